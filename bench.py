@@ -1,0 +1,408 @@
+"""Benchmark of the gart hot path on B200: one step = bounds -> tile map -> forward -> backward of one view.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config unbounded6m] [--tile-size 8]
+    python bench.py --impl reference ...      # the float64 CPU oracle on the host cores, bounded sample
+
+Prints ONE JSON line.  `value` is ray-Gaussian hits per second over the whole step with every input
+resident in HBM; `e2e` is the same metric through the host-buffer entry point (gart_view_host) with
+the host<->device copies inside the timed region.  Per-stage times, the backward's roofline
+fraction, the speedup over the pixel-centric atomic backward, clocks sampled during the timed region
+and the oracle timed on the host cores are reported in the same line.
+
+With N > 1 (torchrun) the views of the orbit are sharded over the ranks; ranks exchange nothing on
+the data path (views are independent), so the scaling is "weak".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gart_scenes as gs  # noqa: E402
+
+METRIC = "ray_gaussian_hits_per_s"
+UNIT = "hits/s"
+HBM_FALLBACK_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------------------- host logic
+def shard_views(n_views: int, rank: int, world: int):
+    """Views handled by `rank`: round-robin, every rank gets at least one (wrapping if world > n_views)."""
+    mine = [v for v in range(n_views) if v % world == rank]
+    return mine if mine else [rank % n_views]
+
+
+def launches_per_step(n_tiles: int) -> int:
+    """Kernel launches of one step (memsets are not kernels)."""
+    bits = 1
+    while (1 << bits) < n_tiles:
+        bits += 1
+    passes = (bits + 7) // 8
+    bounds = 1
+    tile_map = 1 + 3 + 1 + 1 + passes * (1 + 3 + 1) + 1
+    forward = 1 + 3 + 3 + 1 + 1 + 1
+    backward = 2
+    return bounds + tile_map + forward + backward
+
+
+def algorithmic_bytes_backward(H, P, n_vis, n_pixels, K, mask_words):
+    """Bytes the primitive-centric backward must move once: LT entries of the hits, the pair list with
+    its masks and offsets, each visible Gaussian's record and SH read once, its gradient written once,
+    the upstream gradient read once."""
+    return 16 * H + (4 + 4 * mask_words + 4) * P + 4 * (20 + 3 * K) * n_vis + 4 * (11 + 3 * K) * n_vis + 12 * n_pixels
+
+
+def fp32_instr_backward(H, K):
+    """FP32-pipe instructions per hit of the backward: evaluation 31, maximum-response point 9, colour and
+    SH gradient 2*3K, alpha gradient 14, moments 13."""
+    return H * (31 + 9 + 6 * K + 14 + 13)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured", float(d.get("sm_max_mhz", 1965.0))
+        except Exception:
+            pass
+    return HBM_FALLBACK_GBS, "fallback", 1965.0
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        q = "clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+            "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q, "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------- workload
+def make_workload(name: str, n_views=None):
+    kw = {}
+    if n_views is not None and name in ("shell200k", "unbounded1m", "unbounded6m"):
+        kw["n_views"] = n_views
+    scene, cams = gs.make(name, **kw)
+    return scene, cams
+
+
+def oracle_sample(scene, cam, seed=0, frac=0.02, tile=8):
+    """Pixel mask for the oracle's bounded sample: a random subset of 8x8 tiles of the view."""
+    rng = np.random.default_rng([seed, 0x51])
+    tx, ty = -(-cam.width // tile), -(-cam.height // tile)
+    pick = rng.random((ty, tx)) < frac
+    mask = np.repeat(np.repeat(pick, tile, axis=0), tile, axis=1)[:cam.height, :cam.width]
+    return np.ascontiguousarray(mask.astype(np.uint8))
+
+
+def time_oracle(scene, cam, dL_dC, frac, threads=None):
+    """Oracle (as it stands) on a bounded sample of the view: hit discovery + ordering + compositing +
+    backward for the sampled rays.  Returns (hits, seconds, threads)."""
+    from oracle import gart_oracle as orc
+    if threads:
+        orc.set_threads(threads)
+    osc = orc.OracleScene.from_scene(scene)
+    mask = oracle_sample(scene, cam, frac=frac)
+    t0 = time.perf_counter()
+    v = orc.View(osc, cam, alpha_min=float(np.float32(1.0 / 255.0)), near=float(np.float32(0.01)))
+    H = v.find_hits(orc.PREFILTER, mask)
+    v.composite()
+    v.backward(np.asarray(dL_dC, dtype=np.float64))
+    dt = time.perf_counter() - t0
+    v.close()
+    return H, dt, orc.max_threads(), int(mask.sum())
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    scene, cams = make_workload(args.config)
+    frac = args.oracle_frac / 4.0     # per step; keeps a K-step run within minutes
+    times, hits = [], 0
+    for s in range(args.warmup + args.steps):
+        cam = cams[s % len(cams)]
+        g = gs.upstream_gradient(cam, s % len(cams))
+        H, dt, thr, npx = time_oracle(scene, cam, g, frac)
+        if s >= args.warmup:
+            times.append(dt); hits += H
+    total = sum(times)
+    val = hits / total if total > 0 else 0.0
+    sample = "random %.0f%% of the 8x8 tiles of each view (%d rays), all Gaussians" % (100 * frac, npx)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.config, "n_gaussians": scene.n, "width": cams[0].width, "height": cams[0].height,
+                       "sh_degree": scene.sh_degree},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2608_17298_b200.gart as G
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback for the gart library")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    cfg = G.Config(tile_size=args.tile_size)
+    scene, cams = make_workload(args.config)
+    mine = shard_views(len(cams), rank, world)
+    g = G.Gaussians.from_numpy(scene, dev)
+    K = (scene.sh_degree + 1) ** 2
+    dls = {v: torch.from_numpy(gs.upstream_gradient(cams[v], v)).to(dev) for v in mine}
+
+    # capacities: exact pair count and slot bound of this rank's first view, with slack for the other views
+    P0, S0 = G.size_view(cfg, g, cams[mine[0]], slack=1.0, device=dev)
+    cap_pairs, cap_hits = int(P0 * args.slack) + 1024, int(S0 * args.slack) + 1024
+    buf = G.ViewBuffers(g.n, g.sh_degree, cams[0], cfg, cap_pairs, cap_hits, dev)
+    stream = torch.cuda.current_stream()
+
+    def step(v, ev=None):
+        cam = cams[v]
+        if ev: ev[0].record(stream)
+        G.run_bounds_tile_map(cfg, g, cam, buf, stream)
+        if ev: ev[1].record(stream)
+        G.run_forward(cfg, g, cam, buf, stream)
+        if ev: ev[2].record(stream)
+        G.run_backward(cfg, g, cam, buf, dls[v], None, stream)
+        if ev: ev[3].record(stream)
+
+    for s in range(args.warmup):
+        step(mine[s % len(mine)])
+    torch.cuda.synchronize()
+    cnt = G.gart_read_counts(buf.counts)
+    if cnt[G.CNT_ERROR]:
+        raise RuntimeError("capacity exceeded during warm-up: counts=%s cap_pairs=%d cap_hits=%d" % (cnt, cap_pairs, cap_hits))
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    hits_ev = []
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    t_start = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    counts_log = torch.zeros((args.steps, G.COUNTS_WORDS), dtype=torch.int32, device=dev)
+    t_start.record(stream)
+    for s in range(args.steps):
+        step(mine[s % len(mine)], evs[s])
+        counts_log[s].copy_(buf.counts)          # device-to-device, 32 bytes: keeps per-view counts without a host sync
+    t_end.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = t_start.elapsed_time(t_end)
+    cl = counts_log.cpu().numpy().view(np.uint32).astype(np.int64)
+    if (cl[:, G.CNT_ERROR] != 0).any():
+        raise RuntimeError("capacity exceeded inside the timed region: %s" % cl.tolist())
+    hits_total = int(cl[:, G.CNT_HITS].sum())
+    stage = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(3)] for e in evs])   # maps, forward, backward
+    bwd_ms = float(np.mean(stage[:, 2]))
+
+    # whole-job aggregate: total hits of all ranks / max time over ranks
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        h = torch.tensor([hits_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(h, op=dist.ReduceOp.SUM)
+        total_ms_all, hits_all = float(t.item()), float(h.item())
+    else:
+        total_ms_all, hits_all = total_ms, float(hits_total)
+
+    # ---- atomic backward (pixel-centric baseline) on the last view's buffers
+    last_v = mine[(args.steps - 1) % len(mine)]
+    ga = torch.empty_like(buf.grad)
+    at = []
+    for i in range(args.atomic_reps + 1):
+        a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        G.run_backward_atomic(cfg, g, cams[last_v], buf, dls[last_v], ga, stream)
+        a1.record(stream)
+        torch.cuda.synchronize()
+        if i > 0:
+            at.append(a0.elapsed_time(a1))
+    atomic_ms = float(np.mean(at)) if at else None
+    last = cl[-1]
+    prim_last_ms = float(stage[-1, 2])
+    del ga
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if args.e2e_steps > 0:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+        class HS:
+            pass
+        hs = HS()
+        hs.mean, hs.scale, hs.quat, hs.opacity, hs.sh = pin(scene.mean), pin(scene.scale), pin(scene.quat), pin(scene.opacity), pin(scene.sh)
+        hs.sh_degree = scene.sh_degree
+        hdl = {v: pin(gs.upstream_gradient(cams[v], v)) for v in mine}
+        cam0 = cams[0]
+        color_h = torch.empty((cam0.height, cam0.width, 3), dtype=torch.float32).pin_memory()
+        grad_h = torch.empty((scene.n, G.GRAD_WORDS), dtype=torch.float32).pin_memory()
+        # free the resident buffers first: the arena holds its own copy of everything
+        del buf
+        torch.cuda.empty_cache()
+        arena = torch.empty(G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam0.width, cam0.height, cfg.tile_size,
+                                                         cap_pairs, cap_hits), dtype=torch.uint8, device=dev)
+        e_hits, e_t = 0, 0.0
+        for s in range(args.e2e_steps + 1):
+            v = mine[s % len(mine)]
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            c = G.gart_view_host(cfg, hs, cams[v], hdl[v], color_h, grad_h, cap_pairs, cap_hits, arena, stream)
+            dt = time.perf_counter() - t0
+            if s > 0:
+                e_hits += c[G.CNT_HITS]; e_t += dt
+        e_val = e_hits / e_t
+        if world > 1:
+            tt = torch.tensor([e_t], dtype=torch.float64, device=dev); dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            hh = torch.tensor([e_hits], dtype=torch.float64, device=dev); dist.all_reduce(hh, op=dist.ReduceOp.SUM)
+            e_val = float(hh.item()) / float(tt.item())
+        h2d = 4 * scene.n * (3 + 3 + 4 + 1 + 3 * K) + 12 * cam0.width * cam0.height
+        d2h = 4 * scene.n * G.GRAD_WORDS + 12 * cam0.width * cam0.height + 4 * G.COUNTS_WORDS
+        e2e = {"value": e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * e_t / args.e2e_steps, "steps": args.e2e_steps}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant call (gart_backward: zeroing + pair kernel + per-Gaussian conversion)
+    hbm, hbm_src, sm_max = measured_peaks()
+    mw = cfg.tile_size ** 2 // 32
+    n_pix = cams[0].width * cams[0].height
+    Hm, Pm, Nv = float(np.mean(cl[:, G.CNT_HITS])), float(np.mean(cl[:, G.CNT_PAIRS])), float(np.mean(cl[:, G.CNT_VISIBLE]))
+    B = algorithmic_bytes_backward(Hm, Pm, Nv, n_pix, K, mw)
+    achieved = B / (bwd_ms * 1e-3) / 1e9
+    F = fp32_instr_backward(Hm, K)
+    alu_peak = 148 * 128 * sm_max * 1e6            # FP32 lane-instructions per second at the maximum SM clock
+    roof = {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
+            "peak_source": hbm_src, "kernel": "gart_backward (memset + bwd_pairs_kernel + bwd_finalize_kernel)",
+            "algorithmic_bytes": B, "ms": bwd_ms,
+            "alu": {"fp32_lane_instr": F, "peak_lane_instr_per_s": alu_peak, "frac": F / (bwd_ms * 1e-3) / alu_peak}}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            t = json.load(open(prof))
+            if t.get("config") == args.config and t.get("tile_size") == cfg.tile_size:
+                roof["traffic"] = t.get("dram_bytes_per_launch")
+        except Exception:
+            pass
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cam = cams[mine[0]]
+        H, dt, thr, npx = time_oracle(scene, cam, gs.upstream_gradient(cam, mine[0]), args.oracle_frac)
+        cpu = {"value": H / dt, "unit": UNIT, "cores": thr, "kind": "oracle",
+               "sample": "random %.0f%% of the 8x8 tiles of view %d (%d rays, %d hits), all Gaussians, %.1f s" % (
+                   100 * args.oracle_frac, mine[0], npx, H, dt)}
+
+    line = {
+        "metric": METRIC, "value": hits_all / (total_ms_all * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms_all / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.config, "n_gaussians": scene.n, "width": cams[0].width, "height": cams[0].height,
+                   "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "views": len(cams),
+                   "l2": "inputs larger than L2 (parameters %.2f GB, LT %.2f GB per view)" % (
+                       4e-9 * scene.n * (11 + 3 * K), 16e-9 * Hm),
+                   "hits_per_view": Hm, "pairs_per_view": Pm, "visible_per_view": Nv},
+        "stages_ms": {"bounds_tile_map": float(np.mean(stage[:, 0])), "forward": float(np.mean(stage[:, 1])),
+                      "backward": bwd_ms, "backward_median": float(np.median(stage[:, 2]))},
+        "backward_hits_per_s": Hm / (bwd_ms * 1e-3),
+        "backward_atomic_ms": atomic_ms,
+        "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(G.tiles(cams[0], cfg.tile_size)) * args.steps,
+        "roofline": roof, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="unbounded6m", choices=list(gs.CONFIGS))
+    ap.add_argument("--tile-size", type=int, default=8, choices=[8, 16])
+    ap.add_argument("--slack", type=float, default=1.25)
+    ap.add_argument("--atomic-reps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--oracle-frac", type=float, default=0.02)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

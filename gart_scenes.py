@@ -99,11 +99,12 @@ def _unit_quats(rng, n):
 
 
 def _sh(rng, n, degree):
+    """DC ~ U(0,1), higher bands ~ N(0, 0.1); drawn in fp32 (the arrays are fp32 anyway)."""
     K = (degree + 1) ** 2
-    sh = np.empty((n, K, 3), dtype=np.float64)
-    sh[:, 0, :] = rng.uniform(0.0, 1.0, (n, 3))
+    sh = np.empty((n, K, 3), dtype=np.float32)
+    sh[:, 0, :] = rng.random((n, 3), dtype=np.float32)
     if K > 1:
-        sh[:, 1:, :] = rng.normal(0.0, 0.1, (n, K - 1, 3))
+        sh[:, 1:, :] = rng.standard_normal((n, K - 1, 3), dtype=np.float32) * np.float32(0.1)
     return sh
 
 
@@ -181,12 +182,13 @@ def _unbounded(rng, n, fg_log_scale, fg_sigma, bg_log_scale, bg_sigma, sh_degree
     s_fg = np.exp(rng.normal(fg_log_scale, fg_sigma, (n_fg, 3)))
     s_bg = np.minimum(2.0, np.exp(rng.normal(bg_log_scale, bg_sigma, (n_bg, 3))) * r_bg / 10.0)
     scale = np.concatenate([s_fg, s_bg], axis=0)
+    # interleave foreground and background so that ids carry no depth information
+    perm = rng.permutation(n)
+    mean, scale = mean[perm], scale[perm]
     quat = _unit_quats(rng, n)
     opacity = _sigmoid(rng.normal(1.0, 1.0, n))
     sh = _sh(rng, n, sh_degree)
-    # interleave foreground and background so that ids carry no depth information
-    perm = rng.permutation(n)
-    return _pack(mean[perm], scale[perm], quat[perm], opacity[perm], sh[perm], sh_degree)
+    return _pack(mean, scale, quat, opacity, sh, sh_degree)
 
 
 def unbounded_camera(view: int = 0, n_orbit: int = 64, width: int = 1237, height: int = 822) -> Camera:

@@ -1,0 +1,210 @@
+/*
+ * gart.h -- C ABI of the B200 (sm_100a) library for the hot path of primitive-centric
+ * ray-traced Gaussian rendering (3DGART).
+ *
+ * One view is processed by four calls, in this order:
+ *
+ *   gart_bounds    per-Gaussian conservative screen rectangle and ray-evaluation record
+ *   gart_tile_map  (tile, Gaussian) pair list, radix-sorted by tile, and the tile offset table
+ *   gart_forward   ray evaluation: hits ordered by maximum-response distance, compositing,
+ *                  and the compact per-hit buffer LT = (colour behind the hit, transmittance)
+ *   gart_backward  primitive-centric backward: one thread per (tile, Gaussian) pair gathers
+ *                  the gradients of that Gaussian over the pair's hit pixels
+ *   gart_backward_atomic   the pixel-centric baseline: one thread per ray, atomicAdd per hit
+ *
+ * Conventions
+ *   - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
+ *     "host".  Arrays are dense, row-major, fp32 unless the type says otherwise.
+ *   - The library allocates no device memory.  Scratch comes from a caller-supplied
+ *     workspace whose size is returned by the matching *_workspace_bytes query; the
+ *     workspace must be 256-byte aligned and may be reused by the next call on the
+ *     same stream.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All calls
+ *     are asynchronous; none synchronises with the host.
+ *   - Return value: GART_OK or an error code from argument checking / kernel launch.
+ *     Conditions only the device can see (a capacity that turns out too small) are
+ *     recorded in the counts block (GART_CNT_ERROR) and skip the affected work; read
+ *     the block back with gart_read_counts after synchronising.
+ *   - Camera: pinhole, x right, y down, z forward; pixel (x,y) has its centre at
+ *     (x+0.5, y+0.5); world-to-camera matrix [R|t] row-major; unit ray direction
+ *     d = normalize(R^T ((x+0.5-cx)/fx, (y+0.5-cy)/fy, 1)), origin o = -R^T t.
+ *   - Quaternions are (w,x,y,z) and used as given (no normalisation).
+ *   - Tiles are tile_size x tile_size pixels (8 or 16); tile id = ty * tiles_x + tx with
+ *     tiles_x = ceil(width / tile_size).
+ */
+#ifndef GART_H
+#define GART_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GART_OK = 0,
+    GART_ERR_INVALID_ARG = 1,
+    GART_ERR_WORKSPACE_TOO_SMALL = 2,
+    GART_ERR_CAPACITY_EXCEEDED = 3,
+    GART_ERR_CUDA = 4
+} gart_status;
+
+/* Host struct. */
+typedef struct {
+    float alpha_min;      /* minimum response of a hit; the paper uses 1/255 (Sec. 3.4) */
+    float near_z;         /* depth of the near plane used only to classify Gaussians */
+    float background[3];  /* colour multiplied by the final transmittance */
+    int32_t tile_size;    /* 8 (the paper's choice, Sec. 4.4) or 16 */
+} gart_config;
+
+/* Host struct. */
+typedef struct {
+    int32_t width, height;
+    double fx, fy, cx, cy;
+    double w2c[12];       /* row-major [R | t] */
+} gart_camera;
+
+/* Host struct holding device pointers (Sec. 3.1: mean, Sigma = R S S^T R^T, opacity, SH radiance). */
+typedef struct {
+    int64_t n;
+    int32_t sh_degree;     /* 0..3; K = (sh_degree+1)^2 coefficients per channel */
+    const float *mean;     /* [n,3] */
+    const float *scale;    /* [n,3] */
+    const float *quat;     /* [n,4] (w,x,y,z) */
+    const float *opacity;  /* [n]   */
+    const float *sh;       /* [n,K,3] */
+} gart_gaussians;
+
+/* Words of the counts block (device memory, GART_COUNTS_WORDS x uint32, zeroed by gart_bounds). */
+enum {
+    GART_CNT_VISIBLE = 0,   /* Gaussians with a non-empty rectangle */
+    GART_CNT_PAIRS = 1,     /* P: (tile, Gaussian) pairs */
+    GART_CNT_SLOTS_LO = 2,  /* S = sum of rectangle areas, low/high words: the capacity bound */
+    GART_CNT_SLOTS_HI = 3,  /*     of the intermediate buffer (Eq. 15 with lambda_s = 1)      */
+    GART_CNT_HITS = 4,      /* H: ray-Gaussian hits of the view = entries used in LT */
+    GART_CNT_ERROR = 5,     /* bit 0: pair capacity exceeded; bit 1: hit capacity exceeded */
+    GART_CNT_MAX_RAY_HITS = 6,
+    GART_CNT_STRADDLE = 7,  /* Gaussians whose support crosses the near plane */
+    GART_COUNTS_WORDS = 8
+};
+#define GART_ERRBIT_PAIRS 1u
+#define GART_ERRBIT_HITS 2u
+
+#define GART_PRE_WORDS 20   /* fp32 words of the per-Gaussian ray-evaluation record */
+#define GART_GRAD_WORDS 64  /* stride of a gradient record: mean 3, scale 3, quat 4, opacity 1,
+                               sh 3K (coefficient-major, channel-minor, as the input), zero padding */
+
+const char *gart_status_string(gart_status s);
+
+/* Words (uint32) of hit mask per pair: tile_size^2 / 32. */
+int32_t gart_mask_words(int32_t tile_size);
+
+/*
+ * Step 1 -- conservative perspective-correct bounds (Sec. 4.2, Eq. 11-14) with the opacity
+ * dependent clamping radius alpha_c = sqrt(2 ln(sigma/alpha_min)) (Eq. 10), evaluated in
+ * double precision, and the pre-computations of the ray evaluation (W = S^-1 R^T and o_g of
+ * Eq. 5, expressed relative to a per-Gaussian reference pixel so that fp32 evaluation stays
+ * well conditioned).
+ *   rect   [n,4] int32 out: inclusive pixel range x0,y0,x1,y1 of pixel centres inside the
+ *                bound, clipped to the image; (0,0,-1,-1) if empty.
+ *   cls    [n]   uint8 out: 0 culled (sigma <= alpha_min, or support entirely at depth <= near_z),
+ *                1 in front of the near plane, 2 straddling it (rectangle = whole image unless
+ *                the bounding sphere is outside a side plane of the frustum).
+ *   pre    [n,GART_PRE_WORDS] fp32 out; contents are private to the library.
+ *   counts [GART_COUNTS_WORDS] uint32 out: zeroed, then VISIBLE and STRADDLE are set.
+ * Errors: INVALID_ARG for null pointers, n < 0, sh_degree outside 0..3, tile size not 8/16,
+ * non-positive image size.
+ */
+gart_status gart_bounds(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,
+                        int32_t *rect, uint8_t *cls, float *pre, uint32_t *counts, void *stream);
+
+/*
+ * Step 2 -- reverse tile mapping (Sec. 4.3): every Gaussian emits one (tile, id) pair per tile
+ * its rectangle overlaps; the pairs are radix-sorted by tile (stable, so ids ascend inside a
+ * tile) and the tile offset table is the prefix sum of pairs per tile.  Also sums the
+ * rectangle areas (the footprint prefix sum of "Primitive offset", kept as the total S).
+ *   tile_off [T+1] uint32 out, T = tiles_x * tiles_y; tile t owns pair_gid[tile_off[t] .. tile_off[t+1]).
+ *   pair_gid [cap_pairs] uint32 out.
+ *   counts: PAIRS, SLOTS set.  If P > cap_pairs the error bit GART_ERRBIT_PAIRS is set,
+ *   tile_off is all zero and later calls do nothing.
+ */
+size_t gart_tile_map_workspace_bytes(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs);
+gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n, int32_t width, int32_t height,
+                          uint32_t *tile_off, uint32_t *pair_gid, int64_t cap_pairs, uint32_t *counts,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Step 3 -- forward ray evaluation (Sec. 3.2-3.3, Eq. 3-8; intermediate buffer of Sec. 4.2-4.3).
+ * For every pixel ray and every Gaussian of its tile list: t* = -(o_g.d_g)/(d_g.d_g),
+ * alpha = sigma exp(-|o_g + t* d_g|^2 / 2); a hit iff alpha >= alpha_min and t* > 0.  Hits of a
+ * ray are ordered by (t*, id) and composited front to back, C = sum T_i alpha_i c_i + T_final bg,
+ * c_i = max(0, 0.5 + sum_k Y_k(d) sh_ik).
+ *   color      [H,W,3] out;  t_final [H,W] out;  hit_count [H,W] uint32 out.
+ *   pair_mask  [cap_pairs, gart_mask_words] uint32 out: bit p of pair j = pixel p of the tile
+ *              (p = ly * tile_size + lx) is hit by the pair's Gaussian.
+ *   pair_lt_off[cap_pairs+1] uint32 out: exclusive prefix sum of hits per pair; the hit of pair j
+ *              at pixel p lives at lt[pair_lt_off[j] + (number of set mask bits below p)]:
+ *              primitive-tile-major, then pixel, every hit with a collision-free slot.
+ *   lt         [cap_hits,4] out: per hit (R_r, R_g, R_b, T): colour composited BEHIND the hit
+ *              (including the background term) and transmittance in front of it.
+ *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
+ *              compositing order, the Gaussian id and LT slot of each hit.
+ *   counts: HITS, MAX_RAY_HITS.  If H > cap_hits, GART_ERRBIT_HITS is set and color, t_final,
+ *   lt, ray_gid, ray_slot are not written.
+ */
+size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
+gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
+                         const uint32_t *tile_off, const uint32_t *pair_gid, int64_t cap_pairs,
+                         float *color, float *t_final, uint32_t *hit_count,
+                         uint32_t *pair_mask, uint32_t *pair_lt_off, float *lt, int64_t cap_hits,
+                         uint32_t *ray_off, uint32_t *ray_gid, uint32_t *ray_slot, uint32_t *counts,
+                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Step 4 -- primitive-centric backward (Sec. 4.4): one thread block per tile, one thread per
+ * (tile, Gaussian) pair; the thread walks the pair's hit pixels, reads their LT entries (one
+ * contiguous run), accumulates in registers and performs one vector atomic update of the
+ * Gaussian's gradient record per pair.  No per-pixel atomics.
+ *   dL_dcolor [H,W,3] in.
+ *   grad [n,GART_GRAD_WORDS] out, fully overwritten: d mean, d scale, d quat, d opacity, d sh
+ *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
+ */
+gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
+                          const uint32_t *tile_off, const uint32_t *pair_gid, const uint32_t *pair_mask,
+                          const uint32_t *pair_lt_off, const float *lt, const float *dL_dcolor,
+                          float *grad, const uint32_t *counts, void *stream);
+
+/*
+ * Pixel-centric baseline (Sec. 3.5): one thread per ray walks the ray's hits and issues one
+ * atomicAdd per gradient word per hit (11 + 3K; 59 at degree 3).  Same result as gart_backward
+ * up to summation order.
+ */
+gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,
+                                 const float *pre, const uint32_t *ray_off, const uint32_t *ray_gid,
+                                 const uint32_t *ray_slot, const float *lt, const float *dL_dcolor,
+                                 float *grad, const uint32_t *counts, void *stream);
+
+/* Copy the counts block to host memory (synchronises the stream). counts_host: host, GART_COUNTS_WORDS words. */
+gart_status gart_read_counts(const uint32_t *counts, uint32_t *counts_host, void *stream);
+
+/*
+ * End-to-end convenience for callers holding HOST arrays: uploads the scene and dL_dcolor,
+ * runs the four steps for one view, downloads color [H,W,3] and grad [n,GART_GRAD_WORDS].
+ * All five array arguments and the members of `g_host` are HOST pointers.  `arena` is a device
+ * buffer of `arena_bytes` bytes from which every device array is carved; query the size with
+ * gart_view_host_arena_bytes (cap_pairs / cap_hits are capacities chosen by the caller).
+ * counts_host (host, GART_COUNTS_WORDS words) receives the counts block.  Synchronous.
+ * Returns GART_ERR_CAPACITY_EXCEEDED if a capacity was too small.
+ */
+size_t gart_view_host_arena_bytes(int64_t n, int32_t sh_degree, int32_t width, int32_t height, int32_t tile_size,
+                                  int64_t cap_pairs, int64_t cap_hits);
+gart_status gart_view_host(const gart_config *cfg, const gart_gaussians *g_host, const gart_camera *cam,
+                           const float *dL_dcolor_host, float *color_host, float *grad_host,
+                           int64_t cap_pairs, int64_t cap_hits, uint32_t *counts_host,
+                           void *arena, size_t arena_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GART_H */

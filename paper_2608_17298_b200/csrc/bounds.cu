@@ -1,0 +1,172 @@
+// gart_bounds: conservative perspective-correct screen rectangles (Sec. 4.2, Eq. 11-14), the
+// opacity-dependent clamping radius (Eq. 10) and the ray-evaluation record (Eq. 5), one thread
+// per Gaussian, in double precision: the rectangle edges are integer decisions (ceil / floor of
+// p -/+ h) and the pass is O(n), so fp64 costs nothing that matters and keeps the edges exact.
+#include "common.cuh"
+
+namespace gart {
+
+struct CamD {
+    int width, height;
+    double fx, fy, cx, cy;
+    double w2c[12];
+};
+
+__device__ __forceinline__ void quat_to_rot(const double w, const double x, const double y, const double z, double* R) {
+    R[0] = 1.0 - 2.0 * (y * y + z * z); R[1] = 2.0 * (x * y - w * z); R[2] = 2.0 * (x * z + w * y);
+    R[3] = 2.0 * (x * y + w * z); R[4] = 1.0 - 2.0 * (x * x + z * z); R[5] = 2.0 * (y * z - w * x);
+    R[6] = 2.0 * (x * z - w * y); R[7] = 2.0 * (y * z + w * x); R[8] = 1.0 - 2.0 * (x * x + y * y);
+}
+
+__global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
+                                                     const float* __restrict__ quat, const float* __restrict__ opacity,
+                                                     CamD cam, double alpha_min, double near_z,
+                                                     int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
+                                                     float4* __restrict__ pre4, uint32_t* __restrict__ counts) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int vis = 0, straddle = 0;
+    if (i < n) {
+        int x0 = 0, y0 = 0, x1 = -1, y1 = -1, c = 0;
+        float4 q0 = make_float4(0, 0, 0, 0), q1 = q0, q2 = q0, q3 = q0, q4 = q0;
+        const double sigma = (double)opacity[i];
+        if (sigma > alpha_min) {
+            const double alpha_c = sqrt(2.0 * log(sigma / alpha_min));  // Eq. 10
+            double R[9];
+            quat_to_rot((double)quat[4 * i], (double)quat[4 * i + 1], (double)quat[4 * i + 2], (double)quat[4 * i + 3], R);
+            const double s[3] = {(double)scale[3 * i], (double)scale[3 * i + 1], (double)scale[3 * i + 2]};
+            const double mu[3] = {(double)mean[3 * i], (double)mean[3 * i + 1], (double)mean[3 * i + 2]};
+            const double* M = cam.w2c;
+            // camera-space support axes  Ac = Rc * (R S alpha_c)  and centre
+            double Ac[9], muc[3];
+#pragma unroll
+            for (int r = 0; r < 3; ++r) {
+#pragma unroll
+                for (int k = 0; k < 3; ++k)
+                    Ac[3 * r + k] = (M[4 * r] * R[k] + M[4 * r + 1] * R[3 + k] + M[4 * r + 2] * R[6 + k]) * s[k] * alpha_c;
+                muc[r] = M[4 * r] * mu[0] + M[4 * r + 1] * mu[1] + M[4 * r + 2] * mu[2] + M[4 * r + 3];
+            }
+            const double ez = sqrt(Ac[6] * Ac[6] + Ac[7] * Ac[7] + Ac[8] * Ac[8]);
+            if (muc[2] + ez > near_z) {
+                c = (muc[2] - ez >= near_z) ? 1 : 2;
+                if (c == 1) {
+                    // rows x, y, w of T' in pixel units; v = (1,1,1,-1)
+                    double sden = -muc[2] * muc[2], pxn = 0.0, pyn = 0.0, qxn = 0.0, qyn = 0.0;
+                    const double tx3 = cam.fx * muc[0] + cam.cx * muc[2], ty3 = cam.fy * muc[1] + cam.cy * muc[2];
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) {
+                        const double tw = Ac[6 + k];
+                        const double tx = cam.fx * Ac[k] + cam.cx * tw, ty = cam.fy * Ac[3 + k] + cam.cy * tw;
+                        sden += tw * tw;
+                        pxn += tx * tw; pyn += ty * tw;
+                        qxn += tx * tx; qyn += ty * ty;
+                    }
+                    pxn -= tx3 * muc[2]; pyn -= ty3 * muc[2];
+                    qxn -= tx3 * tx3;   qyn -= ty3 * ty3;
+                    const double px = pxn / sden, py = pyn / sden;
+                    const double hx = sqrt(fmax(0.0, px * px - qxn / sden)), hy = sqrt(fmax(0.0, py * py - qyn / sden));
+                    const double fx0 = fmax(0.0, ceil(px - hx - 0.5)), fx1 = fmin((double)(cam.width - 1), floor(px + hx - 0.5));
+                    const double fy0 = fmax(0.0, ceil(py - hy - 0.5)), fy1 = fmin((double)(cam.height - 1), floor(py + hy - 0.5));
+                    if (fx1 >= fx0 && fy1 >= fy0) { x0 = (int)fx0; y0 = (int)fy0; x1 = (int)fx1; y1 = (int)fy1; }
+                } else {
+                    const double rad = alpha_c * fmax(s[0], fmax(s[1], s[2]));
+                    const double pl[4][3] = {{cam.fx, 0.0, cam.cx}, {-cam.fx, 0.0, cam.width - cam.cx},
+                                             {0.0, cam.fy, cam.cy}, {0.0, -cam.fy, cam.height - cam.cy}};
+                    bool outside = false;
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        const double len = sqrt(pl[p][0] * pl[p][0] + pl[p][1] * pl[p][1] + pl[p][2] * pl[p][2]);
+                        const double dist = (pl[p][0] * muc[0] + pl[p][1] * muc[1] + pl[p][2] * muc[2]) / len;
+                        outside = outside || (dist < -rad);
+                    }
+                    if (!outside) { x0 = 0; y0 = 0; x1 = cam.width - 1; y1 = cam.height - 1; }
+                    straddle = 1;
+                }
+                if (x1 >= x0) {
+                    vis = 1;
+                    // ---- ray-evaluation record
+                    // W = S^-1 R^T ; Wc = W Rc^T ; m = W (mu - o), o = -Rc^T t
+                    double Wc[9], m[3];
+                    const double o[3] = {-(M[0] * M[3] + M[4] * M[7] + M[8] * M[11]),
+                                         -(M[1] * M[3] + M[5] * M[7] + M[9] * M[11]),
+                                         -(M[2] * M[3] + M[6] * M[7] + M[10] * M[11])};
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) {
+                        const double w0 = R[k] / s[k], w1 = R[3 + k] / s[k], w2 = R[6 + k] / s[k];  // row k of W
+#pragma unroll
+                        for (int j = 0; j < 3; ++j) Wc[3 * k + j] = w0 * M[4 * j] + w1 * M[4 * j + 1] + w2 * M[4 * j + 2];
+                        m[k] = w0 * (mu[0] - o[0]) + w1 * (mu[1] - o[1]) + w2 * (mu[2] - o[2]);
+                    }
+                    // reference position: projected centre when that is a sane pixel coordinate
+                    double rpx = cam.cx, rpy = cam.cy;
+                    if (c == 1) {
+                        const double ppx = cam.fx * muc[0] / muc[2] + cam.cx, ppy = cam.fy * muc[1] / muc[2] + cam.cy;
+                        if (fabs(ppx) < 1.0e6 && fabs(ppy) < 1.0e6) { rpx = ppx; rpy = ppy; }
+                    }
+                    const double fix = floor(rpx), fiy = floor(rpy);
+                    const float rx = (float)(rpx - 0.5 - fix), ry = (float)(rpy - 0.5 - fiy);
+                    const double ex_px = fix + 0.5 + (double)rx, ex_py = fiy + 0.5 + (double)ry;  // exactly what the kernels use
+                    const double du = (ex_px - cam.cx) / cam.fx, dv = (ex_py - cam.cy) / cam.fy;
+                    double dgr[3], kk[3];
+#pragma unroll
+                    for (int k = 0; k < 3; ++k) dgr[k] = Wc[3 * k] * du + Wc[3 * k + 1] * dv + Wc[3 * k + 2];
+                    // k = o_g x dgr = dgr x m
+                    kk[0] = dgr[1] * m[2] - dgr[2] * m[1];
+                    kk[1] = dgr[2] * m[0] - dgr[0] * m[2];
+                    kk[2] = dgr[0] * m[1] - dgr[1] * m[0];
+                    q0 = make_float4((float)(Wc[0] / cam.fx), (float)(Wc[3] / cam.fx), (float)(Wc[6] / cam.fx), (float)(Wc[1] / cam.fy));
+                    q1 = make_float4((float)(Wc[4] / cam.fy), (float)(Wc[7] / cam.fy), (float)dgr[0], (float)dgr[1]);
+                    q2 = make_float4((float)dgr[2], (float)m[0], (float)m[1], (float)m[2]);
+                    q3 = make_float4((float)kk[0], (float)kk[1], (float)kk[2], (float)sigma);
+                    q4 = make_float4(rx, ry, __int_as_float((int)fix), __int_as_float((int)fiy));
+                }
+            }
+        }
+        reinterpret_cast<int4*>(rect)[i] = make_int4(x0, y0, x1, y1);
+        cls[i] = (uint8_t)c;
+        float4* p = pre4 + (size_t)i * 5;
+        p[0] = q0; p[1] = q1; p[2] = q2; p[3] = q3; p[4] = q4;
+    }
+    const unsigned bv = __ballot_sync(0xffffffffu, vis), bs = __ballot_sync(0xffffffffu, straddle);
+    if ((threadIdx.x & 31) == 0) {
+        if (bv) atomicAdd(&counts[GART_CNT_VISIBLE], __popc(bv));
+        if (bs) atomicAdd(&counts[GART_CNT_STRADDLE], __popc(bs));
+    }
+}
+
+}  // namespace gart
+
+extern "C" const char* gart_status_string(gart_status s) {
+    switch (s) {
+        case GART_OK: return "ok";
+        case GART_ERR_INVALID_ARG: return "invalid argument";
+        case GART_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case GART_ERR_CAPACITY_EXCEEDED: return "capacity exceeded";
+        case GART_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+extern "C" int32_t gart_mask_words(int32_t tile_size) { return tile_size * tile_size / 32; }
+
+extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam,
+                                   int32_t* rect, uint8_t* cls, float* pre, uint32_t* counts, void* stream) {
+    if (!cfg || !g || !cam || !counts) return GART_ERR_INVALID_ARG;
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
+    if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
+    if (cam->width <= 0 || cam->height <= 0 || !(cam->fx > 0.0) || !(cam->fy > 0.0)) return GART_ERR_INVALID_ARG;
+    if (g->n > 0 && (!g->mean || !g->scale || !g->quat || !g->opacity || !rect || !cls || !pre)) return GART_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(counts, 0, GART_COUNTS_WORDS * sizeof(uint32_t), st) != cudaSuccess) return GART_ERR_CUDA;
+    if (g->n == 0) return GART_OK;
+    gart::CamD c;
+    c.width = cam->width; c.height = cam->height;
+    c.fx = cam->fx; c.fy = cam->fy; c.cx = cam->cx; c.cy = cam->cy;
+    for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
+    const int threads = 128;
+    const int64_t blocks = gart::ceil_div(g->n, threads);
+    gart::bounds_kernel<<<(unsigned)blocks, threads, 0, st>>>(g->n, g->mean, g->scale, g->quat, g->opacity, c,
+                                                             (double)cfg->alpha_min, (double)cfg->near_z, rect, cls,
+                                                             reinterpret_cast<float4*>(pre), counts);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}

@@ -1,0 +1,299 @@
+// Shared device/host helpers of the gart CUDA library (sm_100a).
+//
+// Contents: launch-error macro, the fp32 camera block passed to kernels by value, the
+// per-Gaussian ray-evaluation record and the single ray/Gaussian evaluation routine that
+// every kernel uses (Eq. 4, 5, 8 of the 3DGART paper in a cancellation-free form), the real
+// spherical-harmonics basis, and a three-kernel exclusive scan without device-side waiting.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gart.h"
+
+#define GART_LAUNCH_CHECK()                                   \
+    do {                                                      \
+        if (cudaGetLastError() != cudaSuccess) return GART_ERR_CUDA; \
+    } while (0)
+
+namespace gart {
+
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// ---------------------------------------------------------------------------------------------
+// Camera, fp32, by value.
+struct CamF {
+    int width, height;
+    int tiles_x, tiles_y;
+    float fx, fy, cx, cy;
+    float r[9];  // world-to-camera rotation, row-major; world direction of d_c is r^T d_c
+};
+
+static inline CamF make_camf(const gart_camera* cam, int ts) {
+    CamF c;
+    c.width = cam->width;
+    c.height = cam->height;
+    c.tiles_x = (cam->width + ts - 1) / ts;
+    c.tiles_y = (cam->height + ts - 1) / ts;
+    c.fx = (float)cam->fx; c.fy = (float)cam->fy; c.cx = (float)cam->cx; c.cy = (float)cam->cy;
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) c.r[3 * i + j] = (float)cam->w2c[4 * i + j];
+    return c;
+}
+
+// Unit world-space direction of the ray through the centre of pixel (x, y).
+__device__ __forceinline__ float3 pixel_dir(const CamF& c, int x, int y) {
+    const float u = ((float)x + 0.5f - c.cx) / c.fx;
+    const float v = ((float)y + 0.5f - c.cy) / c.fy;
+    float wx = fmaf(c.r[0], u, fmaf(c.r[3], v, c.r[6]));
+    float wy = fmaf(c.r[1], u, fmaf(c.r[4], v, c.r[7]));
+    float wz = fmaf(c.r[2], u, fmaf(c.r[5], v, c.r[8]));
+    const float inv = rsqrtf(fmaf(wx, wx, fmaf(wy, wy, wz * wz)));
+    return make_float3(wx * inv, wy * inv, wz * inv);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Per-Gaussian ray-evaluation record: GART_PRE_WORDS = 20 floats = 5 float4.
+//
+// With W = S^-1 R^T (Eq. 5), the camera rotation Rc and origin o, and the un-normalised ray
+// direction d_c = ((x+.5-cx)/fx, (y+.5-cy)/fy, 1) in camera space:
+//   c0, c1 : columns 0 and 1 of W Rc^T divided by fx, fy -> d_g changes by c0*dx + c1*dy when
+//            the pixel moves by (dx, dy) pixels away from the reference pixel position
+//   dgr    : d_g at the reference position (the projected centre for Gaussians in front)
+//   m      : -o_g = W (mu - o)
+//   k      : o_g x dgr (zero up to rounding when the reference is the projected centre)
+//   sigma  : opacity
+//   rx, ry : fractional part of the reference position, ix, iy its integer part:
+//            dx = float(x - ix) - rx is exact to one rounding however far the pixel is from 0.
+// Then o_g x d_g = k + e x m with e = c0*dx + c1*dy, and
+//   D^2 = |o_g x d_g|^2 / |d_g|^2,  x_g = d_g x (o_g x d_g) / |d_g|^2,  t* = (m . d_g) / |d_g|^2,
+// none of which subtracts large nearly equal numbers (the textbook |o_g|^2 - (o_g.d_g)^2/|d_g|^2
+// loses all digits in fp32 when the Gaussian is small and far).
+struct PreRec {
+    float3 c0, c1, dgr, m, k;
+    float sigma, rx, ry;
+    int ix, iy;
+};
+
+__device__ __forceinline__ PreRec unpack_pre(const float4& a, const float4& b, const float4& c,
+                                             const float4& d, const float4& e) {
+    PreRec p;
+    p.c0 = make_float3(a.x, a.y, a.z);
+    p.c1 = make_float3(a.w, b.x, b.y);
+    p.dgr = make_float3(b.z, b.w, c.x);
+    p.m = make_float3(c.y, c.z, c.w);
+    p.k = make_float3(d.x, d.y, d.z);
+    p.sigma = d.w;
+    p.rx = e.x;
+    p.ry = e.y;
+    p.ix = __float_as_int(e.z);
+    p.iy = __float_as_int(e.w);
+    return p;
+}
+
+__device__ __forceinline__ PreRec load_pre(const float4* __restrict__ pre4, uint32_t gid) {
+    const float4* p = pre4 + (size_t)gid * 5;
+    return unpack_pre(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3), __ldg(p + 4));
+}
+
+struct RayEval {
+    float alpha;   // sigma * exp(-D^2 / 2)
+    float tnum;    // m . d_g : same sign as t*
+    float inv_a;   // 1 / |d_g|^2
+    float3 dg;     // d_g
+    float3 cr;     // o_g x d_g
+};
+
+// Response of the Gaussian along the ray through the pixel at offset (dx, dy) pixels from the
+// record's reference position.
+__device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy) {
+    RayEval r;
+    const float ex = fmaf(p.c0.x, dx, p.c1.x * dy);
+    const float ey = fmaf(p.c0.y, dx, p.c1.y * dy);
+    const float ez = fmaf(p.c0.z, dx, p.c1.z * dy);
+    r.dg = make_float3(p.dgr.x + ex, p.dgr.y + ey, p.dgr.z + ez);
+    r.cr.x = fmaf(ey, p.m.z, fmaf(-ez, p.m.y, p.k.x));
+    r.cr.y = fmaf(ez, p.m.x, fmaf(-ex, p.m.z, p.k.y));
+    r.cr.z = fmaf(ex, p.m.y, fmaf(-ey, p.m.x, p.k.z));
+    const float a = fmaf(r.dg.x, r.dg.x, fmaf(r.dg.y, r.dg.y, r.dg.z * r.dg.z));
+    const float cc = fmaf(r.cr.x, r.cr.x, fmaf(r.cr.y, r.cr.y, r.cr.z * r.cr.z));
+    r.inv_a = __frcp_rn(a);
+    const float D2 = cc * r.inv_a;
+    r.alpha = p.sigma * exp2f(-0.72134752044448170f * D2);
+    r.tnum = fmaf(p.m.x, r.dg.x, fmaf(p.m.y, r.dg.y, p.m.z * r.dg.z));
+    return r;
+}
+
+// Maximum-response point in the Gaussian's normalised space.
+__device__ __forceinline__ float3 ray_xg(const RayEval& r) {
+    return make_float3((r.dg.y * r.cr.z - r.dg.z * r.cr.y) * r.inv_a,
+                       (r.dg.z * r.cr.x - r.dg.x * r.cr.z) * r.inv_a,
+                       (r.dg.x * r.cr.y - r.dg.y * r.cr.x) * r.inv_a);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Real spherical harmonics (index k = l(l+1)+m) of a unit vector, first K values.
+template <int K>
+__device__ __forceinline__ void sh_basis(const float3 d, float* Y) {
+    Y[0] = 0.28209479177387814f;
+    if (K > 1) {
+        Y[1] = -0.4886025119029199f * d.y;
+        Y[2] = 0.4886025119029199f * d.z;
+        Y[3] = -0.4886025119029199f * d.x;
+    }
+    if (K > 4) {
+        const float xx = d.x * d.x, yy = d.y * d.y, zz = d.z * d.z;
+        const float xy = d.x * d.y, yz = d.y * d.z, xz = d.x * d.z;
+        Y[4] = 1.0925484305920792f * xy;
+        Y[5] = -1.0925484305920792f * yz;
+        Y[6] = 0.31539156525252005f * (2.0f * zz - xx - yy);
+        Y[7] = -1.0925484305920792f * xz;
+        Y[8] = 0.5462742152960396f * (xx - yy);
+        if (K > 9) {
+            Y[9] = -0.5900435899266435f * d.y * (3.0f * xx - yy);
+            Y[10] = 2.890611442640554f * xy * d.z;
+            Y[11] = -0.4570457994644658f * d.y * (4.0f * zz - xx - yy);
+            Y[12] = 0.3731763325901154f * d.z * (2.0f * zz - 3.0f * xx - 3.0f * yy);
+            Y[13] = -0.4570457994644658f * d.x * (4.0f * zz - xx - yy);
+            Y[14] = 1.445305721320277f * d.z * (xx - yy);
+            Y[15] = -0.5900435899266435f * d.x * (xx - 3.0f * yy);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exclusive scan of f(0..n_cap-1) into out[0..n_cap] (uint32; out[n_cap] = total) with three
+// launches and no waiting between blocks: per-block sums, one block scans the sums, per-block
+// rescan.  Sums are carried in 64 bits so that an overflowing total is seen (total64_out).
+// f(i) is a device functor returning uint32.
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 16;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
+
+// Block-wide exclusive scan of one value per thread (SCAN_THREADS threads); returns the
+// exclusive prefix and the block total.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* total) {
+    __shared__ uint32_t wsum[SCAN_THREADS / 32];
+    __shared__ uint32_t wtot;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t inc = warp_incl_scan(v);
+    __syncthreads();
+    if (lane == 31) wsum[w] = inc;
+    __syncthreads();
+    if (w == 0) {
+        const uint32_t s = lane < SCAN_THREADS / 32 ? wsum[lane] : 0u;
+        const uint32_t si = warp_incl_scan(s);
+        if (lane < SCAN_THREADS / 32) wsum[lane] = si - s;
+        if (lane == SCAN_THREADS / 32 - 1) wtot = si;
+    }
+    __syncthreads();
+    *total = wtot;
+    return inc - v + wsum[w];
+}
+
+template <class F>
+__global__ void __launch_bounds__(SCAN_THREADS) scan_reduce_kernel(F f, int64_t n_cap, uint64_t* block_sums) {
+    const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    uint32_t s = 0;
+#pragma unroll 4
+    for (int i = 0; i < SCAN_ITEMS; ++i) {
+        const int64_t idx = base + i;
+        if (idx < n_cap) s += f(idx);
+    }
+    uint32_t tot;
+    block_excl_scan(s, &tot);
+    if (threadIdx.x == 0) block_sums[blockIdx.x] = tot;
+}
+
+// One block: exclusive scan of block_sums in place (uint64), total to total64_out[0].
+static __global__ void __launch_bounds__(1024) scan_blocks_kernel(uint64_t* block_sums, int nb, uint64_t* total64_out) {
+    __shared__ uint64_t wsum[32];
+    __shared__ uint64_t carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int base = 0; base < nb; base += 1024) {
+        const int i = base + threadIdx.x;
+        const uint64_t v = i < nb ? block_sums[i] : 0ull;
+        uint64_t inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint64_t t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) wsum[w] = inc;
+        __syncthreads();
+        if (w == 0) {
+            const uint64_t s = wsum[lane];
+            uint64_t si = s;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint64_t t = __shfl_up_sync(0xffffffffu, si, o);
+                if (lane >= o) si += t;
+            }
+            wsum[lane] = si - s;
+        }
+        __syncthreads();
+        const uint64_t carry = carry_s;
+        const uint64_t excl = carry + wsum[w] + inc - v;
+        if (i < nb) block_sums[i] = excl;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = excl + v;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) total64_out[0] = carry_s;
+}
+
+template <class F>
+__global__ void __launch_bounds__(SCAN_THREADS) scan_apply_kernel(F f, int64_t n_cap, const uint64_t* block_offs, uint32_t* out) {
+    const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+    uint32_t v[SCAN_ITEMS];
+    uint32_t s = 0;
+#pragma unroll
+    for (int i = 0; i < SCAN_ITEMS; ++i) {
+        const int64_t idx = base + i;
+        v[i] = idx < n_cap ? f(idx) : 0u;
+        s += v[i];
+    }
+    uint32_t tot;
+    uint32_t run = block_excl_scan(s, &tot) + (uint32_t)block_offs[blockIdx.x];
+#pragma unroll
+    for (int i = 0; i < SCAN_ITEMS; ++i) {
+        const int64_t idx = base + i;
+        if (idx < n_cap) out[idx] = run;
+        run += v[i];
+        if (idx == n_cap - 1) out[n_cap] = run;
+    }
+}
+
+static inline size_t scan_workspace_bytes(int64_t n_cap) {
+    return align256((size_t)(ceil_div(n_cap > 0 ? n_cap : 1, SCAN_TILE) + 1) * sizeof(uint64_t)) + 256;
+}
+
+// out[0..n_cap] = exclusive scan of f; total64 (device, 8-byte aligned) receives the 64-bit total.
+// ws must hold scan_workspace_bytes(n_cap) bytes.  n_cap >= 1.
+template <class F>
+static inline gart_status exclusive_scan(F f, int64_t n_cap, uint32_t* out, uint64_t* total64, void* ws, cudaStream_t st) {
+    const int nb = (int)ceil_div(n_cap, SCAN_TILE);
+    uint64_t* block_sums = (uint64_t*)ws;
+    scan_reduce_kernel<F><<<nb, SCAN_THREADS, 0, st>>>(f, n_cap, block_sums);
+    GART_LAUNCH_CHECK();
+    scan_blocks_kernel<<<1, 1024, 0, st>>>(block_sums, nb, total64);
+    GART_LAUNCH_CHECK();
+    scan_apply_kernel<F><<<nb, SCAN_THREADS, 0, st>>>(f, n_cap, block_sums, out);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}
+
+}  // namespace gart

@@ -1,0 +1,343 @@
+"""Thin Python binding of ``libgart.so`` (ctypes).
+
+Only argument marshalling lives here: PyTorch provides device memory and streams, every step
+of the path runs in the CUDA library.  The functions carry the names of the C entry points
+(``include/gart.h``) and take torch CUDA tensors where the C ABI takes device pointers.
+
+The library must have been built (``python -m paper_2608_17298_b200.build``); loading fails
+loudly otherwise -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import dataclasses
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgart.so")
+
+GART_OK = 0
+STATUS_NAMES = {0: "GART_OK", 1: "GART_ERR_INVALID_ARG", 2: "GART_ERR_WORKSPACE_TOO_SMALL",
+                3: "GART_ERR_CAPACITY_EXCEEDED", 4: "GART_ERR_CUDA"}
+CNT_VISIBLE, CNT_PAIRS, CNT_SLOTS_LO, CNT_SLOTS_HI, CNT_HITS, CNT_ERROR, CNT_MAX_RAY_HITS, CNT_STRADDLE = range(8)
+COUNTS_WORDS = 8
+PRE_WORDS = 20
+GRAD_WORDS = 64
+
+EXPORTS = [
+    "gart_status_string", "gart_mask_words", "gart_bounds", "gart_tile_map_workspace_bytes", "gart_tile_map",
+    "gart_forward_workspace_bytes", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_read_counts",
+    "gart_view_host_arena_bytes", "gart_view_host",
+]
+
+
+class GartError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__("%s returned %s" % (where, STATUS_NAMES.get(int(status), status)))
+
+
+class _Config(C.Structure):
+    _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32)]
+
+
+class _Camera(C.Structure):
+    _fields_ = [("width", C.c_int32), ("height", C.c_int32), ("fx", C.c_double), ("fy", C.c_double),
+                ("cx", C.c_double), ("cy", C.c_double), ("w2c", C.c_double * 12)]
+
+
+class _Gaussians(C.Structure):
+    _fields_ = [("n", C.c_int64), ("sh_degree", C.c_int32), ("mean", C.c_void_p), ("scale", C.c_void_p),
+                ("quat", C.c_void_p), ("opacity", C.c_void_p), ("sh", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libgart.so is missing: build it with `python -m paper_2608_17298_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        L.gart_status_string.restype = C.c_char_p
+        L.gart_status_string.argtypes = [C.c_int]
+        L.gart_mask_words.restype = i32
+        L.gart_mask_words.argtypes = [i32]
+        L.gart_bounds.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.gart_tile_map_workspace_bytes.restype = sz
+        L.gart_tile_map_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
+        L.gart_tile_map.argtypes = [vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, sz, vp]
+        L.gart_forward_workspace_bytes.restype = sz
+        L.gart_forward_workspace_bytes.argtypes = [i32, i32, i32, i64, i64]
+        L.gart_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.gart_backward.argtypes = [vp] * 13
+        L.gart_backward_atomic.argtypes = [vp] * 12
+        L.gart_read_counts.argtypes = [vp, vp, vp]
+        L.gart_view_host_arena_bytes.restype = sz
+        L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
+        L.gart_view_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
+        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic",
+                   "gart_read_counts", "gart_view_host"):
+            getattr(L, fn).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+# ----------------------------------------------------------------------------------------- host structs
+@dataclasses.dataclass
+class Config:
+    alpha_min: float = 1.0 / 255.0
+    near_z: float = 0.01
+    background: tuple = (0.0, 0.0, 0.0)
+    tile_size: int = 8
+
+    def c(self) -> _Config:
+        s = _Config()
+        s.alpha_min, s.near_z, s.tile_size = self.alpha_min, self.near_z, int(self.tile_size)
+        for i in range(3):
+            s.background[i] = float(self.background[i])
+        return s
+
+    @property
+    def alpha_min_f32(self) -> float:
+        """The threshold as the library sees it (rounded to fp32)."""
+        return float(C.c_float(self.alpha_min).value)
+
+    @property
+    def near_f32(self) -> float:
+        return float(C.c_float(self.near_z).value)
+
+
+def camera_struct(cam) -> _Camera:
+    """``cam`` has width, height, fx, fy, cx, cy and a [3,4] world-to-camera matrix ``w2c``."""
+    s = _Camera()
+    s.width, s.height = int(cam.width), int(cam.height)
+    s.fx, s.fy, s.cx, s.cy = float(cam.fx), float(cam.fy), float(cam.cx), float(cam.cy)
+    flat = [float(v) for row in cam.w2c for v in row]
+    for i in range(12):
+        s.w2c[i] = flat[i]
+    return s
+
+
+def _dev(t, dtype, what):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CUDA tensor of dtype %s" % (what, dtype))
+    return t.data_ptr()
+
+
+@dataclasses.dataclass
+class Gaussians:
+    """Device-resident scene: fp32 CUDA tensors mean [n,3], scale [n,3], quat [n,4], opacity [n], sh [n,K,3]."""
+    mean: torch.Tensor
+    scale: torch.Tensor
+    quat: torch.Tensor
+    opacity: torch.Tensor
+    sh: torch.Tensor
+    sh_degree: int
+
+    @property
+    def n(self):
+        return int(self.mean.shape[0])
+
+    @classmethod
+    def from_numpy(cls, scene, device="cuda"):
+        f = lambda a: torch.from_numpy(a).to(device=device, dtype=torch.float32).contiguous()
+        return cls(f(scene.mean), f(scene.scale), f(scene.quat), f(scene.opacity), f(scene.sh), int(scene.sh_degree))
+
+    def c(self) -> _Gaussians:
+        K = (self.sh_degree + 1) ** 2
+        n = self.n
+        assert self.sh.shape == (n, K, 3) and self.scale.shape == (n, 3) and self.quat.shape == (n, 4)
+        s = _Gaussians()
+        s.n, s.sh_degree = n, int(self.sh_degree)
+        s.mean, s.scale = _dev(self.mean, torch.float32, "mean"), _dev(self.scale, torch.float32, "scale")
+        s.quat, s.opacity = _dev(self.quat, torch.float32, "quat"), _dev(self.opacity, torch.float32, "opacity")
+        s.sh = _dev(self.sh, torch.float32, "sh")
+        return s
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(status, where):
+    if status != GART_OK:
+        raise GartError(status, where)
+
+
+def tiles(cam, tile_size):
+    return -(-int(cam.width) // tile_size) * -(-int(cam.height) // tile_size)
+
+
+def gart_mask_words(tile_size: int) -> int:
+    return int(lib().gart_mask_words(int(tile_size)))
+
+
+# ----------------------------------------------------------------------------------------- the calls
+def gart_bounds(cfg: Config, g: Gaussians, cam, rect, cls, pre, counts, stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    _check(lib().gart_bounds(C.byref(c), C.byref(gs), C.byref(cs), _dev(rect, torch.int32, "rect"),
+                             _dev(cls, torch.uint8, "cls"), _dev(pre, torch.float32, "pre"),
+                             _dev(counts, torch.int32, "counts"), _stream_ptr(stream)), "gart_bounds")
+
+
+def gart_tile_map_workspace_bytes(n, width, height, tile_size, cap_pairs) -> int:
+    return int(lib().gart_tile_map_workspace_bytes(int(n), int(width), int(height), int(tile_size), int(cap_pairs)))
+
+
+def gart_tile_map(cfg: Config, rect, n, cam, tile_off, pair_gid, cap_pairs, counts, workspace, stream=None):
+    c = cfg.c()
+    _check(lib().gart_tile_map(C.byref(c), _dev(rect, torch.int32, "rect"), int(n), int(cam.width), int(cam.height),
+                               _dev(tile_off, torch.int32, "tile_off"), _dev(pair_gid, torch.int32, "pair_gid"),
+                               int(cap_pairs), _dev(counts, torch.int32, "counts"),
+                               _dev(workspace, torch.uint8, "workspace"), workspace.numel() if workspace is not None else 0,
+                               _stream_ptr(stream)), "gart_tile_map")
+
+
+def gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits) -> int:
+    return int(lib().gart_forward_workspace_bytes(int(width), int(height), int(tile_size), int(cap_pairs), int(cap_hits)))
+
+
+def gart_forward(cfg: Config, g: Gaussians, cam, pre, tile_off, pair_gid, cap_pairs, color, t_final, hit_count,
+                 pair_mask, pair_lt_off, lt, cap_hits, ray_off, ray_gid, ray_slot, counts, workspace, stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    i32, f32 = torch.int32, torch.float32
+    _check(lib().gart_forward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
+                              _dev(pair_gid, i32, "pair_gid"), int(cap_pairs), _dev(color, f32, "color"),
+                              _dev(t_final, f32, "t_final"), _dev(hit_count, i32, "hit_count"),
+                              _dev(pair_mask, i32, "pair_mask"), _dev(pair_lt_off, i32, "pair_lt_off"),
+                              _dev(lt, f32, "lt"), int(cap_hits), _dev(ray_off, i32, "ray_off"),
+                              _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"),
+                              _dev(counts, i32, "counts"), _dev(workspace, torch.uint8, "workspace"),
+                              workspace.numel() if workspace is not None else 0, _stream_ptr(stream)), "gart_forward")
+
+
+def gart_backward(cfg: Config, g: Gaussians, cam, pre, tile_off, pair_gid, pair_mask, pair_lt_off, lt, dL_dcolor,
+                  grad, counts, stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    i32, f32 = torch.int32, torch.float32
+    _check(lib().gart_backward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
+                               _dev(pair_gid, i32, "pair_gid"), _dev(pair_mask, i32, "pair_mask"),
+                               _dev(pair_lt_off, i32, "pair_lt_off"), _dev(lt, f32, "lt"),
+                               _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"), _dev(counts, i32, "counts"),
+                               _stream_ptr(stream)), "gart_backward")
+
+
+def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, ray_off, ray_gid, ray_slot, lt, dL_dcolor, grad, counts,
+                         stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    i32, f32 = torch.int32, torch.float32
+    _check(lib().gart_backward_atomic(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                                      _dev(ray_off, i32, "ray_off"), _dev(ray_gid, i32, "ray_gid"),
+                                      _dev(ray_slot, i32, "ray_slot"), _dev(lt, f32, "lt"),
+                                      _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
+                                      _dev(counts, i32, "counts"), _stream_ptr(stream)), "gart_backward_atomic")
+
+
+def gart_read_counts(counts, stream=None):
+    """Counts block as a list of 8 unsigned ints (synchronises the stream)."""
+    host = (C.c_uint32 * COUNTS_WORDS)()
+    _check(lib().gart_read_counts(_dev(counts, torch.int32, "counts"), host, _stream_ptr(stream)), "gart_read_counts")
+    return [int(v) for v in host]
+
+
+def gart_view_host_arena_bytes(n, sh_degree, width, height, tile_size, cap_pairs, cap_hits) -> int:
+    return int(lib().gart_view_host_arena_bytes(int(n), int(sh_degree), int(width), int(height), int(tile_size),
+                                                int(cap_pairs), int(cap_hits)))
+
+
+def gart_view_host(cfg: Config, scene, cam, dL_dcolor, color_out, grad_out, cap_pairs, cap_hits, arena, stream=None):
+    """End-to-end call on HOST (CPU, ideally pinned) fp32 tensors; ``arena`` is a CUDA uint8 tensor.
+
+    ``scene`` has CPU tensors mean, scale, quat, opacity, sh and ``sh_degree``.  Returns the counts block.
+    """
+    def host(t, what):
+        if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+            raise TypeError("%s must be a contiguous CPU float32 tensor" % what)
+        return t.data_ptr()
+    gs = _Gaussians()
+    gs.n, gs.sh_degree = int(scene.mean.shape[0]), int(scene.sh_degree)
+    gs.mean, gs.scale, gs.quat = host(scene.mean, "mean"), host(scene.scale, "scale"), host(scene.quat, "quat")
+    gs.opacity, gs.sh = host(scene.opacity, "opacity"), host(scene.sh, "sh")
+    c, cs = cfg.c(), camera_struct(cam)
+    counts = (C.c_uint32 * COUNTS_WORDS)()
+    st = lib().gart_view_host(C.byref(c), C.byref(gs), C.byref(cs), host(dL_dcolor, "dL_dcolor"), host(color_out, "color_out"),
+                              host(grad_out, "grad_out"), int(cap_pairs), int(cap_hits), counts,
+                              _dev(arena, torch.uint8, "arena"), arena.numel(), _stream_ptr(stream))
+    out = [int(v) for v in counts]
+    if st != GART_OK:
+        err = GartError(st, "gart_view_host")
+        err.counts = out
+        raise err
+    return out
+
+
+# ----------------------------------------------------------------------------------------- buffer plumbing
+class ViewBuffers:
+    """Device buffers of one view, allocated once for given capacities and reused across views."""
+
+    def __init__(self, n, sh_degree, cam, cfg: Config, cap_pairs, cap_hits, device="cuda"):
+        ts = cfg.tile_size
+        self.n, self.cap_pairs, self.cap_hits = int(n), int(cap_pairs), int(cap_hits)
+        H, W = int(cam.height), int(cam.width)
+        T = tiles(cam, ts)
+        mw = ts * ts // 32
+        i32, f32, u8 = torch.int32, torch.float32, torch.uint8
+        e = lambda shape, dt: torch.empty(shape, dtype=dt, device=device)
+        n1, cp, ch = max(self.n, 1), max(self.cap_pairs, 1), max(self.cap_hits, 1)
+        self.rect, self.cls, self.pre = e((n1, 4), i32), e((n1,), u8), e((n1, PRE_WORDS), f32)
+        self.counts = torch.zeros(COUNTS_WORDS, dtype=i32, device=device)
+        self.tile_off, self.pair_gid = e((T + 1,), i32), e((cp,), i32)
+        self.pair_mask, self.pair_lt_off = e((cp, mw), i32), e((cp + 1,), i32)
+        self.color, self.t_final, self.hit_count = e((H, W, 3), f32), e((H, W), f32), e((H, W), i32)
+        self.lt = e((ch, 4), f32)
+        self.ray_off, self.ray_gid, self.ray_slot = e((H * W + 1,), i32), e((ch,), i32), e((ch,), i32)
+        self.grad = e((n1, GRAD_WORDS), f32)
+        ws = max(gart_tile_map_workspace_bytes(n1, W, H, ts, cap_pairs), gart_forward_workspace_bytes(W, H, ts, cap_pairs, cap_hits))
+        self.workspace = e((ws,), u8)
+
+    def bytes(self):
+        return sum(t.numel() * t.element_size() for t in vars(self).values() if isinstance(t, torch.Tensor))
+
+
+def run_bounds_tile_map(cfg, g, cam, buf: ViewBuffers, stream=None):
+    gart_bounds(cfg, g, cam, buf.rect, buf.cls, buf.pre, buf.counts, stream)
+    gart_tile_map(cfg, buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.counts, buf.workspace, stream)
+
+
+def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None):
+    gart_forward(cfg, g, cam, buf.pre, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color, buf.t_final, buf.hit_count,
+                 buf.pair_mask, buf.pair_lt_off, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot,
+                 buf.counts, buf.workspace, stream)
+
+
+def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
+    gart_backward(cfg, g, cam, buf.pre, buf.tile_off, buf.pair_gid, buf.pair_mask, buf.pair_lt_off, buf.lt, dL_dcolor,
+                  buf.grad if grad is None else grad, buf.counts, stream)
+
+
+def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):
+    gart_backward_atomic(cfg, g, cam, buf.pre, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.lt, dL_dcolor, grad,
+                         buf.counts, stream)
+
+
+def size_view(cfg, g, cam, slack=1.0, device="cuda"):
+    """Run bounds + tile map with a probing allocation and return (P, S): exact pair count and the
+    capacity bound of the intermediate buffer (sum of rectangle areas).  Two host round trips; meant
+    for set-up, not for the steady state."""
+    probe = ViewBuffers(g.n, g.sh_degree, cam, cfg, 0, 0, device)
+    run_bounds_tile_map(cfg, g, cam, probe)
+    cnt = gart_read_counts(probe.counts)
+    P = cnt[CNT_PAIRS]
+    S = cnt[CNT_SLOTS_LO] | (cnt[CNT_SLOTS_HI] << 32)
+    return int(P * slack) + 1, int(S * slack) + 1

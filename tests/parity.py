@@ -1,0 +1,196 @@
+"""Helpers of the GPU parity tests: run the CUDA path, run the oracle, compare.
+
+Comparison protocol
+-------------------
+Integer artefacts (rectangles, classes, tile lists) must be identical, except for a Gaussian
+whose float64 decision margin is below 1e-9 (a pixel-centre exactly on a bound).
+
+Hit decisions and the per-ray order are taken in fp32 on the GPU and in float64 by the oracle.
+A decision may differ only inside a guard band: a hit present on one side only must have
+|ln(alpha / alpha_min)| < BAND_HIT in float64, and the GPU's order of two consecutive hits
+may differ from the (t*, id) order only if their float64 t* agree within BAND_ORDER (relative).
+Such cases are counted and reported; the oracle then composites and differentiates the GPU's
+own hit lists ("replay"), so that colour and gradient tolerances apply to every ray.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import paper_2608_17298_b200.gart as G
+from oracle import gart_oracle as orc
+
+BAND_HIT = 2e-4
+BAND_ORDER = 2e-5
+
+
+def to_np(t):
+    return t.detach().cpu().numpy()
+
+
+def u32(a):
+    return a.view(np.uint32) if a.dtype == np.int32 else a
+
+
+def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, atomic=True):
+    """Full device path for one view; returns numpy copies of every output."""
+    g = G.Gaussians.from_numpy(scene)
+    if cap_pairs is None or cap_hits is None:
+        P, S = G.size_view(cfg, g, cam, slack=1.0)
+        cap_pairs = P if cap_pairs is None else cap_pairs
+        cap_hits = S if cap_hits is None else cap_hits
+    buf = G.ViewBuffers(g.n, g.sh_degree, cam, cfg, cap_pairs, cap_hits)
+    dl = torch.from_numpy(np.ascontiguousarray(dL_dC, dtype=np.float32)).cuda()
+    G.run_bounds_tile_map(cfg, g, cam, buf)
+    G.run_forward(cfg, g, cam, buf)
+    G.run_backward(cfg, g, cam, buf, dl)
+    counts = G.gart_read_counts(buf.counts)
+    out = {"counts": counts, "buf": buf, "g": g, "dl": dl}
+    P, H = counts[G.CNT_PAIRS], counts[G.CNT_HITS]
+    out["rect"], out["cls"] = to_np(buf.rect)[:g.n], to_np(buf.cls)[:g.n]
+    out["tile_off"] = u32(to_np(buf.tile_off))
+    if counts[G.CNT_ERROR]:
+        return out
+    out["pair_gid"] = u32(to_np(buf.pair_gid))[:P]
+    out["pair_mask"] = u32(to_np(buf.pair_mask))[:P]
+    out["pair_lt_off"] = u32(to_np(buf.pair_lt_off))[:P + 1]
+    out["color"], out["t_final"] = to_np(buf.color), to_np(buf.t_final)
+    out["hit_count"] = u32(to_np(buf.hit_count))
+    out["ray_off"] = u32(to_np(buf.ray_off))
+    out["ray_gid"] = u32(to_np(buf.ray_gid))[:H]
+    out["ray_slot"] = u32(to_np(buf.ray_slot))[:H]
+    out["lt"] = to_np(buf.lt)[:H]
+    out["grad"] = to_np(buf.grad)[:g.n].copy()
+    if atomic:
+        ga = torch.empty_like(buf.grad)
+        G.run_backward_atomic(cfg, g, cam, buf, dl, ga)
+        torch.cuda.synchronize()
+        out["grad_atomic"] = to_np(ga)[:g.n]
+    return out
+
+
+def check_maps(scene, cam, cfg: G.Config, gpu):
+    """Rectangles, classes and tile lists against the oracle (bit-exact outside the 1e-9 margin)."""
+    osc = orc.OracleScene.from_scene(scene)
+    rect, cls, margin = orc.bounds(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    safe = margin > 1e-9
+    assert safe.mean() > 0.999
+    assert np.array_equal(gpu["cls"][safe], cls[safe])
+    assert np.array_equal(gpu["rect"][safe], rect[safe])
+    same = np.array_equal(gpu["rect"], rect)
+    # tile lists follow from the rectangles: check them against the oracle on the GPU's rectangles
+    # (identical to the oracle's own unless a sub-1e-9 margin flipped an edge)
+    tile_off, pair_gid, slots = orc.tile_map(gpu["rect"], cam.width, cam.height, cfg.tile_size)
+    assert np.array_equal(gpu["tile_off"], tile_off)
+    assert np.array_equal(gpu["pair_gid"], pair_gid)
+    c = gpu["counts"]
+    assert c[G.CNT_PAIRS] == len(pair_gid)
+    assert (c[G.CNT_SLOTS_LO] | (c[G.CNT_SLOTS_HI] << 32)) == slots
+    assert c[G.CNT_VISIBLE] == int((gpu["rect"][:, 2] >= gpu["rect"][:, 0]).sum())
+    return {"rect_identical": bool(same), "n_unsafe": int((~safe).sum()), "osc": osc}
+
+
+def check_structure(cam, cfg: G.Config, gpu):
+    """Properties that hold at any size, checked on the whole view without the oracle."""
+    H = gpu["counts"][G.CNT_HITS]
+    ray_off, hit_count = gpu["ray_off"].astype(np.int64), gpu["hit_count"].reshape(-1).astype(np.int64)
+    assert ray_off[0] == 0 and ray_off[-1] == H and np.array_equal(np.diff(ray_off), hit_count)
+    # pair masks: popcounts give the LT offsets; every hit owns exactly one slot
+    pc = np.unpackbits(gpu["pair_mask"].view(np.uint8), axis=1).sum(axis=1).astype(np.int64)
+    off = gpu["pair_lt_off"].astype(np.int64)
+    assert off[0] == 0 and off[-1] == H and np.array_equal(np.diff(off), pc)
+    slots = np.sort(gpu["ray_slot"].astype(np.int64))
+    assert np.array_equal(slots, np.arange(H))
+    assert gpu["counts"][G.CNT_MAX_RAY_HITS] == (hit_count.max() if hit_count.size else 0)
+    # a hit's slot belongs to the pair (tile of the ray, its Gaussian)
+    ts = cfg.tile_size
+    tiles_x = -(-cam.width // ts)
+    rays = np.repeat(np.arange(hit_count.size), hit_count)
+    tile = (rays // cam.width) // ts * tiles_x + (rays % cam.width) // ts
+    pair = np.searchsorted(off, gpu["ray_slot"].astype(np.int64), side="right") - 1
+    assert np.array_equal(gpu["pair_gid"][pair], gpu["ray_gid"])
+    tile_of_pair = np.searchsorted(gpu["tile_off"].astype(np.int64), pair, side="right") - 1
+    assert np.array_equal(tile_of_pair, tile)
+    # LT: transmittance of the first hit of a ray is 1; of later hits in (0, 1]; colours finite
+    lt = gpu["lt"]
+    first = ray_off[:-1][hit_count > 0]
+    assert np.all(lt[gpu["ray_slot"][first].astype(np.int64), 3] == 1.0)
+    assert np.all(np.isfinite(lt)) and np.all(lt[:, 3] >= 0) and np.all(lt[:, 3] <= 1.0)
+    assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
+
+
+def _lists_for(ray_off, gid, rays):
+    """Sub-lists of the selected rays as (ray_off_full [n_rays+1], gid) with other rays empty."""
+    n_rays = ray_off.size - 1
+    cnt = np.zeros(n_rays, dtype=np.int64)
+    cnt[rays] = (ray_off[rays + 1] - ray_off[rays]).astype(np.int64)
+    new_off = np.zeros(n_rays + 1, dtype=np.uint64)
+    new_off[1:] = np.cumsum(cnt)
+    idx = np.concatenate([np.arange(ray_off[r], ray_off[r + 1], dtype=np.int64) for r in rays]) if len(rays) else np.zeros(0, np.int64)
+    return new_off, gid[idx].astype(np.uint32)
+
+
+def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, mode=orc.BRUTE):
+    """Compare the GPU's per-ray hit lists with the oracle's on the selected rays, under the guard
+    band protocol; then replay the GPU's lists through the oracle.  Returns the replayed view's
+    colour, t_final, gradient, gradient conditioning and statistics."""
+    n_rays = cam.width * cam.height
+    sel = np.arange(n_rays) if pixel_mask is None else np.nonzero(pixel_mask.reshape(-1))[0]
+    v = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background)
+    v.find_hits(mode, pixel_mask)
+    o_off, o_gid, o_t, o_alpha = v.hits()
+    g_off, g_gid = gpu["ray_off"].astype(np.int64), gpu["ray_gid"]
+    o_off = o_off.astype(np.int64)
+    stats = {"rays": int(sel.size), "oracle_hits": int(o_off[-1]), "band_hit": 0, "band_order": 0}
+    g_cnt, o_cnt = g_off[sel + 1] - g_off[sel], o_off[sel + 1] - o_off[sel]
+    # fast path: concatenate selected lists and compare wholesale
+    g_new_off, g_sel_gid = _lists_for(gpu["ray_off"].astype(np.int64), g_gid, sel)
+    identical = np.array_equal(g_cnt, o_cnt) and np.array_equal(g_sel_gid, o_gid)
+    if not identical:
+        amin = cfg.alpha_min_f32
+        for k, r in enumerate(sel):
+            gl = g_gid[g_off[r]:g_off[r + 1]]
+            ol = o_gid[o_off[r]:o_off[r + 1]]
+            if gl.size == ol.size and np.array_equal(gl, ol):
+                continue
+            gs, os_ = set(gl.tolist()), set(ol.tolist())
+            for gid in gs ^ os_:
+                alpha, t = v.eval_pair(int(r), int(gid))
+                assert abs(np.log(alpha / amin)) < BAND_HIT or (alpha >= amin and abs(t) < 1e-6), \
+                    ("hit decision differs outside the guard band", int(r), int(gid), alpha, t)
+                stats["band_hit"] += 1
+            # order of the GPU list must be non-decreasing in float64 t* up to the band
+            ts_ = np.array([v.eval_pair(int(r), int(gid))[1] for gid in gl])
+            if ts_.size > 1:
+                viol = ts_[:-1] > ts_[1:] * (1 + BAND_ORDER)
+                assert not viol.any(), ("order differs outside the guard band", int(r))
+                eq = np.abs(ts_[:-1] - ts_[1:]) <= BAND_ORDER * np.abs(ts_[1:])
+                # equal within the band: either order accepted; exact ties must ascend in id
+                exact = ts_[:-1] == ts_[1:]
+                assert np.all(gl[:-1][exact] < gl[1:][exact])
+                common = [x for x in gl.tolist() if x in os_]
+                common_o = [x for x in ol.tolist() if x in gs]
+                stats["band_order"] += int(common != common_o)
+    stats["identical_lists"] = bool(identical)
+    assert stats["band_hit"] + stats["band_order"] <= max(2, 1e-3 * stats["oracle_hits"])
+    # replay the GPU's lists
+    v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background)
+    v2.set_hits(g_new_off, g_sel_gid)
+    color, t_final, cnt = v2.composite()
+    grad, gabs = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True)
+    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "stats": stats, "sel": sel, "view": v2}
+
+
+def color_errors(gpu, ref, sel, cam):
+    c_g = gpu["color"].reshape(-1, 3)[sel].astype(np.float64)
+    c_o = ref["color"].reshape(-1, 3)[sel]
+    t_g = gpu["t_final"].reshape(-1)[sel].astype(np.float64)
+    t_o = ref["t_final"].reshape(-1)[sel]
+    return np.abs(c_g - c_o), np.abs(c_o), np.abs(t_g - t_o), np.abs(t_o)
+
+
+def pack_grad(grad64, K):
+    """Oracle layout [n, 11+3K] -> library layout [n, 64]."""
+    out = np.zeros((grad64.shape[0], G.GRAD_WORDS))
+    out[:, :11 + 3 * K] = grad64
+    return out

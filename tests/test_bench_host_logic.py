@@ -1,0 +1,56 @@
+"""Host logic of the benchmark: view sharding, launch counting, byte accounting, and the
+max-over-ranks / sum-over-ranks aggregation on two gloo ranks (CPU)."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import bench
+
+
+def test_shard_views_partition():
+    for world in (1, 2, 3, 4, 8, 16, 32):
+        seen = []
+        for r in range(world):
+            mine = bench.shard_views(16, r, world)
+            assert len(mine) >= 1
+            seen += mine
+        if world <= 16:
+            assert sorted(seen) == list(range(16))
+
+
+def test_launch_count_and_bytes():
+    assert bench.launches_per_step(155 * 103) == 1 + (7 + 2 * 5) + 10 + 2     # 14 tile bits -> 2 radix passes
+    assert bench.launches_per_step(64) == 1 + (7 + 5) + 10 + 2
+    B = bench.algorithmic_bytes_backward(H=100, P=10, n_vis=5, n_pixels=64, K=16, mask_words=2)
+    assert B == 1600 + 160 + 4 * 68 * 5 + 4 * 59 * 5 + 768
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = bench.shard_views(16, rank, world)
+    t = torch.tensor([10.0 + rank], dtype=torch.float64)
+    h = torch.tensor([float(len(mine))], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(h, op=dist.ReduceOp.SUM)
+    if rank == 0:
+        out.put((t.item(), h.item()))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_aggregation_gloo():
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    tmax, hsum = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    assert tmax == 11.0 and hsum == 16.0

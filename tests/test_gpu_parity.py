@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA path (through the C ABI) against the float64 oracle, element by element.
+
+Tolerances (written here, derived in the design doc):
+  * rectangles, classes, tile offsets, pair lists, per-ray hit counts and ordered hit lists:
+    bit-exact, up to the guard-band protocol of tests/parity.py;
+  * colour: |gpu - ref| <= 1e-4 |ref| + 1e-7; final transmittance: 1e-4 |ref| + 1e-6;
+  * gradients (all 11+3K words, both backward variants): |gpu - ref| <= 1e-3 max(|ref|, COND * A)
+    or <= 1e-6, where A is the sum of the absolute values of the per-hit terms of that word (its
+    conditioning).  A sum whose terms cancel to less than COND = 2% of their mass cannot reach a
+    relative 1e-3 in fp32 in any summation order, so the relative bar is measured against that floor.
+"""
+import numpy as np
+import pytest
+import torch
+
+import gart_scenes as gs
+import paper_2608_17298_b200.gart as G
+from oracle import gart_oracle as orc
+
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+COND = 0.02
+
+
+def assert_color(gpu, ref, sel, cam):
+    dc, ac, dt, at = P.color_errors(gpu, ref, sel, cam)
+    assert np.all(dc <= 1e-4 * ac + 1e-7), float((dc / np.maximum(ac, 1e-30)).max())
+    assert np.all(dt <= 1e-4 * at + 1e-6)
+
+
+def assert_grad(gpu_grad, ref, K, rows=None):
+    gw = 11 + 3 * K
+    rows = np.arange(ref["grad"].shape[0]) if rows is None else rows
+    g = gpu_grad[rows][:, :gw].astype(np.float64)
+    r, a = ref["grad"][rows], ref["gabs"][rows]
+    d = np.abs(g - r)
+    ok = (d <= 1e-3 * np.maximum(np.abs(r), COND * a)) | (d <= 1e-6)
+    assert ok.all(), ("gradient outside tolerance", int((~ok).sum()), float(d[~ok].max()))
+    assert np.all(gpu_grad[rows][:, gw:] == 0)
+    strict = (d <= 1e-3 * np.abs(r)) | (d <= 1e-6)
+    return float(strict.mean())
+
+
+def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
+    g = gs.upstream_gradient(cam, 0) if g is None else g
+    gpu = P.run_gpu(scene, cam, cfg, g)
+    assert gpu["counts"][G.CNT_ERROR] == 0
+    m = P.check_maps(scene, cam, cfg, gpu)
+    P.check_structure(cam, cfg, gpu)
+    ref = P.check_hits_and_replay(m["osc"], cam, cfg, gpu, g, None, mode)
+    assert_color(gpu, ref, ref["sel"], cam)
+    K = (scene.sh_degree + 1) ** 2
+    s1 = assert_grad(gpu["grad"], ref, K)
+    s2 = assert_grad(gpu["grad_atomic"], ref, K)
+    assert s1 > 0.995 and s2 > 0.995            # the conditioning floor is the exception, not the rule
+    return gpu, ref
+
+
+# ------------------------------------------------------------------------------------------ small configs, every ray
+@pytest.mark.parametrize("ts", [8, 16])
+def test_tiny_exact_lists_and_values(ts):
+    scene, cams = gs.config_tiny()
+    gpu, ref = full_parity(scene, cams[0], G.Config(tile_size=ts))
+    st = ref["stats"]
+    assert st["identical_lists"] and st["band_hit"] == 0 and st["band_order"] == 0   # no guard-band case at all on Tiny
+    assert gpu["counts"][G.CNT_HITS] == st["oracle_hits"]
+
+
+@pytest.mark.parametrize("deg", [0, 1, 2, 3])
+def test_tiny_all_sh_degrees(deg):
+    scene, cams = gs.config_tiny(sh_degree=deg, seed=deg + 1)
+    full_parity(scene, cams[0], G.Config(tile_size=8))
+
+
+@pytest.mark.parametrize("ts", [8, 16])
+def test_cluster10k_every_ray(ts):
+    scene, cams = gs.config_cluster()
+    gpu, ref = full_parity(scene, cams[0], G.Config(tile_size=ts))
+    assert ref["stats"]["band_hit"] + ref["stats"]["band_order"] <= 1e-4 * ref["stats"]["oracle_hits"]
+
+
+def test_ragged_image_and_background():
+    scene, cams = gs.config_tiny(width=61, height=37, sh_degree=2, seed=5)
+    for ts in (8, 16):
+        full_parity(scene, cams[0], G.Config(tile_size=ts, background=(0.2, 0.5, 0.1)))
+
+
+def test_straddling_gaussian_and_culling_rules():
+    scene, cams = gs.config_tiny(n=64, seed=9)
+    scene.mean[0] = (0.05, -0.02, 0.3); scene.scale[0] = (0.4, 0.5, 0.45); scene.opacity[0] = 0.6   # crosses the camera plane
+    scene.mean[1] = (9.0, 0.0, 0.2); scene.scale[1] = (0.3, 0.3, 0.3)                              # straddles, outside the frustum
+    scene.mean[2] = (0.0, 0.0, -2.0)                                                                 # behind
+    scene.opacity[3] = 0.003                                                                          # below alpha_min
+    scene.mean[4] = (30.0, 0.0, 3.0)                                                                  # off screen
+    gpu, ref = full_parity(scene, cams[0], G.Config(tile_size=8))
+    assert list(gpu["cls"][:5]) == [2, 2, 0, 0, 1]
+    assert list(gpu["rect"][0]) == [0, 0, 63, 63] and list(gpu["rect"][1]) == [0, 0, -1, -1]
+    assert gpu["counts"][G.CNT_STRADDLE] == 2
+    assert np.any(gpu["grad"][0] != 0) and np.all(gpu["grad"][1:5] == 0)
+
+
+def test_rays_longer_than_the_shared_memory_sort():
+    """More than 1024 hits on a ray: the per-ray sort falls back to global memory."""
+    rng = np.random.default_rng(3)
+    n = 1400
+    mean = np.stack([rng.normal(0, 0.02, n), rng.normal(0, 0.02, n), rng.uniform(2.0, 6.0, n)], 1)
+    scene = gs.Scene(mean.astype(np.float32), np.full((n, 3), 0.25, np.float32) * rng.uniform(0.8, 1.2, (n, 3)).astype(np.float32),
+                     gs._unit_quats(rng, n).astype(np.float32), rng.uniform(0.01, 0.03, n).astype(np.float32),
+                     gs._sh(rng, n, 1), 1)
+    cam = gs.pinhole(16, 16, 20.0)
+    gpu, ref = full_parity(scene, cam, G.Config(tile_size=8))
+    assert gpu["counts"][G.CNT_MAX_RAY_HITS] > 1024
+
+
+def test_primitive_and_atomic_backward_agree():
+    scene, cams = gs.config_cluster(n=3000, width=128, height=96)
+    g = gs.upstream_gradient(cams[0], 1)
+    gpu = P.run_gpu(scene, cams[0], G.Config(tile_size=8), g)
+    a, b = gpu["grad"].astype(np.float64), gpu["grad_atomic"].astype(np.float64)
+    scale = np.maximum(np.abs(a), np.abs(b))
+    close = np.abs(a - b) <= 1e-3 * scale + 1e-5 * np.abs(a).max(axis=1, keepdims=True) + 1e-6
+    assert close.all()
+
+
+# ------------------------------------------------------------------------------------------ full-size configs, sampled
+def sampled_parity(scene, cam, cfg, view_seed, n_gauss=300, n_tiles=60, max_area=3000):
+    """Full-size view on the GPU; the oracle handles a sample: random tiles plus every pixel of the
+    rectangles of randomly chosen Gaussians, so that those Gaussians' gradients are complete."""
+    g = gs.upstream_gradient(cam, view_seed)
+    gpu = P.run_gpu(scene, cam, cfg, g, atomic=True)
+    assert gpu["counts"][G.CNT_ERROR] == 0
+    m = P.check_maps(scene, cam, cfg, gpu)
+    P.check_structure(cam, cfg, gpu)
+    rng = np.random.default_rng([view_seed, 77])
+    rect = gpu["rect"]
+    area = (rect[:, 2] - rect[:, 0] + 1) * (rect[:, 3] - rect[:, 1] + 1)
+    cand = np.nonzero((rect[:, 2] >= rect[:, 0]) & (area <= max_area))[0]
+    gsel = rng.choice(cand, size=min(n_gauss, cand.size), replace=False)
+    mask = np.zeros((cam.height, cam.width), np.uint8)
+    for i in gsel:
+        x0, y0, x1, y1 = rect[i]
+        mask[y0:y1 + 1, x0:x1 + 1] = 1
+    ts = 8
+    for _ in range(n_tiles):
+        ty, tx = int(rng.integers(-(-cam.height // ts))), int(rng.integers(-(-cam.width // ts)))
+        mask[ty * ts:(ty + 1) * ts, tx * ts:(tx + 1) * ts] = 1
+    ref = P.check_hits_and_replay(m["osc"], cam, cfg, gpu, g, mask, orc.PREFILTER)
+    assert ref["stats"]["oracle_hits"] > 1000
+    assert_color(gpu, ref, ref["sel"], cam)
+    K = (scene.sh_degree + 1) ** 2
+    assert_grad(gpu["grad"], ref, K, gsel)
+    assert_grad(gpu["grad_atomic"], ref, K, gsel)
+    # the prefilter of the oracle is audited by true all-pairs brute force on a few rays
+    audit = np.zeros_like(mask)
+    ys, xs = np.nonzero(mask)
+    pick = rng.choice(ys.size, size=min(24, ys.size), replace=False)
+    audit[ys[pick], xs[pick]] = 1
+    va = orc.View(m["osc"], cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    va.find_hits(orc.BRUTE, audit)
+    vb = orc.View(m["osc"], cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    vb.find_hits(orc.PREFILTER, audit)
+    for p, q in zip(va.hits(), vb.hits()):
+        assert np.array_equal(p, q)
+    return gpu, ref
+
+
+@pytest.mark.parametrize("view", [0, 2])
+def test_shell200k_sampled(view):
+    scene, cams = gs.config_shell()
+    sampled_parity(scene, cams[view], G.Config(tile_size=8), view)
+
+
+def test_unbounded1m_sampled():
+    scene, cams = gs.config_unbounded_1m()
+    sampled_parity(scene, cams[0], G.Config(tile_size=8), 0)
+    sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=100, n_tiles=20)
+
+
+def test_unbounded6m_sampled():
+    """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles)."""
+    scene, cams = gs.config_unbounded_6m()
+    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=200, n_tiles=40)
+    assert gpu["counts"][G.CNT_HITS] > 1e8
+
+
+# ------------------------------------------------------------------------------------------ edge cases and errors
+def _empty_scene(deg=1):
+    K = (deg + 1) ** 2
+    z = lambda *s: np.zeros(s, np.float32)
+    return gs.Scene(z(0, 3), z(0, 3), z(0, 4), z(0), z(0, K, 3), deg)
+
+
+def test_no_gaussians():
+    cam = gs.pinhole(40, 24, 50.0)
+    cfg = G.Config(tile_size=8, background=(0.3, 0.1, 0.7))
+    gpu = P.run_gpu(_empty_scene(), cam, cfg, gs.upstream_gradient(cam, 0), cap_pairs=0, cap_hits=0, atomic=False)
+    c = gpu["counts"]
+    assert c[G.CNT_PAIRS] == 0 and c[G.CNT_HITS] == 0 and c[G.CNT_ERROR] == 0
+    assert np.all(gpu["tile_off"] == 0) and np.all(gpu["hit_count"] == 0)
+    assert np.allclose(gpu["color"], np.array([0.3, 0.1, 0.7], np.float32)) and np.all(gpu["t_final"] == 1)
+
+
+def test_everything_culled():
+    scene, cams = gs.config_tiny(n=50)
+    scene.opacity[:] = 0.002
+    gpu = P.run_gpu(scene, cams[0], G.Config(), gs.upstream_gradient(cams[0], 0), atomic=True)
+    assert gpu["counts"][G.CNT_VISIBLE] == 0 and gpu["counts"][G.CNT_PAIRS] == 0 and gpu["counts"][G.CNT_HITS] == 0
+    assert np.all(gpu["grad"] == 0) and np.all(gpu["grad_atomic"] == 0) and np.all(gpu["color"] == 0)
+    assert np.all(gpu["cls"] == 0) and np.all(gpu["rect"] == np.array([0, 0, -1, -1]))
+
+
+def test_capacity_errors_are_reported_not_fatal():
+    scene, cams = gs.config_tiny()
+    cam, cfg = cams[0], G.Config()
+    g = gs.upstream_gradient(cam, 0)
+    gpu = P.run_gpu(scene, cam, cfg, g, cap_pairs=100, cap_hits=20000, atomic=False)
+    assert gpu["counts"][G.CNT_ERROR] & 1 and gpu["counts"][G.CNT_PAIRS] == 683 and np.all(gpu["tile_off"] == 0)
+    gpu = P.run_gpu(scene, cam, cfg, g, cap_pairs=700, cap_hits=500, atomic=False)
+    assert gpu["counts"][G.CNT_ERROR] == 2 and gpu["counts"][G.CNT_HITS] == 7373
+    # and the context is still usable afterwards
+    gpu = P.run_gpu(scene, cam, cfg, g, atomic=False)
+    assert gpu["counts"][G.CNT_ERROR] == 0 and gpu["counts"][G.CNT_HITS] == 7373
+
+
+def test_invalid_arguments_return_status():
+    scene, cams = gs.config_tiny(n=8)
+    cam = cams[0]
+    g = G.Gaussians.from_numpy(scene)
+    buf = G.ViewBuffers(g.n, 0, cam, G.Config(), 100, 1000)
+    with pytest.raises(G.GartError) as e:
+        G.gart_bounds(G.Config(tile_size=12), g, cam, buf.rect, buf.cls, buf.pre, buf.counts)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
+        G.gart_bounds(G.Config(), g, cam, None, buf.cls, buf.pre, buf.counts)
+    assert e.value.status == 1
+    G.gart_bounds(G.Config(), g, cam, buf.rect, buf.cls, buf.pre, buf.counts)
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(G.GartError) as e:
+        G.gart_tile_map(G.Config(), buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, 100, buf.counts, small)
+    assert e.value.status == 2
+    with pytest.raises(G.GartError) as e:
+        G.gart_tile_map(G.Config(), buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, 100, buf.counts, buf.workspace[1:])
+    assert e.value.status == 1                     # workspace not 256-byte aligned
+    g.sh_degree = 3
+    with pytest.raises(AssertionError):
+        g.c()
+    assert G.lib().gart_status_string(3) == b"capacity exceeded"
+    torch.cuda.synchronize()
+
+
+def test_host_entry_point_matches_device_path():
+    scene, cams = gs.config_cluster(n=2000, width=96, height=64)
+    cam, cfg = cams[0], G.Config(tile_size=8)
+    g = gs.upstream_gradient(cam, 0)
+    gpu = P.run_gpu(scene, cam, cfg, g, atomic=False)
+    Pn, Hn = gpu["counts"][G.CNT_PAIRS], gpu["counts"][G.CNT_HITS]
+
+    class HS:
+        pass
+    hs = HS()
+    for k in ("mean", "scale", "quat", "opacity", "sh"):
+        setattr(hs, k, torch.from_numpy(getattr(scene, k)).pin_memory())
+    hs.sh_degree = scene.sh_degree
+    color = torch.empty((cam.height, cam.width, 3), dtype=torch.float32).pin_memory()
+    grad = torch.empty((scene.n, G.GRAD_WORDS), dtype=torch.float32).pin_memory()
+    arena = torch.empty(G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam.width, cam.height, 8, Pn + 5, Hn + 5),
+                        dtype=torch.uint8, device="cuda")
+    counts = G.gart_view_host(cfg, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Hn + 5, arena)
+    assert counts[G.CNT_HITS] == Hn and counts[G.CNT_PAIRS] == Pn
+    assert np.array_equal(color.numpy(), gpu["color"])
+    a, b = grad.numpy().astype(np.float64), gpu["grad"].astype(np.float64)
+    assert np.all(np.abs(a - b) <= 1e-4 * np.abs(b) + 1e-5 * np.abs(b).max(axis=1, keepdims=True) + 1e-7)
+    with pytest.raises(G.GartError) as e:
+        G.gart_view_host(cfg, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Hn // 2, arena)
+    assert e.value.status == 3

@@ -1,0 +1,37 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import os
+import re
+
+import paper_2608_17298_b200.gart as G
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "gart.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gart_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    from paper_2608_17298_b200 import build
+    build.build()
+    L = G.lib()
+    names = _declared()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(G.EXPORTS)
+
+
+def test_host_only_queries():
+    assert G.gart_mask_words(8) == 2 and G.gart_mask_words(16) == 8
+    assert G.lib().gart_status_string(0) == b"ok" and G.lib().gart_status_string(2) == b"workspace too small"
+    a = G.gart_tile_map_workspace_bytes(1000, 640, 480, 8, 10_000)
+    b = G.gart_tile_map_workspace_bytes(1000, 640, 480, 8, 20_000)
+    assert 0 < a < b and a % 256 == 0
+    f1 = G.gart_forward_workspace_bytes(640, 480, 8, 10_000, 100_000)
+    f2 = G.gart_forward_workspace_bytes(640, 480, 8, 10_000, 200_000)
+    assert abs((f2 - f1) - 100_000 * 32) <= 4 * 256    # 32 bytes of scratch per hit of capacity (+- alignment)
+    assert G.gart_view_host_arena_bytes(1000, 3, 640, 480, 8, 10_000, 100_000) > f1
+    assert G.gart_view_host_arena_bytes(1000, 5, 640, 480, 8, 10_000, 100_000) == 0
