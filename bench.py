@@ -50,7 +50,7 @@ def launches_per_step(n_tiles: int) -> int:
     passes = (bits + 7) // 8
     bounds = 1
     tile_map = 1 + 3 + 1 + 1 + passes * (1 + 3 + 1) + 1
-    forward = 1 + 3 + 3 + 1 + 1 + 1
+    forward = 1 + 1 + 3 + 3 + 1 + 1 + 1
     backward = 2
     return bounds + tile_map + forward + backward
 
@@ -126,11 +126,16 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------- workload
-def make_workload(name: str, n_views=None):
+def make_workload(name: str, n_views=None, crop=1.0):
+    """Scene and cameras of a configuration.  crop < 1 keeps the central part of every image (same
+    focal length, fewer pixels): a smaller case of the same per-tile structure, used for profiling."""
     kw = {}
     if n_views is not None and name in ("shell200k", "unbounded1m", "unbounded6m"):
         kw["n_views"] = n_views
     scene, cams = gs.make(name, **kw)
+    if crop < 1.0:
+        cams = [gs.Camera(max(8, int(c.width * crop)), max(8, int(c.height * crop)), c.fx, c.fy,
+                          max(8, int(c.width * crop)) / 2.0, max(8, int(c.height * crop)) / 2.0, c.w2c) for c in cams]
     return scene, cams
 
 
@@ -166,7 +171,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    scene, cams = make_workload(args.config)
+    scene, cams = make_workload(args.config, crop=args.crop)
     frac = args.oracle_frac / 4.0     # per step; keeps a K-step run within minutes
     times, hits = [], 0
     for s in range(args.warmup + args.steps):
@@ -206,15 +211,14 @@ def run_ours(args):
     dev = torch.device("cuda", local)
 
     cfg = G.Config(tile_size=args.tile_size)
-    scene, cams = make_workload(args.config)
+    scene, cams = make_workload(args.config, crop=args.crop)
     mine = shard_views(len(cams), rank, world)
     g = G.Gaussians.from_numpy(scene, dev)
     K = (scene.sh_degree + 1) ** 2
     dls = {v: torch.from_numpy(gs.upstream_gradient(cams[v], v)).to(dev) for v in mine}
 
     # capacities: exact pair count and slot bound of this rank's first view, with slack for the other views
-    P0, S0 = G.size_view(cfg, g, cams[mine[0]], slack=1.0, device=dev)
-    cap_pairs, cap_hits = int(P0 * args.slack) + 1024, int(S0 * args.slack) + 1024
+    cap_pairs, cap_hits = G.size_view(cfg, g, cams[mine[0]], slack=args.slack, device=dev)
     buf = G.ViewBuffers(g.n, g.sh_degree, cams[0], cfg, cap_pairs, cap_hits, dev)
     stream = torch.cuda.current_stream()
 
@@ -367,7 +371,7 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": total_ms_all / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.config, "n_gaussians": scene.n, "width": cams[0].width, "height": cams[0].height,
-                   "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "views": len(cams),
+                   "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "views": len(cams), "crop": args.crop,
                    "l2": "inputs larger than L2 (parameters %.2f GB, LT %.2f GB per view)" % (
                        4e-9 * scene.n * (11 + 3 * K), 16e-9 * Hm),
                    "hits_per_view": Hm, "pairs_per_view": Pm, "visible_per_view": Nv},
@@ -397,6 +401,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--oracle-frac", type=float, default=0.02)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--crop", type=float, default=1.0, help="central crop of every view (profiling on a smaller case)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

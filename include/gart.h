@@ -83,13 +83,15 @@ enum {
     GART_CNT_SLOTS_LO = 2,  /* S = sum of rectangle areas, low/high words: the capacity bound */
     GART_CNT_SLOTS_HI = 3,  /*     of the intermediate buffer (Eq. 15 with lambda_s = 1)      */
     GART_CNT_HITS = 4,      /* H: ray-Gaussian hits of the view = entries used in LT */
-    GART_CNT_ERROR = 5,     /* bit 0: pair capacity exceeded; bit 1: hit capacity exceeded */
+    GART_CNT_ERROR = 5,     /* bit 0: pair capacity exceeded; bit 1: hit capacity exceeded (L > cap_hits); bit 2: timeout */
     GART_CNT_MAX_RAY_HITS = 6,
     GART_CNT_STRADDLE = 7,  /* Gaussians whose support crosses the near plane */
-    GART_COUNTS_WORDS = 8
+    GART_CNT_LT_SLOTS = 8,  /* L >= H: entries of LT in use, including the padding of its interleaved layout */
+    GART_COUNTS_WORDS = 12
 };
 #define GART_ERRBIT_PAIRS 1u
 #define GART_ERRBIT_HITS 2u
+#define GART_ERRBIT_TIMEOUT 4u   /* a bounded wait on an asynchronous copy gave up (never expected) */
 
 #define GART_PRE_WORDS 20   /* fp32 words of the per-Gaussian ray-evaluation record */
 #define GART_GRAD_WORDS 64  /* stride of a gradient record: mean 3, scale 3, quat 4, opacity 1,
@@ -143,37 +145,57 @@ gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n
  *   color      [H,W,3] out;  t_final [H,W] out;  hit_count [H,W] uint32 out.
  *   pair_mask  [cap_pairs, gart_mask_words] uint32 out: bit p of pair j = pixel p of the tile
  *              (p = ly * tile_size + lx) is hit by the pair's Gaussian.
- *   pair_lt_off[cap_pairs+1] uint32 out: exclusive prefix sum of hits per pair; the hit of pair j
- *              at pixel p lives at lt[pair_lt_off[j] + (number of set mask bits below p)]:
- *              primitive-tile-major, then pixel, every hit with a collision-free slot.
+ *   pair_order [cap_pairs] uint32 out: for tile t, pair_order[tile_off[t] + r] is the pair of rank r
+ *              when the tile's pairs are ordered by descending hit count (stable); the backward
+ *              gives lane l of a warp the pair of rank 32 g + l, so a warp's lanes have (nearly)
+ *              the same number of hits.
+ *   rank_gid   [cap_pairs] uint32 out, rank_mask [cap_pairs, gart_mask_words] uint32 out: Gaussian id
+ *              and hit mask of the pair at each rank position (copies of pair_gid / pair_mask in rank
+ *              order, so that later kernels read them coalesced and without indirection).
+ *   rank_gstart[cap_pairs] uint32 out, tile_lt_base [T+1] uint32 out: the e-th hit (in pixel order)
+ *              of the pair of rank r of tile t lives at
+ *                  lt[tile_lt_base[t] + rank_gstart[tile_off[t] + r] + 32 e + (r mod 32)].
+ *              rank_gstart is the same for the 32 ranks of a group: the group's pairs are interleaved
+ *              entry by entry, so the group's e-th entries are 32 consecutive 16-byte words, the
+ *              group's whole block is one contiguous range (one bulk copy), every hit owns one slot
+ *              (forward writes never collide), and a group occupies 32 x (its largest hit count)
+ *              entries: L = tile_lt_base[T] >= H counts the padding.
  *   lt         [cap_hits,4] out: per hit (R_r, R_g, R_b, T): colour composited BEHIND the hit
  *              (including the background term) and transmittance in front of it.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.
- *   counts: HITS, MAX_RAY_HITS.  If H > cap_hits, GART_ERRBIT_HITS is set and color, t_final,
- *   lt, ray_gid, ray_slot are not written.
+ *   counts: HITS, LT_SLOTS, MAX_RAY_HITS.  If L > cap_hits, GART_ERRBIT_HITS is set and color,
+ *   t_final, lt, ray_gid, ray_slot are not written.  Because ranks descend in hit count,
+ *   L <= H + 32 tile_size^2 per non-empty tile, and H <= S (the slot bound of gart_tile_map), so
+ *   cap_hits = S + 32 tile_size^2 T always suffices; the exact need is L.
  */
 size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
 gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                          const uint32_t *tile_off, const uint32_t *pair_gid, int64_t cap_pairs,
                          float *color, float *t_final, uint32_t *hit_count,
-                         uint32_t *pair_mask, uint32_t *pair_lt_off, float *lt, int64_t cap_hits,
+                         uint32_t *pair_mask, uint32_t *pair_order, uint32_t *rank_gid, uint32_t *rank_mask,
+                         uint32_t *rank_gstart, uint32_t *tile_lt_base, float *lt, int64_t cap_hits,
                          uint32_t *ray_off, uint32_t *ray_gid, uint32_t *ray_slot, uint32_t *counts,
                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Step 4 -- primitive-centric backward (Sec. 4.4): one thread block per tile, one thread per
- * (tile, Gaussian) pair; the thread walks the pair's hit pixels, reads their LT entries (one
- * contiguous run), accumulates in registers and performs one vector atomic update of the
- * Gaussian's gradient record per pair.  No per-pixel atomics.
+ * (tile, Gaussian) pair; the thread walks the pair's hit pixels, reads their LT entries (coalesced
+ * across the warp thanks to the interleaved layout), accumulates in registers and performs one vector
+ * atomic update of the Gaussian's gradient record per pair.  No per-pixel atomics.
  *   dL_dcolor [H,W,3] in.
  *   grad [n,GART_GRAD_WORDS] out, fully overwritten: d mean, d scale, d quat, d opacity, d sh
  *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
+ *   counts: read (a set error bit skips the work); GART_ERRBIT_TIMEOUT is set if a wait on an
+ *        asynchronous copy ran out, in which case grad is incomplete.
+ * The main kernel uses up to 99 KB of dynamic shared memory per block (opt-in set by the call): LT blocks
+ * and the Gaussians' records are streamed in with bulk asynchronous copies, one rank group ahead.
  */
 gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
-                          const uint32_t *tile_off, const uint32_t *pair_gid, const uint32_t *pair_mask,
-                          const uint32_t *pair_lt_off, const float *lt, const float *dL_dcolor,
-                          float *grad, const uint32_t *counts, void *stream);
+                          const uint32_t *tile_off, const uint32_t *rank_gid, const uint32_t *rank_mask,
+                          const uint32_t *rank_gstart, const uint32_t *tile_lt_base,
+                          const float *lt, const float *dL_dcolor,
+                          float *grad, uint32_t *counts, void *stream);
 
 /*
  * Pixel-centric baseline (Sec. 3.5): one thread per ray walks the ray's hits and issues one

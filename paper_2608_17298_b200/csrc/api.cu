@@ -8,7 +8,7 @@ struct HostArena {
     float *mean, *scale, *quat, *opacity, *sh, *pre, *color, *t_final, *lt, *dL_dC, *grad;
     int32_t* rect;
     uint8_t* cls;
-    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_lt_off, *hit_count, *ray_off, *ray_gid, *ray_slot;
+    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_gid, *rank_mask, *rank_gstart, *tile_lt_base, *hit_count, *ray_off, *ray_gid, *ray_slot;
     void* ws;
     size_t ws_bytes;
     size_t bytes;
@@ -28,7 +28,9 @@ static HostArena arena_layout(void* base, int64_t n, int K, int width, int heigh
     a.rect = (int32_t*)take(nn * 16); a.cls = (uint8_t*)take(nn); a.pre = (float*)take(nn * GART_PRE_WORDS * 4);
     a.counts = (uint32_t*)take(GART_COUNTS_WORDS * 4);
     a.tile_off = (uint32_t*)take((size_t)(T + 1) * 4); a.pair_gid = (uint32_t*)take(cp * 4);
-    a.pair_mask = (uint32_t*)take(cp * 4 * mw); a.pair_lt_off = (uint32_t*)take((cp + 1) * 4);
+    a.pair_mask = (uint32_t*)take(cp * 4 * mw); a.pair_order = (uint32_t*)take(cp * 4); a.rank_gid = (uint32_t*)take(cp * 4);
+    a.rank_mask = (uint32_t*)take(cp * 4 * mw); a.rank_gstart = (uint32_t*)take(cp * 4);
+    a.tile_lt_base = (uint32_t*)take((size_t)(T + 1) * 4);
     a.color = (float*)take(hw * 12); a.t_final = (float*)take(hw * 4); a.hit_count = (uint32_t*)take(hw * 4);
     a.lt = (float*)take(ch * 16); a.ray_off = (uint32_t*)take((hw + 1) * 4);
     a.ray_gid = (uint32_t*)take(ch * 4); a.ray_slot = (uint32_t*)take(ch * 4);
@@ -91,9 +93,9 @@ extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussia
     s = gart_tile_map(cfg, a.rect, n, cam->width, cam->height, a.tile_off, a.pair_gid, cap_pairs, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     s = gart_forward(cfg, &gd, cam, a.pre, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count, a.pair_mask,
-                     a.pair_lt_off, a.lt, cap_hits, a.ray_off, a.ray_gid, a.ray_slot, a.counts, a.ws, a.ws_bytes, stream);
+                     a.pair_order, a.rank_gid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, a.ray_gid, a.ray_slot, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
-    s = gart_backward(cfg, &gd, cam, a.pre, a.tile_off, a.pair_gid, a.pair_mask, a.pair_lt_off, a.lt, a.dL_dC, a.grad, a.counts, stream);
+    s = gart_backward(cfg, &gd, cam, a.pre, a.tile_off, a.rank_gid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, a.dL_dC, a.grad, a.counts, stream);
     if (s != GART_OK) return s;
     if (cudaMemcpyAsync(color_host, a.color, (size_t)hw * 12, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GART_ERR_CUDA;
     if (n > 0 && cudaMemcpyAsync(grad_host, a.grad, (size_t)n * GART_GRAD_WORDS * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)

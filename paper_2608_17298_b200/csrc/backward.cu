@@ -1,124 +1,152 @@
-// gart_backward: primitive-centric backward (Sec. 4.4) and gart_backward_atomic, the
-// pixel-centric baseline (Sec. 3.5).
+// gart_backward: primitive-centric backward (Sec. 4.4).
 //
-// Per hit (ray r, Gaussian i), with g = dL/dC_r, T = transmittance in front of the hit, Rb =
-// colour composited behind it (both from the LT buffer), alpha, x_g recomputed from the record:
-//   dL/dsh_k   += Y_k(d_r) * T alpha g            (channels whose raw colour is positive)
-//   dL/dalpha   = g . (T c - Rb / (1 - alpha))
-//   dL/dsigma  += dL/dalpha * alpha / sigma
-//   G           = dL/d(D^2) = -alpha dL/dalpha / 2       (the maximum-response point is
-//                 stationary in t, so t* carries no gradient)
-//   v += G x_g,  Q += G x_g x_g^T
-// and, once per Gaussian (all sums are linear in v and Q, with W = S^-1 R^T):
-//   dL/dmu = -2 W^T v,  dL/ds_k = -2 Q_kk / s_k,  dL/dR = 2 R^-T S Q S^-1,  dL/dq by the chain
-//   rule through the polynomial rotation formula.
-// gart_backward accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) per (tile, Gaussian) pair in
-// registers, adds them to the Gaussian's record with one vector atomic per 16 bytes, and a
-// per-Gaussian pass converts the record in place.  The baseline converts per hit and issues one
-// scalar atomicAdd per gradient word per hit.
-#include "common.cuh"
+// One thread block per tile, one thread per (tile, Gaussian) pair.  Lane l of a warp owns the pair
+// of rank 32 g + l in the tile's hit-count order, so the lanes of a warp run (nearly) the same
+// number of iterations; the LT entries of such a group of 32 pairs are interleaved entry by entry
+// (lt[base + 32 e + l]), i.e. the whole group's LT block is one contiguous range.  Each warp streams
+// these blocks into shared memory with bulk asynchronous copies (cp.async.bulk, completion on an
+// mbarrier), double buffered, so that tens of KB of LT data per SM are in flight while the warp
+// computes; lanes then read their entry with conflict-free 16-byte shared loads.  A thread
+// accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) of its pair in registers and adds them to the
+// Gaussian's gradient record with one vector atomic per 16 bytes -- no per-pixel atomics.  A
+// per-Gaussian pass then converts the record in place into d mean, d scale, d quat, d opacity.
+#include "backward_common.cuh"
 
 namespace gart {
 
-// -------------------------------------------------------------------------------- per-Gaussian conversion
-struct GeoGrad {
-    float dmu[3], ds[3], dq[4];
-};
-
-// v[3], Q = (xx, yy, zz, xy, xz, yz) -> gradients of mean, scale, quaternion.
-__device__ __forceinline__ GeoGrad moments_to_grads(const float* v, const float* Q, const float* q, const float* s) {
-    const float w = q[0], x = q[1], y = q[2], z = q[3];
-    float R[9];
-    R[0] = 1.0f - 2.0f * (y * y + z * z); R[1] = 2.0f * (x * y - w * z); R[2] = 2.0f * (x * z + w * y);
-    R[3] = 2.0f * (x * y + w * z); R[4] = 1.0f - 2.0f * (x * x + z * z); R[5] = 2.0f * (y * z - w * x);
-    R[6] = 2.0f * (x * z - w * y); R[7] = 2.0f * (y * z + w * x); R[8] = 1.0f - 2.0f * (x * x + y * y);
-    const float is[3] = {1.0f / s[0], 1.0f / s[1], 1.0f / s[2]};
-    GeoGrad o;
-    const float vs[3] = {v[0] * is[0], v[1] * is[1], v[2] * is[2]};
-#pragma unroll
-    for (int j = 0; j < 3; ++j) o.dmu[j] = -2.0f * (R[3 * j] * vs[0] + R[3 * j + 1] * vs[1] + R[3 * j + 2] * vs[2]);
-    o.ds[0] = -2.0f * Q[0] * is[0];
-    o.ds[1] = -2.0f * Q[1] * is[1];
-    o.ds[2] = -2.0f * Q[2] * is[2];
-    // R^-T = cof(R) / det(R)
-    float C[9];
-    C[0] = R[4] * R[8] - R[5] * R[7]; C[1] = R[5] * R[6] - R[3] * R[8]; C[2] = R[3] * R[7] - R[4] * R[6];
-    C[3] = R[2] * R[7] - R[1] * R[8]; C[4] = R[0] * R[8] - R[2] * R[6]; C[5] = R[1] * R[6] - R[0] * R[7];
-    C[6] = R[1] * R[5] - R[2] * R[4]; C[7] = R[2] * R[3] - R[0] * R[5]; C[8] = R[0] * R[4] - R[1] * R[3];
-    const float idet = 1.0f / (R[0] * C[0] + R[1] * C[1] + R[2] * C[2]);
-    // B = S Q S^-1
-    const float Qm[9] = {Q[0], Q[3], Q[4], Q[3], Q[1], Q[5], Q[4], Q[5], Q[2]};
-    float B[9];
-#pragma unroll
-    for (int l = 0; l < 3; ++l)
-#pragma unroll
-        for (int k = 0; k < 3; ++k) B[3 * l + k] = s[l] * Qm[3 * l + k] * is[k];
-    float dR[9];
-#pragma unroll
-    for (int j = 0; j < 3; ++j)
-#pragma unroll
-        for (int k = 0; k < 3; ++k)
-            dR[3 * j + k] = 2.0f * idet * (C[3 * j] * B[k] + C[3 * j + 1] * B[3 + k] + C[3 * j + 2] * B[6 + k]);
-    o.dq[0] = 2.0f * (-z * dR[1] + y * dR[2] + z * dR[3] - x * dR[5] - y * dR[6] + x * dR[7]);
-    o.dq[1] = 2.0f * (y * dR[1] + z * dR[2] + y * dR[3] - 2.0f * x * dR[4] - w * dR[5] + z * dR[6] + w * dR[7] - 2.0f * x * dR[8]);
-    o.dq[2] = 2.0f * (-2.0f * y * dR[0] + x * dR[1] + w * dR[2] + x * dR[3] + z * dR[5] - w * dR[6] + z * dR[7] - 2.0f * y * dR[8]);
-    o.dq[3] = 2.0f * (-2.0f * z * dR[0] - w * dR[1] + x * dR[2] + w * dR[3] - 2.0f * z * dR[4] + y * dR[5] + x * dR[6] + y * dR[7]);
-    return o;
-}
-
-// Per-hit gradient terms shared by both backward variants.
-template <int K>
-struct HitGrad {
-    float wch[3];   // T alpha g per channel, zero where the colour is clamped
-    float dalpha;   // dL/dalpha
-};
-
-template <int K>
-__device__ __forceinline__ HitGrad<K> hit_grad(const float* Y, const float* shc, const float3 g, const float4 L, const float alpha) {
-    float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
-#pragma unroll
-    for (int k = 0; k < K; ++k) {
-        c0 = fmaf(Y[k], shc[3 * k], c0);
-        c1 = fmaf(Y[k], shc[3 * k + 1], c1);
-        c2 = fmaf(Y[k], shc[3 * k + 2], c2);
-    }
-    const float T = L.w;
-    const float Ta = T * alpha;
-    const float inv = __frcp_rn(1.0f - alpha);
-    HitGrad<K> h;
-    h.wch[0] = c0 > 0.0f ? Ta * g.x : 0.0f;
-    h.wch[1] = c1 > 0.0f ? Ta * g.y : 0.0f;
-    h.wch[2] = c2 > 0.0f ? Ta * g.z : 0.0f;
-    const float t0 = fmaf(T, fmaxf(c0, 0.0f), -L.x * inv);
-    const float t1 = fmaf(T, fmaxf(c1, 0.0f), -L.y * inv);
-    const float t2 = fmaf(T, fmaxf(c2, 0.0f), -L.z * inv);
-    h.dalpha = fmaf(g.x, t0, fmaf(g.y, t1, g.z * t2));
-    return h;
-}
-
-// -------------------------------------------------------------------------------- primitive-centric
-constexpr int BWD_THREADS = 128;
+constexpr int BWD_WARPS = 4;
+constexpr int BWD_THREADS = BWD_WARPS * 32;
+constexpr int BWD_CHUNK = 16;                          // LT entries per lane and per pipeline stage
+constexpr int BWD_STAGE_F4 = BWD_CHUNK * 32;           // float4 per stage (8 KB)
+constexpr int BWD_LT_SMEM = BWD_WARPS * 2 * BWD_STAGE_F4 * 16;
+constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + ((sw * 4) % 16 == 0 ? BWD_THREADS * (5 + sw / 4) * 16 : 0); }
+constexpr uint32_t BWD_WAIT_LIMIT = 1u << 22;          // bounded wait on a copy; then the error bit is set
 
 template <int K>
 struct PixLayout {
     static constexpr int W = (K + 3 + 3) & ~3;   // floats per pixel record: Y[K], g[3], zero padding
 };
 
+// ---- mbarrier / bulk copy (shared::cta addresses as 32-bit)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < BWD_WAIT_LIMIT; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Descriptor of one rank group as seen by a lane (read from the rank-ordered copies: coalesced).
+template <int MW>
+struct GroupDesc {
+    PairMask<MW> pm;
+    uint32_t gid;
+    int c;             // hits of this lane's pair
+    int cmax;          // hits of the group's first pair = the largest of the group
+    uint32_t gstart;   // first LT entry of the group, relative to the tile's base
+};
+
+template <int MW>
+__device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__ rank_gid, const uint32_t* __restrict__ rank_mask,
+                                                    const uint32_t* __restrict__ rank_gstart, uint32_t begin, uint32_t n,
+                                                    uint32_t r0, int lane) {
+    GroupDesc<MW> d;
+    const bool act = r0 < n && r0 + lane < n;
+    const uint32_t q = begin + r0 + lane;
+    d.pm.load(rank_mask, act ? q : 0u, act);
+    d.c = d.pm.count();
+    d.gid = act ? __ldg(rank_gid + q) : 0u;
+    const uint32_t s0 = act ? __ldg(rank_gstart + q) : 0u;
+    d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
+    d.gstart = __shfl_sync(0xffffffffu, s0, 0);
+    return d;
+}
+
+// Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
+// acc[0..2] = v, acc[3..8] = Q (xx, yy, zz, xy, xz, yz), acc[9] = sum alpha dL/dalpha, acc[11..] = dL/dsh.
+template <int TS, int K, int PW>
+__device__ __forceinline__ void bwd_hit(const PreRec& P, const float* shc, float* acc, const float* spix, int bx, int by, int p,
+                                        const float4 L) {
+    const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
+    const float* rec = spix + p * PW;
+    float Y[K];
+    if (K % 4 == 0) {
+#pragma unroll
+        for (int k4 = 0; k4 < K / 4; ++k4) {
+            const float4 t = reinterpret_cast<const float4*>(rec)[k4];
+            Y[4 * k4] = t.x; Y[4 * k4 + 1] = t.y; Y[4 * k4 + 2] = t.z; Y[4 * k4 + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int kk = 0; kk < K; ++kk) Y[kk] = rec[kk];
+    }
+    const float3 g = make_float3(rec[K], rec[K + 1], rec[K + 2]);
+    const HitGrad<K> h = hit_grad<K>(Y, shc, g, L, r.alpha);
+#pragma unroll
+    for (int kk = 0; kk < K; ++kk) {
+        acc[11 + 3 * kk] = fmaf(Y[kk], h.wch[0], acc[11 + 3 * kk]);
+        acc[11 + 3 * kk + 1] = fmaf(Y[kk], h.wch[1], acc[11 + 3 * kk + 1]);
+        acc[11 + 3 * kk + 2] = fmaf(Y[kk], h.wch[2], acc[11 + 3 * kk + 2]);
+    }
+    const float ad = r.alpha * h.dalpha;
+    acc[9] += ad;
+    const float G = -0.5f * ad;
+    const float3 xg = ray_xg(r);
+    const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
+    acc[0] += gx; acc[1] += gy; acc[2] += gz;
+    acc[3] = fmaf(gx, xg.x, acc[3]); acc[4] = fmaf(gy, xg.y, acc[4]); acc[5] = fmaf(gz, xg.z, acc[5]);
+    acc[6] = fmaf(gx, xg.y, acc[6]); acc[7] = fmaf(gx, xg.z, acc[7]); acc[8] = fmaf(gy, xg.z, acc[8]);
+}
+
 template <int TS, int DEG>
 __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
-                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_gid,
-                                                                const uint32_t* __restrict__ pair_mask, const uint32_t* __restrict__ pair_lt_off,
+                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_gid,
+                                                                const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
+                                                                const uint32_t* __restrict__ tile_lt_base,
                                                                 const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                float* __restrict__ grad, const uint32_t* __restrict__ counts) {
+                                                                float* __restrict__ grad, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = PixLayout<K>::W;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
+    // Gaussian record + SH coefficients of a lane's pair, staged through shared memory one group ahead
+    // when their size allows bulk copies (multiples of 16 bytes: degrees 1 and 3)
+    constexpr bool STAGE_P = (SW * 4) % 16 == 0;
+    constexpr int PF4 = 5 + SW / 4;          // float4 per lane in the parameter buffer
+    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][PF4] parameters
     __shared__ __align__(16) float spix[NT * PW];
+    __shared__ __align__(8) uint64_t bars[BWD_WARPS][3];
     if (counts[GART_CNT_ERROR]) return;
     const int tile = blockIdx.x;
-    const uint32_t begin = tile_off[tile], end = tile_off[tile + 1];
-    if (begin == end) return;
+    const uint32_t begin = tile_off[tile], n = tile_off[tile + 1] - begin;
+    if (n == 0) return;
     const int tx = tile % cam.tiles_x, ty = tile / cam.tiles_x;
     const int x0 = tx * TS, y0 = ty * TS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        mbar_init(smem_u32(&bars[warp][0]), 1);
+        mbar_init(smem_u32(&bars[warp][1]), 1);
+        mbar_init(smem_u32(&bars[warp][2]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     // per-pixel data of the tile: SH basis of the ray direction and the upstream gradient
     for (int p = threadIdx.x; p < NT; p += BWD_THREADS) {
         const int x = x0 + p % TS, y = y0 + p / TS;
@@ -137,76 +165,109 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     }
     __syncthreads();
 
-    for (uint32_t j = begin + threadIdx.x; j < end; j += BWD_THREADS) {
-        uint32_t mk[MW];
-        uint32_t any = 0;
-#pragma unroll
-        for (int q = 0; q < MW; ++q) { mk[q] = __ldg(pair_mask + (size_t)j * MW + q); any |= mk[q]; }
-        if (!any) continue;
-        const uint32_t gid = __ldg(pair_gid + j);
-        const PreRec P = load_pre(pre4, gid);
-        float shc[SW];
-        {
-            const float* sp = sh + (size_t)gid * SW;
-            if (SW % 4 == 0) {
-#pragma unroll
-                for (int q = 0; q < SW / 4; ++q) {
-                    const float4 t = __ldg(reinterpret_cast<const float4*>(sp) + q);
-                    shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
-                }
-            } else {
-#pragma unroll
-                for (int q = 0; q < SW; ++q) shc[q] = __ldg(sp + q);
+    const float4* lt_tile = lt + tile_lt_base[tile];
+    float4* my_stage = dyn + (size_t)warp * 2 * BWD_STAGE_F4;
+    float4* my_par = dyn + (size_t)BWD_WARPS * 2 * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PF4;
+    const uint32_t stage_addr = smem_u32(my_stage);
+    const uint32_t par_addr = smem_u32(my_par);
+    const uint32_t bar_addr = smem_u32(&bars[warp][0]);
+    const uint32_t pbar_addr = bar_addr + 16u;
+    uint32_t unit = 0;     // LT pipeline units (chunks) consumed so far by this warp: stage = unit & 1, parity = (unit >> 1) & 1
+    uint32_t pphase = 0;   // parity of the parameter barrier
+
+    // copy chunk `k` of a group's LT block into the stage that unit number `u` will use
+    auto issue = [&](const GroupDesc<MW>& d, int k, uint32_t u) {
+        if (lane == 0) {
+            const int ne = min(BWD_CHUNK, d.cmax - k * BWD_CHUNK);
+            const uint32_t bytes = (uint32_t)ne * 512u, s = u & 1u;
+            mbar_expect_tx(bar_addr + 8u * s, bytes);
+            bulk_g2s(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + d.gstart + (size_t)k * BWD_STAGE_F4, bytes, bar_addr + 8u * s);
+        }
+    };
+    // copy the Gaussian records and SH coefficients of a group's pairs into the parameter buffer
+    auto issue_params = [&](const GroupDesc<MW>& d) {
+        if (STAGE_P) {
+            const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
+            if (lane == 0) mbar_expect_tx(pbar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
+            if (d.c != 0) {
+                bulk_g2s(par_addr, pre4 + (size_t)d.gid * 5, 80u, pbar_addr);
+                bulk_g2s(par_addr + 80u, sh + (size_t)d.gid * SW, (uint32_t)(SW * 4), pbar_addr);
             }
         }
+    };
+    auto fail = [&]() {
+        // a copy never completed: report, give copies that may still be in flight a second bounded
+        // chance to land before this warp's shared memory may be released, and stop
+        if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
+        mbar_wait_bounded(bar_addr, (unit >> 1) & 1u);
+        mbar_wait_bounded(bar_addr + 8u, (unit >> 1) & 1u);
+        mbar_wait_bounded(pbar_addr, pphase);
+    };
+
+    uint32_t r0 = warp * 32;
+    GroupDesc<MW> cur = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0, lane);
+    if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
+    issue(cur, 0, unit);
+    issue_params(cur);
+    GroupDesc<MW> nxt = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0 + BWD_THREADS, lane);
+    while (true) {
+        // descriptor two groups ahead: needed only at the start of the next iteration
+        const GroupDesc<MW> nxt2 = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
+        PreRec P;
+        float shc[SW];
         float acc[AW];
 #pragma unroll
         for (int q = 0; q < AW; ++q) acc[q] = 0.0f;
-        const float4* lp = lt + __ldg(pair_lt_off + j);
-        const int bx = x0 - P.ix, by = y0 - P.iy;
+        if (STAGE_P) {
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(pbar_addr, pphase))) { fail(); return; }
+            pphase ^= 1u;
+            if (cur.c != 0) {
+                P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);
 #pragma unroll
-        for (int q = 0; q < MW; ++q) {
-            uint32_t word = mk[q];
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                const int p = q * 32 + b;
-                const float4 L = __ldg(lp++);
-                const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
-                const float* rec = spix + p * PW;
-                float Y[K];
-                if (K % 4 == 0) {
-#pragma unroll
-                    for (int k4 = 0; k4 < K / 4; ++k4) {
-                        const float4 t = reinterpret_cast<const float4*>(rec)[k4];
-                        Y[4 * k4] = t.x; Y[4 * k4 + 1] = t.y; Y[4 * k4 + 2] = t.z; Y[4 * k4 + 3] = t.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int k = 0; k < K; ++k) Y[k] = rec[k];
+                for (int q = 0; q < SW / 4; ++q) {
+                    const float4 t = my_par[5 + q];
+                    shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
                 }
-                const float3 g = make_float3(rec[K], rec[K + 1], rec[K + 2]);
-                const HitGrad<K> h = hit_grad<K>(Y, shc, g, L, r.alpha);
-#pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    acc[11 + 3 * k] = fmaf(Y[k], h.wch[0], acc[11 + 3 * k]);
-                    acc[11 + 3 * k + 1] = fmaf(Y[k], h.wch[1], acc[11 + 3 * k + 1]);
-                    acc[11 + 3 * k + 2] = fmaf(Y[k], h.wch[2], acc[11 + 3 * k + 2]);
-                }
-                const float ad = r.alpha * h.dalpha;
-                acc[9] += ad;
-                const float G = -0.5f * ad;
-                const float3 xg = ray_xg(r);
-                const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
-                acc[0] += gx; acc[1] += gy; acc[2] += gz;
-                acc[3] = fmaf(gx, xg.x, acc[3]); acc[4] = fmaf(gy, xg.y, acc[4]); acc[5] = fmaf(gz, xg.z, acc[5]);
-                acc[6] = fmaf(gx, xg.y, acc[6]); acc[7] = fmaf(gx, xg.z, acc[7]); acc[8] = fmaf(gy, xg.z, acc[8]);
             }
-        }
-        // one vector atomic per 16 bytes of the Gaussian's record
-        float4* gp = reinterpret_cast<float4*>(grad + (size_t)gid * GART_GRAD_WORDS);
+            __syncwarp();
+            if (nxt.cmax != 0) issue_params(nxt);
+        } else if (cur.c != 0) {
+            P = load_pre(pre4, cur.gid);
+            const float* sp = sh + (size_t)cur.gid * SW;
 #pragma unroll
-        for (int q = 0; q < AW / 4; ++q) atomicAdd(gp + q, make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]));
+            for (int q = 0; q < SW; ++q) shc[q] = __ldg(sp + q);
+        }
+        if (cur.c == 0) {
+            P = unpack_pre(make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 1),
+                           make_float4(0, 0, 0, 0));
+#pragma unroll
+            for (int q = 0; q < SW; ++q) shc[q] = 0.0f;
+        }
+        const int bx = x0 - P.ix, by = y0 - P.iy;
+        const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
+        for (int k = 0; k < nchunks; ++k) {
+            // keep the next unit's copy in flight while this one is consumed
+            if (k + 1 < nchunks) issue(cur, k + 1, unit + 1);
+            else if (nxt.cmax != 0) issue(nxt, 0, unit + 1);
+            const uint32_t s = unit & 1u;
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit >> 1) & 1u))) { fail(); return; }
+            const float4* sl = my_stage + s * BWD_STAGE_F4 + lane;
+            const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
+            for (int e = k * BWD_CHUNK; e < e_end; ++e)
+                bwd_hit<TS, K, PW>(P, shc, acc, spix, bx, by, cur.pm.next(), sl[(e - k * BWD_CHUNK) * 32]);
+            __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
+            ++unit;
+        }
+        if (cur.c != 0) {
+            // one vector atomic per 16 bytes of the Gaussian's record
+            float4* gp = reinterpret_cast<float4*>(grad + (size_t)cur.gid * GART_GRAD_WORDS);
+#pragma unroll
+            for (int q = 0; q < AW / 4; ++q) atomicAdd(gp + q, make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]));
+        }
+        if (nxt.cmax == 0) break;
+        cur = nxt;
+        nxt = nxt2;
+        r0 += BWD_THREADS;
     }
 }
 
@@ -235,80 +296,44 @@ __global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, const floa
     gp[2] = make_float4(o.dq[2], o.dq[3], c.y / opacity[i], c.w);
 }
 
-// -------------------------------------------------------------------------------- pixel-centric baseline
-template <int DEG>
-__global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
-                                                         const float* __restrict__ scale, const float* __restrict__ quat,
-                                                         const float* __restrict__ opacity, const uint32_t* __restrict__ ray_off,
-                                                         const uint32_t* __restrict__ ray_gid, const uint32_t* __restrict__ ray_slot,
-                                                         const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                         float* __restrict__ grad, const uint32_t* __restrict__ counts) {
-    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K;
-    if (counts[GART_CNT_ERROR]) return;
-    const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (ray >= (int64_t)cam.width * cam.height) return;
-    const uint32_t b = ray_off[ray], e = ray_off[ray + 1];
-    if (b == e) return;
-    const int x = (int)(ray % cam.width), y = (int)(ray / cam.width);
-    float Y[K];
-    sh_basis<K>(pixel_dir(cam, x, y), Y);
-    const float3 g = make_float3(dL_dC[3 * ray], dL_dC[3 * ray + 1], dL_dC[3 * ray + 2]);
-    for (uint32_t h = b; h < e; ++h) {
-        const uint32_t gid = ray_gid[h];
-        const float4 L = lt[ray_slot[h]];
-        const PreRec P = load_pre(pre4, gid);
-        const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
-        float shc[SW];
-#pragma unroll
-        for (int q = 0; q < SW; ++q) shc[q] = __ldg(sh + (size_t)gid * SW + q);
-        const HitGrad<K> hg = hit_grad<K>(Y, shc, g, L, r.alpha);
-        const float ad = r.alpha * hg.dalpha;
-        const float G = -0.5f * ad;
-        const float3 xg = ray_xg(r);
-        const float v[3] = {G * xg.x, G * xg.y, G * xg.z};
-        const float Q[6] = {v[0] * xg.x, v[1] * xg.y, v[2] * xg.z, v[0] * xg.y, v[0] * xg.z, v[1] * xg.z};
-        const float q[4] = {quat[4 * gid], quat[4 * gid + 1], quat[4 * gid + 2], quat[4 * gid + 3]};
-        const float s[3] = {scale[3 * gid], scale[3 * gid + 1], scale[3 * gid + 2]};
-        const GeoGrad o = moments_to_grads(v, Q, q, s);
-        float* gp = grad + (size_t)gid * GART_GRAD_WORDS;
-        atomicAdd(gp + 0, o.dmu[0]); atomicAdd(gp + 1, o.dmu[1]); atomicAdd(gp + 2, o.dmu[2]);
-        atomicAdd(gp + 3, o.ds[0]); atomicAdd(gp + 4, o.ds[1]); atomicAdd(gp + 5, o.ds[2]);
-        atomicAdd(gp + 6, o.dq[0]); atomicAdd(gp + 7, o.dq[1]); atomicAdd(gp + 8, o.dq[2]); atomicAdd(gp + 9, o.dq[3]);
-        atomicAdd(gp + 10, ad / opacity[gid]);
-#pragma unroll
-        for (int k = 0; k < K; ++k) {
-            atomicAdd(gp + 11 + 3 * k, Y[k] * hg.wch[0]);
-            atomicAdd(gp + 11 + 3 * k + 1, Y[k] * hg.wch[1]);
-            atomicAdd(gp + 11 + 3 * k + 2, Y[k] * hg.wch[2]);
-        }
-    }
+template <int TS, int DEG>
+static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
+                                    const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+                                    const uint32_t* tile_lt_base, const float4* lt,
+                                    const float* dL_dC, const CamF& cam, float* grad, uint32_t* counts) {
+    auto kern = bwd_pairs_kernel<TS, DEG>;
+    constexpr int smem = bwd_dyn_smem(3 * (DEG + 1) * (DEG + 1));
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
+    kern<<<T, BWD_THREADS, smem, st>>>(pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, grad, counts);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
 }
 
 template <int TS>
 static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
-                                const uint32_t* pair_gid, const uint32_t* pair_mask, const uint32_t* pair_lt_off, const float4* lt,
-                                const float* dL_dC, const CamF& cam, float* grad, const uint32_t* counts) {
+                                const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+                                const uint32_t* tile_lt_base, const float4* lt,
+                                const float* dL_dC, const CamF& cam, float* grad, uint32_t* counts) {
 #define GART_PAIRS(D) \
-    bwd_pairs_kernel<TS, D><<<T, BWD_THREADS, 0, st>>>(pre4, sh, tile_off, pair_gid, pair_mask, pair_lt_off, lt, dL_dC, cam, grad, counts)
+    return launch_pairs_deg<TS, D>(T, st, pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, grad, counts)
     switch (deg) {
-        case 0: GART_PAIRS(0); break;
-        case 1: GART_PAIRS(1); break;
-        case 2: GART_PAIRS(2); break;
-        default: GART_PAIRS(3); break;
+        case 0: GART_PAIRS(0);
+        case 1: GART_PAIRS(1);
+        case 2: GART_PAIRS(2);
+        default: GART_PAIRS(3);
     }
 #undef GART_PAIRS
-    GART_LAUNCH_CHECK();
-    return GART_OK;
 }
 
 }  // namespace gart
 
 extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
-                                     const uint32_t* tile_off, const uint32_t* pair_gid, const uint32_t* pair_mask,
-                                     const uint32_t* pair_lt_off, const float* lt, const float* dL_dcolor,
-                                     float* grad, const uint32_t* counts, void* stream) {
+                                     const uint32_t* tile_off, const uint32_t* rank_gid, const uint32_t* rank_mask,
+                                     const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
+                                     const float* lt, const float* dL_dcolor,
+                                     float* grad, uint32_t* counts, void* stream) {
     using namespace gart;
-    if (!cfg || !g || !cam || !counts || !tile_off || !pair_lt_off || !dL_dcolor) return GART_ERR_INVALID_ARG;
+    if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
@@ -320,40 +345,10 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     const float4* pre4 = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
     gart_status s;
-    if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, pair_gid, pair_mask, pair_lt_off, lt4, dL_dcolor, cf, grad, counts);
-    else s = launch_pairs<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, pair_gid, pair_mask, pair_lt_off, lt4, dL_dcolor, cf, grad, counts);
+    if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, grad, counts);
+    else s = launch_pairs<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, grad, counts);
     if (s != GART_OK) return s;
     bwd_finalize_kernel<<<(unsigned)ceil_div(g->n, 256), 256, 0, st>>>(g->n, g->scale, g->quat, g->opacity, grad, counts);
-    GART_LAUNCH_CHECK();
-    return GART_OK;
-}
-
-extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam,
-                                            const float* pre, const uint32_t* ray_off, const uint32_t* ray_gid,
-                                            const uint32_t* ray_slot, const float* lt, const float* dL_dcolor,
-                                            float* grad, const uint32_t* counts, void* stream) {
-    using namespace gart;
-    if (!cfg || !g || !cam || !counts || !ray_off || !dL_dcolor) return GART_ERR_INVALID_ARG;
-    if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
-    if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !g->scale || !g->quat || !g->opacity || !g->sh) return GART_ERR_INVALID_ARG;
-    cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(grad, 0, (size_t)g->n * GART_GRAD_WORDS * sizeof(float), st) != cudaSuccess) return GART_ERR_CUDA;
-    const CamF cf = make_camf(cam, cfg->tile_size);
-    const int64_t n_rays = (int64_t)cam->width * cam->height;
-    const float4* pre4 = reinterpret_cast<const float4*>(pre);
-    const float4* lt4 = reinterpret_cast<const float4*>(lt);
-    const unsigned blocks = (unsigned)ceil_div(n_rays, 128);
-#define GART_ATOMIC(D) \
-    bwd_atomic_kernel<D><<<blocks, 128, 0, st>>>(pre4, g->sh, g->scale, g->quat, g->opacity, ray_off, ray_gid, ray_slot, lt4, dL_dcolor, cf, grad, counts)
-    switch (g->sh_degree) {
-        case 0: GART_ATOMIC(0); break;
-        case 1: GART_ATOMIC(1); break;
-        case 2: GART_ATOMIC(2); break;
-        default: GART_ATOMIC(3); break;
-    }
-#undef GART_ATOMIC
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

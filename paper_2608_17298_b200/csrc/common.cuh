@@ -132,6 +132,49 @@ __device__ __forceinline__ float3 ray_xg(const RayEval& r) {
                        (r.dg.x * r.cr.y - r.dg.y * r.cr.x) * r.inv_a);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Hit mask of a (tile, Gaussian) pair held as 64-bit words, walked bit by bit in pixel order.
+// One loop over all words, so that the trip count of a lane is its hit count (lanes of a warp
+// own pairs of nearly equal hit count) whatever the distribution of the bits over the words.
+template <int MW>
+struct PairMask {
+    static constexpr int N64 = MW / 2;
+    unsigned long long w[N64];
+    unsigned long long cur;
+    int qi;
+    __device__ __forceinline__ void load(const uint32_t* __restrict__ pair_mask, uint32_t j, bool act) {
+#pragma unroll
+        for (int q = 0; q < N64; ++q) {
+            const uint2 t = act ? __ldg(reinterpret_cast<const uint2*>(pair_mask + (size_t)j * MW) + q) : make_uint2(0u, 0u);
+            w[q] = ((unsigned long long)t.y << 32) | t.x;
+        }
+        cur = w[0];
+        qi = 0;
+    }
+    __device__ __forceinline__ int count() const {
+        int c = 0;
+#pragma unroll
+        for (int q = 0; q < N64; ++q) c += __popcll(w[q]);
+        return c;
+    }
+    // index (pixel of the tile) of the next set bit; call at most count() times
+    __device__ __forceinline__ int next() {
+        if (N64 > 1) {
+            while (cur == 0ull) {
+                ++qi;
+                cur = qi == 1 ? w[1 % N64] : (qi == 2 ? w[2 % N64] : w[3 % N64]);
+            }
+        }
+        const int b = __ffsll((long long)cur) - 1;
+        cur &= cur - 1ull;
+        return qi * 64 + b;
+    }
+};
+
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 // ---------------------------------------------------------------------------------------------
 // Real spherical harmonics (index k = l(l+1)+m) of a unit vector, first K values.
 template <int K>

@@ -3,20 +3,22 @@
 //
 // The paper finds the hits of a ray with hardware ray tracing over a BVH of bounded proxies;
 // here candidates come from the tile lists (same hit set: a hit is alpha >= alpha_min, i.e.
-// the ray meets the clamped ellipsoid whose projection the rectangle bounds).  Four phases:
-//   1. fwd_mask   block per tile, thread per pixel: every pixel of the tile evaluates every
-//                 Gaussian of the tile list (records broadcast from shared memory); a warp
-//                 ballot yields the pair's hit mask; pixels count their hits.
-//   2. scans      hits per pair -> pair_lt_off (slot base of every pair in LT: pair-major,
-//                 then pixel -- each hit owns one slot, so forward writes never collide and
-//                 the backward thread of a pair reads one contiguous run); hits per ray ->
-//                 ray_off.
-//   3. fwd_keys   block per tile, thread per pixel: for every set mask bit compute t*, alpha
-//                 and the SH colour (SH coefficients staged per tile in shared memory) and
-//                 append (t*, index) keys plus payload to the ray's segment.
+// the ray meets the clamped ellipsoid whose projection the rectangle bounds).  Phases:
+//   1. fwd_mask    block per tile, thread per pixel: every pixel of the tile evaluates every
+//                  Gaussian of the tile list (records broadcast from shared memory); a warp
+//                  ballot yields the pair's hit mask; pixels count their hits.
+//   2. tile_sort   warp per tile: stable counting sort of the tile's pairs by descending hit
+//                  count -> pair_order, with copies of id and mask in rank order (rank_gid,
+//                  rank_mask: read coalesced later); groups of 32 consecutive ranks share an LT
+//                  block in which entry e of lane l sits at 32 e + l -> rank_gstart; per-tile LT size.
+//      scans       LT size per tile -> tile_lt_base; hits per ray -> ray_off.
+//   3. fwd_eval    block per tile, one thread per (tile, Gaussian) pair, warps walk rank groups:
+//                  for every hit pixel of the pair compute t*, alpha and the SH colour with the
+//                  Gaussian in registers, and append a 32-byte record to the ray's segment
+//                  (position from a shared-memory cursor per pixel).
 //   4. fwd_sort_sweep  warp per ray: sort the segment by (t*, id), scan the transmittance
-//                 front to back, then sum colour back to front so that each hit gets the
-//                 colour composited behind it without cancellation; write LT, C, T_final.
+//                  front to back, then sum colour back to front so that each hit gets the
+//                  colour composited behind it without cancellation; write LT, C, T_final.
 #include "common.cuh"
 
 namespace gart {
@@ -68,16 +70,82 @@ __global__ void __launch_bounds__(TS * TS) fwd_mask_kernel(const float4* __restr
 }
 
 // ------------------------------------------------------------------------------------------ phase 2
-struct PairHitsF {
-    const uint32_t* mask;
-    const uint32_t* counts;
-    int mw;
-    __device__ __forceinline__ uint32_t operator()(int64_t i) const {
-        if (counts[GART_CNT_ERROR] || i >= counts[GART_CNT_PAIRS]) return 0u;
-        uint32_t s = 0;
-        for (int q = 0; q < mw; ++q) s += __popc(mask[(size_t)i * mw + q]);
-        return s;
+constexpr int SORT_WARPS = 4;
+
+template <int MW>
+__device__ __forceinline__ uint32_t mask_popc(const uint32_t* __restrict__ pair_mask, uint32_t j) {
+    uint32_t c = 0;
+#pragma unroll
+    for (int q = 0; q < MW; ++q) c += __popc(__ldg(pair_mask + (size_t)j * MW + q));
+    return c;
+}
+
+template <int TS>
+__global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_gid,
+                                                                    const uint32_t* __restrict__ pair_mask, int T, uint32_t* pair_order,
+                                                                    uint32_t* __restrict__ rank_gid, uint32_t* __restrict__ rank_mask,
+                                                                    uint32_t* __restrict__ rank_gstart,
+                                                                    uint32_t* __restrict__ tile_slots, const uint32_t* __restrict__ counts) {
+    constexpr int NT = TS * TS, MW = NT / 32, NB = NT + 1;
+    __shared__ uint32_t hist[SORT_WARPS][NB];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int tile = blockIdx.x * SORT_WARPS + w;
+    if (tile >= T) return;
+    if (counts[GART_CNT_ERROR]) { if (lane == 0) tile_slots[tile] = 0; return; }
+    const uint32_t begin = tile_off[tile], n = tile_off[tile + 1] - begin;
+    if (n == 0) { if (lane == 0) tile_slots[tile] = 0; return; }
+    for (int d = lane; d < NB; d += 32) hist[w][d] = 0;
+    __syncwarp();
+    for (uint32_t r0 = 0; r0 < n; r0 += 32)
+        if (r0 + lane < n) atomicAdd(&hist[w][mask_popc<MW>(pair_mask, begin + r0 + lane)], 1u);
+    __syncwarp();
+    if (lane == 0) {   // first rank of every hit count, largest count first
+        uint32_t run = 0;
+        for (int c = NT; c >= 0; --c) { const uint32_t t = hist[w][c]; hist[w][c] = run; run += t; }
     }
+    __syncwarp();
+    for (uint32_t r0 = 0; r0 < n; r0 += 32) {
+        const bool act = r0 + lane < n;
+        const unsigned amask = __ballot_sync(0xffffffffu, act);
+        if (act) {
+            const uint32_t j = begin + r0 + lane;
+            const uint32_t c = mask_popc<MW>(pair_mask, j);
+            const unsigned peers = __match_any_sync(amask, c);
+            const uint32_t rk = __popc(peers & ((1u << lane) - 1u));
+            const uint32_t pos = hist[w][c] + rk;
+            __syncwarp(amask);
+            if (rk == 0) hist[w][c] += __popc(peers);
+            __syncwarp(amask);
+            pair_order[begin + pos] = j;
+        }
+    }
+    __threadfence_block();
+    __syncwarp();
+    uint32_t run = 0;
+    for (uint32_t r0 = 0; r0 < n; r0 += 32) {
+        const bool act = r0 + lane < n;
+        const uint32_t j = act ? __ldcg(pair_order + begin + r0 + lane) : 0u;
+        uint32_t c = 0;
+        if (act) {
+            const size_t q = (size_t)begin + r0 + lane;
+#pragma unroll
+            for (int m = 0; m < MW; ++m) {
+                const uint32_t wv = __ldg(pair_mask + (size_t)j * MW + m);
+                rank_mask[q * MW + m] = wv;
+                c += __popc(wv);
+            }
+            rank_gid[q] = __ldg(pair_gid + j);
+            rank_gstart[q] = run;
+        }
+        const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
+        run += 32u * cmax;
+    }
+    if (lane == 0) tile_slots[tile] = run;
+}
+
+struct TileSlotsF {
+    const uint32_t* tile_slots;
+    __device__ __forceinline__ uint32_t operator()(int64_t i) const { return tile_slots[i]; }
 };
 
 struct RayHitsF {
@@ -88,81 +156,89 @@ struct RayHitsF {
     }
 };
 
-__global__ void hits_total_kernel(const uint64_t* total64, int64_t cap_hits, uint32_t* counts) {
-    const uint64_t H = total64[0];
+__global__ void hits_total_kernel(const uint64_t* total_slots, const uint64_t* total_hits, int64_t cap_hits, uint32_t* counts) {
+    const uint64_t L = total_slots[0], H = total_hits[0];
     counts[GART_CNT_HITS] = H > 0xffffffffull ? 0xffffffffu : (uint32_t)H;
-    if (H > (uint64_t)cap_hits) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_HITS);
+    counts[GART_CNT_LT_SLOTS] = L > 0xffffffffull ? 0xffffffffu : (uint32_t)L;
+    if (L > (uint64_t)cap_hits || H > (uint64_t)cap_hits) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_HITS);
 }
 
 // ------------------------------------------------------------------------------------------ phase 3
+constexpr int EVAL_THREADS = 128;
+
 template <int TS, int DEG>
-__global__ void __launch_bounds__(TS * TS) fwd_keys_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
-                                                           const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_gid,
-                                                           const uint32_t* __restrict__ pair_mask, const uint32_t* __restrict__ pair_lt_off,
-                                                           const uint32_t* __restrict__ ray_off, CamF cam,
-                                                           uint64_t* __restrict__ keys, float4* __restrict__ payload,
-                                                           uint32_t* __restrict__ hit_gid, uint32_t* __restrict__ hit_slot,
-                                                           const uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, CH = 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K;
-    __shared__ float4 sp[CH * 5];
-    __shared__ float ssh[CH * SW];
-    __shared__ uint32_t smask[CH * MW];
-    __shared__ uint32_t sbase[CH];
-    __shared__ uint32_t sgid[CH];
+__global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
+                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_gid,
+                                                                const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
+                                                                const uint32_t* __restrict__ tile_lt_base,
+                                                                const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
+                                                                const uint32_t* __restrict__ counts) {
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3;
+    __shared__ __align__(16) float spix[NT * PW];
+    __shared__ uint32_t sro[NT];
+    __shared__ uint32_t scur[NT];
     if (counts[GART_CNT_ERROR]) return;
     const int tile = blockIdx.x;
+    const uint32_t begin = tile_off[tile], n = tile_off[tile + 1] - begin;
+    if (n == 0) return;
     const int tx = tile % cam.tiles_x, ty = tile / cam.tiles_x;
-    const int p = threadIdx.x, lane = p & 31, warp = p >> 5;
-    const int x = tx * TS + p % TS, y = ty * TS + p / TS;
-    const bool inside = x < cam.width && y < cam.height;
-    const uint32_t begin = tile_off[tile], end = tile_off[tile + 1];
-    if (begin == end) return;
-    float Y[K];
-    sh_basis<K>(pixel_dir(cam, min(x, cam.width - 1), min(y, cam.height - 1)), Y);
-    size_t w = inside ? (size_t)ray_off[(size_t)y * cam.width + x] : 0;
-    uint32_t local = 0;
-    for (uint32_t base = begin; base < end; base += CH) {
-        const int nb = min((uint32_t)CH, end - base);
-        for (int i = p; i < nb; i += NT) {
-            sgid[i] = __ldg(pair_gid + base + i);
-            sbase[i] = __ldg(pair_lt_off + base + i);
-        }
-        for (int i = p; i < nb * MW; i += NT) smask[i] = __ldg(pair_mask + (size_t)base * MW + i);
-        __syncthreads();
-        for (int i = p; i < nb * 5; i += NT) {
-            const int pair = i / 5, q = i - pair * 5;
-            sp[i] = __ldg(pre4 + (size_t)sgid[pair] * 5 + q);
-        }
-        for (int i = p; i < nb * SW; i += NT) {
-            const int pair = i / SW, q = i - pair * SW;
-            ssh[i] = __ldg(sh + (size_t)sgid[pair] * SW + q);
-        }
-        __syncthreads();
-        for (int j = 0; j < nb; ++j) {
-            const uint32_t word = smask[j * MW + warp];
-            if ((word >> lane) & 1u) {
-                const PreRec P = unpack_pre(sp[j * 5], sp[j * 5 + 1], sp[j * 5 + 2], sp[j * 5 + 3], sp[j * 5 + 4]);
-                const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
-                const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
-                float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
-                const float* s = ssh + j * SW;
+    const int x0 = tx * TS, y0 = ty * TS;
+    for (int p = threadIdx.x; p < NT; p += EVAL_THREADS) {
+        const int x = x0 + p % TS, y = y0 + p / TS;
+        float Y[K];
+        sh_basis<K>(pixel_dir(cam, min(x, cam.width - 1), min(y, cam.height - 1)), Y);
 #pragma unroll
-                for (int k = 0; k < K; ++k) {
-                    c0 = fmaf(Y[k], s[3 * k], c0);
-                    c1 = fmaf(Y[k], s[3 * k + 1], c1);
-                    c2 = fmaf(Y[k], s[3 * k + 2], c2);
+        for (int k = 0; k < K; ++k) spix[p * PW + k] = Y[k];
+        sro[p] = (x < cam.width && y < cam.height) ? ray_off[(size_t)y * cam.width + x] : 0u;
+        scur[p] = 0u;
+    }
+    __syncthreads();
+    const uint32_t lt_base = tile_lt_base[tile];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t r0 = warp * 32; r0 < n; r0 += EVAL_THREADS) {
+        const bool act = r0 + lane < n;
+        const uint32_t q = begin + r0 + lane;
+        PairMask<MW> pm;
+        pm.load(rank_mask, act ? q : 0u, act);
+        const int c = pm.count();
+        if (__ballot_sync(0xffffffffu, c != 0) == 0u) break;   // ranks descend in hit count: nothing left in this tile
+        if (c == 0) continue;
+        const uint32_t gid = __ldg(rank_gid + q);
+        const PreRec P = load_pre(pre4, gid);
+        float shc[SW];
+        {
+            const float* sp = sh + (size_t)gid * SW;
+            if (SW % 4 == 0) {
+#pragma unroll
+                for (int q = 0; q < SW / 4; ++q) {
+                    const float4 t = __ldg(reinterpret_cast<const float4*>(sp) + q);
+                    shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
                 }
-                uint32_t slot = sbase[j] + __popc(word & ((1u << lane) - 1u));
-                for (int q = 0; q < warp; ++q) slot += __popc(smask[j * MW + q]);
-                keys[w] = ((uint64_t)__float_as_uint(t) << 32) | (uint64_t)local;
-                payload[w] = make_float4(r.alpha, fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f));
-                hit_gid[w] = sgid[j];
-                hit_slot[w] = slot;
-                ++w;
-                ++local;
+            } else {
+#pragma unroll
+                for (int q = 0; q < SW; ++q) shc[q] = __ldg(sp + q);
             }
         }
-        __syncthreads();
+        uint32_t slot = lt_base + __ldg(rank_gstart + q) + lane;
+        const int bx = x0 - P.ix, by = y0 - P.iy;
+        for (int e = 0; e < c; ++e) {
+            const int p = pm.next();
+            const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
+            const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
+            const float* Y = spix + p * PW;
+            float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                c0 = fmaf(Y[k], shc[3 * k], c0);
+                c1 = fmaf(Y[k], shc[3 * k + 1], c1);
+                c2 = fmaf(Y[k], shc[3 * k + 2], c2);
+            }
+            const uint32_t pos = atomicAdd(&scur[p], 1u);
+            float4* rec = recs + ((size_t)sro[p] + pos) * 2;
+            rec[0] = make_float4(t, __uint_as_float(gid), __uint_as_float(slot), r.alpha);
+            rec[1] = make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f);
+            slot += 32u;
+        }
     }
 }
 
@@ -199,9 +275,10 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
     }
 }
 
-__global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, uint64_t* __restrict__ keys,
-                                                                          const float4* __restrict__ payload, const uint32_t* __restrict__ hit_gid,
-                                                                          const uint32_t* __restrict__ hit_slot, int64_t n_rays,
+// Keys are (t* bits << 32) | record index.  A ray's records arrive in arbitrary order, so hits with
+// bit-identical t* are put in ascending Gaussian id afterwards (rare: one lane, insertion sort).
+__global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs,
+                                                                          uint64_t* __restrict__ long_keys, int64_t n_rays,
                                                                           float bg0, float bg1, float bg2,
                                                                           float* __restrict__ color, float* __restrict__ t_final,
                                                                           float4* __restrict__ lt, uint32_t* __restrict__ ray_gid,
@@ -220,23 +297,36 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         }
         return;
     }
-    uint64_t* kp;
-    if (n <= SORT_CAP) {
-        kp = skeys[warp];
-        for (int i = lane; i < n; i += 32) kp[i] = keys[b + i];
-    } else {
-        kp = keys + b;
-    }
+    const float4* rec = recs + b * 2;
+    uint64_t* kp = n <= SORT_CAP ? skeys[warp] : long_keys + b;
+    for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
     __syncwarp();
     warp_sort(kp, n, lane);
+    bool tie = false;
+    for (int i = lane; i + 1 < n; i += 32) tie = tie || ((uint32_t)(kp[i] >> 32) == (uint32_t)(kp[i + 1] >> 32));
+    if (__any_sync(0xffffffffu, tie)) {
+        if (lane == 0) {
+            for (int i = 1; i < n; ++i) {
+                const uint64_t x = kp[i];
+                const uint32_t tx = (uint32_t)(x >> 32), gx = __float_as_uint(rec[2 * (uint32_t)x].y);
+                int m = i;
+                while (m > 0 && (uint32_t)(kp[m - 1] >> 32) == tx && __float_as_uint(rec[2 * (uint32_t)kp[m - 1]].y) > gx) {
+                    kp[m] = kp[m - 1];
+                    --m;
+                }
+                kp[m] = x;
+            }
+        }
+        __syncwarp();
+    }
 
-    // front to back: transmittance in front of every hit (Eq. 7); stored in the key's high word
+    // front to back: transmittance in front of every hit (Eq. 7); kept in the key's high word
     float carryT = 1.0f;
     for (int base = 0; base < n; base += 32) {
         const int i = base + lane;
         const bool valid = i < n;
         const uint32_t c = valid ? (uint32_t)kp[i] : 0u;
-        const float alpha = valid ? payload[b + c].x : 0.0f;
+        const float alpha = valid ? __ldg(&rec[2 * c].w) : 0.0f;
         float prod = 1.0f - alpha;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -258,14 +348,15 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         const int i = n - 1 - (base + lane);
         const bool valid = i >= 0;
         float T = 0.0f, v0 = 0.0f, v1 = 0.0f, v2 = 0.0f;
-        uint32_t c = 0;
+        float4 ra = make_float4(0.f, 0.f, 0.f, 0.f);
         if (valid) {
             const uint64_t key = kp[i];
-            c = (uint32_t)key;
+            const uint32_t c = (uint32_t)key;
             T = __uint_as_float((uint32_t)(key >> 32));
-            const float4 pl = payload[b + c];
-            const float wgt = T * pl.x;
-            v0 = wgt * pl.y; v1 = wgt * pl.z; v2 = wgt * pl.w;
+            ra = __ldg(&rec[2 * c]);
+            const float4 rb = __ldg(&rec[2 * c + 1]);
+            const float wgt = T * ra.w;
+            v0 = wgt * rb.x; v1 = wgt * rb.y; v2 = wgt * rb.z;
         }
         float s0 = v0, s1 = v1, s2 = v2;
 #pragma unroll
@@ -278,9 +369,9 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         float e0 = __shfl_up_sync(0xffffffffu, s0, 1), e1 = __shfl_up_sync(0xffffffffu, s1, 1), e2 = __shfl_up_sync(0xffffffffu, s2, 1);
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
-            const uint32_t slot = hit_slot[b + c];
+            const uint32_t slot = __float_as_uint(ra.z);
             lt[slot] = make_float4(k0 + e0, k1 + e1, k2 + e2, T);
-            ray_gid[b + i] = hit_gid[b + c];
+            ray_gid[b + i] = __float_as_uint(ra.y);
             ray_slot[b + i] = slot;
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -295,44 +386,45 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
 
 // ------------------------------------------------------------------------------------------ host
 struct ForwardWs {
-    uint64_t* total64;
+    uint64_t *total_slots, *total_hits;
     void* scan_ws;
-    uint64_t* keys;
-    float4* payload;
-    uint32_t *hit_gid, *hit_slot;
+    uint32_t* tile_slots;
+    float4* recs;
+    uint64_t* long_keys;
     size_t bytes;
 };
 
-static ForwardWs forward_layout(void* base, int64_t n_rays, int64_t cap_pairs, int64_t cap_hits) {
+static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_hits) {
     ForwardWs w;
     char* p = (char*)base;
     size_t off = 0;
     auto take = [&](size_t b) { void* r = p ? (void*)(p + off) : nullptr; off += align256(b); return r; };
     const int64_t ch = cap_hits > 0 ? cap_hits : 1;
-    w.total64 = (uint64_t*)take(256);
-    w.scan_ws = take(scan_workspace_bytes(cap_pairs > n_rays ? cap_pairs : n_rays));
-    w.keys = (uint64_t*)take((size_t)ch * 8);
-    w.payload = (float4*)take((size_t)ch * 16);
-    w.hit_gid = (uint32_t*)take((size_t)ch * 4);
-    w.hit_slot = (uint32_t*)take((size_t)ch * 4);
+    w.total_slots = (uint64_t*)take(256);
+    w.total_hits = (uint64_t*)take(256);
+    w.scan_ws = take(scan_workspace_bytes(n_rays > T ? n_rays : T));
+    w.tile_slots = (uint32_t*)take((size_t)(T + 1) * 4);
+    w.recs = (float4*)take((size_t)ch * 32);
+    w.long_keys = (uint64_t*)take((size_t)ch * 8);
     w.bytes = off;
     return w;
 }
 
 template <int TS>
-static gart_status launch_keys(int deg, int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
-                               const uint32_t* pair_gid, const uint32_t* pair_mask, const uint32_t* pair_lt_off,
-                               const uint32_t* ray_off, const CamF& cam, const ForwardWs& w, const uint32_t* counts) {
-#define GART_KEYS(D)                                                                                                   \
-    fwd_keys_kernel<TS, D><<<T, TS * TS, 0, st>>>(pre4, sh, tile_off, pair_gid, pair_mask, pair_lt_off, ray_off, cam, \
-                                                  w.keys, w.payload, w.hit_gid, w.hit_slot, counts)
+static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
+                               const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+                               const uint32_t* tile_lt_base, const uint32_t* ray_off,
+                               const CamF& cam, const ForwardWs& w, const uint32_t* counts) {
+#define GART_EVAL(D)                                                                                                      \
+    fwd_eval_kernel<TS, D><<<T, EVAL_THREADS, 0, st>>>(pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart,             \
+                                                       tile_lt_base, ray_off, cam, w.recs, counts)
     switch (deg) {
-        case 0: GART_KEYS(0); break;
-        case 1: GART_KEYS(1); break;
-        case 2: GART_KEYS(2); break;
-        default: GART_KEYS(3); break;
+        case 0: GART_EVAL(0); break;
+        case 1: GART_EVAL(1); break;
+        case 2: GART_EVAL(2); break;
+        default: GART_EVAL(3); break;
     }
-#undef GART_KEYS
+#undef GART_EVAL
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
@@ -340,31 +432,34 @@ static gart_status launch_keys(int deg, int T, cudaStream_t st, const float4* pr
 }  // namespace gart
 
 extern "C" size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits) {
-    (void)tile_size;
-    return gart::forward_layout(nullptr, (int64_t)width * height, cap_pairs > 0 ? cap_pairs : 1, cap_hits).bytes;
+    (void)cap_pairs;
+    if (tile_size != 8 && tile_size != 16) return 0;
+    const int T = ((width + tile_size - 1) / tile_size) * ((height + tile_size - 1) / tile_size);
+    return gart::forward_layout(nullptr, (int64_t)width * height, T, cap_hits).bytes;
 }
 
 extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                     const uint32_t* tile_off, const uint32_t* pair_gid, int64_t cap_pairs,
                                     float* color, float* t_final, uint32_t* hit_count,
-                                    uint32_t* pair_mask, uint32_t* pair_lt_off, float* lt, int64_t cap_hits,
+                                    uint32_t* pair_mask, uint32_t* pair_order, uint32_t* rank_gid, uint32_t* rank_mask,
+                                    uint32_t* rank_gstart, uint32_t* tile_lt_base,
+                                    float* lt, int64_t cap_hits,
                                     uint32_t* ray_off, uint32_t* ray_gid, uint32_t* ray_slot, uint32_t* counts,
                                     void* workspace, size_t workspace_bytes, void* stream) {
     using namespace gart;
-    if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !pair_lt_off || !ray_off || !counts)
+    if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !tile_lt_base || !ray_off || !counts)
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
-    if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pre || !g->sh)) return GART_ERR_INVALID_ARG;
+    if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_gid || !rank_mask || !rank_gstart || !pre || !g->sh)) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0 && (!lt || !ray_gid || !ray_slot)) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     const int ts = cfg->tile_size;
     const CamF cf = make_camf(cam, ts);
     const int T = cf.tiles_x * cf.tiles_y;
     const int64_t n_rays = (int64_t)cam->width * cam->height;
-    const int64_t cp = cap_pairs > 0 ? cap_pairs : 1;
-    ForwardWs w = forward_layout(workspace, n_rays, cp, cap_hits);
+    ForwardWs w = forward_layout(workspace, n_rays, T, cap_hits);
     if (w.bytes > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     const float4* pre4 = reinterpret_cast<const float4*>(pre);
@@ -373,21 +468,26 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     else fwd_mask_kernel<16><<<T, 256, 0, st>>>(pre4, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
     GART_LAUNCH_CHECK();
 
-    PairHitsF pf{pair_mask, counts, ts * ts / 32};
-    gart_status s = exclusive_scan(pf, cp, pair_lt_off, w.total64, w.scan_ws, st);
-    if (s != GART_OK) return s;
-    RayHitsF rf{hit_count, counts};
-    s = exclusive_scan(rf, n_rays, ray_off, w.total64, w.scan_ws, st);
-    if (s != GART_OK) return s;
-    hits_total_kernel<<<1, 1, 0, st>>>(w.total64, cap_hits, counts);
+    const int sblocks = (int)ceil_div(T, SORT_WARPS);
+    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, pair_mask, T, pair_order, rank_gid, rank_mask, rank_gstart, w.tile_slots, counts);
+    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, pair_mask, T, pair_order, rank_gid, rank_mask, rank_gstart, w.tile_slots, counts);
     GART_LAUNCH_CHECK();
 
-    if (ts == 8) s = launch_keys<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, pair_gid, pair_mask, pair_lt_off, ray_off, cf, w, counts);
-    else s = launch_keys<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, pair_gid, pair_mask, pair_lt_off, ray_off, cf, w, counts);
+    TileSlotsF tf{w.tile_slots};
+    gart_status s = exclusive_scan(tf, (int64_t)T, tile_lt_base, w.total_slots, w.scan_ws, st);
+    if (s != GART_OK) return s;
+    RayHitsF rf{hit_count, counts};
+    s = exclusive_scan(rf, n_rays, ray_off, w.total_hits, w.scan_ws, st);
+    if (s != GART_OK) return s;
+    hits_total_kernel<<<1, 1, 0, st>>>(w.total_slots, w.total_hits, cap_hits, counts);
+    GART_LAUNCH_CHECK();
+
+    if (ts == 8) s = launch_eval<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
+    else s = launch_eval<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);
-    fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, 0, st>>>(ray_off, w.keys, w.payload, w.hit_gid, w.hit_slot, n_rays,
+    fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, 0, st>>>(ray_off, w.recs, w.long_keys, n_rays,
                                                                          cfg->background[0], cfg->background[1], cfg->background[2],
                                                                          color, t_final, reinterpret_cast<float4*>(lt), ray_gid,
                                                                          ray_slot, counts);

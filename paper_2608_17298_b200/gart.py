@@ -21,8 +21,8 @@ LIB_PATH = os.path.join(_HERE, "libgart.so")
 GART_OK = 0
 STATUS_NAMES = {0: "GART_OK", 1: "GART_ERR_INVALID_ARG", 2: "GART_ERR_WORKSPACE_TOO_SMALL",
                 3: "GART_ERR_CAPACITY_EXCEEDED", 4: "GART_ERR_CUDA"}
-CNT_VISIBLE, CNT_PAIRS, CNT_SLOTS_LO, CNT_SLOTS_HI, CNT_HITS, CNT_ERROR, CNT_MAX_RAY_HITS, CNT_STRADDLE = range(8)
-COUNTS_WORDS = 8
+CNT_VISIBLE, CNT_PAIRS, CNT_SLOTS_LO, CNT_SLOTS_HI, CNT_HITS, CNT_ERROR, CNT_MAX_RAY_HITS, CNT_STRADDLE, CNT_LT_SLOTS = range(9)
+COUNTS_WORDS = 12
 PRE_WORDS = 20
 GRAD_WORDS = 64
 
@@ -75,8 +75,8 @@ def lib():
         L.gart_tile_map.argtypes = [vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, sz, vp]
         L.gart_forward_workspace_bytes.restype = sz
         L.gart_forward_workspace_bytes.argtypes = [i32, i32, i32, i64, i64]
-        L.gart_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
-        L.gart_backward.argtypes = [vp] * 13
+        L.gart_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.gart_backward.argtypes = [vp] * 14
         L.gart_backward_atomic.argtypes = [vp] * 12
         L.gart_read_counts.argtypes = [vp, vp, vp]
         L.gart_view_host_arena_bytes.restype = sz
@@ -209,26 +209,30 @@ def gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits) 
 
 
 def gart_forward(cfg: Config, g: Gaussians, cam, pre, tile_off, pair_gid, cap_pairs, color, t_final, hit_count,
-                 pair_mask, pair_lt_off, lt, cap_hits, ray_off, ray_gid, ray_slot, counts, workspace, stream=None):
+                 pair_mask, pair_order, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, cap_hits, ray_off, ray_gid,
+                 ray_slot, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     _check(lib().gart_forward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
                               _dev(pair_gid, i32, "pair_gid"), int(cap_pairs), _dev(color, f32, "color"),
                               _dev(t_final, f32, "t_final"), _dev(hit_count, i32, "hit_count"),
-                              _dev(pair_mask, i32, "pair_mask"), _dev(pair_lt_off, i32, "pair_lt_off"),
+                              _dev(pair_mask, i32, "pair_mask"), _dev(pair_order, i32, "pair_order"),
+                              _dev(rank_gid, i32, "rank_gid"), _dev(rank_mask, i32, "rank_mask"),
+                              _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
                               _dev(lt, f32, "lt"), int(cap_hits), _dev(ray_off, i32, "ray_off"),
                               _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"),
                               _dev(counts, i32, "counts"), _dev(workspace, torch.uint8, "workspace"),
                               workspace.numel() if workspace is not None else 0, _stream_ptr(stream)), "gart_forward")
 
 
-def gart_backward(cfg: Config, g: Gaussians, cam, pre, tile_off, pair_gid, pair_mask, pair_lt_off, lt, dL_dcolor,
-                  grad, counts, stream=None):
+def gart_backward(cfg: Config, g: Gaussians, cam, pre, tile_off, rank_gid, rank_mask, rank_gstart,
+                  tile_lt_base, lt, dL_dcolor, grad, counts, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     _check(lib().gart_backward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
-                               _dev(pair_gid, i32, "pair_gid"), _dev(pair_mask, i32, "pair_mask"),
-                               _dev(pair_lt_off, i32, "pair_lt_off"), _dev(lt, f32, "lt"),
+                               _dev(rank_gid, i32, "rank_gid"), _dev(rank_mask, i32, "rank_mask"),
+                               _dev(rank_gstart, i32, "rank_gstart"),
+                               _dev(tile_lt_base, i32, "tile_lt_base"), _dev(lt, f32, "lt"),
                                _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"), _dev(counts, i32, "counts"),
                                _stream_ptr(stream)), "gart_backward")
 
@@ -298,7 +302,9 @@ class ViewBuffers:
         self.rect, self.cls, self.pre = e((n1, 4), i32), e((n1,), u8), e((n1, PRE_WORDS), f32)
         self.counts = torch.zeros(COUNTS_WORDS, dtype=i32, device=device)
         self.tile_off, self.pair_gid = e((T + 1,), i32), e((cp,), i32)
-        self.pair_mask, self.pair_lt_off = e((cp, mw), i32), e((cp + 1,), i32)
+        self.pair_mask, self.pair_order = e((cp, mw), i32), e((cp,), i32)
+        self.rank_gid, self.rank_mask, self.rank_gstart = e((cp,), i32), e((cp, mw), i32), e((cp,), i32)
+        self.tile_lt_base = e((T + 1,), i32)
         self.color, self.t_final, self.hit_count = e((H, W, 3), f32), e((H, W), f32), e((H, W), i32)
         self.lt = e((ch, 4), f32)
         self.ray_off, self.ray_gid, self.ray_slot = e((H * W + 1,), i32), e((ch,), i32), e((ch,), i32)
@@ -317,13 +323,13 @@ def run_bounds_tile_map(cfg, g, cam, buf: ViewBuffers, stream=None):
 
 def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None):
     gart_forward(cfg, g, cam, buf.pre, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color, buf.t_final, buf.hit_count,
-                 buf.pair_mask, buf.pair_lt_off, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot,
-                 buf.counts, buf.workspace, stream)
+                 buf.pair_mask, buf.pair_order, buf.rank_gid, buf.rank_mask, buf.rank_gstart, buf.tile_lt_base, buf.lt,
+                 buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.counts, buf.workspace, stream)
 
 
 def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
-    gart_backward(cfg, g, cam, buf.pre, buf.tile_off, buf.pair_gid, buf.pair_mask, buf.pair_lt_off, buf.lt, dL_dcolor,
-                  buf.grad if grad is None else grad, buf.counts, stream)
+    gart_backward(cfg, g, cam, buf.pre, buf.tile_off, buf.rank_gid, buf.rank_mask, buf.rank_gstart,
+                  buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts, stream)
 
 
 def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):
@@ -332,12 +338,14 @@ def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=N
 
 
 def size_view(cfg, g, cam, slack=1.0, device="cuda"):
-    """Run bounds + tile map with a probing allocation and return (P, S): exact pair count and the
-    capacity bound of the intermediate buffer (sum of rectangle areas).  Two host round trips; meant
-    for set-up, not for the steady state."""
+    """Run bounds + tile map with a probing allocation and return (cap_pairs, cap_hits): the exact pair
+    count and a capacity that always holds the intermediate buffer (sum of rectangle areas plus the
+    worst-case padding of its interleaved layout), each times `slack`.  Two host round trips; meant for
+    set-up, not for the steady state."""
     probe = ViewBuffers(g.n, g.sh_degree, cam, cfg, 0, 0, device)
     run_bounds_tile_map(cfg, g, cam, probe)
     cnt = gart_read_counts(probe.counts)
     P = cnt[CNT_PAIRS]
     S = cnt[CNT_SLOTS_LO] | (cnt[CNT_SLOTS_HI] << 32)
-    return int(P * slack) + 1, int(S * slack) + 1
+    pad = 32 * cfg.tile_size ** 2 * min(tiles(cam, cfg.tile_size), P)
+    return int(P * slack) + 1, int(S * slack) + pad + 1

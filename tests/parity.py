@@ -53,13 +53,17 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         return out
     out["pair_gid"] = u32(to_np(buf.pair_gid))[:P]
     out["pair_mask"] = u32(to_np(buf.pair_mask))[:P]
-    out["pair_lt_off"] = u32(to_np(buf.pair_lt_off))[:P + 1]
+    out["pair_order"] = u32(to_np(buf.pair_order))[:P]
+    out["rank_gid"] = u32(to_np(buf.rank_gid))[:P]
+    out["rank_mask"] = u32(to_np(buf.rank_mask))[:P]
+    out["rank_gstart"] = u32(to_np(buf.rank_gstart))[:P]
+    out["tile_lt_base"] = u32(to_np(buf.tile_lt_base))
     out["color"], out["t_final"] = to_np(buf.color), to_np(buf.t_final)
     out["hit_count"] = u32(to_np(buf.hit_count))
     out["ray_off"] = u32(to_np(buf.ray_off))
     out["ray_gid"] = u32(to_np(buf.ray_gid))[:H]
     out["ray_slot"] = u32(to_np(buf.ray_slot))[:H]
-    out["lt"] = to_np(buf.lt)[:H]
+    out["lt"] = to_np(buf.lt)[:counts[G.CNT_LT_SLOTS]]
     out["grad"] = to_np(buf.grad)[:g.n].copy()
     if atomic:
         ga = torch.empty_like(buf.grad)
@@ -90,32 +94,92 @@ def check_maps(scene, cam, cfg: G.Config, gpu):
     return {"rect_identical": bool(same), "n_unsafe": int((~safe).sum()), "osc": osc}
 
 
-def check_structure(cam, cfg: G.Config, gpu):
-    """Properties that hold at any size, checked on the whole view without the oracle."""
+def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
+    """Properties that hold at any size, checked on the whole view without the oracle (the per-hit
+    part on a random subset of rays when the view has more than a few million hits)."""
     H = gpu["counts"][G.CNT_HITS]
+    L = gpu["counts"][G.CNT_LT_SLOTS]
     ray_off, hit_count = gpu["ray_off"].astype(np.int64), gpu["hit_count"].reshape(-1).astype(np.int64)
     assert ray_off[0] == 0 and ray_off[-1] == H and np.array_equal(np.diff(ray_off), hit_count)
-    # pair masks: popcounts give the LT offsets; every hit owns exactly one slot
-    pc = np.unpackbits(gpu["pair_mask"].view(np.uint8), axis=1).sum(axis=1).astype(np.int64)
-    off = gpu["pair_lt_off"].astype(np.int64)
-    assert off[0] == 0 and off[-1] == H and np.array_equal(np.diff(off), pc)
-    slots = np.sort(gpu["ray_slot"].astype(np.int64))
-    assert np.array_equal(slots, np.arange(H))
     assert gpu["counts"][G.CNT_MAX_RAY_HITS] == (hit_count.max() if hit_count.size else 0)
-    # a hit's slot belongs to the pair (tile of the ray, its Gaussian)
+    pc = np.bitwise_count(gpu["pair_mask"]).sum(axis=1).astype(np.int64)
+    assert pc.sum() == H and L >= H
+    # every hit owns exactly one slot
+    slots_all = gpu["ray_slot"]
+    assert np.unique(slots_all).size == H and (int(slots_all.max()) if H else -1) < L
     ts = cfg.tile_size
     tiles_x = -(-cam.width // ts)
-    rays = np.repeat(np.arange(hit_count.size), hit_count)
+    tile_off, base = gpu["tile_off"].astype(np.int64), gpu["tile_lt_base"].astype(np.int64)
+    assert base[0] == 0 and base[-1] == L and np.all(np.diff(base) >= 0)
+    n_tile = np.diff(tile_off)
+    P = pc.size
+    tile_of_pair = np.repeat(np.arange(n_tile.size), n_tile)
+    # pair_order: a permutation of each tile's pairs in descending hit count, stable
+    order = gpu["pair_order"].astype(np.int64)
+    seen = np.zeros(P, bool)
+    seen[order] = True
+    assert seen.all()
+    assert np.array_equal(tile_of_pair[order], tile_of_pair)
+    rank = np.arange(P) - tile_off[tile_of_pair]                 # rank of position q within its tile
+    po = pc[order]
+    same_tile = tile_of_pair[1:] == tile_of_pair[:-1]
+    assert np.all((po[:-1] >= po[1:]) | ~same_tile)
+    assert np.all((order[:-1] < order[1:]) | (po[:-1] != po[1:]) | ~same_tile)
+    # copies in rank order
+    assert np.array_equal(gpu["rank_gid"], gpu["pair_gid"][order]) and np.array_equal(gpu["rank_mask"], gpu["pair_mask"][order])
+    # rank_gstart: start of the 32-rank group; a group spans 32 x its largest (= first) count
+    gs_ = gpu["rank_gstart"].astype(np.int64)                   # by position in rank order
+    first = rank % 32 == 0
+    grp_start, grp_tile, grp_size = gs_[first], tile_of_pair[first], 32 * po[first]
+    assert np.array_equal(np.repeat(grp_start, np.diff(np.r_[np.nonzero(first)[0], P])), gs_)
+    slot0 = np.empty(P, np.int64)
+    slot0[order] = gs_ + rank % 32                               # per pair: first LT entry relative to the tile
+    nxt_same = grp_tile[1:] == grp_tile[:-1]
+    assert np.all((grp_start[1:] == grp_start[:-1] + grp_size[:-1]) | ~nxt_same)
+    assert np.all(grp_start[np.r_[True, ~nxt_same]] == 0)
+    last_of_tile = np.r_[~nxt_same, True]
+    tile_len = np.zeros(n_tile.size, np.int64)
+    tile_len[grp_tile[last_of_tile]] = (grp_start + grp_size)[last_of_tile]
+    assert np.array_equal(tile_len, np.diff(base))
+    # ---- per hit: on all rays, or on a random subset of them
+    n_rays = hit_count.size
+    if H > 5_000_000:
+        rsel = np.sort(np.random.default_rng(seed).choice(n_rays, size=max_rays, replace=False))
+    else:
+        rsel = np.arange(n_rays)
+    cnt = hit_count[rsel]
+    idx = np.repeat(ray_off[rsel], cnt) + (np.arange(cnt.sum()) - np.repeat(np.cumsum(cnt) - cnt, cnt))
+    rays = np.repeat(rsel, cnt)
+    slots = gpu["ray_slot"][idx].astype(np.int64)
+    gids = gpu["ray_gid"][idx].astype(np.int64)
     tile = (rays // cam.width) // ts * tiles_x + (rays % cam.width) // ts
-    pair = np.searchsorted(off, gpu["ray_slot"].astype(np.int64), side="right") - 1
-    assert np.array_equal(gpu["pair_gid"][pair], gpu["ray_gid"])
-    tile_of_pair = np.searchsorted(gpu["tile_off"].astype(np.int64), pair, side="right") - 1
-    assert np.array_equal(tile_of_pair, tile)
-    # LT: transmittance of the first hit of a ray is 1; of later hits in (0, 1]; colours finite
+    rel = slots - base[tile]
+    assert np.all(rel >= 0) and np.all(slots < base[tile + 1])
+    # locate the pair: among the tile's pairs, the one whose Gaussian is the hit's (ids ascend in a tile)
+    pair_gid = gpu["pair_gid"].astype(np.int64)
+    mul = int(pair_gid.max()) + 1 if P else 1
+    key = tile_of_pair * mul + pair_gid
+    want = tile * mul + gids
+    pair = np.searchsorted(key, want)
+    assert np.array_equal(key[pair], want)
+    e = rel - slot0[pair]
+    assert np.all(e % 32 == 0) and np.all(e >= 0) and np.all(e // 32 < pc[pair])
+    # the e-th hit of a pair is its e-th set mask bit in pixel order
+    px = (rays % cam.width) % ts + ((rays // cam.width) % ts) * ts
+    words = gpu["pair_mask"][pair]                                  # [h, MW]
+    w_idx, b_idx = px // 32, px % 32
+    word = words[np.arange(pair.size), w_idx].astype(np.uint64)
+    assert np.all((word >> b_idx.astype(np.uint64)) & np.uint64(1))
+    below = np.bitwise_count(word & ((np.uint64(1) << b_idx.astype(np.uint64)) - np.uint64(1))).astype(np.int64)
+    for q in range(words.shape[1]):
+        below += np.where(q < w_idx, np.bitwise_count(words[:, q]).astype(np.int64), 0)
+    assert np.array_equal(below, e // 32)
+    # LT: transmittance of the first hit of a ray is 1; of later hits in [0, 1]; colours finite
     lt = gpu["lt"]
-    first = ray_off[:-1][hit_count > 0]
-    assert np.all(lt[gpu["ray_slot"][first].astype(np.int64), 3] == 1.0)
-    assert np.all(np.isfinite(lt)) and np.all(lt[:, 3] >= 0) and np.all(lt[:, 3] <= 1.0)
+    first_hit = ray_off[:-1][hit_count > 0]
+    assert np.all(lt[gpu["ray_slot"][first_hit].astype(np.int64), 3] == 1.0)
+    used = lt[slots]
+    assert np.all(np.isfinite(used)) and np.all(used[:, 3] >= 0) and np.all(used[:, 3] <= 1.0)
     assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
 
 

@@ -32,6 +32,6 @@ def test_host_only_queries():
     assert 0 < a < b and a % 256 == 0
     f1 = G.gart_forward_workspace_bytes(640, 480, 8, 10_000, 100_000)
     f2 = G.gart_forward_workspace_bytes(640, 480, 8, 10_000, 200_000)
-    assert abs((f2 - f1) - 100_000 * 32) <= 4 * 256    # 32 bytes of scratch per hit of capacity (+- alignment)
+    assert abs((f2 - f1) - 100_000 * 40) <= 4 * 256    # 40 bytes of scratch per hit of capacity (+- alignment)
     assert G.gart_view_host_arena_bytes(1000, 3, 640, 480, 8, 10_000, 100_000) > f1
     assert G.gart_view_host_arena_bytes(1000, 5, 640, 480, 8, 10_000, 100_000) == 0
