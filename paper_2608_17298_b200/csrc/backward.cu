@@ -82,10 +82,75 @@ __device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__
     return d;
 }
 
+// SH coefficients of a pair's Gaussian and the pair's dL/dsh accumulators, in registers.  For an even
+// number of coefficients both are kept as (k, k+1) pairs per channel, so that colour evaluation and
+// gradient accumulation issue packed two-wide FMAs (fma.rn.f32x2: half the issue slots).
+template <int K, bool PACKED = (K % 2 == 0)>
+struct ShRegs;
+
+template <int K>
+struct ShRegs<K, false> {
+    float sh[3 * K], acc[3 * K];
+    __device__ __forceinline__ void set(int e, float v) { sh[e] = v; acc[e] = 0.0f; }   // e = 3 k + channel
+    __device__ __forceinline__ float word(int e) const { return acc[e]; }
+    __device__ __forceinline__ void colour(const float* Y, float* c) const {
+        c[0] = 0.5f; c[1] = 0.5f; c[2] = 0.5f;
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            c[0] = fmaf(Y[k], sh[3 * k], c[0]);
+            c[1] = fmaf(Y[k], sh[3 * k + 1], c[1]);
+            c[2] = fmaf(Y[k], sh[3 * k + 2], c[2]);
+        }
+    }
+    __device__ __forceinline__ void accumulate(const float* Y, const float* w) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            acc[3 * k] = fmaf(Y[k], w[0], acc[3 * k]);
+            acc[3 * k + 1] = fmaf(Y[k], w[1], acc[3 * k + 1]);
+            acc[3 * k + 2] = fmaf(Y[k], w[2], acc[3 * k + 2]);
+        }
+    }
+};
+
+template <int K>
+struct ShRegs<K, true> {
+    float2 sh[3][K / 2], acc[3][K / 2];
+    __device__ __forceinline__ void set(int e, float v) {
+        const int k = e / 3, c = e % 3;
+        if (k & 1) { sh[c][k >> 1].y = v; acc[c][k >> 1].y = 0.0f; }
+        else { sh[c][k >> 1].x = v; acc[c][k >> 1].x = 0.0f; }
+    }
+    __device__ __forceinline__ float word(int e) const {
+        const int k = e / 3, c = e % 3;
+        return (k & 1) ? acc[c][k >> 1].y : acc[c][k >> 1].x;
+    }
+    __device__ __forceinline__ void colour(const float* Y, float* c) const {
+        float2 a0 = make_float2(0.5f, 0.0f), a1 = a0, a2 = a0;
+#pragma unroll
+        for (int i = 0; i < K / 2; ++i) {
+            const float2 y = make_float2(Y[2 * i], Y[2 * i + 1]);
+            a0 = __ffma2_rn(y, sh[0][i], a0);
+            a1 = __ffma2_rn(y, sh[1][i], a1);
+            a2 = __ffma2_rn(y, sh[2][i], a2);
+        }
+        c[0] = a0.x + a0.y; c[1] = a1.x + a1.y; c[2] = a2.x + a2.y;
+    }
+    __device__ __forceinline__ void accumulate(const float* Y, const float* w) {
+        const float2 w0 = make_float2(w[0], w[0]), w1 = make_float2(w[1], w[1]), w2 = make_float2(w[2], w[2]);
+#pragma unroll
+        for (int i = 0; i < K / 2; ++i) {
+            const float2 y = make_float2(Y[2 * i], Y[2 * i + 1]);
+            acc[0][i] = __ffma2_rn(y, w0, acc[0][i]);
+            acc[1][i] = __ffma2_rn(y, w1, acc[1][i]);
+            acc[2][i] = __ffma2_rn(y, w2, acc[2][i]);
+        }
+    }
+};
+
 // Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
-// acc[0..2] = v, acc[3..8] = Q (xx, yy, zz, xy, xz, yz), acc[9] = sum alpha dL/dalpha, acc[11..] = dL/dsh.
+// geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz), geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh.
 template <int TS, int K, int PW>
-__device__ __forceinline__ void bwd_hit(const PreRec& P, const float* shc, float* acc, const float* spix, int bx, int by, int p,
+__device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* geo, const float* spix, int bx, int by, int p,
                                         const float4 L) {
     const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
     const float* rec = spix + p * PW;
@@ -101,21 +166,26 @@ __device__ __forceinline__ void bwd_hit(const PreRec& P, const float* shc, float
         for (int kk = 0; kk < K; ++kk) Y[kk] = rec[kk];
     }
     const float3 g = make_float3(rec[K], rec[K + 1], rec[K + 2]);
-    const HitGrad<K> h = hit_grad<K>(Y, shc, g, L, r.alpha);
-#pragma unroll
-    for (int kk = 0; kk < K; ++kk) {
-        acc[11 + 3 * kk] = fmaf(Y[kk], h.wch[0], acc[11 + 3 * kk]);
-        acc[11 + 3 * kk + 1] = fmaf(Y[kk], h.wch[1], acc[11 + 3 * kk + 1]);
-        acc[11 + 3 * kk + 2] = fmaf(Y[kk], h.wch[2], acc[11 + 3 * kk + 2]);
-    }
-    const float ad = r.alpha * h.dalpha;
-    acc[9] += ad;
+    float c[3], w[3];
+    R.colour(Y, c);
+    const float T = L.w, Ta = T * r.alpha;
+    const float inv = fast_rcp(1.0f - r.alpha);
+    w[0] = c[0] > 0.0f ? Ta * g.x : 0.0f;
+    w[1] = c[1] > 0.0f ? Ta * g.y : 0.0f;
+    w[2] = c[2] > 0.0f ? Ta * g.z : 0.0f;
+    const float t0 = fmaf(T, fmaxf(c[0], 0.0f), -L.x * inv);
+    const float t1 = fmaf(T, fmaxf(c[1], 0.0f), -L.y * inv);
+    const float t2 = fmaf(T, fmaxf(c[2], 0.0f), -L.z * inv);
+    const float dalpha = fmaf(g.x, t0, fmaf(g.y, t1, g.z * t2));
+    R.accumulate(Y, w);
+    const float ad = r.alpha * dalpha;
+    geo[9] += ad;
     const float G = -0.5f * ad;
     const float3 xg = ray_xg(r);
     const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
-    acc[0] += gx; acc[1] += gy; acc[2] += gz;
-    acc[3] = fmaf(gx, xg.x, acc[3]); acc[4] = fmaf(gy, xg.y, acc[4]); acc[5] = fmaf(gz, xg.z, acc[5]);
-    acc[6] = fmaf(gx, xg.y, acc[6]); acc[7] = fmaf(gx, xg.z, acc[7]); acc[8] = fmaf(gy, xg.z, acc[8]);
+    geo[0] += gx; geo[1] += gy; geo[2] += gz;
+    geo[3] = fmaf(gx, xg.x, geo[3]); geo[4] = fmaf(gy, xg.y, geo[4]); geo[5] = fmaf(gz, xg.z, geo[5]);
+    geo[6] = fmaf(gx, xg.y, geo[6]); geo[7] = fmaf(gx, xg.z, geo[7]); geo[8] = fmaf(gy, xg.z, geo[8]);
 }
 
 template <int TS, int DEG>
@@ -214,34 +284,27 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
         // descriptor two groups ahead: needed only at the start of the next iteration
         const GroupDesc<MW> nxt2 = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
         PreRec P;
-        float shc[SW];
-        float acc[AW];
+        ShRegs<K> R;
+        float geo[11];
 #pragma unroll
-        for (int q = 0; q < AW; ++q) acc[q] = 0.0f;
+        for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
         if (STAGE_P) {
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(pbar_addr, pphase))) { fail(); return; }
             pphase ^= 1u;
-            if (cur.c != 0) {
-                P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);
+            P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);
 #pragma unroll
-                for (int q = 0; q < SW / 4; ++q) {
-                    const float4 t = my_par[5 + q];
-                    shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
-                }
+            for (int q = 0; q < SW / 4; ++q) {
+                const float4 t = my_par[5 + q];
+                R.set(4 * q, t.x); R.set(4 * q + 1, t.y); R.set(4 * q + 2, t.z); R.set(4 * q + 3, t.w);
             }
             __syncwarp();
             if (nxt.cmax != 0) issue_params(nxt);
-        } else if (cur.c != 0) {
-            P = load_pre(pre4, cur.gid);
-            const float* sp = sh + (size_t)cur.gid * SW;
+        } else {
+            const uint32_t gg = cur.c != 0 ? cur.gid : 0u;   // lanes without hits read a valid record they never use
+            P = load_pre(pre4, gg);
+            const float* sp = sh + (size_t)gg * SW;
 #pragma unroll
-            for (int q = 0; q < SW; ++q) shc[q] = __ldg(sp + q);
-        }
-        if (cur.c == 0) {
-            P = unpack_pre(make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 0), make_float4(0, 0, 0, 1),
-                           make_float4(0, 0, 0, 0));
-#pragma unroll
-            for (int q = 0; q < SW; ++q) shc[q] = 0.0f;
+            for (int q = 0; q < SW; ++q) R.set(q, __ldg(sp + q));
         }
         const int bx = x0 - P.ix, by = y0 - P.iy;
         const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
@@ -254,7 +317,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
             const float4* sl = my_stage + s * BWD_STAGE_F4 + lane;
             const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
             for (int e = k * BWD_CHUNK; e < e_end; ++e)
-                bwd_hit<TS, K, PW>(P, shc, acc, spix, bx, by, cur.pm.next(), sl[(e - k * BWD_CHUNK) * 32]);
+                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, cur.pm.next(), sl[(e - k * BWD_CHUNK) * 32]);
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
         }
@@ -262,7 +325,15 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
             // one vector atomic per 16 bytes of the Gaussian's record
             float4* gp = reinterpret_cast<float4*>(grad + (size_t)cur.gid * GART_GRAD_WORDS);
 #pragma unroll
-            for (int q = 0; q < AW / 4; ++q) atomicAdd(gp + q, make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]));
+            for (int q = 0; q < AW / 4; ++q) {
+                float v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int wd = 4 * q + i;
+                    v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? R.word(wd - 11) : 0.0f);
+                }
+                atomicAdd(gp + q, make_float4(v[0], v[1], v[2], v[3]));
+            }
         }
         if (nxt.cmax == 0) break;
         cur = nxt;

@@ -82,7 +82,7 @@ __device__ __forceinline__ HitGrad<K> hit_grad(const float* Y, const float* shc,
     }
     const float T = L.w;
     const float Ta = T * alpha;
-    const float inv = __frcp_rn(1.0f - alpha);
+    const float inv = fast_rcp(1.0f - alpha);
     HitGrad<K> h;
     h.wch[0] = c0 > 0.0f ? Ta * g.x : 0.0f;
     h.wch[1] = c1 > 0.0f ? Ta * g.y : 0.0f;

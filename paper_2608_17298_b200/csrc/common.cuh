@@ -97,6 +97,18 @@ __device__ __forceinline__ PreRec load_pre(const float4* __restrict__ pre4, uint
     return unpack_pre(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3), __ldg(p + 4));
 }
 
+// One-instruction reciprocal and 2^x of the special-function unit (about 1 and 2 ulp).
+__device__ __forceinline__ float fast_rcp(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 struct RayEval {
     float alpha;   // sigma * exp(-D^2 / 2)
     float tnum;    // m . d_g : same sign as t*
@@ -118,9 +130,9 @@ __device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy)
     r.cr.z = fmaf(ex, p.m.y, fmaf(-ey, p.m.x, p.k.z));
     const float a = fmaf(r.dg.x, r.dg.x, fmaf(r.dg.y, r.dg.y, r.dg.z * r.dg.z));
     const float cc = fmaf(r.cr.x, r.cr.x, fmaf(r.cr.y, r.cr.y, r.cr.z * r.cr.z));
-    r.inv_a = __frcp_rn(a);
+    r.inv_a = fast_rcp(a);
     const float D2 = cc * r.inv_a;
-    r.alpha = p.sigma * exp2f(-0.72134752044448170f * D2);
+    r.alpha = p.sigma * fast_exp2(-0.72134752044448170f * D2);
     r.tnum = fmaf(p.m.x, r.dg.x, fmaf(p.m.y, r.dg.y, p.m.z * r.dg.z));
     return r;
 }
@@ -160,15 +172,31 @@ struct PairMask {
     }
     // index (pixel of the tile) of the next set bit; call at most count() times
     __device__ __forceinline__ int next() {
-        if (N64 > 1) {
-            while (cur == 0ull) {
-                ++qi;
-                cur = qi == 1 ? w[1 % N64] : (qi == 2 ? w[2 % N64] : w[3 % N64]);
-            }
+        while (cur == 0ull) {
+            ++qi;
+            cur = qi == 1 ? w[1 % N64] : (qi == 2 ? w[2 % N64] : w[3 % N64]);
         }
         const int b = __ffsll((long long)cur) - 1;
         cur &= cur - 1ull;
         return qi * 64 + b;
+    }
+};
+
+// 64-pixel tiles: two 32-bit words walked with 32-bit operations.
+template <>
+struct PairMask<2> {
+    uint32_t lo, hi;
+    int base;
+    __device__ __forceinline__ void load(const uint32_t* __restrict__ pair_mask, uint32_t j, bool act) {
+        const uint2 t = act ? __ldg(reinterpret_cast<const uint2*>(pair_mask + (size_t)j * 2)) : make_uint2(0u, 0u);
+        lo = t.x; hi = t.y; base = 0;
+    }
+    __device__ __forceinline__ int count() const { return __popc(lo) + __popc(hi); }
+    __device__ __forceinline__ int next() {
+        if (lo == 0u) { lo = hi; hi = 0u; base = 32; }
+        const int b = __ffs((int)lo) - 1;
+        lo &= lo - 1u;
+        return base + b;
     }
 };
 
