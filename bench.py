@@ -48,10 +48,10 @@ def launches_per_step(n_tiles: int) -> int:
     while (1 << bits) < n_tiles:
         bits += 1
     passes = (bits + 7) // 8
-    bounds = 1
+    bounds = 1 + 2 * (1 + 3 + 1) + 1          # bounds kernel, two radix passes, record gather
     tile_map = 1 + 3 + 1 + 1 + passes * (1 + 3 + 1) + 1
     forward = 1 + 1 + 3 + 3 + 1 + 1 + 1
-    backward = 2
+    backward = 3                                # zero, pair kernel, per-Gaussian conversion
     return bounds + tile_map + forward + backward
 
 

@@ -93,7 +93,6 @@ enum {
 #define GART_ERRBIT_HITS 2u
 #define GART_ERRBIT_TIMEOUT 4u   /* a bounded wait on an asynchronous copy gave up (never expected) */
 
-#define GART_PRE_WORDS 20   /* fp32 words of the per-Gaussian ray-evaluation record */
 #define GART_GRAD_WORDS 64  /* stride of a gradient record: mean 3, scale 3, quat 4, opacity 1,
                                sh 3K (coefficient-major, channel-minor, as the input), zero padding */
 
@@ -107,19 +106,29 @@ int32_t gart_mask_words(int32_t tile_size);
  * dependent clamping radius alpha_c = sqrt(2 ln(sigma/alpha_min)) (Eq. 10), evaluated in
  * double precision, and the pre-computations of the ray evaluation (W = S^-1 R^T and o_g of
  * Eq. 5, expressed relative to a per-Gaussian reference pixel so that fp32 evaluation stays
- * well conditioned).
+ * well conditioned).  Gaussians with a non-empty rectangle are renumbered for the view: a stable
+ * sort on the tile of the rectangle's corner (x0, y0) gives each a slot 0..V-1 (V = counts[VISIBLE]);
+ * later steps read and update per-Gaussian data by slot, which keeps the accesses of neighbouring
+ * tiles close in memory.
  *   rect   [n,4] int32 out: inclusive pixel range x0,y0,x1,y1 of pixel centres inside the
  *                bound, clipped to the image; (0,0,-1,-1) if empty.
  *   cls    [n]   uint8 out: 0 culled (sigma <= alpha_min, or support entirely at depth <= near_z),
  *                1 in front of the near plane, 2 straddling it (rectangle = whole image unless
  *                the bounding sphere is outside a side plane of the frustum).
- *   pre    [n,GART_PRE_WORDS] fp32 out; contents are private to the library.
+ *   pre    [n * gart_pre_words(sh_degree)] fp32 out: per slot, the evaluation record followed by a copy
+ *                of the Gaussian's SH coefficients, and behind all records a copy of quaternion, scale
+ *                and opacity in slot order; contents are private to the library.
+ *   slot_of_gid [n] uint32 out: slot of every Gaussian, 0xffffffff if it has none.
+ *   gid_of_slot [n] uint32 out: the inverse (first V entries; 0xffffffff beyond).
  *   counts [GART_COUNTS_WORDS] uint32 out: zeroed, then VISIBLE and STRADDLE are set.
  * Errors: INVALID_ARG for null pointers, n < 0, sh_degree outside 0..3, tile size not 8/16,
- * non-positive image size.
+ * non-positive image size, unaligned workspace; WORKSPACE_TOO_SMALL.
  */
+int32_t gart_pre_words(int32_t sh_degree);
+size_t gart_bounds_workspace_bytes(int64_t n);
 gart_status gart_bounds(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,
-                        int32_t *rect, uint8_t *cls, float *pre, uint32_t *counts, void *stream);
+                        int32_t *rect, uint8_t *cls, float *pre, uint32_t *slot_of_gid, uint32_t *gid_of_slot,
+                        uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Step 2 -- reverse tile mapping (Sec. 4.3): every Gaussian emits one (tile, id) pair per tile
@@ -149,9 +158,10 @@ gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n
  *              when the tile's pairs are ordered by descending hit count (stable); the backward
  *              gives lane l of a warp the pair of rank 32 g + l, so a warp's lanes have (nearly)
  *              the same number of hits.
- *   rank_gid   [cap_pairs] uint32 out, rank_mask [cap_pairs, gart_mask_words] uint32 out: Gaussian id
- *              and hit mask of the pair at each rank position (copies of pair_gid / pair_mask in rank
- *              order, so that later kernels read them coalesced and without indirection).
+ *   rank_sid   [cap_pairs] uint32 out, rank_mask [cap_pairs, gart_mask_words] uint32 out: slot of the
+ *              Gaussian and hit mask of the pair at each rank position (slot_of_gid[pair_gid[.]] and
+ *              pair_mask[.] in rank order, so that later kernels read them coalesced and without
+ *              indirection).
  *   rank_gstart[cap_pairs] uint32 out, tile_lt_base [T+1] uint32 out: the e-th hit (in pixel order)
  *              of the pair of rank r of tile t lives at
  *                  lt[tile_lt_base[t] + rank_gstart[tile_off[t] + r] + 32 e + (r mod 32)].
@@ -171,9 +181,9 @@ gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n
  */
 size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
 gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
-                         const uint32_t *tile_off, const uint32_t *pair_gid, int64_t cap_pairs,
+                         const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off, const uint32_t *pair_gid, int64_t cap_pairs,
                          float *color, float *t_final, uint32_t *hit_count,
-                         uint32_t *pair_mask, uint32_t *pair_order, uint32_t *rank_gid, uint32_t *rank_mask,
+                         uint32_t *pair_mask, uint32_t *pair_order, uint32_t *rank_sid, uint32_t *rank_mask,
                          uint32_t *rank_gstart, uint32_t *tile_lt_base, float *lt, int64_t cap_hits,
                          uint32_t *ray_off, uint32_t *ray_gid, uint32_t *ray_slot, uint32_t *counts,
                          void *workspace, size_t workspace_bytes, void *stream);
@@ -182,7 +192,8 @@ gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const 
  * Step 4 -- primitive-centric backward (Sec. 4.4): one thread block per tile, one thread per
  * (tile, Gaussian) pair; the thread walks the pair's hit pixels, reads their LT entries (coalesced
  * across the warp thanks to the interleaved layout), accumulates in registers and performs one vector
- * atomic update of the Gaussian's gradient record per pair.  No per-pixel atomics.
+ * atomic update per pair of the accumulation record of the Gaussian's slot.  No per-pixel atomics.
+ * A per-Gaussian pass then converts the accumulated moments and writes the gradient records.
  *   dL_dcolor [H,W,3] in.
  *   grad [n,GART_GRAD_WORDS] out, fully overwritten: d mean, d scale, d quat, d opacity, d sh
  *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
@@ -191,11 +202,13 @@ gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const 
  * The main kernel uses up to 99 KB of dynamic shared memory per block (opt-in set by the call): LT blocks
  * and the Gaussians' records are streamed in with bulk asynchronous copies, one rank group ahead.
  */
+size_t gart_backward_workspace_bytes(int64_t n);
 gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
-                          const uint32_t *tile_off, const uint32_t *rank_gid, const uint32_t *rank_mask,
-                          const uint32_t *rank_gstart, const uint32_t *tile_lt_base,
+                          const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
+                          const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
+                          const uint32_t *tile_lt_base,
                           const float *lt, const float *dL_dcolor,
-                          float *grad, uint32_t *counts, void *stream);
+                          float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Pixel-centric baseline (Sec. 3.5): one thread per ray walks the ray's hits and issues one
@@ -203,7 +216,7 @@ gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const
  * up to summation order.
  */
 gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,
-                                 const float *pre, const uint32_t *ray_off, const uint32_t *ray_gid,
+                                 const float *pre, const uint32_t *slot_of_gid, const uint32_t *ray_off, const uint32_t *ray_gid,
                                  const uint32_t *ray_slot, const float *lt, const float *dL_dcolor,
                                  float *grad, const uint32_t *counts, void *stream);
 

@@ -8,7 +8,7 @@ struct HostArena {
     float *mean, *scale, *quat, *opacity, *sh, *pre, *color, *t_final, *lt, *dL_dC, *grad;
     int32_t* rect;
     uint8_t* cls;
-    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_gid, *rank_mask, *rank_gstart, *tile_lt_base, *hit_count, *ray_off, *ray_gid, *ray_slot;
+    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_sid, *rank_mask, *rank_gstart, *tile_lt_base, *slot_of_gid, *gid_of_slot, *hit_count, *ray_off, *ray_gid, *ray_slot;
     void* ws;
     size_t ws_bytes;
     size_t bytes;
@@ -25,19 +25,25 @@ static HostArena arena_layout(void* base, int64_t n, int K, int width, int heigh
     const int mw = ts * ts / 32;
     a.mean = (float*)take(nn * 12); a.scale = (float*)take(nn * 12); a.quat = (float*)take(nn * 16);
     a.opacity = (float*)take(nn * 4); a.sh = (float*)take(nn * 12 * K);
-    a.rect = (int32_t*)take(nn * 16); a.cls = (uint8_t*)take(nn); a.pre = (float*)take(nn * GART_PRE_WORDS * 4);
+    a.rect = (int32_t*)take(nn * 16); a.cls = (uint8_t*)take(nn); a.pre = (float*)take(nn * 4 * (size_t)(((20 + 3 * K + 3) & ~3) + 8));
+    a.slot_of_gid = (uint32_t*)take(nn * 4); a.gid_of_slot = (uint32_t*)take(nn * 4);
     a.counts = (uint32_t*)take(GART_COUNTS_WORDS * 4);
     a.tile_off = (uint32_t*)take((size_t)(T + 1) * 4); a.pair_gid = (uint32_t*)take(cp * 4);
-    a.pair_mask = (uint32_t*)take(cp * 4 * mw); a.pair_order = (uint32_t*)take(cp * 4); a.rank_gid = (uint32_t*)take(cp * 4);
+    a.pair_mask = (uint32_t*)take(cp * 4 * mw); a.pair_order = (uint32_t*)take(cp * 4); a.rank_sid = (uint32_t*)take(cp * 4);
     a.rank_mask = (uint32_t*)take(cp * 4 * mw); a.rank_gstart = (uint32_t*)take(cp * 4);
     a.tile_lt_base = (uint32_t*)take((size_t)(T + 1) * 4);
     a.color = (float*)take(hw * 12); a.t_final = (float*)take(hw * 4); a.hit_count = (uint32_t*)take(hw * 4);
     a.lt = (float*)take(ch * 16); a.ray_off = (uint32_t*)take((hw + 1) * 4);
     a.ray_gid = (uint32_t*)take(ch * 4); a.ray_slot = (uint32_t*)take(ch * 4);
     a.dL_dC = (float*)take(hw * 12); a.grad = (float*)take(nn * GART_GRAD_WORDS * 4);
+    const size_t w0 = gart_bounds_workspace_bytes(nn);
     const size_t w1 = gart_tile_map_workspace_bytes(nn, width, height, ts, cap_pairs);
     const size_t w2 = gart_forward_workspace_bytes(width, height, ts, cap_pairs, cap_hits);
-    a.ws_bytes = w1 > w2 ? w1 : w2;
+    const size_t w3 = gart_backward_workspace_bytes(nn);
+    a.ws_bytes = w0;
+    if (w1 > a.ws_bytes) a.ws_bytes = w1;
+    if (w2 > a.ws_bytes) a.ws_bytes = w2;
+    if (w3 > a.ws_bytes) a.ws_bytes = w3;
     a.ws = take(a.ws_bytes);
     a.bytes = off;
     return a;
@@ -88,14 +94,15 @@ extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussia
 #undef GART_H2D
     gart_gaussians gd = *gh;
     gd.mean = a.mean; gd.scale = a.scale; gd.quat = a.quat; gd.opacity = a.opacity; gd.sh = a.sh;
-    gart_status s = gart_bounds(cfg, &gd, cam, a.rect, a.cls, a.pre, a.counts, stream);
+    gart_status s = gart_bounds(cfg, &gd, cam, a.rect, a.cls, a.pre, a.slot_of_gid, a.gid_of_slot, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     s = gart_tile_map(cfg, a.rect, n, cam->width, cam->height, a.tile_off, a.pair_gid, cap_pairs, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
-    s = gart_forward(cfg, &gd, cam, a.pre, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count, a.pair_mask,
-                     a.pair_order, a.rank_gid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, a.ray_gid, a.ray_slot, a.counts, a.ws, a.ws_bytes, stream);
+    s = gart_forward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count, a.pair_mask,
+                     a.pair_order, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, a.ray_gid, a.ray_slot, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
-    s = gart_backward(cfg, &gd, cam, a.pre, a.tile_off, a.rank_gid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, a.dL_dC, a.grad, a.counts, stream);
+    s = gart_backward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, a.dL_dC,
+                      a.grad, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     if (cudaMemcpyAsync(color_host, a.color, (size_t)hw * 12, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GART_ERR_CUDA;
     if (n > 0 && cudaMemcpyAsync(grad_host, a.grad, (size_t)n * GART_GRAD_WORDS * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)

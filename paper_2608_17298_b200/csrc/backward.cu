@@ -6,10 +6,13 @@
 // (lt[base + 32 e + l]), i.e. the whole group's LT block is one contiguous range.  Each warp streams
 // these blocks into shared memory with bulk asynchronous copies (cp.async.bulk, completion on an
 // mbarrier), double buffered, so that tens of KB of LT data per SM are in flight while the warp
-// computes; lanes then read their entry with conflict-free 16-byte shared loads.  A thread
-// accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) of its pair in registers and adds them to the
-// Gaussian's gradient record with one vector atomic per 16 bytes -- no per-pixel atomics.  A
-// per-Gaussian pass then converts the record in place into d mean, d scale, d quat, d opacity.
+// computes; lanes then read their entry with conflict-free 16-byte shared loads.  The records of the
+// next group's Gaussians (evaluation record + SH coefficients, one contiguous piece per slot of the
+// view's order) arrive the same way.  A thread accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) of its
+// pair in registers and adds them to the accumulation record of the Gaussian's slot with one vector
+// atomic per 16 bytes -- no per-pixel atomics; slots are ordered by tile, so neighbouring tiles update
+// neighbouring memory.  A per-Gaussian pass then converts the moments into d mean, d scale, d quat,
+// d opacity and writes the caller's gradient records.
 #include "backward_common.cuh"
 
 namespace gart {
@@ -19,7 +22,7 @@ constexpr int BWD_THREADS = BWD_WARPS * 32;
 constexpr int BWD_CHUNK = 16;                          // LT entries per lane and per pipeline stage
 constexpr int BWD_STAGE_F4 = BWD_CHUNK * 32;           // float4 per stage (8 KB)
 constexpr int BWD_LT_SMEM = BWD_WARPS * 2 * BWD_STAGE_F4 * 16;
-constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + ((sw * 4) % 16 == 0 ? BWD_THREADS * (5 + sw / 4) * 16 : 0); }
+constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + BWD_THREADS * ((20 + sw + 3) / 4) * 16; }
 constexpr uint32_t BWD_WAIT_LIMIT = 1u << 22;          // bounded wait on a copy; then the error bit is set
 
 template <int K>
@@ -60,14 +63,14 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 template <int MW>
 struct GroupDesc {
     PairMask<MW> pm;
-    uint32_t gid;
+    uint32_t sid;      // slot of the pair's Gaussian in the view's order
     int c;             // hits of this lane's pair
     int cmax;          // hits of the group's first pair = the largest of the group
     uint32_t gstart;   // first LT entry of the group, relative to the tile's base
 };
 
 template <int MW>
-__device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__ rank_gid, const uint32_t* __restrict__ rank_mask,
+__device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
                                                     const uint32_t* __restrict__ rank_gstart, uint32_t begin, uint32_t n,
                                                     uint32_t r0, int lane) {
     GroupDesc<MW> d;
@@ -75,7 +78,7 @@ __device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__
     const uint32_t q = begin + r0 + lane;
     d.pm.load(rank_mask, act ? q : 0u, act);
     d.c = d.pm.count();
-    d.gid = act ? __ldg(rank_gid + q) : 0u;
+    d.sid = act ? __ldg(rank_sid + q) : 0u;
     const uint32_t s0 = act ? __ldg(rank_gstart + q) : 0u;
     d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
     d.gstart = __shfl_sync(0xffffffffu, s0, 0);
@@ -189,18 +192,17 @@ __device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* ge
 }
 
 template <int TS, int DEG>
-__global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
-                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_gid,
+__global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __restrict__ rec,
+                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                float* __restrict__ grad, uint32_t* __restrict__ counts) {
+                                                                float* __restrict__ gacc, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = PixLayout<K>::W;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
-    // Gaussian record + SH coefficients of a lane's pair, staged through shared memory one group ahead
-    // when their size allows bulk copies (multiples of 16 bytes: degrees 1 and 3)
-    constexpr bool STAGE_P = (SW * 4) % 16 == 0;
-    constexpr int PF4 = 5 + SW / 4;          // float4 per lane in the parameter buffer
+    // record (evaluation record + SH coefficients) of a lane's Gaussian, staged through shared memory one
+    // group ahead; PF4 float4 per lane
+    constexpr int PF4 = (20 + SW + 3) / 4;
     extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][PF4] parameters
     __shared__ __align__(16) float spix[NT * PW];
     __shared__ __align__(8) uint64_t bars[BWD_WARPS][3];
@@ -256,14 +258,9 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     };
     // copy the Gaussian records and SH coefficients of a group's pairs into the parameter buffer
     auto issue_params = [&](const GroupDesc<MW>& d) {
-        if (STAGE_P) {
-            const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
-            if (lane == 0) mbar_expect_tx(pbar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
-            if (d.c != 0) {
-                bulk_g2s(par_addr, pre4 + (size_t)d.gid * 5, 80u, pbar_addr);
-                bulk_g2s(par_addr + 80u, sh + (size_t)d.gid * SW, (uint32_t)(SW * 4), pbar_addr);
-            }
-        }
+        const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
+        if (lane == 0) mbar_expect_tx(pbar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
+        if (d.c != 0) bulk_g2s(par_addr, rec + (size_t)d.sid * PF4, (uint32_t)(PF4 * 16), pbar_addr);
     };
     auto fail = [&]() {
         // a copy never completed: report, give copies that may still be in flight a second bounded
@@ -275,37 +272,32 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     };
 
     uint32_t r0 = warp * 32;
-    GroupDesc<MW> cur = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0, lane);
+    GroupDesc<MW> cur = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0, lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
     issue(cur, 0, unit);
     issue_params(cur);
-    GroupDesc<MW> nxt = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0 + BWD_THREADS, lane);
+    GroupDesc<MW> nxt = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + BWD_THREADS, lane);
     while (true) {
         // descriptor two groups ahead: needed only at the start of the next iteration
-        const GroupDesc<MW> nxt2 = load_group<MW>(rank_gid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
+        const GroupDesc<MW> nxt2 = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
         PreRec P;
         ShRegs<K> R;
         float geo[11];
 #pragma unroll
         for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
-        if (STAGE_P) {
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(pbar_addr, pphase))) { fail(); return; }
-            pphase ^= 1u;
-            P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(pbar_addr, pphase))) { fail(); return; }
+        pphase ^= 1u;
+        P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale data for lanes without hits: never used)
 #pragma unroll
-            for (int q = 0; q < SW / 4; ++q) {
-                const float4 t = my_par[5 + q];
-                R.set(4 * q, t.x); R.set(4 * q + 1, t.y); R.set(4 * q + 2, t.z); R.set(4 * q + 3, t.w);
-            }
-            __syncwarp();
-            if (nxt.cmax != 0) issue_params(nxt);
-        } else {
-            const uint32_t gg = cur.c != 0 ? cur.gid : 0u;   // lanes without hits read a valid record they never use
-            P = load_pre(pre4, gg);
-            const float* sp = sh + (size_t)gg * SW;
-#pragma unroll
-            for (int q = 0; q < SW; ++q) R.set(q, __ldg(sp + q));
+        for (int q = 0; q < (SW + 3) / 4; ++q) {
+            const float4 t = my_par[5 + q];
+            R.set(4 * q, t.x);
+            if (4 * q + 1 < SW) R.set(4 * q + 1, t.y);
+            if (4 * q + 2 < SW) R.set(4 * q + 2, t.z);
+            if (4 * q + 3 < SW) R.set(4 * q + 3, t.w);
         }
+        __syncwarp();
+        if (nxt.cmax != 0) issue_params(nxt);
         const int bx = x0 - P.ix, by = y0 - P.iy;
         const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
         for (int k = 0; k < nchunks; ++k) {
@@ -323,7 +315,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
         }
         if (cur.c != 0) {
             // one vector atomic per 16 bytes of the Gaussian's record
-            float4* gp = reinterpret_cast<float4*>(grad + (size_t)cur.gid * GART_GRAD_WORDS);
+            float4* gp = reinterpret_cast<float4*>(gacc + (size_t)cur.sid * GART_GRAD_WORDS);
 #pragma unroll
             for (int q = 0; q < AW / 4; ++q) {
                 float v[4];
@@ -342,51 +334,67 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     }
 }
 
-// In-place conversion of the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity.
-__global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, const float* __restrict__ scale, const float* __restrict__ quat,
-                                                           const float* __restrict__ opacity, float* __restrict__ grad,
+// Zero the accumulation records of the view's slots (their number lives on the device).
+__global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc4, const uint32_t* __restrict__ counts) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4)) gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// Two roles by block range, 16 lanes per record.  Blocks [0, slot_blocks): per slot, in slot order,
+// convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity, copy the SH
+// gradient and write the Gaussian's whole gradient record (reads are sequential, the 256-byte writes
+// scattered).  The remaining blocks: per Gaussian, zero the record if it has no slot.
+__global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, int64_t slot_blocks, const float4* __restrict__ qs,
+                                                           const uint32_t* __restrict__ slot_of_gid, const uint32_t* __restrict__ gid_of_slot,
+                                                           const float4* __restrict__ gacc4, float4* __restrict__ grad4,
                                                            const uint32_t* __restrict__ counts) {
     if (counts[GART_CNT_ERROR]) return;
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    float4* gp = reinterpret_cast<float4*>(grad + (size_t)i * GART_GRAD_WORDS);
-    const float4 a = gp[0], b = gp[1], c = gp[2];
-    const float v[3] = {a.x, a.y, a.z};
-    const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
-    bool nz = c.y != 0.0f;
-#pragma unroll
-    for (int k = 0; k < 3; ++k) nz = nz || v[k] != 0.0f;
-#pragma unroll
-    for (int k = 0; k < 6; ++k) nz = nz || Q[k] != 0.0f;
-    if (!nz) return;
-    const float q[4] = {quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]};
-    const float s[3] = {scale[3 * i], scale[3 * i + 1], scale[3 * i + 2]};
-    const GeoGrad o = moments_to_grads(v, Q, q, s);
-    gp[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
-    gp[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
-    gp[2] = make_float4(o.dq[2], o.dq[3], c.y / opacity[i], c.w);
+    const int l = threadIdx.x & 15;
+    if ((int64_t)blockIdx.x < slot_blocks) {
+        const int64_t sid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;
+        if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+        const float4* gp = gacc4 + (size_t)sid * (GART_GRAD_WORDS / 4);
+        float4 out = gp[l];
+        if (l < 3) {
+            const float4 a = gp[0], b = gp[1], c = gp[2];
+            const float v[3] = {a.x, a.y, a.z};
+            const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
+            const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
+            const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+            const float sc[3] = {s4.x, s4.y, s4.z};
+            const GeoGrad o = moments_to_grads(v, Q, q, sc);
+            if (l == 0) out = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
+            else if (l == 1) out = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
+            else out = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
+        }
+        grad4[(size_t)gid_of_slot[sid] * (GART_GRAD_WORDS / 4) + l] = out;
+    } else {
+        const int64_t i = (((int64_t)blockIdx.x - slot_blocks) * blockDim.x + threadIdx.x) >> 4;
+        if (i >= n) return;
+        if (slot_of_gid[i] == 0xffffffffu) grad4[(size_t)i * (GART_GRAD_WORDS / 4) + l] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
 }
 
 template <int TS, int DEG>
-static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
-                                    const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
+                                    const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                     const uint32_t* tile_lt_base, const float4* lt,
-                                    const float* dL_dC, const CamF& cam, float* grad, uint32_t* counts) {
+                                    const float* dL_dC, const CamF& cam, float* gacc, uint32_t* counts) {
     auto kern = bwd_pairs_kernel<TS, DEG>;
     constexpr int smem = bwd_dyn_smem(3 * (DEG + 1) * (DEG + 1));
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
-    kern<<<T, BWD_THREADS, smem, st>>>(pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, grad, counts);
+    kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
 
 template <int TS>
-static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
-                                const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
+                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                 const uint32_t* tile_lt_base, const float4* lt,
-                                const float* dL_dC, const CamF& cam, float* grad, uint32_t* counts) {
+                                const float* dL_dC, const CamF& cam, float* gacc, uint32_t* counts) {
 #define GART_PAIRS(D) \
-    return launch_pairs_deg<TS, D>(T, st, pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, grad, counts)
+    return launch_pairs_deg<TS, D>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts)
     switch (deg) {
         case 0: GART_PAIRS(0);
         case 1: GART_PAIRS(1);
@@ -398,28 +406,40 @@ static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* p
 
 }  // namespace gart
 
+extern "C" size_t gart_backward_workspace_bytes(int64_t n) {
+    return gart::align256((size_t)(n > 0 ? n : 1) * GART_GRAD_WORDS * sizeof(float));
+}
+
 extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
-                                     const uint32_t* tile_off, const uint32_t* rank_gid, const uint32_t* rank_mask,
-                                     const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
+                                     const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
                                      const float* lt, const float* dL_dcolor,
-                                     float* grad, uint32_t* counts, void* stream) {
+                                     float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace gart;
     if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !g->scale || !g->quat || !g->opacity || !g->sh) return GART_ERR_INVALID_ARG;
+    if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
+    if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(grad, 0, (size_t)g->n * GART_GRAD_WORDS * sizeof(float), st) != cudaSuccess) return GART_ERR_CUDA;
+    float* gacc = reinterpret_cast<float*>(workspace);
+    const int64_t f4 = g->n * (GART_GRAD_WORDS / 4);
+    bwd_zero_kernel<<<(unsigned)ceil_div(f4, 256), 256, 0, st>>>(reinterpret_cast<float4*>(gacc), counts);
+    GART_LAUNCH_CHECK();
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int T = cf.tiles_x * cf.tiles_y;
-    const float4* pre4 = reinterpret_cast<const float4*>(pre);
+    const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
     gart_status s;
-    if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, grad, counts);
-    else s = launch_pairs<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, grad, counts);
+    if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
+    else s = launch_pairs<16>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
     if (s != GART_OK) return s;
-    bwd_finalize_kernel<<<(unsigned)ceil_div(g->n, 256), 256, 0, st>>>(g->n, g->scale, g->quat, g->opacity, grad, counts);
+    const int64_t fblocks = ceil_div(g->n * 16, 256);
+    const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
+    bwd_finalize_kernel<<<(unsigned)(2 * fblocks), 256, 0, st>>>(g->n, fblocks, qs, slot_of_gid, gid_of_slot,
+                                                                 reinterpret_cast<const float4*>(gacc), reinterpret_cast<float4*>(grad), counts);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

@@ -8,13 +8,13 @@ namespace gart {
 
 // -------------------------------------------------------------------------------- pixel-centric baseline
 template <int DEG>
-__global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
+__global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ slot_of_gid,
                                                          const float* __restrict__ scale, const float* __restrict__ quat,
                                                          const float* __restrict__ opacity, const uint32_t* __restrict__ ray_off,
                                                          const uint32_t* __restrict__ ray_gid, const uint32_t* __restrict__ ray_slot,
                                                          const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
                                                          float* __restrict__ grad, const uint32_t* __restrict__ counts) {
-    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K;
+    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (ray >= (int64_t)cam.width * cam.height) return;
@@ -27,11 +27,11 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
     for (uint32_t h = b; h < e; ++h) {
         const uint32_t gid = ray_gid[h];
         const float4 L = lt[ray_slot[h]];
-        const PreRec P = load_pre(pre4, gid);
+        const float4* rp = rec + (size_t)__ldg(slot_of_gid + gid) * RS4;
+        const PreRec P = load_pre(rp);
         const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
         float shc[SW];
-#pragma unroll
-        for (int q = 0; q < SW; ++q) shc[q] = __ldg(sh + (size_t)gid * SW + q);
+        load_sh<SW>(rp, shc);
         const HitGrad<K> hg = hit_grad<K>(Y, shc, g, L, r.alpha);
         const float ad = r.alpha * hg.dalpha;
         const float G = -0.5f * ad;
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
 }  // namespace gart
 
 extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam,
-                                            const float* pre, const uint32_t* ray_off, const uint32_t* ray_gid,
+                                            const float* pre, const uint32_t* slot_of_gid, const uint32_t* ray_off, const uint32_t* ray_gid,
                                             const uint32_t* ray_slot, const float* lt, const float* dL_dcolor,
                                             float* grad, const uint32_t* counts, void* stream) {
     using namespace gart;
@@ -66,16 +66,16 @@ extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_g
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !g->scale || !g->quat || !g->opacity || !g->sh) return GART_ERR_INVALID_ARG;
+    if (!grad || !pre || !slot_of_gid || !g->scale || !g->quat || !g->opacity) return GART_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(grad, 0, (size_t)g->n * GART_GRAD_WORDS * sizeof(float), st) != cudaSuccess) return GART_ERR_CUDA;
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int64_t n_rays = (int64_t)cam->width * cam->height;
-    const float4* pre4 = reinterpret_cast<const float4*>(pre);
+    const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
     const unsigned blocks = (unsigned)ceil_div(n_rays, 128);
 #define GART_ATOMIC(D) \
-    bwd_atomic_kernel<D><<<blocks, 128, 0, st>>>(pre4, g->sh, g->scale, g->quat, g->opacity, ray_off, ray_gid, ray_slot, lt4, dL_dcolor, cf, grad, counts)
+    bwd_atomic_kernel<D><<<blocks, 128, 0, st>>>(rec, slot_of_gid, g->scale, g->quat, g->opacity, ray_off, ray_gid, ray_slot, lt4, dL_dcolor, cf, grad, counts)
     switch (g->sh_degree) {
         case 0: GART_ATOMIC(0); break;
         case 1: GART_ATOMIC(1); break;

@@ -2,7 +2,14 @@
 // opacity-dependent clamping radius (Eq. 10) and the ray-evaluation record (Eq. 5), one thread
 // per Gaussian, in double precision: the rectangle edges are integer decisions (ceil / floor of
 // p -/+ h) and the pass is O(n), so fp64 costs nothing that matters and keeps the edges exact.
-#include "common.cuh"
+//
+// The Gaussians that reach the image are then renumbered for this view: a stable radix sort on the
+// tile of the rectangle's first corner gives every visible Gaussian a "slot", and its evaluation
+// record and SH coefficients are gathered into one contiguous record per slot.  Tiles are processed
+// in tile order, so the per-pair reads of these records and the per-pair gradient updates of the
+// backward touch memory that neighbouring tiles also touch, instead of random 200-byte pieces of
+// gigabyte-sized arrays.
+#include "radix.cuh"
 
 namespace gart {
 
@@ -21,8 +28,10 @@ __device__ __forceinline__ void quat_to_rot(const double w, const double x, cons
 __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
                                                      const float* __restrict__ quat, const float* __restrict__ opacity,
                                                      CamD cam, double alpha_min, double near_z,
+                                                     int ts, int tiles_x, uint32_t key_none,
                                                      int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
-                                                     float4* __restrict__ pre4, uint32_t* __restrict__ counts) {
+                                                     float4* __restrict__ pre4, uint32_t* __restrict__ keys,
+                                                     uint32_t* __restrict__ vals, uint32_t* __restrict__ counts) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int vis = 0, straddle = 0;
     if (i < n) {
@@ -125,12 +134,76 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
         cls[i] = (uint8_t)c;
         float4* p = pre4 + (size_t)i * 5;
         p[0] = q0; p[1] = q1; p[2] = q2; p[3] = q3; p[4] = q4;
+        keys[i] = vis ? (uint32_t)((y0 / ts) * tiles_x + x0 / ts) : key_none;
+        vals[i] = (uint32_t)i;
     }
     const unsigned bv = __ballot_sync(0xffffffffu, vis), bs = __ballot_sync(0xffffffffu, straddle);
     if ((threadIdx.x & 31) == 0) {
         if (bv) atomicAdd(&counts[GART_CNT_VISIBLE], __popc(bv));
         if (bs) atomicAdd(&counts[GART_CNT_STRADDLE], __popc(bs));
     }
+}
+
+// One thread per 16 bytes of a slot's record: 5 float4 of the evaluation record, then the SH
+// coefficients (zero padded to the record stride).  Also fills the two maps between ids and slots.
+__global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4, int sw, uint32_t key_none,
+                                                             const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
+                                                             const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
+                                                             const float* __restrict__ quat, const float* __restrict__ scale,
+                                                             const float* __restrict__ opacity,
+                                                             float4* __restrict__ rec, float4* __restrict__ qs,
+                                                             uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t slot = t / rs4;
+    const int q = (int)(t - slot * rs4);
+    if (slot >= n) return;
+    const uint32_t gid = vals_sorted[slot];
+    const bool vis = keys_sorted[slot] != key_none;
+    if (q == 0) {
+        slot_of_gid[gid] = vis ? (uint32_t)slot : 0xffffffffu;
+        gid_of_slot[slot] = vis ? gid : 0xffffffffu;
+    }
+    if (!vis) return;
+    if (q == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
+        qs[2 * slot] = make_float4(quat[4 * (size_t)gid], quat[4 * (size_t)gid + 1], quat[4 * (size_t)gid + 2], quat[4 * (size_t)gid + 3]);
+        qs[2 * slot + 1] = make_float4(scale[3 * (size_t)gid], scale[3 * (size_t)gid + 1], scale[3 * (size_t)gid + 2], opacity[gid]);
+    }
+    float4 v;
+    if (q < 5) {
+        v = pre_tmp[(size_t)gid * 5 + q];
+    } else {
+        const int e = (q - 5) * 4;
+        const float* sp = sh + (size_t)gid * sw;
+        v.x = e < sw ? sp[e] : 0.0f;
+        v.y = e + 1 < sw ? sp[e + 1] : 0.0f;
+        v.z = e + 2 < sw ? sp[e + 2] : 0.0f;
+        v.w = e + 3 < sw ? sp[e + 3] : 0.0f;
+    }
+    rec[(size_t)slot * rs4 + q] = v;
+}
+
+struct BoundsWs {
+    float4* pre_tmp;
+    uint32_t *keys0, *keys1, *vals0, *vals1, *table;
+    uint64_t* total64;
+    void* scan_ws;
+    size_t bytes;
+};
+
+static BoundsWs bounds_layout(void* base, int64_t n) {
+    BoundsWs w;
+    char* p = (char*)base;
+    size_t off = 0;
+    auto take = [&](size_t b) { void* r = p ? (void*)(p + off) : nullptr; off += align256(b); return r; };
+    const int64_t nn = n > 0 ? n : 1;
+    w.total64 = (uint64_t*)take(256);
+    w.pre_tmp = (float4*)take((size_t)nn * 80);
+    w.keys0 = (uint32_t*)take((size_t)nn * 4); w.keys1 = (uint32_t*)take((size_t)nn * 4);
+    w.vals0 = (uint32_t*)take((size_t)nn * 4); w.vals1 = (uint32_t*)take((size_t)nn * 4);
+    w.table = (uint32_t*)take(radix_table_bytes(nn));
+    w.scan_ws = take(radix_scan_bytes(nn));
+    w.bytes = off;
+    return w;
 }
 
 }  // namespace gart
@@ -148,25 +221,55 @@ extern "C" const char* gart_status_string(gart_status s) {
 
 extern "C" int32_t gart_mask_words(int32_t tile_size) { return tile_size * tile_size / 32; }
 
+// Per Gaussian: the slot record (evaluation record + SH coefficients, padded to 16 bytes) and, in a
+// second block behind all records, 8 words (quaternion, scale, opacity) in slot order.
+extern "C" int32_t gart_pre_words(int32_t sh_degree) { return 4 * gart::rec_f4(sh_degree) + 8; }
+
+extern "C" size_t gart_bounds_workspace_bytes(int64_t n) { return gart::bounds_layout(nullptr, n).bytes; }
+
 extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam,
-                                   int32_t* rect, uint8_t* cls, float* pre, uint32_t* counts, void* stream) {
+                                   int32_t* rect, uint8_t* cls, float* pre, uint32_t* slot_of_gid, uint32_t* gid_of_slot,
+                                   uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace gart;
     if (!cfg || !g || !cam || !counts) return GART_ERR_INVALID_ARG;
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
+    if (g->n < 0 || g->n > 0xfffffff0ll || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0 || !(cam->fx > 0.0) || !(cam->fy > 0.0)) return GART_ERR_INVALID_ARG;
-    if (g->n > 0 && (!g->mean || !g->scale || !g->quat || !g->opacity || !rect || !cls || !pre)) return GART_ERR_INVALID_ARG;
+    if (g->n > 0 && (!g->mean || !g->scale || !g->quat || !g->opacity || !g->sh || !rect || !cls || !pre || !slot_of_gid || !gid_of_slot))
+        return GART_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(counts, 0, GART_COUNTS_WORDS * sizeof(uint32_t), st) != cudaSuccess) return GART_ERR_CUDA;
     if (g->n == 0) return GART_OK;
+    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
+    BoundsWs w = bounds_layout(workspace, g->n);
+    if (w.bytes > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     gart::CamD c;
     c.width = cam->width; c.height = cam->height;
     c.fx = cam->fx; c.fy = cam->fy; c.cx = cam->cx; c.cy = cam->cy;
     for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
+    const int ts = cfg->tile_size;
+    const int tiles_x = (cam->width + ts - 1) / ts, tiles_y = (cam->height + ts - 1) / ts;
+    const uint32_t key_none = (uint32_t)(tiles_x * tiles_y);   // sorts after every tile
+    int bits = 1;
+    while ((1u << bits) <= key_none) ++bits;
+    uint32_t* const kbuf[2] = {w.keys0, w.keys1};
+    uint32_t* const vbuf[2] = {w.vals0, w.vals1};
+    const int cur = radix_passes(bits) & 1;   // after the passes the sorted arrays are at index 0
     const int threads = 128;
-    const int64_t blocks = gart::ceil_div(g->n, threads);
-    gart::bounds_kernel<<<(unsigned)blocks, threads, 0, st>>>(g->n, g->mean, g->scale, g->quat, g->opacity, c,
-                                                             (double)cfg->alpha_min, (double)cfg->near_z, rect, cls,
-                                                             reinterpret_cast<float4*>(pre), counts);
+    const int64_t blocks = ceil_div(g->n, threads);
+    bounds_kernel<<<(unsigned)blocks, threads, 0, st>>>(g->n, g->mean, g->scale, g->quat, g->opacity, c,
+                                                       (double)cfg->alpha_min, (double)cfg->near_z, ts, tiles_x, key_none, rect, cls,
+                                                       w.pre_tmp, kbuf[cur], vbuf[cur], counts);
+    GART_LAUNCH_CHECK();
+    gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);
+    if (s != GART_OK) return s;
+    const int K = (g->sh_degree + 1) * (g->sh_degree + 1);
+    const int rs4 = rec_f4(g->sh_degree);
+    const int64_t gthreads = g->n * rs4;
+    gather_records_kernel<<<(unsigned)ceil_div(gthreads, 256), 256, 0, st>>>(g->n, rs4, 3 * K, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh,
+                                                                            g->quat, g->scale, g->opacity, reinterpret_cast<float4*>(pre),
+                                                                            reinterpret_cast<float4*>(pre) + (size_t)g->n * rs4, slot_of_gid,
+                                                                            gid_of_slot);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

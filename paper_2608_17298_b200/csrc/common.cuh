@@ -54,7 +54,7 @@ __device__ __forceinline__ float3 pixel_dir(const CamF& c, int x, int y) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Per-Gaussian ray-evaluation record: GART_PRE_WORDS = 20 floats = 5 float4.
+// Per-Gaussian ray-evaluation record: 20 floats = 5 float4 (the head of a slot's record).
 //
 // With W = S^-1 R^T (Eq. 5), the camera rotation Rc and origin o, and the un-normalised ray
 // direction d_c = ((x+.5-cx)/fx, (y+.5-cy)/fy, 1) in camera space:
@@ -92,9 +92,25 @@ __device__ __forceinline__ PreRec unpack_pre(const float4& a, const float4& b, c
     return p;
 }
 
-__device__ __forceinline__ PreRec load_pre(const float4* __restrict__ pre4, uint32_t gid) {
-    const float4* p = pre4 + (size_t)gid * 5;
-    return unpack_pre(__ldg(p), __ldg(p + 1), __ldg(p + 2), __ldg(p + 3), __ldg(p + 4));
+// A slot's record: 5 float4 of PreRec, then the 3K SH coefficients (coefficient-major, channel-minor),
+// zero padded to a multiple of 4 floats.  rs4 = float4 per record.
+static inline int rec_f4(int sh_degree) { return ((20 + 3 * (sh_degree + 1) * (sh_degree + 1) + 3) & ~3) / 4; }
+
+__device__ __forceinline__ PreRec load_pre(const float4* __restrict__ rec) {
+    return unpack_pre(__ldg(rec), __ldg(rec + 1), __ldg(rec + 2), __ldg(rec + 3), __ldg(rec + 4));
+}
+
+// SH coefficients of a record into registers, by 16-byte loads (the padding is loaded and dropped).
+template <int SW>
+__device__ __forceinline__ void load_sh(const float4* __restrict__ rec, float* shc) {
+#pragma unroll
+    for (int q = 0; q < (SW + 3) / 4; ++q) {
+        const float4 t = __ldg(rec + 5 + q);
+        shc[4 * q] = t.x;
+        if (4 * q + 1 < SW) shc[4 * q + 1] = t.y;
+        if (4 * q + 2 < SW) shc[4 * q + 2] = t.z;
+        if (4 * q + 3 < SW) shc[4 * q + 3] = t.w;
+    }
 }
 
 // One-instruction reciprocal and 2^x of the special-function unit (about 1 and 2 ulp).

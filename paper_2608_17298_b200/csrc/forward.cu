@@ -8,7 +8,7 @@
 //                  Gaussian of the tile list (records broadcast from shared memory); a warp
 //                  ballot yields the pair's hit mask; pixels count their hits.
 //   2. tile_sort   warp per tile: stable counting sort of the tile's pairs by descending hit
-//                  count -> pair_order, with copies of id and mask in rank order (rank_gid,
+//                  count -> pair_order, with copies of slot id and mask in rank order (rank_sid,
 //                  rank_mask: read coalesced later); groups of 32 consecutive ranks share an LT
 //                  block in which entry e of lane l sits at 32 e + l -> rank_gstart; per-tile LT size.
 //      scans       LT size per tile -> tile_lt_base; hits per ray -> ray_off.
@@ -25,7 +25,8 @@ namespace gart {
 
 // ------------------------------------------------------------------------------------------ phase 1
 template <int TS>
-__global__ void __launch_bounds__(TS * TS) fwd_mask_kernel(const float4* __restrict__ pre4, const uint32_t* __restrict__ tile_off,
+__global__ void __launch_bounds__(TS * TS) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
+                                                           const uint32_t* __restrict__ tile_off,
                                                            const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
                                                            uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ hit_count,
                                                            uint32_t* __restrict__ counts) {
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(TS * TS) fwd_mask_kernel(const float4* __restr
         const int nb = min((uint32_t)CH, end - base);
         for (int i = p; i < nb * 5; i += NT) {
             const int pair = i / 5, q = i - pair * 5;
-            sp[i] = __ldg(pre4 + (size_t)__ldg(pair_gid + base + pair) * 5 + q);
+            sp[i] = __ldg(rec + (size_t)__ldg(slot_of_gid + __ldg(pair_gid + base + pair)) * rs4 + q);
         }
         __syncthreads();
         for (int j = 0; j < nb; ++j) {
@@ -82,8 +83,9 @@ __device__ __forceinline__ uint32_t mask_popc(const uint32_t* __restrict__ pair_
 
 template <int TS>
 __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_gid,
+                                                                    const uint32_t* __restrict__ slot_of_gid,
                                                                     const uint32_t* __restrict__ pair_mask, int T, uint32_t* pair_order,
-                                                                    uint32_t* __restrict__ rank_gid, uint32_t* __restrict__ rank_mask,
+                                                                    uint32_t* __restrict__ rank_sid, uint32_t* __restrict__ rank_mask,
                                                                     uint32_t* __restrict__ rank_gstart,
                                                                     uint32_t* __restrict__ tile_slots, const uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, NB = NT + 1;
@@ -134,7 +136,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
                 rank_mask[q * MW + m] = wv;
                 c += __popc(wv);
             }
-            rank_gid[q] = __ldg(pair_gid + j);
+            rank_sid[q] = __ldg(slot_of_gid + __ldg(pair_gid + j));
             rank_gstart[q] = run;
         }
         const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
@@ -167,13 +169,13 @@ __global__ void hits_total_kernel(const uint64_t* total_slots, const uint64_t* t
 constexpr int EVAL_THREADS = 128;
 
 template <int TS, int DEG>
-__global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ pre4, const float* __restrict__ sh,
-                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_gid,
+__global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
+                                                                const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
                                                                 const uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3;
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3, RS4 = (20 + SW + 3) / 4;
     __shared__ __align__(16) float spix[NT * PW];
     __shared__ uint32_t sro[NT];
     __shared__ uint32_t scur[NT];
@@ -203,22 +205,12 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         const int c = pm.count();
         if (__ballot_sync(0xffffffffu, c != 0) == 0u) break;   // ranks descend in hit count: nothing left in this tile
         if (c == 0) continue;
-        const uint32_t gid = __ldg(rank_gid + q);
-        const PreRec P = load_pre(pre4, gid);
+        const uint32_t sid = __ldg(rank_sid + q);
+        const uint32_t gid = __ldg(gid_of_slot + sid);
+        const float4* rp = rec + (size_t)sid * RS4;
+        const PreRec P = load_pre(rp);
         float shc[SW];
-        {
-            const float* sp = sh + (size_t)gid * SW;
-            if (SW % 4 == 0) {
-#pragma unroll
-                for (int q = 0; q < SW / 4; ++q) {
-                    const float4 t = __ldg(reinterpret_cast<const float4*>(sp) + q);
-                    shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
-                }
-            } else {
-#pragma unroll
-                for (int q = 0; q < SW; ++q) shc[q] = __ldg(sp + q);
-            }
-        }
+        load_sh<SW>(rp, shc);
         uint32_t slot = lt_base + __ldg(rank_gstart + q) + lane;
         const int bx = x0 - P.ix, by = y0 - P.iy;
         for (int e = 0; e < c; ++e) {
@@ -411,12 +403,12 @@ static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_h
 }
 
 template <int TS>
-static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* pre4, const float* sh, const uint32_t* tile_off,
-                               const uint32_t* rank_gid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
+static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                               const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                const uint32_t* tile_lt_base, const uint32_t* ray_off,
                                const CamF& cam, const ForwardWs& w, const uint32_t* counts) {
 #define GART_EVAL(D)                                                                                                      \
-    fwd_eval_kernel<TS, D><<<T, EVAL_THREADS, 0, st>>>(pre4, sh, tile_off, rank_gid, rank_mask, rank_gstart,             \
+    fwd_eval_kernel<TS, D><<<T, EVAL_THREADS, 0, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart,    \
                                                        tile_lt_base, ray_off, cam, w.recs, counts)
     switch (deg) {
         case 0: GART_EVAL(0); break;
@@ -439,9 +431,9 @@ extern "C" size_t gart_forward_workspace_bytes(int32_t width, int32_t height, in
 }
 
 extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
-                                    const uint32_t* tile_off, const uint32_t* pair_gid, int64_t cap_pairs,
+                                    const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off, const uint32_t* pair_gid, int64_t cap_pairs,
                                     float* color, float* t_final, uint32_t* hit_count,
-                                    uint32_t* pair_mask, uint32_t* pair_order, uint32_t* rank_gid, uint32_t* rank_mask,
+                                    uint32_t* pair_mask, uint32_t* pair_order, uint32_t* rank_sid, uint32_t* rank_mask,
                                     uint32_t* rank_gstart, uint32_t* tile_lt_base,
                                     float* lt, int64_t cap_hits,
                                     uint32_t* ray_off, uint32_t* ray_gid, uint32_t* ray_slot, uint32_t* counts,
@@ -452,7 +444,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
-    if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_gid || !rank_mask || !rank_gstart || !pre || !g->sh)) return GART_ERR_INVALID_ARG;
+    if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_sid || !rank_mask || !rank_gstart || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0 && (!lt || !ray_gid || !ray_slot)) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     const int ts = cfg->tile_size;
@@ -462,15 +454,16 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     ForwardWs w = forward_layout(workspace, n_rays, T, cap_hits);
     if (w.bytes > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
-    const float4* pre4 = reinterpret_cast<const float4*>(pre);
+    const float4* rec = reinterpret_cast<const float4*>(pre);
+    const int rs4 = rec_f4(g->sh_degree);
 
-    if (ts == 8) fwd_mask_kernel<8><<<T, 64, 0, st>>>(pre4, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, 256, 0, st>>>(pre4, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
+    if (ts == 8) fwd_mask_kernel<8><<<T, 64, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, 256, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
-    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, pair_mask, T, pair_order, rank_gid, rank_mask, rank_gstart, w.tile_slots, counts);
-    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, pair_mask, T, pair_order, rank_gid, rank_mask, rank_gstart, w.tile_slots, counts);
+    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, slot_of_gid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
+    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, slot_of_gid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
     GART_LAUNCH_CHECK();
 
     TileSlotsF tf{w.tile_slots};
@@ -482,8 +475,8 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     hits_total_kernel<<<1, 1, 0, st>>>(w.total_slots, w.total_hits, cap_hits, counts);
     GART_LAUNCH_CHECK();
 
-    if (ts == 8) s = launch_eval<8>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
-    else s = launch_eval<16>(g->sh_degree, T, st, pre4, g->sh, tile_off, rank_gid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
+    if (ts == 8) s = launch_eval<8>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
+    else s = launch_eval<16>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);

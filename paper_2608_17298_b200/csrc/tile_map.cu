@@ -3,7 +3,7 @@
 // tile (ids stay ascending inside a tile because emission is id-major); the tile offset table
 // marks the group boundaries.  The pair count lives on the device: kernels are sized by the
 // caller's capacity and read the actual count.
-#include "common.cuh"
+#include "radix.cuh"
 
 namespace gart {
 
@@ -62,68 +62,6 @@ __global__ void __launch_bounds__(256) emit_pairs_kernel(const int4* __restrict_
     vals[p] = (uint32_t)lo;
 }
 
-// ---- stable LSD radix sort, 8-bit digits, one warp per chunk of RADIX_CHUNK consecutive items
-constexpr int RADIX_CHUNK = 2048;
-constexpr int RADIX_WARPS = 4;
-
-__global__ void __launch_bounds__(RADIX_WARPS * 32) radix_hist_kernel(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ counts,
-                                                                      int shift, int nchunks, uint32_t* __restrict__ table) {
-    __shared__ uint32_t hist[RADIX_WARPS][256];
-    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int chunk = blockIdx.x * RADIX_WARPS + w;
-    for (int d = lane; d < 256; d += 32) hist[w][d] = 0;
-    __syncwarp();
-    const uint32_t P = counts[GART_CNT_ERROR] ? 0u : counts[GART_CNT_PAIRS];
-    if (chunk < nchunks) {
-        const int64_t base = (int64_t)chunk * RADIX_CHUNK;
-        for (int r = 0; r < RADIX_CHUNK / 32; ++r) {
-            const int64_t i = base + r * 32 + lane;
-            if (i < P) atomicAdd(&hist[w][(keys[i] >> shift) & 255u], 1u);
-        }
-        __syncwarp();
-        for (int d = lane; d < 256; d += 32) table[(size_t)d * nchunks + chunk] = hist[w][d];
-    }
-}
-
-struct TableF {
-    const uint32_t* t;
-    __device__ __forceinline__ uint32_t operator()(int64_t i) const { return t[i]; }
-};
-
-__global__ void __launch_bounds__(RADIX_WARPS * 32) radix_scatter_kernel(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
-                                                                         const uint32_t* __restrict__ counts, int shift, int nchunks,
-                                                                         const uint32_t* __restrict__ table_scanned,
-                                                                         uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out) {
-    __shared__ uint32_t cursor[RADIX_WARPS][256];
-    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int chunk = blockIdx.x * RADIX_WARPS + w;
-    if (chunk >= nchunks) return;
-    const uint32_t P = counts[GART_CNT_ERROR] ? 0u : counts[GART_CNT_PAIRS];
-    const int64_t base = (int64_t)chunk * RADIX_CHUNK;
-    if (base >= P) return;
-    for (int d = lane; d < 256; d += 32) cursor[w][d] = table_scanned[(size_t)d * nchunks + chunk];
-    __syncwarp();
-    for (int r = 0; r < RADIX_CHUNK / 32; ++r) {
-        const int64_t i = base + r * 32 + lane;
-        const bool act = i < P;
-        const unsigned amask = __ballot_sync(0xffffffffu, act);
-        if (act) {
-            const uint32_t k = keys_in[i];
-            const uint32_t v = vals_in[i];
-            const uint32_t d = (k >> shift) & 255u;
-            const unsigned peers = __match_any_sync(amask, d);
-            const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
-            const uint32_t pos = cursor[w][d] + rank;
-            __syncwarp(amask);
-            if (rank == 0) cursor[w][d] += __popc(peers);
-            __syncwarp(amask);
-            keys_out[pos] = k;
-            vals_out[pos] = v;
-        }
-        if (amask != 0xffffffffu) break;
-    }
-}
-
 // tile_off[t] = first sorted position whose tile id is >= t; tile_off[T] = P.
 __global__ void __launch_bounds__(256) tile_offsets_kernel(const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ counts,
                                                            int T, uint32_t* __restrict__ tile_off) {
@@ -151,15 +89,14 @@ static TileMapWs tile_map_layout(void* base, int64_t n, int64_t cap_pairs) {
     size_t off = 0;
     auto take = [&](size_t b) { void* r = p ? (void*)(p + off) : nullptr; off += align256(b); return r; };
     const int64_t cp = cap_pairs > 0 ? cap_pairs : 1;
-    const int64_t nchunks = ceil_div(cp, RADIX_CHUNK);
     w.total64 = (uint64_t*)take(256);
     w.emit_off = (uint32_t*)take((size_t)(n + 1) * 4);
     w.keys0 = (uint32_t*)take((size_t)cp * 4);
     w.keys1 = (uint32_t*)take((size_t)cp * 4);
     w.vals1 = (uint32_t*)take((size_t)cp * 4);
-    w.table = (uint32_t*)take((size_t)(256 * nchunks + 1) * 4);
-    const int64_t scan_n = (n > 256 * nchunks ? n : 256 * nchunks);
-    w.scan_ws = take(scan_workspace_bytes(scan_n));
+    w.table = (uint32_t*)take(radix_table_bytes(cp));
+    const size_t s1 = scan_workspace_bytes(n), s2 = radix_scan_bytes(cp);
+    w.scan_ws = take(s1 > s2 ? s1 : s2);
     w.bytes = off;
     return w;
 }
@@ -202,31 +139,17 @@ extern "C" gart_status gart_tile_map(const gart_config* cfg, const int32_t* rect
 
     int bits = 1;
     while ((1 << bits) < T) ++bits;
-    const int passes = (bits + 7) / 8;
-    // value buffers alternate between pair_gid and ws.vals1 so that the last pass lands in pair_gid
-    uint32_t* vbuf[2] = {pair_gid, w.vals1};
-    uint32_t* kbuf[2] = {w.keys0, w.keys1};
-    int cur = passes & 1;  // emission target: after `passes` flips we are at index 0 = pair_gid
+    // value buffers alternate between pair_gid and a scratch array so that the last pass lands in pair_gid
+    uint32_t* const vbuf[2] = {pair_gid, w.vals1};
+    uint32_t* const kbuf[2] = {w.keys0, w.keys1};
+    const int cur = radix_passes(bits) & 1;   // emission target: after the passes the result is at index 0
     const int64_t pair_blocks = ceil_div(cap_pairs, 256);
     emit_pairs_kernel<<<(unsigned)pair_blocks, 256, 0, st>>>(rect4, w.emit_off, n, ts, tiles_x, counts, kbuf[cur], vbuf[cur]);
     GART_LAUNCH_CHECK();
-    const int nchunks = (int)ceil_div(cap_pairs, RADIX_CHUNK);
-    const int rblocks = (int)ceil_div(nchunks, RADIX_WARPS);
-    for (int pass = 0; pass < passes; ++pass) {
-        const int shift = 8 * pass;
-        radix_hist_kernel<<<rblocks, RADIX_WARPS * 32, 0, st>>>(kbuf[cur], counts, shift, nchunks, w.table);
-        GART_LAUNCH_CHECK();
-        TableF tf{w.table};
-        // in-place scan is safe: every block reads its items before any block's apply phase runs
-        // (separate launches), and apply re-reads through the functor before writing the same index
-        s = exclusive_scan(tf, (int64_t)256 * nchunks, w.table, w.total64, w.scan_ws, st);
-        if (s != GART_OK) return s;
-        radix_scatter_kernel<<<rblocks, RADIX_WARPS * 32, 0, st>>>(kbuf[cur], vbuf[cur], counts, shift, nchunks, w.table,
-                                                                   kbuf[cur ^ 1], vbuf[cur ^ 1]);
-        GART_LAUNCH_CHECK();
-        cur ^= 1;
-    }
-    tile_offsets_kernel<<<(unsigned)pair_blocks, 256, 0, st>>>(kbuf[cur], counts, T, tile_off);
+    s = radix_sort_pairs(kbuf, vbuf, cur, bits, cap_pairs, counts + GART_CNT_PAIRS, 0u, counts + GART_CNT_ERROR, w.table, w.scan_ws,
+                         w.total64, st);
+    if (s != GART_OK) return s;
+    tile_offsets_kernel<<<(unsigned)pair_blocks, 256, 0, st>>>(kbuf[0], counts, T, tile_off);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

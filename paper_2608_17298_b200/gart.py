@@ -23,12 +23,12 @@ STATUS_NAMES = {0: "GART_OK", 1: "GART_ERR_INVALID_ARG", 2: "GART_ERR_WORKSPACE_
                 3: "GART_ERR_CAPACITY_EXCEEDED", 4: "GART_ERR_CUDA"}
 CNT_VISIBLE, CNT_PAIRS, CNT_SLOTS_LO, CNT_SLOTS_HI, CNT_HITS, CNT_ERROR, CNT_MAX_RAY_HITS, CNT_STRADDLE, CNT_LT_SLOTS = range(9)
 COUNTS_WORDS = 12
-PRE_WORDS = 20
 GRAD_WORDS = 64
 
 EXPORTS = [
-    "gart_status_string", "gart_mask_words", "gart_bounds", "gart_tile_map_workspace_bytes", "gart_tile_map",
-    "gart_forward_workspace_bytes", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_read_counts",
+    "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
+    "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_forward_workspace_bytes", "gart_forward",
+    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_read_counts",
     "gart_view_host_arena_bytes", "gart_view_host",
 ]
 
@@ -69,15 +69,21 @@ def lib():
         L.gart_status_string.argtypes = [C.c_int]
         L.gart_mask_words.restype = i32
         L.gart_mask_words.argtypes = [i32]
-        L.gart_bounds.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+        L.gart_pre_words.restype = i32
+        L.gart_pre_words.argtypes = [i32]
+        L.gart_bounds_workspace_bytes.restype = sz
+        L.gart_bounds_workspace_bytes.argtypes = [i64]
+        L.gart_bounds.argtypes = [vp] * 10 + [sz, vp]
         L.gart_tile_map_workspace_bytes.restype = sz
         L.gart_tile_map_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
         L.gart_tile_map.argtypes = [vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, sz, vp]
         L.gart_forward_workspace_bytes.restype = sz
         L.gart_forward_workspace_bytes.argtypes = [i32, i32, i32, i64, i64]
-        L.gart_forward.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
-        L.gart_backward.argtypes = [vp] * 14
-        L.gart_backward_atomic.argtypes = [vp] * 12
+        L.gart_forward.argtypes = [vp] * 8 + [i64] + [vp] * 10 + [i64] + [vp] * 5 + [sz, vp]
+        L.gart_backward_workspace_bytes.restype = sz
+        L.gart_backward_workspace_bytes.argtypes = [i64]
+        L.gart_backward.argtypes = [vp] * 16 + [sz, vp]
+        L.gart_backward_atomic.argtypes = [vp] * 13
         L.gart_read_counts.argtypes = [vp, vp, vp]
         L.gart_view_host_arena_bytes.restype = sz
         L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
@@ -184,11 +190,26 @@ def gart_mask_words(tile_size: int) -> int:
 
 
 # ----------------------------------------------------------------------------------------- the calls
-def gart_bounds(cfg: Config, g: Gaussians, cam, rect, cls, pre, counts, stream=None):
+def _ws(workspace):
+    return _dev(workspace, torch.uint8, "workspace"), (workspace.numel() if workspace is not None else 0)
+
+
+def gart_pre_words(sh_degree: int) -> int:
+    return int(lib().gart_pre_words(int(sh_degree)))
+
+
+def gart_bounds_workspace_bytes(n) -> int:
+    return int(lib().gart_bounds_workspace_bytes(int(n)))
+
+
+def gart_bounds(cfg: Config, g: Gaussians, cam, rect, cls, pre, slot_of_gid, gid_of_slot, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
-    _check(lib().gart_bounds(C.byref(c), C.byref(gs), C.byref(cs), _dev(rect, torch.int32, "rect"),
-                             _dev(cls, torch.uint8, "cls"), _dev(pre, torch.float32, "pre"),
-                             _dev(counts, torch.int32, "counts"), _stream_ptr(stream)), "gart_bounds")
+    i32 = torch.int32
+    wp, wb = _ws(workspace)
+    _check(lib().gart_bounds(C.byref(c), C.byref(gs), C.byref(cs), _dev(rect, i32, "rect"), _dev(cls, torch.uint8, "cls"),
+                             _dev(pre, torch.float32, "pre"), _dev(slot_of_gid, i32, "slot_of_gid"),
+                             _dev(gid_of_slot, i32, "gid_of_slot"), _dev(counts, i32, "counts"), wp, wb,
+                             _stream_ptr(stream)), "gart_bounds")
 
 
 def gart_tile_map_workspace_bytes(n, width, height, tile_size, cap_pairs) -> int:
@@ -197,59 +218,65 @@ def gart_tile_map_workspace_bytes(n, width, height, tile_size, cap_pairs) -> int
 
 def gart_tile_map(cfg: Config, rect, n, cam, tile_off, pair_gid, cap_pairs, counts, workspace, stream=None):
     c = cfg.c()
+    wp, wb = _ws(workspace)
     _check(lib().gart_tile_map(C.byref(c), _dev(rect, torch.int32, "rect"), int(n), int(cam.width), int(cam.height),
                                _dev(tile_off, torch.int32, "tile_off"), _dev(pair_gid, torch.int32, "pair_gid"),
-                               int(cap_pairs), _dev(counts, torch.int32, "counts"),
-                               _dev(workspace, torch.uint8, "workspace"), workspace.numel() if workspace is not None else 0,
-                               _stream_ptr(stream)), "gart_tile_map")
+                               int(cap_pairs), _dev(counts, torch.int32, "counts"), wp, wb, _stream_ptr(stream)), "gart_tile_map")
 
 
 def gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits) -> int:
     return int(lib().gart_forward_workspace_bytes(int(width), int(height), int(tile_size), int(cap_pairs), int(cap_hits)))
 
 
-def gart_forward(cfg: Config, g: Gaussians, cam, pre, tile_off, pair_gid, cap_pairs, color, t_final, hit_count,
-                 pair_mask, pair_order, rank_gid, rank_mask, rank_gstart, tile_lt_base, lt, cap_hits, ray_off, ray_gid,
-                 ray_slot, counts, workspace, stream=None):
+def gart_forward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, pair_gid, cap_pairs, color,
+                 t_final, hit_count, pair_mask, pair_order, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, cap_hits,
+                 ray_off, ray_gid, ray_slot, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
-    _check(lib().gart_forward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
-                              _dev(pair_gid, i32, "pair_gid"), int(cap_pairs), _dev(color, f32, "color"),
-                              _dev(t_final, f32, "t_final"), _dev(hit_count, i32, "hit_count"),
+    wp, wb = _ws(workspace)
+    _check(lib().gart_forward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                              _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
+                              _dev(tile_off, i32, "tile_off"), _dev(pair_gid, i32, "pair_gid"), int(cap_pairs),
+                              _dev(color, f32, "color"), _dev(t_final, f32, "t_final"), _dev(hit_count, i32, "hit_count"),
                               _dev(pair_mask, i32, "pair_mask"), _dev(pair_order, i32, "pair_order"),
-                              _dev(rank_gid, i32, "rank_gid"), _dev(rank_mask, i32, "rank_mask"),
+                              _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
                               _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
                               _dev(lt, f32, "lt"), int(cap_hits), _dev(ray_off, i32, "ray_off"),
                               _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"),
-                              _dev(counts, i32, "counts"), _dev(workspace, torch.uint8, "workspace"),
-                              workspace.numel() if workspace is not None else 0, _stream_ptr(stream)), "gart_forward")
+                              _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_forward")
 
 
-def gart_backward(cfg: Config, g: Gaussians, cam, pre, tile_off, rank_gid, rank_mask, rank_gstart,
-                  tile_lt_base, lt, dL_dcolor, grad, counts, stream=None):
+def gart_backward_workspace_bytes(n) -> int:
+    return int(lib().gart_backward_workspace_bytes(int(n)))
+
+
+def gart_backward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
+                  rank_gstart, tile_lt_base, lt, dL_dcolor, grad, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
-    _check(lib().gart_backward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"), _dev(tile_off, i32, "tile_off"),
-                               _dev(rank_gid, i32, "rank_gid"), _dev(rank_mask, i32, "rank_mask"),
-                               _dev(rank_gstart, i32, "rank_gstart"),
-                               _dev(tile_lt_base, i32, "tile_lt_base"), _dev(lt, f32, "lt"),
-                               _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"), _dev(counts, i32, "counts"),
-                               _stream_ptr(stream)), "gart_backward")
+    wp, wb = _ws(workspace)
+    _check(lib().gart_backward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                               _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
+                               _dev(tile_off, i32, "tile_off"),
+                               _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
+                               _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
+                               _dev(lt, f32, "lt"), _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
+                               _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward")
 
 
-def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, ray_off, ray_gid, ray_slot, lt, dL_dcolor, grad, counts,
-                         stream=None):
+def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, ray_off, ray_gid, ray_slot, lt, dL_dcolor,
+                         grad, counts, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     _check(lib().gart_backward_atomic(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
-                                      _dev(ray_off, i32, "ray_off"), _dev(ray_gid, i32, "ray_gid"),
-                                      _dev(ray_slot, i32, "ray_slot"), _dev(lt, f32, "lt"),
+                                      _dev(slot_of_gid, i32, "slot_of_gid"), _dev(ray_off, i32, "ray_off"),
+                                      _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"), _dev(lt, f32, "lt"),
                                       _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
                                       _dev(counts, i32, "counts"), _stream_ptr(stream)), "gart_backward_atomic")
 
 
 def gart_read_counts(counts, stream=None):
-    """Counts block as a list of 8 unsigned ints (synchronises the stream)."""
+    """Counts block as a list of unsigned ints (synchronises the stream)."""
     host = (C.c_uint32 * COUNTS_WORDS)()
     _check(lib().gart_read_counts(_dev(counts, torch.int32, "counts"), host, _stream_ptr(stream)), "gart_read_counts")
     return [int(v) for v in host]
@@ -299,17 +326,19 @@ class ViewBuffers:
         i32, f32, u8 = torch.int32, torch.float32, torch.uint8
         e = lambda shape, dt: torch.empty(shape, dtype=dt, device=device)
         n1, cp, ch = max(self.n, 1), max(self.cap_pairs, 1), max(self.cap_hits, 1)
-        self.rect, self.cls, self.pre = e((n1, 4), i32), e((n1,), u8), e((n1, PRE_WORDS), f32)
+        self.rect, self.cls, self.pre = e((n1, 4), i32), e((n1,), u8), e((n1, gart_pre_words(sh_degree)), f32)
+        self.slot_of_gid, self.gid_of_slot = e((n1,), i32), e((n1,), i32)
         self.counts = torch.zeros(COUNTS_WORDS, dtype=i32, device=device)
         self.tile_off, self.pair_gid = e((T + 1,), i32), e((cp,), i32)
         self.pair_mask, self.pair_order = e((cp, mw), i32), e((cp,), i32)
-        self.rank_gid, self.rank_mask, self.rank_gstart = e((cp,), i32), e((cp, mw), i32), e((cp,), i32)
+        self.rank_sid, self.rank_mask, self.rank_gstart = e((cp,), i32), e((cp, mw), i32), e((cp,), i32)
         self.tile_lt_base = e((T + 1,), i32)
         self.color, self.t_final, self.hit_count = e((H, W, 3), f32), e((H, W), f32), e((H, W), i32)
         self.lt = e((ch, 4), f32)
         self.ray_off, self.ray_gid, self.ray_slot = e((H * W + 1,), i32), e((ch,), i32), e((ch,), i32)
         self.grad = e((n1, GRAD_WORDS), f32)
-        ws = max(gart_tile_map_workspace_bytes(n1, W, H, ts, cap_pairs), gart_forward_workspace_bytes(W, H, ts, cap_pairs, cap_hits))
+        ws = max(gart_bounds_workspace_bytes(n1), gart_tile_map_workspace_bytes(n1, W, H, ts, cap_pairs),
+                 gart_forward_workspace_bytes(W, H, ts, cap_pairs, cap_hits), gart_backward_workspace_bytes(n1))
         self.workspace = e((ws,), u8)
 
     def bytes(self):
@@ -317,24 +346,25 @@ class ViewBuffers:
 
 
 def run_bounds_tile_map(cfg, g, cam, buf: ViewBuffers, stream=None):
-    gart_bounds(cfg, g, cam, buf.rect, buf.cls, buf.pre, buf.counts, stream)
+    gart_bounds(cfg, g, cam, buf.rect, buf.cls, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.counts, buf.workspace, stream)
     gart_tile_map(cfg, buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.counts, buf.workspace, stream)
 
 
 def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None):
-    gart_forward(cfg, g, cam, buf.pre, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color, buf.t_final, buf.hit_count,
-                 buf.pair_mask, buf.pair_order, buf.rank_gid, buf.rank_mask, buf.rank_gstart, buf.tile_lt_base, buf.lt,
-                 buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.counts, buf.workspace, stream)
+    gart_forward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color,
+                 buf.t_final, buf.hit_count, buf.pair_mask, buf.pair_order, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
+                 buf.tile_lt_base, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.counts, buf.workspace,
+                 stream)
 
 
 def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
-    gart_backward(cfg, g, cam, buf.pre, buf.tile_off, buf.rank_gid, buf.rank_mask, buf.rank_gstart,
-                  buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts, stream)
+    gart_backward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
+                  buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
 
 
 def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):
-    gart_backward_atomic(cfg, g, cam, buf.pre, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.lt, dL_dcolor, grad,
-                         buf.counts, stream)
+    gart_backward_atomic(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.lt, dL_dcolor,
+                         grad, buf.counts, stream)
 
 
 def size_view(cfg, g, cam, slack=1.0, device="cuda"):

@@ -54,7 +54,8 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
     out["pair_gid"] = u32(to_np(buf.pair_gid))[:P]
     out["pair_mask"] = u32(to_np(buf.pair_mask))[:P]
     out["pair_order"] = u32(to_np(buf.pair_order))[:P]
-    out["rank_gid"] = u32(to_np(buf.rank_gid))[:P]
+    out["rank_sid"] = u32(to_np(buf.rank_sid))[:P]
+    out["slot_of_gid"], out["gid_of_slot"] = u32(to_np(buf.slot_of_gid))[:g.n], u32(to_np(buf.gid_of_slot))[:g.n]
     out["rank_mask"] = u32(to_np(buf.rank_mask))[:P]
     out["rank_gstart"] = u32(to_np(buf.rank_gstart))[:P]
     out["tile_lt_base"] = u32(to_np(buf.tile_lt_base))
@@ -126,7 +127,18 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     assert np.all((po[:-1] >= po[1:]) | ~same_tile)
     assert np.all((order[:-1] < order[1:]) | (po[:-1] != po[1:]) | ~same_tile)
     # copies in rank order
-    assert np.array_equal(gpu["rank_gid"], gpu["pair_gid"][order]) and np.array_equal(gpu["rank_mask"], gpu["pair_mask"][order])
+    assert np.array_equal(gpu["rank_sid"], gpu["slot_of_gid"][gpu["pair_gid"][order]])
+    assert np.array_equal(gpu["rank_mask"], gpu["pair_mask"][order])
+    # slots: visible Gaussians in the order of the tile of their rectangle's corner, ids ascending inside a tile
+    rect_ = gpu["rect"]
+    vis = rect_[:, 2] >= rect_[:, 0]
+    V = int(vis.sum())
+    key_ = (rect_[:, 1] // ts) * tiles_x + rect_[:, 0] // ts
+    want_order = np.nonzero(vis)[0][np.argsort(key_[vis], kind="stable")]
+    assert np.array_equal(gpu["gid_of_slot"][:V], want_order.astype(np.uint32)) and np.all(gpu["gid_of_slot"][V:] == 0xffffffff)
+    inv = np.full(rect_.shape[0], 0xffffffff, np.uint32)
+    inv[want_order] = np.arange(V, dtype=np.uint32)
+    assert np.array_equal(gpu["slot_of_gid"], inv)
     # rank_gstart: start of the 32-rank group; a group spans 32 x its largest (= first) count
     gs_ = gpu["rank_gstart"].astype(np.int64)                   # by position in rank order
     first = rank % 32 == 0

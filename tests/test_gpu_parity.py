@@ -229,13 +229,17 @@ def test_invalid_arguments_return_status():
     cam = cams[0]
     g = G.Gaussians.from_numpy(scene)
     buf = G.ViewBuffers(g.n, 0, cam, G.Config(), 100, 1000)
+    args = (buf.slot_of_gid, buf.gid_of_slot, buf.counts)
     with pytest.raises(G.GartError) as e:
-        G.gart_bounds(G.Config(tile_size=12), g, cam, buf.rect, buf.cls, buf.pre, buf.counts)
+        G.gart_bounds(G.Config(tile_size=12), g, cam, buf.rect, buf.cls, buf.pre, *args, buf.workspace)
     assert e.value.status == 1
     with pytest.raises(G.GartError) as e:
-        G.gart_bounds(G.Config(), g, cam, None, buf.cls, buf.pre, buf.counts)
+        G.gart_bounds(G.Config(), g, cam, None, buf.cls, buf.pre, *args, buf.workspace)
     assert e.value.status == 1
-    G.gart_bounds(G.Config(), g, cam, buf.rect, buf.cls, buf.pre, buf.counts)
+    with pytest.raises(G.GartError) as e:
+        G.gart_bounds(G.Config(), g, cam, buf.rect, buf.cls, buf.pre, *args, buf.workspace[:512])
+    assert e.value.status == 2
+    G.gart_bounds(G.Config(), g, cam, buf.rect, buf.cls, buf.pre, *args, buf.workspace)
     small = torch.empty(256, dtype=torch.uint8, device="cuda")
     with pytest.raises(G.GartError) as e:
         G.gart_tile_map(G.Config(), buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, 100, buf.counts, small)
