@@ -235,9 +235,157 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
 }
 
 // ------------------------------------------------------------------------------------------ phase 4
-constexpr int SORT_CAP = 1024;   // keys per warp held in shared memory; longer rays sort in global memory
+constexpr int SORT_CAP = 512;    // hits per ray sorted in registers; longer rays sort in global memory
 constexpr int SWEEP_WARPS = 4;
 
+// ---- rays of up to SORT_CAP hits: one warp, keys in registers (R per lane, lane l holds positions l R .. l R + R - 1)
+// Keys are (t* bits << 32) | record index; padding keys are all ones and sort last.
+template <int R>
+__device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) {
+    constexpr int N = 32 * R;
+#pragma unroll
+    for (int kk = 2; kk <= N; kk <<= 1) {
+#pragma unroll
+        for (int j = kk >> 1; j >= 1; j >>= 1) {
+            if (j >= R) {   // partner in another lane, same register
+                const int lj = j / R;
+                const bool lower = (lane & lj) == 0;
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    const unsigned long long o = __shfl_xor_sync(0xffffffffu, k[r], lj);
+                    const bool asc = ((lane * R + r) & kk) == 0;
+                    k[r] = ((o < k[r]) == (lower == asc)) ? o : k[r];
+                }
+            } else {        // partner in this lane
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if ((r ^ j) > r) {
+                        const bool asc = ((lane * R + r) & kk) == 0;
+                        const unsigned long long x = k[r], y = k[r ^ j];
+                        const bool sw = (x > y) == asc;
+                        k[r] = sw ? y : x;
+                        k[r ^ j] = sw ? x : y;
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int R>
+__device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
+                                               float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
+                                               float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
+    unsigned long long k[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        // load striped (coalesced), the network does not care about the initial arrangement
+        const int i = r * 32 + lane;
+        k[r] = i < n ? (((unsigned long long)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (unsigned long long)i) : ~0ull;
+    }
+    sort_regs<R>(k, lane);
+    // hits with bit-identical t* must ascend in Gaussian id (records arrive in arbitrary order)
+    {
+        bool tie = false;
+#pragma unroll
+        for (int r = 0; r + 1 < R; ++r) tie = tie || ((uint32_t)(k[r] >> 32) == (uint32_t)(k[r + 1] >> 32) && lane * R + r + 1 < n);
+        const unsigned long long nb = __shfl_down_sync(0xffffffffu, k[0], 1);
+        tie = tie || (lane < 31 && (uint32_t)(k[R - 1] >> 32) == (uint32_t)(nb >> 32) && (lane + 1) * R < n);
+        if (__any_sync(0xffffffffu, tie)) {
+            // rare: odd-even transposition on (t*, id) between neighbours with equal t*, n rounds at most
+            for (int round = 0; round < n; ++round) {
+                bool moved = false;
+#pragma unroll
+                for (int r = 0; r + 1 < R; ++r) {
+                    if (lane * R + r + 1 < n && (uint32_t)(k[r] >> 32) == (uint32_t)(k[r + 1] >> 32) &&
+                        __float_as_uint(rec[2 * (uint32_t)k[r]].y) > __float_as_uint(rec[2 * (uint32_t)k[r + 1]].y)) {
+                        const unsigned long long t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
+                    }
+                }
+                // across the lane boundary: even lanes lead on even rounds, odd lanes on odd rounds
+                const unsigned long long up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
+                const bool lead = ((lane ^ round) & 1) == 0;
+                if (lead) {
+                    if (lane < 31 && (lane + 1) * R < n && (uint32_t)(k[R - 1] >> 32) == (uint32_t)(up >> 32) &&
+                        __float_as_uint(rec[2 * (uint32_t)k[R - 1]].y) > __float_as_uint(rec[2 * (uint32_t)up].y)) { k[R - 1] = up; moved = true; }
+                } else {
+                    if (lane > 0 && lane * R < n && (uint32_t)(dn >> 32) == (uint32_t)(k[0] >> 32) &&
+                        __float_as_uint(rec[2 * (uint32_t)dn].y) > __float_as_uint(rec[2 * (uint32_t)k[0]].y)) { k[0] = dn; moved = true; }
+                }
+                if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
+            }
+        }
+    }
+    // front to back: transmittance in front of every hit (Eq. 7)
+    float al[R];
+    float lp = 1.0f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        al[r] = lane * R + r < n ? __ldg(&rec[2 * (uint32_t)k[r]].w) : 0.0f;
+        lp *= 1.0f - al[r];
+    }
+    float inc = lp;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc *= t;
+    }
+    float T0 = __shfl_up_sync(0xffffffffu, inc, 1);
+    if (lane == 0) T0 = 1.0f;
+    const float Tfin = __shfl_sync(0xffffffffu, inc, 31);
+    // back to front: colour composited behind every hit; first the lane totals ...
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f;
+    {
+        float T = T0;
+        float w0[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) { w0[r] = T * al[r]; T *= 1.0f - al[r]; }
+#pragma unroll
+        for (int r = R - 1; r >= 0; --r) {
+            if (lane * R + r < n) {
+                const float4 c = __ldg(&rec[2 * (uint32_t)k[r] + 1]);
+                s0 = fmaf(w0[r], c.x, s0); s1 = fmaf(w0[r], c.y, s1); s2 = fmaf(w0[r], c.z, s2);
+            }
+        }
+    }
+    float u0 = s0, u1 = s1, u2 = s2;   // inclusive suffix over lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float a0 = __shfl_down_sync(0xffffffffu, u0, o), a1 = __shfl_down_sync(0xffffffffu, u1, o), a2 = __shfl_down_sync(0xffffffffu, u2, o);
+        if (lane + o < 32) { u0 += a0; u1 += a1; u2 += a2; }
+    }
+    float e0 = __shfl_down_sync(0xffffffffu, u0, 1), e1 = __shfl_down_sync(0xffffffffu, u1, 1), e2 = __shfl_down_sync(0xffffffffu, u2, 1);
+    if (lane == 31) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
+    // ... then every hit: background term + lanes behind + hits behind inside the lane
+    float k0 = fmaf(Tfin, bg0, e0), k1 = fmaf(Tfin, bg1, e1), k2 = fmaf(Tfin, bg2, e2);
+    {
+        float Ts[R];
+        float T = T0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) { Ts[r] = T; T *= 1.0f - al[r]; }
+#pragma unroll
+        for (int r = R - 1; r >= 0; --r) {
+            const int i = lane * R + r;
+            if (i < n) {
+                const uint32_t c = (uint32_t)k[r];
+                const float4 ra = __ldg(&rec[2 * c]);
+                const float4 rb = __ldg(&rec[2 * c + 1]);
+                const uint32_t slot = __float_as_uint(ra.z);
+                lt[slot] = make_float4(k0, k1, k2, Ts[r]);
+                ray_gid[b + i] = __float_as_uint(ra.y);
+                ray_slot[b + i] = slot;
+                const float wgt = Ts[r] * al[r];
+                k0 = fmaf(wgt, rb.x, k0); k1 = fmaf(wgt, rb.y, k1); k2 = fmaf(wgt, rb.z, k2);
+            }
+        }
+    }
+    if (lane == 0) {   // lane 0's running sum has reached the front of the ray
+        color[3 * r_idx] = k0; color[3 * r_idx + 1] = k1; color[3 * r_idx + 2] = k2;
+        t_final[r_idx] = Tfin;
+    }
+}
+
+// ---- longer rays: keys in global memory, sorting network over memory
 __device__ __forceinline__ void cmp_swap(uint64_t* a, int i, int l) {
     const uint64_t x = a[i], y = a[l];
     if (x > y) { a[i] = y; a[l] = x; }
@@ -267,37 +415,16 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
     }
 }
 
-// Keys are (t* bits << 32) | record index.  A ray's records arrive in arbitrary order, so hits with
-// bit-identical t* are put in ascending Gaussian id afterwards (rare: one lane, insertion sort).
-__global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs,
-                                                                          uint64_t* __restrict__ long_keys, int64_t n_rays,
-                                                                          float bg0, float bg1, float bg2,
-                                                                          float* __restrict__ color, float* __restrict__ t_final,
-                                                                          float4* __restrict__ lt, uint32_t* __restrict__ ray_gid,
-                                                                          uint32_t* __restrict__ ray_slot, const uint32_t* __restrict__ counts) {
-    __shared__ uint64_t skeys[SWEEP_WARPS][SORT_CAP];
-    if (counts[GART_CNT_ERROR]) return;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t r = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
-    if (r >= n_rays) return;
-    const size_t b = ray_off[r];
-    const int n = (int)(ray_off[r + 1] - ray_off[r]);
-    if (n == 0) {
-        if (lane == 0) {
-            color[3 * r] = bg0; color[3 * r + 1] = bg1; color[3 * r + 2] = bg2;
-            t_final[r] = 1.0f;
-        }
-        return;
-    }
-    const float4* rec = recs + b * 2;
-    uint64_t* kp = n <= SORT_CAP ? skeys[warp] : long_keys + b;
+__device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int lane, size_t b, int64_t r,
+                                            float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
+                                            float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
     for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
     __syncwarp();
     warp_sort(kp, n, lane);
     bool tie = false;
     for (int i = lane; i + 1 < n; i += 32) tie = tie || ((uint32_t)(kp[i] >> 32) == (uint32_t)(kp[i + 1] >> 32));
     if (__any_sync(0xffffffffu, tie)) {
-        if (lane == 0) {
+        if (lane == 0) {   // insertion sort of the runs of equal t* by Gaussian id
             for (int i = 1; i < n; ++i) {
                 const uint64_t x = kp[i];
                 const uint32_t tx = (uint32_t)(x >> 32), gx = __float_as_uint(rec[2 * (uint32_t)x].y);
@@ -311,8 +438,6 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         }
         __syncwarp();
     }
-
-    // front to back: transmittance in front of every hit (Eq. 7); kept in the key's high word
     float carryT = 1.0f;
     for (int base = 0; base < n; base += 32) {
         const int i = base + lane;
@@ -333,8 +458,6 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
     }
     __syncwarp();
     const float Tfin = carryT;
-
-    // back to front: colour composited behind every hit (background term first)
     float k0 = Tfin * bg0, k1 = Tfin * bg1, k2 = Tfin * bg2;
     for (int base = 0; base < n; base += 32) {
         const int i = n - 1 - (base + lane);
@@ -374,6 +497,36 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         color[3 * r] = k0; color[3 * r + 1] = k1; color[3 * r + 2] = k2;
         t_final[r] = Tfin;
     }
+}
+
+__global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs,
+                                                                          uint64_t* __restrict__ long_keys, int64_t n_rays,
+                                                                          float bg0, float bg1, float bg2,
+                                                                          float* __restrict__ color, float* __restrict__ t_final,
+                                                                          float4* __restrict__ lt, uint32_t* __restrict__ ray_gid,
+                                                                          uint32_t* __restrict__ ray_slot, const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t r = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
+    if (r >= n_rays) return;
+    const size_t b = ray_off[r];
+    const int n = (int)(ray_off[r + 1] - ray_off[r]);
+    if (n == 0) {
+        if (lane == 0) {
+            color[3 * r] = bg0; color[3 * r + 1] = bg1; color[3 * r + 2] = bg2;
+            t_final[r] = 1.0f;
+        }
+        return;
+    }
+    const float4* rec = recs + b * 2;
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot)
+    if (n <= 32) GART_SWEEP(1);
+    else if (n <= 64) GART_SWEEP(2);
+    else if (n <= 128) GART_SWEEP(4);
+    else if (n <= 256) GART_SWEEP(8);
+    else if (n <= SORT_CAP) GART_SWEEP(16);
+    else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot);
+#undef GART_SWEEP
 }
 
 // ------------------------------------------------------------------------------------------ host
