@@ -217,7 +217,12 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
             const int p = pm.next();
             const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
             const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
-            const float* Y = spix + p * PW;
+            float Y[PW];
+#pragma unroll
+            for (int k4 = 0; k4 < PW / 4; ++k4) {   // 16-byte shared loads of the pixel's SH basis
+                const float4 t4 = reinterpret_cast<const float4*>(spix + p * PW)[k4];
+                Y[4 * k4] = t4.x; Y[4 * k4 + 1] = t4.y; Y[4 * k4 + 2] = t4.z; Y[4 * k4 + 3] = t4.w;
+            }
             float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
 #pragma unroll
             for (int k = 0; k < K; ++k) {
@@ -243,20 +248,23 @@ constexpr int SWEEP_WARPS = 4;
 template <int R>
 __device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) {
     constexpr int N = 32 * R;
-#pragma unroll
+    // the merge sizes and the cross-lane distances are run-time loops (small code: the instruction cache
+    // matters more here than the loop overhead); register indices stay compile-time
+#pragma unroll 1
     for (int kk = 2; kk <= N; kk <<= 1) {
+#pragma unroll 1
+        for (int lj = (kk >> 1) / R; lj >= 1; lj >>= 1) {   // partner in another lane, same register
+            const bool lower = (lane & lj) == 0;
 #pragma unroll
-        for (int j = kk >> 1; j >= 1; j >>= 1) {
-            if (j >= R) {   // partner in another lane, same register
-                const int lj = j / R;
-                const bool lower = (lane & lj) == 0;
+            for (int r = 0; r < R; ++r) {
+                const unsigned long long o = __shfl_xor_sync(0xffffffffu, k[r], lj);
+                const bool asc = ((lane * R + r) & kk) == 0;
+                k[r] = ((o < k[r]) == (lower == asc)) ? o : k[r];
+            }
+        }
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    const unsigned long long o = __shfl_xor_sync(0xffffffffu, k[r], lj);
-                    const bool asc = ((lane * R + r) & kk) == 0;
-                    k[r] = ((o < k[r]) == (lower == asc)) ? o : k[r];
-                }
-            } else {        // partner in this lane
+        for (int j = R >> 1; j >= 1; j >>= 1) {             // partner in this lane
+            if (j < kk) {
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
                     if ((r ^ j) > r) {
