@@ -22,7 +22,7 @@ constexpr int BWD_THREADS = BWD_WARPS * 32;
 constexpr int BWD_CHUNK = 16;                          // LT entries per lane and per pipeline stage
 constexpr int BWD_STAGE_F4 = BWD_CHUNK * 32;           // float4 per stage (8 KB)
 constexpr int BWD_LT_SMEM = BWD_WARPS * 2 * BWD_STAGE_F4 * 16;
-constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + BWD_THREADS * ((20 + sw + 3) / 4) * 16; }
+constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + BWD_THREADS * (((20 + sw + 3) / 4) | 1) * 16; }
 constexpr uint32_t BWD_WAIT_LIMIT = 1u << 22;          // bounded wait on a copy; then the error bit is set
 
 template <int K>
@@ -53,6 +53,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return false;
 }
 // global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
+// Orders this thread's earlier shared-memory accesses (generic proxy) before later accesses of the
+// asynchronous proxy: issued before a bulk copy overwrites a buffer that was just read.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
@@ -203,6 +206,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     // record (evaluation record + SH coefficients) of a lane's Gaussian, staged through shared memory one
     // group ahead; PF4 float4 per lane
     constexpr int PF4 = (20 + SW + 3) / 4;
+    constexpr int PSTR = PF4 | 1;   // lane stride in the buffer, odd: the lanes' 16-byte reads fall into distinct banks
     extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][PF4] parameters
     __shared__ __align__(16) float spix[NT * PW];
     __shared__ __align__(8) uint64_t bars[BWD_WARPS][3];
@@ -239,7 +243,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
 
     const float4* lt_tile = lt + tile_lt_base[tile];
     float4* my_stage = dyn + (size_t)warp * 2 * BWD_STAGE_F4;
-    float4* my_par = dyn + (size_t)BWD_WARPS * 2 * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PF4;
+    float4* my_par = dyn + (size_t)BWD_WARPS * 2 * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PSTR;
     const uint32_t stage_addr = smem_u32(my_stage);
     const uint32_t par_addr = smem_u32(my_par);
     const uint32_t bar_addr = smem_u32(&bars[warp][0]);
@@ -296,7 +300,8 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
             if (4 * q + 2 < SW) R.set(4 * q + 2, t.z);
             if (4 * q + 3 < SW) R.set(4 * q + 3, t.w);
         }
-        __syncwarp();
+        fence_proxy_async();
+        __syncwarp();   // every lane has read its record: the buffer may be overwritten
         if (nxt.cmax != 0) issue_params(nxt);
         const int bx = x0 - P.ix, by = y0 - P.iy;
         const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
@@ -310,6 +315,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
             const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
             for (int e = k * BWD_CHUNK; e < e_end; ++e)
                 bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, cur.pm.next(), sl[(e - k * BWD_CHUNK) * 32]);
+            fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
         }

@@ -114,6 +114,21 @@ def test_rays_longer_than_the_shared_memory_sort():
     assert gpu["counts"][G.CNT_MAX_RAY_HITS] > 1024
 
 
+@pytest.mark.parametrize("deg", [0, 1, 2, 3])
+def test_many_rank_groups_and_multi_chunk_pairs(deg):
+    """Hundreds of pairs per tile, every pair hitting (almost) all 64 pixels: each warp of the backward walks
+    several rank groups and several LT chunks per group, re-using its shared-memory buffers every time."""
+    rng = np.random.default_rng(11 + deg)
+    n = 400
+    mean = np.stack([rng.normal(0, 0.02, n), rng.normal(0, 0.02, n), rng.uniform(2.0, 6.0, n)], 1)
+    scene = gs.Scene(mean.astype(np.float32), np.full((n, 3), 0.25, np.float32) * rng.uniform(0.8, 1.2, (n, 3)).astype(np.float32),
+                     gs._unit_quats(rng, n).astype(np.float32), rng.uniform(0.01, 0.03, n).astype(np.float32),
+                     gs._sh(rng, n, deg), deg)
+    cam = gs.pinhole(16, 16, 20.0)
+    for rep in range(3):          # a race would not fail every time
+        full_parity(scene, cam, G.Config(tile_size=8), g=gs.upstream_gradient(cam, rep))
+
+
 def test_primitive_and_atomic_backward_agree():
     scene, cams = gs.config_cluster(n=3000, width=128, height=96)
     g = gs.upstream_gradient(cams[0], 1)
