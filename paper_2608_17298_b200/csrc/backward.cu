@@ -313,8 +313,17 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit >> 1) & 1u))) { fail(); return; }
             const float4* sl = my_stage + s * BWD_STAGE_F4 + lane;
             const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
-            for (int e = k * BWD_CHUNK; e < e_end; ++e)
-                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, cur.pm.next(), sl[(e - k * BWD_CHUNK) * 32]);
+            // two hits per iteration: two independent dependency chains for the scheduler to interleave
+            int e = k * BWD_CHUNK;
+            const float4* se = sl;
+            for (; e + 1 < e_end; e += 2, se += 64) {
+                const int p0 = cur.pm.next();
+                const int p1 = cur.pm.next();
+                const float4 L0 = se[0], L1 = se[32];
+                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, p0, L0);
+                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, p1, L1);
+            }
+            if (e < e_end) bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, cur.pm.next(), se[0]);
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
@@ -346,38 +355,47 @@ __global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc
     if (i < (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4)) gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
-// Two roles by block range, 16 lanes per record.  Blocks [0, slot_blocks): per slot, in slot order,
-// convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity, copy the SH
-// gradient and write the Gaussian's whole gradient record (reads are sequential, the 256-byte writes
-// scattered).  The remaining blocks: per Gaussian, zero the record if it has no slot.
-__global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, int64_t slot_blocks, const float4* __restrict__ qs,
+// Three roles by block range; every write covers whole 32-byte sectors of a gradient record.
+//   [0, conv_blocks)            one thread per slot: convert the accumulated moments (words 0..9) into
+//                               d mean, d scale, d quat, d opacity and write words 0..15 of the record
+//                               (all 32 lanes busy with the ~300-instruction conversion);
+//   [conv_blocks, +copy_blocks) 16 lanes per slot, 12 of them copy words 16..63 (SH gradient);
+//   the rest                    16 lanes per Gaussian: zero the record if the Gaussian has no slot.
+// Reads run in slot order (sequential), the writes scatter by Gaussian id.
+__global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, int64_t conv_blocks, int64_t copy_blocks, const float4* __restrict__ qs,
                                                            const uint32_t* __restrict__ slot_of_gid, const uint32_t* __restrict__ gid_of_slot,
                                                            const float4* __restrict__ gacc4, float4* __restrict__ grad4,
                                                            const uint32_t* __restrict__ counts) {
     if (counts[GART_CNT_ERROR]) return;
-    const int l = threadIdx.x & 15;
-    if ((int64_t)blockIdx.x < slot_blocks) {
-        const int64_t sid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;
-        if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
-        const float4* gp = gacc4 + (size_t)sid * (GART_GRAD_WORDS / 4);
-        float4 out = gp[l];
-        if (l < 3) {
-            const float4 a = gp[0], b = gp[1], c = gp[2];
-            const float v[3] = {a.x, a.y, a.z};
-            const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
-            const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
-            const float q[4] = {q4.x, q4.y, q4.z, q4.w};
-            const float sc[3] = {s4.x, s4.y, s4.z};
-            const GeoGrad o = moments_to_grads(v, Q, q, sc);
-            if (l == 0) out = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
-            else if (l == 1) out = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
-            else out = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
-        }
-        grad4[(size_t)gid_of_slot[sid] * (GART_GRAD_WORDS / 4) + l] = out;
+    constexpr int F4 = GART_GRAD_WORDS / 4;
+    const int64_t V = counts[GART_CNT_VISIBLE];
+    if ((int64_t)blockIdx.x < conv_blocks) {
+        const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        if (sid >= V) return;
+        const float4* gp = gacc4 + (size_t)sid * F4;
+        const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
+        const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
+        float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
+        const float v[3] = {a.x, a.y, a.z};
+        const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
+        const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+        const float sc[3] = {s4.x, s4.y, s4.z};
+        const GeoGrad o = moments_to_grads(v, Q, q, sc);
+        out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
+        out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
+        out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
+        out[3] = d;
+    } else if ((int64_t)blockIdx.x < conv_blocks + copy_blocks) {
+        const int64_t t = ((int64_t)blockIdx.x - conv_blocks) * blockDim.x + threadIdx.x;
+        const int64_t sid = t >> 4;
+        const int l = (int)(t & 15);
+        if (sid >= V || l < 4) return;
+        grad4[(size_t)gid_of_slot[sid] * F4 + l] = gacc4[(size_t)sid * F4 + l];
     } else {
-        const int64_t i = (((int64_t)blockIdx.x - slot_blocks) * blockDim.x + threadIdx.x) >> 4;
+        const int64_t t = ((int64_t)blockIdx.x - conv_blocks - copy_blocks) * blockDim.x + threadIdx.x;
+        const int64_t i = t >> 4;
         if (i >= n) return;
-        if (slot_of_gid[i] == 0xffffffffu) grad4[(size_t)i * (GART_GRAD_WORDS / 4) + l] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (slot_of_gid[i] == 0xffffffffu) grad4[(size_t)i * F4 + (t & 15)] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
 
@@ -442,10 +460,11 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
     else s = launch_pairs<16>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
     if (s != GART_OK) return s;
-    const int64_t fblocks = ceil_div(g->n * 16, 256);
+    const int64_t conv_blocks = ceil_div(g->n, 256), copy_blocks = ceil_div(g->n * 16, 256);
     const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
-    bwd_finalize_kernel<<<(unsigned)(2 * fblocks), 256, 0, st>>>(g->n, fblocks, qs, slot_of_gid, gid_of_slot,
-                                                                 reinterpret_cast<const float4*>(gacc), reinterpret_cast<float4*>(grad), counts);
+    bwd_finalize_kernel<<<(unsigned)(conv_blocks + 2 * copy_blocks), 256, 0, st>>>(g->n, conv_blocks, copy_blocks, qs, slot_of_gid, gid_of_slot,
+                                                                                  reinterpret_cast<const float4*>(gacc),
+                                                                                  reinterpret_cast<float4*>(grad), counts);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

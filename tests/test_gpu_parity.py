@@ -275,6 +275,7 @@ def test_host_entry_point_matches_device_path():
     g = gs.upstream_gradient(cam, 0)
     gpu = P.run_gpu(scene, cam, cfg, g, atomic=False)
     Pn, Hn = gpu["counts"][G.CNT_PAIRS], gpu["counts"][G.CNT_HITS]
+    Ln = gpu["counts"][G.CNT_LT_SLOTS]          # LT entries including the padding of the interleaved layout
 
     class HS:
         pass
@@ -284,9 +285,9 @@ def test_host_entry_point_matches_device_path():
     hs.sh_degree = scene.sh_degree
     color = torch.empty((cam.height, cam.width, 3), dtype=torch.float32).pin_memory()
     grad = torch.empty((scene.n, G.GRAD_WORDS), dtype=torch.float32).pin_memory()
-    arena = torch.empty(G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam.width, cam.height, 8, Pn + 5, Hn + 5),
+    arena = torch.empty(G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam.width, cam.height, 8, Pn + 5, Ln + 5),
                         dtype=torch.uint8, device="cuda")
-    counts = G.gart_view_host(cfg, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Hn + 5, arena)
+    counts = G.gart_view_host(cfg, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Ln + 5, arena)
     assert counts[G.CNT_HITS] == Hn and counts[G.CNT_PAIRS] == Pn
     assert np.array_equal(color.numpy(), gpu["color"])
     a, b = grad.numpy().astype(np.float64), gpu["grad"].astype(np.float64)
