@@ -244,9 +244,16 @@ constexpr int SORT_CAP = 512;    // hits per ray sorted in registers; longer ray
 constexpr int SWEEP_WARPS = 4;
 
 // ---- rays of up to SORT_CAP hits: one warp, keys in registers (R per lane, lane l holds positions l R .. l R + R - 1)
-// Keys are (t* bits << 32) | record index; padding keys are all ones and sort last.
+// A key is one 32-bit word: the bits of t* (a non-negative float: its bit pattern orders like its value)
+// with the low KEY_IDX_BITS mantissa bits replaced by the record index.  Sorting these orders the hits
+// by t* up to a relative 2^-14; neighbours whose truncated t* coincide are then put in exact (t*, id)
+// order by a few odd-even exchanges on the full values (rare).  Padding keys are all ones and sort last.
+constexpr int KEY_IDX_BITS = 9;
+static_assert((1 << KEY_IDX_BITS) >= SORT_CAP, "record index must fit the key");
+constexpr uint32_t KEY_IDX_MASK = (1u << KEY_IDX_BITS) - 1u;
+
 template <int R>
-__device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) {
+__device__ __forceinline__ void sort_regs(uint32_t (&k)[R], int lane) {
     constexpr int N = 32 * R;
     // the merge sizes and the cross-lane distances are run-time loops (small code: the instruction cache
     // matters more here than the loop overhead); register indices stay compile-time
@@ -257,9 +264,9 @@ __device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) 
             const bool lower = (lane & lj) == 0;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const unsigned long long o = __shfl_xor_sync(0xffffffffu, k[r], lj);
+                const uint32_t o = __shfl_xor_sync(0xffffffffu, k[r], lj);
                 const bool asc = ((lane * R + r) & kk) == 0;
-                k[r] = ((o < k[r]) == (lower == asc)) ? o : k[r];
+                k[r] = (lower == asc) ? min(k[r], o) : max(k[r], o);
             }
         }
 #pragma unroll
@@ -269,10 +276,9 @@ __device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) 
                 for (int r = 0; r < R; ++r) {
                     if ((r ^ j) > r) {
                         const bool asc = ((lane * R + r) & kk) == 0;
-                        const unsigned long long x = k[r], y = k[r ^ j];
-                        const bool sw = (x > y) == asc;
-                        k[r] = sw ? y : x;
-                        k[r ^ j] = sw ? x : y;
+                        const uint32_t lo = min(k[r], k[r ^ j]), hi = max(k[r], k[r ^ j]);
+                        k[r] = asc ? lo : hi;
+                        k[r ^ j] = asc ? hi : lo;
                     }
                 }
             }
@@ -280,45 +286,47 @@ __device__ __forceinline__ void sort_regs(unsigned long long (&k)[R], int lane) 
     }
 }
 
+// true if record a must come after record b: larger t*, or equal t* and larger Gaussian id
+__device__ __forceinline__ bool rec_after(const float4* __restrict__ rec, uint32_t ka, uint32_t kb) {
+    const float4 a = __ldg(&rec[2 * (ka & KEY_IDX_MASK)]), b = __ldg(&rec[2 * (kb & KEY_IDX_MASK)]);
+    return a.x > b.x || (a.x == b.x && __float_as_uint(a.y) > __float_as_uint(b.y));
+}
+
 template <int R>
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
-    unsigned long long k[R];
+    uint32_t k[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         // load striped (coalesced), the network does not care about the initial arrangement
         const int i = r * 32 + lane;
-        k[r] = i < n ? (((unsigned long long)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (unsigned long long)i) : ~0ull;
+        k[r] = i < n ? ((__float_as_uint(__ldg(&rec[2 * i].x)) & ~KEY_IDX_MASK) | (uint32_t)i) : 0xffffffffu;
     }
     sort_regs<R>(k, lane);
-    // hits with bit-identical t* must ascend in Gaussian id (records arrive in arbitrary order)
     {
+        // neighbours with the same truncated t*: exact order by odd-even exchanges, n rounds at most
         bool tie = false;
 #pragma unroll
-        for (int r = 0; r + 1 < R; ++r) tie = tie || ((uint32_t)(k[r] >> 32) == (uint32_t)(k[r + 1] >> 32) && lane * R + r + 1 < n);
-        const unsigned long long nb = __shfl_down_sync(0xffffffffu, k[0], 1);
-        tie = tie || (lane < 31 && (uint32_t)(k[R - 1] >> 32) == (uint32_t)(nb >> 32) && (lane + 1) * R < n);
+        for (int r = 0; r + 1 < R; ++r) tie = tie || ((k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && lane * R + r + 1 < n);
+        const uint32_t nb = __shfl_down_sync(0xffffffffu, k[0], 1);
+        tie = tie || (lane < 31 && (k[R - 1] >> KEY_IDX_BITS) == (nb >> KEY_IDX_BITS) && (lane + 1) * R < n);
         if (__any_sync(0xffffffffu, tie)) {
-            // rare: odd-even transposition on (t*, id) between neighbours with equal t*, n rounds at most
             for (int round = 0; round < n; ++round) {
                 bool moved = false;
 #pragma unroll
                 for (int r = 0; r + 1 < R; ++r) {
-                    if (lane * R + r + 1 < n && (uint32_t)(k[r] >> 32) == (uint32_t)(k[r + 1] >> 32) &&
-                        __float_as_uint(rec[2 * (uint32_t)k[r]].y) > __float_as_uint(rec[2 * (uint32_t)k[r + 1]].y)) {
-                        const unsigned long long t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
+                    if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(rec, k[r], k[r + 1])) {
+                        const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
                     }
                 }
                 // across the lane boundary: even lanes lead on even rounds, odd lanes on odd rounds
-                const unsigned long long up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
+                const uint32_t up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
                 const bool lead = ((lane ^ round) & 1) == 0;
                 if (lead) {
-                    if (lane < 31 && (lane + 1) * R < n && (uint32_t)(k[R - 1] >> 32) == (uint32_t)(up >> 32) &&
-                        __float_as_uint(rec[2 * (uint32_t)k[R - 1]].y) > __float_as_uint(rec[2 * (uint32_t)up].y)) { k[R - 1] = up; moved = true; }
+                    if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(rec, k[R - 1], up)) { k[R - 1] = up; moved = true; }
                 } else {
-                    if (lane > 0 && lane * R < n && (uint32_t)(dn >> 32) == (uint32_t)(k[0] >> 32) &&
-                        __float_as_uint(rec[2 * (uint32_t)dn].y) > __float_as_uint(rec[2 * (uint32_t)k[0]].y)) { k[0] = dn; moved = true; }
+                    if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(rec, dn, k[0])) { k[0] = dn; moved = true; }
                 }
                 if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
             }
@@ -329,7 +337,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
     float lp = 1.0f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        al[r] = lane * R + r < n ? __ldg(&rec[2 * (uint32_t)k[r]].w) : 0.0f;
+        al[r] = lane * R + r < n ? __ldg(&rec[2 * (k[r] & KEY_IDX_MASK)].w) : 0.0f;
         lp *= 1.0f - al[r];
     }
     float inc = lp;
@@ -351,7 +359,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
 #pragma unroll
         for (int r = R - 1; r >= 0; --r) {
             if (lane * R + r < n) {
-                const float4 c = __ldg(&rec[2 * (uint32_t)k[r] + 1]);
+                const float4 c = __ldg(&rec[2 * (k[r] & KEY_IDX_MASK) + 1]);
                 s0 = fmaf(w0[r], c.x, s0); s1 = fmaf(w0[r], c.y, s1); s2 = fmaf(w0[r], c.z, s2);
             }
         }
@@ -375,7 +383,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
         for (int r = R - 1; r >= 0; --r) {
             const int i = lane * R + r;
             if (i < n) {
-                const uint32_t c = (uint32_t)k[r];
+                const uint32_t c = k[r] & KEY_IDX_MASK;
                 const float4 ra = __ldg(&rec[2 * c]);
                 const float4 rb = __ldg(&rec[2 * c + 1]);
                 const uint32_t slot = __float_as_uint(ra.z);
