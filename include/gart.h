@@ -146,6 +146,27 @@ gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n
                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same tile map for callers that cannot hand over scratch memory (the paper has no counterpart:
+ * this entry point exists for hosts in which device allocations are not possible at call time -- an
+ * engine that gave its whole device budget to its own arena, a plug-in under a memory quota, a loop
+ * that must not touch the allocator).  Arguments, results and errors are those of gart_tile_map; the
+ * scratch is a fixed array of GART_TILE_MAP_STATIC_BYTES inside the library, which every GPU that
+ * loads the library keeps allocated until the process exits.  The call allocates nothing.
+ *   - Limit: gart_tile_map_workspace_bytes(n, width, height, tile_size, cap_pairs) must not exceed
+ *     GART_TILE_MAP_STATIC_BYTES (about n + 3 cap_pairs words: e.g. n = 200k with cap_pairs = 500k);
+ *     larger problems are refused with GART_ERR_WORKSPACE_TOO_SMALL before any work is queued.
+ *   - The first call on a device looks up the array's device address (a host-side query, done with
+ *     that device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the array: calls that may overlap on the GPU (different streams
+ *     without ordering) race on it.  The array keeps the previous call's contents; the tile map
+ *     writes every scratch word before reading it, so nothing has to be cleared.
+ */
+#define GART_TILE_MAP_STATIC_BYTES (8u << 20)
+gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, int64_t n, int32_t width, int32_t height,
+                                 uint32_t *tile_off, uint32_t *pair_gid, int64_t cap_pairs, uint32_t *counts,
+                                 void *stream);
+
+/*
  * Step 3 -- forward ray evaluation (Sec. 3.2-3.3, Eq. 3-8; intermediate buffer of Sec. 4.2-4.3).
  * For every pixel ray and every Gaussian of its tile list: t* = -(o_g.d_g)/(d_g.d_g),
  * alpha = sigma exp(-|o_g + t* d_g|^2 / 2); a hit iff alpha >= alpha_min and t* > 0.  Hits of a

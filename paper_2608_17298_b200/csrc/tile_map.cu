@@ -153,3 +153,42 @@ extern "C" gart_status gart_tile_map(const gart_config* cfg, const int32_t* rect
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// gart_tile_map_static: the tile map for callers that cannot provide scratch memory.
+//
+// Some hosts cannot allocate device memory at the point where they call this library: an engine that
+// hands its whole device budget to its own arena at start-up and forbids later driver allocations,
+// a plug-in running under a memory quota, a real-time loop in which an allocation (which may
+// synchronise the device or fail on a fragmented heap) is not acceptable.  For them the scratch of
+// gart_tile_map lives in a fixed array inside the library image: every GPU that loads libgart.so
+// holds GART_TILE_MAP_STATIC_BYTES of device memory for it until the process exits.
+//
+// The array is shared by every call on a device and keeps the previous call's contents.  Nothing in
+// the tile map relies on zero-initialised scratch (every word is written before it is read), so
+// nothing needs clearing; but two calls that overlap on the GPU (different streams, no ordering
+// between them) would race on it.
+static __device__ __align__(256) unsigned char g_tile_map_scratch[GART_TILE_MAP_STATIC_BYTES];
+
+// In host code the array's name is only a stand-in for the symbol, not a device address: the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device
+// current.
+static void* g_tile_map_scratch_ptr[64] = {nullptr};
+
+extern "C" gart_status gart_tile_map_static(const gart_config* cfg, const int32_t* rect, int64_t n, int32_t width, int32_t height,
+                                            uint32_t* tile_off, uint32_t* pair_gid, int64_t cap_pairs, uint32_t* counts,
+                                            void* stream) {
+    if (n < 0 || cap_pairs < 0 || width <= 0 || height <= 0) return GART_ERR_INVALID_ARG;
+    // sizes beyond the fixed array are refused before anything is launched
+    if (gart_tile_map_workspace_bytes(n, width, height, cfg ? cfg->tile_size : 8, cap_pairs) > (size_t)GART_TILE_MAP_STATIC_BYTES)
+        return GART_ERR_WORKSPACE_TOO_SMALL;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GART_ERR_CUDA;
+    if (!g_tile_map_scratch_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_tile_map_scratch) != cudaSuccess || !p) return GART_ERR_CUDA;
+        g_tile_map_scratch_ptr[dev] = p;
+    }
+    return gart_tile_map(cfg, rect, n, width, height, tile_off, pair_gid, cap_pairs, counts, g_tile_map_scratch_ptr[dev],
+                         (size_t)GART_TILE_MAP_STATIC_BYTES, stream);
+}

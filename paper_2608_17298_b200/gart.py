@@ -27,7 +27,7 @@ GRAD_WORDS = 64
 
 EXPORTS = [
     "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
-    "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_forward_workspace_bytes", "gart_forward",
+    "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_forward_workspace_bytes", "gart_forward",
     "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_read_counts",
     "gart_view_host_arena_bytes", "gart_view_host",
 ]
@@ -77,6 +77,8 @@ def lib():
         L.gart_tile_map_workspace_bytes.restype = sz
         L.gart_tile_map_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
         L.gart_tile_map.argtypes = [vp, vp, i64, i32, i32, vp, vp, i64, vp, vp, sz, vp]
+        L.gart_tile_map_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, i64, vp, vp]
+        L.gart_tile_map_static.restype = C.c_int
         L.gart_forward_workspace_bytes.restype = sz
         L.gart_forward_workspace_bytes.argtypes = [i32, i32, i32, i64, i64]
         L.gart_forward.argtypes = [vp] * 8 + [i64] + [vp] * 10 + [i64] + [vp] * 5 + [sz, vp]
@@ -222,6 +224,20 @@ def gart_tile_map(cfg: Config, rect, n, cam, tile_off, pair_gid, cap_pairs, coun
     _check(lib().gart_tile_map(C.byref(c), _dev(rect, torch.int32, "rect"), int(n), int(cam.width), int(cam.height),
                                _dev(tile_off, torch.int32, "tile_off"), _dev(pair_gid, torch.int32, "pair_gid"),
                                int(cap_pairs), _dev(counts, torch.int32, "counts"), wp, wb, _stream_ptr(stream)), "gart_tile_map")
+
+
+TILE_MAP_STATIC_BYTES = 8 << 20
+
+
+def gart_tile_map_static(cfg: Config, rect, n, cam, tile_off, pair_gid, cap_pairs, counts, stream=None):
+    """gart_tile_map without a workspace argument: the scratch is a fixed array inside the library
+    (for callers that cannot allocate device memory when they call).  Problems whose scratch need
+    exceeds TILE_MAP_STATIC_BYTES are refused with GART_ERR_WORKSPACE_TOO_SMALL."""
+    c = cfg.c()
+    _check(lib().gart_tile_map_static(C.byref(c), _dev(rect, torch.int32, "rect"), int(n), int(cam.width), int(cam.height),
+                                      _dev(tile_off, torch.int32, "tile_off"), _dev(pair_gid, torch.int32, "pair_gid"),
+                                      int(cap_pairs), _dev(counts, torch.int32, "counts"), _stream_ptr(stream)),
+           "gart_tile_map_static")
 
 
 def gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits) -> int:
