@@ -250,6 +250,110 @@ __device__ __forceinline__ void sh_basis(const float3 d, float* Y) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Asynchronous bulk copies global -> shared with completion on an mbarrier.  Every wait is bounded.
+constexpr uint32_t ASYNC_WAIT_LIMIT = 1u << 22;   // polls before a wait gives up (then the caller sets an error bit)
+
+// ---- mbarrier / bulk copy (shared::cta addresses as 32-bit)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < ASYNC_WAIT_LIMIT; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
+// Orders this thread's earlier shared-memory accesses (generic proxy) before later accesses of the
+// asynchronous proxy: issued before a bulk copy overwrites a buffer that was just read.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// SH coefficients of a pair's Gaussian and the pair's dL/dsh accumulators, in registers.  For an even
+// number of coefficients both are kept as (k, k+1) pairs per channel, so that colour evaluation and
+// gradient accumulation issue packed two-wide FMAs (fma.rn.f32x2: half the issue slots).
+template <int K, bool PACKED = (K % 2 == 0)>
+struct ShRegs;
+
+template <int K>
+struct ShRegs<K, false> {
+    float sh[3 * K], acc[3 * K];
+    __device__ __forceinline__ void set(int e, float v) { sh[e] = v; acc[e] = 0.0f; }   // e = 3 k + channel
+    __device__ __forceinline__ float word(int e) const { return acc[e]; }
+    __device__ __forceinline__ void colour(const float* Y, float* c) const {
+        c[0] = 0.5f; c[1] = 0.5f; c[2] = 0.5f;
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            c[0] = fmaf(Y[k], sh[3 * k], c[0]);
+            c[1] = fmaf(Y[k], sh[3 * k + 1], c[1]);
+            c[2] = fmaf(Y[k], sh[3 * k + 2], c[2]);
+        }
+    }
+    __device__ __forceinline__ void accumulate(const float* Y, const float* w) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            acc[3 * k] = fmaf(Y[k], w[0], acc[3 * k]);
+            acc[3 * k + 1] = fmaf(Y[k], w[1], acc[3 * k + 1]);
+            acc[3 * k + 2] = fmaf(Y[k], w[2], acc[3 * k + 2]);
+        }
+    }
+};
+
+template <int K>
+struct ShRegs<K, true> {
+    float2 sh[3][K / 2], acc[3][K / 2];
+    __device__ __forceinline__ void set(int e, float v) {
+        const int k = e / 3, c = e % 3;
+        if (k & 1) { sh[c][k >> 1].y = v; acc[c][k >> 1].y = 0.0f; }
+        else { sh[c][k >> 1].x = v; acc[c][k >> 1].x = 0.0f; }
+    }
+    __device__ __forceinline__ float word(int e) const {
+        const int k = e / 3, c = e % 3;
+        return (k & 1) ? acc[c][k >> 1].y : acc[c][k >> 1].x;
+    }
+    __device__ __forceinline__ void colour(const float* Y, float* c) const {
+        float2 a0 = make_float2(0.5f, 0.0f), a1 = a0, a2 = a0;
+#pragma unroll
+        for (int i = 0; i < K / 2; ++i) {
+            const float2 y = make_float2(Y[2 * i], Y[2 * i + 1]);
+            a0 = __ffma2_rn(y, sh[0][i], a0);
+            a1 = __ffma2_rn(y, sh[1][i], a1);
+            a2 = __ffma2_rn(y, sh[2][i], a2);
+        }
+        c[0] = a0.x + a0.y; c[1] = a1.x + a1.y; c[2] = a2.x + a2.y;
+    }
+    __device__ __forceinline__ void accumulate(const float* Y, const float* w) {
+        const float2 w0 = make_float2(w[0], w[0]), w1 = make_float2(w[1], w[1]), w2 = make_float2(w[2], w[2]);
+#pragma unroll
+        for (int i = 0; i < K / 2; ++i) {
+            const float2 y = make_float2(Y[2 * i], Y[2 * i + 1]);
+            acc[0][i] = __ffma2_rn(y, w0, acc[0][i]);
+            acc[1][i] = __ffma2_rn(y, w1, acc[1][i]);
+            acc[2][i] = __ffma2_rn(y, w2, acc[2][i]);
+        }
+    }
+};
+
+
+// ---------------------------------------------------------------------------------------------
 // Exclusive scan of f(0..n_cap-1) into out[0..n_cap] (uint32; out[n_cap] = total) with three
 // launches and no waiting between blocks: per-block sums, one block scans the sums, per-block
 // rescan.  Sums are carried in 64 bits so that an overflowing total is seen (total64_out).

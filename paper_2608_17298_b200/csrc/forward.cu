@@ -166,17 +166,48 @@ __global__ void hits_total_kernel(const uint64_t* total_slots, const uint64_t* t
 }
 
 // ------------------------------------------------------------------------------------------ phase 3
-constexpr int EVAL_THREADS = 128;
+constexpr int EVAL_WARPS = 4;
+constexpr int EVAL_THREADS = EVAL_WARPS * 32;
 
+// What a lane needs to know about its pair of a rank group (read coalesced from the rank-ordered copies).
+template <int MW>
+struct EvalDesc {
+    PairMask<MW> pm;
+    uint32_t sid, gstart;
+    int c;      // hits of this lane's pair
+    int cmax;   // hits of the group's first pair (the largest)
+};
+
+template <int MW>
+__device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
+                                                       const uint32_t* __restrict__ rank_gstart, uint32_t begin, uint32_t n,
+                                                       uint32_t r0, int lane) {
+    EvalDesc<MW> d;
+    const bool act = r0 < n && r0 + lane < n;
+    const uint32_t q = begin + r0 + lane;
+    d.pm.load(rank_mask, act ? q : 0u, act);
+    d.c = d.pm.count();
+    d.sid = act ? __ldg(rank_sid + q) : 0u;
+    d.gstart = act ? __ldg(rank_gstart + q) : 0u;
+    d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
+    return d;
+}
+
+// Block per tile, one thread per (tile, Gaussian) pair; warps walk the rank groups.  The records of the
+// next group's Gaussians are copied into shared memory (bulk asynchronous copy per lane, completion on an
+// mbarrier) while the current group is evaluated.
 template <int TS, int DEG>
 __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
-                                                                const uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3, RS4 = (20 + SW + 3) / 4;
+                                                                uint32_t* __restrict__ counts) {
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3, PF4 = (20 + SW + 3) / 4;
+    constexpr int PSTR = PF4 | 1;   // odd lane stride: the lanes' 16-byte reads fall into distinct banks
     __shared__ __align__(16) float spix[NT * PW];
+    extern __shared__ __align__(128) float4 spar[];   // [EVAL_THREADS][PSTR] staged records
+    __shared__ __align__(8) uint64_t bars[EVAL_WARPS];
     __shared__ uint32_t sro[NT];
     __shared__ uint32_t scur[NT];
     if (counts[GART_CNT_ERROR]) return;
@@ -185,6 +216,11 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     if (n == 0) return;
     const int tx = tile % cam.tiles_x, ty = tile / cam.tiles_x;
     const int x0 = tx * TS, y0 = ty * TS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        mbar_init(smem_u32(&bars[warp]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     for (int p = threadIdx.x; p < NT; p += EVAL_THREADS) {
         const int x = x0 + p % TS, y = y0 + p / TS;
         float Y[K];
@@ -196,25 +232,45 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     }
     __syncthreads();
     const uint32_t lt_base = tile_lt_base[tile];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (uint32_t r0 = warp * 32; r0 < n; r0 += EVAL_THREADS) {
-        const bool act = r0 + lane < n;
-        const uint32_t q = begin + r0 + lane;
-        PairMask<MW> pm;
-        pm.load(rank_mask, act ? q : 0u, act);
-        const int c = pm.count();
-        if (__ballot_sync(0xffffffffu, c != 0) == 0u) break;   // ranks descend in hit count: nothing left in this tile
-        if (c == 0) continue;
-        const uint32_t sid = __ldg(rank_sid + q);
-        const uint32_t gid = __ldg(gid_of_slot + sid);
-        const float4* rp = rec + (size_t)sid * RS4;
-        const PreRec P = load_pre(rp);
-        float shc[SW];
-        load_sh<SW>(rp, shc);
-        uint32_t slot = lt_base + __ldg(rank_gstart + q) + lane;
+    float4* my_par = spar + (size_t)(warp * 32 + lane) * PSTR;
+    const uint32_t par_addr = smem_u32(my_par), bar_addr = smem_u32(&bars[warp]);
+    uint32_t phase = 0;
+    auto issue_params = [&](const EvalDesc<MW>& d) {
+        const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
+        if (lane == 0) mbar_expect_tx(bar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
+        if (d.c != 0) bulk_g2s(par_addr, rec + (size_t)d.sid * PF4, (uint32_t)(PF4 * 16), bar_addr);
+    };
+
+    uint32_t r0 = warp * 32;
+    EvalDesc<MW> cur = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0, lane);
+    if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
+    issue_params(cur);
+    EvalDesc<MW> nxt = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + EVAL_THREADS, lane);
+    while (true) {
+        const EvalDesc<MW> nxt2 = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * EVAL_THREADS, lane);
+        const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr, phase))) {
+            // the copy never completed: report, give it a second bounded chance to land before this
+            // warp's shared memory may be released, and stop
+            if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
+            mbar_wait_bounded(bar_addr, phase);
+            return;
+        }
+        phase ^= 1u;
+        const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale for lanes without hits: unused)
+        float shc[SW + 3];
+#pragma unroll
+        for (int q = 0; q < (SW + 3) / 4; ++q) {
+            const float4 t = my_par[5 + q];
+            shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
+        }
+        fence_proxy_async();
+        __syncwarp();   // every lane has read its record: the buffer may be overwritten
+        if (nxt.cmax != 0) issue_params(nxt);
+        uint32_t slot = lt_base + cur.gstart + lane;
         const int bx = x0 - P.ix, by = y0 - P.iy;
-        for (int e = 0; e < c; ++e) {
-            const int p = pm.next();
+        for (int e = 0; e < cur.c; ++e) {
+            const int p = cur.pm.next();
             const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
             const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
             float Y[PW];
@@ -231,11 +287,15 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                 c2 = fmaf(Y[k], shc[3 * k + 2], c2);
             }
             const uint32_t pos = atomicAdd(&scur[p], 1u);
-            float4* rec = recs + ((size_t)sro[p] + pos) * 2;
-            rec[0] = make_float4(t, __uint_as_float(gid), __uint_as_float(slot), r.alpha);
-            rec[1] = make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f);
+            float4* out = recs + ((size_t)sro[p] + pos) * 2;
+            out[0] = make_float4(t, __uint_as_float(gid), __uint_as_float(slot), r.alpha);
+            out[1] = make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f);
             slot += 32u;
         }
+        if (nxt.cmax == 0) break;
+        cur = nxt;
+        nxt = nxt2;
+        r0 += EVAL_THREADS;
     }
 }
 
@@ -575,10 +635,15 @@ template <int TS>
 static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                const uint32_t* tile_lt_base, const uint32_t* ray_off,
-                               const CamF& cam, const ForwardWs& w, const uint32_t* counts) {
-#define GART_EVAL(D)                                                                                                      \
-    fwd_eval_kernel<TS, D><<<T, EVAL_THREADS, 0, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart,    \
-                                                       tile_lt_base, ray_off, cam, w.recs, counts)
+                               const CamF& cam, const ForwardWs& w, uint32_t* counts) {
+#define GART_EVAL(D)                                                                                                        \
+    {                                                                                                                      \
+        auto kern = fwd_eval_kernel<TS, D>;                                                                                \
+        constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
+        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cam, \
+                                            w.recs, counts);                                                               \
+    }
     switch (deg) {
         case 0: GART_EVAL(0); break;
         case 1: GART_EVAL(1); break;
