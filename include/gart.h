@@ -194,7 +194,8 @@ gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, in
  *   lt         [cap_hits,4] out: per hit (R_r, R_g, R_b, T): colour composited BEHIND the hit
  *              (including the background term) and transmittance in front of it.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
- *              compositing order, the Gaussian id and LT slot of each hit.
+ *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
+ *              baseline and parity checks read the two lists: pass NULL for both to skip them.
  *   counts: HITS, LT_SLOTS, MAX_RAY_HITS.  If L > cap_hits, GART_ERRBIT_HITS is set and color,
  *   t_final, lt, ray_gid, ray_slot are not written.  Because ranks descend in hit count,
  *   L <= H + 32 tile_size^2 per non-empty tile, and H <= S (the slot bound of gart_tile_map), so

@@ -8,7 +8,7 @@ struct HostArena {
     float *mean, *scale, *quat, *opacity, *sh, *pre, *color, *t_final, *lt, *dL_dC, *grad;
     int32_t* rect;
     uint8_t* cls;
-    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_sid, *rank_mask, *rank_gstart, *tile_lt_base, *slot_of_gid, *gid_of_slot, *hit_count, *ray_off, *ray_gid, *ray_slot;
+    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_sid, *rank_mask, *rank_gstart, *tile_lt_base, *slot_of_gid, *gid_of_slot, *hit_count, *ray_off;
     void* ws;
     size_t ws_bytes;
     size_t bytes;
@@ -34,7 +34,6 @@ static HostArena arena_layout(void* base, int64_t n, int K, int width, int heigh
     a.tile_lt_base = (uint32_t*)take((size_t)(T + 1) * 4);
     a.color = (float*)take(hw * 12); a.t_final = (float*)take(hw * 4); a.hit_count = (uint32_t*)take(hw * 4);
     a.lt = (float*)take(ch * 16); a.ray_off = (uint32_t*)take((hw + 1) * 4);
-    a.ray_gid = (uint32_t*)take(ch * 4); a.ray_slot = (uint32_t*)take(ch * 4);
     a.dL_dC = (float*)take(hw * 12); a.grad = (float*)take(nn * GART_GRAD_WORDS * 4);
     const size_t w0 = gart_bounds_workspace_bytes(nn);
     const size_t w1 = gart_tile_map_workspace_bytes(nn, width, height, ts, cap_pairs);
@@ -99,7 +98,7 @@ extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussia
     s = gart_tile_map(cfg, a.rect, n, cam->width, cam->height, a.tile_off, a.pair_gid, cap_pairs, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     s = gart_forward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count, a.pair_mask,
-                     a.pair_order, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, a.ray_gid, a.ray_slot, a.counts, a.ws, a.ws_bytes, stream);
+                     a.pair_order, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, nullptr, nullptr, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     s = gart_backward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, a.dL_dC,
                       a.grad, a.counts, a.ws, a.ws_bytes, stream);

@@ -13,6 +13,8 @@
 
 namespace gart {
 
+constexpr int PRE_TMP_F4 = 7;   // float4 per Gaussian in the id-ordered temporary: 5 of the record, quaternion, scale + opacity
+
 struct CamD {
     int width, height;
     double fx, fy, cx, cy;
@@ -132,8 +134,12 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
         }
         reinterpret_cast<int4*>(rect)[i] = make_int4(x0, y0, x1, y1);
         cls[i] = (uint8_t)c;
-        float4* p = pre4 + (size_t)i * 5;
+        float4* p = pre4 + (size_t)i * PRE_TMP_F4;
         p[0] = q0; p[1] = q1; p[2] = q2; p[3] = q3; p[4] = q4;
+        if (vis) {   // quaternion, scale, opacity ride along so that the gather reads one contiguous piece
+            p[5] = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
+            p[6] = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
+        }
         keys[i] = vis ? (uint32_t)((y0 / ts) * tiles_x + x0 / ts) : key_none;
         vals[i] = (uint32_t)i;
     }
@@ -149,8 +155,6 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
 __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4, int sw, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
                                                              const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
-                                                             const float* __restrict__ quat, const float* __restrict__ scale,
-                                                             const float* __restrict__ opacity,
                                                              float4* __restrict__ rec, float4* __restrict__ qs,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -165,12 +169,12 @@ __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4,
     }
     if (!vis) return;
     if (q == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
-        qs[2 * slot] = make_float4(quat[4 * (size_t)gid], quat[4 * (size_t)gid + 1], quat[4 * (size_t)gid + 2], quat[4 * (size_t)gid + 3]);
-        qs[2 * slot + 1] = make_float4(scale[3 * (size_t)gid], scale[3 * (size_t)gid + 1], scale[3 * (size_t)gid + 2], opacity[gid]);
+        qs[2 * slot] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 5];
+        qs[2 * slot + 1] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 6];
     }
     float4 v;
     if (q < 5) {
-        v = pre_tmp[(size_t)gid * 5 + q];
+        v = pre_tmp[(size_t)gid * PRE_TMP_F4 + q];
     } else {
         const int e = (q - 5) * 4;
         const float* sp = sh + (size_t)gid * sw;
@@ -197,7 +201,7 @@ static BoundsWs bounds_layout(void* base, int64_t n) {
     auto take = [&](size_t b) { void* r = p ? (void*)(p + off) : nullptr; off += align256(b); return r; };
     const int64_t nn = n > 0 ? n : 1;
     w.total64 = (uint64_t*)take(256);
-    w.pre_tmp = (float4*)take((size_t)nn * 80);
+    w.pre_tmp = (float4*)take((size_t)nn * PRE_TMP_F4 * 16);
     w.keys0 = (uint32_t*)take((size_t)nn * 4); w.keys1 = (uint32_t*)take((size_t)nn * 4);
     w.vals0 = (uint32_t*)take((size_t)nn * 4); w.vals1 = (uint32_t*)take((size_t)nn * 4);
     w.table = (uint32_t*)take(radix_table_bytes(nn));
@@ -267,7 +271,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     const int rs4 = rec_f4(g->sh_degree);
     const int64_t gthreads = g->n * rs4;
     gather_records_kernel<<<(unsigned)ceil_div(gthreads, 256), 256, 0, st>>>(g->n, rs4, 3 * K, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh,
-                                                                            g->quat, g->scale, g->opacity, reinterpret_cast<float4*>(pre),
+                                                                            reinterpret_cast<float4*>(pre),
                                                                             reinterpret_cast<float4*>(pre) + (size_t)g->n * rs4, slot_of_gid,
                                                                             gid_of_slot);
     GART_LAUNCH_CHECK();

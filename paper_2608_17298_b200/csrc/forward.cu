@@ -448,8 +448,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const float4 rb = __ldg(&rec[2 * c + 1]);
                 const uint32_t slot = __float_as_uint(ra.z);
                 lt[slot] = make_float4(k0, k1, k2, Ts[r]);
-                ray_gid[b + i] = __float_as_uint(ra.y);
-                ray_slot[b + i] = slot;
+                if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
                 const float wgt = Ts[r] * al[r];
                 k0 = fmaf(wgt, rb.x, k0); k1 = fmaf(wgt, rb.y, k1); k2 = fmaf(wgt, rb.z, k2);
             }
@@ -562,8 +561,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
             lt[slot] = make_float4(k0 + e0, k1 + e1, k2 + e2, T);
-            ray_gid[b + i] = __float_as_uint(ra.y);
-            ray_slot[b + i] = slot;
+            if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
         k1 += __shfl_sync(0xffffffffu, s1, 31);
@@ -679,7 +677,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
     if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_sid || !rank_mask || !rank_gstart || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
-    if (cap_hits > 0 && (!lt || !ray_gid || !ray_slot)) return GART_ERR_INVALID_ARG;
+    if (cap_hits > 0 && (!lt || (ray_gid == nullptr) != (ray_slot == nullptr))) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     const int ts = cfg->tile_size;
     const CamF cf = make_camf(cam, ts);

@@ -366,11 +366,12 @@ def run_bounds_tile_map(cfg, g, cam, buf: ViewBuffers, stream=None):
     gart_tile_map(cfg, buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.counts, buf.workspace, stream)
 
 
-def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None):
+def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None, ray_lists=True):
+    """ray_lists=False skips the per-ray ordered hit lists (needed only by the atomic baseline and by parity checks)."""
     gart_forward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color,
                  buf.t_final, buf.hit_count, buf.pair_mask, buf.pair_order, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
-                 buf.tile_lt_base, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.counts, buf.workspace,
-                 stream)
+                 buf.tile_lt_base, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid if ray_lists else None,
+                 buf.ray_slot if ray_lists else None, buf.counts, buf.workspace, stream)
 
 
 def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
