@@ -191,8 +191,12 @@ gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, in
  *              group's whole block is one contiguous range (one bulk copy), every hit owns one slot
  *              (forward writes never collide), and a group occupies 32 x (its largest hit count)
  *              entries: L = tile_lt_base[T] >= H counts the padding.
- *   lt         [cap_hits,4] out: per hit (R_r, R_g, R_b, T): colour composited BEHIND the hit
- *              (including the background term) and transmittance in front of it.
+ *   lt         [cap_hits,4] out: per hit, with w = T alpha its blending weight (T the transmittance
+ *              in front of it), c its clamped colour and B the colour composited BEHIND it
+ *              (background term included): words 0..2 = w c - alpha / (1 - alpha) B, which is
+ *              alpha dC/dalpha by Eq. 6-8; word 3 = w, whose three low mantissa bits are replaced by
+ *              flags "channel r, g, b of c is not clamped".  This is all the backward pass needs of
+ *              the ray's state, and nothing in it is a difference of nearly equal sums.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
  *              baseline and parity checks read the two lists: pass NULL for both to skip them.

@@ -7,9 +7,10 @@
 // these blocks into shared memory with bulk asynchronous copies (cp.async.bulk, completion on an
 // mbarrier), double buffered, so that tens of KB of LT data per SM are in flight while the warp
 // computes; lanes then read their entry with conflict-free 16-byte shared loads.  The records of the
-// next group's Gaussians (evaluation record + SH coefficients, one contiguous piece per slot of the
-// view's order) arrive the same way.  A thread accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) of its
-// pair in registers and adds them to the accumulation record of the Gaussian's slot with one vector
+// next group's Gaussians (80 bytes each, the head of the slot's record) arrive the same way.  The LT
+// entry carries alpha dC/dalpha and the blending weight, so a hit costs the geometry of the maximum-
+// response point, one dot product and the SH outer product: no exponential, no colour evaluation.
+// A thread accumulates (v, Q, sum alpha dL/dalpha, dL/dsh) of its pair in registers and adds them to the accumulation record of the Gaussian's slot with one vector
 // atomic per 16 bytes -- no per-pixel atomics; slots are ordered by tile, so neighbouring tiles update
 // neighbouring memory.  A per-Gaussian pass then converts the moments into d mean, d scale, d quat,
 // d opacity and writes the caller's gradient records.
@@ -19,14 +20,24 @@ namespace gart {
 
 constexpr int BWD_WARPS = 4;
 constexpr int BWD_THREADS = BWD_WARPS * 32;
-constexpr int BWD_CHUNK = 16;                          // LT entries per lane and per pipeline stage
+constexpr int BWD_CHUNK = 8;                           // LT entries per lane and per pipeline stage
 constexpr int BWD_STAGE_F4 = BWD_CHUNK * 32;           // float4 per stage (8 KB)
-constexpr int BWD_LT_SMEM = BWD_WARPS * 2 * BWD_STAGE_F4 * 16;
-constexpr int bwd_dyn_smem(int sw) { return BWD_LT_SMEM + BWD_THREADS * (((20 + sw + 3) / 4) | 1) * 16; }
+constexpr int BWD_STAGES = 3;                          // LT pipeline depth per warp
+constexpr int BWD_LT_SMEM = BWD_WARPS * BWD_STAGES * BWD_STAGE_F4 * 16;
+constexpr int BWD_PF4 = 5;                             // float4 per lane of the staged evaluation record
+constexpr int BWD_DYN_SMEM = BWD_LT_SMEM + BWD_THREADS * BWD_PF4 * 16;
 
-template <int K>
+// Per-pixel data of the tile in shared memory: two float4 per pixel, (d.x, d.y, d.z, x) and (g.r, g.g, g.b, y)
+// with d the unit ray direction, g = dL/dC and (x, y) the pixel's position in the tile.  Lanes of a warp read
+// DIFFERENT pixels at the same time, so a single copy suffers bank conflicts at random; with 8 copies, copy j
+// laid out in the 16-byte bank group j only and lane l reading copy l mod 8, the 8 lanes that a 16-byte shared
+// load serves together never collide.  (Tiles of 256 pixels keep one copy, 3 float4 apart.)
+template <int TS>
 struct PixLayout {
-    static constexpr int W = (K + 3 + 3) & ~3;   // floats per pixel record: Y[K], g[3], zero padding
+    static constexpr int COPIES = TS == 8 ? 8 : 1;
+    static constexpr int STRIDE = COPIES == 1 ? 3 : 2;                 // float4 per pixel within a copy
+    static constexpr int F4 = TS * TS * STRIDE * COPIES;               // float4 in all
+    __device__ static __forceinline__ int index(int p, int h, int copy) { return (p * STRIDE + h) * COPIES + copy; }
 };
 
 // Descriptor of one rank group as seen by a lane (read from the rank-ordered copies: coalesced).
@@ -57,36 +68,18 @@ __device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__
 
 // Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
 // geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz), geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh.
-template <int TS, int K, int PW>
-__device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* geo, const float* spix, int bx, int by, int p,
+template <int TS, int K>
+__device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* geo, const float4* spix, float fbx, float fby, int p,
                                         const float4 L) {
-    const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
-    const float* rec = spix + p * PW;
+    const float4 pa = spix[PixLayout<TS>::index(p, 0, 0)], pb = spix[PixLayout<TS>::index(p, 1, 0)];   // spix points at the lane's copy
+    const RayGeo r = ray_geo(P, (fbx + pa.w) - P.rx, (fby + pb.w) - P.ry);   // small integers: the sums are exact
     float Y[K];
-    if (K % 4 == 0) {
-#pragma unroll
-        for (int k4 = 0; k4 < K / 4; ++k4) {
-            const float4 t = reinterpret_cast<const float4*>(rec)[k4];
-            Y[4 * k4] = t.x; Y[4 * k4 + 1] = t.y; Y[4 * k4 + 2] = t.z; Y[4 * k4 + 3] = t.w;
-        }
-    } else {
-#pragma unroll
-        for (int kk = 0; kk < K; ++kk) Y[kk] = rec[kk];
-    }
-    const float3 g = make_float3(rec[K], rec[K + 1], rec[K + 2]);
-    float c[3], w[3];
-    R.colour(Y, c);
-    const float T = L.w, Ta = T * r.alpha;
-    const float inv = fast_rcp(1.0f - r.alpha);
-    w[0] = c[0] > 0.0f ? Ta * g.x : 0.0f;
-    w[1] = c[1] > 0.0f ? Ta * g.y : 0.0f;
-    w[2] = c[2] > 0.0f ? Ta * g.z : 0.0f;
-    const float t0 = fmaf(T, fmaxf(c[0], 0.0f), -L.x * inv);
-    const float t1 = fmaf(T, fmaxf(c[1], 0.0f), -L.y * inv);
-    const float t2 = fmaf(T, fmaxf(c[2], 0.0f), -L.z * inv);
-    const float dalpha = fmaf(g.x, t0, fmaf(g.y, t1, g.z * t2));
+    sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
+    const float3 g = make_float3(pb.x, pb.y, pb.z);
+    float w[3];
+    lt_weights(L, g, w);
     R.accumulate(Y, w);
-    const float ad = r.alpha * dalpha;
+    const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
     geo[9] += ad;
     const float G = -0.5f * ad;
     const float3 xg = ray_xg(r);
@@ -97,21 +90,21 @@ __device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* ge
 }
 
 template <int TS, int DEG>
-__global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __restrict__ rec,
+__global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4* __restrict__ rec,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
                                                                 float* __restrict__ gacc, uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = PixLayout<K>::W;
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
-    // record (evaluation record + SH coefficients) of a lane's Gaussian, staged through shared memory one
-    // group ahead; PF4 float4 per lane
-    constexpr int PF4 = (20 + SW + 3) / 4;
-    constexpr int PSTR = PF4 | 1;   // lane stride in the buffer, odd: the lanes' 16-byte reads fall into distinct banks
-    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][PF4] parameters
-    __shared__ __align__(16) float spix[NT * PW];
-    __shared__ __align__(8) uint64_t bars[BWD_WARPS][3];
+    // evaluation record of a lane's Gaussian (the first 5 float4 of the slot's record), staged through shared
+    // memory one group ahead
+    constexpr int PF4 = BWD_PF4, RS4 = (20 + SW + 3) / 4;
+    constexpr int PSTR = PF4;       // lane stride in the buffer, odd: the lanes' 16-byte reads fall into distinct banks
+    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][5] evaluation records
+    __shared__ __align__(16) float4 spix[PIXF4];
+    __shared__ __align__(8) uint64_t bars[BWD_WARPS][BWD_STAGES];   // one per LT stage
     if (counts[GART_CNT_ERROR]) return;
     const int tile = blockIdx.x;
     const uint32_t begin = tile_off[tile], n = tile_off[tile + 1] - begin;
@@ -120,99 +113,103 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
     const int x0 = tx * TS, y0 = ty * TS;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (lane == 0) {
-        mbar_init(smem_u32(&bars[warp][0]), 1);
-        mbar_init(smem_u32(&bars[warp][1]), 1);
-        mbar_init(smem_u32(&bars[warp][2]), 1);
+#pragma unroll
+        for (int q = 0; q < BWD_STAGES; ++q) mbar_init(smem_u32(&bars[warp][q]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // per-pixel data of the tile: SH basis of the ray direction and the upstream gradient
-    for (int p = threadIdx.x; p < NT; p += BWD_THREADS) {
+    // per-pixel data of the tile: ray direction, upstream gradient, position in the tile
+    for (int t = threadIdx.x; t < 2 * NT; t += BWD_THREADS) {
+        const int p = t >> 1, h = t & 1;
         const int x = x0 + p % TS, y = y0 + p / TS;
-        float* rec = spix + p * PW;
+        float4 v = make_float4(0.f, 0.f, 0.f, h ? (float)(p / TS) : (float)(p % TS));
         if (x < cam.width && y < cam.height) {
-            float Y[K];
-            sh_basis<K>(pixel_dir(cam, x, y), Y);
-#pragma unroll
-            for (int k = 0; k < K; ++k) rec[k] = Y[k];
-            const float* gp = dL_dC + ((size_t)y * cam.width + x) * 3;
-            rec[K] = gp[0]; rec[K + 1] = gp[1]; rec[K + 2] = gp[2];
-        } else {
-#pragma unroll
-            for (int k = 0; k < K + 3; ++k) rec[k] = 0.0f;
+            if (h) {
+                const float* gp = dL_dC + ((size_t)y * cam.width + x) * 3;
+                v.x = gp[0]; v.y = gp[1]; v.z = gp[2];
+            } else {
+                const float3 d = pixel_dir(cam, x, y);
+                v.x = d.x; v.y = d.y; v.z = d.z;
+            }
         }
+#pragma unroll
+        for (int c = 0; c < PixLayout<TS>::COPIES; ++c) spix[PixLayout<TS>::index(p, h, c)] = v;
     }
     __syncthreads();
 
     const float4* lt_tile = lt + tile_lt_base[tile];
-    float4* my_stage = dyn + (size_t)warp * 2 * BWD_STAGE_F4;
-    float4* my_par = dyn + (size_t)BWD_WARPS * 2 * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PSTR;
+    const float4* spix_lane = spix + (lane & (PixLayout<TS>::COPIES - 1));
+    float4* my_stage = dyn + (size_t)warp * BWD_STAGES * BWD_STAGE_F4;
+    float4* my_par = dyn + (size_t)BWD_WARPS * BWD_STAGES * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PSTR;
     const uint32_t stage_addr = smem_u32(my_stage);
     const uint32_t par_addr = smem_u32(my_par);
     const uint32_t bar_addr = smem_u32(&bars[warp][0]);
-    const uint32_t pbar_addr = bar_addr + 16u;
-    uint32_t unit = 0;     // LT pipeline units (chunks) consumed so far by this warp: stage = unit & 1, parity = (unit >> 1) & 1
-    uint32_t pphase = 0;   // parity of the parameter barrier
+    const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
+    // LT pipeline: unit u (a chunk of BWD_CHUNK entries per lane) uses stage u % BWD_STAGES, and the wait for
+    // it uses parity (u / BWD_STAGES) & 1.  `unit` counts the units consumed, `produced` the units whose copy
+    // has been issued; the producer cursor (pw, pk) = (group relative to the current one, chunk) runs up to
+    // BWD_STAGES units and two groups ahead of the consumer.
+    uint32_t unit = 0, produced = 0;
+    int pw = 0, pk = 0;
 
-    // copy chunk `k` of a group's LT block into the stage that unit number `u` will use
-    auto issue = [&](const GroupDesc<MW>& d, int k, uint32_t u) {
-        if (lane == 0) {
-            const int ne = min(BWD_CHUNK, d.cmax - k * BWD_CHUNK);
-            const uint32_t bytes = (uint32_t)ne * 512u, s = u & 1u;
-            mbar_expect_tx(bar_addr + 8u * s, bytes);
-            bulk_g2s(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + d.gstart + (size_t)k * BWD_STAGE_F4, bytes, bar_addr + 8u * s);
+    // issue copies while fewer than BWD_STAGES units are in flight; looks at most `maxw` groups ahead of the current one
+    auto produce = [&](const GroupDesc<MW>& a, const GroupDesc<MW>& b, const GroupDesc<MW>& c, const int maxw) {
+        while (produced - unit < (uint32_t)BWD_STAGES && pw <= maxw) {
+            int cm;
+            uint32_t gs;
+            if (pw == 0) { cm = a.cmax; gs = a.gstart; }
+            else if (pw == 1) { cm = b.cmax; gs = b.gstart; }
+            else { cm = c.cmax; gs = c.gstart; }
+            if (cm == 0) break;                                   // ranks descend in hit count: no later group has hits
+            if (pk * BWD_CHUNK >= cm) { ++pw; pk = 0; continue; }
+            if (lane == 0) {
+                const int ne = min(BWD_CHUNK, cm - pk * BWD_CHUNK);
+                const uint32_t bytes = (uint32_t)ne * 512u, s = produced % BWD_STAGES;
+                mbar_expect_tx(bar_addr + 8u * s, bytes);
+                bulk_g2s_hint(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + gs + (size_t)pk * BWD_STAGE_F4, bytes, bar_addr + 8u * s, pol_stream);
+            }
+            ++produced;
+            ++pk;
         }
     };
-    // copy the Gaussian records and SH coefficients of a group's pairs into the parameter buffer
+    // copy the evaluation records of a group's Gaussians into the parameter buffer
     auto issue_params = [&](const GroupDesc<MW>& d) {
-        const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
-        if (lane == 0) mbar_expect_tx(pbar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
-        if (d.c != 0) bulk_g2s(par_addr, rec + (size_t)d.sid * PF4, (uint32_t)(PF4 * 16), pbar_addr);
+        if (d.c != 0) {
+            const float4* src = rec + (size_t)d.sid * RS4;
+#pragma unroll
+            for (int q = 0; q < PF4; ++q) cp_async16(par_addr + 16u * q, src + q);
+        }
     };
     auto fail = [&]() {
         // a copy never completed: report, give copies that may still be in flight a second bounded
         // chance to land before this warp's shared memory may be released, and stop
         if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
-        mbar_wait_bounded(bar_addr, (unit >> 1) & 1u);
-        mbar_wait_bounded(bar_addr + 8u, (unit >> 1) & 1u);
-        mbar_wait_bounded(pbar_addr, pphase);
+        for (uint32_t u = unit; u != produced; ++u) mbar_wait_bounded(bar_addr + 8u * (u % BWD_STAGES), (u / BWD_STAGES) & 1u);
+        cp_async_wait_all();
     };
 
     uint32_t r0 = warp * 32;
     GroupDesc<MW> cur = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0, lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
-    issue(cur, 0, unit);
     issue_params(cur);
     GroupDesc<MW> nxt = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + BWD_THREADS, lane);
     while (true) {
-        // descriptor two groups ahead: needed only at the start of the next iteration
+        // descriptor two groups ahead: the producer may reach it later in this group (not yet: its loads are in flight)
         const GroupDesc<MW> nxt2 = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
+        produce(cur, nxt, nxt2, 1);
         PreRec P;
         ShRegs<K> R;
         float geo[11];
 #pragma unroll
         for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(pbar_addr, pphase))) { fail(); return; }
-        pphase ^= 1u;
+        cp_async_wait_all();   // this lane's record has landed (a lane reads only what it copied itself)
         P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale data for lanes without hits: never used)
-#pragma unroll
-        for (int q = 0; q < (SW + 3) / 4; ++q) {
-            const float4 t = my_par[5 + q];
-            R.set(4 * q, t.x);
-            if (4 * q + 1 < SW) R.set(4 * q + 1, t.y);
-            if (4 * q + 2 < SW) R.set(4 * q + 2, t.z);
-            if (4 * q + 3 < SW) R.set(4 * q + 3, t.w);
-        }
-        fence_proxy_async();
-        __syncwarp();   // every lane has read its record: the buffer may be overwritten
-        if (nxt.cmax != 0) issue_params(nxt);
-        const int bx = x0 - P.ix, by = y0 - P.iy;
+        R.clear();
+        if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
+        const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
         const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
         for (int k = 0; k < nchunks; ++k) {
-            // keep the next unit's copy in flight while this one is consumed
-            if (k + 1 < nchunks) issue(cur, k + 1, unit + 1);
-            else if (nxt.cmax != 0) issue(nxt, 0, unit + 1);
-            const uint32_t s = unit & 1u;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit >> 1) & 1u))) { fail(); return; }
+            const uint32_t s = unit % BWD_STAGES;
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / BWD_STAGES) & 1u))) { fail(); return; }
             const float4* sl = my_stage + s * BWD_STAGE_F4 + lane;
             const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
             // two hits per iteration: two independent dependency chains for the scheduler to interleave
@@ -222,13 +219,14 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
                 const int p0 = cur.pm.next();
                 const int p1 = cur.pm.next();
                 const float4 L0 = se[0], L1 = se[32];
-                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, p0, L0);
-                bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, p1, L1);
+                bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, p0, L0);
+                bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, p1, L1);
             }
-            if (e < e_end) bwd_hit<TS, K, PW>(P, R, geo, spix, bx, by, cur.pm.next(), se[0]);
+            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, cur.pm.next(), se[0]);
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
+            produce(cur, nxt, nxt2, 2);   // refill the stage just released
         }
         if (cur.c != 0) {
             // one vector atomic per 16 bytes of the Gaussian's record
@@ -239,15 +237,16 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_kernel(const float4* __
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int wd = 4 * q + i;
-                    v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? R.word(wd - 11) : 0.0f);
+                    v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f);   // constants left out by sh_poly
                 }
-                atomicAdd(gp + q, make_float4(v[0], v[1], v[2], v[3]));
+                red_add_f4_hint(gp + q, v[0], v[1], v[2], v[3], pol_keep);
             }
         }
         if (nxt.cmax == 0) break;
         cur = nxt;
         nxt = nxt2;
         r0 += BWD_THREADS;
+        --pw;   // the producer is never behind the consumer: pw >= 1 here
     }
 }
 
@@ -257,48 +256,52 @@ __global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc
     if (i < (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4)) gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
-// Three roles by block range; every write covers whole 32-byte sectors of a gradient record.
-//   [0, conv_blocks)            one thread per slot: convert the accumulated moments (words 0..9) into
-//                               d mean, d scale, d quat, d opacity and write words 0..15 of the record
-//                               (all 32 lanes busy with the ~300-instruction conversion);
-//   [conv_blocks, +copy_blocks) 16 lanes per slot, 12 of them copy words 16..63 (SH gradient);
-//   the rest                    16 lanes per Gaussian: zero the record if the Gaussian has no slot.
-// Reads run in slot order (sequential), the writes scatter by Gaussian id.
-__global__ void __launch_bounds__(256) bwd_finalize_kernel(int64_t n, int64_t conv_blocks, int64_t copy_blocks, const float4* __restrict__ qs,
-                                                           const uint32_t* __restrict__ slot_of_gid, const uint32_t* __restrict__ gid_of_slot,
-                                                           const float4* __restrict__ gacc4, float4* __restrict__ grad4,
-                                                           const uint32_t* __restrict__ counts) {
+// One thread per slot: convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity and
+// write words 0..15 of the Gaussian's gradient record (all 32 lanes busy with the ~300-instruction conversion).
+__global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* __restrict__ qs, const uint32_t* __restrict__ gid_of_slot,
+                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          const uint32_t* __restrict__ counts) {
     if (counts[GART_CNT_ERROR]) return;
     constexpr int F4 = GART_GRAD_WORDS / 4;
-    const int64_t V = counts[GART_CNT_VISIBLE];
-    if ((int64_t)blockIdx.x < conv_blocks) {
-        const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-        if (sid >= V) return;
-        const float4* gp = gacc4 + (size_t)sid * F4;
-        const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
-        const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
-        float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
-        const float v[3] = {a.x, a.y, a.z};
-        const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
-        const float q[4] = {q4.x, q4.y, q4.z, q4.w};
-        const float sc[3] = {s4.x, s4.y, s4.z};
-        const GeoGrad o = moments_to_grads(v, Q, q, sc);
-        out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
-        out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
-        out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
-        out[3] = d;
-    } else if ((int64_t)blockIdx.x < conv_blocks + copy_blocks) {
-        const int64_t t = ((int64_t)blockIdx.x - conv_blocks) * blockDim.x + threadIdx.x;
-        const int64_t sid = t >> 4;
-        const int l = (int)(t & 15);
-        if (sid >= V || l < 4) return;
-        grad4[(size_t)gid_of_slot[sid] * F4 + l] = gacc4[(size_t)sid * F4 + l];
-    } else {
-        const int64_t t = ((int64_t)blockIdx.x - conv_blocks - copy_blocks) * blockDim.x + threadIdx.x;
-        const int64_t i = t >> 4;
-        if (i >= n) return;
-        if (slot_of_gid[i] == 0xffffffffu) grad4[(size_t)i * F4 + (t & 15)] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
+    const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+    const float4* gp = gacc4 + (size_t)sid * F4;
+    const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
+    const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
+    float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
+    const float v[3] = {a.x, a.y, a.z};
+    const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
+    const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+    const float sc[3] = {s4.x, s4.y, s4.z};
+    const GeoGrad o = moments_to_grads(v, Q, q, sc);
+    out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
+    out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
+    out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
+    out[3] = d;
+}
+
+// In the order of the gradient records (sequential writes): 16 lanes per Gaussian; a Gaussian without a slot gets
+// a zero record, the others words 16..63 (dL/dsh) of their slot's accumulation record.  A half-warp handles
+// FIN_ROWS Gaussians with all their loads in flight at once.
+constexpr int FIN_ROWS = 4;
+__global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, const uint32_t* __restrict__ slot_of_gid,
+                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    constexpr int F4 = GART_GRAD_WORDS / 4;
+    const int64_t hw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // half-warp
+    const int l = threadIdx.x & 15;
+    const int64_t i0 = hw * FIN_ROWS;
+    uint32_t s[FIN_ROWS];
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r) s[r] = i0 + r < n ? __ldg(slot_of_gid + i0 + r) : 0xffffffffu;
+    float4 v[FIN_ROWS];
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r)
+        v[r] = (s[r] != 0xffffffffu && l >= 4) ? __ldcs(gacc4 + (size_t)s[r] * F4 + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r)
+        if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu)) __stcs(grad4 + (size_t)(i0 + r) * F4 + l, v[r]);
 }
 
 template <int TS, int DEG>
@@ -307,7 +310,7 @@ static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, c
                                     const uint32_t* tile_lt_base, const float4* lt,
                                     const float* dL_dC, const CamF& cam, float* gacc, uint32_t* counts) {
     auto kern = bwd_pairs_kernel<TS, DEG>;
-    constexpr int smem = bwd_dyn_smem(3 * (DEG + 1) * (DEG + 1));
+    constexpr int smem = BWD_DYN_SMEM;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
     kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts);
     GART_LAUNCH_CHECK();
@@ -362,11 +365,12 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
     else s = launch_pairs<16>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
     if (s != GART_OK) return s;
-    const int64_t conv_blocks = ceil_div(g->n, 256), copy_blocks = ceil_div(g->n * 16, 256);
     const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
-    bwd_finalize_kernel<<<(unsigned)(conv_blocks + 2 * copy_blocks), 256, 0, st>>>(g->n, conv_blocks, copy_blocks, qs, slot_of_gid, gid_of_slot,
-                                                                                  reinterpret_cast<const float4*>(gacc),
-                                                                                  reinterpret_cast<float4*>(grad), counts);
+    bwd_convert_kernel<<<(unsigned)ceil_div(g->n, 256), 256, 0, st>>>(qs, gid_of_slot, reinterpret_cast<const float4*>(gacc),
+                                                                      reinterpret_cast<float4*>(grad), counts);
+    GART_LAUNCH_CHECK();
+    bwd_scatter_kernel<<<(unsigned)ceil_div(ceil_div(g->n, FIN_ROWS) * 16, 256), 256, 0, st>>>(g->n, slot_of_gid, reinterpret_cast<const float4*>(gacc),
+                                                                                               reinterpret_cast<float4*>(grad), counts);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

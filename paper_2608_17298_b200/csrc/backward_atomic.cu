@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
                                                          const uint32_t* __restrict__ ray_gid, const uint32_t* __restrict__ ray_slot,
                                                          const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
                                                          float* __restrict__ grad, const uint32_t* __restrict__ counts) {
-    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int K = (DEG + 1) * (DEG + 1), RS4 = (20 + 3 * K + 3) / 4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (ray >= (int64_t)cam.width * cam.height) return;
@@ -30,10 +30,9 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
         const float4* rp = rec + (size_t)__ldg(slot_of_gid + gid) * RS4;
         const PreRec P = load_pre(rp);
         const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
-        float shc[SW];
-        load_sh<SW>(rp, shc);
-        const HitGrad<K> hg = hit_grad<K>(Y, shc, g, L, r.alpha);
-        const float ad = r.alpha * hg.dalpha;
+        float wch[3];
+        lt_weights(L, g, wch);
+        const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
         const float G = -0.5f * ad;
         const float3 xg = ray_xg(r);
         const float v[3] = {G * xg.x, G * xg.y, G * xg.z};
@@ -48,9 +47,9 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
         atomicAdd(gp + 10, ad / opacity[gid]);
 #pragma unroll
         for (int k = 0; k < K; ++k) {
-            atomicAdd(gp + 11 + 3 * k, Y[k] * hg.wch[0]);
-            atomicAdd(gp + 11 + 3 * k + 1, Y[k] * hg.wch[1]);
-            atomicAdd(gp + 11 + 3 * k + 2, Y[k] * hg.wch[2]);
+            atomicAdd(gp + 11 + 3 * k, Y[k] * wch[0]);
+            atomicAdd(gp + 11 + 3 * k + 1, Y[k] * wch[1]);
+            atomicAdd(gp + 11 + 3 * k + 2, Y[k] * wch[2]);
         }
     }
 }

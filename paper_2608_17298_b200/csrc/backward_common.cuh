@@ -64,34 +64,4 @@ __device__ __forceinline__ GeoGrad moments_to_grads(const float* v, const float*
     return o;
 }
 
-// Per-hit gradient terms shared by both backward variants.
-template <int K>
-struct HitGrad {
-    float wch[3];   // T alpha g per channel, zero where the colour is clamped
-    float dalpha;   // dL/dalpha
-};
-
-template <int K>
-__device__ __forceinline__ HitGrad<K> hit_grad(const float* Y, const float* shc, const float3 g, const float4 L, const float alpha) {
-    float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
-#pragma unroll
-    for (int k = 0; k < K; ++k) {
-        c0 = fmaf(Y[k], shc[3 * k], c0);
-        c1 = fmaf(Y[k], shc[3 * k + 1], c1);
-        c2 = fmaf(Y[k], shc[3 * k + 2], c2);
-    }
-    const float T = L.w;
-    const float Ta = T * alpha;
-    const float inv = fast_rcp(1.0f - alpha);
-    HitGrad<K> h;
-    h.wch[0] = c0 > 0.0f ? Ta * g.x : 0.0f;
-    h.wch[1] = c1 > 0.0f ? Ta * g.y : 0.0f;
-    h.wch[2] = c2 > 0.0f ? Ta * g.z : 0.0f;
-    const float t0 = fmaf(T, fmaxf(c0, 0.0f), -L.x * inv);
-    const float t1 = fmaf(T, fmaxf(c1, 0.0f), -L.y * inv);
-    const float t2 = fmaf(T, fmaxf(c2, 0.0f), -L.z * inv);
-    h.dalpha = fmaf(g.x, t0, fmaf(g.y, t1, g.z * t2));
-    return h;
-}
-
 }  // namespace gart

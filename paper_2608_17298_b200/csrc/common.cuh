@@ -153,13 +153,58 @@ __device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy)
     return r;
 }
 
+// The geometric part alone (no response): what the point of maximum response needs.
+struct RayGeo {
+    float inv_a;   // 1 / |d_g|^2
+    float3 dg;     // d_g
+    float3 cr;     // o_g x d_g
+};
+
+__device__ __forceinline__ RayGeo ray_geo(const PreRec& p, float dx, float dy) {
+    RayGeo r;
+    const float ex = fmaf(p.c0.x, dx, p.c1.x * dy);
+    const float ey = fmaf(p.c0.y, dx, p.c1.y * dy);
+    const float ez = fmaf(p.c0.z, dx, p.c1.z * dy);
+    r.dg = make_float3(p.dgr.x + ex, p.dgr.y + ey, p.dgr.z + ez);
+    r.cr.x = fmaf(ey, p.m.z, fmaf(-ez, p.m.y, p.k.x));
+    r.cr.y = fmaf(ez, p.m.x, fmaf(-ex, p.m.z, p.k.y));
+    r.cr.z = fmaf(ex, p.m.y, fmaf(-ey, p.m.x, p.k.z));
+    r.inv_a = fast_rcp(fmaf(r.dg.x, r.dg.x, fmaf(r.dg.y, r.dg.y, r.dg.z * r.dg.z)));
+    return r;
+}
+
 // Maximum-response point in the Gaussian's normalised space.
-__device__ __forceinline__ float3 ray_xg(const RayEval& r) {
+template <class RayT>
+__device__ __forceinline__ float3 ray_xg(const RayT& r) {
     return make_float3((r.dg.y * r.cr.z - r.dg.z * r.cr.y) * r.inv_a,
                        (r.dg.z * r.cr.x - r.dg.x * r.cr.z) * r.inv_a,
                        (r.dg.x * r.cr.y - r.dg.y * r.cr.x) * r.inv_a);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// LT entry of a hit: what the backward pass needs of the ray's compositing state (Sec. 4.2), 16 bytes.
+// With w = T alpha the hit's blending weight, c its clamped colour and B the colour composited behind
+// it (background included), the pixel colour C satisfies
+//     alpha dC/dalpha = w c - alpha / (1 - alpha) B        (from Eq. 6-8)
+// so the entry holds that vector and w.  The backward pass then needs neither alpha nor the hit's
+// colour again: alpha dL/dalpha = <dL/dC, xyz>, and dL/dc = w dL/dC on the channels that are not
+// clamped, flagged in the three low mantissa bits of w (a relative change of w below 2^-20).
+__device__ __forceinline__ float4 lt_entry(float w, float alpha, float c0, float c1, float c2, float b0, float b1, float b2) {
+    const float r = alpha / (1.0f - alpha);
+    const uint32_t flags = (c0 > 0.0f ? 1u : 0u) | (c1 > 0.0f ? 2u : 0u) | (c2 > 0.0f ? 4u : 0u);
+    return make_float4(fmaf(w, c0, -r * b0), fmaf(w, c1, -r * b1), fmaf(w, c2, -r * b2),
+                       __uint_as_float((__float_as_uint(w) & ~7u) | flags));
+}
+
+// The per-channel weights dL/dc = w g of an LT entry (zero on clamped channels).
+__device__ __forceinline__ void lt_weights(const float4 L, const float3 g, float* wch) {
+    const uint32_t b = __float_as_uint(L.w);
+    const float w = __uint_as_float(b & ~7u);
+    wch[0] = (b & 1u) ? w * g.x : 0.0f;
+    wch[1] = (b & 2u) ? w * g.y : 0.0f;
+    wch[2] = (b & 4u) ? w * g.z : 0.0f;
+}
 
 // ---------------------------------------------------------------------------------------------
 // Hit mask of a (tile, Gaussian) pair held as 64-bit words, walked bit by bit in pixel order.
@@ -249,6 +294,43 @@ __device__ __forceinline__ void sh_basis(const float3 d, float* Y) {
     }
 }
 
+// The same basis without its normalisation constants: Y[k] = sh_norm(k) * B[k].  A sum of B[k] * (weights) over
+// many directions can take the constant once at the end; the first four B cost nothing (1, y, z, x).
+template <int K>
+__device__ __forceinline__ void sh_poly(const float3 d, float* B) {
+    B[0] = 1.0f;
+    if (K > 1) { B[1] = d.y; B[2] = d.z; B[3] = d.x; }
+    if (K > 4) {
+        const float xx = d.x * d.x, yy = d.y * d.y, zz = d.z * d.z;
+        const float xy = d.x * d.y;
+        const float e = xx - yy;
+        B[4] = xy;
+        B[5] = d.y * d.z;
+        B[6] = fmaf(2.0f, zz, -xx) - yy;
+        B[7] = d.x * d.z;
+        B[8] = e;
+        if (K > 9) {
+            const float t = fmaf(4.0f, zz, -xx) - yy;
+            B[9] = d.y * fmaf(3.0f, xx, -yy);
+            B[10] = xy * d.z;
+            B[11] = d.y * t;
+            B[12] = d.z * fmaf(-3.0f, xx + yy, 2.0f * zz);
+            B[13] = d.x * t;
+            B[14] = d.z * e;
+            B[15] = d.x * fmaf(-3.0f, yy, xx);
+        }
+    }
+}
+__device__ __forceinline__ constexpr float sh_norm(int k) {
+    return k == 0 ? 0.28209479177387814f
+         : k == 1 ? -0.4886025119029199f : k == 2 ? 0.4886025119029199f : k == 3 ? -0.4886025119029199f
+         : k == 4 ? 1.0925484305920792f : k == 5 ? -1.0925484305920792f : k == 6 ? 0.31539156525252005f
+         : k == 7 ? -1.0925484305920792f : k == 8 ? 0.5462742152960396f
+         : k == 9 ? -0.5900435899266435f : k == 10 ? 2.890611442640554f : k == 11 ? -0.4570457994644658f
+         : k == 12 ? 0.3731763325901154f : k == 13 ? -0.4570457994644658f : k == 14 ? 1.445305721320277f
+         : -0.5900435899266435f;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Asynchronous bulk copies global -> shared with completion on an mbarrier.  Every wait is bounded.
 constexpr uint32_t ASYNC_WAIT_LIMIT = 1u << 22;   // polls before a wait gives up (then the caller sets an error bit)
@@ -279,6 +361,35 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 // Orders this thread's earlier shared-memory accesses (generic proxy) before later accesses of the
 // asynchronous proxy: issued before a bulk copy overwrites a buffer that was just read.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Per-thread asynchronous 16-byte copies global -> shared (one warp instruction serves all lanes, unlike a bulk
+// copy, which every lane would have to issue by itself); completion by cp.async.wait_all of the issuing thread.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// L2 eviction policies for data read once (streamed) and for data that is re-used soon.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+                 : "memory");
+}
+// 16-byte vector reduction into global memory with an L2 eviction policy
+__device__ __forceinline__ void red_add_f4_hint(float4* dst, float a, float b, float c, float d, uint64_t policy) {
+    asm volatile("red.global.add.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d), "l"(policy)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
@@ -297,6 +408,10 @@ template <int K>
 struct ShRegs<K, false> {
     float sh[3 * K], acc[3 * K];
     __device__ __forceinline__ void set(int e, float v) { sh[e] = v; acc[e] = 0.0f; }   // e = 3 k + channel
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int e = 0; e < 3 * K; ++e) acc[e] = 0.0f;
+    }
     __device__ __forceinline__ float word(int e) const { return acc[e]; }
     __device__ __forceinline__ void colour(const float* Y, float* c) const {
         c[0] = 0.5f; c[1] = 0.5f; c[2] = 0.5f;
@@ -324,6 +439,12 @@ struct ShRegs<K, true> {
         const int k = e / 3, c = e % 3;
         if (k & 1) { sh[c][k >> 1].y = v; acc[c][k >> 1].y = 0.0f; }
         else { sh[c][k >> 1].x = v; acc[c][k >> 1].x = 0.0f; }
+    }
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int c = 0; c < 3; ++c)
+#pragma unroll
+            for (int i = 0; i < K / 2; ++i) acc[c][i] = make_float2(0.0f, 0.0f);
     }
     __device__ __forceinline__ float word(int e) const {
         const int k = e / 3, c = e % 3;

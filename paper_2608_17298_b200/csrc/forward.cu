@@ -447,9 +447,9 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const float4 ra = __ldg(&rec[2 * c]);
                 const float4 rb = __ldg(&rec[2 * c + 1]);
                 const uint32_t slot = __float_as_uint(ra.z);
-                lt[slot] = make_float4(k0, k1, k2, Ts[r]);
-                if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
                 const float wgt = Ts[r] * al[r];
+                lt[slot] = lt_entry(wgt, al[r], rb.x, rb.y, rb.z, k0, k1, k2);
+                if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, rb.x, k0); k1 = fmaf(wgt, rb.y, k1); k2 = fmaf(wgt, rb.z, k2);
             }
         }
@@ -537,15 +537,14 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
     for (int base = 0; base < n; base += 32) {
         const int i = n - 1 - (base + lane);
         const bool valid = i >= 0;
-        float T = 0.0f, v0 = 0.0f, v1 = 0.0f, v2 = 0.0f;
-        float4 ra = make_float4(0.f, 0.f, 0.f, 0.f);
+        float wgt = 0.0f, v0 = 0.0f, v1 = 0.0f, v2 = 0.0f;
+        float4 ra = make_float4(0.f, 0.f, 0.f, 0.f), rb = ra;
         if (valid) {
             const uint64_t key = kp[i];
             const uint32_t c = (uint32_t)key;
-            T = __uint_as_float((uint32_t)(key >> 32));
             ra = __ldg(&rec[2 * c]);
-            const float4 rb = __ldg(&rec[2 * c + 1]);
-            const float wgt = T * ra.w;
+            rb = __ldg(&rec[2 * c + 1]);
+            wgt = __uint_as_float((uint32_t)(key >> 32)) * ra.w;
             v0 = wgt * rb.x; v1 = wgt * rb.y; v2 = wgt * rb.z;
         }
         float s0 = v0, s1 = v1, s2 = v2;
@@ -560,7 +559,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
-            lt[slot] = make_float4(k0 + e0, k1 + e1, k2 + e2, T);
+            lt[slot] = lt_entry(wgt, ra.w, rb.x, rb.y, rb.z, k0 + e0, k1 + e1, k2 + e2);
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);

@@ -186,12 +186,11 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     for q in range(words.shape[1]):
         below += np.where(q < w_idx, np.bitwise_count(words[:, q]).astype(np.int64), 0)
     assert np.array_equal(below, e // 32)
-    # LT: transmittance of the first hit of a ray is 1; of later hits in [0, 1]; colours finite
-    lt = gpu["lt"]
-    first_hit = ray_off[:-1][hit_count > 0]
-    assert np.all(lt[gpu["ray_slot"][first_hit].astype(np.int64), 3] == 1.0)
-    used = lt[slots]
-    assert np.all(np.isfinite(used)) and np.all(used[:, 3] >= 0) and np.all(used[:, 3] <= 1.0)
+    # LT: word 3 is the blending weight T alpha in (0, 1) with the three clamp flags in its low mantissa
+    # bits; the vector part is finite.  (The values themselves are checked through the gradients.)
+    used = gpu["lt"][slots]
+    wgt = (np.ascontiguousarray(used[:, 3]).view(np.uint32) & np.uint32(0xFFFFFFF8)).view(np.float32)
+    assert np.all(np.isfinite(used)) and np.all(wgt >= 0) and np.all(wgt < 1.0)
     assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
 
 
