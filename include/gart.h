@@ -116,7 +116,7 @@ int32_t gart_mask_words(int32_t tile_size);
  *                1 in front of the near plane, 2 straddling it (rectangle = whole image unless
  *                the bounding sphere is outside a side plane of the frustum).
  *   pre    [n * gart_pre_words(sh_degree)] fp32 out: per slot, the evaluation record followed by a copy
- *                of the Gaussian's SH coefficients, and behind all records a copy of quaternion, scale
+ *                of its SH coefficients (times the basis constants), and behind all records quaternion, scale
  *                and opacity in slot order; contents are private to the library.
  *   slot_of_gid [n] uint32 out: slot of every Gaussian, 0xffffffff if it has none.
  *   gid_of_slot [n] uint32 out: the inverse (first V entries; 0xffffffff beyond).

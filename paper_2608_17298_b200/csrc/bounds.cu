@@ -152,6 +152,9 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
 
 // One thread per 16 bytes of a slot's record: 5 float4 of the evaluation record, then the SH
 // coefficients (zero padded to the record stride).  Also fills the two maps between ids and slots.
+__constant__ float c_sh_norm[16] = {sh_norm(0), sh_norm(1), sh_norm(2), sh_norm(3), sh_norm(4), sh_norm(5), sh_norm(6), sh_norm(7),
+                                    sh_norm(8), sh_norm(9), sh_norm(10), sh_norm(11), sh_norm(12), sh_norm(13), sh_norm(14), sh_norm(15)};
+
 __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4, int sw, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
                                                              const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
@@ -178,10 +181,11 @@ __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4,
     } else {
         const int e = (q - 5) * 4;
         const float* sp = sh + (size_t)gid * sw;
-        v.x = e < sw ? sp[e] : 0.0f;
-        v.y = e + 1 < sw ? sp[e + 1] : 0.0f;
-        v.z = e + 2 < sw ? sp[e + 2] : 0.0f;
-        v.w = e + 3 < sw ? sp[e + 3] : 0.0f;
+        // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
+        v.x = e < sw ? c_sh_norm[e / 3] * sp[e] : 0.0f;
+        v.y = e + 1 < sw ? c_sh_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
+        v.z = e + 2 < sw ? c_sh_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
+        v.w = e + 3 < sw ? c_sh_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
     }
     rec[(size_t)slot * rs4 + q] = v;
 }

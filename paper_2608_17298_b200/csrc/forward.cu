@@ -193,9 +193,22 @@ __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restric
     return d;
 }
 
+// Per-pixel data of the tile in shared memory, two float4 per pixel: (d.x, d.y, d.z, x) and (y, ray_off, -, -), d the
+// unit ray direction, (x, y) the position in the tile, ray_off the start of the ray's segment of hit records.
+// Lanes read DIFFERENT pixels at the same time; with 8 copies, copy j confined to the 16-byte bank group j and
+// lane l reading copy l mod 8, the 8 lanes served together by a 16-byte shared load never collide.
+template <int TS>
+struct EvalPix {
+    static constexpr int COPIES = TS == 8 ? 8 : 1;
+    static constexpr int STRIDE = COPIES == 1 ? 3 : 2;
+    static constexpr int F4 = TS * TS * STRIDE * COPIES;
+    __device__ static __forceinline__ int index(int p, int h, int copy) { return (p * STRIDE + h) * COPIES + copy; }
+};
+
 // Block per tile, one thread per (tile, Gaussian) pair; warps walk the rank groups.  The records of the
-// next group's Gaussians are copied into shared memory (bulk asynchronous copy per lane, completion on an
-// mbarrier) while the current group is evaluated.
+// next group's Gaussians are copied into shared memory (16-byte asynchronous copies of each lane) while the
+// current group is evaluated.  The colour is 0.5 + sum_k B_k(d) sh'_k with the bare SH polynomials B_k and
+// the record's coefficients sh'_k, which carry the normalisation constants.
 template <int TS, int DEG>
 __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
@@ -203,12 +216,10 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
                                                                 uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PW = (K + 3) & ~3, PF4 = (20 + SW + 3) / 4;
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PF4 = (20 + SW + 3) / 4;
     constexpr int PSTR = PF4 | 1;   // odd lane stride: the lanes' 16-byte reads fall into distinct banks
-    __shared__ __align__(16) float spix[NT * PW];
+    __shared__ __align__(16) float4 spix[EvalPix<TS>::F4];
     extern __shared__ __align__(128) float4 spar[];   // [EVAL_THREADS][PSTR] staged records
-    __shared__ __align__(8) uint64_t bars[EVAL_WARPS];
-    __shared__ uint32_t sro[NT];
     __shared__ uint32_t scur[NT];
     if (counts[GART_CNT_ERROR]) return;
     const int tile = blockIdx.x;
@@ -217,28 +228,30 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     const int tx = tile % cam.tiles_x, ty = tile / cam.tiles_x;
     const int x0 = tx * TS, y0 = ty * TS;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) {
-        mbar_init(smem_u32(&bars[warp]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
     for (int p = threadIdx.x; p < NT; p += EVAL_THREADS) {
         const int x = x0 + p % TS, y = y0 + p / TS;
-        float Y[K];
-        sh_basis<K>(pixel_dir(cam, min(x, cam.width - 1), min(y, cam.height - 1)), Y);
+        const float3 d = pixel_dir(cam, min(x, cam.width - 1), min(y, cam.height - 1));
+        const uint32_t ro = (x < cam.width && y < cam.height) ? ray_off[(size_t)y * cam.width + x] : 0u;
+        const float4 a = make_float4(d.x, d.y, d.z, (float)(p % TS));
+        const float4 b = make_float4((float)(p / TS), __uint_as_float(ro), 0.0f, 0.0f);
 #pragma unroll
-        for (int k = 0; k < K; ++k) spix[p * PW + k] = Y[k];
-        sro[p] = (x < cam.width && y < cam.height) ? ray_off[(size_t)y * cam.width + x] : 0u;
+        for (int c = 0; c < EvalPix<TS>::COPIES; ++c) {
+            spix[EvalPix<TS>::index(p, 0, c)] = a;
+            spix[EvalPix<TS>::index(p, 1, c)] = b;
+        }
         scur[p] = 0u;
     }
     __syncthreads();
     const uint32_t lt_base = tile_lt_base[tile];
+    const float4* spix_lane = spix + (lane & (EvalPix<TS>::COPIES - 1));
     float4* my_par = spar + (size_t)(warp * 32 + lane) * PSTR;
-    const uint32_t par_addr = smem_u32(my_par), bar_addr = smem_u32(&bars[warp]);
-    uint32_t phase = 0;
+    const uint32_t par_addr = smem_u32(my_par);
     auto issue_params = [&](const EvalDesc<MW>& d) {
-        const unsigned m = __ballot_sync(0xffffffffu, d.c != 0);
-        if (lane == 0) mbar_expect_tx(bar_addr, (uint32_t)__popc(m) * (uint32_t)(PF4 * 16));
-        if (d.c != 0) bulk_g2s(par_addr, rec + (size_t)d.sid * PF4, (uint32_t)(PF4 * 16), bar_addr);
+        if (d.c != 0) {
+            const float4* src = rec + (size_t)d.sid * PF4;
+#pragma unroll
+            for (int q = 0; q < PF4; ++q) cp_async16(par_addr + 16u * q, src + q);
+        }
     };
 
     uint32_t r0 = warp * 32;
@@ -249,14 +262,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     while (true) {
         const EvalDesc<MW> nxt2 = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * EVAL_THREADS, lane);
         const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr, phase))) {
-            // the copy never completed: report, give it a second bounded chance to land before this
-            // warp's shared memory may be released, and stop
-            if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
-            mbar_wait_bounded(bar_addr, phase);
-            return;
-        }
-        phase ^= 1u;
+        cp_async_wait_all();   // this lane's record has landed (a lane reads only what it copied itself)
         const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale for lanes without hits: unused)
         float shc[SW + 3];
 #pragma unroll
@@ -264,34 +270,38 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
             const float4 t = my_par[5 + q];
             shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
         }
-        fence_proxy_async();
-        __syncwarp();   // every lane has read its record: the buffer may be overwritten
-        if (nxt.cmax != 0) issue_params(nxt);
+        if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
         uint32_t slot = lt_base + cur.gstart + lane;
-        const int bx = x0 - P.ix, by = y0 - P.iy;
-        for (int e = 0; e < cur.c; ++e) {
-            const int p = cur.pm.next();
-            const RayEval r = ray_eval(P, (float)(bx + p % TS) - P.rx, (float)(by + p / TS) - P.ry);
+        const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
+        // one hit: evaluate, take the next free place of the ray's segment, write the 32-byte record
+        auto hit = [&](const int p, const uint32_t slot_e) {
+            const float4 pa = spix_lane[EvalPix<TS>::index(p, 0, 0)], pb = spix_lane[EvalPix<TS>::index(p, 1, 0)];
+            const uint32_t pos = atomicAdd(&scur[p], 1u);
+            const RayEval r = ray_eval(P, (fbx + pa.w) - P.rx, (fby + pb.x) - P.ry);   // small integers: the sums are exact
             const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
-            float Y[PW];
-#pragma unroll
-            for (int k4 = 0; k4 < PW / 4; ++k4) {   // 16-byte shared loads of the pixel's SH basis
-                const float4 t4 = reinterpret_cast<const float4*>(spix + p * PW)[k4];
-                Y[4 * k4] = t4.x; Y[4 * k4 + 1] = t4.y; Y[4 * k4 + 2] = t4.z; Y[4 * k4 + 3] = t4.w;
-            }
+            float B[K];
+            sh_poly<K>(make_float3(pa.x, pa.y, pa.z), B);
             float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                c0 = fmaf(Y[k], shc[3 * k], c0);
-                c1 = fmaf(Y[k], shc[3 * k + 1], c1);
-                c2 = fmaf(Y[k], shc[3 * k + 2], c2);
+                c0 = fmaf(B[k], shc[3 * k], c0);
+                c1 = fmaf(B[k], shc[3 * k + 1], c1);
+                c2 = fmaf(B[k], shc[3 * k + 2], c2);
             }
-            const uint32_t pos = atomicAdd(&scur[p], 1u);
-            float4* out = recs + ((size_t)sro[p] + pos) * 2;
-            out[0] = make_float4(t, __uint_as_float(gid), __uint_as_float(slot), r.alpha);
-            out[1] = make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f);
-            slot += 32u;
+            float4* out = recs + ((size_t)__float_as_uint(pb.y) + pos) * 2;
+            st_global_32B(out, make_float4(t, __uint_as_float(gid), __uint_as_float(slot_e), r.alpha),
+                          make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f));
+        };
+        // two hits per iteration: two independent dependency chains for the scheduler to interleave
+        int e = 0;
+        for (; e + 1 < cur.c; e += 2) {
+            const int p0 = cur.pm.next();
+            const int p1 = cur.pm.next();
+            hit(p0, slot);
+            hit(p1, slot + 32u);
+            slot += 64u;
         }
+        if (e < cur.c) hit(cur.pm.next(), slot);
         if (nxt.cmax == 0) break;
         cur = nxt;
         nxt = nxt2;
@@ -444,8 +454,8 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             const int i = lane * R + r;
             if (i < n) {
                 const uint32_t c = k[r] & KEY_IDX_MASK;
-                const float4 ra = __ldg(&rec[2 * c]);
-                const float4 rb = __ldg(&rec[2 * c + 1]);
+                float4 ra, rb;
+                ld_global_nc_32B(&rec[2 * c], ra, rb);
                 const uint32_t slot = __float_as_uint(ra.z);
                 const float wgt = Ts[r] * al[r];
                 lt[slot] = lt_entry(wgt, al[r], rb.x, rb.y, rb.z, k0, k1, k2);
