@@ -4,9 +4,9 @@
 // The paper finds the hits of a ray with hardware ray tracing over a BVH of bounded proxies;
 // here candidates come from the tile lists (same hit set: a hit is alpha >= alpha_min, i.e.
 // the ray meets the clamped ellipsoid whose projection the rectangle bounds).  Phases:
-//   1. fwd_mask    block per tile, thread per pixel: every pixel of the tile evaluates every
-//                  Gaussian of the tile list (records broadcast from shared memory); a warp
-//                  ballot yields the pair's hit mask; pixels count their hits.
+//   1. fwd_mask    block per tile, thread per (tile, Gaussian) pair: per image row the interval of
+//                  columns where the response reaches alpha_min (roots of a quadratic, settled on
+//                  the test itself) -> the pair's hit mask; ballots transpose masks into hits per pixel.
 //   2. tile_sort   warp per tile: stable counting sort of the tile's pairs by descending hit
 //                  count -> pair_order, with copies of slot id and mask in rank order (rank_sid,
 //                  rank_mask: read coalesced later); groups of 32 consecutive ranks share an LT
@@ -24,50 +24,139 @@
 namespace gart {
 
 // ------------------------------------------------------------------------------------------ phase 1
+// Hit test without the exponential: alpha >= alpha_min  <=>  D^2 <= tau := 2 ln(sigma / alpha_min), and with
+// D^2 = |o_g x d_g|^2 / |d_g|^2 and both vectors affine in the pixel position, the hit pixels of one image row are
+// those where a quadratic in the column u,  q(u) = qA u^2 + 2 qBh u + qC <= 0, and t* > 0 is t1 u + t0 > 0.
+// The projected ellipsoid is convex, so (qA > 0) a row's hits are one interval: its ends come from the roots and
+// are then settled by evaluating q at the neighbouring columns, so the mask is exactly {u : q(u) <= 0, t(u) > 0}
+// as evaluated in fp32.  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
+constexpr int MASK_WARPS = 4;
+
+struct RowQuad {
+    float qA, qB2, qC, t1, t0;   // qB2 = 2 qBh
+    __device__ __forceinline__ bool hit(float u) const {
+        return fmaf(fmaf(qA, u, qB2), u, qC) <= 0.0f && fmaf(t1, u, t0) > 0.0f;
+    }
+};
+
+// Bits 0..ncol-1: the columns of one row that the Gaussian's response reaches.
 template <int TS>
-__global__ void __launch_bounds__(TS * TS) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
-                                                           const uint32_t* __restrict__ tile_off,
-                                                           const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
-                                                           uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ hit_count,
-                                                           uint32_t* __restrict__ counts) {
-    constexpr int NT = TS * TS, MW = NT / 32, CH = 64;
-    __shared__ float4 sp[CH * 5];
-    __shared__ uint32_t smax[NT / 32];
+__device__ __forceinline__ uint32_t row_hits(const RowQuad& q, float inv_qA, int ncol) {
+    uint32_t bits = 0u;
+    const float qBh = 0.5f * q.qB2;
+    const float disc = fmaf(qBh, qBh, -q.qA * q.qC);
+    if (q.qA > 0.0f && disc == disc) {
+        if (disc < 0.0f) return 0u;
+        const float sq = sqrtf(disc);
+        float ulo = (-qBh - sq) * inv_qA, uhi = (-qBh + sq) * inv_qA;
+        // t* > 0 on one side of u = -t0 / t1
+        if (q.t1 > 0.0f) ulo = fmaxf(ulo, __fdividef(-q.t0, q.t1));
+        else if (q.t1 < 0.0f) uhi = fminf(uhi, __fdividef(-q.t0, q.t1));
+        else if (!(q.t0 > 0.0f)) return 0u;
+        if (!(ulo <= (float)(ncol - 1) && uhi >= 0.0f)) return 0u;
+        int lo = max(0, (int)ceilf(ulo)), hi = min(ncol - 1, (int)floorf(uhi));
+        // settle the ends on the test itself (the roots carry rounding)
+        if (lo <= hi) {
+            if (!q.hit((float)lo)) ++lo;
+            else if (lo > 0 && q.hit((float)(lo - 1))) --lo;
+        }
+        if (lo <= hi) {
+            if (!q.hit((float)hi)) --hi;
+            else if (hi < ncol - 1 && q.hit((float)(hi + 1))) ++hi;
+        }
+        if (lo <= hi) bits = (2u << hi) - (1u << lo);
+    } else {
+#pragma unroll
+        for (int c = 0; c < TS; ++c)
+            if (c < ncol && q.hit((float)c)) bits |= 1u << c;
+    }
+    return bits;
+}
+
+// Block per tile, thread per (tile, Gaussian) pair: row by row the interval of hit columns -> the pair's mask.
+// Hits per pixel: the lanes' masks are transposed with ballots (lane l counts pixels l, l + 32, ...).
+template <int TS>
+__global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
+                                                                   const uint32_t* __restrict__ tile_off,
+                                                                   const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
+                                                                   uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ hit_count,
+                                                                   uint32_t* __restrict__ counts) {
+    constexpr int NT = TS * TS, MW = NT / 32, RPW = 32 / TS;   // rows per mask word
+    __shared__ uint32_t scnt[NT];
     if (counts[GART_CNT_ERROR]) return;
     const int tile = blockIdx.x;
     const int tx = tile % cam.tiles_x, ty = tile / cam.tiles_x;
-    const int p = threadIdx.x, lane = p & 31, warp = p >> 5;
-    const int x = tx * TS + p % TS, y = ty * TS + p / TS;
-    const bool inside = x < cam.width && y < cam.height;
+    const int x0 = tx * TS, y0 = ty * TS;
+    const int lane = threadIdx.x & 31;
+    const int ncol = min(TS, cam.width - x0), nrow = min(TS, cam.height - y0);
     const uint32_t begin = tile_off[tile], end = tile_off[tile + 1];
-    uint32_t cnt = 0;
-    for (uint32_t base = begin; base < end; base += CH) {
-        const int nb = min((uint32_t)CH, end - base);
-        for (int i = p; i < nb * 5; i += NT) {
-            const int pair = i / 5, q = i - pair * 5;
-            sp[i] = __ldg(rec + (size_t)__ldg(slot_of_gid + __ldg(pair_gid + base + pair)) * rs4 + q);
+    for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) scnt[p] = 0u;
+    __syncthreads();
+    uint32_t cnt[MW];
+#pragma unroll
+    for (int q = 0; q < MW; ++q) cnt[q] = 0u;
+    const float inv_amin = 1.0f / alpha_min;
+    for (uint32_t j0 = begin + (threadIdx.x & ~31u); j0 < end; j0 += MASK_WARPS * 32) {
+        const uint32_t j = j0 + lane;
+        uint32_t w[MW];
+#pragma unroll
+        for (int q = 0; q < MW; ++q) w[q] = 0u;
+        if (j < end) {
+            const PreRec P = load_pre(rec + (size_t)__ldg(slot_of_gid + __ldg(pair_gid + j)) * rs4);
+            const float tau = 1.3862943611198906f * __log2f(P.sigma * inv_amin);   // 2 ln(sigma / alpha_min)
+            const float3 a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
+            const float3 b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
+            RowQuad rq;
+            rq.qA = fmaf(a1.x, a1.x, fmaf(a1.y, a1.y, a1.z * a1.z)) - tau * fmaf(P.c0.x, P.c0.x, fmaf(P.c0.y, P.c0.y, P.c0.z * P.c0.z));
+            rq.t1 = fmaf(P.m.x, P.c0.x, fmaf(P.m.y, P.c0.y, P.m.z * P.c0.z));
+            const float inv_qA = fast_rcp(rq.qA);
+            const float dx0 = (float)(x0 - P.ix) - P.rx;
+            // values at column 0 of row 0, then row by row
+            const float dy0 = (float)(y0 - P.iy) - P.ry;
+#pragma unroll
+            for (int r = 0; r < TS; ++r) {
+                if (r < nrow) {
+                    const float dy = dy0 + (float)r;
+                    const float3 dg0 = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy, P.dgr.y)),
+                                                   fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy, P.dgr.z)));
+                    const float3 cr0 = make_float3(fmaf(a1.x, dx0, fmaf(b1.x, dy, P.k.x)), fmaf(a1.y, dx0, fmaf(b1.y, dy, P.k.y)),
+                                                   fmaf(a1.z, dx0, fmaf(b1.z, dy, P.k.z)));
+                    rq.qC = fmaf(cr0.x, cr0.x, fmaf(cr0.y, cr0.y, cr0.z * cr0.z)) - tau * fmaf(dg0.x, dg0.x, fmaf(dg0.y, dg0.y, dg0.z * dg0.z));
+                    rq.qB2 = 2.0f * (fmaf(cr0.x, a1.x, fmaf(cr0.y, a1.y, cr0.z * a1.z)) - tau * fmaf(dg0.x, P.c0.x, fmaf(dg0.y, P.c0.y, dg0.z * P.c0.z)));
+                    rq.t0 = fmaf(P.m.x, dg0.x, fmaf(P.m.y, dg0.y, P.m.z * dg0.z));
+                    w[r / RPW] |= row_hits<TS>(rq, inv_qA, ncol) << ((r % RPW) * TS);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < MW; ++q) pair_mask[(size_t)j * MW + q] = w[q];
         }
-        __syncthreads();
-        for (int j = 0; j < nb; ++j) {
-            const PreRec P = unpack_pre(sp[j * 5], sp[j * 5 + 1], sp[j * 5 + 2], sp[j * 5 + 3], sp[j * 5 + 4]);
-            const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
-            const bool hit = inside && (r.alpha >= alpha_min) && (r.tnum > 0.0f);
-            const unsigned b = __ballot_sync(0xffffffffu, hit);
-            if (lane == 0) pair_mask[(size_t)(base + j) * MW + warp] = b;
-            cnt += hit ? 1u : 0u;
+        // hits per pixel over these 32 pairs
+#pragma unroll
+        for (int q = 0; q < MW; ++q) {
+            if (__any_sync(0xffffffffu, w[q] != 0u)) {
+#pragma unroll 8
+                for (int b = 0; b < 32; ++b) {
+                    const unsigned bal = __ballot_sync(0xffffffffu, (w[q] >> b) & 1u);
+                    if (lane == b) cnt[q] += __popc(bal);
+                }
+            }
         }
-        __syncthreads();
     }
-    if (inside) hit_count[(size_t)y * cam.width + x] = cnt;
-    uint32_t m = cnt;
+#pragma unroll
+    for (int q = 0; q < MW; ++q)
+        if (cnt[q]) atomicAdd(&scnt[q * 32 + lane], cnt[q]);
+    __syncthreads();
+    uint32_t m = 0;
+    for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) {
+        const int x = x0 + p % TS, y = y0 + p / TS;
+        if (x < cam.width && y < cam.height) {
+            hit_count[(size_t)y * cam.width + x] = scnt[p];
+            m = max(m, scnt[p]);
+        }
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_down_sync(0xffffffffu, m, o));
-    if (lane == 0) smax[warp] = m;
-    __syncthreads();
-    if (p == 0) {
-        for (int w = 1; w < NT / 32; ++w) m = max(m, smax[w]);
-        if (m) atomicMax(&counts[GART_CNT_MAX_RAY_HITS], m);
-    }
+    if (lane == 0 && m) atomicMax(&counts[GART_CNT_MAX_RAY_HITS], m);
 }
 
 // ------------------------------------------------------------------------------------------ phase 2
@@ -698,8 +787,8 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const int rs4 = rec_f4(g->sh_degree);
 
-    if (ts == 8) fwd_mask_kernel<8><<<T, 64, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, 256, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
+    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
