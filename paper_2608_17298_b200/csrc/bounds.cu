@@ -160,6 +160,9 @@ __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4,
                                                              const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
                                                              float4* __restrict__ rec, float4* __restrict__ qs,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
+    __shared__ float s_norm[16];   // lanes index it divergently: shared memory, not the constant bank
+    if (threadIdx.x < 16) s_norm[threadIdx.x] = c_sh_norm[threadIdx.x];
+    __syncthreads();
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t slot = t / rs4;
     const int q = (int)(t - slot * rs4);
@@ -182,10 +185,10 @@ __global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4,
         const int e = (q - 5) * 4;
         const float* sp = sh + (size_t)gid * sw;
         // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
-        v.x = e < sw ? c_sh_norm[e / 3] * sp[e] : 0.0f;
-        v.y = e + 1 < sw ? c_sh_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
-        v.z = e + 2 < sw ? c_sh_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
-        v.w = e + 3 < sw ? c_sh_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
+        v.x = e < sw ? s_norm[e / 3] * sp[e] : 0.0f;
+        v.y = e + 1 < sw ? s_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
+        v.z = e + 2 < sw ? s_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
+        v.w = e + 3 < sw ? s_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
     }
     rec[(size_t)slot * rs4 + q] = v;
 }

@@ -25,11 +25,12 @@ namespace gart {
 
 // ------------------------------------------------------------------------------------------ phase 1
 // Hit test without the exponential: alpha >= alpha_min  <=>  D^2 <= tau := 2 ln(sigma / alpha_min), and with
-// D^2 = |o_g x d_g|^2 / |d_g|^2 and both vectors affine in the pixel position, the hit pixels of one image row are
-// those where a quadratic in the column u,  q(u) = qA u^2 + 2 qBh u + qC <= 0, and t* > 0 is t1 u + t0 > 0.
-// The projected ellipsoid is convex, so (qA > 0) a row's hits are one interval: its ends come from the roots and
-// are then settled by evaluating q at the neighbouring columns, so the mask is exactly {u : q(u) <= 0, t(u) > 0}
-// as evaluated in fp32.  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
+// D^2 = |o_g x d_g|^2 / |d_g|^2 and both vectors affine in the pixel position (u, v) inside the tile,
+//     Q(u, v) = |o_g x d_g|^2 - tau |d_g|^2 = Quu u^2 + 2 Quv u v + Qvv v^2 + 2 Qu u + 2 Qv v + Q0 <= 0,
+// and t* > 0 is t1 u + t2 v + tA > 0.  On row v the hit columns are those with q(u) = qA u^2 + 2 qBh u + qC <= 0.
+// The projected ellipsoid is convex, so (qA > 0) they form one interval: its ends come from the roots and are then
+// settled by evaluating q at the neighbouring columns, so the mask is exactly {u : q(u) <= 0, t(u) > 0} as
+// evaluated in fp32.  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
 constexpr int MASK_WARPS = 4;
 
 struct RowQuad {
@@ -39,32 +40,35 @@ struct RowQuad {
     }
 };
 
-// Bits 0..ncol-1: the columns of one row that the Gaussian's response reaches.
+__device__ __forceinline__ float fast_sqrt(float x) {
+    float y;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Bits 0..ncol-1: the columns of one row that the Gaussian's response reaches.  `regular`: qA > 0 and t1 != 0,
+// with inv_qA = 1 / qA and inv_t1 = 1 / t1.
 template <int TS>
-__device__ __forceinline__ uint32_t row_hits(const RowQuad& q, float inv_qA, int ncol) {
+__device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, float inv_qA, float inv_t1, int ncol) {
     uint32_t bits = 0u;
-    const float qBh = 0.5f * q.qB2;
-    const float disc = fmaf(qBh, qBh, -q.qA * q.qC);
-    if (q.qA > 0.0f && disc == disc) {
-        if (disc < 0.0f) return 0u;
-        const float sq = sqrtf(disc);
-        float ulo = (-qBh - sq) * inv_qA, uhi = (-qBh + sq) * inv_qA;
-        // t* > 0 on one side of u = -t0 / t1
-        if (q.t1 > 0.0f) ulo = fmaxf(ulo, __fdividef(-q.t0, q.t1));
-        else if (q.t1 < 0.0f) uhi = fminf(uhi, __fdividef(-q.t0, q.t1));
-        else if (!(q.t0 > 0.0f)) return 0u;
-        if (!(ulo <= (float)(ncol - 1) && uhi >= 0.0f)) return 0u;
-        int lo = max(0, (int)ceilf(ulo)), hi = min(ncol - 1, (int)floorf(uhi));
-        // settle the ends on the test itself (the roots carry rounding)
-        if (lo <= hi) {
-            if (!q.hit((float)lo)) ++lo;
-            else if (lo > 0 && q.hit((float)(lo - 1))) --lo;
+    if (regular) {
+        const float qBh = 0.5f * q.qB2;
+        const float disc = fmaf(qBh, qBh, -q.qA * q.qC);
+        if (disc >= 0.0f) {
+            const float sq = fast_sqrt(disc);
+            float ulo = (-qBh - sq) * inv_qA, uhi = (-qBh + sq) * inv_qA;
+            const float ut = -q.t0 * inv_t1;   // t* > 0 on one side of it
+            ulo = q.t1 > 0.0f ? fmaxf(ulo, ut) : ulo;
+            uhi = q.t1 > 0.0f ? uhi : fminf(uhi, ut);
+            const float last = (float)(ncol - 1);
+            float flo = fmaxf(ceilf(ulo), 0.0f), fhi = fminf(floorf(uhi), last);
+            // settle the ends on the test itself (the roots carry rounding)
+            const bool l0 = q.hit(flo), l1 = flo > 0.0f && q.hit(flo - 1.0f);
+            const bool h0 = q.hit(fhi), h1 = fhi < last && q.hit(fhi + 1.0f);
+            flo = l0 ? (l1 ? flo - 1.0f : flo) : flo + 1.0f;
+            fhi = h0 ? (h1 ? fhi + 1.0f : fhi) : fhi - 1.0f;
+            if (flo <= fhi) bits = (2u << (int)fhi) - (1u << (int)flo);   // (NaN compares false)
         }
-        if (lo <= hi) {
-            if (!q.hit((float)hi)) --hi;
-            else if (hi < ncol - 1 && q.hit((float)(hi + 1))) ++hi;
-        }
-        if (lo <= hi) bits = (2u << hi) - (1u << lo);
     } else {
 #pragma unroll
         for (int c = 0; c < TS; ++c)
@@ -96,35 +100,58 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
 #pragma unroll
     for (int q = 0; q < MW; ++q) cnt[q] = 0u;
     const float inv_amin = 1.0f / alpha_min;
-    for (uint32_t j0 = begin + (threadIdx.x & ~31u); j0 < end; j0 += MASK_WARPS * 32) {
+    // the chain pair -> Gaussian -> slot -> record is three dependent loads: slot ids run two iterations ahead,
+    // records one
+    constexpr uint32_t STEP = MASK_WARPS * 32;
+    auto load_sid = [&](uint32_t jj) { return jj < end ? __ldg(slot_of_gid + __ldg(pair_gid + jj)) : 0u; };
+    const uint32_t jfirst = begin + threadIdx.x;
+    uint32_t sid_nx = load_sid(jfirst + STEP);
+    float4 ra[5];
+    {
+        const uint32_t sid0 = load_sid(jfirst);
+#pragma unroll
+        for (int q = 0; q < 5; ++q) ra[q] = jfirst < end ? __ldg(rec + (size_t)sid0 * rs4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (uint32_t j0 = begin + (threadIdx.x & ~31u); j0 < end; j0 += STEP) {
         const uint32_t j = j0 + lane;
+        const uint32_t sid_nx2 = load_sid(j + 2 * STEP);
+        float4 rb[5];
+#pragma unroll
+        for (int q = 0; q < 5; ++q) rb[q] = j + STEP < end ? __ldg(rec + (size_t)sid_nx * rs4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        sid_nx = sid_nx2;
         uint32_t w[MW];
 #pragma unroll
         for (int q = 0; q < MW; ++q) w[q] = 0u;
         if (j < end) {
-            const PreRec P = load_pre(rec + (size_t)__ldg(slot_of_gid + __ldg(pair_gid + j)) * rs4);
+            const PreRec P = unpack_pre(ra[0], ra[1], ra[2], ra[3], ra[4]);
             const float tau = 1.3862943611198906f * __log2f(P.sigma * inv_amin);   // 2 ln(sigma / alpha_min)
             const float3 a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
             const float3 b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
+            // o_g x d_g and d_g at the tile's first pixel
+            const float dx0 = (float)(x0 - P.ix) - P.rx, dy0 = (float)(y0 - P.iy) - P.ry;
+            const float3 dgA = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy0, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy0, P.dgr.y)),
+                                           fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy0, P.dgr.z)));
+            const float3 crA = make_float3(fmaf(a1.x, dx0, fmaf(b1.x, dy0, P.k.x)), fmaf(a1.y, dx0, fmaf(b1.y, dy0, P.k.y)),
+                                           fmaf(a1.z, dx0, fmaf(b1.z, dy0, P.k.z)));
+            auto dot = [](const float3 a, const float3 b) { return fmaf(a.x, b.x, fmaf(a.y, b.y, a.z * b.z)); };
+            const float Quu = dot(a1, a1) - tau * dot(P.c0, P.c0), Qvv = dot(b1, b1) - tau * dot(P.c1, P.c1);
+            const float Quv = dot(a1, b1) - tau * dot(P.c0, P.c1);
+            const float Qu = dot(crA, a1) - tau * dot(dgA, P.c0), Qv = dot(crA, b1) - tau * dot(dgA, P.c1);
+            const float Q0 = dot(crA, crA) - tau * dot(dgA, dgA);
+            const float tA = dot(P.m, dgA), t2 = dot(P.m, P.c1);
             RowQuad rq;
-            rq.qA = fmaf(a1.x, a1.x, fmaf(a1.y, a1.y, a1.z * a1.z)) - tau * fmaf(P.c0.x, P.c0.x, fmaf(P.c0.y, P.c0.y, P.c0.z * P.c0.z));
-            rq.t1 = fmaf(P.m.x, P.c0.x, fmaf(P.m.y, P.c0.y, P.m.z * P.c0.z));
-            const float inv_qA = fast_rcp(rq.qA);
-            const float dx0 = (float)(x0 - P.ix) - P.rx;
-            // values at column 0 of row 0, then row by row
-            const float dy0 = (float)(y0 - P.iy) - P.ry;
+            rq.qA = Quu;
+            rq.t1 = dot(P.m, P.c0);
+            const bool regular = rq.qA > 0.0f && rq.t1 != 0.0f;
+            const float inv_qA = fast_rcp(rq.qA), inv_t1 = fast_rcp(rq.t1);
 #pragma unroll
             for (int r = 0; r < TS; ++r) {
                 if (r < nrow) {
-                    const float dy = dy0 + (float)r;
-                    const float3 dg0 = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy, P.dgr.y)),
-                                                   fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy, P.dgr.z)));
-                    const float3 cr0 = make_float3(fmaf(a1.x, dx0, fmaf(b1.x, dy, P.k.x)), fmaf(a1.y, dx0, fmaf(b1.y, dy, P.k.y)),
-                                                   fmaf(a1.z, dx0, fmaf(b1.z, dy, P.k.z)));
-                    rq.qC = fmaf(cr0.x, cr0.x, fmaf(cr0.y, cr0.y, cr0.z * cr0.z)) - tau * fmaf(dg0.x, dg0.x, fmaf(dg0.y, dg0.y, dg0.z * dg0.z));
-                    rq.qB2 = 2.0f * (fmaf(cr0.x, a1.x, fmaf(cr0.y, a1.y, cr0.z * a1.z)) - tau * fmaf(dg0.x, P.c0.x, fmaf(dg0.y, P.c0.y, dg0.z * P.c0.z)));
-                    rq.t0 = fmaf(P.m.x, dg0.x, fmaf(P.m.y, dg0.y, P.m.z * dg0.z));
-                    w[r / RPW] |= row_hits<TS>(rq, inv_qA, ncol) << ((r % RPW) * TS);
+                    const float v = (float)r;
+                    rq.qB2 = 2.0f * fmaf(Quv, v, Qu);
+                    rq.qC = fmaf(fmaf(Qvv, v, 2.0f * Qv), v, Q0);
+                    rq.t0 = fmaf(t2, v, tA);
+                    w[r / RPW] |= row_hits<TS>(rq, regular, inv_qA, inv_t1, ncol) << ((r % RPW) * TS);
                 }
             }
 #pragma unroll
@@ -141,6 +168,8 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
                 }
             }
         }
+#pragma unroll
+        for (int q = 0; q < 5; ++q) ra[q] = rb[q];
     }
 #pragma unroll
     for (int q = 0; q < MW; ++q)
