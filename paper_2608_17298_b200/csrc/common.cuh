@@ -191,7 +191,7 @@ __device__ __forceinline__ float3 ray_xg(const RayT& r) {
 // colour again: alpha dL/dalpha = <dL/dC, xyz>, and dL/dc = w dL/dC on the channels that are not
 // clamped, flagged in the three low mantissa bits of w (a relative change of w below 2^-20).
 __device__ __forceinline__ float4 lt_entry(float w, float alpha, float c0, float c1, float c2, float b0, float b1, float b2) {
-    const float r = alpha / (1.0f - alpha);
+    const float r = __fdividef(alpha, 1.0f - alpha);
     const uint32_t flags = (c0 > 0.0f ? 1u : 0u) | (c1 > 0.0f ? 2u : 0u) | (c2 > 0.0f ? 4u : 0u);
     return make_float4(fmaf(w, c0, -r * b0), fmaf(w, c1, -r * b1), fmaf(w, c2, -r * b2),
                        __uint_as_float((__float_as_uint(w) & ~7u) | flags));

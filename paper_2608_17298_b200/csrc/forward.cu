@@ -440,37 +440,59 @@ constexpr int KEY_IDX_BITS = 9;
 static_assert((1 << KEY_IDX_BITS) >= SORT_CAP, "record index must fit the key");
 constexpr uint32_t KEY_IDX_MASK = (1u << KEY_IDX_BITS) - 1u;
 
+// Ascending bitonic sort of the 32 R keys of a warp (lane l holds positions l R .. l R + R - 1), in the form whose
+// compare-exchanges all put the smaller key at the lower position: a merge of size kk first pairs position i with
+// i ^ (kk - 1), then with i ^ j for j = kk/4 ... 1.  No direction flags; partners inside a lane are compile-time
+// register pairs, partners in another lane cost one shuffle and one min-or-max chosen per lane.
 template <int R>
 __device__ __forceinline__ void sort_regs(uint32_t (&k)[R], int lane) {
-    constexpr int N = 32 * R;
-    // the merge sizes and the cross-lane distances are run-time loops (small code: the instruction cache
-    // matters more here than the loop overhead); register indices stay compile-time
+    auto cmpswap = [](uint32_t& a, uint32_t& b) {
+        const uint32_t lo = min(a, b), hi = max(a, b);
+        a = lo; b = hi;
+    };
+    // merges inside a lane
+#pragma unroll
+    for (int kk = 2; kk <= R; kk <<= 1) {
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+            if ((r ^ (kk - 1)) > r) cmpswap(k[r], k[r ^ (kk - 1)]);
+#pragma unroll
+        for (int j = kk >> 2; j >= 1; j >>= 1)
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if ((r ^ j) > r) cmpswap(k[r], k[r ^ j]);
+    }
+    // merges across m lanes (run-time loops: small code, the instruction cache matters more than loop overhead)
 #pragma unroll 1
-    for (int kk = 2; kk <= N; kk <<= 1) {
+    for (int m = 2; m <= 32; m <<= 1) {
+        {
+            const bool lower = (lane & (m >> 1)) == 0;
+            if (R == 1) {
+                const uint32_t o = __shfl_xor_sync(0xffffffffu, k[0], m - 1);
+                k[0] = lower ? min(k[0], o) : max(k[0], o);
+            }
+#pragma unroll
+            for (int r = 0; r < R / 2; ++r) {   // registers r and R - 1 - r meet each other's mirror image
+                const uint32_t oa = __shfl_xor_sync(0xffffffffu, k[R - 1 - r], m - 1);
+                const uint32_t ob = __shfl_xor_sync(0xffffffffu, k[r], m - 1);
+                k[r] = lower ? min(k[r], oa) : max(k[r], oa);
+                k[R - 1 - r] = lower ? min(k[R - 1 - r], ob) : max(k[R - 1 - r], ob);
+            }
+        }
 #pragma unroll 1
-        for (int lj = (kk >> 1) / R; lj >= 1; lj >>= 1) {   // partner in another lane, same register
+        for (int lj = m >> 2; lj >= 1; lj >>= 1) {
             const bool lower = (lane & lj) == 0;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const uint32_t o = __shfl_xor_sync(0xffffffffu, k[r], lj);
-                const bool asc = ((lane * R + r) & kk) == 0;
-                k[r] = (lower == asc) ? min(k[r], o) : max(k[r], o);
+                k[r] = lower ? min(k[r], o) : max(k[r], o);
             }
         }
 #pragma unroll
-        for (int j = R >> 1; j >= 1; j >>= 1) {             // partner in this lane
-            if (j < kk) {
+        for (int j = R >> 1; j >= 1; j >>= 1)
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if ((r ^ j) > r) {
-                        const bool asc = ((lane * R + r) & kk) == 0;
-                        const uint32_t lo = min(k[r], k[r ^ j]), hi = max(k[r], k[r ^ j]);
-                        k[r] = asc ? lo : hi;
-                        k[r ^ j] = asc ? hi : lo;
-                    }
-                }
-            }
-        }
+            for (int r = 0; r < R; ++r)
+                if ((r ^ j) > r) cmpswap(k[r], k[r ^ j]);
     }
 }
 
