@@ -502,17 +502,28 @@ __device__ __forceinline__ bool rec_after(const float4* __restrict__ rec, uint32
     return a.x > b.x || (a.x == b.x && __float_as_uint(a.y) > __float_as_uint(b.y));
 }
 
+// The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
+// slot as one float4, alpha apart; after the sort the three passes gather from there by sorted index.
 template <int R>
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
-                                               float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
+                                               float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
+                                               float4* __restrict__ s_cs, float* __restrict__ s_al) {
     uint32_t k[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         // load striped (coalesced), the network does not care about the initial arrangement
         const int i = r * 32 + lane;
-        k[r] = i < n ? ((__float_as_uint(__ldg(&rec[2 * i].x)) & ~KEY_IDX_MASK) | (uint32_t)i) : 0xffffffffu;
+        k[r] = 0xffffffffu;
+        if (i < n) {
+            float4 ra, rb;
+            ld_global_nc_32B(&rec[2 * i], ra, rb);
+            k[r] = (__float_as_uint(ra.x) & ~KEY_IDX_MASK) | (uint32_t)i;
+            s_cs[i] = make_float4(rb.x, rb.y, rb.z, ra.z);
+            s_al[i] = ra.w;
+        }
     }
+    __syncwarp();
     sort_regs<R>(k, lane);
     {
         // neighbours with the same truncated t*: exact order by odd-even exchanges, n rounds at most
@@ -542,12 +553,12 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             }
         }
     }
-    // front to back: transmittance in front of every hit (Eq. 7)
+    // front to back: transmittance in front of every hit (Eq. 7); padding positions get alpha = 0
     float al[R];
     float lp = 1.0f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        al[r] = lane * R + r < n ? __ldg(&rec[2 * (k[r] & KEY_IDX_MASK)].w) : 0.0f;
+        al[r] = lane * R + r < n ? s_al[k[r] & KEY_IDX_MASK] : 0.0f;
         lp *= 1.0f - al[r];
     }
     float inc = lp;
@@ -563,15 +574,12 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
     float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f;
     {
         float T = T0;
-        float w0[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) { w0[r] = T * al[r]; T *= 1.0f - al[r]; }
-#pragma unroll
-        for (int r = R - 1; r >= 0; --r) {
-            if (lane * R + r < n) {
-                const float4 c = __ldg(&rec[2 * (k[r] & KEY_IDX_MASK) + 1]);
-                s0 = fmaf(w0[r], c.x, s0); s1 = fmaf(w0[r], c.y, s1); s2 = fmaf(w0[r], c.z, s2);
-            }
+        for (int r = 0; r < R; ++r) {
+            const float w0 = T * al[r];   // zero on padding positions
+            const float4 c = s_cs[lane * R + r < n ? (k[r] & KEY_IDX_MASK) : 0u];
+            s0 = fmaf(w0, c.x, s0); s1 = fmaf(w0, c.y, s1); s2 = fmaf(w0, c.z, s2);
+            T *= 1.0f - al[r];
         }
     }
     float u0 = s0, u1 = s1, u2 = s2;   // inclusive suffix over lanes
@@ -594,13 +602,12 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             const int i = lane * R + r;
             if (i < n) {
                 const uint32_t c = k[r] & KEY_IDX_MASK;
-                float4 ra, rb;
-                ld_global_nc_32B(&rec[2 * c], ra, rb);
-                const uint32_t slot = __float_as_uint(ra.z);
+                const float4 cs = s_cs[c];
+                const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
-                lt[slot] = lt_entry(wgt, al[r], rb.x, rb.y, rb.z, k0, k1, k2);
-                if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
-                k0 = fmaf(wgt, rb.x, k0); k1 = fmaf(wgt, rb.y, k1); k2 = fmaf(wgt, rb.z, k2);
+                lt[slot] = lt_entry(wgt, al[r], cs.x, cs.y, cs.z, k0, k1, k2);
+                if (ray_gid) { ray_gid[b + i] = __float_as_uint(__ldg(&rec[2 * c].y)); ray_slot[b + i] = slot; }
+                k0 = fmaf(wgt, cs.x, k0); k1 = fmaf(wgt, cs.y, k1); k2 = fmaf(wgt, cs.z, k2);
             }
         }
     }
@@ -742,7 +749,10 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         return;
     }
     const float4* rec = recs + b * 2;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot)
+    extern __shared__ __align__(16) float4 sweep_smem[];   // per warp: SORT_CAP float4 (colour, slot), then SORT_CAP floats (alpha)
+    float4* s_cs = sweep_smem + (size_t)warp * SORT_CAP;
+    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP) + (size_t)warp * SORT_CAP;
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot, s_cs, s_al)
     if (n <= 32) GART_SWEEP(1);
     else if (n <= 64) GART_SWEEP(2);
     else if (n <= 128) GART_SWEEP(4);
@@ -861,7 +871,9 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);
-    fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, 0, st>>>(ray_off, w.recs, w.long_keys, n_rays,
+    constexpr int sweep_smem = SWEEP_WARPS * SORT_CAP * 20;
+    if (cudaFuncSetAttribute(fwd_sort_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sweep_smem) != cudaSuccess) return GART_ERR_CUDA;
+    fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, sweep_smem, st>>>(ray_off, w.recs, w.long_keys, n_rays,
                                                                          cfg->background[0], cfg->background[1], cfg->background[2],
                                                                          color, t_final, reinterpret_cast<float4*>(lt), ray_gid,
                                                                          ray_slot, counts);
