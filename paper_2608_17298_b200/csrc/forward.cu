@@ -496,10 +496,10 @@ __device__ __forceinline__ void sort_regs(uint32_t (&k)[R], int lane) {
     }
 }
 
-// true if record a must come after record b: larger t*, or equal t* and larger Gaussian id
-__device__ __forceinline__ bool rec_after(const float4* __restrict__ rec, uint32_t ka, uint32_t kb) {
-    const float4 a = __ldg(&rec[2 * (ka & KEY_IDX_MASK)]), b = __ldg(&rec[2 * (kb & KEY_IDX_MASK)]);
-    return a.x > b.x || (a.x == b.x && __float_as_uint(a.y) > __float_as_uint(b.y));
+// true if record a must come after record b: larger t*, or equal t* and larger Gaussian id  (s_tg: t* bits and id per record)
+__device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32_t ka, uint32_t kb) {
+    const uint2 a = s_tg[ka & KEY_IDX_MASK], b = s_tg[kb & KEY_IDX_MASK];
+    return a.x > b.x || (a.x == b.x && a.y > b.y);   // t* >= 0: its bit pattern orders like its value
 }
 
 // The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
@@ -508,7 +508,7 @@ template <int R>
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
-                                               float4* __restrict__ s_cs, float* __restrict__ s_al) {
+                                               float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
     uint32_t k[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -521,6 +521,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             k[r] = (__float_as_uint(ra.x) & ~KEY_IDX_MASK) | (uint32_t)i;
             s_cs[i] = make_float4(rb.x, rb.y, rb.z, ra.z);
             s_al[i] = ra.w;
+            s_tg[i] = make_uint2(__float_as_uint(ra.x), __float_as_uint(ra.y));
         }
     }
     __syncwarp();
@@ -537,7 +538,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 bool moved = false;
 #pragma unroll
                 for (int r = 0; r + 1 < R; ++r) {
-                    if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(rec, k[r], k[r + 1])) {
+                    if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(s_tg, k[r], k[r + 1])) {
                         const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
                     }
                 }
@@ -545,9 +546,9 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const uint32_t up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
                 const bool lead = ((lane ^ round) & 1) == 0;
                 if (lead) {
-                    if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(rec, k[R - 1], up)) { k[R - 1] = up; moved = true; }
+                    if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(s_tg, k[R - 1], up)) { k[R - 1] = up; moved = true; }
                 } else {
-                    if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(rec, dn, k[0])) { k[0] = dn; moved = true; }
+                    if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(s_tg, dn, k[0])) { k[0] = dn; moved = true; }
                 }
                 if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
             }
@@ -606,7 +607,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
                 lt[slot] = lt_entry(wgt, al[r], cs.x, cs.y, cs.z, k0, k1, k2);
-                if (ray_gid) { ray_gid[b + i] = __float_as_uint(__ldg(&rec[2 * c].y)); ray_slot[b + i] = slot; }
+                if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cs.x, k0); k1 = fmaf(wgt, cs.y, k1); k2 = fmaf(wgt, cs.z, k2);
             }
         }
@@ -749,10 +750,11 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
         return;
     }
     const float4* rec = recs + b * 2;
-    extern __shared__ __align__(16) float4 sweep_smem[];   // per warp: SORT_CAP float4 (colour, slot), then SORT_CAP floats (alpha)
+    extern __shared__ __align__(16) float4 sweep_smem[];   // SORT_CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
     float4* s_cs = sweep_smem + (size_t)warp * SORT_CAP;
-    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP) + (size_t)warp * SORT_CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot, s_cs, s_al)
+    uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP) + (size_t)warp * SORT_CAP;
+    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP * 3 / 2) + (size_t)warp * SORT_CAP;
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (n <= 32) GART_SWEEP(1);
     else if (n <= 64) GART_SWEEP(2);
     else if (n <= 128) GART_SWEEP(4);
@@ -871,7 +873,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);
-    constexpr int sweep_smem = SWEEP_WARPS * SORT_CAP * 20;
+    constexpr int sweep_smem = SWEEP_WARPS * SORT_CAP * 28;
     if (cudaFuncSetAttribute(fwd_sort_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sweep_smem) != cudaSuccess) return GART_ERR_CUDA;
     fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, sweep_smem, st>>>(ray_off, w.recs, w.long_keys, n_rays,
                                                                          cfg->background[0], cfg->background[1], cfg->background[2],
