@@ -250,10 +250,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     }
 }
 
-// Zero the accumulation records of the view's slots (their number lives on the device).
+// Zero the accumulation records of the view's slots (their number lives on the device): grid-stride.
 __global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc4, const uint32_t* __restrict__ counts) {
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4)) gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const size_t total = (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+        gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
 // One thread per slot: convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity and
@@ -355,7 +356,8 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     cudaStream_t st = (cudaStream_t)stream;
     float* gacc = reinterpret_cast<float*>(workspace);
     const int64_t f4 = g->n * (GART_GRAD_WORDS / 4);
-    bwd_zero_kernel<<<(unsigned)ceil_div(f4, 256), 256, 0, st>>>(reinterpret_cast<float4*>(gacc), counts);
+    const int64_t zero_blocks = ceil_div(f4, 256);
+    bwd_zero_kernel<<<(unsigned)(zero_blocks < 148 * 32 ? zero_blocks : 148 * 32), 256, 0, st>>>(reinterpret_cast<float4*>(gacc), counts);
     GART_LAUNCH_CHECK();
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int T = cf.tiles_x * cf.tiles_y;

@@ -22,10 +22,14 @@ def test_shard_views_partition():
 
 
 def test_launch_count_and_bytes():
-    assert bench.launches_per_step(155 * 103) == 12 + (7 + 2 * 5) + 11 + 3     # 14 tile bits -> 2 radix passes
-    assert bench.launches_per_step(64) == 12 + (7 + 5) + 11 + 3
-    B = bench.algorithmic_bytes_backward(H=100, P=10, n_vis=5, n_pixels=64, K=16, mask_words=2)
-    assert B == 1600 + 160 + 4 * 68 * 5 + 4 * 59 * 5 + 768
+    assert bench.launches_per_step(155 * 103) == 12 + (7 + 2 * 5) + 11 + 4     # 14 tile bits -> 2 radix passes
+    assert bench.launches_per_step(64) == 12 + (7 + 5) + 11 + 4
+    B = bench.algorithmic_bytes_backward(H=100, P=10, n_vis=5, n_pixels=64, K=16)
+    assert B == 1600 + 40 + 4 * 61 * 5 + 4 * 59 * 5 + 28 * 64
+    # the traffic model adds its per-unit figures
+    t = bench.TRAFFIC_MODEL
+    assert bench.measured_traffic_backward(0, 0, 10) == 10 * t["scatter_write_per_gaussian"]
+    assert bench.measured_traffic_backward(7, 0, 0) == 7 * t["pairs_per_hit"]
 
 
 def _worker(rank, world, port, out):
