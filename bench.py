@@ -50,7 +50,7 @@ def launches_per_step(n_tiles: int) -> int:
     passes = (bits + 7) // 8
     bounds = 1 + 2 * (1 + 3 + 1) + 1          # bounds kernel, two radix passes, record gather
     tile_map = 1 + 3 + 1 + 1 + passes * (1 + 3 + 1) + 1
-    forward = 1 + 1 + 3 + 3 + 1 + 1 + 1
+    forward = 1 + 1 + 3 + 3 + 1 + 1 + 3          # mask, tile sort, two scans, totals, evaluation, sweep per ray-length class
     backward = 4                                # zero, pair kernel, per-slot conversion, scatter of the SH gradient
     return bounds + tile_map + forward + backward
 

@@ -730,12 +730,25 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
     }
 }
 
-__global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs,
-                                                                          uint64_t* __restrict__ long_keys, int64_t n_rays,
-                                                                          float bg0, float bg1, float bg2,
-                                                                          float* __restrict__ color, float* __restrict__ t_final,
-                                                                          float4* __restrict__ lt, uint32_t* __restrict__ ray_gid,
-                                                                          uint32_t* __restrict__ ray_slot, const uint32_t* __restrict__ counts) {
+// One launch per class of ray length, so that each gets the registers and the shared memory it needs and no more
+// (short rays then run at several times the occupancy of the longest): class 0 up to 64 hits, class 1 up to 256,
+// class 2 beyond.  Every launch walks all rays and a warp returns at once if its ray belongs to another class;
+// class 0 also writes the background colour of rays without hits.
+template <int CLS>
+struct SweepClass {
+    static constexpr int LO = CLS == 0 ? 0 : (CLS == 1 ? 64 : 256);                 // exclusive lower bound of n
+    static constexpr int CAP = CLS == 0 ? 64 : (CLS == 1 ? 256 : SORT_CAP);         // entries staged per warp
+    static constexpr int MIN_BLOCKS = CLS == 0 ? 12 : (CLS == 1 ? 6 : 4);
+    static constexpr int SMEM = SWEEP_WARPS * CAP * 28;
+};
+
+template <int CLS>
+__global__ void __launch_bounds__(SWEEP_WARPS * 32, SweepClass<CLS>::MIN_BLOCKS)
+fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs, uint64_t* __restrict__ long_keys, int64_t n_rays,
+                      float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
+                      float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
+                      const uint32_t* __restrict__ counts) {
+    constexpr int CAP = SweepClass<CLS>::CAP;
     if (counts[GART_CNT_ERROR]) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t r = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
@@ -743,24 +756,29 @@ __global__ void __launch_bounds__(SWEEP_WARPS * 32) fwd_sort_sweep_kernel(const 
     const size_t b = ray_off[r];
     const int n = (int)(ray_off[r + 1] - ray_off[r]);
     if (n == 0) {
-        if (lane == 0) {
+        if (CLS == 0 && lane == 0) {
             color[3 * r] = bg0; color[3 * r + 1] = bg1; color[3 * r + 2] = bg2;
             t_final[r] = 1.0f;
         }
         return;
     }
+    if (n <= SweepClass<CLS>::LO || (CLS < 2 && n > CAP)) return;
     const float4* rec = recs + b * 2;
-    extern __shared__ __align__(16) float4 sweep_smem[];   // SORT_CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
-    float4* s_cs = sweep_smem + (size_t)warp * SORT_CAP;
-    uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP) + (size_t)warp * SORT_CAP;
-    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * SORT_CAP * 3 / 2) + (size_t)warp * SORT_CAP;
+    extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
+    float4* s_cs = sweep_smem + (size_t)warp * CAP;
+    uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
+    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
 #define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot, s_cs, s_al, s_tg)
-    if (n <= 32) GART_SWEEP(1);
-    else if (n <= 64) GART_SWEEP(2);
-    else if (n <= 128) GART_SWEEP(4);
-    else if (n <= 256) GART_SWEEP(8);
-    else if (n <= SORT_CAP) GART_SWEEP(16);
-    else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot);
+    if (CLS == 0) {
+        if (n <= 32) GART_SWEEP(1);
+        else GART_SWEEP(2);
+    } else if (CLS == 1) {
+        if (n <= 128) GART_SWEEP(4);
+        else GART_SWEEP(8);
+    } else {
+        if (n <= SORT_CAP) GART_SWEEP(16);
+        else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, ray_gid, ray_slot);
+    }
 #undef GART_SWEEP
 }
 
@@ -873,12 +891,18 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);
-    constexpr int sweep_smem = SWEEP_WARPS * SORT_CAP * 28;
-    if (cudaFuncSetAttribute(fwd_sort_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sweep_smem) != cudaSuccess) return GART_ERR_CUDA;
-    fwd_sort_sweep_kernel<<<(unsigned)blocks, SWEEP_WARPS * 32, sweep_smem, st>>>(ray_off, w.recs, w.long_keys, n_rays,
-                                                                         cfg->background[0], cfg->background[1], cfg->background[2],
-                                                                         color, t_final, reinterpret_cast<float4*>(lt), ray_gid,
-                                                                         ray_slot, counts);
+    float4* lt4 = reinterpret_cast<float4*>(lt);
+    const float* bg = cfg->background;
+#define GART_SWEEP_LAUNCH(C)                                                                                                                    \
+    if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess)        \
+        return GART_ERR_CUDA;                                                                                                                   \
+    fwd_sort_sweep_kernel<C><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, bg[0], bg[1], \
+                                                                                             bg[2], color, t_final, lt4, ray_gid, ray_slot, counts); \
+    GART_LAUNCH_CHECK();
+    GART_SWEEP_LAUNCH(2)   // the longest rays first
+    GART_SWEEP_LAUNCH(1)
+    GART_SWEEP_LAUNCH(0)
+#undef GART_SWEEP_LAUNCH
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
