@@ -20,9 +20,9 @@ namespace gart {
 
 constexpr int BWD_WARPS = 4;
 constexpr int BWD_THREADS = BWD_WARPS * 32;
-constexpr int BWD_CHUNK = 8;                           // LT entries per lane and per pipeline stage
+constexpr int BWD_CHUNK = 7;                           // LT entries per lane and per pipeline stage
 constexpr int BWD_STAGE_F4 = BWD_CHUNK * 32;           // float4 per stage (8 KB)
-constexpr int BWD_STAGES = 3;                          // LT pipeline depth per warp
+constexpr int BWD_STAGES = 2;                          // LT pipeline depth per warp
 constexpr int BWD_LT_SMEM = BWD_WARPS * BWD_STAGES * BWD_STAGE_F4 * 16;
 constexpr int BWD_PF4 = 5;                             // float4 per lane of the staged evaluation record
 constexpr int BWD_DYN_SMEM = BWD_LT_SMEM + BWD_THREADS * BWD_PF4 * 16;
