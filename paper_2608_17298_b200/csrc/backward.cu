@@ -66,13 +66,38 @@ __device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__
     return d;
 }
 
+// A pair's geometry, affine in the pixel position (u, v) inside the tile: d_g = dgA + u c0 + v c1 and
+// o_g x d_g = crA + u a1 + v b1 (a1 = c0 x m, b1 = c1 x m; dgA, crA the values at the tile's first pixel).
+struct PairGeo {
+    float3 c0, c1, dgA, a1, b1, crA;
+};
+
+__device__ __forceinline__ PairGeo pair_geo(const PreRec& P, int x0, int y0) {
+    PairGeo g;
+    g.c0 = P.c0; g.c1 = P.c1;
+    g.a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
+    g.b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
+    const float dx0 = (float)(x0 - P.ix) - P.rx, dy0 = (float)(y0 - P.iy) - P.ry;
+    g.dgA = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy0, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy0, P.dgr.y)),
+                        fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy0, P.dgr.z)));
+    g.crA = make_float3(fmaf(g.a1.x, dx0, fmaf(g.b1.x, dy0, P.k.x)), fmaf(g.a1.y, dx0, fmaf(g.b1.y, dy0, P.k.y)),
+                        fmaf(g.a1.z, dx0, fmaf(g.b1.z, dy0, P.k.z)));
+    return g;
+}
+
 // Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
 // geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz), geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh.
+// With y = d_g x (o_g x d_g) and a = |d_g|^2 the maximum-response point is x_g = y / a, so
+// G x_g = (G / a) y and G x_g x_g^T = (G / a^2) y y^T.
 template <int TS, int K>
-__device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* geo, const float4* spix, float fbx, float fby, int p,
-                                        const float4 L) {
+__device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* geo, const float4* spix, int p, const float4 L) {
     const float4 pa = spix[PixLayout<TS>::index(p, 0, 0)], pb = spix[PixLayout<TS>::index(p, 1, 0)];   // spix points at the lane's copy
-    const RayGeo r = ray_geo(P, (fbx + pa.w) - P.rx, (fby + pb.w) - P.ry);   // small integers: the sums are exact
+    const float u = pa.w, v = pb.w;
+    const float3 dg = make_float3(fmaf(P.c0.x, u, fmaf(P.c1.x, v, P.dgA.x)), fmaf(P.c0.y, u, fmaf(P.c1.y, v, P.dgA.y)),
+                                  fmaf(P.c0.z, u, fmaf(P.c1.z, v, P.dgA.z)));
+    const float3 cr = make_float3(fmaf(P.a1.x, u, fmaf(P.b1.x, v, P.crA.x)), fmaf(P.a1.y, u, fmaf(P.b1.y, v, P.crA.y)),
+                                  fmaf(P.a1.z, u, fmaf(P.b1.z, v, P.crA.z)));
+    const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
     float Y[K];
     sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
     const float3 g = make_float3(pb.x, pb.y, pb.z);
@@ -81,12 +106,12 @@ __device__ __forceinline__ void bwd_hit(const PreRec& P, ShRegs<K>& R, float* ge
     R.accumulate(Y, w);
     const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
     geo[9] += ad;
-    const float G = -0.5f * ad;
-    const float3 xg = ray_xg(r);
-    const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
-    geo[0] += gx; geo[1] += gy; geo[2] += gz;
-    geo[3] = fmaf(gx, xg.x, geo[3]); geo[4] = fmaf(gy, xg.y, geo[4]); geo[5] = fmaf(gz, xg.z, geo[5]);
-    geo[6] = fmaf(gx, xg.y, geo[6]); geo[7] = fmaf(gx, xg.z, geo[7]); geo[8] = fmaf(gy, xg.z, geo[8]);
+    const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
+    const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+    geo[0] = fmaf(s1, yx, geo[0]); geo[1] = fmaf(s1, yy, geo[1]); geo[2] = fmaf(s1, yz, geo[2]);
+    const float tx = s2 * yx, ty = s2 * yy, tz = s2 * yz;
+    geo[3] = fmaf(tx, yx, geo[3]); geo[4] = fmaf(ty, yy, geo[4]); geo[5] = fmaf(tz, yz, geo[5]);
+    geo[6] = fmaf(tx, yy, geo[6]); geo[7] = fmaf(tx, yz, geo[7]); geo[8] = fmaf(ty, yz, geo[8]);
 }
 
 template <int TS, int DEG>
@@ -196,16 +221,14 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         // descriptor two groups ahead: the producer may reach it later in this group (not yet: its loads are in flight)
         const GroupDesc<MW> nxt2 = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
         produce(cur, nxt, nxt2, 1);
-        PreRec P;
         ShRegs<K> R;
         float geo[11];
 #pragma unroll
         for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
         cp_async_wait_all();   // this lane's record has landed (a lane reads only what it copied itself)
-        P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale data for lanes without hits: never used)
+        const PairGeo P = pair_geo(unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]), x0, y0);   // (stale data for lanes without hits: never used)
         R.clear();
         if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
-        const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
         const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % BWD_STAGES;
@@ -219,10 +242,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                 const int p0 = cur.pm.next();
                 const int p1 = cur.pm.next();
                 const float4 L0 = se[0], L1 = se[32];
-                bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, p0, L0);
-                bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, p1, L1);
+                bwd_hit<TS, K>(P, R, geo, spix_lane, p0, L0);
+                bwd_hit<TS, K>(P, R, geo, spix_lane, p1, L1);
             }
-            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, fbx, fby, cur.pm.next(), se[0]);
+            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, cur.pm.next(), se[0]);
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
