@@ -87,6 +87,35 @@ def test_ragged_image_and_background():
         full_parity(scene, cams[0], G.Config(tile_size=ts, background=(0.2, 0.5, 0.1)))
 
 
+def test_forward_without_ray_lists_gives_the_same_view():
+    """The per-ray ordered lists are optional outputs: without them colour, T_final, LT and the gradient are the
+    same bits (the lists only serve the pixel-centric baseline and the parity checks)."""
+    scene, cams = gs.config_cluster(n=3000, width=96, height=80, seed=11)
+    cam, cfg = cams[0], G.Config()
+    g = G.Gaussians.from_numpy(scene)
+    dl = torch.from_numpy(gs.upstream_gradient(cam, 0)).cuda()
+    cap_pairs, cap_hits = G.size_view(cfg, g, cam, slack=1.0)
+    outs = []
+    for lists in (True, False):
+        buf = G.ViewBuffers(g.n, g.sh_degree, cam, cfg, cap_pairs, cap_hits)
+        buf.ray_gid.fill_(-1)
+        G.run_bounds_tile_map(cfg, g, cam, buf)
+        G.run_forward(cfg, g, cam, buf, ray_lists=lists)
+        G.run_backward(cfg, g, cam, buf, dl)
+        torch.cuda.synchronize()
+        cnt = G.gart_read_counts(buf.counts)
+        assert cnt[G.CNT_ERROR] == 0 and cnt[G.CNT_HITS] > 0
+        outs.append((buf.color.cpu().numpy().copy(), buf.t_final.cpu().numpy().copy(),
+                     buf.lt.cpu().numpy()[:cnt[G.CNT_LT_SLOTS]].copy(), buf.ray_gid.cpu().numpy().copy(), cnt))
+        grad = buf.grad.cpu().numpy()[:g.n]
+        outs[-1] += (grad.copy(),)
+    a, b = outs
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and list(a[4]) == list(b[4])
+    # LT entries are written once each (padding is never written: compare the written ones through the gradient)
+    assert np.allclose(a[5], b[5], rtol=1e-5, atol=1e-7)          # atomics: summation order may differ
+    assert np.all(b[3] == -1) and np.any(a[3] != -1)               # the list was left untouched
+
+
 def test_straddling_gaussian_and_culling_rules():
     scene, cams = gs.config_tiny(n=64, seed=9)
     scene.mean[0] = (0.05, -0.02, 0.3); scene.scale[0] = (0.4, 0.5, 0.45); scene.opacity[0] = 0.6   # crosses the camera plane
