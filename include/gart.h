@@ -107,9 +107,9 @@ int32_t gart_mask_words(int32_t tile_size);
  * double precision, and the pre-computations of the ray evaluation (W = S^-1 R^T and o_g of
  * Eq. 5, expressed relative to a per-Gaussian reference pixel so that fp32 evaluation stays
  * well conditioned).  Gaussians with a non-empty rectangle are renumbered for the view: a stable
- * sort on the tile of the rectangle's corner (x0, y0) gives each a slot 0..V-1 (V = counts[VISIBLE]);
- * later steps read and update per-Gaussian data by slot, which keeps the accesses of neighbouring
- * tiles close in memory.
+ * sort on the tile row of the rectangle's corner (y0 / tile_size) gives each a slot 0..V-1
+ * (V = counts[VISIBLE]); later steps read and update per-Gaussian data by slot, so that what a row of
+ * tiles touches is a few MB that stay in L2 (the scene's own order carries no such locality).
  *   rect   [n,4] int32 out: inclusive pixel range x0,y0,x1,y1 of pixel centres inside the
  *                bound, clipped to the image; (0,0,-1,-1) if empty.
  *   cls    [n]   uint8 out: 0 culled (sigma <= alpha_min, or support entirely at depth <= near_z),

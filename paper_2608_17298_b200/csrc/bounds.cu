@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
             p[5] = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
             p[6] = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
         }
-        keys[i] = vis ? (uint32_t)((y0 / ts) * tiles_x + x0 / ts) : key_none;
+        keys[i] = vis ? (uint32_t)(y0 / ts) : key_none;   // tile row of the rectangle's corner
         vals[i] = (uint32_t)i;
     }
     const unsigned bv = __ballot_sync(0xffffffffu, vis), bs = __ballot_sync(0xffffffffu, straddle);
@@ -260,7 +260,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
     const int ts = cfg->tile_size;
     const int tiles_x = (cam->width + ts - 1) / ts, tiles_y = (cam->height + ts - 1) / ts;
-    const uint32_t key_none = (uint32_t)(tiles_x * tiles_y);   // sorts after every tile
+    const uint32_t key_none = (uint32_t)tiles_y;   // sorts after every tile row
     int bits = 1;
     while ((1u << bits) <= key_none) ++bits;
     uint32_t* const kbuf[2] = {w.keys0, w.keys1};

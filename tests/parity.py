@@ -129,11 +129,11 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     # copies in rank order
     assert np.array_equal(gpu["rank_sid"], gpu["slot_of_gid"][gpu["pair_gid"][order]])
     assert np.array_equal(gpu["rank_mask"], gpu["pair_mask"][order])
-    # slots: visible Gaussians in the order of the tile of their rectangle's corner, ids ascending inside a tile
+    # slots: visible Gaussians in the order of the tile row of their rectangle's corner, ids ascending inside a row
     rect_ = gpu["rect"]
     vis = rect_[:, 2] >= rect_[:, 0]
     V = int(vis.sum())
-    key_ = (rect_[:, 1] // ts) * tiles_x + rect_[:, 0] // ts
+    key_ = rect_[:, 1] // ts
     want_order = np.nonzero(vis)[0][np.argsort(key_[vis], kind="stable")]
     assert np.array_equal(gpu["gid_of_slot"][:V], want_order.astype(np.uint32)) and np.all(gpu["gid_of_slot"][V:] == 0xffffffff)
     inv = np.full(rect_.shape[0], 0xffffffff, np.uint32)
