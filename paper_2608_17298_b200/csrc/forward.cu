@@ -216,49 +216,71 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
     if (n == 0) { if (lane == 0) tile_slots[tile] = 0; return; }
     for (int d = lane; d < NB; d += 32) hist[w][d] = 0;
     __syncwarp();
-    for (uint32_t r0 = 0; r0 < n; r0 += 32)
-        if (r0 + lane < n) atomicAdd(&hist[w][mask_popc<MW>(pair_mask, begin + r0 + lane)], 1u);
+    // every pass walks the tile's pairs 32 at a time; TSU chunks are loaded together so that their (dependent)
+    // loads overlap
+    constexpr int TSU = 4;
+    for (uint32_t r0 = 0; r0 < n; r0 += 32 * TSU) {
+        uint32_t c[TSU];
+#pragma unroll
+        for (int u = 0; u < TSU; ++u) c[u] = r0 + 32 * u + lane < n ? mask_popc<MW>(pair_mask, begin + r0 + 32 * u + lane) : 0xffffffffu;
+#pragma unroll
+        for (int u = 0; u < TSU; ++u)
+            if (c[u] != 0xffffffffu) atomicAdd(&hist[w][c[u]], 1u);
+    }
     __syncwarp();
     if (lane == 0) {   // first rank of every hit count, largest count first
         uint32_t run = 0;
         for (int c = NT; c >= 0; --c) { const uint32_t t = hist[w][c]; hist[w][c] = run; run += t; }
     }
     __syncwarp();
-    for (uint32_t r0 = 0; r0 < n; r0 += 32) {
-        const bool act = r0 + lane < n;
-        const unsigned amask = __ballot_sync(0xffffffffu, act);
-        if (act) {
-            const uint32_t j = begin + r0 + lane;
-            const uint32_t c = mask_popc<MW>(pair_mask, j);
-            const unsigned peers = __match_any_sync(amask, c);
-            const uint32_t rk = __popc(peers & ((1u << lane) - 1u));
-            const uint32_t pos = hist[w][c] + rk;
-            __syncwarp(amask);
-            if (rk == 0) hist[w][c] += __popc(peers);
-            __syncwarp(amask);
-            pair_order[begin + pos] = j;
+    for (uint32_t r0 = 0; r0 < n; r0 += 32 * TSU) {
+        uint32_t c[TSU];
+#pragma unroll
+        for (int u = 0; u < TSU; ++u) c[u] = r0 + 32 * u + lane < n ? mask_popc<MW>(pair_mask, begin + r0 + 32 * u + lane) : 0xffffffffu;
+#pragma unroll
+        for (int u = 0; u < TSU; ++u) {   // in order: equal counts keep the order of the pair list
+            const bool act = c[u] != 0xffffffffu;
+            const unsigned amask = __ballot_sync(0xffffffffu, act);
+            if (act) {
+                const unsigned peers = __match_any_sync(amask, c[u]);
+                const uint32_t rk = __popc(peers & ((1u << lane) - 1u));
+                const uint32_t pos = hist[w][c[u]] + rk;
+                __syncwarp(amask);
+                if (rk == 0) hist[w][c[u]] += __popc(peers);
+                __syncwarp(amask);
+                pair_order[begin + pos] = begin + r0 + 32 * u + lane;
+            }
         }
     }
     __threadfence_block();
     __syncwarp();
     uint32_t run = 0;
-    for (uint32_t r0 = 0; r0 < n; r0 += 32) {
-        const bool act = r0 + lane < n;
-        const uint32_t j = act ? __ldcg(pair_order + begin + r0 + lane) : 0u;
-        uint32_t c = 0;
-        if (act) {
-            const size_t q = (size_t)begin + r0 + lane;
+    for (uint32_t r0 = 0; r0 < n; r0 += 32 * TSU) {
+        uint32_t j[TSU], sid[TSU], wv[TSU][MW];
 #pragma unroll
-            for (int m = 0; m < MW; ++m) {
-                const uint32_t wv = __ldg(pair_mask + (size_t)j * MW + m);
-                rank_mask[q * MW + m] = wv;
-                c += __popc(wv);
-            }
-            rank_sid[q] = __ldg(slot_of_gid + __ldg(pair_gid + j));
-            rank_gstart[q] = run;
+        for (int u = 0; u < TSU; ++u) j[u] = r0 + 32 * u + lane < n ? __ldcg(pair_order + begin + r0 + 32 * u + lane) : 0xffffffffu;
+#pragma unroll
+        for (int u = 0; u < TSU; ++u) {
+            const bool act = j[u] != 0xffffffffu;
+#pragma unroll
+            for (int m = 0; m < MW; ++m) wv[u][m] = act ? __ldg(pair_mask + (size_t)j[u] * MW + m) : 0u;
+            sid[u] = act ? __ldg(slot_of_gid + __ldg(pair_gid + j[u])) : 0u;
         }
-        const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
-        run += 32u * cmax;
+#pragma unroll
+        for (int u = 0; u < TSU; ++u) {
+            uint32_t c = 0;
+#pragma unroll
+            for (int m = 0; m < MW; ++m) c += __popc(wv[u][m]);
+            if (j[u] != 0xffffffffu) {
+                const size_t q = (size_t)begin + r0 + 32 * u + lane;
+#pragma unroll
+                for (int m = 0; m < MW; ++m) rank_mask[q * MW + m] = wv[u][m];
+                rank_sid[q] = sid[u];
+                rank_gstart[q] = run;
+            }
+            const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
+            run += 32u * cmax;
+        }
     }
     if (lane == 0) tile_slots[tile] = run;
 }
