@@ -100,19 +100,6 @@ __device__ __forceinline__ PreRec load_pre(const float4* __restrict__ rec) {
     return unpack_pre(__ldg(rec), __ldg(rec + 1), __ldg(rec + 2), __ldg(rec + 3), __ldg(rec + 4));
 }
 
-// SH coefficients of a record into registers, by 16-byte loads (the padding is loaded and dropped).
-template <int SW>
-__device__ __forceinline__ void load_sh(const float4* __restrict__ rec, float* shc) {
-#pragma unroll
-    for (int q = 0; q < (SW + 3) / 4; ++q) {
-        const float4 t = __ldg(rec + 5 + q);
-        shc[4 * q] = t.x;
-        if (4 * q + 1 < SW) shc[4 * q + 1] = t.y;
-        if (4 * q + 2 < SW) shc[4 * q + 2] = t.z;
-        if (4 * q + 3 < SW) shc[4 * q + 3] = t.w;
-    }
-}
-
 // One-instruction reciprocal and 2^x of the special-function unit (about 1 and 2 ulp).
 __device__ __forceinline__ float fast_rcp(float x) {
     float y;
@@ -150,26 +137,6 @@ __device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy)
     const float D2 = cc * r.inv_a;
     r.alpha = p.sigma * fast_exp2(-0.72134752044448170f * D2);
     r.tnum = fmaf(p.m.x, r.dg.x, fmaf(p.m.y, r.dg.y, p.m.z * r.dg.z));
-    return r;
-}
-
-// The geometric part alone (no response): what the point of maximum response needs.
-struct RayGeo {
-    float inv_a;   // 1 / |d_g|^2
-    float3 dg;     // d_g
-    float3 cr;     // o_g x d_g
-};
-
-__device__ __forceinline__ RayGeo ray_geo(const PreRec& p, float dx, float dy) {
-    RayGeo r;
-    const float ex = fmaf(p.c0.x, dx, p.c1.x * dy);
-    const float ey = fmaf(p.c0.y, dx, p.c1.y * dy);
-    const float ez = fmaf(p.c0.z, dx, p.c1.z * dy);
-    r.dg = make_float3(p.dgr.x + ex, p.dgr.y + ey, p.dgr.z + ez);
-    r.cr.x = fmaf(ey, p.m.z, fmaf(-ez, p.m.y, p.k.x));
-    r.cr.y = fmaf(ez, p.m.x, fmaf(-ex, p.m.z, p.k.y));
-    r.cr.z = fmaf(ex, p.m.y, fmaf(-ey, p.m.x, p.k.z));
-    r.inv_a = fast_rcp(fmaf(r.dg.x, r.dg.x, fmaf(r.dg.y, r.dg.y, r.dg.z * r.dg.z)));
     return r;
 }
 
@@ -260,9 +227,6 @@ struct PairMask<2> {
         return base + b;
     }
 };
-
-__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // ---------------------------------------------------------------------------------------------
 // Real spherical harmonics (index k = l(l+1)+m) of a unit vector, first K values.
@@ -357,7 +321,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
-// global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned)
 // Orders this thread's earlier shared-memory accesses (generic proxy) before later accesses of the
 // asynchronous proxy: issued before a bulk copy overwrites a buffer that was just read.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -391,6 +354,7 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
+// global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned) with an L2 eviction policy
 __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
@@ -400,11 +364,6 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uin
 __device__ __forceinline__ void red_add_f4_hint(float4* dst, float a, float b, float c, float d, uint64_t policy) {
     asm volatile("red.global.add.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
                  ::"l"(dst), "f"(a), "f"(b), "f"(c), "f"(d), "l"(policy)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
 
