@@ -304,6 +304,22 @@ def run_ours(args):
         if i > 0:
             at.append(a0.elapsed_time(a1))
     atomic_ms = float(np.mean(at)) if at else None
+    # ---- hybrid backward (colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric), same view
+    hybrid_ms = None
+    if args.hybrid_reps > 0:
+        import dataclasses
+        cfg_h = dataclasses.replace(cfg, lt_format=1)
+        G.run_forward(cfg_h, g, cams[last_v], buf, stream, ray_lists=True)
+        ht = []
+        for i in range(args.hybrid_reps + 1):                    # one untimed run first
+            a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            G.run_backward_hybrid(cfg_h, g, cams[last_v], buf, dls[last_v], ga, stream)
+            a1.record(stream)
+            torch.cuda.synchronize()
+            if i > 0:
+                ht.append(a0.elapsed_time(a1))
+        hybrid_ms = float(np.mean(ht))
     last = cl[-1]
     prim_last_ms = float(stage[-1, 2])
     del ga
@@ -391,6 +407,7 @@ def run_ours(args):
         "backward_hits_per_s": Hm / (bwd_ms * 1e-3),
         "backward_atomic_ms": atomic_ms,
         "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
+        "backward_hybrid_ms": hybrid_ms,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(G.tiles(cams[0], cfg.tile_size)) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
     }
@@ -409,6 +426,7 @@ def main():
     ap.add_argument("--tile-size", type=int, default=8, choices=[8, 16])
     ap.add_argument("--slack", type=float, default=1.25)
     ap.add_argument("--atomic-reps", type=int, default=2)
+    ap.add_argument("--hybrid-reps", type=int, default=1, help="timed runs of the hybrid backward on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--oracle-frac", type=float, default=0.08)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -11,6 +11,7 @@
  *   gart_backward  primitive-centric backward: one thread per (tile, Gaussian) pair gathers
  *                  the gradients of that Gaussian over the pair's hit pixels
  *   gart_backward_atomic   the pixel-centric baseline: one thread per ray, atomicAdd per hit
+ *   gart_backward_hybrid   colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric
  *
  * Conventions
  *   - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
@@ -56,6 +57,9 @@ typedef struct {
     float near_z;         /* depth of the near plane used only to classify Gaussians */
     float background[3];  /* colour multiplied by the final transmittance */
     int32_t tile_size;    /* 8 (the paper's choice, Sec. 4.4) or 16 */
+    int32_t lt_format;    /* what gart_forward stores per hit: 0 = the 16-byte entry that gart_backward reads,
+                             1 = only its fourth word, 4 bytes per hit (for gart_backward_hybrid, Sec. 4.4
+                             "Hybrid approach"); lt then holds cap_hits floats */
 } gart_config;
 
 /* Host struct. */
@@ -245,6 +249,22 @@ gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g
                                  const float *pre, const uint32_t *slot_of_gid, const uint32_t *ray_off, const uint32_t *ray_gid,
                                  const uint32_t *ray_slot, const float *lt, const float *dL_dcolor,
                                  float *grad, const uint32_t *counts, void *stream);
+
+/*
+ * Hybrid backward (Sec. 4.4 "Hybrid approach"; "Hybrid" of Sec. 5.1): the colour gradients dL/dsh are accumulated
+ * primitive-centric from an intermediate buffer of ONE word per hit, the remaining terms (mean, scale,
+ * quaternion, opacity) pixel-centric with 10 scalar atomicAdd per hit.  Needs gart_forward run with
+ * cfg->lt_format = 1 (lt_w [cap_hits] fp32: word 3 of the full entry, same slot layout) and with the per-ray id
+ * list (ray_off, ray_gid); the 4 + 4 bytes per hit replace the 16 of the full entry (the paper, which re-traces
+ * the ray in its pixel-centric part, keeps 4).  Same result as gart_backward up to rounding and summation order;
+ * same workspace as gart_backward.  Errors as gart_backward; INVALID_ARG if cfg->lt_format != 1.
+ */
+gart_status gart_backward_hybrid(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
+                                 const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
+                                 const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
+                                 const uint32_t *tile_lt_base, const float *lt_w, const uint32_t *ray_off, const uint32_t *ray_gid,
+                                 const float *dL_dcolor, float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes,
+                                 void *stream);
 
 /* Copy the counts block to host memory (synchronises the stream). counts_host: host, GART_COUNTS_WORDS words. */
 gart_status gart_read_counts(const uint32_t *counts, uint32_t *counts_host, void *stream);

@@ -64,4 +64,118 @@ __device__ __forceinline__ GeoGrad moments_to_grads(const float* v, const float*
     return o;
 }
 
+// Per-pixel data of the tile in shared memory: two float4 per pixel, (d.x, d.y, d.z, x) and (g.r, g.g, g.b, y)
+// with d the unit ray direction, g = dL/dC and (x, y) the pixel's position in the tile.  Lanes of a warp read
+// DIFFERENT pixels at the same time, so a single copy suffers bank conflicts at random; with 8 copies, copy j
+// laid out in the 16-byte bank group j only and lane l reading copy l mod 8, the 8 lanes that a 16-byte shared
+// load serves together never collide.  (Tiles of 256 pixels keep one copy, 3 float4 apart.)
+template <int TS>
+struct PixLayout {
+    static constexpr int COPIES = TS == 8 ? 8 : 1;
+    static constexpr int STRIDE = COPIES == 1 ? 3 : 2;                 // float4 per pixel within a copy
+    static constexpr int F4 = TS * TS * STRIDE * COPIES;               // float4 in all
+    __device__ static __forceinline__ int index(int p, int h, int copy) { return (p * STRIDE + h) * COPIES + copy; }
+};
+
+// Descriptor of one rank group as seen by a lane (read from the rank-ordered copies: coalesced).
+template <int MW>
+struct GroupDesc {
+    PairMask<MW> pm;
+    uint32_t sid;      // slot of the pair's Gaussian in the view's order
+    int c;             // hits of this lane's pair
+    int cmax;          // hits of the group's first pair = the largest of the group
+    uint32_t gstart;   // first LT entry of the group, relative to the tile's base
+};
+
+template <int MW>
+__device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
+                                                    const uint32_t* __restrict__ rank_gstart, uint32_t begin, uint32_t n,
+                                                    uint32_t r0, int lane) {
+    GroupDesc<MW> d;
+    const bool act = r0 < n && r0 + lane < n;
+    const uint32_t q = begin + r0 + lane;
+    d.pm.load(rank_mask, act ? q : 0u, act);
+    d.c = d.pm.count();
+    d.sid = act ? __ldg(rank_sid + q) : 0u;
+    const uint32_t s0 = act ? __ldg(rank_gstart + q) : 0u;
+    d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
+    d.gstart = __shfl_sync(0xffffffffu, s0, 0);
+    return d;
+}
+
+// Zero the accumulation records of the view's slots (their number lives on the device): grid-stride.
+static __global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc4, const uint32_t* __restrict__ counts) {
+    const size_t total = (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
+        gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// One thread per slot: convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity and
+// write words 0..15 of the Gaussian's gradient record (all 32 lanes busy with the ~300-instruction conversion).
+static __global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* __restrict__ qs, const uint32_t* __restrict__ gid_of_slot,
+                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    constexpr int F4 = GART_GRAD_WORDS / 4;
+    const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+    const float4* gp = gacc4 + (size_t)sid * F4;
+    const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
+    const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
+    float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
+    const float v[3] = {a.x, a.y, a.z};
+    const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
+    const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+    const float sc[3] = {s4.x, s4.y, s4.z};
+    const GeoGrad o = moments_to_grads(v, Q, q, sc);
+    out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
+    out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
+    out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
+    out[3] = d;
+}
+
+// In the order of the gradient records (sequential writes): 16 lanes per Gaussian; a Gaussian without a slot gets
+// a zero record, the others words 16..63 (dL/dsh) of their slot's accumulation record.  A half-warp handles
+// FIN_ROWS Gaussians with all their loads in flight at once.
+constexpr int FIN_ROWS = 4;
+static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, const uint32_t* __restrict__ slot_of_gid,
+                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    constexpr int F4 = GART_GRAD_WORDS / 4;
+    const int64_t hw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // half-warp
+    const int l = threadIdx.x & 15;
+    const int64_t i0 = hw * FIN_ROWS;
+    uint32_t s[FIN_ROWS];
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r) s[r] = i0 + r < n ? __ldg(slot_of_gid + i0 + r) : 0xffffffffu;
+    float4 v[FIN_ROWS];
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r)
+        v[r] = (s[r] != 0xffffffffu && l >= 4) ? __ldcs(gacc4 + (size_t)s[r] * F4 + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int r = 0; r < FIN_ROWS; ++r)
+        if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu)) __stcs(grad4 + (size_t)(i0 + r) * F4 + l, v[r]);
+}
+
+
+// Launches shared by the backward variants: zero the accumulation records of the view's slots; after the
+// accumulation, convert the moments per slot and write the caller's gradient records.
+static inline gart_status launch_zero_accumulators(float* gacc, int64_t n, const uint32_t* counts, cudaStream_t st) {
+    const int64_t zero_blocks = ceil_div(n * (GART_GRAD_WORDS / 4), 256);
+    bwd_zero_kernel<<<(unsigned)(zero_blocks < 148 * 32 ? zero_blocks : 148 * 32), 256, 0, st>>>(reinterpret_cast<float4*>(gacc), counts);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}
+static inline gart_status launch_finalize(int64_t n, const float4* qs, const uint32_t* slot_of_gid, const uint32_t* gid_of_slot,
+                                          const float* gacc, float* grad, const uint32_t* counts, cudaStream_t st) {
+    bwd_convert_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(qs, gid_of_slot, reinterpret_cast<const float4*>(gacc),
+                                                                   reinterpret_cast<float4*>(grad), counts);
+    GART_LAUNCH_CHECK();
+    bwd_scatter_kernel<<<(unsigned)ceil_div(ceil_div(n, FIN_ROWS) * 16, 256), 256, 0, st>>>(n, slot_of_gid, reinterpret_cast<const float4*>(gacc),
+                                                                                            reinterpret_cast<float4*>(grad), counts);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}
+
 }  // namespace gart

@@ -28,7 +28,7 @@ GRAD_WORDS = 64
 EXPORTS = [
     "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
     "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_forward_workspace_bytes", "gart_forward",
-    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_read_counts",
+    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_read_counts",
     "gart_view_host_arena_bytes", "gart_view_host",
 ]
 
@@ -40,7 +40,8 @@ class GartError(RuntimeError):
 
 
 class _Config(C.Structure):
-    _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32)]
+    _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
+                ("lt_format", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -86,11 +87,12 @@ def lib():
         L.gart_backward_workspace_bytes.argtypes = [i64]
         L.gart_backward.argtypes = [vp] * 16 + [sz, vp]
         L.gart_backward_atomic.argtypes = [vp] * 13
+        L.gart_backward_hybrid.argtypes = [vp] * 18 + [sz, vp]
         L.gart_read_counts.argtypes = [vp, vp, vp]
         L.gart_view_host_arena_bytes.restype = sz
         L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
         L.gart_view_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
-        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic",
+        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid",
                    "gart_read_counts", "gart_view_host"):
             getattr(L, fn).restype = C.c_int
         _lib = L
@@ -104,10 +106,12 @@ class Config:
     near_z: float = 0.01
     background: tuple = (0.0, 0.0, 0.0)
     tile_size: int = 8
+    lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid)
 
     def c(self) -> _Config:
         s = _Config()
         s.alpha_min, s.near_z, s.tile_size = self.alpha_min, self.near_z, int(self.tile_size)
+        s.lt_format = int(self.lt_format)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s
@@ -291,6 +295,21 @@ def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, ray_o
                                       _dev(counts, i32, "counts"), _stream_ptr(stream)), "gart_backward_atomic")
 
 
+def gart_backward_hybrid(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
+                         rank_gstart, tile_lt_base, lt_w, ray_off, ray_gid, dL_dcolor, grad, counts, workspace, stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    i32, f32 = torch.int32, torch.float32
+    wp, wb = _ws(workspace)
+    _check(lib().gart_backward_hybrid(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                                      _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
+                                      _dev(tile_off, i32, "tile_off"),
+                                      _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
+                                      _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
+                                      _dev(lt_w, f32, "lt_w"), _dev(ray_off, i32, "ray_off"), _dev(ray_gid, i32, "ray_gid"),
+                                      _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
+                                      _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward_hybrid")
+
+
 def gart_read_counts(counts, stream=None):
     """Counts block as a list of unsigned ints (synchronises the stream)."""
     host = (C.c_uint32 * COUNTS_WORDS)()
@@ -382,6 +401,13 @@ def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=Non
 def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):
     gart_backward_atomic(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.ray_off, buf.ray_gid, buf.ray_slot, buf.lt, dL_dcolor,
                          grad, buf.counts, stream)
+
+
+def run_backward_hybrid(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
+    """cfg.lt_format must be 1 and the forward must have run with the same cfg and with the ray lists."""
+    gart_backward_hybrid(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask,
+                         buf.rank_gstart, buf.tile_lt_base, buf.lt, buf.ray_off, buf.ray_gid, dL_dcolor,
+                         buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
 
 
 def size_view(cfg, g, cam, slack=1.0, device="cuda"):

@@ -71,6 +71,17 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         G.run_backward_atomic(cfg, g, cam, buf, dl, ga)
         torch.cuda.synchronize()
         out["grad_atomic"] = to_np(ga)[:g.n]
+        # hybrid backward: the forward again with 4-byte LT entries (same buffers, everything else unchanged)
+        import dataclasses
+        cfg_h = dataclasses.replace(cfg, lt_format=1)
+        G.run_forward(cfg_h, g, cam, buf)
+        gh = torch.empty_like(buf.grad)
+        G.run_backward_hybrid(cfg_h, g, cam, buf, dl, gh)
+        torch.cuda.synchronize()
+        assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
+        out["grad_hybrid"] = to_np(gh)[:g.n]
+        # the other outputs of the forward do not depend on the LT format
+        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
     return out
 
 

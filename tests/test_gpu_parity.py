@@ -54,7 +54,8 @@ def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
     K = (scene.sh_degree + 1) ** 2
     s1 = assert_grad(gpu["grad"], ref, K)
     s2 = assert_grad(gpu["grad_atomic"], ref, K)
-    assert s1 > 0.995 and s2 > 0.995            # the conditioning floor is the exception, not the rule
+    s3 = assert_grad(gpu["grad_hybrid"], ref, K)
+    assert s1 > 0.995 and s2 > 0.995 and s3 > 0.995   # the conditioning floor is the exception, not the rule
     return gpu, ref
 
 
