@@ -304,6 +304,21 @@ def run_ours(args):
         if i > 0:
             at.append(a0.elapsed_time(a1))
     atomic_ms = float(np.mean(at)) if at else None
+    # ---- ownership ablation: a warp per pair instead of a thread (same buffers, after the atomic runs restored the lists)
+    warp_ms = None
+    if args.warp_reps > 0:
+        if args.atomic_reps <= 0:
+            G.run_forward(cfg, g, cams[last_v], buf, stream, ray_lists=False)
+        wt = []
+        for i in range(args.warp_reps + 1):
+            a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            G.run_backward_warp(cfg, g, cams[last_v], buf, dls[last_v], ga, stream)
+            a1.record(stream)
+            torch.cuda.synchronize()
+            if i > 0:
+                wt.append(a0.elapsed_time(a1))
+        warp_ms = float(np.mean(wt))
     # ---- hybrid backward (colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric), same view
     hybrid_ms = None
     if args.hybrid_reps > 0:
@@ -408,6 +423,7 @@ def run_ours(args):
         "backward_atomic_ms": atomic_ms,
         "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
         "backward_hybrid_ms": hybrid_ms,
+        "backward_warp_per_pair_ms": warp_ms,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(G.tiles(cams[0], cfg.tile_size)) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
     }
@@ -426,6 +442,7 @@ def main():
     ap.add_argument("--tile-size", type=int, default=8, choices=[8, 16])
     ap.add_argument("--slack", type=float, default=1.25)
     ap.add_argument("--atomic-reps", type=int, default=2)
+    ap.add_argument("--warp-reps", type=int, default=1, help="timed runs of the warp-per-pair backward on the last view (0: skip)")
     ap.add_argument("--hybrid-reps", type=int, default=1, help="timed runs of the hybrid backward on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--oracle-frac", type=float, default=0.08)

@@ -11,6 +11,7 @@
  *   gart_backward  primitive-centric backward: one thread per (tile, Gaussian) pair gathers
  *                  the gradients of that Gaussian over the pair's hit pixels
  *   gart_backward_atomic   the pixel-centric baseline: one thread per ray, atomicAdd per hit
+ *   gart_backward_warp     gart_backward with a warp per pair (ownership ablation)
  *   gart_backward_hybrid   colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric
  *
  * Conventions
@@ -249,6 +250,17 @@ gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g
                                  const float *pre, const uint32_t *slot_of_gid, const uint32_t *ray_off, const uint32_t *ray_gid,
                                  const uint32_t *ray_slot, const float *lt, const float *dL_dcolor,
                                  float *grad, const uint32_t *counts, void *stream);
+
+/*
+ * Ownership ablation (Sec. 4.4): gart_backward with one warp, not one thread, per (tile, Gaussian) pair.  Same
+ * arguments, same result up to summation order; the paper found it less efficient and so it is here.
+ */
+gart_status gart_backward_warp(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
+                               const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
+                               const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
+                               const uint32_t *tile_lt_base,
+                               const float *lt, const float *dL_dcolor,
+                               float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Hybrid backward (Sec. 4.4 "Hybrid approach"; "Hybrid" of Sec. 5.1): the colour gradients dL/dsh are accumulated

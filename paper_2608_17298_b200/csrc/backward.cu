@@ -297,3 +297,151 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
     return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);
 }
+
+// ------------------------------------------------------------------------------------------------------------
+// Ownership ablation (Sec. 4.4: "assigning a full warp is possible, we found it less efficient"): the same
+// gradient with one WARP per (tile, Gaussian) pair.  Lane e takes the pair's e-th (and e+32nd ...) hit, the 11 + 3K
+// terms are summed over the warp with shuffles, and lanes 0..14 flush one 16-byte piece each.  Reads the LT
+// buffer in the layout made for thread ownership (a pair's entries lie 512 bytes apart).
+namespace gart {
+
+template <int MW>
+__device__ __forceinline__ int nth_set_bit(const uint32_t* m, int e) {   // position of the e-th (0-based) set bit of an MW-word mask
+    int base = 0;
+#pragma unroll
+    for (int q = 0; q < MW; ++q) {
+        const int c = __popc(m[q]);
+        if (e < c) return base + (int)__fns(m[q], 0, e + 1);
+        e -= c;
+        base += 32;
+    }
+    return 0;
+}
+
+template <int TS, int DEG>
+__global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ tile_off,
+                                                                     const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
+                                                                     const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ tile_lt_base,
+                                                                     const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
+                                                                     float* __restrict__ gacc, const uint32_t* __restrict__ counts) {
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int AW = (11 + SW + 3) & ~3;
+    __shared__ __align__(16) float4 spix[NT * 2];   // (d, u), (g, v) per pixel, one copy: the lanes of a warp read different pixels
+    if (counts[GART_CNT_ERROR]) return;
+    const int tile = blockIdx.x;
+    const uint32_t begin = tile_off[tile], n = tile_off[tile + 1] - begin;
+    if (n == 0) return;
+    const int x0 = (tile % cam.tiles_x) * TS, y0 = (tile / cam.tiles_x) * TS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int t = threadIdx.x; t < 2 * NT; t += BWD_THREADS) {
+        const int p = t >> 1, h = t & 1;
+        const int x = x0 + p % TS, y = y0 + p / TS;
+        float4 v = make_float4(0.f, 0.f, 0.f, h ? (float)(p / TS) : (float)(p % TS));
+        if (x < cam.width && y < cam.height) {
+            if (h) {
+                const float* gp = dL_dC + ((size_t)y * cam.width + x) * 3;
+                v.x = gp[0]; v.y = gp[1]; v.z = gp[2];
+            } else {
+                const float3 d = pixel_dir(cam, x, y);
+                v.x = d.x; v.y = d.y; v.z = d.z;
+            }
+        }
+        spix[2 * p + h] = v;
+    }
+    __syncthreads();
+    const float4* lt_tile = lt + tile_lt_base[tile];
+    for (uint32_t r = warp; r < n; r += BWD_WARPS) {
+        const uint32_t q = begin + r;
+        uint32_t m[MW];
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) { m[i] = __ldg(rank_mask + (size_t)q * MW + i); c += __popc(m[i]); }
+        if (c == 0) break;   // ranks descend in hit count
+        const uint32_t sid = __ldg(rank_sid + q);
+        const float4* rp = rec + (size_t)sid * RS4;
+        const PairGeo P = pair_geo(unpack_pre(__ldg(rp), __ldg(rp + 1), __ldg(rp + 2), __ldg(rp + 3), __ldg(rp + 4)), x0, y0);
+        const float4* lp = lt_tile + __ldg(rank_gstart + q) + (r & 31u);
+        float acc[AW];
+#pragma unroll
+        for (int i = 0; i < AW; ++i) acc[i] = 0.0f;
+        for (int e = lane; e < c; e += 32) {
+            const int p = nth_set_bit<MW>(m, e);
+            const float4 L = __ldg(lp + (size_t)32 * e);
+            const float4 pa = spix[2 * p], pb = spix[2 * p + 1];
+            const float u = pa.w, v = pb.w;
+            const float3 dg = make_float3(fmaf(P.c0.x, u, fmaf(P.c1.x, v, P.dgA.x)), fmaf(P.c0.y, u, fmaf(P.c1.y, v, P.dgA.y)),
+                                          fmaf(P.c0.z, u, fmaf(P.c1.z, v, P.dgA.z)));
+            const float3 cr = make_float3(fmaf(P.a1.x, u, fmaf(P.b1.x, v, P.crA.x)), fmaf(P.a1.y, u, fmaf(P.b1.y, v, P.crA.y)),
+                                          fmaf(P.a1.z, u, fmaf(P.b1.z, v, P.crA.z)));
+            const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
+            float Y[K], w[3];
+            sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
+            const float3 g = make_float3(pb.x, pb.y, pb.z);
+            lt_weights(L, g, w);
+            const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));
+            const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
+            const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+            acc[0] = fmaf(s1, yx, acc[0]); acc[1] = fmaf(s1, yy, acc[1]); acc[2] = fmaf(s1, yz, acc[2]);
+            acc[3] = fmaf(s2 * yx, yx, acc[3]); acc[4] = fmaf(s2 * yy, yy, acc[4]); acc[5] = fmaf(s2 * yz, yz, acc[5]);
+            acc[6] = fmaf(s2 * yx, yy, acc[6]); acc[7] = fmaf(s2 * yx, yz, acc[7]); acc[8] = fmaf(s2 * yy, yz, acc[8]);
+            acc[9] += ad;
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                acc[11 + 3 * k] = fmaf(sh_norm(k) * Y[k], w[0], acc[11 + 3 * k]);
+                acc[11 + 3 * k + 1] = fmaf(sh_norm(k) * Y[k], w[1], acc[11 + 3 * k + 1]);
+                acc[11 + 3 * k + 2] = fmaf(sh_norm(k) * Y[k], w[2], acc[11 + 3 * k + 2]);
+            }
+        }
+        // sum over the warp; lane i ends up with piece i (words 4 i .. 4 i + 3)
+        float4 mine = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < AW; ++i) {
+            float v = acc[i];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == i / 4) {
+                if (i % 4 == 0) mine.x = v;
+                else if (i % 4 == 1) mine.y = v;
+                else if (i % 4 == 2) mine.z = v;
+                else mine.w = v;
+            }
+        }
+        if (lane < AW / 4) atomicAdd(reinterpret_cast<float4*>(gacc + (size_t)sid * GART_GRAD_WORDS) + lane, mine);
+    }
+}
+
+}  // namespace gart
+
+extern "C" gart_status gart_backward_warp(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
+                                          const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                                          const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
+                                          const float* lt, const float* dL_dcolor,
+                                          float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace gart;
+    if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
+    if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
+    if (g->n == 0) return GART_OK;
+    if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
+    if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    float* gacc = reinterpret_cast<float*>(workspace);
+    gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
+    if (s != GART_OK) return s;
+    const CamF cf = make_camf(cam, cfg->tile_size);
+    const int T = cf.tiles_x * cf.tiles_y;
+    const float4* rec = reinterpret_cast<const float4*>(pre);
+    const float4* lt4 = reinterpret_cast<const float4*>(lt);
+#define GART_WARP(TS, D) bwd_pairs_warp_kernel<TS, D><<<T, BWD_THREADS, 0, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts)
+    if (cfg->tile_size == 8) {
+        switch (g->sh_degree) { case 0: GART_WARP(8, 0); break; case 1: GART_WARP(8, 1); break; case 2: GART_WARP(8, 2); break; default: GART_WARP(8, 3); break; }
+    } else {
+        switch (g->sh_degree) { case 0: GART_WARP(16, 0); break; case 1: GART_WARP(16, 1); break; case 2: GART_WARP(16, 2); break; default: GART_WARP(16, 3); break; }
+    }
+#undef GART_WARP
+    GART_LAUNCH_CHECK();
+    const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);
+    return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);
+}

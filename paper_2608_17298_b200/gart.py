@@ -28,7 +28,7 @@ GRAD_WORDS = 64
 EXPORTS = [
     "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
     "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_forward_workspace_bytes", "gart_forward",
-    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_read_counts",
+    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp", "gart_read_counts",
     "gart_view_host_arena_bytes", "gart_view_host",
 ]
 
@@ -88,11 +88,12 @@ def lib():
         L.gart_backward.argtypes = [vp] * 16 + [sz, vp]
         L.gart_backward_atomic.argtypes = [vp] * 13
         L.gart_backward_hybrid.argtypes = [vp] * 18 + [sz, vp]
+        L.gart_backward_warp.argtypes = [vp] * 16 + [sz, vp]
         L.gart_read_counts.argtypes = [vp, vp, vp]
         L.gart_view_host_arena_bytes.restype = sz
         L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
         L.gart_view_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
-        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid",
+        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp",
                    "gart_read_counts", "gart_view_host"):
             getattr(L, fn).restype = C.c_int
         _lib = L
@@ -284,6 +285,20 @@ def gart_backward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot,
                                _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward")
 
 
+def gart_backward_warp(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
+                       rank_gstart, tile_lt_base, lt, dL_dcolor, grad, counts, workspace, stream=None):
+    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
+    i32, f32 = torch.int32, torch.float32
+    wp, wb = _ws(workspace)
+    _check(lib().gart_backward_warp(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                                    _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
+                                    _dev(tile_off, i32, "tile_off"),
+                                    _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
+                                    _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
+                                    _dev(lt, f32, "lt"), _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
+                                    _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward_warp")
+
+
 def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, ray_off, ray_gid, ray_slot, lt, dL_dcolor,
                          grad, counts, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
@@ -396,6 +411,12 @@ def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None, ray_lists=True):
 def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
     gart_backward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
                   buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
+
+
+def run_backward_warp(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
+    gart_backward_warp(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask,
+                       buf.rank_gstart, buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts,
+                       buf.workspace, stream)
 
 
 def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):

@@ -71,6 +71,10 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         G.run_backward_atomic(cfg, g, cam, buf, dl, ga)
         torch.cuda.synchronize()
         out["grad_atomic"] = to_np(ga)[:g.n]
+        gw = torch.empty_like(buf.grad)
+        G.run_backward_warp(cfg, g, cam, buf, dl, gw)          # ownership ablation: a warp per pair
+        torch.cuda.synchronize()
+        out["grad_warp"] = to_np(gw)[:g.n]
         # hybrid backward: the forward again with 4-byte LT entries (same buffers, everything else unchanged)
         import dataclasses
         cfg_h = dataclasses.replace(cfg, lt_format=1)
