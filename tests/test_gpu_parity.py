@@ -1,10 +1,11 @@
 """GPU parity: the CUDA path (through the C ABI) against the float64 oracle, element by element.
 
-Tolerances (written here, derived in the design doc):
+Tolerances (each fp32 term carries a relative error of a few 1e-6, so a sum is off by about 1e-5 of the mass of its
+terms whatever the summation order):
   * rectangles, classes, tile offsets, pair lists, per-ray hit counts and ordered hit lists:
     bit-exact, up to the guard-band protocol of tests/parity.py;
   * colour: |gpu - ref| <= 1e-4 |ref| + 1e-7; final transmittance: 1e-4 |ref| + 1e-6;
-  * gradients (all 11+3K words, both backward variants): |gpu - ref| <= 1e-3 max(|ref|, COND * A)
+  * gradients (all 11+3K words, every backward variant): |gpu - ref| <= 1e-3 max(|ref|, COND * A)
     or <= 1e-6, where A is the sum of the absolute values of the per-hit terms of that word (its
     conditioning).  A sum whose terms cancel to less than COND = 2% of their mass cannot reach a
     relative 1e-3 in fp32 in any summation order, so the relative bar is measured against that floor.
