@@ -110,14 +110,22 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / HYB_STAGES) & 1u))) { fail(); return; }
             const float* sl = &stage[warp][s][lane];
             const int e_end = min(cur.c, (k + 1) * HYB_CHUNK);
-            for (int e = k * HYB_CHUNK; e < e_end; ++e, sl += 32) {
-                const int p = cur.pm.next();
+            auto hit = [&](const int p, const float wv) {
                 const float4 pa = spix_lane[PixLayout<TS>::index(p, 0, 0)], pb = spix_lane[PixLayout<TS>::index(p, 1, 0)];
                 float Y[K], w[3];
                 sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
-                lt_weights(make_float4(0.f, 0.f, 0.f, *sl), make_float3(pb.x, pb.y, pb.z), w);
+                lt_weights(make_float4(0.f, 0.f, 0.f, wv), make_float3(pb.x, pb.y, pb.z), w);
                 R.accumulate(Y, w);
+            };
+            int e = k * HYB_CHUNK;
+            for (; e + 1 < e_end; e += 2, sl += 64) {   // two hits per iteration: independent chains to interleave
+                const int p0 = cur.pm.next();
+                const int p1 = cur.pm.next();
+                const float w0 = sl[0], w1 = sl[32];
+                hit(p0, w0);
+                hit(p1, w1);
             }
+            if (e < e_end) hit(cur.pm.next(), sl[0]);
             fence_proxy_async();
             __syncwarp();
             ++unit;
