@@ -42,24 +42,46 @@ __global__ void pairs_total_kernel(const uint64_t* total64, int64_t cap_pairs, u
     }
 }
 
-// One thread per pair slot: find the owning Gaussian by bisection of the emission offsets.
+// One thread per Gaussian writes its pairs (row-major over the tiles of its rectangle) from its emission offset.
+// Rectangles of more than EMIT_SERIAL tiles (large or near Gaussians; a straddler covers every tile) are written
+// by the whole warp, one such lane at a time.
+constexpr int EMIT_SERIAL = 16;
 __global__ void __launch_bounds__(256) emit_pairs_kernel(const int4* __restrict__ rect, const uint32_t* __restrict__ emit_off,
                                                          int64_t n, int ts, int tiles_x, const uint32_t* __restrict__ counts,
                                                          uint32_t* __restrict__ keys, uint32_t* __restrict__ vals) {
     if (counts[GART_CNT_ERROR]) return;
-    const uint32_t P = counts[GART_CNT_PAIRS];
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= P) return;
-    int64_t lo = 0, hi = n;  // emit_off[lo] <= p < emit_off[hi]
-    while (hi - lo > 1) {
-        const int64_t mid = (lo + hi) >> 1;
-        if (emit_off[mid] <= (uint32_t)p) lo = mid; else hi = mid;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    int tx0 = 0, ty0 = 0, ntx = 0, cnt = 0;
+    uint32_t off = 0;
+    if (i < n) {
+        const int4 r = rect[i];
+        if (r.z >= r.x && r.w >= r.y) {
+            tx0 = r.x / ts; ty0 = r.y / ts;
+            ntx = r.z / ts - tx0 + 1;
+            cnt = ntx * (r.w / ts - ty0 + 1);
+            off = emit_off[i];
+        }
     }
-    const int4 r = rect[lo];
-    const int tx0 = r.x / ts, ntx = r.z / ts - tx0 + 1, ty0 = r.y / ts;
-    const int local = (int)((uint32_t)p - emit_off[lo]);
-    keys[p] = (uint32_t)((ty0 + local / ntx) * tiles_x + tx0 + local % ntx);
-    vals[p] = (uint32_t)lo;
+    if (cnt <= EMIT_SERIAL) {
+        for (int l = 0; l < cnt; ++l) {
+            keys[off + l] = (uint32_t)((ty0 + l / ntx) * tiles_x + tx0 + l % ntx);
+            vals[off + l] = (uint32_t)i;
+        }
+    }
+    unsigned big = __ballot_sync(0xffffffffu, cnt > EMIT_SERIAL);
+    while (big) {
+        const int src = __ffs((int)big) - 1;
+        big &= big - 1u;
+        const int c = __shfl_sync(0xffffffffu, cnt, src), w = __shfl_sync(0xffffffffu, ntx, src);
+        const int bx = __shfl_sync(0xffffffffu, tx0, src), by = __shfl_sync(0xffffffffu, ty0, src);
+        const uint32_t o = __shfl_sync(0xffffffffu, off, src);
+        const uint32_t id = (uint32_t)(i - lane + src);
+        for (int l = lane; l < c; l += 32) {
+            keys[o + l] = (uint32_t)((by + l / w) * tiles_x + bx + l % w);
+            vals[o + l] = id;
+        }
+    }
 }
 
 // tile_off[t] = first sorted position whose tile id is >= t; tile_off[T] = P.
@@ -144,7 +166,7 @@ extern "C" gart_status gart_tile_map(const gart_config* cfg, const int32_t* rect
     uint32_t* const kbuf[2] = {w.keys0, w.keys1};
     const int cur = radix_passes(bits) & 1;   // emission target: after the passes the result is at index 0
     const int64_t pair_blocks = ceil_div(cap_pairs, 256);
-    emit_pairs_kernel<<<(unsigned)pair_blocks, 256, 0, st>>>(rect4, w.emit_off, n, ts, tiles_x, counts, kbuf[cur], vbuf[cur]);
+    emit_pairs_kernel<<<(unsigned)ceil_div(n > 0 ? n : 1, 256), 256, 0, st>>>(rect4, w.emit_off, n, ts, tiles_x, counts, kbuf[cur], vbuf[cur]);
     GART_LAUNCH_CHECK();
     s = radix_sort_pairs(kbuf, vbuf, cur, bits, cap_pairs, counts + GART_CNT_PAIRS, 0u, counts + GART_CNT_ERROR, w.table, w.scan_ws,
                          w.total64, st);
