@@ -27,7 +27,7 @@ __device__ __forceinline__ void quat_to_rot(const double w, const double x, cons
     R[6] = 2.0 * (x * z - w * y); R[7] = 2.0 * (y * z + w * x); R[8] = 1.0 - 2.0 * (x * x + y * y);
 }
 
-__global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
+__global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
                                                      const float* __restrict__ quat, const float* __restrict__ opacity,
                                                      CamD cam, double alpha_min, double near_z,
                                                      int ts, int tiles_x, uint32_t key_none,
@@ -155,42 +155,49 @@ __global__ void __launch_bounds__(128) bounds_kernel(int64_t n, const float* __r
 __constant__ float c_sh_norm[16] = {sh_norm(0), sh_norm(1), sh_norm(2), sh_norm(3), sh_norm(4), sh_norm(5), sh_norm(6), sh_norm(7),
                                     sh_norm(8), sh_norm(9), sh_norm(10), sh_norm(11), sh_norm(12), sh_norm(13), sh_norm(14), sh_norm(15)};
 
-__global__ void __launch_bounds__(256) gather_records_kernel(int64_t n, int rs4, int sw, uint32_t key_none,
+template <int DEG>
+__global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
                                                              const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
                                                              float4* __restrict__ rec, float4* __restrict__ qs,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
+    constexpr uint32_t SW = 3 * (DEG + 1) * (DEG + 1), RS4 = (20 + SW + 3) / 4;   // (compile-time: the divisions below are multiplications)
     __shared__ float s_norm[16];   // lanes index it divergently: shared memory, not the constant bank
     if (threadIdx.x < 16) s_norm[threadIdx.x] = c_sh_norm[threadIdx.x];
     __syncthreads();
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t slot = t / rs4;
-    const int q = (int)(t - slot * rs4);
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t slot = t / RS4;
+    const uint32_t q = t - slot * RS4;
     if (slot >= n) return;
     const uint32_t gid = vals_sorted[slot];
     const bool vis = keys_sorted[slot] != key_none;
     if (q == 0) {
-        slot_of_gid[gid] = vis ? (uint32_t)slot : 0xffffffffu;
+        slot_of_gid[gid] = vis ? slot : 0xffffffffu;
         gid_of_slot[slot] = vis ? gid : 0xffffffffu;
     }
     if (!vis) return;
     if (q == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
-        qs[2 * slot] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 5];
-        qs[2 * slot + 1] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 6];
+        qs[2 * (size_t)slot] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 5];
+        qs[2 * (size_t)slot + 1] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 6];
     }
     float4 v;
     if (q < 5) {
         v = pre_tmp[(size_t)gid * PRE_TMP_F4 + q];
     } else {
-        const int e = (q - 5) * 4;
-        const float* sp = sh + (size_t)gid * sw;
+        const uint32_t e = (q - 5) * 4;
+        const float* sp = sh + (size_t)gid * SW;
         // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
-        v.x = e < sw ? s_norm[e / 3] * sp[e] : 0.0f;
-        v.y = e + 1 < sw ? s_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
-        v.z = e + 2 < sw ? s_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
-        v.w = e + 3 < sw ? s_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
+        if (SW % 4 == 0) {
+            const float4 c = __ldg(reinterpret_cast<const float4*>(sp + e));
+            v = make_float4(s_norm[e / 3] * c.x, s_norm[(e + 1) / 3] * c.y, s_norm[(e + 2) / 3] * c.z, s_norm[(e + 3) / 3] * c.w);
+        } else {
+            v.x = e < SW ? s_norm[e / 3] * sp[e] : 0.0f;
+            v.y = e + 1 < SW ? s_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
+            v.z = e + 2 < SW ? s_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
+            v.w = e + 3 < SW ? s_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
+        }
     }
-    rec[(size_t)slot * rs4 + q] = v;
+    rec[(size_t)slot * RS4 + q] = v;
 }
 
 struct BoundsWs {
@@ -274,13 +281,20 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     GART_LAUNCH_CHECK();
     gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);
     if (s != GART_OK) return s;
-    const int K = (g->sh_degree + 1) * (g->sh_degree + 1);
     const int rs4 = rec_f4(g->sh_degree);
     const int64_t gthreads = g->n * rs4;
-    gather_records_kernel<<<(unsigned)ceil_div(gthreads, 256), 256, 0, st>>>(g->n, rs4, 3 * K, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh,
-                                                                            reinterpret_cast<float4*>(pre),
-                                                                            reinterpret_cast<float4*>(pre) + (size_t)g->n * rs4, slot_of_gid,
-                                                                            gid_of_slot);
+    if (gthreads >= (int64_t)1 << 32) return GART_ERR_INVALID_ARG;   // (n beyond 1e8 at SH degree 3: 32-bit thread indices)
+    float4* rec_out = reinterpret_cast<float4*>(pre);
+#define GART_GATHER(D)                                                                                                                        \
+    gather_records_kernel<D><<<(unsigned)ceil_div(gthreads, 256), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh, \
+                                                                                rec_out, rec_out + (size_t)g->n * rs4, slot_of_gid, gid_of_slot)
+    switch (g->sh_degree) {
+        case 0: GART_GATHER(0); break;
+        case 1: GART_GATHER(1); break;
+        case 2: GART_GATHER(2); break;
+        default: GART_GATHER(3); break;
+    }
+#undef GART_GATHER
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
