@@ -83,8 +83,8 @@ template <int TS>
 __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
                                                                    const uint32_t* __restrict__ tile_off,
                                                                    const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
-                                                                   uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ hit_count,
-                                                                   uint32_t* __restrict__ counts) {
+                                                                   uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ pair_sid,
+                                                                   uint32_t* __restrict__ hit_count, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, RPW = 32 / TS;   // rows per mask word
     __shared__ uint32_t scnt[NT];
     if (counts[GART_CNT_ERROR]) return;
@@ -103,7 +103,12 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
     // the chain pair -> Gaussian -> slot -> record is three dependent loads: slot ids run two iterations ahead,
     // records one
     constexpr uint32_t STEP = MASK_WARPS * 32;
-    auto load_sid = [&](uint32_t jj) { return jj < end ? __ldg(slot_of_gid + __ldg(pair_gid + jj)) : 0u; };
+    auto load_sid = [&](uint32_t jj) {   // (each pair once: the slot id is also left for the tile sort, in pair order)
+        if (jj >= end) return 0u;
+        const uint32_t sid = __ldg(slot_of_gid + __ldg(pair_gid + jj));
+        pair_sid[jj] = sid;
+        return sid;
+    };
     const uint32_t jfirst = begin + threadIdx.x;
     uint32_t sid_nx = load_sid(jfirst + STEP);
     float4 ra[5];
@@ -200,8 +205,7 @@ __device__ __forceinline__ uint32_t mask_popc(const uint32_t* __restrict__ pair_
 }
 
 template <int TS>
-__global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_gid,
-                                                                    const uint32_t* __restrict__ slot_of_gid,
+__global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_sid,
                                                                     const uint32_t* __restrict__ pair_mask, int T, uint32_t* pair_order,
                                                                     uint32_t* __restrict__ rank_sid, uint32_t* __restrict__ rank_mask,
                                                                     uint32_t* __restrict__ rank_gstart,
@@ -264,7 +268,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
             const bool act = j[u] != 0xffffffffu;
 #pragma unroll
             for (int m = 0; m < MW; ++m) wv[u][m] = act ? __ldg(pair_mask + (size_t)j[u] * MW + m) : 0u;
-            sid[u] = act ? __ldg(slot_of_gid + __ldg(pair_gid + j[u])) : 0u;
+            sid[u] = act ? __ldg(pair_sid + j[u]) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < TSU; ++u) {
@@ -815,12 +819,13 @@ struct ForwardWs {
     uint64_t *total_slots, *total_hits;
     void* scan_ws;
     uint32_t* tile_slots;
+    uint32_t* pair_sid;     // slot of every pair's Gaussian, in pair order (written by fwd_mask, read by tile_sort)
     float4* recs;
     uint64_t* long_keys;
     size_t bytes;
 };
 
-static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_hits) {
+static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_pairs, int64_t cap_hits) {
     ForwardWs w;
     char* p = (char*)base;
     size_t off = 0;
@@ -830,6 +835,7 @@ static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_h
     w.total_hits = (uint64_t*)take(256);
     w.scan_ws = take(scan_workspace_bytes(n_rays > T ? n_rays : T));
     w.tile_slots = (uint32_t*)take((size_t)(T + 1) * 4);
+    w.pair_sid = (uint32_t*)take((size_t)(cap_pairs > 0 ? cap_pairs : 1) * 4);
     w.recs = (float4*)take((size_t)ch * 32);
     w.long_keys = (uint64_t*)take((size_t)ch * 8);
     w.bytes = off;
@@ -863,10 +869,9 @@ static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* re
 }  // namespace gart
 
 extern "C" size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits) {
-    (void)cap_pairs;
     if (tile_size != 8 && tile_size != 16) return 0;
     const int T = ((width + tile_size - 1) / tile_size) * ((height + tile_size - 1) / tile_size);
-    return gart::forward_layout(nullptr, (int64_t)width * height, T, cap_hits).bytes;
+    return gart::forward_layout(nullptr, (int64_t)width * height, T, cap_pairs, cap_hits).bytes;
 }
 
 extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
@@ -891,19 +896,19 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const CamF cf = make_camf(cam, ts);
     const int T = cf.tiles_x * cf.tiles_y;
     const int64_t n_rays = (int64_t)cam->width * cam->height;
-    ForwardWs w = forward_layout(workspace, n_rays, T, cap_hits);
+    ForwardWs w = forward_layout(workspace, n_rays, T, cap_pairs, cap_hits);
     if (w.bytes > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const int rs4 = rec_f4(g->sh_degree);
 
-    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, hit_count, counts);
+    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, w.pair_sid, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, w.pair_sid, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
-    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, slot_of_gid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
-    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, pair_gid, slot_of_gid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
+    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
+    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
     GART_LAUNCH_CHECK();
 
     TileSlotsF tf{w.tile_slots};
