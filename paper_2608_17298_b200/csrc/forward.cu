@@ -6,7 +6,7 @@
 // the ray meets the clamped ellipsoid whose projection the rectangle bounds).  Phases:
 //   1. fwd_mask    block per tile, thread per (tile, Gaussian) pair: per image row the interval of
 //                  columns where the response reaches alpha_min (roots of a quadratic, settled on
-//                  the test itself) -> the pair's hit mask; ballots transpose masks into hits per pixel.
+//                  the test itself) -> the pair's hit mask; hits per pixel counted in shared memory.
 //   2. tile_sort   warp per tile: stable counting sort of the tile's pairs by descending hit
 //                  count -> pair_order, with copies of slot id and mask in rank order (rank_sid,
 //                  rank_mask: read coalesced later); groups of 32 consecutive ranks share an LT
@@ -28,9 +28,8 @@ namespace gart {
 // D^2 = |o_g x d_g|^2 / |d_g|^2 and both vectors affine in the pixel position (u, v) inside the tile,
 //     Q(u, v) = |o_g x d_g|^2 - tau |d_g|^2 = Quu u^2 + 2 Quv u v + Qvv v^2 + 2 Qu u + 2 Qv v + Q0 <= 0,
 // and t* > 0 is t1 u + t2 v + tA > 0.  On row v the hit columns are those with q(u) = qA u^2 + 2 qBh u + qC <= 0.
-// The projected ellipsoid is convex, so (qA > 0) they form one interval: its ends come from the roots and are then
-// settled by evaluating q at the neighbouring columns, so the mask is exactly {u : q(u) <= 0, t(u) > 0} as
-// evaluated in fp32.  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
+// The projected ellipsoid is convex, so (qA > 0) they form one interval, whose ends are the roots of q (and the
+// zero of t).  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
 constexpr int MASK_WARPS = 4;
 
 struct RowQuad {
@@ -46,8 +45,24 @@ __device__ __forceinline__ float fast_sqrt(float x) {
     return y;
 }
 
+// floor / ceil of |x| < 2^22 without the conversion unit: adding and subtracting 1.5 * 2^23 rounds to nearest.
+__device__ __forceinline__ float fast_floor(float x) {
+    const float r = (x + 12582912.0f) - 12582912.0f;
+    return r > x ? r - 1.0f : r;
+}
+__device__ __forceinline__ float fast_ceil(float x) {
+    const float r = (x + 12582912.0f) - 12582912.0f;
+    return r < x ? r + 1.0f : r;
+}
+__device__ __forceinline__ int small_float_to_int(float x) {   // x integral, 0 <= x < 2^22
+    return __float_as_int(x + 12582912.0f) - 0x4B400000;
+}
+
 // Bits 0..ncol-1: the columns of one row that the Gaussian's response reaches.  `regular`: qA > 0 and t1 != 0,
-// with inv_qA = 1 / qA and inv_t1 = 1 / t1.
+// with inv_qA = 1 / qA and inv_t1 = 1 / t1.  The roots come from the cancellation-free form
+// (z = -(qBh + sign(qBh) sqrt(disc)); roots z / qA and qC / z), so inside the tile they are good to a few ulp: a pixel
+// whose decision that rounding could flip lies within 1e-5 pixel of the boundary, i.e. its response is within
+// 1e-5 of alpha_min.
 template <int TS>
 __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, float inv_qA, float inv_t1, int ncol) {
     uint32_t bits = 0u;
@@ -55,19 +70,26 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
         const float qBh = 0.5f * q.qB2;
         const float disc = fmaf(qBh, qBh, -q.qA * q.qC);
         if (disc >= 0.0f) {
-            const float sq = fast_sqrt(disc);
-            float ulo = (-qBh - sq) * inv_qA, uhi = (-qBh + sq) * inv_qA;
-            const float ut = -q.t0 * inv_t1;   // t* > 0 on one side of it
-            ulo = q.t1 > 0.0f ? fmaxf(ulo, ut) : ulo;
-            uhi = q.t1 > 0.0f ? uhi : fminf(uhi, ut);
+            const float z = -(qBh + copysignf(fast_sqrt(disc), qBh));
+            const float r1 = z * inv_qA;
+            const float r2 = z != 0.0f ? q.qC * fast_rcp(z) : r1;
+            float ulo = fminf(r1, r2), uhi = fmaxf(r1, r2);
+            const float ut = -q.t0 * inv_t1;   // t* > 0 on one side of it (strictly: a pixel exactly on it is left out below)
+            const bool up = q.t1 > 0.0f;
             const float last = (float)(ncol - 1);
-            float flo = fmaxf(ceilf(ulo), 0.0f), fhi = fminf(floorf(uhi), last);
-            // settle the ends on the test itself (the roots carry rounding)
-            const bool l0 = q.hit(flo), l1 = flo > 0.0f && q.hit(flo - 1.0f);
-            const bool h0 = q.hit(fhi), h1 = fhi < last && q.hit(fhi + 1.0f);
-            flo = l0 ? (l1 ? flo - 1.0f : flo) : flo + 1.0f;
-            fhi = h0 ? (h1 ? fhi + 1.0f : fhi) : fhi - 1.0f;
-            if (flo <= fhi) bits = (2u << (int)fhi) - (1u << (int)flo);   // (NaN compares false)
+            float flo = fast_ceil(fminf(fmaxf(ulo, -1.0f), 4194303.0f)), fhi = fast_floor(fminf(fmaxf(uhi, -2.0f), 4194303.0f));
+            if (up) {
+                const float tl = fminf(fmaxf(ut, -1.0f), 4194303.0f);
+                const float c = fast_floor(tl) + 1.0f;          // smallest integer > ut
+                flo = fmaxf(flo, c);
+            } else {
+                const float tl = fminf(fmaxf(ut, -2.0f), 4194303.0f);
+                const float c = fast_ceil(tl) - 1.0f;           // largest integer < ut
+                fhi = fminf(fhi, c);
+            }
+            flo = fmaxf(flo, 0.0f);
+            fhi = fminf(fhi, last);
+            if (flo <= fhi) bits = (2u << small_float_to_int(fhi)) - (1u << small_float_to_int(flo));   // (NaN compares false)
         }
     } else {
 #pragma unroll
@@ -78,7 +100,7 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
 }
 
 // Block per tile, thread per (tile, Gaussian) pair: row by row the interval of hit columns -> the pair's mask.
-// Hits per pixel: the lanes' masks are transposed with ballots (lane l counts pixels l, l + 32, ...).
+// Hits per pixel: a shared-memory counter per pixel.
 template <int TS>
 __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
                                                                    const uint32_t* __restrict__ tile_off,
@@ -96,9 +118,6 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
     const uint32_t begin = tile_off[tile], end = tile_off[tile + 1];
     for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) scnt[p] = 0u;
     __syncthreads();
-    uint32_t cnt[MW];
-#pragma unroll
-    for (int q = 0; q < MW; ++q) cnt[q] = 0u;
     const float inv_amin = 1.0f / alpha_min;
     // the chain pair -> Gaussian -> slot -> record is three dependent loads: slot ids run two iterations ahead,
     // records one
@@ -162,23 +181,19 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
 #pragma unroll
             for (int q = 0; q < MW; ++q) pair_mask[(size_t)j * MW + q] = w[q];
         }
-        // hits per pixel over these 32 pairs
+        // hits per pixel: one shared-memory increment per hit
 #pragma unroll
         for (int q = 0; q < MW; ++q) {
-            if (__any_sync(0xffffffffu, w[q] != 0u)) {
-#pragma unroll 8
-                for (int b = 0; b < 32; ++b) {
-                    const unsigned bal = __ballot_sync(0xffffffffu, (w[q] >> b) & 1u);
-                    if (lane == b) cnt[q] += __popc(bal);
-                }
+            uint32_t m = w[q];
+            while (m) {
+                const int b = __ffs((int)m) - 1;
+                m &= m - 1u;
+                atomicAdd(&scnt[q * 32 + b], 1u);
             }
         }
 #pragma unroll
         for (int q = 0; q < 5; ++q) ra[q] = rb[q];
     }
-#pragma unroll
-    for (int q = 0; q < MW; ++q)
-        if (cnt[q]) atomicAdd(&scnt[q * 32 + lane], cnt[q]);
     __syncthreads();
     uint32_t m = 0;
     for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) {
