@@ -69,28 +69,21 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
     if (regular) {
         const float qBh = 0.5f * q.qB2;
         const float disc = fmaf(qBh, qBh, -q.qA * q.qC);
-        if (disc >= 0.0f) {
-            const float z = -(qBh + copysignf(fast_sqrt(disc), qBh));
-            const float r1 = z * inv_qA;
-            const float r2 = z != 0.0f ? q.qC * fast_rcp(z) : r1;
-            float ulo = fminf(r1, r2), uhi = fmaxf(r1, r2);
-            const float ut = -q.t0 * inv_t1;   // t* > 0 on one side of it (strictly: a pixel exactly on it is left out below)
-            const bool up = q.t1 > 0.0f;
-            const float last = (float)(ncol - 1);
-            float flo = fast_ceil(fminf(fmaxf(ulo, -1.0f), 4194303.0f)), fhi = fast_floor(fminf(fmaxf(uhi, -2.0f), 4194303.0f));
-            if (up) {
-                const float tl = fminf(fmaxf(ut, -1.0f), 4194303.0f);
-                const float c = fast_floor(tl) + 1.0f;          // smallest integer > ut
-                flo = fmaxf(flo, c);
-            } else {
-                const float tl = fminf(fmaxf(ut, -2.0f), 4194303.0f);
-                const float c = fast_ceil(tl) - 1.0f;           // largest integer < ut
-                fhi = fminf(fhi, c);
-            }
-            flo = fmaxf(flo, 0.0f);
-            fhi = fminf(fhi, last);
-            if (flo <= fhi) bits = (2u << small_float_to_int(fhi)) - (1u << small_float_to_int(flo));   // (NaN compares false)
-        }
+        // no branch on the sign of disc: the lanes of a warp stay together, the result is masked at the end
+        const float z = -(qBh + copysignf(fast_sqrt(fmaxf(disc, 0.0f)), qBh));
+        const float r1 = z * inv_qA;
+        const float r2 = z != 0.0f ? q.qC * fast_rcp(z) : r1;
+        const float ulo = fminf(r1, r2), uhi = fmaxf(r1, r2);
+        const float ut = fminf(fmaxf(-q.t0 * inv_t1, -2.0f), 4194303.0f);   // t* > 0 on one side of it, strictly
+        const bool up = q.t1 > 0.0f;
+        float flo = fast_ceil(fminf(fmaxf(ulo, -1.0f), 4194303.0f)), fhi = fast_floor(fminf(fmaxf(uhi, -2.0f), 4194303.0f));
+        flo = up ? fmaxf(flo, fast_floor(ut) + 1.0f) : flo;     // smallest integer > ut
+        fhi = up ? fhi : fminf(fhi, fast_ceil(ut) - 1.0f);      // largest integer < ut
+        flo = fmaxf(flo, 0.0f);
+        fhi = fminf(fhi, (float)(ncol - 1));
+        const bool any = disc >= 0.0f && flo <= fhi;             // (NaN compares false)
+        const uint32_t span = (2u << (small_float_to_int(fhi) & 31)) - (1u << (small_float_to_int(flo) & 31));
+        bits = any ? span : 0u;
     } else {
 #pragma unroll
         for (int c = 0; c < TS; ++c)
