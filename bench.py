@@ -42,14 +42,17 @@ def shard_views(n_views: int, rank: int, world: int):
     return mine if mine else [rank % n_views]
 
 
-def launches_per_step(n_tiles: int) -> int:
-    """Kernel launches of one step (memsets are not kernels)."""
+def _radix_passes(n_keys: int) -> int:
     bits = 1
-    while (1 << bits) < n_tiles:
+    while (1 << bits) <= n_keys:          # keys 0 .. n_keys (the last one marks "none")
         bits += 1
-    passes = (bits + 7) // 8
-    bounds = 1 + 2 * (1 + 3 + 1) + 1          # bounds kernel, two radix passes, record gather
-    tile_map = 1 + 3 + 1 + 1 + passes * (1 + 3 + 1) + 1
+    return (bits + 7) // 8
+
+
+def launches_per_step(tiles_x: int, tiles_y: int) -> int:
+    """Kernel launches of one step (memsets are not kernels).  A radix pass is histogram + three scan kernels + scatter."""
+    bounds = 1 + _radix_passes(tiles_y) * 5 + 1                  # bounds kernel, slot sort on the tile row, record gather
+    tile_map = 1 + 3 + 1 + 1 + _radix_passes(tiles_x * tiles_y - 1) * 5 + 1   # areas, scan, total, emission, pair sort, offsets
     forward = 1 + 1 + 3 + 3 + 1 + 1 + 3          # mask, tile sort, two scans, totals, evaluation, sweep per ray-length class
     backward = 4                                # zero, pair kernel, per-slot conversion, scatter of the SH gradient
     return bounds + tile_map + forward + backward
@@ -424,7 +427,7 @@ def run_ours(args):
         "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
         "backward_hybrid_ms": hybrid_ms,
         "backward_warp_per_pair_ms": warp_ms,
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(G.tiles(cams[0], cfg.tile_size)) * args.steps,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(-(-cams[0].width // cfg.tile_size), -(-cams[0].height // cfg.tile_size)) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
