@@ -567,30 +567,51 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
     __syncwarp();
     sort_regs<R>(k, lane);
     {
-        // neighbours with the same truncated t*: exact order by odd-even exchanges, n rounds at most
-        bool tie = false;
+        // neighbours with the same truncated t* (a padding key never ties: t* is finite): bit r of tm says that positions
+        // r and r + 1 of this lane tie (r + 1 = R: the next lane's first)
+        uint32_t tm = 0u;
 #pragma unroll
-        for (int r = 0; r + 1 < R; ++r) tie = tie || ((k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && lane * R + r + 1 < n);
+        for (int r = 0; r + 1 < R; ++r) tm |= (uint32_t)(((k[r] ^ k[r + 1]) >> KEY_IDX_BITS) == 0u && k[r + 1] != 0xffffffffu) << r;
         const uint32_t nb = __shfl_down_sync(0xffffffffu, k[0], 1);
-        tie = tie || (lane < 31 && (k[R - 1] >> KEY_IDX_BITS) == (nb >> KEY_IDX_BITS) && (lane + 1) * R < n);
-        if (__any_sync(0xffffffffu, tie)) {
-            for (int round = 0; round < n; ++round) {
-                bool moved = false;
+        tm |= (uint32_t)(lane < 31 && ((k[R - 1] ^ nb) >> KEY_IDX_BITS) == 0u && nb != 0xffffffffu) << (R - 1);
+        if (__any_sync(0xffffffffu, tm != 0u)) {
+            // a tie directly after a tie means a run of three or more equal keys
+            const uint32_t tm_next = __shfl_down_sync(0xffffffffu, tm, 1);
+            const bool chain = (tm & (tm << 1)) != 0u || (lane < 31 && ((tm >> (R - 1)) & 1u) && (tm_next & 1u));
+            if (!__any_sync(0xffffffffu, chain)) {
+                // isolated pairs (the usual case): one exact comparison each
 #pragma unroll
                 for (int r = 0; r + 1 < R; ++r) {
-                    if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(s_tg, k[r], k[r + 1])) {
-                        const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
+                    if (((tm >> r) & 1u) && rec_after(s_tg, k[r], k[r + 1])) { const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; }
+                }
+                const bool mine = (tm >> (R - 1)) & 1u;
+                if (__any_sync(0xffffffffu, mine)) {   // pairs across a lane boundary
+                    const bool swap = mine && rec_after(s_tg, k[R - 1], nb);
+                    const uint32_t from_prev = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
+                    const bool prev_swapped = __shfl_up_sync(0xffffffffu, (int)swap, 1) != 0 && lane > 0;
+                    if (swap) k[R - 1] = nb;
+                    if (prev_swapped) k[0] = from_prev;
+                }
+            } else {
+                // general case: odd-even exchanges on the exact values until nothing moves, n rounds at most
+                for (int round = 0; round < n; ++round) {
+                    bool moved = false;
+#pragma unroll
+                    for (int r = 0; r + 1 < R; ++r) {
+                        if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(s_tg, k[r], k[r + 1])) {
+                            const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
+                        }
                     }
+                    // across the lane boundary: even lanes lead on even rounds, odd lanes on odd rounds
+                    const uint32_t up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
+                    const bool lead = ((lane ^ round) & 1) == 0;
+                    if (lead) {
+                        if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(s_tg, k[R - 1], up)) { k[R - 1] = up; moved = true; }
+                    } else {
+                        if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(s_tg, dn, k[0])) { k[0] = dn; moved = true; }
+                    }
+                    if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
                 }
-                // across the lane boundary: even lanes lead on even rounds, odd lanes on odd rounds
-                const uint32_t up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
-                const bool lead = ((lane ^ round) & 1) == 0;
-                if (lead) {
-                    if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(s_tg, k[R - 1], up)) { k[R - 1] = up; moved = true; }
-                } else {
-                    if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(s_tg, dn, k[0])) { k[0] = dn; moved = true; }
-                }
-                if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
             }
         }
     }
