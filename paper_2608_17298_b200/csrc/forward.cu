@@ -806,14 +806,22 @@ struct SweepClass {
 template <int CLS>
 __global__ void __launch_bounds__(SWEEP_WARPS * 32, SweepClass<CLS>::MIN_BLOCKS)
 fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs, uint64_t* __restrict__ long_keys, int64_t n_rays,
+                      int width, int tile_size, int tiles_x,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                       float4* __restrict__ lt, bool w_only, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                       const uint32_t* __restrict__ counts) {
     constexpr int CAP = SweepClass<CLS>::CAP;
     if (counts[GART_CNT_ERROR]) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t r = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
-    if (r >= n_rays) return;
+    // rays in tile-major order: the 64 (256) rays of a tile are taken by neighbouring blocks, so the two halves of an
+    // LT sector (entries of two pairs of the same tile) are written close in time and merge in L2
+    const int64_t lin = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
+    const int nt = tile_size * tile_size;
+    const int64_t tile = lin / nt;
+    const int pix = (int)(lin - tile * nt);
+    const int x = (int)(tile % tiles_x) * tile_size + pix % tile_size, y = (int)(tile / tiles_x) * tile_size + pix / tile_size;
+    if (x >= width || y * (int64_t)width + x >= n_rays) return;
+    const int64_t r = (int64_t)y * width + x;
     const size_t b = ray_off[r];
     const int n = (int)(ray_off[r + 1] - ray_off[r]);
     if (n == 0) {
@@ -953,14 +961,14 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     else s = launch_eval<16>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
     if (s != GART_OK) return s;
 
-    const int64_t blocks = ceil_div(n_rays, SWEEP_WARPS);
+    const int64_t blocks = ceil_div((int64_t)T * ts * ts, SWEEP_WARPS);
     float4* lt4 = reinterpret_cast<float4*>(lt);
     const bool w_only = cfg->lt_format == 1;
     const float* bg = cfg->background;
 #define GART_SWEEP_LAUNCH(C)                                                                                                                    \
     if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess)        \
         return GART_ERR_CUDA;                                                                                                                   \
-    fwd_sort_sweep_kernel<C><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, bg[0], bg[1], \
+    fwd_sort_sweep_kernel<C><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0], bg[1], \
                                                                                              bg[2], color, t_final, lt4, w_only, ray_gid, ray_slot, counts); \
     GART_LAUNCH_CHECK();
     GART_SWEEP_LAUNCH(2)   // the longest rays first
