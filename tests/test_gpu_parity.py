@@ -295,6 +295,20 @@ def test_invalid_arguments_return_status():
     with pytest.raises(G.GartError) as e:
         G.gart_tile_map(G.Config(), buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, 100, buf.counts, buf.workspace[1:])
     assert e.value.status == 1                     # workspace not 256-byte aligned
+    # each backward variant wants its own LT format, and the forward knows two
+    dl = torch.zeros((cam.height, cam.width, 3), dtype=torch.float32, device="cuda")
+    with pytest.raises(G.GartError) as e:
+        G.run_backward(G.Config(lt_format=1), g, cam, buf, dl)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
+        G.run_backward_warp(G.Config(lt_format=1), g, cam, buf, dl)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
+        G.run_backward_hybrid(G.Config(lt_format=0), g, cam, buf, dl)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
+        G.run_forward(G.Config(lt_format=2), g, cam, buf)
+    assert e.value.status == 1
     g.sh_degree = 3
     with pytest.raises(AssertionError):
         g.c()
