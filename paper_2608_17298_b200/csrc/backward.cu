@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                float* __restrict__ gacc, uint32_t* __restrict__ counts) {
+                                                                Gacc gacc, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
     // evaluation record of a lane's Gaussian (the first 5 float4 of the slot's record), staged through shared
@@ -214,7 +214,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         }
         if (cur.c != 0) {
             // one vector atomic per 16 bytes of the Gaussian's record
-            float4* gp = reinterpret_cast<float4*>(gacc + (size_t)cur.sid * GART_GRAD_WORDS);
 #pragma unroll
             for (int q = 0; q < AW / 4; ++q) {
                 float v[4];
@@ -223,7 +222,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                     const int wd = 4 * q + i;
                     v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f);   // constants left out by sh_poly
                 }
-                red_add_f4_hint(gp + q, v[0], v[1], v[2], v[3], pol_keep);
+                red_add_f4_hint(gacc_piece(gacc, cur.sid, q), v[0], v[1], v[2], v[3], pol_keep);
             }
         }
         if (nxt.cmax == 0) break;
@@ -238,7 +237,7 @@ template <int TS, int DEG>
 static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                     const uint32_t* tile_lt_base, const float4* lt,
-                                    const float* dL_dC, const CamF& cam, float* gacc, uint32_t* counts) {
+                                    const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
     auto kern = bwd_pairs_kernel<TS, DEG>;
     constexpr int smem = BWD_DYN_SMEM;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
@@ -251,7 +250,7 @@ template <int TS>
 static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                 const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                 const uint32_t* tile_lt_base, const float4* lt,
-                                const float* dL_dC, const CamF& cam, float* gacc, uint32_t* counts) {
+                                const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
 #define GART_PAIRS(D) \
     return launch_pairs_deg<TS, D>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts)
     switch (deg) {
@@ -265,9 +264,7 @@ static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* r
 
 }  // namespace gart
 
-extern "C" size_t gart_backward_workspace_bytes(int64_t n) {
-    return gart::align256((size_t)(n > 0 ? n : 1) * GART_GRAD_WORDS * sizeof(float));
-}
+extern "C" size_t gart_backward_workspace_bytes(int64_t n) { return gart::gacc_bytes(n > 0 ? n : 1); }
 
 extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                      const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
@@ -284,7 +281,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
-    float* gacc = reinterpret_cast<float*>(workspace);
+    const Gacc gacc = make_gacc(workspace, g->n);
     gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
     if (s != GART_OK) return s;
     const CamF cf = make_camf(cam, cfg->tile_size);
@@ -323,7 +320,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
                                                                      const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
                                                                      const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ tile_lt_base,
                                                                      const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                     float* __restrict__ gacc, const uint32_t* __restrict__ counts) {
+                                                                     Gacc gacc, const uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     constexpr int AW = (11 + SW + 3) & ~3;
     __shared__ __align__(16) float4 spix[NT * 2];   // (d, u), (g, v) per pixel, one copy: the lanes of a warp read different pixels
@@ -406,7 +403,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
                 else mine.w = v;
             }
         }
-        if (lane < AW / 4) atomicAdd(reinterpret_cast<float4*>(gacc + (size_t)sid * GART_GRAD_WORDS) + lane, mine);
+        if (lane < AW / 4) atomicAdd(gacc_piece(gacc, sid, lane), mine);
     }
 }
 
@@ -427,7 +424,7 @@ extern "C" gart_status gart_backward_warp(const gart_config* cfg, const gart_gau
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
-    float* gacc = reinterpret_cast<float*>(workspace);
+    const Gacc gacc = make_gacc(workspace, g->n);
     gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
     if (s != GART_OK) return s;
     const CamF cf = make_camf(cam, cfg->tile_size);

@@ -103,23 +103,50 @@ __device__ __forceinline__ GroupDesc<MW> load_group(const uint32_t* __restrict__
     return d;
 }
 
+// The accumulation record of a slot, as the gradient record's words 0..59 in two pieces: words 0..15 (moments v, Q,
+// sum alpha dL/dalpha, one unused word, the first five dL/dsh words) in one array of 64-byte rows, words 16..59 (the
+// rest of dL/dsh) in another of 176-byte rows.  The conversion then reads compact, coalesced rows, and nothing is
+// moved or zeroed for the record's four padding words.
+constexpr int GACC_A_WORDS = 16, GACC_B_WORDS = 44;
+struct Gacc {
+    float* a;   // [n][GACC_A_WORDS]
+    float* b;   // [n][GACC_B_WORDS]
+};
+static inline size_t gacc_bytes(int64_t n) { return align256((size_t)n * GACC_A_WORDS * 4) + align256((size_t)n * GACC_B_WORDS * 4); }
+static inline Gacc make_gacc(void* workspace, int64_t n) {
+    Gacc g;
+    g.a = reinterpret_cast<float*>(workspace);
+    g.b = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + align256((size_t)n * GACC_A_WORDS * 4));
+    return g;
+}
+// float4 number q (0..14) of slot sid's record
+__device__ __forceinline__ float4* gacc_piece(const Gacc& g, uint32_t sid, int q) {
+    return q < 4 ? reinterpret_cast<float4*>(g.a + (size_t)sid * GACC_A_WORDS) + q
+                 : reinterpret_cast<float4*>(g.b + (size_t)sid * GACC_B_WORDS) + (q - 4);
+}
+
 // Zero the accumulation records of the view's slots (their number lives on the device): grid-stride.
-static __global__ void __launch_bounds__(256) bwd_zero_kernel(float4* __restrict__ gacc4, const uint32_t* __restrict__ counts) {
-    const size_t total = (size_t)counts[GART_CNT_VISIBLE] * (GART_GRAD_WORDS / 4);
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x)
-        gacc4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+static __global__ void __launch_bounds__(256) bwd_zero_kernel(Gacc gacc, const uint32_t* __restrict__ counts) {
+    const size_t V = counts[GART_CNT_VISIBLE];
+    const size_t na = V * (GACC_A_WORDS / 4), total = na + V * (GACC_B_WORDS / 4);
+    float4* a4 = reinterpret_cast<float4*>(gacc.a);
+    float4* b4 = reinterpret_cast<float4*>(gacc.b);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        if (i < na) a4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        else b4[i - na] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
 }
 
 // One thread per slot: convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity and
 // write words 0..15 of the Gaussian's gradient record (all 32 lanes busy with the ~300-instruction conversion).
 static __global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* __restrict__ qs, const uint32_t* __restrict__ gid_of_slot,
-                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          Gacc gacc, float4* __restrict__ grad4,
                                                           const uint32_t* __restrict__ counts) {
     if (counts[GART_CNT_ERROR]) return;
     constexpr int F4 = GART_GRAD_WORDS / 4;
     const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
-    const float4* gp = gacc4 + (size_t)sid * F4;
+    const float4* gp = reinterpret_cast<const float4*>(gacc.a) + (size_t)sid * (GACC_A_WORDS / 4);
     const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
     const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];   // quaternion; scale and opacity
     float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
@@ -139,10 +166,11 @@ static __global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* _
 // FIN_ROWS Gaussians with all their loads in flight at once.
 constexpr int FIN_ROWS = 4;
 static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, const uint32_t* __restrict__ slot_of_gid,
-                                                          const float4* __restrict__ gacc4, float4* __restrict__ grad4,
+                                                          Gacc gacc, float4* __restrict__ grad4,
                                                           const uint32_t* __restrict__ counts) {
     if (counts[GART_CNT_ERROR]) return;
     constexpr int F4 = GART_GRAD_WORDS / 4;
+    const float4* b4 = reinterpret_cast<const float4*>(gacc.b);
     const int64_t hw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // half-warp
     const int l = threadIdx.x & 15;
     const int64_t i0 = hw * FIN_ROWS;
@@ -152,7 +180,7 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
     float4 v[FIN_ROWS];
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r)
-        v[r] = (s[r] != 0xffffffffu && l >= 4) ? __ldcs(gacc4 + (size_t)s[r] * F4 + l) : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[r] = (s[r] != 0xffffffffu && l >= 4 && l < 15) ? __ldcs(b4 + (size_t)s[r] * (GACC_B_WORDS / 4) + (l - 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r)
         if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu)) __stcs(grad4 + (size_t)(i0 + r) * F4 + l, v[r]);
@@ -161,18 +189,18 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
 
 // Launches shared by the backward variants: zero the accumulation records of the view's slots; after the
 // accumulation, convert the moments per slot and write the caller's gradient records.
-static inline gart_status launch_zero_accumulators(float* gacc, int64_t n, const uint32_t* counts, cudaStream_t st) {
-    const int64_t zero_blocks = ceil_div(n * (GART_GRAD_WORDS / 4), 256);
-    bwd_zero_kernel<<<(unsigned)(zero_blocks < 148 * 32 ? zero_blocks : 148 * 32), 256, 0, st>>>(reinterpret_cast<float4*>(gacc), counts);
+static inline gart_status launch_zero_accumulators(const Gacc& gacc, int64_t n, const uint32_t* counts, cudaStream_t st) {
+    const int64_t zero_blocks = ceil_div(n * ((GACC_A_WORDS + GACC_B_WORDS) / 4), 256);
+    bwd_zero_kernel<<<(unsigned)(zero_blocks < 148 * 32 ? zero_blocks : 148 * 32), 256, 0, st>>>(gacc, counts);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
 static inline gart_status launch_finalize(int64_t n, const float4* qs, const uint32_t* slot_of_gid, const uint32_t* gid_of_slot,
-                                          const float* gacc, float* grad, const uint32_t* counts, cudaStream_t st) {
-    bwd_convert_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(qs, gid_of_slot, reinterpret_cast<const float4*>(gacc),
+                                          const Gacc& gacc, float* grad, const uint32_t* counts, cudaStream_t st) {
+    bwd_convert_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(qs, gid_of_slot, gacc,
                                                                    reinterpret_cast<float4*>(grad), counts);
     GART_LAUNCH_CHECK();
-    bwd_scatter_kernel<<<(unsigned)ceil_div(ceil_div(n, FIN_ROWS) * 16, 256), 256, 0, st>>>(n, slot_of_gid, reinterpret_cast<const float4*>(gacc),
+    bwd_scatter_kernel<<<(unsigned)ceil_div(ceil_div(n, FIN_ROWS) * 16, 256), 256, 0, st>>>(n, slot_of_gid, gacc,
                                                                                             reinterpret_cast<float4*>(grad), counts);
     GART_LAUNCH_CHECK();
     return GART_OK;

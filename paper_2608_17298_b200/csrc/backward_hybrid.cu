@@ -27,7 +27,7 @@ template <int TS, int DEG>
 __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                              const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                              const uint32_t* __restrict__ tile_lt_base, const float* __restrict__ lt_w,
-                                                             const float* __restrict__ dL_dC, CamF cam, float* __restrict__ gacc,
+                                                             const float* __restrict__ dL_dC, CamF cam, Gacc gacc,
                                                              uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;
@@ -133,7 +133,6 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
         }
         if (cur.c != 0) {
             // words 11 .. 10 + 3K of the slot's accumulation record (the float4 holding word 11 starts at word 8)
-            float4* gp = reinterpret_cast<float4*>(gacc + (size_t)cur.sid * GART_GRAD_WORDS);
 #pragma unroll
             for (int q = 2; q < AW / 4; ++q) {
                 float v[4];
@@ -142,7 +141,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
                     const int wd = 4 * q + i;
                     v[i] = (wd >= 11 && wd < 11 + SW) ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f;
                 }
-                red_add_f4_hint(gp + q, v[0], v[1], v[2], v[3], pol_keep);
+                red_add_f4_hint(gacc_piece(gacc, cur.sid, q), v[0], v[1], v[2], v[3], pol_keep);
             }
         }
         if (nxt.cmax == 0) break;
@@ -160,7 +159,7 @@ template <int DEG>
 __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ slot_of_gid,
                                                             const uint32_t* __restrict__ ray_off, const uint32_t* __restrict__ ray_gid,
                                                             const float* __restrict__ dL_dC, CamF cam, float bg0, float bg1, float bg2,
-                                                            float* __restrict__ gacc, const uint32_t* __restrict__ counts) {
+                                                            Gacc gacc, const uint32_t* __restrict__ counts) {
     constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -208,7 +207,7 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
         const float G = -0.5f * ad;
         const float3 xg = ray_xg(r);
         const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
-        float* gp = gacc + (size_t)sid * GART_GRAD_WORDS;
+        float* gp = gacc.a + (size_t)sid * GACC_A_WORDS;
         atomicAdd(gp + 0, gx); atomicAdd(gp + 1, gy); atomicAdd(gp + 2, gz);
         atomicAdd(gp + 3, gx * xg.x); atomicAdd(gp + 4, gy * xg.y); atomicAdd(gp + 5, gz * xg.z);
         atomicAdd(gp + 6, gx * xg.y); atomicAdd(gp + 7, gx * xg.z); atomicAdd(gp + 8, gy * xg.z);
@@ -221,7 +220,7 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
 template <int TS>
 static gart_status launch_sh(int deg, int T, cudaStream_t st, const uint32_t* tile_off, const uint32_t* rank_sid, const uint32_t* rank_mask,
                              const uint32_t* rank_gstart, const uint32_t* tile_lt_base, const float* lt_w, const float* dL_dC,
-                             const CamF& cam, float* gacc, uint32_t* counts) {
+                             const CamF& cam, const Gacc& gacc, uint32_t* counts) {
 #define GART_SH(D) bwd_sh_kernel<TS, D><<<T, HYB_THREADS, 0, st>>>(tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dC, cam, gacc, counts)
     switch (deg) {
         case 0: GART_SH(0); break;
@@ -252,7 +251,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
-    float* gacc = reinterpret_cast<float*>(workspace);
+    const Gacc gacc = make_gacc(workspace, g->n);
     gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
     if (s != GART_OK) return s;
     const CamF cf = make_camf(cam, cfg->tile_size);

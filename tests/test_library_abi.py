@@ -27,7 +27,8 @@ def test_every_declared_symbol_is_exported():
 def test_host_only_queries():
     assert G.gart_mask_words(8) == 2 and G.gart_mask_words(16) == 8
     assert [G.gart_pre_words(d) for d in range(4)] == [32, 40, 56, 76]
-    assert G.gart_backward_workspace_bytes(1000) == 256_000 and G.gart_bounds_workspace_bytes(1000) > 80_000
+    # accumulation records: 60 words per Gaussian in two arrays, each rounded up to 256 bytes
+    assert G.gart_backward_workspace_bytes(1000) == 64_000 + 176_128 and G.gart_bounds_workspace_bytes(1000) > 80_000
     assert G.lib().gart_status_string(0) == b"ok" and G.lib().gart_status_string(2) == b"workspace too small"
     a = G.gart_tile_map_workspace_bytes(1000, 640, 480, 8, 10_000)
     b = G.gart_tile_map_workspace_bytes(1000, 640, 480, 8, 20_000)
