@@ -69,8 +69,8 @@ def algorithmic_bytes_backward(H, P, n_vis, n_pixels, K):
 # summarised in profiles/dram_traffic_unbounded6m_crop.md (8x8 tiles, SH degree 3, central crop of a view), each
 # divided by the unit it grows with: the pair kernel by hits, zeroing and conversion by visible Gaussians, the
 # scatter's reads by visible Gaussians and its writes by all Gaussians.
-TRAFFIC_MODEL = {"pairs_per_hit": 45.1, "zero_per_visible": 230.4, "convert_per_visible": 218.6,
-                 "scatter_read_per_visible": 265.8, "scatter_write_per_gaussian": 220.8}
+TRAFFIC_MODEL = {"pairs_per_hit": 46.2, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
+                 "scatter_read_per_visible": 186.0, "scatter_write_per_gaussian": 220.7}
 
 
 def measured_traffic_backward(H, n_vis, n):
