@@ -816,12 +816,16 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     // rays in tile-major order: the 64 (256) rays of a tile are taken by neighbouring blocks, so the two halves of an
     // LT sector (entries of two pairs of the same tile) are written close in time and merge in L2
     const int64_t lin = (int64_t)blockIdx.x * SWEEP_WARPS + warp;
-    const int nt = tile_size * tile_size;
-    const int64_t tile = lin / nt;
-    const int pix = (int)(lin - tile * nt);
-    const int x = (int)(tile % tiles_x) * tile_size + pix % tile_size, y = (int)(tile / tiles_x) * tile_size + pix / tile_size;
-    if (x >= width || y * (int64_t)width + x >= n_rays) return;
-    const int64_t r = (int64_t)y * width + x;
+    int64_t r = lin;
+    if (CLS == 2) {   // (the short rays' launches mostly find blocks with nothing to do: plain order is cheaper there)
+        const int nt = tile_size * tile_size;
+        const int64_t tile = lin / nt;
+        const int pix = (int)(lin - tile * nt);
+        const int x = (int)(tile % tiles_x) * tile_size + pix % tile_size, y = (int)(tile / tiles_x) * tile_size + pix / tile_size;
+        if (x >= width) return;
+        r = (int64_t)y * width + x;
+    }
+    if (r >= n_rays) return;
     const size_t b = ray_off[r];
     const int n = (int)(ray_off[r + 1] - ray_off[r]);
     if (n == 0) {
