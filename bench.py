@@ -53,7 +53,7 @@ def launches_per_step(tiles_x: int, tiles_y: int) -> int:
     """Kernel launches of one step (memsets are not kernels).  A radix pass is histogram + three scan kernels + scatter."""
     bounds = 1 + _radix_passes(tiles_y) * 5 + 1                  # bounds kernel, slot sort on the tile row, record gather
     tile_map = 1 + 3 + 1 + 1 + _radix_passes(tiles_x * tiles_y - 1) * 5 + 1   # areas, scan, total, emission, pair sort, offsets
-    forward = 1 + 1 + 3 + 3 + 1 + 1 + 3          # mask, tile sort, two scans, totals, evaluation, sweep per ray-length class
+    forward = 1 + 1 + 3 + 3 + 1 + 1 + 2          # mask, tile sort, two scans, totals, evaluation, sweep per ray-length class
     backward = 4                                # zero, pair kernel, per-slot conversion, scatter of the SH gradient
     return bounds + tile_map + forward + backward
 

@@ -792,14 +792,15 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
 }
 
 // One launch per class of ray length, so that each gets the registers and the shared memory it needs and no more
-// (short rays then run at several times the occupancy of the longest): class 0 up to 64 hits, class 1 up to 256,
-// class 2 beyond.  Every launch walks all rays and a warp returns at once if its ray belongs to another class;
-// class 0 also writes the background colour of rays without hits.
+// (the shorter rays then run at a higher occupancy than the longest): class 1 up to 256 hits, class 2 beyond.
+// Every launch walks all rays and a warp returns at once if its ray belongs to the other class; class 1 also
+// writes the background colour of rays without hits.
 template <int CLS>
 struct SweepClass {
-    static constexpr int LO = CLS == 0 ? 0 : (CLS == 1 ? 64 : 256);                 // exclusive lower bound of n
-    static constexpr int CAP = CLS == 0 ? 64 : (CLS == 1 ? 256 : SORT_CAP);         // entries staged per warp
-    static constexpr int MIN_BLOCKS = CLS == 0 ? 12 : (CLS == 1 ? 6 : 4);
+    static_assert(CLS == 1 || CLS == 2, "two classes");
+    static constexpr int LO = CLS == 1 ? 0 : 256;                    // exclusive lower bound of n
+    static constexpr int CAP = CLS == 1 ? 256 : SORT_CAP;            // entries staged per warp
+    static constexpr int MIN_BLOCKS = CLS == 1 ? 6 : 4;
     static constexpr int SMEM = SWEEP_WARPS * CAP * 28;
 };
 
@@ -829,7 +830,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     const size_t b = ray_off[r];
     const int n = (int)(ray_off[r + 1] - ray_off[r]);
     if (n == 0) {
-        if (CLS == 0 && lane == 0) {
+        if (CLS == 1 && lane == 0) {
             color[3 * r] = bg0; color[3 * r + 1] = bg1; color[3 * r + 2] = bg2;
             t_final[r] = 1.0f;
         }
@@ -842,11 +843,10 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
 #define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, w_only, ray_gid, ray_slot, s_cs, s_al, s_tg)
-    if (CLS == 0) {
+    if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
-        else GART_SWEEP(2);
-    } else if (CLS == 1) {
-        if (n <= 128) GART_SWEEP(4);
+        else if (n <= 64) GART_SWEEP(2);
+        else if (n <= 128) GART_SWEEP(4);
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
@@ -977,7 +977,6 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     GART_LAUNCH_CHECK();
     GART_SWEEP_LAUNCH(2)   // the longest rays first
     GART_SWEEP_LAUNCH(1)
-    GART_SWEEP_LAUNCH(0)
 #undef GART_SWEEP_LAUNCH
     GART_LAUNCH_CHECK();
     return GART_OK;

@@ -22,8 +22,8 @@ def test_shard_views_partition():
 
 
 def test_launch_count_and_bytes():
-    assert bench.launches_per_step(155, 103) == 7 + (7 + 2 * 5) + 13 + 4     # 7 row bits -> 1 pass, 14 tile bits -> 2 passes
-    assert bench.launches_per_step(8, 8) == 7 + (7 + 5) + 13 + 4
+    assert bench.launches_per_step(155, 103) == 7 + (7 + 2 * 5) + 12 + 4     # 7 row bits -> 1 pass, 14 tile bits -> 2 passes
+    assert bench.launches_per_step(8, 8) == 7 + (7 + 5) + 12 + 4
     B = bench.algorithmic_bytes_backward(H=100, P=10, n_vis=5, n_pixels=64, K=16)
     assert B == 1600 + 40 + 4 * 61 * 5 + 4 * 59 * 5 + 28 * 64
     # the traffic model adds its per-unit figures
