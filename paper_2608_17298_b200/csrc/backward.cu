@@ -210,20 +210,50 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
-            produce(cur, nxt, nxt2, 2);   // refill the stage just released
+            if (k + 1 < nchunks) produce(cur, nxt, nxt2, 2);   // refill the stage just released (after the last chunk it first serves the flush)
         }
-        if (cur.c != 0) {
-            // one vector atomic per 16 bytes of the Gaussian's record
-#pragma unroll
-            for (int q = 0; q < AW / 4; ++q) {
+        {
+            // Flush through the stage just released, so that consecutive lanes add consecutive 16-byte pieces of one
+            // record: the atomics of a record then reach L2 as whole 32-byte sectors (about 9 sector updates per pair
+            // instead of 15).  Two rounds of FLUSH_Q pieces per lane, then the last piece directly.
+            constexpr int NQ = AW / 4, FLUSH_Q = BWD_CHUNK;
+            static_assert(NQ <= 2 * FLUSH_Q + 1 && NQ >= 1, "flush rounds");
+            float4* tb = my_stage + ((unit - 1u) % BWD_STAGES) * BWD_STAGE_F4;
+            const uint32_t tag = cur.c != 0 ? cur.sid : 0xffffffffu;
+            auto piece = [&](int q) {
                 float v[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int wd = 4 * q + i;
                     v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f);   // constants left out by sh_poly
                 }
-                red_add_f4_hint(gacc_piece(gacc, cur.sid, q), v[0], v[1], v[2], v[3], pol_keep);
+                return make_float4(v[0], v[1], v[2], v[3]);
+            };
+#pragma unroll
+            for (int q0 = 0; q0 + 1 < NQ; q0 += FLUSH_Q) {
+                const int nq = NQ - 1 - q0 < FLUSH_Q ? NQ - 1 - q0 : FLUSH_Q;   // compile-time after unrolling
+#pragma unroll
+                for (int j = 0; j < FLUSH_Q; ++j)
+                    if (j < nq) tb[lane * nq + j] = piece(q0 + j);
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < FLUSH_Q; ++j) {
+                    if (j < nq) {
+                        const int i = j * 32 + lane, pr = i / nq, q = q0 + i - pr * nq;
+                        const float4 v = tb[i];
+                        const uint32_t sd = __shfl_sync(0xffffffffu, tag, pr);
+                        if (sd != 0xffffffffu) red_add_f4_hint(gacc_piece(gacc, sd, q), v.x, v.y, v.z, v.w, pol_keep);
+                    }
+                }
+                __syncwarp();
             }
+            if (tag != 0xffffffffu) {
+                const float4 v = piece(NQ - 1);
+                red_add_f4_hint(gacc_piece(gacc, tag, NQ - 1), v.x, v.y, v.z, v.w, pol_keep);
+            }
+            fence_proxy_async();
+            __syncwarp();
+            produce(cur, nxt, nxt2, 2);   // now refill the stage
         }
         if (nxt.cmax == 0) break;
         cur = nxt;
