@@ -173,14 +173,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         cp_async_wait_all();
     };
 
-    uint32_t r0 = warp * 32;
-    GroupDesc<MW> cur = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0, lane);
+    // The warp's j-th group is group j * BWD_WARPS + (j even ? warp : BWD_WARPS - 1 - warp) of the tile: groups descend
+    // in hit count, and this serpentine deal gives every warp of the block nearly the same number of iterations.
+    auto first_rank = [&](uint32_t j) { return 32u * (j * BWD_WARPS + ((j & 1u) ? (uint32_t)(BWD_WARPS - 1 - warp) : (uint32_t)warp)); };
+    uint32_t gj = 0;
+    GroupDesc<MW> cur = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, first_rank(0), lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
     issue_params(cur);
-    GroupDesc<MW> nxt = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + BWD_THREADS, lane);
+    GroupDesc<MW> nxt = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, first_rank(1), lane);
     while (true) {
         // descriptor two groups ahead: the producer may reach it later in this group (not yet: its loads are in flight)
-        const GroupDesc<MW> nxt2 = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * BWD_THREADS, lane);
+        const GroupDesc<MW> nxt2 = load_group<MW>(rank_sid, rank_mask, rank_gstart, begin, n, first_rank(gj + 2), lane);
         produce(cur, nxt, nxt2, 1);
         ShRegs<K> R;
         float geo[11];
@@ -258,7 +261,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         if (nxt.cmax == 0) break;
         cur = nxt;
         nxt = nxt2;
-        r0 += BWD_THREADS;
+        ++gj;
         --pw;   // the producer is never behind the consumer: pw >= 1 here
     }
 }
