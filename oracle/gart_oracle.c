@@ -27,7 +27,9 @@
  * Gaussian; T_final = prod(1 - alpha_i) and the partition-of-unity invariant;
  * a two-Gaussian closed form with permutation invariance; Unsoeld's theorem and
  * numerical orthonormality for the SH table; central finite differences for
- * every gradient word; translation invariance (sum of dL/dmu = -dL/do).
+ * every gradient word; translation invariance (sum of dL/dmu = -dL/do); the per-hit
+ * intermediate-buffer entries against the opacity and SH gradients they must reproduce
+ * (dL/dsigma = sum <g, entry.xyz> / sigma, dL/dsh = sum Y w g on unclamped channels).
  *
  * Readings of the paper used here (the paper is silent or ambiguous):
  *   - pinhole camera, pixel centres at +0.5, unit ray directions;
@@ -578,18 +580,46 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
 }
 
 /*
+ * What the compact intermediate buffer (Sec. 4.3-4.4) has to hold per hit for the primitive-centric
+ * backward, in the reading where the forward stores the derivative of the pixel colour instead of
+ * (T, alpha, colour): from Eq. 6-8, with c the clamped colour of hit i, w = T_i alpha_i and B the colour
+ * composited behind the hit (background included),
+ *     alpha_i dC/dalpha_i = w c - alpha_i / (1 - alpha_i) B.
+ * entry [H,4] receives that vector and w; flags [H] bit ch is set where colour channel ch is not
+ * clamped (its SH gradient is w g_ch Y_k, zero otherwise).  Hit order = the view's lists.
+ * Returns 0, or -1 if the view was not composited.
+ */
+int orc_view_lt_entries(const orc_view *v, double *entry, uint8_t *flags) {
+    if (!v->composited) return -1;
+    const uint64_t Hn = v->ray_off[v->n_rays];
+    for (uint64_t h = 0; h < Hn; ++h) {
+        const double al = v->alpha[h], w = v->T[h] * al;
+        for (int c = 0; c < 3; ++c) entry[4 * h + c] = w * v->col[3 * h + c] - al / (1.0 - al) * v->Rs[3 * h + c];
+        entry[4 * h + 3] = w;
+        if (flags) flags[h] = v->pos[h];
+    }
+    return 0;
+}
+
+/*
  * Analytic backward of L = sum_rays <g_ray, C_ray> for the current (composited) hit lists.
  * dL_dC [n_rays,3].  grad [n, 11+3K] doubles: d mean(3), d scale(3), d quat(4), d opacity(1),
  * d sh(K*3, coefficient-major); fully overwritten.  grad_abs (may be NULL) receives, in
  * the same layout, the sum of absolute values of the per-hit contributions (the
- * conditioning of each sum).  Returns 0, or -1 if the view was not composited.
+ * conditioning of each sum).  grad_abs_elem (may be NULL) is the same with every hit's
+ * contribution split further into its three colour channels: words 0..10 are linear in
+ * alpha dL/dalpha = sum_c g_c (T alpha col_c - alpha Rs_c / (1 - alpha)), and the scale takes
+ * sum_c |g_c (...)_c| in its place.  It bounds what a relative perturbation of the four
+ * per-hit quantities (those three terms and T alpha) can do to a gradient word.
+ * Returns 0, or -1 if the view was not composited.
  */
-int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *grad_abs) {
+int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *grad_abs, double *grad_abs_elem) {
     if (!v->composited) return -1;
     const int K = v->K, G = 11 + 3 * K;
     const int64_t NR = v->n_rays;
     memset(grad, 0, (size_t)v->sc.n * G * sizeof(double));
     if (grad_abs) memset(grad_abs, 0, (size_t)v->sc.n * G * sizeof(double));
+    if (grad_abs_elem) memset(grad_abs_elem, 0, (size_t)v->sc.n * G * sizeof(double));
     double o[3];
     cam_origin(&v->cam, o);
 #pragma omp parallel for schedule(dynamic, 64)
@@ -608,8 +638,12 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
             for (int k = 0; k < K; ++k) for (int c = 0; c < 3; ++c)
                 contrib[11 + 3 * k + c] = ((v->pos[h] >> c) & 1) ? Y[k] * T * al * g[c] : 0.0;
             /* alpha */
-            double dalpha = 0.0;
-            for (int c = 0; c < 3; ++c) dalpha += g[c] * (T * v->col[3 * h + c] - v->Rs[3 * h + c] / (1.0 - al));
+            double dalpha = 0.0, dalpha_abs = 0.0;
+            for (int c = 0; c < 3; ++c) {
+                const double term = g[c] * (T * v->col[3 * h + c] - v->Rs[3 * h + c] / (1.0 - al));
+                dalpha += term;
+                dalpha_abs += fabs(term);
+            }
             const double sigma = v->sc.opacity[i];
             const double rho = al / sigma;
             contrib[10] = dalpha * rho;
@@ -644,6 +678,17 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
                     if (contrib[k] != 0.0) {
 #pragma omp atomic
                         ga[k] += fabs(contrib[k]);
+                    }
+                }
+            }
+            if (grad_abs_elem) {
+                double *ge = grad_abs_elem + (size_t)i * G;
+                const double split = dalpha != 0.0 ? dalpha_abs / fabs(dalpha) : 0.0;   /* >= 1 */
+                for (int k = 0; k < G; ++k) {
+                    if (contrib[k] != 0.0) {
+                        const double a = fabs(contrib[k]) * (k < 11 ? split : 1.0);
+#pragma omp atomic
+                        ge[k] += a;
                     }
                 }
             }

@@ -71,8 +71,10 @@ def lib():
         L.orc_view_num_hits.restype = C.c_int64
         L.orc_view_get_hits.argtypes = [C.c_void_p] + [C.c_void_p] * 4
         L.orc_view_composite.argtypes = [C.c_void_p] + [C.c_void_p] * 3
-        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 3
+        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 4
         L.orc_view_backward.restype = C.c_int
+        L.orc_view_lt_entries.argtypes = [C.c_void_p] + [C.c_void_p] * 2
+        L.orc_view_lt_entries.restype = C.c_int
         _lib = L
     return _lib
 
@@ -235,16 +237,30 @@ class View:
         lib().orc_view_composite(self._h, _ptr(color), _ptr(t_final), _ptr(cnt))
         return color, t_final, cnt
 
-    def backward(self, dL_dC, with_abs=False):
-        """Gradients [n, 11+3K] (mean 3, scale 3, quat 4, opacity 1, sh K*3) of sum <dL_dC, C>."""
+    def backward(self, dL_dC, with_abs=False, with_elem=False):
+        """Gradients [n, 11+3K] (mean 3, scale 3, quat 4, opacity 1, sh K*3) of sum <dL_dC, C>.
+        with_abs adds the sums of absolute per-hit contributions, with_elem those of the contributions
+        split by colour channel (the scale of an error that is relative to the per-hit quantities)."""
         g = _f64(dL_dC).reshape(self.n_rays, 3)
         G = self.scene.grad_words
         grad = np.zeros((self.scene.n, G))
         gabs = np.zeros((self.scene.n, G)) if with_abs else None
-        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs))
+        gelem = np.zeros((self.scene.n, G)) if with_elem else None
+        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs), _ptr(gelem))
         if rc != 0:
             raise RuntimeError("composite() must run before backward()")
-        return (grad, gabs) if with_abs else grad
+        out = (grad,) + ((gabs,) if with_abs else ()) + ((gelem,) if with_elem else ())
+        return out if len(out) > 1 else grad
+
+    def lt_entries(self):
+        """Per hit, in list order: (entry [H,4] = alpha dC/dalpha (3) and w = T alpha; flags [H] uint8, bit ch set
+        where colour channel ch is not clamped)."""
+        H = int(lib().orc_view_num_hits(self._h))
+        entry = np.zeros((max(H, 1), 4))
+        flags = np.zeros(max(H, 1), dtype=np.uint8)
+        if lib().orc_view_lt_entries(self._h, _ptr(entry), _ptr(flags)) != 0:
+            raise RuntimeError("composite() must run before lt_entries()")
+        return entry[:H], flags[:H]
 
 
 def render(scene: OracleScene, cam, dL_dC=None, mode=BRUTE, pixel_mask=None, hit_lists=None, **kw):
