@@ -338,6 +338,23 @@ def run_ours(args):
             if i > 0:
                 ht.append(a0.elapsed_time(a1))
         hybrid_ms = float(np.mean(ht))
+    # ---- 8-byte LT entries (four halves per hit): forward and primitive-centric backward of the same view
+    lt16_ms = None
+    if args.lt16_reps > 0:
+        import dataclasses
+        cfg_8 = dataclasses.replace(cfg, lt_format=2)
+        ft, bt = [], []
+        for i in range(args.lt16_reps + 1):                      # one untimed run first
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record(stream)
+            G.run_forward(cfg_8, g, cams[last_v], buf, stream, ray_lists=False)
+            e1.record(stream)
+            G.run_backward(cfg_8, g, cams[last_v], buf, dls[last_v], ga, stream)
+            e2.record(stream)
+            torch.cuda.synchronize()
+            if i > 0:
+                ft.append(e0.elapsed_time(e1)); bt.append(e1.elapsed_time(e2))
+        lt16_ms = {"forward": float(np.mean(ft)), "backward": float(np.mean(bt))}
     last = cl[-1]
     prim_last_ms = float(stage[-1, 2])
     del ga
@@ -426,6 +443,7 @@ def run_ours(args):
         "backward_atomic_ms": atomic_ms,
         "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
         "backward_hybrid_ms": hybrid_ms,
+        "lt_8byte_ms": lt16_ms,
         "backward_warp_per_pair_ms": warp_ms,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(-(-cams[0].width // cfg.tile_size), -(-cams[0].height // cfg.tile_size)) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
@@ -447,6 +465,7 @@ def main():
     ap.add_argument("--atomic-reps", type=int, default=2)
     ap.add_argument("--warp-reps", type=int, default=1, help="timed runs of the warp-per-pair backward on the last view (0: skip)")
     ap.add_argument("--hybrid-reps", type=int, default=1, help="timed runs of the hybrid backward on the last view (0: skip)")
+    ap.add_argument("--lt16-reps", type=int, default=2, help="timed runs of forward + backward with 8-byte LT entries on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--oracle-frac", type=float, default=0.08)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -60,7 +60,10 @@ typedef struct {
     int32_t tile_size;    /* 8 (the paper's choice, Sec. 4.4) or 16 */
     int32_t lt_format;    /* what gart_forward stores per hit: 0 = the 16-byte entry that gart_backward reads,
                              1 = only its fourth word, 4 bytes per hit (for gart_backward_hybrid, Sec. 4.4
-                             "Hybrid approach"); lt then holds cap_hits floats */
+                             "Hybrid approach"); lt then holds cap_hits floats;
+                             2 = the entry as four halves, 8 bytes per hit (the half-precision buffer that the
+                             paper's limitations section, "VRAM Consumption", names as a way to save
+                             memory); gart_backward reads this format too */
 } gart_config;
 
 /* Host struct. */
@@ -202,6 +205,11 @@ gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, in
  *              alpha dC/dalpha by Eq. 6-8; word 3 = w, whose three low mantissa bits are replaced by
  *              flags "channel r, g, b of c is not clamped".  This is all the backward pass needs of
  *              the ray's state, and nothing in it is a difference of nearly equal sums.
+ *              With cfg->lt_format = 2 the entry of slot i is the 8 bytes at lt + 8 i: four IEEE halves
+ *              h0..h3, h_ch = 4096 x word ch (clamped to +-60000) rounded to nine mantissa bits (nearest,
+ *              ties to even) with the half's lowest bit replaced by the flag of channel ch, h3 = the half
+ *              nearest to 4096 w.  A decoded colour word is within 2^-10 (relative) of the fp32 value, the
+ *              weight within 2^-11; magnitudes below 2^-26 lose relative precision, below 2^-37 vanish.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
  *              baseline and parity checks read the two lists: pass NULL for both to skip them.
@@ -230,6 +238,9 @@ gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const 
  *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
  *   counts: read (a set error bit skips the work); GART_ERRBIT_TIMEOUT is set if a wait on an
  *        asynchronous copy ran out, in which case grad is incomplete.
+ * cfg->lt_format must be the one the forward wrote lt with, 0 or 2 (INVALID_ARG otherwise).  With 8-byte
+ * entries every gradient word, being linear in the four words of its hits' entries, moves by at most 2^-10
+ * of the sum of the absolute per-hit, per-channel terms of that word.
  * The main kernel uses up to 99 KB of dynamic shared memory per block (opt-in set by the call): LT blocks
  * and the Gaussians' records are streamed in with bulk asynchronous copies, one rank group ahead.
  */

@@ -75,7 +75,8 @@ __device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* g
     geo[6] = fmaf(tx, yy, geo[6]); geo[7] = fmaf(tx, yz, geo[7]); geo[8] = fmaf(ty, yz, geo[8]);
 }
 
-template <int TS, int DEG>
+// FMT: 0 = 16-byte LT entries, 2 = 8-byte entries (four halves, twice as many per pipeline stage).
+template <int TS, int DEG, int FMT>
 __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4* __restrict__ rec,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
@@ -84,6 +85,8 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                                                                 Gacc gacc, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
+    constexpr int EB = FMT == 2 ? 8 : 16;                  // bytes per LT entry
+    constexpr int CH = BWD_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage
     // evaluation record of a lane's Gaussian (the first 5 float4 of the slot's record), staged through shared
     // memory one group ahead
     constexpr int PF4 = BWD_PF4, RS4 = (20 + SW + 3) / 4;
@@ -122,7 +125,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     }
     __syncthreads();
 
-    const float4* lt_tile = lt + tile_lt_base[tile];
+    const char* lt_tile = reinterpret_cast<const char*>(lt) + (size_t)tile_lt_base[tile] * EB;
     const float4* spix_lane = spix + (lane & (PixLayout<TS>::COPIES - 1));
     float4* my_stage = dyn + (size_t)warp * BWD_STAGES * BWD_STAGE_F4;
     float4* my_par = dyn + (size_t)BWD_WARPS * BWD_STAGES * BWD_STAGE_F4 + (size_t)(warp * 32 + lane) * PSTR;
@@ -146,12 +149,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
             else if (pw == 1) { cm = b.cmax; gs = b.gstart; }
             else { cm = c.cmax; gs = c.gstart; }
             if (cm == 0) break;                                   // ranks descend in hit count: no later group has hits
-            if (pk * BWD_CHUNK >= cm) { ++pw; pk = 0; continue; }
+            if (pk * CH >= cm) { ++pw; pk = 0; continue; }
             if (lane == 0) {
-                const int ne = min(BWD_CHUNK, cm - pk * BWD_CHUNK);
-                const uint32_t bytes = (uint32_t)ne * 512u, s = produced % BWD_STAGES;
+                const int ne = min(CH, cm - pk * CH);
+                const uint32_t bytes = (uint32_t)ne * (32u * EB), s = produced % BWD_STAGES;
                 mbar_expect_tx(bar_addr + 8u * s, bytes);
-                bulk_g2s_hint(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + gs + (size_t)pk * BWD_STAGE_F4, bytes, bar_addr + 8u * s, pol_stream);
+                bulk_g2s_hint(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + ((size_t)gs + (size_t)pk * (CH * 32)) * EB, bytes, bar_addr + 8u * s, pol_stream);
             }
             ++produced;
             ++pk;
@@ -193,23 +196,27 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         const PairGeo P = pair_geo(unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]), x0, y0);   // (stale data for lanes without hits: never used)
         R.clear();
         if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
-        const int nchunks = (cur.cmax + BWD_CHUNK - 1) / BWD_CHUNK;
+        const int nchunks = (cur.cmax + CH - 1) / CH;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % BWD_STAGES;
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / BWD_STAGES) & 1u))) { fail(); return; }
-            const float4* sl = my_stage + s * BWD_STAGE_F4 + lane;
-            const int e_end = min(cur.c, (k + 1) * BWD_CHUNK);
+            const char* sl = reinterpret_cast<const char*>(my_stage + s * BWD_STAGE_F4) + lane * EB;   // entry j of the stage: sl + j * 32 * EB
+            auto entry = [&](const char* q) {
+                if constexpr (FMT == 2) return lt_unpack_half(*reinterpret_cast<const uint2*>(q));
+                else return *reinterpret_cast<const float4*>(q);
+            };
+            const int e_end = min(cur.c, (k + 1) * CH);
             // two hits per iteration: two independent dependency chains for the scheduler to interleave
-            int e = k * BWD_CHUNK;
-            const float4* se = sl;
-            for (; e + 1 < e_end; e += 2, se += 64) {
+            int e = k * CH;
+            const char* se = sl;
+            for (; e + 1 < e_end; e += 2, se += 64 * EB) {
                 const int p0 = cur.pm.next();
                 const int p1 = cur.pm.next();
-                const float4 L0 = se[0], L1 = se[32];
+                const float4 L0 = entry(se), L1 = entry(se + 32 * EB);
                 bwd_hit<TS, K>(P, R, geo, spix_lane, p0, L0);
                 bwd_hit<TS, K>(P, R, geo, spix_lane, p1, L1);
             }
-            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, cur.pm.next(), se[0]);
+            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, cur.pm.next(), entry(se));
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
@@ -266,12 +273,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     }
 }
 
-template <int TS, int DEG>
+template <int TS, int DEG, int FMT>
 static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                     const uint32_t* tile_lt_base, const float4* lt,
                                     const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
-    auto kern = bwd_pairs_kernel<TS, DEG>;
+    auto kern = bwd_pairs_kernel<TS, DEG, FMT>;
     constexpr int smem = BWD_DYN_SMEM;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
     kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts);
@@ -279,13 +286,13 @@ static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, c
     return GART_OK;
 }
 
-template <int TS>
+template <int TS, int FMT>
 static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                 const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                 const uint32_t* tile_lt_base, const float4* lt,
                                 const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
 #define GART_PAIRS(D) \
-    return launch_pairs_deg<TS, D>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts)
+    return launch_pairs_deg<TS, D, FMT>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts)
     switch (deg) {
         case 0: GART_PAIRS(0);
         case 1: GART_PAIRS(1);
@@ -307,7 +314,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     using namespace gart;
     if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte LT entries
+    if (cfg->lt_format != 0 && cfg->lt_format != 2) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte or 8-byte LT entries
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
     if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
@@ -321,8 +328,10 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     const int T = cf.tiles_x * cf.tiles_y;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
-    if (cfg->tile_size == 8) s = launch_pairs<8>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
-    else s = launch_pairs<16>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts);
+#define GART_PAIRS_TS(TSV, F) launch_pairs<TSV, F>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts)
+    if (cfg->lt_format == 0) s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 0) : GART_PAIRS_TS(16, 0);
+    else s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 2) : GART_PAIRS_TS(16, 2);
+#undef GART_PAIRS_TS
     if (s != GART_OK) return s;
     const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
     return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);

@@ -6,6 +6,7 @@
 // spherical-harmonics basis, and a three-kernel exclusive scan without device-side waiting.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -171,6 +172,35 @@ __device__ __forceinline__ void lt_weights(const float4 L, const float3 g, float
     wch[0] = (b & 1u) ? w * g.x : 0.0f;
     wch[1] = (b & 2u) ? w * g.y : 0.0f;
     wch[2] = (b & 4u) ? w * g.z : 0.0f;
+}
+
+// The 8-byte form of an LT entry (lt_format 2): four halves, each the value times 4096 (weights reach down to
+// alpha_min times a small transmittance: the scale keeps them in the half's normal range; +-60000 saturates).  The
+// three colour words are first rounded to nine mantissa bits (nearest, ties to even), so the half's lowest bit is
+// free for the channel's "not clamped" flag: a decoded word is within 2^-10 of its value, the weight within 2^-11.
+constexpr float LT_HALF_SCALE = 4096.0f;
+__device__ __forceinline__ uint32_t lt_half_word9(float x, uint32_t flag) {
+    const float y = fminf(fmaxf(x * LT_HALF_SCALE, -60000.0f), 60000.0f);
+    uint32_t u = __float_as_uint(y);
+    u += 0x1FFFu + ((u >> 14) & 1u);
+    u &= ~0x3FFFu;
+    return ((uint32_t)__half_as_ushort(__float2half_rn(__uint_as_float(u))) & 0xFFFEu) | flag;
+}
+__device__ __forceinline__ uint2 lt_pack_half(const float4 e) {
+    const uint32_t b = __float_as_uint(e.w);
+    const float w = __uint_as_float(b & ~7u);
+    const uint32_t h3 = __half_as_ushort(__float2half_rn(w * LT_HALF_SCALE));
+    return make_uint2(lt_half_word9(e.x, b & 1u) | (lt_half_word9(e.y, (b >> 1) & 1u) << 16),
+                      lt_half_word9(e.z, (b >> 2) & 1u) | (h3 << 16));
+}
+// Back to the layout of the 16-byte entry (flags in the low mantissa bits of w, which a widened half leaves zero).
+__device__ __forceinline__ float4 lt_unpack_half(const uint2 p) {
+    const uint32_t flags = (p.x & 1u) | ((p.x >> 15) & 2u) | ((p.y & 1u) << 2);
+    const uint32_t lo = p.x & 0xFFFEFFFEu, hi = p.y & 0xFFFFFFFEu;
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lo));
+    const float2 c = __half22float2(*reinterpret_cast<const __half2*>(&hi));
+    constexpr float inv = 1.0f / LT_HALF_SCALE;
+    return make_float4(a.x * inv, a.y * inv, c.x * inv, __uint_as_float(__float_as_uint(c.y * inv) | flags));
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -530,10 +530,12 @@ __device__ __forceinline__ void sort_regs(uint32_t (&k)[R], int lane) {
     }
 }
 
-// Store a hit's LT entry: all 16 bytes, or only the weight word where the caller asked for the 4-byte format.
-__device__ __forceinline__ void lt_store(float4* __restrict__ lt, bool w_only, uint32_t slot, const float4 e) {
-    if (w_only) reinterpret_cast<float*>(lt)[slot] = e.w;
-    else lt[slot] = e;
+// Store a hit's LT entry in the format the caller asked for: all 16 bytes, only the weight word (4 bytes), or
+// the four words as halves (8 bytes).
+__device__ __forceinline__ void lt_store(float4* __restrict__ lt, int lt_fmt, uint32_t slot, const float4 e) {
+    if (lt_fmt == 0) lt[slot] = e;
+    else if (lt_fmt == 1) reinterpret_cast<float*>(lt)[slot] = e.w;
+    else reinterpret_cast<uint2*>(lt)[slot] = lt_pack_half(e);
 }
 
 // true if record a must come after record b: larger t*, or equal t* and larger Gaussian id  (s_tg: t* bits and id per record)
@@ -547,7 +549,7 @@ __device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32
 template <int R>
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
-                                               float4* __restrict__ lt, bool w_only, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
+                                               float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                                                float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
     uint32_t k[R];
 #pragma unroll
@@ -667,7 +669,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const float4 cs = s_cs[c];
                 const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
-                lt_store(lt, w_only, slot, lt_entry(wgt, al[r], cs.x, cs.y, cs.z, k0, k1, k2));
+                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cs.x, cs.y, cs.z, k0, k1, k2));
                 if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cs.x, k0); k1 = fmaf(wgt, cs.y, k1); k2 = fmaf(wgt, cs.z, k2);
             }
@@ -711,7 +713,7 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
 
 __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int lane, size_t b, int64_t r,
                                             float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
-                                            float4* __restrict__ lt, bool w_only, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
+                                            float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
     for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
     __syncwarp();
     warp_sort(kp, n, lane);
@@ -778,7 +780,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
-            lt_store(lt, w_only, slot, lt_entry(wgt, ra.w, rb.x, rb.y, rb.z, k0 + e0, k1 + e1, k2 + e2));
+            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, rb.x, rb.y, rb.z, k0 + e0, k1 + e1, k2 + e2));
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -804,14 +806,15 @@ struct SweepClass {
     static constexpr int SMEM = SWEEP_WARPS * CAP * 28;
 };
 
-template <int CLS>
+template <int CLS, int FMT>   // FMT: the LT format (a compile-time constant keeps the store of the usual format free of tests)
 __global__ void __launch_bounds__(SWEEP_WARPS * 32, SweepClass<CLS>::MIN_BLOCKS)
 fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs, uint64_t* __restrict__ long_keys, int64_t n_rays,
                       int width, int tile_size, int tiles_x,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
-                      float4* __restrict__ lt, bool w_only, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
+                      float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                       const uint32_t* __restrict__ counts) {
     constexpr int CAP = SweepClass<CLS>::CAP;
+    constexpr int lt_fmt = FMT;
     if (counts[GART_CNT_ERROR]) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // rays in tile-major order: the 64 (256) rays of a tile are taken by neighbouring blocks, so the two halves of an
@@ -842,7 +845,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, w_only, ray_gid, ray_slot, s_cs, s_al, s_tg)
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
@@ -850,7 +853,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
-        else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, w_only, ray_gid, ray_slot);
+        else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
     }
 #undef GART_SWEEP
 }
@@ -927,7 +930,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !tile_lt_base || !ray_off || !counts)
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 0 && cfg->lt_format != 1) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format < 0 || cfg->lt_format > 2) return GART_ERR_INVALID_ARG;
     if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
     if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_sid || !rank_mask || !rank_gstart || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
@@ -967,16 +970,21 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
 
     const int64_t blocks = ceil_div((int64_t)T * ts * ts, SWEEP_WARPS);
     float4* lt4 = reinterpret_cast<float4*>(lt);
-    const bool w_only = cfg->lt_format == 1;
+    const int lt_fmt = cfg->lt_format;
     const float* bg = cfg->background;
-#define GART_SWEEP_LAUNCH(C)                                                                                                                    \
-    if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess)        \
-        return GART_ERR_CUDA;                                                                                                                   \
-    fwd_sort_sweep_kernel<C><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0], bg[1], \
-                                                                                             bg[2], color, t_final, lt4, w_only, ray_gid, ray_slot, counts); \
-    GART_LAUNCH_CHECK();
-    GART_SWEEP_LAUNCH(2)   // the longest rays first
-    GART_SWEEP_LAUNCH(1)
+#define GART_SWEEP_LAUNCH(C, F)                                                                                                                 \
+    {                                                                                                                                           \
+        if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
+            return GART_ERR_CUDA;                                                                                                               \
+        fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0], \
+                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, counts); \
+        GART_LAUNCH_CHECK();                                                                                                                    \
+    }
+#define GART_SWEEP_BOTH(F) GART_SWEEP_LAUNCH(2, F) GART_SWEEP_LAUNCH(1, F)   // the longest rays first
+    if (lt_fmt == 0) { GART_SWEEP_BOTH(0) }
+    else if (lt_fmt == 1) { GART_SWEEP_BOTH(1) }
+    else { GART_SWEEP_BOTH(2) }
+#undef GART_SWEEP_BOTH
 #undef GART_SWEEP_LAUNCH
     GART_LAUNCH_CHECK();
     return GART_OK;

@@ -107,7 +107,7 @@ class Config:
     near_z: float = 0.01
     background: tuple = (0.0, 0.0, 0.0)
     tile_size: int = 8
-    lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid)
+    lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid); 2: 8 bytes (gart_backward)
 
     def c(self) -> _Config:
         s = _Config()

@@ -86,6 +86,16 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         out["grad_hybrid"] = to_np(gh)[:g.n]
         # the other outputs of the forward do not depend on the LT format
         assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
+        # 8-byte LT entries (four halves per hit) and the primitive-centric backward on them
+        cfg_8 = dataclasses.replace(cfg, lt_format=2)
+        G.run_forward(cfg_8, g, cam, buf)
+        g8 = torch.empty_like(buf.grad)
+        G.run_backward(cfg_8, g, cam, buf, dl, g8)
+        torch.cuda.synchronize()
+        assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
+        out["grad_lt16"] = to_np(g8)[:g.n]
+        out["lt16"] = to_np(buf.lt).reshape(-1).view(np.uint16)[:4 * counts[G.CNT_LT_SLOTS]].reshape(-1, 4).copy()
+        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_slot))[:H], out["ray_slot"])
     return out
 
 
@@ -267,8 +277,28 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background)
     v2.set_hits(g_new_off, g_sel_gid)
     color, t_final, cnt = v2.composite()
-    grad, gabs = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True)
-    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "stats": stats, "sel": sel, "view": v2}
+    grad, gabs, gelem = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True)
+    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "gelem": gelem, "stats": stats, "sel": sel, "view": v2}
+
+
+def check_lt16(gpu, ref):
+    """The 8-byte entries the forward wrote (lt_format 2) against the oracle's entries of the same hits: flags
+    identical, every colour word within the encoding's 2^-10 and the weight within 2^-11, plus the fp32 error of
+    the encoder's input (the colour word is a difference of two products of size about w and alpha/(1-alpha) B).
+    Only for a replay of every ray (the oracle's hit order is then the GPU's list order)."""
+    import lt16
+    entry, flags = ref["view"].lt_entries()
+    slots = gpu["ray_slot"].astype(np.int64)
+    assert entry.shape[0] == slots.size
+    dec, f = lt16.decode(gpu["lt16"][slots])
+    assert np.array_equal(f, flags)
+    x, w = entry[:, :3], entry[:, 3]
+    fp32 = 1e-5 * (np.abs(x) + 8.0 * w[:, None])
+    assert np.all(np.abs(dec[:, :3] - x) <= 1.02 * lt16.REL_X * np.abs(x) + fp32 + lt16.ABS_SUB)
+    assert np.all(np.abs(dec[:, 3] - w) <= 1.02 * lt16.REL_W * w + 1e-5 * w + lt16.ABS_SUB)
+    # and the encoding is used to its precision: the typical error is that of nine / ten mantissa bits, not more
+    big = np.abs(x) > 1e-6
+    assert np.median(np.abs(dec[:, :3] - x)[big] / np.abs(x)[big]) > 2.0 ** -14
 
 
 def color_errors(gpu, ref, sel, cam):

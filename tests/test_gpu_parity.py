@@ -8,7 +8,11 @@ terms whatever the summation order):
   * gradients (all 11+3K words, every backward variant): |gpu - ref| <= 1e-3 max(|ref|, COND * A)
     or <= 1e-6, where A is the sum of the absolute values of the per-hit terms of that word (its
     conditioning).  A sum whose terms cancel to less than COND = 2% of their mass cannot reach a
-    relative 1e-3 in fp32 in any summation order, so the relative bar is measured against that floor.
+    relative 1e-3 in fp32 in any summation order, so the relative bar is measured against that floor;
+  * gradients from 8-byte LT entries (lt_format 2): the same bar plus 1.05 * 2^-10 * E, where E is the sum of
+    the absolute per-hit terms split by colour channel.  Every gradient word is linear in the four words of the
+    hit's entry, each stored to a relative 2^-10 (2^-11 for the weight), so that is the bound of the encoding;
+    the entries themselves are compared with the oracle's (tests/parity.py: check_lt16).
 """
 import numpy as np
 import pytest
@@ -44,6 +48,18 @@ def assert_grad(gpu_grad, ref, K, rows=None):
     return float(strict.mean())
 
 
+def assert_grad_lt16(gpu_grad, ref, K):
+    gw = 11 + 3 * K
+    g = gpu_grad[:, :gw].astype(np.float64)
+    r, a, e = ref["grad"], ref["gabs"], ref["gelem"]
+    d = np.abs(g - r)
+    ok = d <= 1.05 * 2.0 ** -10 * e + np.maximum(1e-3 * np.maximum(np.abs(r), COND * a), 1e-6)
+    assert ok.all(), ("gradient from 8-byte entries outside tolerance", int((~ok).sum()), float(d[~ok].max()))
+    assert np.all(gpu_grad[:, gw:] == 0)
+    # the encoding costs precision but not much: most words stay within 0.3 % of the oracle's
+    return float(((d <= 3e-3 * np.maximum(np.abs(r), COND * a)) | (d <= 1e-6)).mean())
+
+
 def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
     g = gs.upstream_gradient(cam, 0) if g is None else g
     gpu = P.run_gpu(scene, cam, cfg, g)
@@ -58,6 +74,8 @@ def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
     s3 = assert_grad(gpu["grad_hybrid"], ref, K)
     s4 = assert_grad(gpu["grad_warp"], ref, K)
     assert min(s1, s2, s3, s4) > 0.995            # the conditioning floor is the exception, not the rule
+    P.check_lt16(gpu, ref)
+    assert assert_grad_lt16(gpu["grad_lt16"], ref, K) > 0.85
     return gpu, ref
 
 
@@ -295,7 +313,7 @@ def test_invalid_arguments_return_status():
     with pytest.raises(G.GartError) as e:
         G.gart_tile_map(G.Config(), buf.rect, g.n, cam, buf.tile_off, buf.pair_gid, 100, buf.counts, buf.workspace[1:])
     assert e.value.status == 1                     # workspace not 256-byte aligned
-    # each backward variant wants its own LT format, and the forward knows two
+    # each backward variant wants its own LT format, and the forward knows three
     dl = torch.zeros((cam.height, cam.width, 3), dtype=torch.float32, device="cuda")
     with pytest.raises(G.GartError) as e:
         G.run_backward(G.Config(lt_format=1), g, cam, buf, dl)
@@ -304,10 +322,16 @@ def test_invalid_arguments_return_status():
         G.run_backward_warp(G.Config(lt_format=1), g, cam, buf, dl)
     assert e.value.status == 1
     with pytest.raises(G.GartError) as e:
+        G.run_backward_warp(G.Config(lt_format=2), g, cam, buf, dl)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
+        G.run_backward_hybrid(G.Config(lt_format=2), g, cam, buf, dl)
+    assert e.value.status == 1
+    with pytest.raises(G.GartError) as e:
         G.run_backward_hybrid(G.Config(lt_format=0), g, cam, buf, dl)
     assert e.value.status == 1
     with pytest.raises(G.GartError) as e:
-        G.run_forward(G.Config(lt_format=2), g, cam, buf)
+        G.run_forward(G.Config(lt_format=3), g, cam, buf)
     assert e.value.status == 1
     g.sh_degree = 3
     with pytest.raises(AssertionError):
