@@ -69,7 +69,7 @@ def algorithmic_bytes_backward(H, P, n_vis, n_pixels, K):
 # summarised in profiles/dram_traffic_unbounded6m_crop.md (8x8 tiles, SH degree 3, central crop of a view), each
 # divided by the unit it grows with: the pair kernel by hits, zeroing and conversion by visible Gaussians, the
 # scatter's reads by visible Gaussians and its writes by all Gaussians.
-TRAFFIC_MODEL = {"pairs_per_hit": 46.2, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
+TRAFFIC_MODEL = {"pairs_per_hit": 45.0, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
                  "scatter_read_per_visible": 186.0, "scatter_write_per_gaussian": 220.7}
 
 
