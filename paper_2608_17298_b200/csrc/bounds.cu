@@ -155,6 +155,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
 __constant__ float c_sh_norm[16] = {sh_norm(0), sh_norm(1), sh_norm(2), sh_norm(3), sh_norm(4), sh_norm(5), sh_norm(6), sh_norm(7),
                                     sh_norm(8), sh_norm(9), sh_norm(10), sh_norm(11), sh_norm(12), sh_norm(13), sh_norm(14), sh_norm(15)};
 
+constexpr int GATHER_UNROLL = 4;
+
 template <int DEG>
 __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
@@ -165,39 +167,59 @@ __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_
     __shared__ float s_norm[16];   // lanes index it divergently: shared memory, not the constant bank
     if (threadIdx.x < 16) s_norm[threadIdx.x] = c_sh_norm[threadIdx.x];
     __syncthreads();
-    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t slot = t / RS4;
-    const uint32_t q = t - slot * RS4;
-    if (slot >= n) return;
-    const uint32_t gid = vals_sorted[slot];
-    const bool vis = keys_sorted[slot] != key_none;
-    if (q == 0) {
-        slot_of_gid[gid] = vis ? slot : 0xffffffffu;
-        gid_of_slot[slot] = vis ? gid : 0xffffffffu;
-    }
-    if (!vis) return;
-    if (q == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
-        qs[2 * (size_t)slot] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 5];
-        qs[2 * (size_t)slot + 1] = pre_tmp[(size_t)gid * PRE_TMP_F4 + 6];
-    }
-    float4 v;
-    if (q < 5) {
-        v = pre_tmp[(size_t)gid * PRE_TMP_F4 + q];
-    } else {
-        const uint32_t e = (q - 5) * 4;
-        const float* sp = sh + (size_t)gid * SW;
-        // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
-        if (SW % 4 == 0) {
-            const float4 c = __ldg(reinterpret_cast<const float4*>(sp + e));
-            v = make_float4(s_norm[e / 3] * c.x, s_norm[(e + 1) / 3] * c.y, s_norm[(e + 2) / 3] * c.z, s_norm[(e + 3) / 3] * c.w);
-        } else {
-            v.x = e < SW ? s_norm[e / 3] * sp[e] : 0.0f;
-            v.y = e + 1 < SW ? s_norm[(e + 1) / 3] * sp[e + 1] : 0.0f;
-            v.z = e + 2 < SW ? s_norm[(e + 2) / 3] * sp[e + 2] : 0.0f;
-            v.w = e + 3 < SW ? s_norm[(e + 3) / 3] * sp[e + 3] : 0.0f;
+    // GATHER_UNROLL pieces per thread, their loads issued together (the chain id -> record otherwise leaves too few bytes in flight)
+    uint32_t slot[GATHER_UNROLL], q[GATHER_UNROLL], gid[GATHER_UNROLL];
+    bool vis[GATHER_UNROLL];
+#pragma unroll
+    for (int u = 0; u < GATHER_UNROLL; ++u) {
+        const uint32_t t = (blockIdx.x * GATHER_UNROLL + u) * blockDim.x + threadIdx.x;
+        slot[u] = t / RS4;
+        q[u] = t - slot[u] * RS4;
+        const bool in = slot[u] < n;
+        gid[u] = in ? vals_sorted[slot[u]] : 0u;
+        vis[u] = in && keys_sorted[slot[u]] != key_none;
+        if (in && q[u] == 0) {
+            slot_of_gid[gid[u]] = vis[u] ? slot[u] : 0xffffffffu;
+            gid_of_slot[slot[u]] = vis[u] ? gid[u] : 0xffffffffu;
         }
     }
-    rec[(size_t)slot * RS4 + q] = v;
+    float4 v[GATHER_UNROLL];
+#pragma unroll
+    for (int u = 0; u < GATHER_UNROLL; ++u) {
+        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!vis[u]) continue;
+        if (q[u] < 5) {
+            v[u] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + q[u]];
+        } else {
+            const uint32_t e = (q[u] - 5) * 4;
+            const float* sp = sh + (size_t)gid[u] * SW;
+            if (SW % 4 == 0) {
+                v[u] = __ldg(reinterpret_cast<const float4*>(sp + e));
+            } else {
+                v[u].x = e < SW ? sp[e] : 0.0f;
+                v[u].y = e + 1 < SW ? sp[e + 1] : 0.0f;
+                v[u].z = e + 2 < SW ? sp[e + 2] : 0.0f;
+                v[u].w = e + 3 < SW ? sp[e + 3] : 0.0f;
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < GATHER_UNROLL; ++u) {
+        if (!vis[u]) continue;
+        if (q[u] == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
+            qs[2 * (size_t)slot[u]] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 5];
+            qs[2 * (size_t)slot[u] + 1] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 6];
+        }
+        if (q[u] >= 5) {
+            // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
+            const uint32_t e = (q[u] - 5) * 4;
+            v[u].x *= e < SW ? s_norm[e / 3] : 0.0f;
+            v[u].y *= e + 1 < SW ? s_norm[(e + 1) / 3] : 0.0f;
+            v[u].z *= e + 2 < SW ? s_norm[(e + 2) / 3] : 0.0f;
+            v[u].w *= e + 3 < SW ? s_norm[(e + 3) / 3] : 0.0f;
+        }
+        rec[(size_t)slot[u] * RS4 + q[u]] = v[u];
+    }
 }
 
 struct BoundsWs {
@@ -286,7 +308,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     if (gthreads >= (int64_t)1 << 32) return GART_ERR_INVALID_ARG;   // (n beyond 1e8 at SH degree 3: 32-bit thread indices)
     float4* rec_out = reinterpret_cast<float4*>(pre);
 #define GART_GATHER(D)                                                                                                                        \
-    gather_records_kernel<D><<<(unsigned)ceil_div(gthreads, 256), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh, \
+    gather_records_kernel<D><<<(unsigned)ceil_div(gthreads, 256 * GATHER_UNROLL), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh, \
                                                                                 rec_out, rec_out + (size_t)g->n * rs4, slot_of_gid, gid_of_slot)
     switch (g->sh_degree) {
         case 0: GART_GATHER(0); break;
