@@ -34,11 +34,12 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
                                                      int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
                                                      float4* __restrict__ pre4, uint32_t* __restrict__ keys,
                                                      uint32_t* __restrict__ vals, uint32_t* __restrict__ counts) {
+    __shared__ float4 s_out[128 * PRE_TMP_F4];   // the block's 128 temporaries, staged so that the stores are whole rows
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int vis = 0, straddle = 0;
+    float4 q0 = make_float4(0, 0, 0, 0), q1 = q0, q2 = q0, q3 = q0, q4 = q0, q5 = q0, q6 = q0;
     if (i < n) {
         int x0 = 0, y0 = 0, x1 = -1, y1 = -1, c = 0;
-        float4 q0 = make_float4(0, 0, 0, 0), q1 = q0, q2 = q0, q3 = q0, q4 = q0;
         const double sigma = (double)opacity[i];
         if (sigma > alpha_min) {
             const double alpha_c = sqrt(2.0 * log(sigma / alpha_min));  // Eq. 10
@@ -134,14 +135,28 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
         }
         reinterpret_cast<int4*>(rect)[i] = make_int4(x0, y0, x1, y1);
         cls[i] = (uint8_t)c;
-        float4* p = pre4 + (size_t)i * PRE_TMP_F4;
-        p[0] = q0; p[1] = q1; p[2] = q2; p[3] = q3; p[4] = q4;
         if (vis) {   // quaternion, scale, opacity ride along so that the gather reads one contiguous piece
-            p[5] = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
-            p[6] = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
+            q5 = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
+            q6 = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
         }
         keys[i] = vis ? (uint32_t)(y0 / ts) : key_none;   // tile row of the rectangle's corner
         vals[i] = (uint32_t)i;
+    }
+    {
+        // a warp's 32 temporaries are contiguous in memory: through shared memory (lane stride 7 float4, odd: no bank
+        // conflicts) and out as 7 coalesced 512-byte rows
+        const int lane = threadIdx.x & 31, wbase = (threadIdx.x & ~31) * PRE_TMP_F4;
+        float4* mine = s_out + wbase + lane * PRE_TMP_F4;
+        mine[0] = q0; mine[1] = q1; mine[2] = q2; mine[3] = q3; mine[4] = q4; mine[5] = q5; mine[6] = q6;
+        __syncwarp();
+        const int64_t i_w = i - lane;                      // first Gaussian of the warp
+        const int64_t left = (n - i_w) * PRE_TMP_F4;       // float4 of this warp that exist
+        float4* dst = pre4 + (size_t)i_w * PRE_TMP_F4;
+#pragma unroll
+        for (int j = 0; j < PRE_TMP_F4; ++j) {
+            const int idx = j * 32 + lane;
+            if (idx < left) dst[idx] = s_out[wbase + idx];
+        }
     }
     const unsigned bv = __ballot_sync(0xffffffffu, vis), bs = __ballot_sync(0xffffffffu, straddle);
     if ((threadIdx.x & 31) == 0) {
