@@ -398,11 +398,24 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     const float4* spix_lane = spix + (lane & (EvalPix<TS>::COPIES - 1));
     float4* my_par = spar + (size_t)(warp * 32 + lane) * PSTR;
     const uint32_t par_addr = smem_u32(my_par);
+    // Copy the records of a group's 32 Gaussians: LP lanes take the first LP 16-byte pieces of one record (contiguous:
+    // whole sectors per request instead of one request per piece), 32 / LP records per instruction; a lane copies the
+    // pieces beyond LP of its own record.  A lane therefore writes other lanes' buffers: warp barriers around the use.
+    constexpr int LP = PF4 <= 8 ? 8 : 16, PPI = 32 / LP;
+    const uint32_t warp_par_addr = smem_u32(spar + (size_t)warp * 32 * PSTR);
     auto issue_params = [&](const EvalDesc<MW>& d) {
+        const uint32_t tag = d.c != 0 ? d.sid : 0xffffffffu;
+        const int piece = lane % LP;
+#pragma unroll
+        for (int i = 0; i < 32 / PPI; ++i) {
+            const int pair = i * PPI + lane / LP;
+            const uint32_t sd = __shfl_sync(0xffffffffu, tag, pair);
+            if (sd != 0xffffffffu && piece < PF4) cp_async16(warp_par_addr + 16u * (uint32_t)(pair * PSTR + piece), rec + (size_t)sd * PF4 + piece);
+        }
         if (d.c != 0) {
             const float4* src = rec + (size_t)d.sid * PF4;
 #pragma unroll
-            for (int q = 0; q < PF4; ++q) cp_async16(par_addr + 16u * q, src + q);
+            for (int q = LP; q < PF4; ++q) cp_async16(par_addr + 16u * q, src + q);
         }
     };
 
@@ -414,7 +427,8 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     while (true) {
         const EvalDesc<MW> nxt2 = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * EVAL_THREADS, lane);
         const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
-        cp_async_wait_all();   // this lane's record has landed (a lane reads only what it copied itself)
+        cp_async_wait_all();   // the copies this lane issued have landed
+        __syncwarp();          // ... and so have those of the other lanes, which hold pieces of this lane's record
         const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale for lanes without hits: unused)
         float shc[SW + 3];
 #pragma unroll
@@ -422,7 +436,8 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
             const float4 t = my_par[5 + q];
             shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
         }
-        if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
+        __syncwarp();                           // every lane has read its record: the buffers may be overwritten
+        if (nxt.cmax != 0) issue_params(nxt);
         uint32_t slot = lt_base + cur.gstart + lane;
         const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
         // one hit: evaluate, take the next free place of the ray's segment, write the 32-byte record
