@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
 __constant__ float c_sh_norm[16] = {sh_norm(0), sh_norm(1), sh_norm(2), sh_norm(3), sh_norm(4), sh_norm(5), sh_norm(6), sh_norm(7),
                                     sh_norm(8), sh_norm(9), sh_norm(10), sh_norm(11), sh_norm(12), sh_norm(13), sh_norm(14), sh_norm(15)};
 
-constexpr int GATHER_UNROLL = 4;
+constexpr int GATHER_UNROLL = 2;
 
 template <int DEG>
 __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
