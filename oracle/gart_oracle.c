@@ -77,6 +77,9 @@ typedef struct {
     double alpha_min;
     double near_z;
     double bg[3];
+    int64_t max_hits; /* 0: every hit is composited (the paper's setting).  m > 0: only the first m hits of a ray in
+                         (t*, id) order, the cap on ray-primitive intersections that the paper lists among the
+                         compromises of 3DGRT (comparison with prior work); later hits weigh nothing */
 } orc_config;
 
 /* ------------------------------------------------------------------ threads */
@@ -530,6 +533,8 @@ void orc_view_get_hits(const orc_view *v, uint64_t *ray_off, uint32_t *gid, doub
  * color [n_rays,3], t_final [n_rays], hit_count [n_rays] (any may be NULL).
  * Also keeps, per hit, T_i, the clamped colour and the colour composited behind
  * the hit (summed back to front), which the backward pass needs.
+ * With a hit cap (cfg.max_hits > 0) the ray ends after its first max_hits hits: the hits behind keep their
+ * place in the lists but get T_i = 0, so they add nothing to the colour, to T_final or to any gradient.
  */
 void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *hit_count) {
     const int64_t NR = v->n_rays;
@@ -551,24 +556,26 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
             orc_sh_basis(d, Y);
             for (uint64_t h = b; h < e; ++h) {
                 const double *sh = v->sc.sh + (size_t)v->gid[h] * K * 3;
+                const int capped = v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits;
                 uint8_t pm = 0;
                 for (int c = 0; c < 3; ++c) {
                     double raw = 0.5;
                     for (int k = 0; k < K; ++k) raw += Y[k] * sh[3 * k + c];
                     if (raw > 0.0) pm |= (uint8_t)(1u << c);
                     v->col[3 * h + c] = raw > 0.0 ? raw : 0.0;
-                    C[c] += T * v->alpha[h] * v->col[3 * h + c];
+                    if (!capped) C[c] += T * v->alpha[h] * v->col[3 * h + c];
                 }
                 v->pos[h] = pm;
-                v->T[h] = T;
-                T *= (1.0 - v->alpha[h]);
+                v->T[h] = capped ? 0.0 : T;
+                if (!capped) T *= (1.0 - v->alpha[h]);
             }
         }
         double Rb[3] = {T * v->cfg.bg[0], T * v->cfg.bg[1], T * v->cfg.bg[2]};
         for (int c = 0; c < 3; ++c) C[c] += Rb[c];
         for (uint64_t h = e; h-- > b;) {
+            const int capped = v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits;
             for (int c = 0; c < 3; ++c) {
-                v->Rs[3 * h + c] = Rb[c];
+                v->Rs[3 * h + c] = capped ? 0.0 : Rb[c];   /* nothing lies behind a hit that is not composited */
                 Rb[c] += v->T[h] * v->alpha[h] * v->col[3 * h + c];
             }
         }

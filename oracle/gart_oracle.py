@@ -43,7 +43,7 @@ class _Scene(C.Structure):
 
 
 class _Config(C.Structure):
-    _fields_ = [("alpha_min", C.c_double), ("near_z", C.c_double), ("bg", C.c_double * 3)]
+    _fields_ = [("alpha_min", C.c_double), ("near_z", C.c_double), ("bg", C.c_double * 3), ("max_hits", C.c_int64)]
 
 
 _lib = None
@@ -105,9 +105,10 @@ def _camera(cam) -> _Camera:
     return c
 
 
-def _config(alpha_min, near, bg) -> _Config:
+def _config(alpha_min, near, bg, max_hits=0) -> _Config:
     c = _Config()
     c.alpha_min, c.near_z = float(alpha_min), float(near)
+    c.max_hits = int(max_hits)
     for i in range(3):
         c.bg[i] = float(bg[i])
     return c
@@ -182,9 +183,10 @@ PREFILTER = 1  # candidates from the projected bounding sphere, padded by one pi
 class View:
     """One camera view of a scene: hit discovery, ordering, compositing, backward."""
 
-    def __init__(self, scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, bg=(0.0, 0.0, 0.0)):
+    def __init__(self, scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, bg=(0.0, 0.0, 0.0), max_hits=0):
+        """max_hits > 0 composites only the first max_hits hits of every ray (0: all of them)."""
         self.scene, self.cam = scene, cam
-        self._c, self._g = _camera(cam), _config(alpha_min, near, bg)
+        self._c, self._g = _camera(cam), _config(alpha_min, near, bg, max_hits)
         self.n_rays = int(cam.width) * int(cam.height)
         self._h = lib().orc_view_create(C.byref(scene.c), C.byref(self._c), C.byref(self._g))
         self._keep = None
