@@ -64,6 +64,12 @@ typedef struct {
                              2 = the entry as four halves, 8 bytes per hit (the half-precision buffer that the
                              paper's limitations section, "VRAM Consumption", names as a way to save
                              memory); gart_backward reads this format too */
+    int32_t max_hits;     /* 0: every hit of a ray is composited (the paper's setting: "no maximum ray intersection
+                             cap").  m > 0: gart_forward composites only the first m hits of a ray in (t*, id)
+                             order, the cap that the paper lists among the compromises of 3DGRT.  The hits behind
+                             the cap keep their place in every list and their LT slot, with a zero entry: they
+                             add nothing to the colour, to T_final or to a gradient (the backward passes that
+                             read lt need no change; gart_backward_hybrid rejects a cap) */
 } gart_config;
 
 /* Host struct. */

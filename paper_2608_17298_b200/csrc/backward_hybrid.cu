@@ -245,6 +245,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor || !ray_off) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 1) return GART_ERR_INVALID_ARG;   // this pass reads the 4-byte LT format
+    if (cfg->max_hits != 0) return GART_ERR_INVALID_ARG;    // its pixel-centric part re-derives every hit's alpha: no cap
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
     if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;

@@ -562,7 +562,7 @@ __device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32
 // The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
 // slot as one float4, alpha apart; after the sort the three passes gather from there by sorted index.
 template <int R>
-__device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int lane, size_t b, int64_t r_idx,
+__device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                                                float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
@@ -632,12 +632,13 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             }
         }
     }
-    // front to back: transmittance in front of every hit (Eq. 7); padding positions get alpha = 0
+    // front to back: transmittance in front of every hit (Eq. 7); padding positions get alpha = 0, and so do the hits
+    // behind a cap on the composited hits (n_comp < n): they keep their place and their LT slot but weigh nothing
     float al[R];
     float lp = 1.0f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        al[r] = lane * R + r < n ? s_al[k[r] & KEY_IDX_MASK] : 0.0f;
+        al[r] = lane * R + r < n_comp ? s_al[k[r] & KEY_IDX_MASK] : 0.0f;
         lp *= 1.0f - al[r];
     }
     float inc = lp;
@@ -726,7 +727,7 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
     }
 }
 
-__device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int lane, size_t b, int64_t r,
+__device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int n_comp, int lane, size_t b, int64_t r,
                                             float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                             float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
     for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
@@ -754,7 +755,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         const int i = base + lane;
         const bool valid = i < n;
         const uint32_t c = valid ? (uint32_t)kp[i] : 0u;
-        const float alpha = valid ? __ldg(&rec[2 * c].w) : 0.0f;
+        const float alpha = i < n_comp ? __ldg(&rec[2 * c].w) : 0.0f;   // (n_comp <= n)
         float prod = 1.0f - alpha;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -780,6 +781,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
             const uint32_t c = (uint32_t)key;
             ra = __ldg(&rec[2 * c]);
             rb = __ldg(&rec[2 * c + 1]);
+            if (i >= n_comp) ra.w = 0.0f;   // behind the cap: not composited
             wgt = __uint_as_float((uint32_t)(key >> 32)) * ra.w;
             v0 = wgt * rb.x; v1 = wgt * rb.y; v2 = wgt * rb.z;
         }
@@ -827,7 +829,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
                       int width, int tile_size, int tiles_x,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                       float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
-                      const uint32_t* __restrict__ counts) {
+                      int max_comp, const uint32_t* __restrict__ counts) {
     constexpr int CAP = SweepClass<CLS>::CAP;
     constexpr int lt_fmt = FMT;
     if (counts[GART_CNT_ERROR]) return;
@@ -855,12 +857,13 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         return;
     }
     if (n <= SweepClass<CLS>::LO || (CLS < 2 && n > CAP)) return;
+    const int n_comp = min(n, max_comp);   // hits that are composited (all of them unless the caller set a cap)
     const float4* rec = recs + b * 2;
     extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
@@ -868,7 +871,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
-        else sweep_ray_long(rec, long_keys + b, n, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
+        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
     }
 #undef GART_SWEEP
 }
@@ -945,7 +948,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !tile_lt_base || !ray_off || !counts)
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format < 0 || cfg->lt_format > 2) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0) return GART_ERR_INVALID_ARG;
     if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
     if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_sid || !rank_mask || !rank_gstart || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
@@ -986,13 +989,14 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const int64_t blocks = ceil_div((int64_t)T * ts * ts, SWEEP_WARPS);
     float4* lt4 = reinterpret_cast<float4*>(lt);
     const int lt_fmt = cfg->lt_format;
+    const int max_comp = cfg->max_hits > 0 ? cfg->max_hits : 0x7fffffff;
     const float* bg = cfg->background;
 #define GART_SWEEP_LAUNCH(C, F)                                                                                                                 \
     {                                                                                                                                           \
         if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
             return GART_ERR_CUDA;                                                                                                               \
         fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0], \
-                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, counts); \
+                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, counts); \
         GART_LAUNCH_CHECK();                                                                                                                    \
     }
 #define GART_SWEEP_BOTH(F) GART_SWEEP_LAUNCH(2, F) GART_SWEEP_LAUNCH(1, F)   // the longest rays first

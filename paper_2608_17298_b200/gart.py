@@ -41,7 +41,7 @@ class GartError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
-                ("lt_format", C.c_int32)]
+                ("lt_format", C.c_int32), ("max_hits", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -108,11 +108,13 @@ class Config:
     background: tuple = (0.0, 0.0, 0.0)
     tile_size: int = 8
     lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid); 2: 8 bytes (gart_backward)
+    max_hits: int = 0           # > 0: only the first max_hits hits of a ray are composited (0: all, the paper's setting)
 
     def c(self) -> _Config:
         s = _Config()
         s.alpha_min, s.near_z, s.tile_size = self.alpha_min, self.near_z, int(self.tile_size)
         s.lt_format = int(self.lt_format)
+        s.max_hits = int(self.max_hits)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s

@@ -75,17 +75,18 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         G.run_backward_warp(cfg, g, cam, buf, dl, gw)          # ownership ablation: a warp per pair
         torch.cuda.synchronize()
         out["grad_warp"] = to_np(gw)[:g.n]
-        # hybrid backward: the forward again with 4-byte LT entries (same buffers, everything else unchanged)
         import dataclasses
-        cfg_h = dataclasses.replace(cfg, lt_format=1)
-        G.run_forward(cfg_h, g, cam, buf)
-        gh = torch.empty_like(buf.grad)
-        G.run_backward_hybrid(cfg_h, g, cam, buf, dl, gh)
-        torch.cuda.synchronize()
-        assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
-        out["grad_hybrid"] = to_np(gh)[:g.n]
-        # the other outputs of the forward do not depend on the LT format
-        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
+        if cfg.max_hits == 0:   # (the hybrid backward re-derives every alpha in its pixel pass: it takes no hit cap)
+            # hybrid backward: the forward again with 4-byte LT entries (same buffers, everything else unchanged)
+            cfg_h = dataclasses.replace(cfg, lt_format=1)
+            G.run_forward(cfg_h, g, cam, buf)
+            gh = torch.empty_like(buf.grad)
+            G.run_backward_hybrid(cfg_h, g, cam, buf, dl, gh)
+            torch.cuda.synchronize()
+            assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
+            out["grad_hybrid"] = to_np(gh)[:g.n]
+            # the other outputs of the forward do not depend on the LT format
+            assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
         # 8-byte LT entries (four halves per hit) and the primitive-centric backward on them
         cfg_8 = dataclasses.replace(cfg, lt_format=2)
         G.run_forward(cfg_8, g, cam, buf)
@@ -274,7 +275,7 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     stats["identical_lists"] = bool(identical)
     assert stats["band_hit"] + stats["band_order"] <= max(2, 1e-3 * stats["oracle_hits"])
     # replay the GPU's lists
-    v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background)
+    v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits)
     v2.set_hits(g_new_off, g_sel_gid)
     color, t_final, cnt = v2.composite()
     grad, gabs, gelem = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True)
