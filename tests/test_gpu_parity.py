@@ -14,6 +14,8 @@ terms whatever the summation order):
     hit's entry, each stored to a relative 2^-10 (2^-11 for the weight), so that is the bound of the encoding;
     the entries themselves are compared with the oracle's (tests/parity.py: check_lt16).
 """
+import dataclasses
+
 import numpy as np
 import pytest
 import torch
@@ -402,3 +404,10 @@ def test_host_entry_point_matches_device_path():
     with pytest.raises(G.GartError) as e:
         G.gart_view_host(cfg, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Hn // 2, arena)
     assert e.value.status == 3
+    # the configuration travels through the host entry point: a hit cap with 8-byte LT entries gives the device path's result
+    cfg2 = G.Config(tile_size=8, max_hits=4, lt_format=2)
+    gpu2 = P.run_gpu(scene, cam, dataclasses.replace(cfg2, lt_format=0), g, atomic=True)
+    G.gart_view_host(cfg2, hs, cam, torch.from_numpy(g).pin_memory(), color, grad, Pn + 5, Ln + 5, arena)
+    assert np.array_equal(color.numpy(), gpu2["color"]) and np.abs(gpu2["color"] - gpu["color"]).max() > 1e-3
+    a, b = grad.numpy().astype(np.float64), gpu2["grad_lt16"].astype(np.float64)
+    assert np.all(np.abs(a - b) <= 1e-4 * np.abs(b) + 1e-5 * np.abs(b).max(axis=1, keepdims=True) + 1e-7)
