@@ -50,10 +50,12 @@ def assert_grad(gpu_grad, ref, K, rows=None):
     return float(strict.mean())
 
 
-def assert_grad_lt16(gpu_grad, ref, K):
+def assert_grad_lt16(gpu_grad, ref, K, rows=None):
     gw = 11 + 3 * K
+    rows = np.arange(ref["grad"].shape[0]) if rows is None else rows
+    gpu_grad = gpu_grad[rows]
     g = gpu_grad[:, :gw].astype(np.float64)
-    r, a, e = ref["grad"], ref["gabs"], ref["gelem"]
+    r, a, e = ref["grad"][rows], ref["gabs"][rows], ref["gelem"][rows]
     d = np.abs(g - r)
     ok = d <= 1.05 * 2.0 ** -10 * e + np.maximum(1e-3 * np.maximum(np.abs(r), COND * a), 1e-6)
     assert ok.all(), ("gradient from 8-byte entries outside tolerance", int((~ok).sum()), float(d[~ok].max()))
@@ -250,6 +252,7 @@ def sampled_parity(scene, cam, cfg, view_seed, n_gauss=300, n_tiles=60, max_area
     K = (scene.sh_degree + 1) ** 2
     for variant in ("grad", "grad_atomic", "grad_hybrid", "grad_warp"):
         assert_grad(gpu[variant], ref, K, gsel)
+    assert assert_grad_lt16(gpu["grad_lt16"], ref, K, gsel) > 0.85      # the backward on 8-byte LT entries
     # the prefilter of the oracle is audited by true all-pairs brute force on a few rays
     audit = np.zeros_like(mask)
     ys, xs = np.nonzero(mask)
