@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
 }
 
 // ------------------------------------------------------------------------------- remaining terms, pixel-centric
-// One thread per ray; per hit 10 scalar atomics on the moments of the Gaussian's accumulation record
+// One thread per ray; per hit three 16-byte vector reductions on the moments of the Gaussian's accumulation record
 // (v, Q, sum alpha dL/dalpha: the same record that the primitive-centric pass fills, converted afterwards).
 template <int DEG>
 __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ slot_of_gid,
@@ -170,6 +170,7 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
     float B[K];
     sh_poly<K>(pixel_dir(cam, x, y), B);   // the records' SH coefficients carry the basis constants
     const float3 g = make_float3(dL_dC[3 * ray], dL_dC[3 * ray + 1], dL_dC[3 * ray + 2]);
+    const uint64_t pol_keep = l2_policy_evict_last();
     // front to back: log of the final transmittance
     float logT = 0.0f;
     for (uint32_t h = b; h < e; ++h) {
@@ -207,11 +208,11 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
         const float G = -0.5f * ad;
         const float3 xg = ray_xg(r);
         const float gx = G * xg.x, gy = G * xg.y, gz = G * xg.z;
-        float* gp = gacc.a + (size_t)sid * GACC_A_WORDS;
-        atomicAdd(gp + 0, gx); atomicAdd(gp + 1, gy); atomicAdd(gp + 2, gz);
-        atomicAdd(gp + 3, gx * xg.x); atomicAdd(gp + 4, gy * xg.y); atomicAdd(gp + 5, gz * xg.z);
-        atomicAdd(gp + 6, gx * xg.y); atomicAdd(gp + 7, gx * xg.z); atomicAdd(gp + 8, gy * xg.z);
-        atomicAdd(gp + 9, ad);
+        // words 0..9 of the slot's accumulation record as three 16-byte vector reductions (word 10 is unused and word
+        // 11, the first SH word, gets + 0)
+        red_add_f4_hint(gacc_piece(gacc, sid, 0), gx, gy, gz, gx * xg.x, pol_keep);
+        red_add_f4_hint(gacc_piece(gacc, sid, 1), gy * xg.y, gz * xg.z, gx * xg.y, gx * xg.z, pol_keep);
+        red_add_f4_hint(gacc_piece(gacc, sid, 2), gy * xg.z, ad, 0.0f, 0.0f, pol_keep);
         const float om = 1.0f - r.alpha;
         cb0 = fmaf(r.alpha, c0, om * cb0); cb1 = fmaf(r.alpha, c1, om * cb1); cb2 = fmaf(r.alpha, c2, om * cb2);
     }
