@@ -27,23 +27,39 @@ constexpr int BWD_LT_SMEM = BWD_WARPS * BWD_STAGES * BWD_STAGE_F4 * 16;
 constexpr int BWD_PF4 = 5;                             // float4 per lane of the staged evaluation record
 constexpr int BWD_DYN_SMEM = BWD_LT_SMEM + BWD_THREADS * BWD_PF4 * 16;
 
-// A pair's geometry, affine in the pixel position (u, v) inside the tile: d_g = dgA + u c0 + v c1 and
-// o_g x d_g = crA + u a1 + v b1 (a1 = c0 x m, b1 = c1 x m; dgA, crA the values at the tile's first pixel).
+// A pair's geometry, affine in the pixel position: with (uc, vc) the pixel of the tile nearest to the Gaussian's
+// reference position, d_g = dgC + (u - uc) c0 + (v - vc) c1 and o_g x d_g = crC + (u - uc) a1 + (v - vc) b1
+// (a1 = c0 x m, b1 = c1 x m; dgC, crC the values at that pixel).  o_g x d_g vanishes at the Gaussian's centre: expanded
+// about the tile's corner instead, a small Gaussian's hits would be differences of numbers up to tile size / offset
+// times larger, and lose that many digits.
 struct PairGeo {
-    float3 c0, c1, dgA, a1, b1, crA;
+    float3 c0, c1, dgC, a1, b1, crC;
+    float uc, vc;
 };
 
+template <int TS>
 __device__ __forceinline__ PairGeo pair_geo(const PreRec& P, int x0, int y0) {
     PairGeo g;
     g.c0 = P.c0; g.c1 = P.c1;
     g.a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
     g.b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
-    const float dx0 = (float)(x0 - P.ix) - P.rx, dy0 = (float)(y0 - P.iy) - P.ry;
-    g.dgA = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy0, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy0, P.dgr.y)),
-                        fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy0, P.dgr.z)));
-    g.crA = make_float3(fmaf(g.a1.x, dx0, fmaf(g.b1.x, dy0, P.k.x)), fmaf(g.a1.y, dx0, fmaf(g.b1.y, dy0, P.k.y)),
-                        fmaf(g.a1.z, dx0, fmaf(g.b1.z, dy0, P.k.z)));
+    const int xc = min(max(P.ix, x0), x0 + TS - 1), yc = min(max(P.iy, y0), y0 + TS - 1);
+    g.uc = (float)(xc - x0); g.vc = (float)(yc - y0);
+    const float dxc = (float)(xc - P.ix) - P.rx, dyc = (float)(yc - P.iy) - P.ry;
+    g.dgC = make_float3(fmaf(P.c0.x, dxc, fmaf(P.c1.x, dyc, P.dgr.x)), fmaf(P.c0.y, dxc, fmaf(P.c1.y, dyc, P.dgr.y)),
+                        fmaf(P.c0.z, dxc, fmaf(P.c1.z, dyc, P.dgr.z)));
+    g.crC = make_float3(fmaf(g.a1.x, dxc, fmaf(g.b1.x, dyc, P.k.x)), fmaf(g.a1.y, dxc, fmaf(g.b1.y, dyc, P.k.y)),
+                        fmaf(g.a1.z, dxc, fmaf(g.b1.z, dyc, P.k.z)));
     return g;
+}
+
+// d_g and o_g x d_g of pixel (u, v) of the tile
+__device__ __forceinline__ void pair_geo_at(const PairGeo& P, float u, float v, float3& dg, float3& cr) {
+    const float du = u - P.uc, dv = v - P.vc;   // small integers: exact
+    dg = make_float3(fmaf(P.c0.x, du, fmaf(P.c1.x, dv, P.dgC.x)), fmaf(P.c0.y, du, fmaf(P.c1.y, dv, P.dgC.y)),
+                     fmaf(P.c0.z, du, fmaf(P.c1.z, dv, P.dgC.z)));
+    cr = make_float3(fmaf(P.a1.x, du, fmaf(P.b1.x, dv, P.crC.x)), fmaf(P.a1.y, du, fmaf(P.b1.y, dv, P.crC.y)),
+                     fmaf(P.a1.z, du, fmaf(P.b1.z, dv, P.crC.z)));
 }
 
 // Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
@@ -53,11 +69,8 @@ __device__ __forceinline__ PairGeo pair_geo(const PreRec& P, int x0, int y0) {
 template <int TS, int K>
 __device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* geo, const float4* spix, int p, const float4 L) {
     const float4 pa = spix[PixLayout<TS>::index(p, 0, 0)], pb = spix[PixLayout<TS>::index(p, 1, 0)];   // spix points at the lane's copy
-    const float u = pa.w, v = pb.w;
-    const float3 dg = make_float3(fmaf(P.c0.x, u, fmaf(P.c1.x, v, P.dgA.x)), fmaf(P.c0.y, u, fmaf(P.c1.y, v, P.dgA.y)),
-                                  fmaf(P.c0.z, u, fmaf(P.c1.z, v, P.dgA.z)));
-    const float3 cr = make_float3(fmaf(P.a1.x, u, fmaf(P.b1.x, v, P.crA.x)), fmaf(P.a1.y, u, fmaf(P.b1.y, v, P.crA.y)),
-                                  fmaf(P.a1.z, u, fmaf(P.b1.z, v, P.crA.z)));
+    float3 dg, cr;
+    pair_geo_at(P, pa.w, pb.w, dg, cr);
     const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
     float Y[K];
     sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
@@ -132,7 +145,6 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     const uint32_t stage_addr = smem_u32(my_stage);
     const uint32_t par_addr = smem_u32(my_par);
     const uint32_t bar_addr = smem_u32(&bars[warp][0]);
-    const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
     // LT pipeline: unit u (a chunk of BWD_CHUNK entries per lane) uses stage u % BWD_STAGES, and the wait for
     // it uses parity (u / BWD_STAGES) & 1.  `unit` counts the units consumed, `produced` the units whose copy
     // has been issued; the producer cursor (pw, pk) = (group relative to the current one, chunk) runs up to
@@ -154,7 +166,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                 const int ne = min(CH, cm - pk * CH);
                 const uint32_t bytes = (uint32_t)ne * (32u * EB), s = produced % BWD_STAGES;
                 mbar_expect_tx(bar_addr + 8u * s, bytes);
-                bulk_g2s_hint(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + ((size_t)gs + (size_t)pk * (CH * 32)) * EB, bytes, bar_addr + 8u * s, pol_stream);
+                bulk_g2s_hint(stage_addr + s * (BWD_STAGE_F4 * 16u), lt_tile + ((size_t)gs + (size_t)pk * (CH * 32)) * EB, bytes, bar_addr + 8u * s, l2_policy_evict_first());
             }
             ++produced;
             ++pk;
@@ -193,7 +205,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
 #pragma unroll
         for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
         cp_async_wait_all();   // this lane's record has landed (a lane reads only what it copied itself)
-        const PairGeo P = pair_geo(unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]), x0, y0);   // (stale data for lanes without hits: never used)
+        const PairGeo P = pair_geo<TS>(unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]), x0, y0);   // (stale data for lanes without hits: never used)
         R.clear();
         if (nxt.cmax != 0) issue_params(nxt);   // the lane has read its record: its buffer may be overwritten
         const int nchunks = (cur.cmax + CH - 1) / CH;
@@ -230,12 +242,13 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
             static_assert(NQ <= 2 * FLUSH_Q + 1 && NQ >= 1, "flush rounds");
             float4* tb = my_stage + ((unit - 1u) % BWD_STAGES) * BWD_STAGE_F4;
             const uint32_t tag = cur.c != 0 ? cur.sid : 0xffffffffu;
+            const uint64_t pol_keep = l2_policy_evict_last();   // (made where they are used: the policies hold no register across the hit loop)
             auto piece = [&](int q) {
                 float v[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int wd = 4 * q + i;
-                    v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f);   // constants left out by sh_poly
+                    v[i] = wd < 11 ? geo[wd] : (wd < 11 + SW ? R.word(wd - 11) : 0.0f);   // (bare polynomials: the basis constants are applied when the records are converted)
                 }
                 return make_float4(v[0], v[1], v[2], v[3]);
             };
@@ -398,7 +411,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
         if (c == 0) break;   // ranks descend in hit count
         const uint32_t sid = __ldg(rank_sid + q);
         const float4* rp = rec + (size_t)sid * RS4;
-        const PairGeo P = pair_geo(unpack_pre(__ldg(rp), __ldg(rp + 1), __ldg(rp + 2), __ldg(rp + 3), __ldg(rp + 4)), x0, y0);
+        const PairGeo P = pair_geo<TS>(unpack_pre(__ldg(rp), __ldg(rp + 1), __ldg(rp + 2), __ldg(rp + 3), __ldg(rp + 4)), x0, y0);
         const float4* lp = lt_tile + __ldg(rank_gstart + q) + (r & 31u);
         float acc[AW];
 #pragma unroll
@@ -407,11 +420,8 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
             const int p = nth_set_bit<MW>(m, e);
             const float4 L = __ldg(lp + (size_t)32 * e);
             const float4 pa = spix[2 * p], pb = spix[2 * p + 1];
-            const float u = pa.w, v = pb.w;
-            const float3 dg = make_float3(fmaf(P.c0.x, u, fmaf(P.c1.x, v, P.dgA.x)), fmaf(P.c0.y, u, fmaf(P.c1.y, v, P.dgA.y)),
-                                          fmaf(P.c0.z, u, fmaf(P.c1.z, v, P.dgA.z)));
-            const float3 cr = make_float3(fmaf(P.a1.x, u, fmaf(P.b1.x, v, P.crA.x)), fmaf(P.a1.y, u, fmaf(P.b1.y, v, P.crA.y)),
-                                          fmaf(P.a1.z, u, fmaf(P.b1.z, v, P.crA.z)));
+            float3 dg, cr;
+            pair_geo_at(P, pa.w, pb.w, dg, cr);
             const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
             float Y[K], w[3];
             sh_poly<K>(make_float3(pa.x, pa.y, pa.z), Y);
@@ -426,9 +436,9 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
             acc[9] += ad;
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                acc[11 + 3 * k] = fmaf(sh_norm(k) * Y[k], w[0], acc[11 + 3 * k]);
-                acc[11 + 3 * k + 1] = fmaf(sh_norm(k) * Y[k], w[1], acc[11 + 3 * k + 1]);
-                acc[11 + 3 * k + 2] = fmaf(sh_norm(k) * Y[k], w[2], acc[11 + 3 * k + 2]);
+                acc[11 + 3 * k] = fmaf(Y[k], w[0], acc[11 + 3 * k]);
+                acc[11 + 3 * k + 1] = fmaf(Y[k], w[1], acc[11 + 3 * k + 1]);
+                acc[11 + 3 * k + 2] = fmaf(Y[k], w[2], acc[11 + 3 * k + 2]);
             }
         }
         // sum over the warp; lane i ends up with piece i (words 4 i .. 4 i + 3)

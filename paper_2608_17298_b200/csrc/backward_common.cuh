@@ -137,6 +137,13 @@ static __global__ void __launch_bounds__(256) bwd_zero_kernel(Gacc gacc, const u
     }
 }
 
+// The accumulation records hold dL/dsh against the bare SH polynomials (the kernels that fill them leave the basis
+// constants out, as the forward does): word 11 + 3 k + c is multiplied by the constant of basis function k when the
+// record is converted into the caller's gradient record.
+__device__ __forceinline__ float sh_word_norm(int word) {   // factor of gradient word `word` (11 <= word < 59)
+    return sh_norm((word - 11) / 3);
+}
+
 // One thread per slot: convert the accumulated moments (words 0..9) into d mean, d scale, d quat, d opacity and
 // write words 0..15 of the Gaussian's gradient record (all 32 lanes busy with the ~300-instruction conversion).
 static __global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* __restrict__ qs, const uint32_t* __restrict__ gid_of_slot,
@@ -157,8 +164,8 @@ static __global__ void __launch_bounds__(256) bwd_convert_kernel(const float4* _
     const GeoGrad o = moments_to_grads(v, Q, q, sc);
     out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
     out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
-    out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, c.w);
-    out[3] = d;
+    out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, sh_word_norm(11) * c.w);
+    out[3] = make_float4(sh_word_norm(12) * d.x, sh_word_norm(13) * d.y, sh_word_norm(14) * d.z, sh_word_norm(15) * d.w);
 }
 
 // In the order of the gradient records (sequential writes): 16 lanes per Gaussian; a Gaussian without a slot gets
@@ -174,6 +181,11 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
     const int64_t hw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // half-warp
     const int l = threadIdx.x & 15;
     const int64_t i0 = hw * FIN_ROWS;
+    // basis constants of this lane's four words (lanes 4..14 carry words 16..59; word 59 is padding)
+    float4 nf = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 4; q < 15; ++q)
+        if (l == q) nf = make_float4(sh_word_norm(4 * q), sh_word_norm(4 * q + 1), sh_word_norm(4 * q + 2), 4 * q + 3 < 59 ? sh_word_norm(4 * q + 3) : 0.0f);
     uint32_t s[FIN_ROWS];
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r) s[r] = i0 + r < n ? __ldg(slot_of_gid + i0 + r) : 0xffffffffu;
@@ -183,7 +195,8 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
         v[r] = (s[r] != 0xffffffffu && l >= 4 && l < 15) ? __ldcs(b4 + (size_t)s[r] * (GACC_B_WORDS / 4) + (l - 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r)
-        if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu)) __stcs(grad4 + (size_t)(i0 + r) * F4 + l, v[r]);
+        if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu))
+            __stcs(grad4 + (size_t)(i0 + r) * F4 + l, make_float4(nf.x * v[r].x, nf.y * v[r].y, nf.z * v[r].z, nf.w * v[r].w));
 }
 
 

@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int wd = 4 * q + i;
-                    v[i] = (wd >= 11 && wd < 11 + SW) ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f;
+                    v[i] = (wd >= 11 && wd < 11 + SW) ? R.word(wd - 11) : 0.0f;
                 }
                 red_add_f4_hint(gacc_piece(gacc, cur.sid, q), v[0], v[1], v[2], v[3], pol_keep);
             }

@@ -126,6 +126,24 @@ def test_hit_cap(m):
     assert hidden.any() and np.all(gpu["grad"][hidden] == 0) and np.all(gpu["grad_atomic"][hidden] == 0)
 
 
+@pytest.mark.parametrize("seed", [101, 102, 103, 104, 105, 106])
+def test_random_configurations(seed):
+    """Random combinations of image size (ragged against both tile sizes), field of view, SH degree, tile size, background,
+    alpha_min and hit cap on a random cluster, every ray and every backward variant against the oracle."""
+    rng = np.random.default_rng(seed)
+    deg = int(rng.integers(0, 4))
+    width, height = int(rng.integers(40, 150)), int(rng.integers(30, 110))
+    scene, cams = gs.config_cluster(n=int(rng.integers(500, 5000)), sh_degree=deg, width=width, height=height, seed=seed)
+    # a camera somewhere around the cluster (centre (0, 0, 3)), looking near its centre, any field of view
+    dirv = rng.normal(size=3)
+    pos = np.array([0.0, 0.0, 3.0]) + float(rng.uniform(2.0, 4.0)) * dirv / np.linalg.norm(dirv)
+    cam = gs.pinhole(width, height, float(rng.uniform(25.0, 75.0)), gs.look_at(pos, np.array([0.0, 0.0, 3.0]) + rng.uniform(-0.2, 0.2, 3)))
+    cfg = G.Config(tile_size=int(rng.choice([8, 16])), background=tuple(float(v) for v in rng.uniform(0, 1, 3)),
+                   alpha_min=float(rng.choice([1.0 / 255.0, 0.01, 0.03])), max_hits=int(rng.choice([0, 0, 3, 17])))
+    gpu, ref = full_parity(scene, cam, cfg, g=gs.upstream_gradient(cam, seed))
+    assert gpu["counts"][G.CNT_HITS] > 100
+
+
 def test_stricter_alpha_min():
     """alpha_min is a parameter (the paper's 1/255 is the default): a stricter threshold drops hits on both sides alike."""
     scene, cams = gs.config_cluster(n=4000, width=120, height=96, seed=22)
