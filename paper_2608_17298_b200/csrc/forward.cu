@@ -32,10 +32,15 @@ namespace gart {
 // zero of t).  qA <= 0 (the camera inside or beside the clamped ellipsoid) tests every column.
 constexpr int MASK_WARPS = 4;
 
+// The quadratic is expanded about the pixel (uc, vc) of the tile nearest to the Gaussian's reference position: Q is a
+// difference of two squares that nearly cancel at the boundary of a small Gaussian, and about the tile's corner its
+// coefficients would be up to (tile size / footprint)^2 times larger than the values that decide.  A row works in
+// u - uc and shifts its roots back by us = uc.
 struct RowQuad {
-    float qA, qB2, qC, t1, t0;   // qB2 = 2 qBh
-    __device__ __forceinline__ bool hit(float u) const {
-        return fmaf(fmaf(qA, u, qB2), u, qC) <= 0.0f && fmaf(t1, u, t0) > 0.0f;
+    float qA, qB2, qC, t1, t0, us;   // qB2 = 2 qBh
+    __device__ __forceinline__ bool hit(float u) const {   // u: column inside the tile
+        const float w = u - us;
+        return fmaf(fmaf(qA, w, qB2), w, qC) <= 0.0f && fmaf(t1, w, t0) > 0.0f;
     }
 };
 
@@ -73,8 +78,8 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
         const float z = -(qBh + copysignf(fast_sqrt(fmaxf(disc, 0.0f)), qBh));
         const float r1 = z * inv_qA;
         const float r2 = z != 0.0f ? q.qC * fast_rcp(z) : r1;
-        const float ulo = fminf(r1, r2), uhi = fmaxf(r1, r2);
-        const float ut = fminf(fmaxf(-q.t0 * inv_t1, -2.0f), 4194303.0f);   // t* > 0 on one side of it, strictly
+        const float ulo = fminf(r1, r2) + q.us, uhi = fmaxf(r1, r2) + q.us;
+        const float ut = fminf(fmaxf(fmaf(-q.t0, inv_t1, q.us), -2.0f), 4194303.0f);   // t* > 0 on one side of it, strictly
         const bool up = q.t1 > 0.0f;
         float flo = fast_ceil(fminf(fmaxf(ulo, -1.0f), 4194303.0f)), fhi = fast_floor(fminf(fmaxf(uhi, -2.0f), 4194303.0f));
         flo = up ? fmaxf(flo, fast_floor(ut) + 1.0f) : flo;     // smallest integer > ut
@@ -144,8 +149,10 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
             const float tau = 1.3862943611198906f * __log2f(P.sigma * inv_amin);   // 2 ln(sigma / alpha_min)
             const float3 a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
             const float3 b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
-            // o_g x d_g and d_g at the tile's first pixel
-            const float dx0 = (float)(x0 - P.ix) - P.rx, dy0 = (float)(y0 - P.iy) - P.ry;
+            // o_g x d_g and d_g at the pixel of the tile nearest to the reference position
+            const int xc = min(max(P.ix, x0), x0 + TS - 1), yc = min(max(P.iy, y0), y0 + TS - 1);
+            const float dx0 = (float)(xc - P.ix) - P.rx, dy0 = (float)(yc - P.iy) - P.ry;
+            const float vc = (float)(yc - y0);
             const float3 dgA = make_float3(fmaf(P.c0.x, dx0, fmaf(P.c1.x, dy0, P.dgr.x)), fmaf(P.c0.y, dx0, fmaf(P.c1.y, dy0, P.dgr.y)),
                                            fmaf(P.c0.z, dx0, fmaf(P.c1.z, dy0, P.dgr.z)));
             const float3 crA = make_float3(fmaf(a1.x, dx0, fmaf(b1.x, dy0, P.k.x)), fmaf(a1.y, dx0, fmaf(b1.y, dy0, P.k.y)),
@@ -159,12 +166,13 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
             RowQuad rq;
             rq.qA = Quu;
             rq.t1 = dot(P.m, P.c0);
+            rq.us = (float)(xc - x0);
             const bool regular = rq.qA > 0.0f && rq.t1 != 0.0f;
             const float inv_qA = fast_rcp(rq.qA), inv_t1 = fast_rcp(rq.t1);
 #pragma unroll
             for (int r = 0; r < TS; ++r) {
                 if (r < nrow) {
-                    const float v = (float)r;
+                    const float v = (float)r - vc;
                     rq.qB2 = 2.0f * fmaf(Quv, v, Qu);
                     rq.qC = fmaf(fmaf(Qvv, v, 2.0f * Qv), v, Q0);
                     rq.t0 = fmaf(t2, v, tA);
