@@ -618,15 +618,20 @@ int orc_view_lt_entries(const orc_view *v, double *entry, uint8_t *flags) {
  * alpha dL/dalpha = sum_c g_c (T alpha col_c - alpha Rs_c / (1 - alpha)), and the scale takes
  * sum_c |g_c (...)_c| in its place.  It bounds what a relative perturbation of the four
  * per-hit quantities (those three terms and T alpha) can do to a gradient word.
+ * grad_abs_terms (may be NULL) splits once more: each channel's term is itself the difference of T alpha col_c and
+ * alpha Rs_c / (1 - alpha), which nearly cancel where a hit has the colour of what lies behind it, and the scale
+ * takes the sum of the two magnitudes: the mass of the products that any evaluation of Eq. 6-8 has to form.
  * Returns 0, or -1 if the view was not composited.
  */
-int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *grad_abs, double *grad_abs_elem) {
+int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *grad_abs, double *grad_abs_elem,
+                      double *grad_abs_terms) {
     if (!v->composited) return -1;
     const int K = v->K, G = 11 + 3 * K;
     const int64_t NR = v->n_rays;
     memset(grad, 0, (size_t)v->sc.n * G * sizeof(double));
     if (grad_abs) memset(grad_abs, 0, (size_t)v->sc.n * G * sizeof(double));
     if (grad_abs_elem) memset(grad_abs_elem, 0, (size_t)v->sc.n * G * sizeof(double));
+    if (grad_abs_terms) memset(grad_abs_terms, 0, (size_t)v->sc.n * G * sizeof(double));
     double o[3];
     cam_origin(&v->cam, o);
 #pragma omp parallel for schedule(dynamic, 64)
@@ -645,11 +650,12 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
             for (int k = 0; k < K; ++k) for (int c = 0; c < 3; ++c)
                 contrib[11 + 3 * k + c] = ((v->pos[h] >> c) & 1) ? Y[k] * T * al * g[c] : 0.0;
             /* alpha */
-            double dalpha = 0.0, dalpha_abs = 0.0;
+            double dalpha = 0.0, dalpha_abs = 0.0, dalpha_terms = 0.0;
             for (int c = 0; c < 3; ++c) {
                 const double term = g[c] * (T * v->col[3 * h + c] - v->Rs[3 * h + c] / (1.0 - al));
                 dalpha += term;
                 dalpha_abs += fabs(term);
+                dalpha_terms += fabs(g[c]) * (fabs(T * v->col[3 * h + c]) + fabs(v->Rs[3 * h + c] / (1.0 - al)));
             }
             const double sigma = v->sc.opacity[i];
             const double rho = al / sigma;
@@ -685,6 +691,17 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
                     if (contrib[k] != 0.0) {
 #pragma omp atomic
                         ga[k] += fabs(contrib[k]);
+                    }
+                }
+            }
+            if (grad_abs_terms) {
+                double *gt = grad_abs_terms + (size_t)i * G;
+                const double split = dalpha != 0.0 ? dalpha_terms / fabs(dalpha) : 0.0;   /* >= 1 */
+                for (int k = 0; k < G; ++k) {
+                    if (contrib[k] != 0.0) {
+                        const double a = fabs(contrib[k]) * (k < 11 ? split : 1.0);
+#pragma omp atomic
+                        gt[k] += a;
                     }
                 }
             }

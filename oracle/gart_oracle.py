@@ -71,7 +71,7 @@ def lib():
         L.orc_view_num_hits.restype = C.c_int64
         L.orc_view_get_hits.argtypes = [C.c_void_p] + [C.c_void_p] * 4
         L.orc_view_composite.argtypes = [C.c_void_p] + [C.c_void_p] * 3
-        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 4
+        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 5
         L.orc_view_backward.restype = C.c_int
         L.orc_view_lt_entries.argtypes = [C.c_void_p] + [C.c_void_p] * 2
         L.orc_view_lt_entries.restype = C.c_int
@@ -239,19 +239,21 @@ class View:
         lib().orc_view_composite(self._h, _ptr(color), _ptr(t_final), _ptr(cnt))
         return color, t_final, cnt
 
-    def backward(self, dL_dC, with_abs=False, with_elem=False):
+    def backward(self, dL_dC, with_abs=False, with_elem=False, with_terms=False):
         """Gradients [n, 11+3K] (mean 3, scale 3, quat 4, opacity 1, sh K*3) of sum <dL_dC, C>.
         with_abs adds the sums of absolute per-hit contributions, with_elem those of the contributions
-        split by colour channel (the scale of an error that is relative to the per-hit quantities)."""
+        split by colour channel (the scale of an error that is relative to the per-hit quantities), with_terms
+        those with each channel's term split again into its two products (hit colour against colour behind)."""
         g = _f64(dL_dC).reshape(self.n_rays, 3)
         G = self.scene.grad_words
         grad = np.zeros((self.scene.n, G))
         gabs = np.zeros((self.scene.n, G)) if with_abs else None
         gelem = np.zeros((self.scene.n, G)) if with_elem else None
-        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs), _ptr(gelem))
+        gterms = np.zeros((self.scene.n, G)) if with_terms else None
+        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs), _ptr(gelem), _ptr(gterms))
         if rc != 0:
             raise RuntimeError("composite() must run before backward()")
-        out = (grad,) + ((gabs,) if with_abs else ()) + ((gelem,) if with_elem else ())
+        out = (grad,) + ((gabs,) if with_abs else ()) + ((gelem,) if with_elem else ()) + ((gterms,) if with_terms else ())
         return out if len(out) > 1 else grad
 
     def lt_entries(self):

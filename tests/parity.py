@@ -278,8 +278,9 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits)
     v2.set_hits(g_new_off, g_sel_gid)
     color, t_final, cnt = v2.composite()
-    grad, gabs, gelem = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True)
-    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "gelem": gelem, "stats": stats, "sel": sel, "view": v2}
+    grad, gabs, gelem, gterms = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True, with_terms=True)
+    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "gelem": gelem, "gterms": gterms, "stats": stats,
+            "sel": sel, "view": v2}
 
 
 def check_lt16(gpu, ref):

@@ -98,6 +98,35 @@ def test_channel_split_conditioning_bounds_the_plain_one():
         assert np.allclose(ratio, ratio[0], rtol=1e-9)
 
 
+def test_product_split_conditioning():
+    """The finest scale splits every channel's term into its two products |g| (T alpha col + alpha Rs / (1 - alpha)):
+    it bounds the channel split, equals it where nothing lies behind a hit (one composited hit per ray, black
+    background), and for the opacity word it is the sum written out from the weights and the entries."""
+    osc, cam, v, bg = _view(sh_degree=1)
+    g = gs.upstream_gradient(cam, 7).astype(np.float64)
+    grad, gabs, gelem, gterms = v.backward(g, with_abs=True, with_elem=True, with_terms=True)
+    assert np.all(gterms >= gelem * (1 - 1e-12)) and np.any(gterms[:, :11] > 1.05 * gelem[:, :11])
+    assert np.allclose(gterms[:, 11:], gabs[:, 11:], rtol=1e-12, atol=0)
+    # opacity word: sum over hits and channels of |g| (w col + (w col - entry)) / sigma, since alpha Rs / (1 - alpha) = w col - entry
+    ray_off, gid, _, _ = v.hits()
+    entry, flags = v.lt_entries()
+    rays = _rays_of_hits(v, ray_off)
+    d = np.stack([orc.ray(cam, r % cam.width, r // cam.width)[1] for r in range(v.n_rays)])
+    Y = np.stack([orc.sh_basis(x) for x in d])[:, :osc.sh.shape[1]]
+    col = np.maximum(0.5 + np.einsum("hk,hkc->hc", Y[rays], osc.sh[gid]), 0.0)
+    wcol = entry[:, 3:4] * col
+    mass = (np.abs(g.reshape(-1, 3)[rays]) * (np.abs(wcol) + np.abs(wcol - entry[:, :3]))).sum(axis=1)
+    want = np.zeros(osc.n)
+    np.add.at(want, gid, mass / osc.opacity[gid])
+    assert np.allclose(gterms[:, 10], want, rtol=1e-9, atol=1e-14)
+    # nothing behind: one composited hit per ray and a black background
+    lone = orc.View(osc, cam, bg=(0.0, 0.0, 0.0), max_hits=1)
+    lone.set_hits(ray_off, gid)
+    lone.composite()
+    _, e1, t1 = lone.backward(g, with_elem=True, with_terms=True)
+    assert np.allclose(t1, e1, rtol=1e-12, atol=0) and np.any(e1[:, :11] > 0)
+
+
 def test_half_entry_encoding_round_trip():
     rng = np.random.default_rng(0)
     H = 200_000
