@@ -181,11 +181,6 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
     const int64_t hw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;   // half-warp
     const int l = threadIdx.x & 15;
     const int64_t i0 = hw * FIN_ROWS;
-    // basis constants of this lane's four words (lanes 4..14 carry words 16..59; word 59 is padding)
-    float4 nf = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int q = 4; q < 15; ++q)
-        if (l == q) nf = make_float4(sh_word_norm(4 * q), sh_word_norm(4 * q + 1), sh_word_norm(4 * q + 2), 4 * q + 3 < 59 ? sh_word_norm(4 * q + 3) : 0.0f);
     uint32_t s[FIN_ROWS];
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r) s[r] = i0 + r < n ? __ldg(slot_of_gid + i0 + r) : 0xffffffffu;
@@ -193,6 +188,11 @@ static __global__ void __launch_bounds__(256) bwd_scatter_kernel(int64_t n, cons
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r)
         v[r] = (s[r] != 0xffffffffu && l >= 4 && l < 15) ? __ldcs(b4 + (size_t)s[r] * (GACC_B_WORDS / 4) + (l - 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    // basis constants of this lane's four words (lanes 4..14 carry words 16..59; word 59 is padding); chosen while the loads are in flight
+    float4 nf = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int q = 4; q < 15; ++q)
+        if (l == q) nf = make_float4(sh_word_norm(4 * q), sh_word_norm(4 * q + 1), sh_word_norm(4 * q + 2), 4 * q + 3 < 59 ? sh_word_norm(4 * q + 3) : 0.0f);
 #pragma unroll
     for (int r = 0; r < FIN_ROWS; ++r)
         if (i0 + r < n && (l >= 4 || s[r] == 0xffffffffu))
