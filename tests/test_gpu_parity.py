@@ -149,6 +149,27 @@ def test_random_configurations(seed):
     assert gpu["counts"][G.CNT_HITS] > 100
 
 
+@pytest.mark.parametrize("seed", [3, 11, 19, 42])
+def test_random_cameras_inside_the_cloud(seed):
+    """Harsher random scenes: scales from sub-pixel needles to screen-filling blobs, the camera inside or beside the
+    cloud (Gaussians behind it, straddling its plane, covering the image), fy != fx and an off-centre principal point."""
+    rng = np.random.default_rng(seed)
+    deg = int(rng.integers(0, 4))
+    n = int(rng.integers(50, 1500))
+    width, height = int(rng.integers(17, 120)), int(rng.integers(9, 100))
+    mean = rng.uniform(-1.0, 1.0, (n, 3))
+    scale = np.exp(rng.uniform(np.log(0.003), np.log(0.6), (n, 3)))
+    scene = gs.Scene(mean.astype(np.float32), scale.astype(np.float32), gs._unit_quats(rng, n).astype(np.float32),
+                     np.minimum(gs._sigmoid(rng.normal(0, 2.0, n)), 0.98).astype(np.float32), gs._sh(rng, n, deg), deg)
+    cam = gs.pinhole(width, height, float(rng.uniform(20.0, 100.0)), gs.look_at(rng.uniform(-1.5, 1.5, 3), rng.uniform(-0.5, 0.5, 3)))
+    cam = gs.Camera(cam.width, cam.height, cam.fx, cam.fx * float(rng.uniform(0.8, 1.25)), cam.cx + float(rng.uniform(-5, 5)),
+                    cam.cy + float(rng.uniform(-5, 5)), cam.w2c)
+    cfg = G.Config(tile_size=int(rng.choice([8, 16])), background=tuple(float(v) for v in rng.uniform(0, 1, 3)),
+                   alpha_min=float(rng.choice([1.0 / 255.0, 0.02])), max_hits=int(rng.choice([0, 0, 0, 5])))
+    gpu, ref = full_parity(scene, cam, cfg, g=gs.upstream_gradient(cam, seed))
+    assert gpu["counts"][G.CNT_HITS] > 0
+
+
 def test_stricter_alpha_min():
     """alpha_min is a parameter (the paper's 1/255 is the default): a stricter threshold drops hits on both sides alike."""
     scene, cams = gs.config_cluster(n=4000, width=120, height=96, seed=22)
