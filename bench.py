@@ -307,26 +307,34 @@ def run_ours(args):
         if i > 0:
             at.append(a0.elapsed_time(a1))
     atomic_ms = float(np.mean(at)) if at else None
-    # ---- ownership ablation: a warp per pair instead of a thread (same buffers, after the atomic runs restored the lists)
-    warp_ms = None
-    if args.warp_reps > 0:
-        if args.atomic_reps <= 0:
-            G.run_forward(cfg, g, cams[last_v], buf, stream, ray_lists=False)
-        wt = []
-        for i in range(args.warp_reps + 1):
+    # ---- the paper's decomposition (block per tile, one vector atomic update per pair) and the ownership ablation (a warp
+    # per pair instead of a thread): the forward again in the tile-major LT layout, same view
+    import dataclasses
+    cfg_t = dataclasses.replace(cfg, lt_layout=G.LT_TILE_MAJOR)
+    warp_ms, tile_ms, tile_fwd_ms = None, None, None
+
+    def timed(fn, reps):
+        ts_ = []
+        for i in range(reps + 1):                                # one untimed run first
             a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
             a0.record(stream)
-            G.run_backward_warp(cfg, g, cams[last_v], buf, dls[last_v], ga, stream)
+            fn()
             a1.record(stream)
             torch.cuda.synchronize()
             if i > 0:
-                wt.append(a0.elapsed_time(a1))
-        warp_ms = float(np.mean(wt))
+                ts_.append(a0.elapsed_time(a1))
+        return float(np.mean(ts_))
+
+    if args.tile_reps > 0 or args.warp_reps > 0:
+        tile_fwd_ms = timed(lambda: G.run_forward(cfg_t, g, cams[last_v], buf, stream, ray_lists=False), max(1, args.tile_reps))
+        if args.tile_reps > 0:
+            tile_ms = timed(lambda: G.run_backward_tile(cfg_t, g, cams[last_v], buf, dls[last_v], ga, stream), args.tile_reps)
+        if args.warp_reps > 0:
+            warp_ms = timed(lambda: G.run_backward_warp(cfg_t, g, cams[last_v], buf, dls[last_v], ga, stream), args.warp_reps)
     # ---- hybrid backward (colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric), same view
     hybrid_ms = None
     if args.hybrid_reps > 0:
-        import dataclasses
-        cfg_h = dataclasses.replace(cfg, lt_format=1)
+        cfg_h = dataclasses.replace(cfg, lt_format=1, lt_layout=G.LT_TILE_MAJOR)
         G.run_forward(cfg_h, g, cams[last_v], buf, stream, ray_lists=True)
         ht = []
         for i in range(args.hybrid_reps + 1):                    # one untimed run first
@@ -341,7 +349,6 @@ def run_ours(args):
     # ---- 8-byte LT entries (four halves per hit): forward and primitive-centric backward of the same view
     lt16_ms = None
     if args.lt16_reps > 0:
-        import dataclasses
         cfg_8 = dataclasses.replace(cfg, lt_format=2)
         ft, bt = [], []
         for i in range(args.lt16_reps + 1):                      # one untimed run first
@@ -445,6 +452,7 @@ def run_ours(args):
         "backward_hybrid_ms": hybrid_ms,
         "lt_8byte_ms": lt16_ms,
         "backward_warp_per_pair_ms": warp_ms,
+        "backward_tile_ms": tile_ms, "forward_tile_major_ms": tile_fwd_ms,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(-(-cams[0].width // cfg.tile_size), -(-cams[0].height // cfg.tile_size)) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
     }
@@ -464,6 +472,7 @@ def main():
     ap.add_argument("--slack", type=float, default=1.25)
     ap.add_argument("--atomic-reps", type=int, default=2)
     ap.add_argument("--warp-reps", type=int, default=1, help="timed runs of the warp-per-pair backward on the last view (0: skip)")
+    ap.add_argument("--tile-reps", type=int, default=2, help="timed runs of the block-per-tile backward (tile-major LT layout) on the last view (0: skip)")
     ap.add_argument("--hybrid-reps", type=int, default=1, help="timed runs of the hybrid backward on the last view (0: skip)")
     ap.add_argument("--lt16-reps", type=int, default=2, help="timed runs of forward + backward with 8-byte LT entries on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)

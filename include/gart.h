@@ -7,20 +7,30 @@
  *   gart_bounds    per-Gaussian conservative screen rectangle and ray-evaluation record
  *   gart_tile_map  (tile, Gaussian) pair list, radix-sorted by tile, and the tile offset table
  *   gart_forward   ray evaluation: hits ordered by maximum-response distance, compositing,
- *                  and the compact per-hit buffer LT = (colour behind the hit, transmittance)
- *   gart_backward  primitive-centric backward: one thread per (tile, Gaussian) pair gathers
- *                  the gradients of that Gaussian over the pair's hit pixels
+ *                  and the compact per-hit buffer LT (16 bytes per hit: alpha dC/dalpha and the
+ *                  blending weight T alpha, see gart_forward)
+ *   gart_backward  primitive-centric backward: a thread gathers the gradients of one Gaussian over
+ *                  the hit pixels of its (tile, Gaussian) pairs, with the sums in registers
+ *   gart_backward_tile     the same pass in the paper's decomposition: block per tile, thread per pair,
+ *                          one vector atomic update per pair
  *   gart_backward_atomic   the pixel-centric baseline: one thread per ray, atomicAdd per hit
- *   gart_backward_warp     gart_backward with a warp per pair (ownership ablation)
+ *   gart_backward_warp     gart_backward_tile with a warp per pair (ownership ablation)
  *   gart_backward_hybrid   colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric
  *
  * Conventions
  *   - Every array pointer is a DEVICE pointer owned by the caller unless the comment says
  *     "host".  Arrays are dense, row-major, fp32 unless the type says otherwise.
  *   - The library allocates no device memory.  Scratch comes from a caller-supplied
- *     workspace whose size is returned by the matching *_workspace_bytes query; the
- *     workspace must be 256-byte aligned and may be reused by the next call on the
- *     same stream.
+ *     workspace whose size is returned by the matching *_workspace_bytes query (or by
+ *     gart_workspace_bytes, the largest of them); the workspace must be 256-byte aligned
+ *     and may be reused by the next call on the same stream.  What gart_forward builds for
+ *     the backward passes beside LT (hit masks, work lists, the LT layout) lives in one
+ *     opaque, caller-owned "view block" of gart_view_bytes bytes, 256-byte aligned, which
+ *     must stay untouched between gart_forward and the backward pass of the same view.
+ *   - There is no context object: the configuration travels with every call as a host
+ *     struct, the per-view state is the caller's buffers, and what the device alone can
+ *     see comes back through the counts block (gart_sync_status reads it and turns its
+ *     error bits into a status).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All calls
  *     are asynchronous; none synchronises with the host.
  *   - Return value: GART_OK or an error code from argument checking / kernel launch.
@@ -49,8 +59,15 @@ typedef enum {
     GART_ERR_INVALID_ARG = 1,
     GART_ERR_WORKSPACE_TOO_SMALL = 2,
     GART_ERR_CAPACITY_EXCEEDED = 3,
-    GART_ERR_CUDA = 4
+    GART_ERR_CUDA = 4,
+    GART_ERR_TIMEOUT = 5          /* a bounded wait on an asynchronous copy inside a kernel ran out (gart_sync_status) */
 } gart_status;
+
+/* Layouts of the intermediate buffer LT (gart_config.lt_layout). */
+enum {
+    GART_LT_PRIMITIVE_MAJOR = 0,  /* hits grouped by Gaussian: what gart_backward reads */
+    GART_LT_TILE_MAJOR = 1        /* hits grouped by (tile, Gaussian) pair inside each tile: gart_backward_tile, _warp, _hybrid */
+};
 
 /* Host struct. */
 typedef struct {
@@ -64,12 +81,14 @@ typedef struct {
                              2 = the entry as four halves, 8 bytes per hit (the half-precision buffer that the
                              paper's limitations section, "VRAM Consumption", names as a way to save
                              memory); gart_backward reads this format too */
-    int32_t max_hits;     /* 0: every hit of a ray is composited (the paper's setting: "no maximum ray intersection
-                             cap").  m > 0: gart_forward composites only the first m hits of a ray in (t*, id)
+    int32_t max_hits;     /* 0: every hit of a ray is composited (the paper's benchmark sets no hit cap, Sec. 5).
+                             m > 0: gart_forward composites only the first m hits of a ray in (t*, id)
                              order, the cap that the paper lists among the compromises of 3DGRT.  The hits behind
                              the cap keep their place in every list and their LT slot, with a zero entry: they
                              add nothing to the colour, to T_final or to a gradient (the backward passes that
                              read lt need no change; gart_backward_hybrid rejects a cap) */
+    int32_t lt_layout;    /* GART_LT_PRIMITIVE_MAJOR (0, for gart_backward) or GART_LT_TILE_MAJOR (the ablation passes):
+                             where gart_forward puts a hit's entry in lt.  The entries' contents are the same. */
 } gart_config;
 
 /* Host struct. */
@@ -121,17 +140,18 @@ int32_t gart_mask_words(int32_t tile_size);
  * double precision, and the pre-computations of the ray evaluation (W = S^-1 R^T and o_g of
  * Eq. 5, expressed relative to a per-Gaussian reference pixel so that fp32 evaluation stays
  * well conditioned).  Gaussians with a non-empty rectangle are renumbered for the view: a stable
- * sort on the tile row of the rectangle's corner (y0 / tile_size) gives each a slot 0..V-1
- * (V = counts[VISIBLE]); later steps read and update per-Gaussian data by slot, so that what a row of
- * tiles touches is a few MB that stay in L2 (the scene's own order carries no such locality).
+ * sort on the 16 x 16-pixel super-tile of the rectangle's corner ((y0 / 16) * ceil(width / 16) + x0 / 16) gives
+ * each a slot 0..V-1 (V = counts[VISIBLE]); later steps read per-Gaussian data by slot, so that what
+ * neighbouring tiles touch is neighbouring memory (the scene's own order carries no such locality), and the
+ * Gaussians that a super-tile owns in the backward pass are one run of slots.
  *   rect   [n,4] int32 out: inclusive pixel range x0,y0,x1,y1 of pixel centres inside the
  *                bound, clipped to the image; (0,0,-1,-1) if empty.
  *   cls    [n]   uint8 out: 0 culled (sigma <= alpha_min, or support entirely at depth <= near_z),
  *                1 in front of the near plane, 2 straddling it (rectangle = whole image unless
  *                the bounding sphere is outside a side plane of the frustum).
  *   pre    [n * gart_pre_words(sh_degree)] fp32 out: per slot, the evaluation record followed by a copy
- *                of its SH coefficients (times the basis constants), and behind all records quaternion, scale
- *                and opacity in slot order; contents are private to the library.
+ *                of its SH coefficients (times the basis constants), and behind all records quaternion, scale,
+ *                opacity and the rectangle in slot order; contents are private to the library.
  *   slot_of_gid [n] uint32 out: slot of every Gaussian, 0xffffffff if it has none.
  *   gid_of_slot [n] uint32 out: the inverse (first V entries; 0xffffffff beyond).
  *   counts [GART_COUNTS_WORDS] uint32 out: zeroed, then VISIBLE and STRADDLE are set.
@@ -181,30 +201,41 @@ gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, in
                                  void *stream);
 
 /*
+ * The view block: private arrays that gart_forward builds and the backward passes read (per pair the hit mask and
+ * its rank in the tile; per Gaussian the work items of the primitive-major order; the LT layout of both orders).
+ * Opaque to the caller, who owns the memory: `view` is a device buffer of at least gart_view_bytes bytes, 256-byte
+ * aligned.  n, image size, tile size and cap_pairs must be the same in the query, in gart_forward and in the backward
+ * pass.  gart_view_array returns offset and size of one named array inside the block (for tests and diagnostics;
+ * the names are not a stable interface).
+ */
+size_t gart_view_bytes(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs);
+enum {
+    GART_VIEW_PAIR_MASK = 0,    /* [cap_pairs, gart_mask_words] bit p of pair j: pixel p = ly * tile_size + lx of its tile is hit */
+    GART_VIEW_PAIR_ORDER = 1,   /* [cap_pairs] per tile, the pairs by descending hit count (stable) */
+    GART_VIEW_RANK_SID = 2,     /* [cap_pairs] slot of the Gaussian, in rank order */
+    GART_VIEW_RANK_MASK = 3,    /* [cap_pairs, gart_mask_words] hit mask, in rank order */
+    GART_VIEW_RANK_GSTART = 4,  /* [cap_pairs] tile-major LT layout: start of the pair's 32-rank group inside its tile */
+    GART_VIEW_TILE_LT_BASE = 5, /* [T+1] tile-major LT layout: first entry of every tile */
+    GART_VIEW_PAIR_GPOS = 6,    /* [cap_pairs] position of the pair in the primitive-major order */
+    GART_VIEW_GPAIR_OFF = 7,    /* [n+1] first primitive-major position of every slot (the slot's tiles follow row by row) */
+    GART_VIEW_GM_MASK = 8,      /* [cap_pairs, gart_mask_words] hit masks in primitive-major order */
+    GART_VIEW_GM_LTB = 9,       /* [cap_pairs] primitive-major LT layout: entry of the first hit of every pair, by primitive-major position */
+    GART_VIEW_ITEM_DESC = 10,   /* [cap_pairs, 4] work items per super-tile in rank order: slot, first pair, dimensions, hits | whole-flag << 16 */
+    GART_VIEW_ITEM_GSTART = 11, /* [cap_pairs] LT entry where the item's 32-rank group starts */
+    GART_VIEW_ST_OFF = 12,      /* [NS+1] first item of every super-tile, NS = ceil(width / 16) * ceil(height / 16) */
+    GART_VIEW_ST_LT_BASE = 13,  /* [NS+1] first LT entry of every super-tile */
+    GART_VIEW_INFO = 14         /* [64] word 0: items, word 1: blocks of the backward pass */
+};
+gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int32_t which,
+                            size_t *offset, size_t *bytes);
+
+/*
  * Step 3 -- forward ray evaluation (Sec. 3.2-3.3, Eq. 3-8; intermediate buffer of Sec. 4.2-4.3).
  * For every pixel ray and every Gaussian of its tile list: t* = -(o_g.d_g)/(d_g.d_g),
  * alpha = sigma exp(-|o_g + t* d_g|^2 / 2); a hit iff alpha >= alpha_min and t* > 0.  Hits of a
  * ray are ordered by (t*, id) and composited front to back, C = sum T_i alpha_i c_i + T_final bg,
  * c_i = max(0, 0.5 + sum_k Y_k(d) sh_ik).
  *   color      [H,W,3] out;  t_final [H,W] out;  hit_count [H,W] uint32 out.
- *   pair_mask  [cap_pairs, gart_mask_words] uint32 out: bit p of pair j = pixel p of the tile
- *              (p = ly * tile_size + lx) is hit by the pair's Gaussian.
- *   pair_order [cap_pairs] uint32 out: for tile t, pair_order[tile_off[t] + r] is the pair of rank r
- *              when the tile's pairs are ordered by descending hit count (stable); the backward
- *              gives lane l of a warp the pair of rank 32 g + l, so a warp's lanes have (nearly)
- *              the same number of hits.
- *   rank_sid   [cap_pairs] uint32 out, rank_mask [cap_pairs, gart_mask_words] uint32 out: slot of the
- *              Gaussian and hit mask of the pair at each rank position (slot_of_gid[pair_gid[.]] and
- *              pair_mask[.] in rank order, so that later kernels read them coalesced and without
- *              indirection).
- *   rank_gstart[cap_pairs] uint32 out, tile_lt_base [T+1] uint32 out: the e-th hit (in pixel order)
- *              of the pair of rank r of tile t lives at
- *                  lt[tile_lt_base[t] + rank_gstart[tile_off[t] + r] + 32 e + (r mod 32)].
- *              rank_gstart is the same for the 32 ranks of a group: the group's pairs are interleaved
- *              entry by entry, so the group's e-th entries are 32 consecutive 16-byte words, the
- *              group's whole block is one contiguous range (one bulk copy), every hit owns one slot
- *              (forward writes never collide), and a group occupies 32 x (its largest hit count)
- *              entries: L = tile_lt_base[T] >= H counts the padding.
  *   lt         [cap_hits,4] out: per hit, with w = T alpha its blending weight (T the transmittance
  *              in front of it), c its clamped colour and B the colour composited BEHIND it
  *              (background term included): words 0..2 = w c - alpha / (1 - alpha) B, which is
@@ -216,52 +247,82 @@ gart_status gart_tile_map_static(const gart_config *cfg, const int32_t *rect, in
  *              ties to even) with the half's lowest bit replaced by the flag of channel ch, h3 = the half
  *              nearest to 4096 w.  A decoded colour word is within 2^-10 (relative) of the fp32 value, the
  *              weight within 2^-11; magnitudes below 2^-26 lose relative precision, below 2^-37 vanish.
+ *              Where a hit's entry lives: every hit owns one slot (forward writes never collide).  Both layouts
+ *              rank work units by descending hit count and interleave the entries of 32 consecutive ranks
+ *              (entry e of rank r of a group at group start + 32 e + r mod 32), so that a warp of the backward
+ *              reads its lanes' e-th entries as one 512-byte row and a group's block is one contiguous range;
+ *              a group occupies 32 x (its largest hit count) entries, L >= H counts that padding.
+ *              GART_LT_TILE_MAJOR: the unit is a (tile, Gaussian) pair, groups are formed inside each tile.
+ *              GART_LT_PRIMITIVE_MAJOR: the unit is a work item -- a Gaussian whose rectangle spans at most two
+ *              16 x 16-pixel super-tiles per axis, else the part of a Gaussian inside one super-tile; its entries are
+ *              those of its (tile, Gaussian) pairs in turn (tiles row by row, pixels in mask order); groups are
+ *              formed among the items owned by one super-tile.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
  *              baseline and parity checks read the two lists: pass NULL for both to skip them.
+ *   view       the view block (above), out.
  *   counts: HITS, LT_SLOTS, MAX_RAY_HITS.  If L > cap_hits, GART_ERRBIT_HITS is set and color,
- *   t_final, lt, ray_gid, ray_slot are not written.  Because ranks descend in hit count,
- *   L <= H + 32 tile_size^2 per non-empty tile, and H <= S (the slot bound of gart_tile_map), so
- *   cap_hits = S + 32 tile_size^2 T always suffices; the exact need is L.
+ *   t_final, lt, ray_gid, ray_slot are not written.  Because ranks descend in hit count, a tile (super-tile) pads
+ *   by less than 32 x its largest count, and H <= S (the slot bound of gart_tile_map), so
+ *   cap_hits = S + 32 tile_size^2 T (tile-major) or S + 32 * 1024 * NS (primitive-major) always suffices; the
+ *   exact need is L.
+ * Errors: INVALID_ARG also for an image wider or higher than 524280 pixels, and for lt_format 1 with the
+ * primitive-major layout (the 4-byte format serves the hybrid pass, which is tile-major).
  */
 size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
 gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                          const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off, const uint32_t *pair_gid, int64_t cap_pairs,
                          float *color, float *t_final, uint32_t *hit_count,
-                         uint32_t *pair_mask, uint32_t *pair_order, uint32_t *rank_sid, uint32_t *rank_mask,
-                         uint32_t *rank_gstart, uint32_t *tile_lt_base, float *lt, int64_t cap_hits,
-                         uint32_t *ray_off, uint32_t *ray_gid, uint32_t *ray_slot, uint32_t *counts,
+                         float *lt, int64_t cap_hits,
+                         uint32_t *ray_off, uint32_t *ray_gid, uint32_t *ray_slot,
+                         void *view, size_t view_bytes, uint32_t *counts,
                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * Step 4 -- primitive-centric backward (Sec. 4.4): one thread block per tile, one thread per
- * (tile, Gaussian) pair; the thread walks the pair's hit pixels, reads their LT entries (coalesced
- * across the warp thanks to the interleaved layout), accumulates in registers and performs one vector
- * atomic update per pair of the accumulation record of the Gaussian's slot.  No per-pixel atomics.
- * A per-Gaussian pass then converts the accumulated moments and writes the gradient records.
+ * Step 4 -- primitive-centric backward (Sec. 4.4).  A thread gathers the gradient sums of ONE work item of the
+ * primitive-major order: it walks the item's (tile, Gaussian) pairs one after the other and, per pair, the pair's hit
+ * pixels, reads their LT entries (coalesced across the warp thanks to the interleaved layout) and accumulates in
+ * registers.  No per-pixel atomics.  An item that is a whole Gaussian (its rectangle fits a 32 x 32-pixel window: nearly
+ * all of them) ends with the conversion of the moments and ONE write of the 256-byte gradient record -- no atomic, no
+ * accumulation record; the pieces of larger Gaussians add to an accumulation record with one vector atomic per 16 bytes
+ * and piece, converted by a small per-slot pass.  Needs gart_forward run with lt_layout = GART_LT_PRIMITIVE_MAJOR.
  *   dL_dcolor [H,W,3] in.
  *   grad [n,GART_GRAD_WORDS] out, fully overwritten: d mean, d scale, d quat, d opacity, d sh
  *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
+ *   view, cap_pairs: the view block that gart_forward filled and the capacity it was laid out for.
  *   counts: read (a set error bit skips the work); GART_ERRBIT_TIMEOUT is set if a wait on an
  *        asynchronous copy ran out, in which case grad is incomplete.
  * cfg->lt_format must be the one the forward wrote lt with, 0 or 2 (INVALID_ARG otherwise).  With 8-byte
  * entries every gradient word, being linear in the four words of its hits' entries, moves by at most 2^-10
  * of the sum of the absolute per-hit, per-channel terms of that word.
- * The main kernel uses up to 99 KB of dynamic shared memory per block (opt-in set by the call): LT blocks
- * and the Gaussians' records are streamed in with bulk asynchronous copies, one rank group ahead.
+ * The main kernel uses 44 KB of dynamic shared memory per block: LT blocks are streamed in with bulk
+ * asynchronous copies, one rank group ahead, beside dL/dC of the block's 32 x 32-pixel window.
  */
 size_t gart_backward_workspace_bytes(int64_t n);
 gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                           const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
-                          const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
-                          const uint32_t *tile_lt_base,
+                          const void *view, size_t view_bytes, int64_t cap_pairs,
                           const float *lt, const float *dL_dcolor,
                           float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same pass in the decomposition that Sec. 4.4 describes: one thread block per tile, one thread per
+ * (tile, Gaussian) pair; the thread walks the pair's hit pixels, accumulates in registers and performs one vector
+ * atomic update per pair of the accumulation record of the Gaussian's slot; a per-Gaussian pass then converts the
+ * accumulated moments and writes the gradient records.  Needs lt_layout = GART_LT_TILE_MAJOR.  Arguments, result
+ * (up to summation order) and errors as gart_backward.  38 KB of dynamic shared memory per block.
+ */
+gart_status gart_backward_tile(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
+                               const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
+                               const void *view, size_t view_bytes, int64_t cap_pairs,
+                               const float *lt, const float *dL_dcolor,
+                               float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Pixel-centric baseline (Sec. 3.5): one thread per ray walks the ray's hits and issues one
  * atomicAdd per gradient word per hit (11 + 3K; 59 at degree 3).  Same result as gart_backward
- * up to summation order.
+ * up to summation order.  Reads 16-byte LT entries through ray_slot, so either layout serves; needs the
+ * per-ray lists of gart_forward (INVALID_ARG if they are NULL).
  */
 gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,
                                  const float *pre, const uint32_t *slot_of_gid, const uint32_t *ray_off, const uint32_t *ray_gid,
@@ -269,34 +330,40 @@ gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g
                                  float *grad, const uint32_t *counts, void *stream);
 
 /*
- * Ownership ablation (Sec. 4.4): gart_backward with one warp, not one thread, per (tile, Gaussian) pair.  Same
- * arguments, same result up to summation order; the paper found it less efficient and so it is here.
+ * Ownership ablation (Sec. 4.4): gart_backward_tile with one warp, not one thread, per (tile, Gaussian) pair.  Same
+ * arguments, same result up to summation order; Sec. 4.4 reports it as slower, and so it is here.  16-byte entries only.
  */
 gart_status gart_backward_warp(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                                const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
-                               const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
-                               const uint32_t *tile_lt_base,
+                               const void *view, size_t view_bytes, int64_t cap_pairs,
                                const float *lt, const float *dL_dcolor,
                                float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Hybrid backward (Sec. 4.4 "Hybrid approach"; "Hybrid" of Sec. 5.1): the colour gradients dL/dsh are accumulated
- * primitive-centric from an intermediate buffer of ONE word per hit, the remaining terms (mean, scale,
- * quaternion, opacity) pixel-centric with 10 scalar atomicAdd per hit.  Needs gart_forward run with
- * cfg->lt_format = 1 (lt_w [cap_hits] fp32: word 3 of the full entry, same slot layout) and with the per-ray id
+ * primitive-centric (block per tile) from an intermediate buffer of ONE word per hit, the remaining terms (mean, scale,
+ * quaternion, opacity) pixel-centric with three vector atomics per hit.  Needs gart_forward run with
+ * cfg->lt_format = 1, lt_layout = GART_LT_TILE_MAJOR (lt_w [cap_hits] fp32: word 3 of the full entry) and with the per-ray id
  * list (ray_off, ray_gid); the 4 + 4 bytes per hit replace the 16 of the full entry (the paper, which re-traces
  * the ray in its pixel-centric part, keeps 4).  Same result as gart_backward up to rounding and summation order;
  * same workspace as gart_backward.  Errors as gart_backward; INVALID_ARG if cfg->lt_format != 1.
  */
 gart_status gart_backward_hybrid(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                                  const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
-                                 const uint32_t *rank_sid, const uint32_t *rank_mask, const uint32_t *rank_gstart,
-                                 const uint32_t *tile_lt_base, const float *lt_w, const uint32_t *ray_off, const uint32_t *ray_gid,
+                                 const void *view, size_t view_bytes, int64_t cap_pairs,
+                                 const float *lt_w, const uint32_t *ray_off, const uint32_t *ray_gid,
                                  const float *dL_dcolor, float *grad, uint32_t *counts, void *workspace, size_t workspace_bytes,
                                  void *stream);
 
+/* The largest of the four per-step workspace needs (bounds, tile map, forward, backward): one buffer serves a whole view. */
+size_t gart_workspace_bytes(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
+
 /* Copy the counts block to host memory (synchronises the stream). counts_host: host, GART_COUNTS_WORDS words. */
 gart_status gart_read_counts(const uint32_t *counts, uint32_t *counts_host, void *stream);
+
+/* gart_read_counts, then the block's error word as a status: GART_ERR_CAPACITY_EXCEEDED (pair or hit capacity),
+ * GART_ERR_TIMEOUT (a bounded wait inside a kernel ran out), else GART_OK.  counts_host may be NULL. */
+gart_status gart_sync_status(const uint32_t *counts, uint32_t *counts_host, void *stream);
 
 /*
  * End-to-end convenience for callers holding HOST arrays: uploads the scene and dL_dcolor,

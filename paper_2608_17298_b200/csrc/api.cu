@@ -8,9 +8,9 @@ struct HostArena {
     float *mean, *scale, *quat, *opacity, *sh, *pre, *color, *t_final, *lt, *dL_dC, *grad;
     int32_t* rect;
     uint8_t* cls;
-    uint32_t *counts, *tile_off, *pair_gid, *pair_mask, *pair_order, *rank_sid, *rank_mask, *rank_gstart, *tile_lt_base, *slot_of_gid, *gid_of_slot, *hit_count, *ray_off;
-    void* ws;
-    size_t ws_bytes;
+    uint32_t *counts, *tile_off, *pair_gid, *slot_of_gid, *gid_of_slot, *hit_count, *ray_off;
+    void *view, *ws;
+    size_t view_bytes, ws_bytes;
     size_t bytes;
 };
 
@@ -22,27 +22,18 @@ static HostArena arena_layout(void* base, int64_t n, int K, int width, int heigh
     const int64_t nn = n > 0 ? n : 1, cp = cap_pairs > 0 ? cap_pairs : 1, ch = cap_hits > 0 ? cap_hits : 1;
     const int64_t hw = (int64_t)width * height;
     const int T = ((width + ts - 1) / ts) * ((height + ts - 1) / ts);
-    const int mw = ts * ts / 32;
     a.mean = (float*)take(nn * 12); a.scale = (float*)take(nn * 12); a.quat = (float*)take(nn * 16);
     a.opacity = (float*)take(nn * 4); a.sh = (float*)take(nn * 12 * K);
-    a.rect = (int32_t*)take(nn * 16); a.cls = (uint8_t*)take(nn); a.pre = (float*)take(nn * 4 * (size_t)(((20 + 3 * K + 3) & ~3) + 8));
+    a.rect = (int32_t*)take(nn * 16); a.cls = (uint8_t*)take(nn); a.pre = (float*)take(nn * 4 * (size_t)(((20 + 3 * K + 3) & ~3) + 8 + 4));
     a.slot_of_gid = (uint32_t*)take(nn * 4); a.gid_of_slot = (uint32_t*)take(nn * 4);
     a.counts = (uint32_t*)take(GART_COUNTS_WORDS * 4);
     a.tile_off = (uint32_t*)take((size_t)(T + 1) * 4); a.pair_gid = (uint32_t*)take(cp * 4);
-    a.pair_mask = (uint32_t*)take(cp * 4 * mw); a.pair_order = (uint32_t*)take(cp * 4); a.rank_sid = (uint32_t*)take(cp * 4);
-    a.rank_mask = (uint32_t*)take(cp * 4 * mw); a.rank_gstart = (uint32_t*)take(cp * 4);
-    a.tile_lt_base = (uint32_t*)take((size_t)(T + 1) * 4);
+    a.view_bytes = gart_view_bytes(nn, width, height, ts, cap_pairs);
+    a.view = take(a.view_bytes);
     a.color = (float*)take(hw * 12); a.t_final = (float*)take(hw * 4); a.hit_count = (uint32_t*)take(hw * 4);
     a.lt = (float*)take(ch * 16); a.ray_off = (uint32_t*)take((hw + 1) * 4);
     a.dL_dC = (float*)take(hw * 12); a.grad = (float*)take(nn * GART_GRAD_WORDS * 4);
-    const size_t w0 = gart_bounds_workspace_bytes(nn);
-    const size_t w1 = gart_tile_map_workspace_bytes(nn, width, height, ts, cap_pairs);
-    const size_t w2 = gart_forward_workspace_bytes(width, height, ts, cap_pairs, cap_hits);
-    const size_t w3 = gart_backward_workspace_bytes(nn);
-    a.ws_bytes = w0;
-    if (w1 > a.ws_bytes) a.ws_bytes = w1;
-    if (w2 > a.ws_bytes) a.ws_bytes = w2;
-    if (w3 > a.ws_bytes) a.ws_bytes = w3;
+    a.ws_bytes = gart_workspace_bytes(nn, width, height, ts, cap_pairs, cap_hits);
     a.ws = take(a.ws_bytes);
     a.bytes = off;
     return a;
@@ -57,6 +48,28 @@ extern "C" gart_status gart_read_counts(const uint32_t* counts, uint32_t* counts
         return GART_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return GART_ERR_CUDA;
     return GART_OK;
+}
+
+extern "C" gart_status gart_sync_status(const uint32_t* counts, uint32_t* counts_host, void* stream) {
+    uint32_t local[GART_COUNTS_WORDS];
+    uint32_t* h = counts_host ? counts_host : local;
+    const gart_status s = gart_read_counts(counts, h, stream);
+    if (s != GART_OK) return s;
+    if (h[GART_CNT_ERROR] & GART_ERRBIT_TIMEOUT) return GART_ERR_TIMEOUT;
+    if (h[GART_CNT_ERROR]) return GART_ERR_CAPACITY_EXCEEDED;
+    return GART_OK;
+}
+
+extern "C" size_t gart_workspace_bytes(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits) {
+    const int64_t nn = n > 0 ? n : 1;
+    size_t b = gart_bounds_workspace_bytes(nn);
+    const size_t w1 = gart_tile_map_workspace_bytes(nn, width, height, tile_size, cap_pairs);
+    const size_t w2 = gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits);
+    const size_t w3 = gart_backward_workspace_bytes(nn);
+    if (w1 > b) b = w1;
+    if (w2 > b) b = w2;
+    if (w3 > b) b = w3;
+    return b;
 }
 
 extern "C" size_t gart_view_host_arena_bytes(int64_t n, int32_t sh_degree, int32_t width, int32_t height, int32_t tile_size,
@@ -97,17 +110,22 @@ extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussia
     if (s != GART_OK) return s;
     s = gart_tile_map(cfg, a.rect, n, cam->width, cam->height, a.tile_off, a.pair_gid, cap_pairs, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
-    s = gart_forward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count, a.pair_mask,
-                     a.pair_order, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, cap_hits, a.ray_off, nullptr, nullptr, a.counts, a.ws, a.ws_bytes, stream);
+    s = gart_forward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.pair_gid, cap_pairs, a.color, a.t_final, a.hit_count,
+                     a.lt, cap_hits, a.ray_off, nullptr, nullptr, a.view, a.view_bytes, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
-    s = gart_backward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.rank_sid, a.rank_mask, a.rank_gstart, a.tile_lt_base, a.lt, a.dL_dC,
-                      a.grad, a.counts, a.ws, a.ws_bytes, stream);
+    if (cfg->lt_layout == GART_LT_TILE_MAJOR)
+        s = gart_backward_tile(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.view, a.view_bytes, cap_pairs, a.lt, a.dL_dC,
+                               a.grad, a.counts, a.ws, a.ws_bytes, stream);
+    else
+        s = gart_backward(cfg, &gd, cam, a.pre, a.slot_of_gid, a.gid_of_slot, a.tile_off, a.view, a.view_bytes, cap_pairs, a.lt, a.dL_dC,
+                          a.grad, a.counts, a.ws, a.ws_bytes, stream);
     if (s != GART_OK) return s;
     if (cudaMemcpyAsync(color_host, a.color, (size_t)hw * 12, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GART_ERR_CUDA;
     if (n > 0 && cudaMemcpyAsync(grad_host, a.grad, (size_t)n * GART_GRAD_WORDS * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return GART_ERR_CUDA;
     s = gart_read_counts(a.counts, counts_host, stream);
     if (s != GART_OK) return s;
+    if (counts_host[GART_CNT_ERROR] & GART_ERRBIT_TIMEOUT) return GART_ERR_TIMEOUT;
     if (counts_host[GART_CNT_ERROR]) return GART_ERR_CAPACITY_EXCEEDED;
     return GART_OK;
 }

@@ -1,4 +1,4 @@
-// gart_backward: primitive-centric backward (Sec. 4.4).
+// gart_backward_tile: primitive-centric backward in the paper's own decomposition (Sec. 4.4): block per tile.
 //
 // One thread block per tile, one thread per (tile, Gaussian) pair.  Lane l of a warp owns the pair
 // of rank 32 g + l in the tile's hit-count order, so the lanes of a warp run (nearly) the same
@@ -15,6 +15,7 @@
 // neighbouring memory.  A per-Gaussian pass then converts the moments into d mean, d scale, d quat,
 // d opacity and writes the caller's gradient records.
 #include "backward_common.cuh"
+#include "view_layout.cuh"
 
 namespace gart {
 
@@ -319,23 +320,41 @@ static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* r
 
 extern "C" size_t gart_backward_workspace_bytes(int64_t n) { return gart::gacc_bytes(n > 0 ? n : 1); }
 
-extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
-                                     const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
-                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
-                                     const float* lt, const float* dL_dcolor,
-                                     float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
-    using namespace gart;
-    if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
+// Argument checks shared by the tile-major passes; on success `v` holds the arrays of the view block.
+static gart_status tile_pass_args(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
+                                  const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                                  const void* view, size_t view_bytes, int64_t cap_pairs, const float* lt, const float* dL_dcolor,
+                                  const float* grad, const uint32_t* counts, const void* workspace, size_t workspace_bytes,
+                                  gart::ViewLayout* v) {
+    if (!cfg || !g || !cam || !counts || !tile_off || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 0 && cfg->lt_format != 2) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte or 8-byte LT entries
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // these passes read LT in the tile-major layout
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
+    if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
+    if (!grad || !pre || !slot_of_gid || !gid_of_slot || !lt || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    *v = gart::view_layout(const_cast<void*>(view), g->n, cam->width, cam->height, cfg->tile_size, cap_pairs);
+    if (v->bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    return GART_OK;
+}
+
+extern "C" gart_status gart_backward_tile(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
+                                          const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                                          const void* view, size_t view_bytes, int64_t cap_pairs,
+                                          const float* lt, const float* dL_dcolor,
+                                          float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace gart;
+    ViewLayout v;
+    gart_status s = tile_pass_args(cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, view_bytes, cap_pairs, lt, dL_dcolor, grad, counts,
+                                   workspace, workspace_bytes, &v);
+    if (s != GART_OK || g->n == 0) return s;
+    if (cfg->lt_format != 0 && cfg->lt_format != 2) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte or 8-byte LT entries
+    const uint32_t *rank_sid = v.rank_sid, *rank_mask = v.rank_mask, *rank_gstart = v.rank_gstart, *tile_lt_base = v.tile_lt_base;
     cudaStream_t st = (cudaStream_t)stream;
     const Gacc gacc = make_gacc(workspace, g->n);
-    gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
+    s = launch_zero_accumulators(gacc, g->n, counts, st);
     if (s != GART_OK) return s;
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int T = cf.tiles_x * cf.tiles_y;
@@ -351,7 +370,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Ownership ablation (Sec. 4.4: "assigning a full warp is possible, we found it less efficient"): the same
+// Ownership ablation (Sec. 4.4 reports warp-per-pair ownership as possible but slower): the same
 // gradient with one WARP per (tile, Gaussian) pair.  Lane e takes the pair's e-th (and e+32nd ...) hit, the 11 + 3K
 // terms are summed over the warp with shuffles, and lanes 0..14 flush one 16-byte piece each.  Reads the LT
 // buffer in the layout made for thread ownership (a pair's entries lie 512 bytes apart).
@@ -463,21 +482,19 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
 
 extern "C" gart_status gart_backward_warp(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                           const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
-                                          const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart, const uint32_t* tile_lt_base,
+                                          const void* view, size_t view_bytes, int64_t cap_pairs,
                                           const float* lt, const float* dL_dcolor,
                                           float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace gart;
-    if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor) return GART_ERR_INVALID_ARG;
-    if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
+    ViewLayout v;
+    gart_status s = tile_pass_args(cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, view_bytes, cap_pairs, lt, dL_dcolor, grad, counts,
+                                   workspace, workspace_bytes, &v);
+    if (s != GART_OK || g->n == 0) return s;
     if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
-    if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
-    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
-    if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    const uint32_t *rank_sid = v.rank_sid, *rank_mask = v.rank_mask, *rank_gstart = v.rank_gstart, *tile_lt_base = v.tile_lt_base;
     cudaStream_t st = (cudaStream_t)stream;
     const Gacc gacc = make_gacc(workspace, g->n);
-    gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);
+    s = launch_zero_accumulators(gacc, g->n, counts, st);
     if (s != GART_OK) return s;
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int T = cf.tiles_x * cf.tiles_y;

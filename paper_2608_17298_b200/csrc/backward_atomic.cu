@@ -65,7 +65,8 @@ extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_g
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !slot_of_gid || !g->scale || !g->quat || !g->opacity) return GART_ERR_INVALID_ARG;
+    if (!grad || !pre || !slot_of_gid || !g->scale || !g->quat || !g->opacity || !ray_gid || !ray_slot || !lt) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;   // reads 16-byte LT entries (either layout: the slot of every hit comes from ray_slot)
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(grad, 0, (size_t)g->n * GART_GRAD_WORDS * sizeof(float), st) != cudaSuccess) return GART_ERR_CUDA;
     const CamF cf = make_camf(cam, cfg->tile_size);

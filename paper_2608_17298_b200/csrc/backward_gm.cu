@@ -1,0 +1,478 @@
+// gart_backward: primitive-centric backward (Sec. 4.4) over the primitive-major work lists.
+//
+// The paper gives a thread one (tile, Gaussian) pair and lets it add its sums to the Gaussian's gradient with one
+// atomic update per pair.  On this GPU the arithmetic of a hit and the bytes of its LT entry are in balance, and what
+// then costs most is exactly those updates: a Gaussian covers 3.6 tiles on average, so its 240-byte record is
+// read, modified and written back several times, by blocks that run tens of microseconds apart (more than the
+// L2 holds), and must be zeroed before and converted after.  Here a thread still gathers (tile, Gaussian) pairs, but
+// it walks ALL pairs of one work item -- a whole Gaussian whenever its rectangle fits a 32 x 32-pixel window, else the
+// part of a large Gaussian inside one 16 x 16 super-tile -- one after the other with the sums in registers.  A whole
+// Gaussian (96 % of them at the benchmark's scale) then needs no atomic and no accumulation record: its thread converts
+// the moments and writes the final 256-byte gradient record once.  Only the pieces of large Gaussians use vector
+// atomics on an accumulation record (one per piece), converted by a small per-slot pass.
+//
+// A block serves up to GM_GROUPS_PER_BLOCK rank groups of one super-tile: it stages dL/dC of the super-tile's window in
+// shared memory (one copy: 16 KB), its warps take the groups in serpentine order, lanes own items of (nearly) equal hit
+// count, and the group's interleaved LT block streams in through bulk asynchronous copies (cp.async.bulk + mbarrier,
+// double buffered, every wait bounded).  The ray direction is affine in the pixel position before normalisation, so a
+// hit recomputes it (12 instructions) instead of loading it: with lanes reading different pixels of a 1024-pixel window,
+// shared-memory loads conflict, and the direction would double them.
+#include "backward_common.cuh"
+#include "view_layout.cuh"
+
+namespace gart {
+
+constexpr int GMB_WARPS = 4;
+constexpr int GMB_THREADS = GMB_WARPS * 32;
+constexpr int GMB_CHUNK = 7;                           // LT entries per lane and per pipeline stage (16-byte entries)
+constexpr int GMB_STAGE_F4 = GMB_CHUNK * 32;           // float4 per stage
+constexpr int GMB_STAGES = 2;
+constexpr int GMB_LT_SMEM = GMB_WARPS * GMB_STAGES * GMB_STAGE_F4 * 16;
+constexpr int GMB_PIX = GM_WIN * GM_WIN;
+constexpr int GMB_DYN_SMEM = GMB_LT_SMEM + GMB_PIX * 16;
+static_assert(GM_GROUPS_PER_BLOCK % GMB_WARPS == 0, "groups are dealt to the warps in rounds");
+
+__device__ __forceinline__ float fast_rsqrt(float x) {
+    float y;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// float of a small non-negative integer without the conversion unit
+__device__ __forceinline__ float small_int_to_float(uint32_t v) { return __uint_as_float(0x4B000000u | v) - 8388608.0f; }
+
+// What a lane knows of its item of a rank group.
+struct GmItem {
+    uint4 d;           // descriptor (view_layout.cuh)
+    uint32_t gstart;   // LT index of the group's block
+    int c;             // hits of this lane's item (0 for a lane without item)
+    int cmax;          // hits of the group's first item = the largest of the group
+    bool valid;        // the lane has an item
+};
+
+__device__ __forceinline__ GmItem gm_load_item(const uint4* __restrict__ rk_desc, const uint32_t* __restrict__ rk_gstart,
+                                               uint32_t begin, uint32_t n, uint32_t r0, bool in_part, int lane) {
+    GmItem g;
+    g.valid = in_part && r0 + lane < n;
+    g.d = g.valid ? __ldg(rk_desc + begin + r0 + lane) : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t gs = g.valid ? __ldg(rk_gstart + begin + r0 + lane) : 0u;
+    g.c = (int)(g.d.w & 0xffffu);
+    g.cmax = __shfl_sync(0xffffffffu, g.c, 0);
+    g.gstart = __shfl_sync(0xffffffffu, gs, 0);
+    return g;
+}
+
+// The item's geometry, affine in the window position (xf, yf): d_g = dgC + (xf - uc) c0 + (yf - vc) c1 and
+// o_g x d_g = crC + (xf - uc) a1 + (yf - vc) b1, expanded about the pixel of the item's extent nearest to the Gaussian's
+// reference position (o_g x d_g vanishes at the centre: about a far corner a small Gaussian's hits would be
+// differences of much larger numbers).
+struct ItemGeo {
+    float3 c0, c1, dgC, a1, b1, crC;
+    float uc, vc;
+};
+
+template <int TS>
+__device__ __forceinline__ ItemGeo item_geo(const PreRec& P, const uint4 d, int wx0, int wy0) {
+    ItemGeo g;
+    const int ntx = (d.z >> 16) & 15, nty = (d.z >> 20) & 15, otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
+    const int xlo = wx0 + otx * TS, ylo = wy0 + oty * TS;
+    g.c0 = P.c0; g.c1 = P.c1;
+    g.a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
+    g.b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
+    const int xc = min(max(P.ix, xlo), xlo + ntx * TS - 1), yc = min(max(P.iy, ylo), ylo + nty * TS - 1);
+    g.uc = (float)(xc - wx0); g.vc = (float)(yc - wy0);
+    const float dxc = (float)(xc - P.ix) - P.rx, dyc = (float)(yc - P.iy) - P.ry;
+    g.dgC = make_float3(fmaf(P.c0.x, dxc, fmaf(P.c1.x, dyc, P.dgr.x)), fmaf(P.c0.y, dxc, fmaf(P.c1.y, dyc, P.dgr.y)),
+                        fmaf(P.c0.z, dxc, fmaf(P.c1.z, dyc, P.dgr.z)));
+    g.crC = make_float3(fmaf(g.a1.x, dxc, fmaf(g.b1.x, dyc, P.k.x)), fmaf(g.a1.y, dxc, fmaf(g.b1.y, dyc, P.k.y)),
+                        fmaf(g.a1.z, dxc, fmaf(g.b1.z, dyc, P.k.z)));
+    return g;
+}
+
+// Walks the hit pixels of an item: its pairs row by row, each pair's mask bit by bit.  next() returns the pixel's index
+// in the window (y * GM_WIN + x); call it at most (hits of the item) times.
+template <int TS>
+struct ItemWalk {
+    static constexpr int MW = TS * TS / 32;
+    const uint32_t* mrow;   // masks of the current tile row of the item
+    uint32_t bits, stride;
+    int ntx, tx, wi, pbase, prow;
+    __device__ __forceinline__ void start(const uint32_t* __restrict__ gm_mask, const uint4 d, bool any) {
+        stride = d.z & 0xffffu;
+        ntx = (d.z >> 16) & 15;
+        const int otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
+        mrow = gm_mask + (size_t)d.y * MW;
+        tx = 0; wi = 0;
+        prow = oty * TS * GM_WIN + otx * TS;
+        pbase = prow;
+        bits = any ? __ldg(mrow) : 0u;
+    }
+    __device__ __forceinline__ int next() {
+        while (bits == 0u) {
+            if (++wi == MW) {
+                wi = 0;
+                pbase += TS;
+                if (++tx == ntx) { tx = 0; mrow += (size_t)stride * MW; prow += TS * GM_WIN; pbase = prow; }
+            }
+            bits = __ldg(mrow + tx * MW + wi);
+        }
+        const int b = __ffs((int)bits) - 1 + wi * 32;
+        bits &= bits - 1u;
+        return pbase + (b / TS) * GM_WIN + (b % TS);
+    }
+};
+
+// Block-uniform coefficients of the un-normalised ray direction D = A xf + B yf + C through window pixel (xf, yf).
+struct DirAffine {
+    float3 A, B, C;
+};
+
+// Gradient terms of one hit added to the item's accumulators: geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz),
+// geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh against the bare SH polynomials.
+template <int K>
+__device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, ShRegs<K>& R, float* geo, const float4* __restrict__ spix, int pix, const float4 L) {
+    const float4 gq = spix[pix];
+    const float xf = small_int_to_float((uint32_t)pix & (GM_WIN - 1)), yf = small_int_to_float((uint32_t)pix / GM_WIN);
+    const float Dx = fmaf(dir.A.x, xf, fmaf(dir.B.x, yf, dir.C.x)), Dy = fmaf(dir.A.y, xf, fmaf(dir.B.y, yf, dir.C.y)),
+                Dz = fmaf(dir.A.z, xf, fmaf(dir.B.z, yf, dir.C.z));
+    const float inv = fast_rsqrt(fmaf(Dx, Dx, fmaf(Dy, Dy, Dz * Dz)));
+    float Y[K];
+    sh_poly<K>(make_float3(Dx * inv, Dy * inv, Dz * inv), Y);
+    const float3 g = make_float3(gq.x, gq.y, gq.z);
+    float w[3];
+    lt_weights(L, g, w);
+    R.accumulate(Y, w);
+    const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
+    geo[9] += ad;
+    const float du = xf - P.uc, dv = yf - P.vc;   // small integers: exact
+    const float3 dg = make_float3(fmaf(P.c0.x, du, fmaf(P.c1.x, dv, P.dgC.x)), fmaf(P.c0.y, du, fmaf(P.c1.y, dv, P.dgC.y)),
+                                  fmaf(P.c0.z, du, fmaf(P.c1.z, dv, P.dgC.z)));
+    const float3 cr = make_float3(fmaf(P.a1.x, du, fmaf(P.b1.x, dv, P.crC.x)), fmaf(P.a1.y, du, fmaf(P.b1.y, dv, P.crC.y)),
+                                  fmaf(P.a1.z, du, fmaf(P.b1.z, dv, P.crC.z)));
+    const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
+    // y = d_g x (o_g x d_g); x_g = y / |d_g|^2
+    const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
+    const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+    geo[0] = fmaf(s1, yx, geo[0]); geo[1] = fmaf(s1, yy, geo[1]); geo[2] = fmaf(s1, yz, geo[2]);
+    const float tx = s2 * yx, ty = s2 * yy, tz = s2 * yz;
+    geo[3] = fmaf(tx, yx, geo[3]); geo[4] = fmaf(ty, yy, geo[4]); geo[5] = fmaf(tz, yz, geo[5]);
+    geo[6] = fmaf(tx, yy, geo[6]); geo[7] = fmaf(tx, yz, geo[7]); geo[8] = fmaf(ty, yz, geo[8]);
+}
+
+// FMT: 0 = 16-byte LT entries, 2 = 8-byte entries (four halves, twice as many per pipeline stage).
+template <int TS, int DEG, int FMT>
+__global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __restrict__ rec, const float4* __restrict__ qs,
+                                                             const uint32_t* __restrict__ gid_of_slot, const uint2* __restrict__ blk_desc,
+                                                             const uint32_t* __restrict__ info, const uint32_t* __restrict__ st_off,
+                                                             const uint4* __restrict__ rk_desc, const uint32_t* __restrict__ rk_gstart,
+                                                             const uint32_t* __restrict__ gm_mask, const float4* __restrict__ lt,
+                                                             const float* __restrict__ dL_dC, CamF cam, int sup_x, Gacc gacc,
+                                                             float4* __restrict__ grad4, uint32_t* __restrict__ counts) {
+    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
+    constexpr int EB = FMT == 2 ? 8 : 16;                  // bytes per LT entry
+    constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage
+    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][GMB_STAGE_F4] LT stages, then dL/dC of the window
+    __shared__ __align__(8) uint64_t bars[GMB_WARPS][GMB_STAGES];
+    if (counts[GART_CNT_ERROR]) return;
+    if (blockIdx.x >= info[GM_INFO_BLOCKS]) return;
+    const uint2 bd = blk_desc[blockIdx.x];
+    const int S = (int)bd.x;
+    const uint32_t begin = st_off[S], n = st_off[S + 1] - begin;
+    const int wx0 = (S % sup_x) * GM_SUP, wy0 = (S / sup_x) * GM_SUP;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+#pragma unroll
+        for (int q = 0; q < GMB_STAGES; ++q) mbar_init(smem_u32(&bars[warp][q]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    float4* spix = dyn + GMB_WARPS * GMB_STAGES * GMB_STAGE_F4;
+    for (int t = threadIdx.x; t < GMB_PIX; t += GMB_THREADS) {
+        const int x = wx0 + (t & (GM_WIN - 1)), y = wy0 + t / GM_WIN;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (x < cam.width && y < cam.height) {
+            const float* gp = dL_dC + ((size_t)y * cam.width + x) * 3;
+            v.x = gp[0]; v.y = gp[1]; v.z = gp[2];
+        }
+        spix[t] = v;
+    }
+    __syncthreads();
+    DirAffine dir;
+    {
+        const float ifx = 1.0f / cam.fx, ify = 1.0f / cam.fy;
+        const float u0 = ((float)wx0 + 0.5f - cam.cx) * ifx, v0 = ((float)wy0 + 0.5f - cam.cy) * ify;
+        dir.A = make_float3(cam.r[0] * ifx, cam.r[1] * ifx, cam.r[2] * ifx);
+        dir.B = make_float3(cam.r[3] * ify, cam.r[4] * ify, cam.r[5] * ify);
+        dir.C = make_float3(fmaf(cam.r[0], u0, fmaf(cam.r[3], v0, cam.r[6])), fmaf(cam.r[1], u0, fmaf(cam.r[4], v0, cam.r[7])),
+                            fmaf(cam.r[2], u0, fmaf(cam.r[5], v0, cam.r[8])));
+    }
+
+    float4* my_stage = dyn + (size_t)warp * GMB_STAGES * GMB_STAGE_F4;
+    const uint32_t stage_addr = smem_u32(my_stage);
+    const uint32_t bar_addr = smem_u32(&bars[warp][0]);
+    const char* lt_bytes = reinterpret_cast<const char*>(lt);
+    // LT pipeline: unit u (a chunk of CH entries per lane) uses stage u % GMB_STAGES, and the wait for it uses parity
+    // (u / GMB_STAGES) & 1.  `unit` counts the units consumed, `produced` those whose copy has been issued; the producer
+    // cursor (pw, pk) = (group relative to the current one, chunk) runs up to GMB_STAGES units and two groups ahead.
+    uint32_t unit = 0, produced = 0;
+    int pw = 0, pk = 0;
+    auto produce = [&](const GmItem& a, const GmItem& b, const GmItem& c, const int maxw) {
+        while (produced - unit < (uint32_t)GMB_STAGES && pw <= maxw) {
+            int cm;
+            uint32_t gs;
+            if (pw == 0) { cm = a.cmax; gs = a.gstart; }
+            else if (pw == 1) { cm = b.cmax; gs = b.gstart; }
+            else { cm = c.cmax; gs = c.gstart; }
+            if (cm == 0) break;                                   // ranks descend in hit count: no later group has hits
+            if (pk * CH >= cm) { ++pw; pk = 0; continue; }
+            if (lane == 0) {
+                const int ne = min(CH, cm - pk * CH);
+                const uint32_t bytes = (uint32_t)ne * (32u * EB), s = produced % GMB_STAGES;
+                mbar_expect_tx(bar_addr + 8u * s, bytes);
+                bulk_g2s_hint(stage_addr + s * (GMB_STAGE_F4 * 16u), lt_bytes + ((size_t)gs + (size_t)pk * (CH * 32)) * EB, bytes, bar_addr + 8u * s, l2_policy_evict_first());
+            }
+            ++produced;
+            ++pk;
+        }
+    };
+    auto fail = [&]() {
+        // a copy never completed: report, give copies that may still be in flight a second bounded chance to land
+        // before this warp's shared memory may be released, and stop
+        if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
+        for (uint32_t u = unit; u != produced; ++u) mbar_wait_bounded(bar_addr + 8u * (u % GMB_STAGES), (u / GMB_STAGES) & 1u);
+    };
+
+    // The block's groups are [g0, g0 + GM_GROUPS_PER_BLOCK) of the super-tile; the warp's j-th group is
+    // g0 + j * GMB_WARPS + (j even ? warp : GMB_WARPS - 1 - warp): groups descend in hit count, and this serpentine deal
+    // gives every warp nearly the same number of iterations.
+    const uint32_t g0 = bd.y * GM_GROUPS_PER_BLOCK;
+    constexpr uint32_t ROUNDS = GM_GROUPS_PER_BLOCK / GMB_WARPS;
+    auto load = [&](uint32_t j) {
+        const uint32_t gi = g0 + j * GMB_WARPS + ((j & 1u) ? (uint32_t)(GMB_WARPS - 1 - warp) : (uint32_t)warp);
+        return gm_load_item(rk_desc, rk_gstart, begin, n, 32u * gi, j < ROUNDS, lane);
+    };
+    uint32_t gj = 0;
+    GmItem cur = load(0);
+    GmItem nxt = load(1);
+    while (__any_sync(0xffffffffu, cur.valid)) {
+        const GmItem nxt2 = load(gj + 2);
+        produce(cur, nxt, nxt2, 1);
+        // the item's Gaussian: evaluation record, and what the final conversion needs
+        const uint32_t sid = cur.d.x;
+        const bool whole = (cur.d.w & GM_DESC_WHOLE) != 0u;
+        PreRec P;
+        if (cur.valid) {
+            P = load_pre(rec + (size_t)sid * RS4);
+        } else {
+            P = unpack_pre(make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 1.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f),
+                           make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f));
+        }
+        const ItemGeo IG = item_geo<TS>(P, cur.d, wx0, wy0);
+        ItemWalk<TS> walk;
+        walk.start(gm_mask, cur.d, cur.c != 0);
+        ShRegs<K> R;
+        R.clear();
+        float geo[11];
+#pragma unroll
+        for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
+        const int nchunks = (cur.cmax + CH - 1) / CH;
+        for (int k = 0; k < nchunks; ++k) {
+            const uint32_t s = unit % GMB_STAGES;
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / GMB_STAGES) & 1u))) { fail(); return; }
+            const char* sl = reinterpret_cast<const char*>(my_stage + s * GMB_STAGE_F4) + lane * EB;   // entry j of the stage: sl + j * 32 * EB
+            auto entry = [&](const char* q) {
+                if constexpr (FMT == 2) return lt_unpack_half(*reinterpret_cast<const uint2*>(q));
+                else return *reinterpret_cast<const float4*>(q);
+            };
+            const int e_end = min(cur.c, (k + 1) * CH);
+            // two hits per iteration: two independent dependency chains for the scheduler to interleave
+            int e = k * CH;
+            const char* se = sl;
+            for (; e + 1 < e_end; e += 2, se += 64 * EB) {
+                const int p0 = walk.next();
+                const int p1 = walk.next();
+                const float4 L0 = entry(se), L1 = entry(se + 32 * EB);
+                gm_hit<K>(IG, dir, R, geo, spix, p0, L0);
+                gm_hit<K>(IG, dir, R, geo, spix, p1, L1);
+            }
+            if (e < e_end) gm_hit<K>(IG, dir, R, geo, spix, walk.next(), entry(se));
+            fence_proxy_async();
+            __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
+            ++unit;
+            produce(cur, nxt, nxt2, 2);
+        }
+        // ---- the item's sums leave the registers
+        if (cur.valid) {
+            if (whole) {
+                // the thread holds every hit of its Gaussian: convert the moments and write the gradient record once
+                // (quaternion, scale, opacity and id are fetched only now: they would occupy registers across the hit loop)
+                const float4 q4 = __ldg(qs + 2 * (size_t)sid), s4 = __ldg(qs + 2 * (size_t)sid + 1);
+                const uint32_t gid = __ldg(gid_of_slot + sid);
+                const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
+                const float sc[3] = {s4.x, s4.y, s4.z};
+                const GeoGrad o = moments_to_grads(geo, geo + 3, qv, sc);
+                const float gw[11] = {o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0], o.ds[1], o.ds[2], o.dq[0], o.dq[1], o.dq[2], o.dq[3], geo[9] / s4.w};
+                float4* out = grad4 + (size_t)gid * (GART_GRAD_WORDS / 4);
+#pragma unroll
+                for (int q = 0; q < GART_GRAD_WORDS / 4; ++q) {
+                    float v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int wd = 4 * q + i;
+                        v[i] = wd < 11 ? gw[wd] : (wd < 11 + SW ? sh_norm((wd - 11) / 3) * R.word(wd - 11) : 0.0f);
+                    }
+                    __stcs(out + q, make_float4(v[0], v[1], v[2], v[3]));
+                }
+            } else if (cur.c != 0) {
+                // a piece of a large Gaussian: one vector atomic per 16 bytes of the slot's accumulation record
+                const uint64_t pol_keep = l2_policy_evict_last();
+#pragma unroll
+                for (int q = 0; q < AW / 4; ++q) {
+                    float v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int wd = 4 * q + i;
+                        v[i] = wd < 10 ? geo[wd] : (wd >= 11 && wd < 11 + SW ? R.word(wd - 11) : 0.0f);
+                    }
+                    red_add_f4_hint(gacc_piece(gacc, sid, q), v[0], v[1], v[2], v[3], pol_keep);
+                }
+            }
+        }
+        cur = nxt;
+        nxt = nxt2;
+        ++gj;
+        --pw;
+        if (pw < 0) { pw = 0; pk = 0; }   // (a group without hits leaves the producer behind: it restarts at the new current group)
+    }
+}
+
+// ---- the large Gaussians (cut into pieces): zero their accumulation records before, convert them after.  One thread
+// per slot looks at the rectangle; the few large ones (a few per cent) do the work.
+static __global__ void __launch_bounds__(256) gm_zero_big_kernel(const int4* __restrict__ srect, Gacc gacc, const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+    if (gm_is_whole(__ldg(srect + sid))) return;
+#pragma unroll
+    for (int q = 0; q < (GACC_A_WORDS + GACC_B_WORDS) / 4; ++q) *gacc_piece(gacc, (uint32_t)sid, q) = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+static __global__ void __launch_bounds__(256) gm_convert_big_kernel(const int4* __restrict__ srect, const float4* __restrict__ qs,
+                                                                    const uint32_t* __restrict__ gid_of_slot, Gacc gacc,
+                                                                    float4* __restrict__ grad4, const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    constexpr int F4 = GART_GRAD_WORDS / 4;
+    const int64_t sid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sid >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+    if (gm_is_whole(__ldg(srect + sid))) return;
+    float4* out = grad4 + (size_t)gid_of_slot[sid] * F4;
+    const float4* gp = reinterpret_cast<const float4*>(gacc.a) + (size_t)sid * (GACC_A_WORDS / 4);
+    const float4 a = gp[0], b = gp[1], c = gp[2], d = gp[3];
+    const float4 q4 = qs[2 * sid], s4 = qs[2 * sid + 1];
+    const float v[3] = {a.x, a.y, a.z};
+    const float Q[6] = {a.w, b.x, b.y, b.z, b.w, c.x};
+    const float q[4] = {q4.x, q4.y, q4.z, q4.w};
+    const float sc[3] = {s4.x, s4.y, s4.z};
+    const GeoGrad o = moments_to_grads(v, Q, q, sc);
+    out[0] = make_float4(o.dmu[0], o.dmu[1], o.dmu[2], o.ds[0]);
+    out[1] = make_float4(o.ds[1], o.ds[2], o.dq[0], o.dq[1]);
+    out[2] = make_float4(o.dq[2], o.dq[3], c.y / s4.w, sh_word_norm(11) * c.w);
+    out[3] = make_float4(sh_word_norm(12) * d.x, sh_word_norm(13) * d.y, sh_word_norm(14) * d.z, sh_word_norm(15) * d.w);
+    const float4* bp = reinterpret_cast<const float4*>(gacc.b) + (size_t)sid * (GACC_B_WORDS / 4);
+#pragma unroll
+    for (int l = 4; l < 15; ++l) {
+        const float4 t = bp[l - 4];
+        out[l] = make_float4(sh_word_norm(4 * l) * t.x, sh_word_norm(4 * l + 1) * t.y, sh_word_norm(4 * l + 2) * t.z,
+                             4 * l + 3 < 59 ? sh_word_norm(4 * l + 3) * t.w : 0.0f);
+    }
+    out[15] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// A zero record for every Gaussian without a slot: a thread looks at one Gaussian, the warp then writes the flagged
+// records two at a time (16 lanes per 256-byte record).
+static __global__ void __launch_bounds__(256) gm_fill_kernel(int64_t n, const uint32_t* __restrict__ slot_of_gid, float4* __restrict__ grad4,
+                                                             const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const bool none = gid < n && __ldg(slot_of_gid + gid) == 0xffffffffu;
+    unsigned m = __ballot_sync(0xffffffffu, none);
+    const int64_t g0 = gid - lane;
+    while (m) {
+        const int a = __ffs((int)m) - 1;
+        m &= m - 1u;
+        int b = -1;
+        if (m) { b = __ffs((int)m) - 1; m &= m - 1u; }
+        const int mine = lane < 16 ? a : b;
+        if (mine >= 0) __stcs(grad4 + (size_t)(g0 + mine) * (GART_GRAD_WORDS / 4) + (lane & 15), make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+}
+
+template <int TS, int FMT>
+static gart_status launch_gm(int deg, unsigned grid, cudaStream_t st, const float4* rec, const float4* qs, const uint32_t* gid_of_slot,
+                             const ViewLayout& v, const float4* lt, const float* dL_dC, const CamF& cam, int sup_x, const Gacc& gacc,
+                             float4* grad4, uint32_t* counts) {
+#define GART_GM(D)                                                                                                                \
+    {                                                                                                                            \
+        auto kern = bwd_gm_kernel<TS, D, FMT>;                                                                                   \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GMB_DYN_SMEM) != cudaSuccess) return GART_ERR_CUDA; \
+        kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, v.gm_mask, lt, \
+                                                      dL_dC, cam, sup_x, gacc, grad4, counts);                                  \
+    }
+    switch (deg) {
+        case 0: GART_GM(0); break;
+        case 1: GART_GM(1); break;
+        case 2: GART_GM(2); break;
+        default: GART_GM(3); break;
+    }
+#undef GART_GM
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}
+
+}  // namespace gart
+
+extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
+                                     const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+                                     const void* view, size_t view_bytes, int64_t cap_pairs,
+                                     const float* lt, const float* dL_dcolor,
+                                     float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace gart;
+    (void)tile_off;
+    if (!cfg || !g || !cam || !counts || !dL_dcolor) return GART_ERR_INVALID_ARG;
+    if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format != 0 && cfg->lt_format != 2) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte or 8-byte LT entries
+    if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR) return GART_ERR_INVALID_ARG;    // ... in the primitive-major layout
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
+    if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
+    if (g->n == 0) return GART_OK;
+    if (!grad || !pre || !slot_of_gid || !gid_of_slot || !lt || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
+    if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    const ViewLayout v = view_layout(const_cast<void*>(view), g->n, cam->width, cam->height, cfg->tile_size, cap_pairs);
+    if (v.bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Gacc gacc = make_gacc(workspace, g->n);
+    const CamF cf = make_camf(cam, cfg->tile_size);
+    const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
+    const float4* rec = reinterpret_cast<const float4*>(pre);
+    const int rs4 = rec_f4(g->sh_degree);
+    const float4* qs = rec + (size_t)g->n * rs4;                                         // per slot: quaternion, scale, opacity
+    const int4* srect = reinterpret_cast<const int4*>(rec + (size_t)g->n * (rs4 + 2));   // per slot: rectangle
+    const float4* lt4 = reinterpret_cast<const float4*>(lt);
+    float4* grad4 = reinterpret_cast<float4*>(grad);
+    const unsigned slot_blocks = (unsigned)ceil_div(g->n, 256);
+    gm_zero_big_kernel<<<slot_blocks, 256, 0, st>>>(srect, gacc, counts);
+    GART_LAUNCH_CHECK();
+    gm_fill_kernel<<<slot_blocks, 256, 0, st>>>(g->n, slot_of_gid, grad4, counts);
+    GART_LAUNCH_CHECK();
+    const unsigned grid = (unsigned)v.blocks_cap;
+    gart_status s;
+#define GART_GM_TS(TSV, F) launch_gm<TSV, F>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts)
+    if (cfg->lt_format == 0) s = cfg->tile_size == 8 ? GART_GM_TS(8, 0) : GART_GM_TS(16, 0);
+    else s = cfg->tile_size == 8 ? GART_GM_TS(8, 2) : GART_GM_TS(16, 2);
+#undef GART_GM_TS
+    if (s != GART_OK) return s;
+    gm_convert_big_kernel<<<slot_blocks, 256, 0, st>>>(srect, qs, gid_of_slot, gacc, grad4, counts);
+    GART_LAUNCH_CHECK();
+    return GART_OK;
+}

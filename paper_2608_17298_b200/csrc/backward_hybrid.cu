@@ -13,6 +13,7 @@
 //     Cb_{i-1} = alpha_i c_i + (1 - alpha_i) Cb_i       (colour behind, not premultiplied; Cb_last = background)
 // so that alpha dL/dalpha = w_i <dL/dC, c_i - Cb_i>  (Eq. 6-8); nothing is a difference of nearly equal sums.
 #include "backward_common.cuh"
+#include "view_layout.cuh"
 
 namespace gart {
 
@@ -238,20 +239,24 @@ static gart_status launch_sh(int deg, int T, cudaStream_t st, const uint32_t* ti
 
 extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                             const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
-                                            const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
-                                            const uint32_t* tile_lt_base, const float* lt_w, const uint32_t* ray_off, const uint32_t* ray_gid,
+                                            const void* view, size_t view_bytes, int64_t cap_pairs,
+                                            const float* lt_w, const uint32_t* ray_off, const uint32_t* ray_gid,
                                             const float* dL_dcolor, float* grad, uint32_t* counts, void* workspace, size_t workspace_bytes,
                                             void* stream) {
     using namespace gart;
-    if (!cfg || !g || !cam || !counts || !tile_off || !tile_lt_base || !dL_dcolor || !ray_off) return GART_ERR_INVALID_ARG;
+    if (!cfg || !g || !cam || !counts || !tile_off || !dL_dcolor || !ray_off) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 1) return GART_ERR_INVALID_ARG;   // this pass reads the 4-byte LT format
+    if (cfg->lt_format != 1 || cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // this pass reads the 4-byte LT format, tile-major
     if (cfg->max_hits != 0) return GART_ERR_INVALID_ARG;    // its pixel-centric part re-derives every hit's alpha: no cap
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
+    if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
-    if (!grad || !pre || !slot_of_gid || !gid_of_slot) return GART_ERR_INVALID_ARG;
+    if (!grad || !pre || !slot_of_gid || !gid_of_slot || !lt_w || !ray_gid || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
     if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    const ViewLayout v = view_layout(const_cast<void*>(view), g->n, cam->width, cam->height, cfg->tile_size, cap_pairs);
+    if (v.bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    const uint32_t *rank_sid = v.rank_sid, *rank_mask = v.rank_mask, *rank_gstart = v.rank_gstart, *tile_lt_base = v.tile_lt_base;
     cudaStream_t st = (cudaStream_t)stream;
     const Gacc gacc = make_gacc(workspace, g->n);
     gart_status s = launch_zero_accumulators(gacc, g->n, counts, st);

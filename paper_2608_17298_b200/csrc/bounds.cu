@@ -4,12 +4,13 @@
 // p -/+ h) and the pass is O(n), so fp64 costs nothing that matters and keeps the edges exact.
 //
 // The Gaussians that reach the image are then renumbered for this view: a stable radix sort on the
-// tile of the rectangle's first corner gives every visible Gaussian a "slot", and its evaluation
-// record and SH coefficients are gathered into one contiguous record per slot.  Tiles are processed
-// in tile order, so the per-pair reads of these records and the per-pair gradient updates of the
-// backward touch memory that neighbouring tiles also touch, instead of random 200-byte pieces of
-// gigabyte-sized arrays.
+// 16 x 16-pixel super-tile of the rectangle's first corner gives every visible Gaussian a "slot", and its
+// evaluation record and SH coefficients are gathered into one contiguous record per slot.  Tiles are
+// processed in tile order and the backward walks the slots in order, so per-pair reads of these records
+// touch memory that neighbouring work also touches, instead of random 200-byte pieces of gigabyte-sized
+// arrays; the Gaussians that one super-tile owns are one contiguous run of slots.
 #include "radix.cuh"
+#include "view_layout.cuh"
 
 namespace gart {
 
@@ -30,7 +31,7 @@ __device__ __forceinline__ void quat_to_rot(const double w, const double x, cons
 __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
                                                      const float* __restrict__ quat, const float* __restrict__ opacity,
                                                      CamD cam, double alpha_min, double near_z,
-                                                     int ts, int tiles_x, uint32_t key_none,
+                                                     int sup_x, uint32_t key_none,
                                                      int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
                                                      float4* __restrict__ pre4, uint32_t* __restrict__ keys,
                                                      uint32_t* __restrict__ vals, uint32_t* __restrict__ counts) {
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
             q5 = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
             q6 = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
         }
-        keys[i] = vis ? (uint32_t)(y0 / ts) : key_none;   // tile row of the rectangle's corner
+        keys[i] = vis ? (uint32_t)((y0 / GM_SUP) * sup_x + x0 / GM_SUP) : key_none;   // super-tile of the rectangle's corner
         vals[i] = (uint32_t)i;
     }
     {
@@ -176,7 +177,8 @@ template <int DEG>
 __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
                                                              const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
-                                                             float4* __restrict__ rec, float4* __restrict__ qs,
+                                                             const int4* __restrict__ rect,
+                                                             float4* __restrict__ rec, float4* __restrict__ qs, int4* __restrict__ srect,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
     constexpr uint32_t SW = 3 * (DEG + 1) * (DEG + 1), RS4 = (20 + SW + 3) / 4;   // (compile-time: the divisions below are multiplications)
     __shared__ float s_norm[16];   // lanes index it divergently: shared memory, not the constant bank
@@ -225,6 +227,7 @@ __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_
             qs[2 * (size_t)slot[u]] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 5];
             qs[2 * (size_t)slot[u] + 1] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 6];
         }
+        if (q[u] == 2) srect[slot[u]] = rect[gid[u]];   // the rectangle in slot order
         if (q[u] >= 5) {
             // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
             const uint32_t e = (q[u] - 5) * 4;
@@ -270,15 +273,16 @@ extern "C" const char* gart_status_string(gart_status s) {
         case GART_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case GART_ERR_CAPACITY_EXCEEDED: return "capacity exceeded";
         case GART_ERR_CUDA: return "CUDA error";
+        case GART_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     }
     return "unknown status";
 }
 
 extern "C" int32_t gart_mask_words(int32_t tile_size) { return tile_size * tile_size / 32; }
 
-// Per Gaussian: the slot record (evaluation record + SH coefficients, padded to 16 bytes) and, in a
-// second block behind all records, 8 words (quaternion, scale, opacity) in slot order.
-extern "C" int32_t gart_pre_words(int32_t sh_degree) { return 4 * gart::rec_f4(sh_degree) + 8; }
+// Per Gaussian: the slot record (evaluation record + SH coefficients, padded to 16 bytes); in a second
+// block behind all records, 8 words (quaternion, scale, opacity) in slot order; in a third, the rectangle.
+extern "C" int32_t gart_pre_words(int32_t sh_degree) { return 4 * gart::rec_f4(sh_degree) + 8 + 4; }
 
 extern "C" size_t gart_bounds_workspace_bytes(int64_t n) { return gart::bounds_layout(nullptr, n).bytes; }
 
@@ -302,9 +306,8 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     c.width = cam->width; c.height = cam->height;
     c.fx = cam->fx; c.fy = cam->fy; c.cx = cam->cx; c.cy = cam->cy;
     for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
-    const int ts = cfg->tile_size;
-    const int tiles_x = (cam->width + ts - 1) / ts, tiles_y = (cam->height + ts - 1) / ts;
-    const uint32_t key_none = (uint32_t)tiles_y;   // sorts after every tile row
+    const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
+    const uint32_t key_none = (uint32_t)gm_super_tiles(cam->width, cam->height);   // sorts after every super-tile
     int bits = 1;
     while ((1u << bits) <= key_none) ++bits;
     uint32_t* const kbuf[2] = {w.keys0, w.keys1};
@@ -313,7 +316,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     const int threads = 128;
     const int64_t blocks = ceil_div(g->n, threads);
     bounds_kernel<<<(unsigned)blocks, threads, 0, st>>>(g->n, g->mean, g->scale, g->quat, g->opacity, c,
-                                                       (double)cfg->alpha_min, (double)cfg->near_z, ts, tiles_x, key_none, rect, cls,
+                                                       (double)cfg->alpha_min, (double)cfg->near_z, sup_x, key_none, rect, cls,
                                                        w.pre_tmp, kbuf[cur], vbuf[cur], counts);
     GART_LAUNCH_CHECK();
     gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);
@@ -324,7 +327,8 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     float4* rec_out = reinterpret_cast<float4*>(pre);
 #define GART_GATHER(D)                                                                                                                        \
     gather_records_kernel<D><<<(unsigned)ceil_div(gthreads, 256 * GATHER_UNROLL), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh, \
-                                                                                rec_out, rec_out + (size_t)g->n * rs4, slot_of_gid, gid_of_slot)
+                                                                                reinterpret_cast<const int4*>(rect), rec_out, rec_out + (size_t)g->n * rs4,        \
+                                                                                reinterpret_cast<int4*>(rec_out + (size_t)g->n * (rs4 + 2)), slot_of_gid, gid_of_slot)
     switch (g->sh_degree) {
         case 0: GART_GATHER(0); break;
         case 1: GART_GATHER(1); break;

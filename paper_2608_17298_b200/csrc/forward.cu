@@ -19,7 +19,7 @@
 //   4. fwd_sort_sweep  warp per ray: sort the segment by (t*, id), scan the transmittance
 //                  front to back, then sum colour back to front so that each hit gets the
 //                  colour composited behind it without cancellation; write LT, C, T_final.
-#include "common.cuh"
+#include "gm_build.cuh"
 
 namespace gart {
 
@@ -104,6 +104,8 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
                                                                    const uint32_t* __restrict__ tile_off,
                                                                    const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
                                                                    uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ pair_sid,
+                                                                   const int4* __restrict__ srect, const uint32_t* __restrict__ gpair_off,
+                                                                   uint32_t* __restrict__ gm_mask, uint32_t* __restrict__ pair_gpos,
                                                                    uint32_t* __restrict__ hit_count, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, RPW = 32 / TS;   // rows per mask word
     __shared__ uint32_t scnt[NT];
@@ -129,10 +131,19 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
     const uint32_t jfirst = begin + threadIdx.x;
     uint32_t sid_nx = load_sid(jfirst + STEP);
     float4 ra[5];
+    // the pair's place in the primitive-major order: first pair of its Gaussian + its tile's index in the rectangle's tiles
+    auto gpos_of = [&](uint32_t sid, bool act) {
+        if (!act) return 0u;
+        const int4 r = __ldg(srect + sid);
+        const int gx0 = r.x / TS, gy0 = r.y / TS;
+        return __ldg(gpair_off + sid) + (uint32_t)((ty - gy0) * (r.z / TS - gx0 + 1) + (tx - gx0));
+    };
+    uint32_t gpa;
     {
         const uint32_t sid0 = load_sid(jfirst);
 #pragma unroll
         for (int q = 0; q < 5; ++q) ra[q] = jfirst < end ? __ldg(rec + (size_t)sid0 * rs4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        gpa = gpos_of(sid0, jfirst < end);
     }
     for (uint32_t j0 = begin + (threadIdx.x & ~31u); j0 < end; j0 += STEP) {
         const uint32_t j = j0 + lane;
@@ -140,6 +151,7 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
         float4 rb[5];
 #pragma unroll
         for (int q = 0; q < 5; ++q) rb[q] = j + STEP < end ? __ldg(rec + (size_t)sid_nx * rs4 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const uint32_t gpb = gpos_of(sid_nx, j + STEP < end);
         sid_nx = sid_nx2;
         uint32_t w[MW];
 #pragma unroll
@@ -181,6 +193,9 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
             }
 #pragma unroll
             for (int q = 0; q < MW; ++q) pair_mask[(size_t)j * MW + q] = w[q];
+#pragma unroll
+            for (int q = 0; q < MW; ++q) gm_mask[(size_t)gpa * MW + q] = w[q];
+            pair_gpos[j] = gpa;
         }
         // hits per pixel: one shared-memory increment per hit
 #pragma unroll
@@ -194,6 +209,7 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
         }
 #pragma unroll
         for (int q = 0; q < 5; ++q) ra[q] = rb[q];
+        gpa = gpb;
     }
     __syncthreads();
     uint32_t m = 0;
@@ -222,9 +238,10 @@ __device__ __forceinline__ uint32_t mask_popc(const uint32_t* __restrict__ pair_
 
 template <int TS>
 __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ pair_sid,
-                                                                    const uint32_t* __restrict__ pair_mask, int T, uint32_t* pair_order,
+                                                                    const uint32_t* __restrict__ pair_mask, const uint32_t* __restrict__ pair_gpos,
+                                                                    int T, uint32_t* pair_order,
                                                                     uint32_t* __restrict__ rank_sid, uint32_t* __restrict__ rank_mask,
-                                                                    uint32_t* __restrict__ rank_gstart,
+                                                                    uint32_t* __restrict__ rank_gstart, uint32_t* __restrict__ rank_gpos,
                                                                     uint32_t* __restrict__ tile_slots, const uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, NB = NT + 1;
     __shared__ uint32_t hist[SORT_WARPS][NB];
@@ -276,7 +293,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
     __syncwarp();
     uint32_t run = 0;
     for (uint32_t r0 = 0; r0 < n; r0 += 32 * TSU) {
-        uint32_t j[TSU], sid[TSU], wv[TSU][MW];
+        uint32_t j[TSU], sid[TSU], gp[TSU], wv[TSU][MW];
 #pragma unroll
         for (int u = 0; u < TSU; ++u) j[u] = r0 + 32 * u + lane < n ? __ldcg(pair_order + begin + r0 + 32 * u + lane) : 0xffffffffu;
 #pragma unroll
@@ -285,6 +302,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
 #pragma unroll
             for (int m = 0; m < MW; ++m) wv[u][m] = act ? __ldg(pair_mask + (size_t)j[u] * MW + m) : 0u;
             sid[u] = act ? __ldg(pair_sid + j[u]) : 0u;
+            gp[u] = act ? __ldg(pair_gpos + j[u]) : 0u;
         }
 #pragma unroll
         for (int u = 0; u < TSU; ++u) {
@@ -296,6 +314,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
 #pragma unroll
                 for (int m = 0; m < MW; ++m) rank_mask[q * MW + m] = wv[u][m];
                 rank_sid[q] = sid[u];
+                rank_gpos[q] = gp[u];
                 rank_gstart[q] = run;
             }
             const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
@@ -338,17 +357,20 @@ struct EvalDesc {
     int cmax;   // hits of the group's first pair (the largest)
 };
 
-template <int MW>
+// GMAJ: the LT slot of the pair's first hit comes from the primitive-major layout (gm_ltb, looked up by the pair's
+// primitive-major position) instead of the tile's rank groups; later hits follow 32 entries apart in both layouts.
+template <int MW, bool GMAJ>
 __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
-                                                       const uint32_t* __restrict__ rank_gstart, uint32_t begin, uint32_t n,
-                                                       uint32_t r0, int lane) {
+                                                       const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ gm_ltb,
+                                                       uint32_t begin, uint32_t n, uint32_t r0, int lane) {
     EvalDesc<MW> d;
     const bool act = r0 < n && r0 + lane < n;
     const uint32_t q = begin + r0 + lane;
     d.pm.load(rank_mask, act ? q : 0u, act);
     d.c = d.pm.count();
     d.sid = act ? __ldg(rank_sid + q) : 0u;
-    d.gstart = act ? __ldg(rank_gstart + q) : 0u;
+    d.gstart = act ? __ldg(rank_gstart + q) : 0u;   // (GMAJ: rank_gstart is the array of primitive-major positions)
+    if (GMAJ) d.gstart = act ? __ldg(gm_ltb + d.gstart) : 0u;
     d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
     return d;
 }
@@ -369,11 +391,11 @@ struct EvalPix {
 // next group's Gaussians are copied into shared memory (16-byte asynchronous copies of each lane) while the
 // current group is evaluated.  The colour is 0.5 + sum_k B_k(d) sh'_k with the bare SH polynomials B_k and
 // the record's coefficients sh'_k, which carry the normalisation constants.
-template <int TS, int DEG>
+template <int TS, int DEG, bool GMAJ>
 __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
-                                                                const uint32_t* __restrict__ tile_lt_base,
+                                                                const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ gm_ltb,
                                                                 const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
                                                                 uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PF4 = (20 + SW + 3) / 4;
@@ -428,12 +450,12 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     };
 
     uint32_t r0 = warp * 32;
-    EvalDesc<MW> cur = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0, lane);
+    EvalDesc<MW> cur = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0, lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
     issue_params(cur);
-    EvalDesc<MW> nxt = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + EVAL_THREADS, lane);
+    EvalDesc<MW> nxt = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0 + EVAL_THREADS, lane);
     while (true) {
-        const EvalDesc<MW> nxt2 = load_eval_desc<MW>(rank_sid, rank_mask, rank_gstart, begin, n, r0 + 2 * EVAL_THREADS, lane);
+        const EvalDesc<MW> nxt2 = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0 + 2 * EVAL_THREADS, lane);
         const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
         cp_async_wait_all();   // the copies this lane issued have landed
         __syncwarp();          // ... and so have those of the other lanes, which hold pieces of this lane's record
@@ -446,7 +468,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         }
         __syncwarp();                           // every lane has read its record: the buffers may be overwritten
         if (nxt.cmax != 0) issue_params(nxt);
-        uint32_t slot = lt_base + cur.gstart + lane;
+        uint32_t slot = GMAJ ? cur.gstart : lt_base + cur.gstart + lane;
         const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
         // one hit: evaluate, take the next free place of the ray's segment, write the 32-byte record
         auto hit = [&](const int p, const uint32_t slot_e) {
@@ -886,10 +908,11 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
 
 // ------------------------------------------------------------------------------------------ host
 struct ForwardWs {
-    uint64_t *total_slots, *total_hits;
+    uint64_t *total_slots, *total_hits, *total_gm;
     void* scan_ws;
     uint32_t* tile_slots;
     uint32_t* pair_sid;     // slot of every pair's Gaussian, in pair order (written by fwd_mask, read by tile_sort)
+    uint32_t *ikeys0, *ikeys1, *ivals0, *ivals1, *itable;   // sort of the primitive-major items by super-tile
     float4* recs;
     uint64_t* long_keys;
     size_t bytes;
@@ -900,29 +923,38 @@ static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_p
     char* p = (char*)base;
     size_t off = 0;
     auto take = [&](size_t b) { void* r = p ? (void*)(p + off) : nullptr; off += align256(b); return r; };
-    const int64_t ch = cap_hits > 0 ? cap_hits : 1;
+    const int64_t ch = cap_hits > 0 ? cap_hits : 1, cp = cap_pairs > 0 ? cap_pairs : 1;
     w.total_slots = (uint64_t*)take(256);
     w.total_hits = (uint64_t*)take(256);
-    w.scan_ws = take(scan_workspace_bytes(n_rays > T ? n_rays : T));
+    w.total_gm = (uint64_t*)take(256);
+    // scans over rays, tiles, super-tiles (fewer than tiles), the slots that have pairs (no more than the pair
+    // capacity) and the radix tables of the item sort
+    const int64_t scan_n = n_rays > T ? n_rays : T;
+    size_t sb = scan_workspace_bytes(scan_n > cp ? scan_n : cp);
+    if (radix_scan_bytes(cp) > sb) sb = radix_scan_bytes(cp);
+    w.scan_ws = take(sb);
     w.tile_slots = (uint32_t*)take((size_t)(T + 1) * 4);
-    w.pair_sid = (uint32_t*)take((size_t)(cap_pairs > 0 ? cap_pairs : 1) * 4);
+    w.pair_sid = (uint32_t*)take((size_t)cp * 4);
+    w.ikeys0 = (uint32_t*)take((size_t)cp * 4); w.ikeys1 = (uint32_t*)take((size_t)cp * 4);
+    w.ivals0 = (uint32_t*)take((size_t)cp * 4); w.ivals1 = (uint32_t*)take((size_t)cp * 4);
+    w.itable = (uint32_t*)take(radix_table_bytes(cp));
     w.recs = (float4*)take((size_t)ch * 32);
     w.long_keys = (uint64_t*)take((size_t)ch * 8);
     w.bytes = off;
     return w;
 }
 
-template <int TS>
+template <int TS, bool GMAJ>
 static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
-                               const uint32_t* tile_lt_base, const uint32_t* ray_off,
+                               const uint32_t* tile_lt_base, const uint32_t* gm_ltb, const uint32_t* ray_off,
                                const CamF& cam, const ForwardWs& w, uint32_t* counts) {
 #define GART_EVAL(D)                                                                                                        \
     {                                                                                                                      \
-        auto kern = fwd_eval_kernel<TS, D>;                                                                                \
+        auto kern = fwd_eval_kernel<TS, D, GMAJ>;                                                                          \
         constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
-        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cam, \
+        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, gm_ltb, ray_off, cam, \
                                             w.recs, counts);                                                               \
     }
     switch (deg) {
@@ -938,6 +970,44 @@ static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* re
 
 }  // namespace gart
 
+extern "C" size_t gart_view_bytes(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs) {
+    if ((tile_size != 8 && tile_size != 16) || width <= 0 || height <= 0 || n < 0 || cap_pairs < 0) return 0;
+    return gart::view_layout(nullptr, n, width, height, tile_size, cap_pairs).bytes;
+}
+
+extern "C" gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int32_t which,
+                                       size_t* offset, size_t* bytes) {
+    using namespace gart;
+    if ((tile_size != 8 && tile_size != 16) || width <= 0 || height <= 0 || n < 0 || cap_pairs < 0 || !offset || !bytes) return GART_ERR_INVALID_ARG;
+    char* const base = reinterpret_cast<char*>((uintptr_t)256);   // (a non-null base: only differences are used)
+    const ViewLayout v = view_layout(base, n, width, height, tile_size, cap_pairs);
+    const int64_t cp = cap_pairs > 0 ? cap_pairs : 1, nn = n > 0 ? n : 1;
+    const int T = ((width + tile_size - 1) / tile_size) * ((height + tile_size - 1) / tile_size), mw = tile_size * tile_size / 32;
+    const void* ptr = nullptr;
+    size_t b = 0;
+    switch (which) {
+        case GART_VIEW_PAIR_MASK: ptr = v.pair_mask; b = (size_t)cp * 4 * mw; break;
+        case GART_VIEW_PAIR_ORDER: ptr = v.pair_order; b = (size_t)cp * 4; break;
+        case GART_VIEW_RANK_SID: ptr = v.rank_sid; b = (size_t)cp * 4; break;
+        case GART_VIEW_RANK_MASK: ptr = v.rank_mask; b = (size_t)cp * 4 * mw; break;
+        case GART_VIEW_RANK_GSTART: ptr = v.rank_gstart; b = (size_t)cp * 4; break;
+        case GART_VIEW_TILE_LT_BASE: ptr = v.tile_lt_base; b = (size_t)(T + 1) * 4; break;
+        case GART_VIEW_PAIR_GPOS: ptr = v.pair_gpos; b = (size_t)cp * 4; break;
+        case GART_VIEW_GPAIR_OFF: ptr = v.gpair_off; b = (size_t)(nn + 1) * 4; break;
+        case GART_VIEW_GM_MASK: ptr = v.gm_mask; b = (size_t)cp * 4 * mw; break;
+        case GART_VIEW_GM_LTB: ptr = v.gm_ltb; b = (size_t)cp * 4; break;
+        case GART_VIEW_ITEM_DESC: ptr = v.rk_desc; b = (size_t)cp * 16; break;
+        case GART_VIEW_ITEM_GSTART: ptr = v.rk_gstart; b = (size_t)cp * 4; break;
+        case GART_VIEW_ST_OFF: ptr = v.st_off; b = (size_t)(v.ns + 1) * 4; break;
+        case GART_VIEW_ST_LT_BASE: ptr = v.st_lt_base; b = (size_t)(v.ns + 1) * 4; break;
+        case GART_VIEW_INFO: ptr = v.info; b = GM_INFO_WORDS * 4; break;
+        default: return GART_ERR_INVALID_ARG;
+    }
+    *offset = (size_t)(reinterpret_cast<const char*>(ptr) - base);
+    *bytes = b;
+    return GART_OK;
+}
+
 extern "C" size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits) {
     if (tile_size != 8 && tile_size != 16) return 0;
     const int T = ((width + tile_size - 1) / tile_size) * ((height + tile_size - 1) / tile_size);
@@ -947,51 +1017,115 @@ extern "C" size_t gart_forward_workspace_bytes(int32_t width, int32_t height, in
 extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                     const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off, const uint32_t* pair_gid, int64_t cap_pairs,
                                     float* color, float* t_final, uint32_t* hit_count,
-                                    uint32_t* pair_mask, uint32_t* pair_order, uint32_t* rank_sid, uint32_t* rank_mask,
-                                    uint32_t* rank_gstart, uint32_t* tile_lt_base,
                                     float* lt, int64_t cap_hits,
-                                    uint32_t* ray_off, uint32_t* ray_gid, uint32_t* ray_slot, uint32_t* counts,
+                                    uint32_t* ray_off, uint32_t* ray_gid, uint32_t* ray_slot,
+                                    void* view, size_t view_bytes, uint32_t* counts,
                                     void* workspace, size_t workspace_bytes, void* stream) {
     using namespace gart;
-    if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !tile_lt_base || !ray_off || !counts)
+    if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !ray_off || !counts)
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0) return GART_ERR_INVALID_ARG;
-    if (g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format == 1 && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // the 4-byte format serves the hybrid pass, which is tile-major
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
-    if (cap_pairs > 0 && (!pair_gid || !pair_mask || !pair_order || !rank_sid || !rank_mask || !rank_gstart || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
+    if (cam->width <= 0 || cam->height <= 0 || cam->width > 65535 * 8 || cam->height > 65535 * 8) return GART_ERR_INVALID_ARG;
+    if (cap_pairs > 0 && (!pair_gid || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0 && (!lt || (ray_gid == nullptr) != (ray_slot == nullptr))) return GART_ERR_INVALID_ARG;
-    if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
     const int ts = cfg->tile_size;
     const CamF cf = make_camf(cam, ts);
     const int T = cf.tiles_x * cf.tiles_y;
     const int64_t n_rays = (int64_t)cam->width * cam->height;
     ForwardWs w = forward_layout(workspace, n_rays, T, cap_pairs, cap_hits);
     if (w.bytes > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    const ViewLayout v = view_layout(view, g->n, cam->width, cam->height, ts, cap_pairs);
+    if (v.bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const int rs4 = rec_f4(g->sh_degree);
+    const int4* srect = reinterpret_cast<const int4*>(rec + (size_t)g->n * (rs4 + 2));   // the rectangles in slot order, behind the records
+    const bool gmaj = cfg->lt_layout == GART_LT_PRIMITIVE_MAJOR;
+    const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
+    gart_status s;
 
-    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, w.pair_sid, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, pair_mask, w.pair_sid, hit_count, counts);
+    // first primitive-major pair position of every slot (the mask kernel files every pair's mask there)
+    if (cudaMemsetAsync(v.info, 0, GM_INFO_WORDS * 4, st) != cudaSuccess) return GART_ERR_CUDA;
+    if (cudaMemsetAsync(v.st_off, 0, (size_t)(v.ns + 1) * 4, st) != cudaSuccess) return GART_ERR_CUDA;
+    // (a visible Gaussian has at least one pair: without a capacity error the slots in use number at most cap_pairs)
+    const int64_t nscan = g->n < cap_pairs ? g->n : cap_pairs;
+    if (nscan > 0) {
+        SlotTilesF tf{srect, counts, ts};
+        s = exclusive_scan(tf, nscan, v.gpair_off, w.total_gm, w.scan_ws, st);
+        if (s != GART_OK) return s;
+    }
+
+    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, v.gm_mask, v.pair_gpos, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, v.gm_mask, v.pair_gpos, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
-    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
-    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, pair_mask, T, pair_order, rank_sid, rank_mask, rank_gstart, w.tile_slots, counts);
+    // (in the primitive-major layout the evaluation looks the LT slot up by the pair's primitive-major position: the
+    // rank-ordered copy of those positions takes the place of the tile layout's group starts)
+    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, v.rank_gpos, w.tile_slots, counts);
+    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, v.rank_gpos, w.tile_slots, counts);
     GART_LAUNCH_CHECK();
 
-    TileSlotsF tf{w.tile_slots};
-    gart_status s = exclusive_scan(tf, (int64_t)T, tile_lt_base, w.total_slots, w.scan_ws, st);
+    TileSlotsF tsf{w.tile_slots};
+    s = exclusive_scan(tsf, (int64_t)T, v.tile_lt_base, w.total_slots, w.scan_ws, st);
     if (s != GART_OK) return s;
+
+    if (gmaj && nscan > 0) {
+        // items: one per Gaussian that fits a window, one per touched super-tile otherwise; grouped by owner
+        SlotItemsF itf{srect, counts};
+        s = exclusive_scan(itf, nscan, v.item_off, w.total_gm, w.scan_ws, st);
+        if (s != GART_OK) return s;
+        gm_items_total_kernel<<<1, 1, 0, st>>>(w.total_gm, cap_pairs, v.info, counts);
+        GART_LAUNCH_CHECK();
+        int bits = 1;
+        while ((1 << bits) < v.ns) ++bits;
+        uint32_t* const kbuf[2] = {w.ikeys0, w.ikeys1};
+        uint32_t* const vbuf[2] = {w.ivals0, w.ivals1};
+        const int cur = radix_passes(bits) & 1;   // after the passes the sorted arrays are at index 0
+        gm_emit_items_kernel<<<(unsigned)ceil_div(nscan, 256), 256, 0, st>>>(srect, v.item_off, sup_x, counts, kbuf[cur], vbuf[cur], v.em_slot);
+        GART_LAUNCH_CHECK();
+        s = radix_sort_pairs(kbuf, vbuf, cur, bits, cap_pairs, v.info + GM_INFO_ITEMS, 0u, counts + GART_CNT_ERROR, w.itable, w.scan_ws, w.total_gm, st);
+        if (s != GART_OK) return s;
+        const unsigned iblocks = (unsigned)ceil_div(cap_pairs, 256);
+        gm_segment_offsets_kernel<<<iblocks, 256, 0, st>>>(kbuf[0], v.info + GM_INFO_ITEMS, counts, v.ns, v.st_off);
+        GART_LAUNCH_CHECK();
+        if (ts == 8) gm_item_desc_kernel<8><<<iblocks, 256, 0, st>>>(kbuf[0], vbuf[0], v.em_slot, v.item_off, srect, v.gpair_off, v.gm_mask, sup_x, v.info, counts, v.it_desc);
+        else gm_item_desc_kernel<16><<<iblocks, 256, 0, st>>>(kbuf[0], vbuf[0], v.em_slot, v.item_off, srect, v.gpair_off, v.gm_mask, sup_x, v.info, counts, v.it_desc);
+        GART_LAUNCH_CHECK();
+        gm_rank_kernel<<<(unsigned)ceil_div(v.ns, GM_RANK_WARPS), GM_RANK_WARPS * 32, 0, st>>>(v.st_off, v.it_desc, v.ns, v.rk_desc, v.rk_gstart, v.st_len, v.st_parts, counts);
+        GART_LAUNCH_CHECK();
+        ArrayF lf{v.st_len};
+        s = exclusive_scan(lf, (int64_t)v.ns, v.st_lt_base, w.total_slots, w.scan_ws, st);   // the LT size of this layout replaces the tile layout's
+        if (s != GART_OK) return s;
+        ArrayF pf{v.st_parts};
+        s = exclusive_scan(pf, (int64_t)v.ns, v.blk_off, w.total_gm, w.scan_ws, st);
+        if (s != GART_OK) return s;
+        gm_blocks_kernel<<<(unsigned)ceil_div(v.ns, 256), 256, 0, st>>>(v.blk_off, v.st_parts, v.ns, v.blocks_cap, v.blk_desc, v.info, counts);
+        GART_LAUNCH_CHECK();
+        if (ts == 8) gm_ltb_kernel<8><<<(unsigned)ceil_div(v.ns, 4), 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, counts);
+        else gm_ltb_kernel<16><<<(unsigned)ceil_div(v.ns, 4), 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, counts);
+        GART_LAUNCH_CHECK();
+    }
+
     RayHitsF rf{hit_count, counts};
     s = exclusive_scan(rf, n_rays, ray_off, w.total_hits, w.scan_ws, st);
     if (s != GART_OK) return s;
     hits_total_kernel<<<1, 1, 0, st>>>(w.total_slots, w.total_hits, cap_hits, counts);
     GART_LAUNCH_CHECK();
 
-    if (ts == 8) s = launch_eval<8>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
-    else s = launch_eval<16>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, ray_off, cf, w, counts);
+    if (gmaj) {
+        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+    } else {
+        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+    }
     if (s != GART_OK) return s;
 
     const int64_t blocks = ceil_div((int64_t)T * ts * ts, SWEEP_WARPS);

@@ -20,15 +20,22 @@ LIB_PATH = os.path.join(_HERE, "libgart.so")
 
 GART_OK = 0
 STATUS_NAMES = {0: "GART_OK", 1: "GART_ERR_INVALID_ARG", 2: "GART_ERR_WORKSPACE_TOO_SMALL",
-                3: "GART_ERR_CAPACITY_EXCEEDED", 4: "GART_ERR_CUDA"}
+                3: "GART_ERR_CAPACITY_EXCEEDED", 4: "GART_ERR_CUDA", 5: "GART_ERR_TIMEOUT"}
+LT_PRIMITIVE_MAJOR, LT_TILE_MAJOR = 0, 1
+# names of the arrays inside the view block (gart_view_array): index, numpy-style dtype width in bytes, columns
+VIEW_ARRAYS = {"pair_mask": 0, "pair_order": 1, "rank_sid": 2, "rank_mask": 3, "rank_gstart": 4, "tile_lt_base": 5,
+               "pair_gpos": 6, "gpair_off": 7, "gm_mask": 8, "gm_ltb": 9, "item_desc": 10, "item_gstart": 11,
+               "st_off": 12, "st_lt_base": 13, "info": 14}
 CNT_VISIBLE, CNT_PAIRS, CNT_SLOTS_LO, CNT_SLOTS_HI, CNT_HITS, CNT_ERROR, CNT_MAX_RAY_HITS, CNT_STRADDLE, CNT_LT_SLOTS = range(9)
 COUNTS_WORDS = 12
 GRAD_WORDS = 64
 
 EXPORTS = [
     "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
-    "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_forward_workspace_bytes", "gart_forward",
-    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp", "gart_read_counts",
+    "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_view_bytes", "gart_view_array",
+    "gart_forward_workspace_bytes", "gart_forward",
+    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_tile", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp",
+    "gart_workspace_bytes", "gart_read_counts", "gart_sync_status",
     "gart_view_host_arena_bytes", "gart_view_host",
 ]
 
@@ -41,7 +48,7 @@ class GartError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
-                ("lt_format", C.c_int32), ("max_hits", C.c_int32)]
+                ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -82,19 +89,25 @@ def lib():
         L.gart_tile_map_static.restype = C.c_int
         L.gart_forward_workspace_bytes.restype = sz
         L.gart_forward_workspace_bytes.argtypes = [i32, i32, i32, i64, i64]
-        L.gart_forward.argtypes = [vp] * 8 + [i64] + [vp] * 10 + [i64] + [vp] * 5 + [sz, vp]
+        L.gart_view_bytes.restype = sz
+        L.gart_view_bytes.argtypes = [i64, i32, i32, i32, i64]
+        L.gart_view_array.argtypes = [i64, i32, i32, i32, i64, i32, C.POINTER(sz), C.POINTER(sz)]
+        L.gart_forward.argtypes = [vp] * 8 + [i64] + [vp] * 4 + [i64] + [vp] * 4 + [sz, vp, vp, sz, vp]
         L.gart_backward_workspace_bytes.restype = sz
         L.gart_backward_workspace_bytes.argtypes = [i64]
-        L.gart_backward.argtypes = [vp] * 16 + [sz, vp]
+        for fn in ("gart_backward", "gart_backward_tile", "gart_backward_warp"):
+            getattr(L, fn).argtypes = [vp] * 8 + [sz, i64] + [vp] * 5 + [sz, vp]
         L.gart_backward_atomic.argtypes = [vp] * 13
-        L.gart_backward_hybrid.argtypes = [vp] * 18 + [sz, vp]
-        L.gart_backward_warp.argtypes = [vp] * 16 + [sz, vp]
+        L.gart_backward_hybrid.argtypes = [vp] * 8 + [sz, i64] + [vp] * 7 + [sz, vp]
+        L.gart_workspace_bytes.restype = sz
+        L.gart_workspace_bytes.argtypes = [i64, i32, i32, i32, i64, i64]
         L.gart_read_counts.argtypes = [vp, vp, vp]
+        L.gart_sync_status.argtypes = [vp, vp, vp]
         L.gart_view_host_arena_bytes.restype = sz
         L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
         L.gart_view_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
-        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp",
-                   "gart_read_counts", "gart_view_host"):
+        for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_tile", "gart_backward_atomic",
+                   "gart_backward_hybrid", "gart_backward_warp", "gart_read_counts", "gart_sync_status", "gart_view_host", "gart_view_array"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -109,12 +122,14 @@ class Config:
     tile_size: int = 8
     lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid); 2: 8 bytes (gart_backward)
     max_hits: int = 0           # > 0: only the first max_hits hits of a ray are composited (0: all, the paper's setting)
+    lt_layout: int = 0          # 0: primitive-major LT (gart_backward); 1: tile-major (gart_backward_tile, _warp, _hybrid)
 
     def c(self) -> _Config:
         s = _Config()
         s.alpha_min, s.near_z, s.tile_size = self.alpha_min, self.near_z, int(self.tile_size)
         s.lt_format = int(self.lt_format)
         s.max_hits = int(self.max_hits)
+        s.lt_layout = int(self.lt_layout)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s
@@ -251,21 +266,38 @@ def gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits) 
     return int(lib().gart_forward_workspace_bytes(int(width), int(height), int(tile_size), int(cap_pairs), int(cap_hits)))
 
 
+def gart_workspace_bytes(n, width, height, tile_size, cap_pairs, cap_hits) -> int:
+    return int(lib().gart_workspace_bytes(int(n), int(width), int(height), int(tile_size), int(cap_pairs), int(cap_hits)))
+
+
+def gart_view_bytes(n, width, height, tile_size, cap_pairs) -> int:
+    return int(lib().gart_view_bytes(int(n), int(width), int(height), int(tile_size), int(cap_pairs)))
+
+
+def gart_view_array(n, width, height, tile_size, cap_pairs, name):
+    """(offset, bytes) of one named private array inside the view block (tests and diagnostics)."""
+    off, nb = C.c_size_t(0), C.c_size_t(0)
+    _check(lib().gart_view_array(int(n), int(width), int(height), int(tile_size), int(cap_pairs), VIEW_ARRAYS[name],
+                                 C.byref(off), C.byref(nb)), "gart_view_array")
+    return int(off.value), int(nb.value)
+
+
+def _view(view):
+    return _dev(view, torch.uint8, "view"), (view.numel() if view is not None else 0)
+
+
 def gart_forward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, pair_gid, cap_pairs, color,
-                 t_final, hit_count, pair_mask, pair_order, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, cap_hits,
-                 ray_off, ray_gid, ray_slot, counts, workspace, stream=None):
+                 t_final, hit_count, lt, cap_hits, ray_off, ray_gid, ray_slot, view, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     wp, wb = _ws(workspace)
+    vp, vb = _view(view)
     _check(lib().gart_forward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
                               _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
                               _dev(tile_off, i32, "tile_off"), _dev(pair_gid, i32, "pair_gid"), int(cap_pairs),
                               _dev(color, f32, "color"), _dev(t_final, f32, "t_final"), _dev(hit_count, i32, "hit_count"),
-                              _dev(pair_mask, i32, "pair_mask"), _dev(pair_order, i32, "pair_order"),
-                              _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
-                              _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
                               _dev(lt, f32, "lt"), int(cap_hits), _dev(ray_off, i32, "ray_off"),
-                              _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"),
+                              _dev(ray_gid, i32, "ray_gid"), _dev(ray_slot, i32, "ray_slot"), vp, vb,
                               _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_forward")
 
 
@@ -273,32 +305,35 @@ def gart_backward_workspace_bytes(n) -> int:
     return int(lib().gart_backward_workspace_bytes(int(n)))
 
 
-def gart_backward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
-                  rank_gstart, tile_lt_base, lt, dL_dcolor, grad, counts, workspace, stream=None):
+def _backward_call(name, cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor, grad, counts,
+                   workspace, stream):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     wp, wb = _ws(workspace)
-    _check(lib().gart_backward(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
-                               _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
-                               _dev(tile_off, i32, "tile_off"),
-                               _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
-                               _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
-                               _dev(lt, f32, "lt"), _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
-                               _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward")
+    vp, vb = _view(view)
+    _check(getattr(lib(), name)(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
+                                _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
+                                _dev(tile_off, i32, "tile_off"), vp, vb, int(cap_pairs),
+                                _dev(lt, f32, "lt"), _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
+                                _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), name)
 
 
-def gart_backward_warp(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
-                       rank_gstart, tile_lt_base, lt, dL_dcolor, grad, counts, workspace, stream=None):
-    c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
-    i32, f32 = torch.int32, torch.float32
-    wp, wb = _ws(workspace)
-    _check(lib().gart_backward_warp(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
-                                    _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
-                                    _dev(tile_off, i32, "tile_off"),
-                                    _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
-                                    _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
-                                    _dev(lt, f32, "lt"), _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
-                                    _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward_warp")
+def gart_backward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor,
+                  grad, counts, workspace, stream=None):
+    _backward_call("gart_backward", cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor, grad,
+                   counts, workspace, stream)
+
+
+def gart_backward_tile(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor,
+                       grad, counts, workspace, stream=None):
+    _backward_call("gart_backward_tile", cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor,
+                   grad, counts, workspace, stream)
+
+
+def gart_backward_warp(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor,
+                       grad, counts, workspace, stream=None):
+    _backward_call("gart_backward_warp", cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor,
+                   grad, counts, workspace, stream)
 
 
 def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, ray_off, ray_gid, ray_slot, lt, dL_dcolor,
@@ -312,16 +347,15 @@ def gart_backward_atomic(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, ray_o
                                       _dev(counts, i32, "counts"), _stream_ptr(stream)), "gart_backward_atomic")
 
 
-def gart_backward_hybrid(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, rank_sid, rank_mask,
-                         rank_gstart, tile_lt_base, lt_w, ray_off, ray_gid, dL_dcolor, grad, counts, workspace, stream=None):
+def gart_backward_hybrid(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt_w, ray_off,
+                         ray_gid, dL_dcolor, grad, counts, workspace, stream=None):
     c, gs, cs = cfg.c(), g.c(), camera_struct(cam)
     i32, f32 = torch.int32, torch.float32
     wp, wb = _ws(workspace)
+    vp, vb = _view(view)
     _check(lib().gart_backward_hybrid(C.byref(c), C.byref(gs), C.byref(cs), _dev(pre, f32, "pre"),
                                       _dev(slot_of_gid, i32, "slot_of_gid"), _dev(gid_of_slot, i32, "gid_of_slot"),
-                                      _dev(tile_off, i32, "tile_off"),
-                                      _dev(rank_sid, i32, "rank_sid"), _dev(rank_mask, i32, "rank_mask"),
-                                      _dev(rank_gstart, i32, "rank_gstart"), _dev(tile_lt_base, i32, "tile_lt_base"),
+                                      _dev(tile_off, i32, "tile_off"), vp, vb, int(cap_pairs),
                                       _dev(lt_w, f32, "lt_w"), _dev(ray_off, i32, "ray_off"), _dev(ray_gid, i32, "ray_gid"),
                                       _dev(dL_dcolor, f32, "dL_dcolor"), _dev(grad, f32, "grad"),
                                       _dev(counts, i32, "counts"), wp, wb, _stream_ptr(stream)), "gart_backward_hybrid")
@@ -332,6 +366,11 @@ def gart_read_counts(counts, stream=None):
     host = (C.c_uint32 * COUNTS_WORDS)()
     _check(lib().gart_read_counts(_dev(counts, torch.int32, "counts"), host, _stream_ptr(stream)), "gart_read_counts")
     return [int(v) for v in host]
+
+
+def gart_sync_status(counts, stream=None) -> int:
+    """Reads the counts block (synchronises the stream) and returns its error word as a status code."""
+    return int(lib().gart_sync_status(_dev(counts, torch.int32, "counts"), None, _stream_ptr(stream)))
 
 
 def gart_view_host_arena_bytes(n, sh_degree, width, height, tile_size, cap_pairs, cap_hits) -> int:
@@ -382,16 +421,18 @@ class ViewBuffers:
         self.slot_of_gid, self.gid_of_slot = e((n1,), i32), e((n1,), i32)
         self.counts = torch.zeros(COUNTS_WORDS, dtype=i32, device=device)
         self.tile_off, self.pair_gid = e((T + 1,), i32), e((cp,), i32)
-        self.pair_mask, self.pair_order = e((cp, mw), i32), e((cp,), i32)
-        self.rank_sid, self.rank_mask, self.rank_gstart = e((cp,), i32), e((cp, mw), i32), e((cp,), i32)
-        self.tile_lt_base = e((T + 1,), i32)
+        self._geom = (n1, W, H, ts, self.cap_pairs)
+        self.view = e((gart_view_bytes(*self._geom),), u8)
         self.color, self.t_final, self.hit_count = e((H, W, 3), f32), e((H, W), f32), e((H, W), i32)
         self.lt = e((ch, 4), f32)
         self.ray_off, self.ray_gid, self.ray_slot = e((H * W + 1,), i32), e((ch,), i32), e((ch,), i32)
         self.grad = e((n1, GRAD_WORDS), f32)
-        ws = max(gart_bounds_workspace_bytes(n1), gart_tile_map_workspace_bytes(n1, W, H, ts, cap_pairs),
-                 gart_forward_workspace_bytes(W, H, ts, cap_pairs, cap_hits), gart_backward_workspace_bytes(n1))
-        self.workspace = e((ws,), u8)
+        self.workspace = e((gart_workspace_bytes(n1, W, H, ts, cap_pairs, cap_hits),), u8)
+
+    def view_array(self, name):
+        """One named private array of the view block as an int32 tensor (a view into the block; tests and diagnostics)."""
+        off, nb = gart_view_array(*self._geom, name)
+        return self.view[off:off + nb].view(torch.int32)
 
     def bytes(self):
         return sum(t.numel() * t.element_size() for t in vars(self).values() if isinstance(t, torch.Tensor))
@@ -405,20 +446,24 @@ def run_bounds_tile_map(cfg, g, cam, buf: ViewBuffers, stream=None):
 def run_forward(cfg, g, cam, buf: ViewBuffers, stream=None, ray_lists=True):
     """ray_lists=False skips the per-ray ordered hit lists (needed only by the atomic baseline and by parity checks)."""
     gart_forward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.pair_gid, buf.cap_pairs, buf.color,
-                 buf.t_final, buf.hit_count, buf.pair_mask, buf.pair_order, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
-                 buf.tile_lt_base, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid if ray_lists else None,
-                 buf.ray_slot if ray_lists else None, buf.counts, buf.workspace, stream)
+                 buf.t_final, buf.hit_count, buf.lt, buf.cap_hits, buf.ray_off, buf.ray_gid if ray_lists else None,
+                 buf.ray_slot if ray_lists else None, buf.view, buf.counts, buf.workspace, stream)
 
 
 def run_backward(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
-    gart_backward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask, buf.rank_gstart,
-                  buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
+    gart_backward(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.view, buf.cap_pairs, buf.lt, dL_dcolor,
+                  buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
+
+
+def run_backward_tile(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
+    """cfg.lt_layout must be LT_TILE_MAJOR and the forward must have run with the same cfg."""
+    gart_backward_tile(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.view, buf.cap_pairs, buf.lt,
+                       dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
 
 
 def run_backward_warp(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
-    gart_backward_warp(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask,
-                       buf.rank_gstart, buf.tile_lt_base, buf.lt, dL_dcolor, buf.grad if grad is None else grad, buf.counts,
-                       buf.workspace, stream)
+    gart_backward_warp(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.view, buf.cap_pairs, buf.lt,
+                       dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
 
 
 def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=None):
@@ -427,10 +472,9 @@ def run_backward_atomic(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad, stream=N
 
 
 def run_backward_hybrid(cfg, g, cam, buf: ViewBuffers, dL_dcolor, grad=None, stream=None):
-    """cfg.lt_format must be 1 and the forward must have run with the same cfg and with the ray lists."""
-    gart_backward_hybrid(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.rank_sid, buf.rank_mask,
-                         buf.rank_gstart, buf.tile_lt_base, buf.lt, buf.ray_off, buf.ray_gid, dL_dcolor,
-                         buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
+    """cfg.lt_format must be 1, cfg.lt_layout LT_TILE_MAJOR, and the forward must have run with the same cfg and the ray lists."""
+    gart_backward_hybrid(cfg, g, cam, buf.pre, buf.slot_of_gid, buf.gid_of_slot, buf.tile_off, buf.view, buf.cap_pairs, buf.lt,
+                         buf.ray_off, buf.ray_gid, dL_dcolor, buf.grad if grad is None else grad, buf.counts, buf.workspace, stream)
 
 
 def size_view(cfg, g, cam, slack=1.0, device="cuda"):
@@ -443,5 +487,8 @@ def size_view(cfg, g, cam, slack=1.0, device="cuda"):
     cnt = gart_read_counts(probe.counts)
     P = cnt[CNT_PAIRS]
     S = cnt[CNT_SLOTS_LO] | (cnt[CNT_SLOTS_HI] << 32)
-    pad = 32 * cfg.tile_size ** 2 * min(tiles(cam, cfg.tile_size), P)
+    # padding of the interleaved layouts: a tile pads by less than 32 x its largest hit count (tile_size^2 at most), a
+    # super-tile of the primitive-major layout by less than 32 x 1024 (the exact need is the LT_SLOTS count after the forward)
+    ns = -(-int(cam.width) // 16) * -(-int(cam.height) // 16)
+    pad = max(32 * cfg.tile_size ** 2 * min(tiles(cam, cfg.tile_size), P), 32 * 1024 * min(ns, P))
     return int(P * slack) + 1, int(S * slack) + pad + 1

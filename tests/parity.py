@@ -32,14 +32,33 @@ def u32(a):
     return a.view(np.uint32) if a.dtype == np.int32 else a
 
 
+def _view_arrays(buf, names, P, mw):
+    out = {}
+    for nme in names:
+        a = u32(to_np(buf.view_array(nme)))
+        if nme in ("pair_mask", "rank_mask", "gm_mask"):
+            a = a.reshape(-1, mw)[:P]
+        elif nme == "item_desc":
+            a = a.reshape(-1, 4)
+        elif nme in ("pair_order", "rank_sid", "rank_gstart", "pair_gpos", "gm_ltb"):
+            a = a[:P]
+        out[nme] = a.copy()
+    return out
+
+
 def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, atomic=True):
-    """Full device path for one view; returns numpy copies of every output."""
+    """Full device path for one view; returns numpy copies of every output.  The view runs in the primitive-major LT
+    layout (gart_backward); with atomic=True the other backward variants follow: the pixel-centric baseline on the
+    same buffers, then the forward again in the tile-major layout for the block-per-tile pass, the warp-per-pair pass
+    and the hybrid pass, and the forward with 8-byte entries for gart_backward on them."""
+    import dataclasses
     g = G.Gaussians.from_numpy(scene)
     if cap_pairs is None or cap_hits is None:
         P, S = G.size_view(cfg, g, cam, slack=1.0)
         cap_pairs = P if cap_pairs is None else cap_pairs
         cap_hits = S if cap_hits is None else cap_hits
     buf = G.ViewBuffers(g.n, g.sh_degree, cam, cfg, cap_pairs, cap_hits)
+    buf.grad.fill_(float("nan"))          # every record must be written by the backward pass
     dl = torch.from_numpy(np.ascontiguousarray(dL_dC, dtype=np.float32)).cuda()
     G.run_bounds_tile_map(cfg, g, cam, buf)
     G.run_forward(cfg, g, cam, buf)
@@ -47,18 +66,15 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
     counts = G.gart_read_counts(buf.counts)
     out = {"counts": counts, "buf": buf, "g": g, "dl": dl}
     P, H = counts[G.CNT_PAIRS], counts[G.CNT_HITS]
+    mw = cfg.tile_size ** 2 // 32
     out["rect"], out["cls"] = to_np(buf.rect)[:g.n], to_np(buf.cls)[:g.n]
     out["tile_off"] = u32(to_np(buf.tile_off))
     if counts[G.CNT_ERROR]:
         return out
     out["pair_gid"] = u32(to_np(buf.pair_gid))[:P]
-    out["pair_mask"] = u32(to_np(buf.pair_mask))[:P]
-    out["pair_order"] = u32(to_np(buf.pair_order))[:P]
-    out["rank_sid"] = u32(to_np(buf.rank_sid))[:P]
     out["slot_of_gid"], out["gid_of_slot"] = u32(to_np(buf.slot_of_gid))[:g.n], u32(to_np(buf.gid_of_slot))[:g.n]
-    out["rank_mask"] = u32(to_np(buf.rank_mask))[:P]
-    out["rank_gstart"] = u32(to_np(buf.rank_gstart))[:P]
-    out["tile_lt_base"] = u32(to_np(buf.tile_lt_base))
+    out.update(_view_arrays(buf, ["pair_mask", "pair_order", "rank_sid", "rank_mask", "pair_gpos", "gpair_off", "gm_mask", "gm_ltb",
+                                  "item_desc", "item_gstart", "st_off", "st_lt_base", "info"], P, mw))
     out["color"], out["t_final"] = to_np(buf.color), to_np(buf.t_final)
     out["hit_count"] = u32(to_np(buf.hit_count))
     out["ray_off"] = u32(to_np(buf.ray_off))
@@ -67,30 +83,48 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
     out["lt"] = to_np(buf.lt)[:counts[G.CNT_LT_SLOTS]]
     out["grad"] = to_np(buf.grad)[:g.n].copy()
     if atomic:
-        ga = torch.empty_like(buf.grad)
+        ga = torch.full_like(buf.grad, float("nan"))
         G.run_backward_atomic(cfg, g, cam, buf, dl, ga)
         torch.cuda.synchronize()
         out["grad_atomic"] = to_np(ga)[:g.n]
-        gw = torch.empty_like(buf.grad)
-        G.run_backward_warp(cfg, g, cam, buf, dl, gw)          # ownership ablation: a warp per pair
-        torch.cuda.synchronize()
-        out["grad_warp"] = to_np(gw)[:g.n]
-        import dataclasses
+        # ---- tile-major layout: block-per-tile pass and warp-per-pair pass (same buffers, the forward again)
+        cfg_t = dataclasses.replace(cfg, lt_layout=G.LT_TILE_MAJOR)
+        G.run_forward(cfg_t, g, cam, buf)
+        for key, fn in (("grad_tile", G.run_backward_tile), ("grad_warp", G.run_backward_warp)):
+            gt = torch.full_like(buf.grad, float("nan"))
+            fn(cfg_t, g, cam, buf, dl, gt)
+            torch.cuda.synchronize()
+            out[key] = to_np(gt)[:g.n]
+        ct = G.gart_read_counts(buf.counts)
+        assert ct[G.CNT_ERROR] == 0 and ct[G.CNT_HITS] == H
+        tile = _view_arrays(buf, ["pair_mask", "pair_order", "rank_sid", "rank_mask", "rank_gstart", "tile_lt_base"], P, mw)
+        tile["ray_slot"] = u32(to_np(buf.ray_slot))[:H].copy()
+        tile["lt"] = to_np(buf.lt)[:ct[G.CNT_LT_SLOTS]].copy()
+        tile["lt_slots"] = ct[G.CNT_LT_SLOTS]
+        out["tile"] = tile
+        # the other outputs of the forward do not depend on the LT layout
+        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
+        assert np.array_equal(tile["pair_mask"], out["pair_mask"])
         if cfg.max_hits == 0:   # (the hybrid backward re-derives every alpha in its pixel pass: it takes no hit cap)
-            # hybrid backward: the forward again with 4-byte LT entries (same buffers, everything else unchanged)
-            cfg_h = dataclasses.replace(cfg, lt_format=1)
+            # hybrid backward: the forward again with 4-byte LT entries
+            cfg_h = dataclasses.replace(cfg_t, lt_format=1)
             G.run_forward(cfg_h, g, cam, buf)
-            gh = torch.empty_like(buf.grad)
+            gh = torch.full_like(buf.grad, float("nan"))
             G.run_backward_hybrid(cfg_h, g, cam, buf, dl, gh)
             torch.cuda.synchronize()
             assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
             out["grad_hybrid"] = to_np(gh)[:g.n]
-            # the other outputs of the forward do not depend on the LT format
             assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
-        # 8-byte LT entries (four halves per hit) and the primitive-centric backward on them
+        # 8-byte LT entries (four halves per hit): gart_backward on them (primitive-major) and the block-per-tile pass
+        cfg_8t = dataclasses.replace(cfg_t, lt_format=2)
+        G.run_forward(cfg_8t, g, cam, buf)
+        g8 = torch.full_like(buf.grad, float("nan"))
+        G.run_backward_tile(cfg_8t, g, cam, buf, dl, g8)
+        torch.cuda.synchronize()
+        out["grad_lt16_tile"] = to_np(g8)[:g.n]
         cfg_8 = dataclasses.replace(cfg, lt_format=2)
         G.run_forward(cfg_8, g, cam, buf)
-        g8 = torch.empty_like(buf.grad)
+        g8 = torch.full_like(buf.grad, float("nan"))
         G.run_backward(cfg_8, g, cam, buf, dl, g8)
         torch.cuda.synchronize()
         assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
@@ -121,11 +155,57 @@ def check_maps(scene, cam, cfg: G.Config, gpu):
     return {"rect_identical": bool(same), "n_unsafe": int((~safe).sum()), "osc": osc}
 
 
+SUP = 16   # super-tile edge of the primitive-major order, pixels
+
+
+def _sample_hits(cam, gpu, max_rays, seed):
+    """(rays, index into the per-ray lists) of every hit, or of the hits of a random subset of rays on large views."""
+    H = gpu["counts"][G.CNT_HITS]
+    ray_off, hit_count = gpu["ray_off"].astype(np.int64), gpu["hit_count"].reshape(-1).astype(np.int64)
+    n_rays = hit_count.size
+    if H > 5_000_000:
+        rsel = np.sort(np.random.default_rng(seed).choice(n_rays, size=max_rays, replace=False))
+    else:
+        rsel = np.arange(n_rays)
+    cnt = hit_count[rsel]
+    idx = np.repeat(ray_off[rsel], cnt) + (np.arange(cnt.sum()) - np.repeat(np.cumsum(cnt) - cnt, cnt))
+    return np.repeat(rsel, cnt), idx
+
+
+def _locate_pairs(cam, cfg, gpu, rays, gids):
+    """Pair index (in the tile-major pair list) of every (ray, Gaussian) hit, and the hit's index among the set bits of the
+    pair's mask (pixel order)."""
+    ts = cfg.tile_size
+    tiles_x = -(-cam.width // ts)
+    tile_off = gpu["tile_off"].astype(np.int64)
+    n_tile = np.diff(tile_off)
+    tile_of_pair = np.repeat(np.arange(n_tile.size), n_tile)
+    tile = (rays // cam.width) // ts * tiles_x + (rays % cam.width) // ts
+    pair_gid = gpu["pair_gid"].astype(np.int64)
+    P = pair_gid.size
+    mul = int(pair_gid.max()) + 1 if P else 1
+    key = tile_of_pair * mul + pair_gid                      # ascending: ids ascend inside a tile
+    want = tile * mul + gids
+    pair = np.searchsorted(key, want)
+    assert np.array_equal(key[pair], want)
+    px = (rays % cam.width) % ts + ((rays // cam.width) % ts) * ts
+    words = gpu["pair_mask"][pair]                                  # [h, MW]
+    w_idx, b_idx = px // 32, px % 32
+    word = words[np.arange(pair.size), w_idx].astype(np.uint64)
+    assert np.all((word >> b_idx.astype(np.uint64)) & np.uint64(1))   # the hit pixel is set in the pair's mask
+    below = np.bitwise_count(word & ((np.uint64(1) << b_idx.astype(np.uint64)) - np.uint64(1))).astype(np.int64)
+    for q in range(words.shape[1]):
+        below += np.where(q < w_idx, np.bitwise_count(words[:, q]).astype(np.int64), 0)
+    return pair, below, tile
+
+
 def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
-    """Properties that hold at any size, checked on the whole view without the oracle (the per-hit
-    part on a random subset of rays when the view has more than a few million hits)."""
+    """Properties that hold at any size, checked on the whole view without the oracle (the per-hit part on a random
+    subset of rays when the view has more than a few million hits): ray offsets, hit masks, slot numbering, and the
+    primitive-major work lists and LT layout re-derived in numpy from rectangles and masks."""
     H = gpu["counts"][G.CNT_HITS]
     L = gpu["counts"][G.CNT_LT_SLOTS]
+    ts = cfg.tile_size
     ray_off, hit_count = gpu["ray_off"].astype(np.int64), gpu["hit_count"].reshape(-1).astype(np.int64)
     assert ray_off[0] == 0 and ray_off[-1] == H and np.array_equal(np.diff(ray_off), hit_count)
     assert gpu["counts"][G.CNT_MAX_RAY_HITS] == (hit_count.max() if hit_count.size else 0)
@@ -134,15 +214,118 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     # every hit owns exactly one slot
     slots_all = gpu["ray_slot"]
     assert np.unique(slots_all).size == H and (int(slots_all.max()) if H else -1) < L
-    ts = cfg.tile_size
+    P = pc.size
+    # ---- slots: visible Gaussians in the order of the super-tile of their rectangle's corner, ids ascending inside one
+    rect_ = gpu["rect"].astype(np.int64)
+    vis = rect_[:, 2] >= rect_[:, 0]
+    V = int(vis.sum())
+    sup_x = -(-cam.width // SUP)
+    key_ = (rect_[:, 1] // SUP) * sup_x + rect_[:, 0] // SUP
+    want_order = np.nonzero(vis)[0][np.argsort(key_[vis], kind="stable")]
+    assert np.array_equal(gpu["gid_of_slot"][:V], want_order.astype(np.uint32)) and np.all(gpu["gid_of_slot"][V:] == 0xffffffff)
+    inv = np.full(rect_.shape[0], 0xffffffff, np.uint32)
+    inv[want_order] = np.arange(V, dtype=np.uint32)
+    assert np.array_equal(gpu["slot_of_gid"], inv)
+    # ---- primitive-major pair positions: a slot's tiles row by row
+    r = rect_[want_order]                                          # rectangles in slot order
+    tx0, ty0, tx1, ty1 = r[:, 0] // ts, r[:, 1] // ts, r[:, 2] // ts, r[:, 3] // ts
+    ntx, nty = tx1 - tx0 + 1, ty1 - ty0 + 1
+    gpo = np.concatenate([[0], np.cumsum(ntx * nty)])
+    assert gpo[-1] == P and np.array_equal(gpu["gpair_off"][:V + 1].astype(np.int64), gpo)
     tiles_x = -(-cam.width // ts)
-    tile_off, base = gpu["tile_off"].astype(np.int64), gpu["tile_lt_base"].astype(np.int64)
+    tile_off = gpu["tile_off"].astype(np.int64)
+    tile_of_pair = np.repeat(np.arange(tile_off.size - 1), np.diff(tile_off))
+    sl = gpu["slot_of_gid"][gpu["pair_gid"]].astype(np.int64)
+    ptx, pty = tile_of_pair % tiles_x, tile_of_pair // tiles_x
+    gpos = gpo[sl] + (pty - ty0[sl]) * ntx[sl] + (ptx - tx0[sl])
+    assert np.array_equal(gpu["pair_gpos"].astype(np.int64), gpos) and np.unique(gpos).size == P
+    assert np.array_equal(gpu["gm_mask"][gpos], gpu["pair_mask"])
+    pc_g = np.empty(P, np.int64)
+    pc_g[gpos] = pc                                                # hits per pair, by primitive-major position
+    # ---- work items: a Gaussian spanning at most two super-tiles per axis is one item owned by the super-tile of its
+    # corner, any other is cut into one item per super-tile it touches; emission order = slot order, pieces row by row
+    sx0, sy0, sx1, sy1 = r[:, 0] // SUP, r[:, 1] // SUP, r[:, 2] // SUP, r[:, 3] // SUP
+    whole = ((sx1 - sx0) <= 1) & ((sy1 - sy0) <= 1)
+    nsx = np.where(whole, 1, sx1 - sx0 + 1)
+    n_it = np.where(whole, 1, (sx1 - sx0 + 1) * (sy1 - sy0 + 1))
+    I = int(n_it.sum())
+    assert gpu["info"][0] == I
+    it_slot = np.repeat(np.arange(V), n_it)
+    local = np.arange(I) - np.repeat(np.cumsum(n_it) - n_it, n_it)
+    it_sx, it_sy = sx0[it_slot] + local % nsx[it_slot], sy0[it_slot] + local // nsx[it_slot]
+    it_whole = whole[it_slot]
+    tps = SUP // ts                                                # tiles per super-tile edge
+    fx = np.where(it_whole, tx0[it_slot], np.maximum(tx0[it_slot], it_sx * tps))
+    lx = np.where(it_whole, tx1[it_slot], np.minimum(tx1[it_slot], it_sx * tps + tps - 1))
+    fy = np.where(it_whole, ty0[it_slot], np.maximum(ty0[it_slot], it_sy * tps))
+    ly = np.where(it_whole, ty1[it_slot], np.minimum(ty1[it_slot], it_sy * tps + tps - 1))
+    it_ntx, it_nty = lx - fx + 1, ly - fy + 1
+    gpos0 = gpo[it_slot] + (fy - ty0[it_slot]) * ntx[it_slot] + (fx - tx0[it_slot])
+    # hits per item and, per pair of an item, the hits of the item's earlier pairs
+    npair = it_ntx * it_nty
+    pi = np.repeat(np.arange(I), npair)
+    kk = np.arange(npair.sum()) - np.repeat(np.cumsum(npair) - npair, npair)
+    pg = gpos0[pi] + (kk // it_ntx[pi]) * ntx[it_slot][pi] + kk % it_ntx[pi]      # primitive-major position of the item's k-th pair
+    assert np.unique(pg).size == P                                  # the items partition the pairs
+    it_cnt = np.bincount(pi, weights=pc_g[pg], minlength=I).astype(np.int64)
+    csum = np.cumsum(pc_g[pg]) - pc_g[pg]
+    before = csum - np.repeat((np.cumsum(it_cnt) - it_cnt), npair)
+    S_own = it_sy * sup_x + it_sx
+    NS = sup_x * -(-cam.height // SUP)
+    order = np.lexsort((np.arange(I), -it_cnt, S_own))              # by super-tile, then descending hits, stable
+    st_off = np.concatenate([[0], np.cumsum(np.bincount(S_own, minlength=NS))])
+    assert np.array_equal(gpu["st_off"].astype(np.int64), st_off)
+    desc = gpu["item_desc"][:I].astype(np.int64)
+    assert np.array_equal(desc[:, 0], it_slot[order]) and np.array_equal(desc[:, 1], gpos0[order])
+    dims = ntx[it_slot] | (it_ntx << 16) | (it_nty << 20) | ((fx - it_sx * tps) << 24) | ((fy - it_sy * tps) << 28)
+    assert np.array_equal(desc[:, 2], dims[order])
+    assert np.array_equal(desc[:, 3], (it_cnt | (it_whole.astype(np.int64) << 16))[order])
+    # groups of 32 ranks inside a super-tile occupy 32 x (largest count) entries
+    So, co = S_own[order], it_cnt[order]
+    rank = np.arange(I) - st_off[So]
+    first = rank % 32 == 0
+    gsize = 32 * co[first]
+    gS = So[first]
+    gstart = np.cumsum(gsize) - gsize                               # super-tiles are laid out one after the other
+    assert np.array_equal(gpu["item_gstart"][:I].astype(np.int64), np.repeat(gstart, np.diff(np.r_[np.nonzero(first)[0], I])))
+    st_len = np.bincount(gS, weights=gsize, minlength=NS).astype(np.int64)
+    assert np.array_equal(gpu["st_lt_base"].astype(np.int64), np.concatenate([[0], np.cumsum(st_len)])) and st_len.sum() == L
+    # first LT entry of every pair
+    pos_of_item = np.empty(I, np.int64)
+    pos_of_item[order] = np.arange(I)
+    g_of_item = gpu["item_gstart"][:I].astype(np.int64)[pos_of_item]
+    ltb = np.empty(P, np.int64)
+    ltb[pg] = g_of_item[pi] + rank[pos_of_item][pi] % 32 + 32 * before
+    assert np.array_equal(gpu["gm_ltb"].astype(np.int64), ltb)
+    # ---- per hit: on all rays, or on a random subset of them
+    rays, idx = _sample_hits(cam, gpu, max_rays, seed)
+    slots = gpu["ray_slot"][idx].astype(np.int64)
+    gids = gpu["ray_gid"][idx].astype(np.int64)
+    pair, below, _ = _locate_pairs(cam, cfg, gpu, rays, gids)
+    assert np.array_equal(slots, ltb[gpos[pair]] + 32 * below)      # the e-th hit of a pair: its e-th set mask bit in pixel order
+    # LT: word 3 is the blending weight T alpha in (0, 1) with the three clamp flags in its low mantissa
+    # bits; the vector part is finite.  (The values themselves are checked against the oracle's entries.)
+    used = gpu["lt"][slots]
+    wgt = (np.ascontiguousarray(used[:, 3]).view(np.uint32) & np.uint32(0xFFFFFFF8)).view(np.float32)
+    assert np.all(np.isfinite(used)) and np.all(wgt >= 0) and np.all(wgt < 1.0)
+    assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
+    return {"items": I, "whole_share": float(whole.mean()) if V else 1.0, "lt_padding": float(L) / max(H, 1)}
+
+
+def check_structure_tile(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
+    """The tile-major work lists and LT layout (the forward run with lt_layout = tile-major: gpu["tile"])."""
+    t = gpu["tile"]
+    H, L = gpu["counts"][G.CNT_HITS], t["lt_slots"]
+    pc = np.bitwise_count(t["pair_mask"]).sum(axis=1).astype(np.int64)
+    slots_all = t["ray_slot"]
+    assert np.unique(slots_all).size == H and (int(slots_all.max()) if H else -1) < L and L >= H
+    tile_off, base = gpu["tile_off"].astype(np.int64), t["tile_lt_base"].astype(np.int64)
     assert base[0] == 0 and base[-1] == L and np.all(np.diff(base) >= 0)
     n_tile = np.diff(tile_off)
     P = pc.size
     tile_of_pair = np.repeat(np.arange(n_tile.size), n_tile)
     # pair_order: a permutation of each tile's pairs in descending hit count, stable
-    order = gpu["pair_order"].astype(np.int64)
+    order = t["pair_order"].astype(np.int64)
     seen = np.zeros(P, bool)
     seen[order] = True
     assert seen.all()
@@ -153,20 +336,10 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     assert np.all((po[:-1] >= po[1:]) | ~same_tile)
     assert np.all((order[:-1] < order[1:]) | (po[:-1] != po[1:]) | ~same_tile)
     # copies in rank order
-    assert np.array_equal(gpu["rank_sid"], gpu["slot_of_gid"][gpu["pair_gid"][order]])
-    assert np.array_equal(gpu["rank_mask"], gpu["pair_mask"][order])
-    # slots: visible Gaussians in the order of the tile row of their rectangle's corner, ids ascending inside a row
-    rect_ = gpu["rect"]
-    vis = rect_[:, 2] >= rect_[:, 0]
-    V = int(vis.sum())
-    key_ = rect_[:, 1] // ts
-    want_order = np.nonzero(vis)[0][np.argsort(key_[vis], kind="stable")]
-    assert np.array_equal(gpu["gid_of_slot"][:V], want_order.astype(np.uint32)) and np.all(gpu["gid_of_slot"][V:] == 0xffffffff)
-    inv = np.full(rect_.shape[0], 0xffffffff, np.uint32)
-    inv[want_order] = np.arange(V, dtype=np.uint32)
-    assert np.array_equal(gpu["slot_of_gid"], inv)
+    assert np.array_equal(t["rank_sid"], gpu["slot_of_gid"][gpu["pair_gid"][order]])
+    assert np.array_equal(t["rank_mask"], t["pair_mask"][order])
     # rank_gstart: start of the 32-rank group; a group spans 32 x its largest (= first) count
-    gs_ = gpu["rank_gstart"].astype(np.int64)                   # by position in rank order
+    gs_ = t["rank_gstart"].astype(np.int64)                   # by position in rank order
     first = rank % 32 == 0
     grp_start, grp_tile, grp_size = gs_[first], tile_of_pair[first], 32 * po[first]
     assert np.array_equal(np.repeat(grp_start, np.diff(np.r_[np.nonzero(first)[0], P])), gs_)
@@ -179,45 +352,15 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     tile_len = np.zeros(n_tile.size, np.int64)
     tile_len[grp_tile[last_of_tile]] = (grp_start + grp_size)[last_of_tile]
     assert np.array_equal(tile_len, np.diff(base))
-    # ---- per hit: on all rays, or on a random subset of them
-    n_rays = hit_count.size
-    if H > 5_000_000:
-        rsel = np.sort(np.random.default_rng(seed).choice(n_rays, size=max_rays, replace=False))
-    else:
-        rsel = np.arange(n_rays)
-    cnt = hit_count[rsel]
-    idx = np.repeat(ray_off[rsel], cnt) + (np.arange(cnt.sum()) - np.repeat(np.cumsum(cnt) - cnt, cnt))
-    rays = np.repeat(rsel, cnt)
-    slots = gpu["ray_slot"][idx].astype(np.int64)
+    rays, idx = _sample_hits(cam, gpu, max_rays, seed)
+    slots = t["ray_slot"][idx].astype(np.int64)
     gids = gpu["ray_gid"][idx].astype(np.int64)
-    tile = (rays // cam.width) // ts * tiles_x + (rays % cam.width) // ts
+    pair, below, tile = _locate_pairs(cam, cfg, gpu, rays, gids)
     rel = slots - base[tile]
     assert np.all(rel >= 0) and np.all(slots < base[tile + 1])
-    # locate the pair: among the tile's pairs, the one whose Gaussian is the hit's (ids ascend in a tile)
-    pair_gid = gpu["pair_gid"].astype(np.int64)
-    mul = int(pair_gid.max()) + 1 if P else 1
-    key = tile_of_pair * mul + pair_gid
-    want = tile * mul + gids
-    pair = np.searchsorted(key, want)
-    assert np.array_equal(key[pair], want)
-    e = rel - slot0[pair]
-    assert np.all(e % 32 == 0) and np.all(e >= 0) and np.all(e // 32 < pc[pair])
-    # the e-th hit of a pair is its e-th set mask bit in pixel order
-    px = (rays % cam.width) % ts + ((rays // cam.width) % ts) * ts
-    words = gpu["pair_mask"][pair]                                  # [h, MW]
-    w_idx, b_idx = px // 32, px % 32
-    word = words[np.arange(pair.size), w_idx].astype(np.uint64)
-    assert np.all((word >> b_idx.astype(np.uint64)) & np.uint64(1))
-    below = np.bitwise_count(word & ((np.uint64(1) << b_idx.astype(np.uint64)) - np.uint64(1))).astype(np.int64)
-    for q in range(words.shape[1]):
-        below += np.where(q < w_idx, np.bitwise_count(words[:, q]).astype(np.int64), 0)
-    assert np.array_equal(below, e // 32)
-    # LT: word 3 is the blending weight T alpha in (0, 1) with the three clamp flags in its low mantissa
-    # bits; the vector part is finite.  (The values themselves are checked through the gradients.)
-    used = gpu["lt"][slots]
-    wgt = (np.ascontiguousarray(used[:, 3]).view(np.uint32) & np.uint32(0xFFFFFFF8)).view(np.float32)
-    assert np.all(np.isfinite(used)) and np.all(wgt >= 0) and np.all(wgt < 1.0)
-    assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
+    assert np.array_equal(rel, slot0[pair] + 32 * below)
+    # the entries are the same numbers in both layouts
+    assert np.array_equal(t["lt"][slots], gpu["lt"][gpu["ray_slot"][idx].astype(np.int64)])
 
 
 def _lists_for(ray_off, gid, rays):
