@@ -443,7 +443,8 @@ def run_ours(args):
                    "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "views": len(cams), "crop": args.crop,
                    "l2": "inputs larger than L2 (parameters %.2f GB, LT %.2f GB per view)" % (
                        4e-9 * scene.n * (11 + 3 * K), 16e-9 * Hm),
-                   "hits_per_view": Hm, "pairs_per_view": Pm, "visible_per_view": Nv},
+                   "hits_per_view": Hm, "pairs_per_view": Pm, "visible_per_view": Nv,
+                   "lt_entries_per_view": float(np.mean(cl[:, G.CNT_LT_SLOTS]))},
         "stages_ms": {"bounds_tile_map": float(np.mean(stage[:, 0])), "forward": float(np.mean(stage[:, 1])),
                       "backward": bwd_ms, "backward_median": float(np.median(stage[:, 2]))},
         "backward_hits_per_s": Hm / (bwd_ms * 1e-3),

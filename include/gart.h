@@ -248,15 +248,17 @@ gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t ti
  *              nearest to 4096 w.  A decoded colour word is within 2^-10 (relative) of the fp32 value, the
  *              weight within 2^-11; magnitudes below 2^-26 lose relative precision, below 2^-37 vanish.
  *              Where a hit's entry lives: every hit owns one slot (forward writes never collide).  Both layouts
- *              rank work units by descending hit count and interleave the entries of 32 consecutive ranks
- *              (entry e of rank r of a group at group start + 32 e + r mod 32), so that a warp of the backward
- *              reads its lanes' e-th entries as one 512-byte row and a group's block is one contiguous range;
- *              a group occupies 32 x (its largest hit count) entries, L >= H counts that padding.
- *              GART_LT_TILE_MAJOR: the unit is a (tile, Gaussian) pair, groups are formed inside each tile.
+ *              rank work units by descending hit count and interleave the entries of 32 consecutive ranks, so that a
+ *              warp of the backward reads its lanes' entries as contiguous rows and a group's block is one contiguous
+ *              range; a group occupies 32 x (its largest hit count) entries, L >= H counts that padding.
+ *              GART_LT_TILE_MAJOR: the unit is a (tile, Gaussian) pair, groups are formed inside each tile; entry e
+ *              of rank r sits at group start + 32 e + r mod 32.
  *              GART_LT_PRIMITIVE_MAJOR: the unit is a work item -- a Gaussian whose rectangle spans at most two
  *              16 x 16-pixel super-tiles per axis, else the part of a Gaussian inside one super-tile; its entries are
  *              those of its (tile, Gaussian) pairs in turn (tiles row by row, pixels in mask order); groups are
- *              formed among the items owned by one super-tile.
+ *              formed among the items owned by one super-tile.  Entries go two by two: entry e of rank r sits at
+ *              group start + 64 (e / 2) + 2 (r mod 32) + e mod 2 (the group's largest count is rounded up to even), so
+ *              that a 32-byte sector holds two neighbouring hits of one Gaussian, which the forward writes close in time.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
  *              baseline and parity checks read the two lists: pass NULL for both to skip them.

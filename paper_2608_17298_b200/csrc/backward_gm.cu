@@ -14,22 +14,34 @@
 // A block serves up to GM_GROUPS_PER_BLOCK rank groups of one super-tile: it stages dL/dC of the super-tile's window in
 // shared memory (one copy: 16 KB), its warps take the groups in serpentine order, lanes own items of (nearly) equal hit
 // count, and the group's interleaved LT block streams in through bulk asynchronous copies (cp.async.bulk + mbarrier,
-// double buffered, every wait bounded).  The ray direction is affine in the pixel position before normalisation, so a
+// double buffered, every wait bounded).  A 16-byte LT entry carries the index of its pixel inside the window in its low
+// mantissa bits, so the hit loop touches no mask: walking per-lane masks costs more than the arithmetic of the hits
+// (every lane changes pair at its own time, and each change stalls the whole warp on that lane's load).  The ray direction is affine in the pixel position before normalisation, so a
 // hit recomputes it (12 instructions) instead of loading it: with lanes reading different pixels of a 1024-pixel window,
 // shared-memory loads conflict, and the direction would double them.
 #include "backward_common.cuh"
 #include "view_layout.cuh"
 
+#ifndef GMB_ABL
+#define GMB_ABL 0
+#endif
+
 namespace gart {
 
 constexpr int GMB_WARPS = 4;
 constexpr int GMB_THREADS = GMB_WARPS * 32;
-constexpr int GMB_CHUNK = 7;                           // LT entries per lane and per pipeline stage (16-byte entries)
+constexpr int GMB_CHUNK = 6;                           // LT entries per lane and per pipeline stage (16-byte entries); even
 constexpr int GMB_STAGE_F4 = GMB_CHUNK * 32;           // float4 per stage
 constexpr int GMB_STAGES = 2;
+#ifndef GMB_MINB
+#define GMB_MINB 4
+#endif
+constexpr int GMB_MIN_BLOCKS = GMB_MINB;                      // resident blocks per SM that the register budget is set for
 constexpr int GMB_LT_SMEM = GMB_WARPS * GMB_STAGES * GMB_STAGE_F4 * 16;
 constexpr int GMB_PIX = GM_WIN * GM_WIN;
-constexpr int GMB_DYN_SMEM = GMB_LT_SMEM + GMB_PIX * 16;
+constexpr int GMB_PF4 = 7;                             // float4 per lane of the staged per-Gaussian data: evaluation record 5, quaternion, scale + opacity
+constexpr int GMB_DYN_SMEM = GMB_LT_SMEM + GMB_PIX * 16 + GMB_THREADS * GMB_PF4 * 16;
+static_assert(GMB_CHUNK % 2 == 0, "entries are interleaved two by two");
 static_assert(GM_GROUPS_PER_BLOCK % GMB_WARPS == 0, "groups are dealt to the warps in rounds");
 
 __device__ __forceinline__ float fast_rsqrt(float x) {
@@ -95,11 +107,12 @@ struct ItemWalk {
     static constexpr int MW = TS * TS / 32;
     const uint32_t* mrow;   // masks of the current tile row of the item
     uint32_t bits, stride;
-    int ntx, tx, wi, pbase, prow;
+    int ntx, tx, wi, pbase, prow, togo;   // togo: pairs of the item after the current one
     __device__ __forceinline__ void start(const uint32_t* __restrict__ gm_mask, const uint4 d, bool any) {
         stride = d.z & 0xffffu;
         ntx = (d.z >> 16) & 15;
         const int otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
+        togo = ntx * (int)((d.z >> 20) & 15) - 1;
         mrow = gm_mask + (size_t)d.y * MW;
         tx = 0; wi = 0;
         prow = oty * TS * GM_WIN + otx * TS;
@@ -109,6 +122,7 @@ struct ItemWalk {
     __device__ __forceinline__ int next() {
         while (bits == 0u) {
             if (++wi == MW) {
+                if (--togo < 0) return 0;   // (never: next() is called once per hit of the item; keeps a broken mask from spinning)
                 wi = 0;
                 pbase += TS;
                 if (++tx == ntx) { tx = 0; mrow += (size_t)stride * MW; prow += TS * GM_WIN; pbase = prow; }
@@ -121,19 +135,79 @@ struct ItemWalk {
     }
 };
 
-// Block-uniform coefficients of the un-normalised ray direction D = A xf + B yf + C through window pixel (xf, yf).
+// 64-pixel tiles: a pair's mask is one 8-byte word pair, and the mask of the pair after the current one is fetched
+// while the current one is walked (a lane changes pair every dozen hits, each lane at its own time: fetched on
+// demand, every change would stall the warp for a trip to L2).
+template <>
+struct ItemWalk<8> {
+    const uint2* mcur;      // mask of the pair being prefetched (row base + column)
+    uint32_t lo, hi, stride;
+    uint2 nx;               // the prefetched mask
+    int ntx, tx, ptx, togo, pbase, prow, boff;   // togo: pairs of the item after the current one
+    // fetch the mask of the pair `ahead` pairs after the current one (the cursor advances row by row)
+    __device__ __forceinline__ void prefetch(int ahead) {
+        if (togo >= ahead) {
+            if (++ptx == ntx) { ptx = 0; mcur += stride; }
+            nx = __ldg(mcur + ptx);
+        } else {
+            nx = make_uint2(0u, 0u);
+        }
+    }
+    __device__ __forceinline__ void start(const uint32_t* __restrict__ gm_mask, const uint4 d, bool any) {
+        stride = d.z & 0xffffu;
+        ntx = (d.z >> 16) & 15;
+        const int nty = (d.z >> 20) & 15, otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
+        mcur = reinterpret_cast<const uint2*>(gm_mask) + d.y;
+        tx = 0; ptx = 0; boff = 0;
+        prow = oty * 8 * GM_WIN + otx * 8;
+        pbase = prow;
+        togo = any ? ntx * nty - 1 : 0;
+        const uint2 m = any ? __ldg(mcur) : make_uint2(0u, 0u);
+        lo = m.x; hi = m.y;
+        prefetch(1);
+    }
+    __device__ __forceinline__ int next() {
+        while (lo == 0u) {
+            if (hi != 0u) { lo = hi; hi = 0u; boff = 32; }
+            else {
+                if (--togo < 0) return 0;   // (never: next() is called once per hit of the item; keeps a broken mask from spinning)
+                lo = nx.x; hi = nx.y; boff = 0;
+                pbase += 8;
+                if (++tx == ntx) { tx = 0; prow += 8 * GM_WIN; pbase = prow; }
+                prefetch(1);
+            }
+        }
+        const int b = __ffs((int)lo) - 1 + boff;
+        lo &= lo - 1u;
+        return pbase + (b >> 3) * GM_WIN + (b & 7);
+    }
+};
+
+// Coefficients of the un-normalised ray direction D = A x + B y + C through pixel (x, y) of the image: the same for the
+// whole launch, passed by value (operands from the constant bank: no registers).
 struct DirAffine {
     float3 A, B, C;
 };
+static inline DirAffine make_dir_affine(const CamF& cam) {
+    DirAffine d;
+    const float ifx = 1.0f / cam.fx, ify = 1.0f / cam.fy;
+    const float u0 = (0.5f - cam.cx) * ifx, v0 = (0.5f - cam.cy) * ify;
+    d.A = make_float3(cam.r[0] * ifx, cam.r[1] * ifx, cam.r[2] * ifx);
+    d.B = make_float3(cam.r[3] * ify, cam.r[4] * ify, cam.r[5] * ify);
+    d.C = make_float3(cam.r[0] * u0 + cam.r[3] * v0 + cam.r[6], cam.r[1] * u0 + cam.r[4] * v0 + cam.r[7],
+                      cam.r[2] * u0 + cam.r[5] * v0 + cam.r[8]);
+    return d;
+}
 
 // Gradient terms of one hit added to the item's accumulators: geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz),
 // geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh against the bare SH polynomials.
 template <int K>
-__device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, ShRegs<K>& R, float* geo, const float4* __restrict__ spix, int pix, const float4 L) {
+__device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, float wxf, float wyf, ShRegs<K>& R, float* geo, const float4* __restrict__ spix, int pix, const float4 L) {
     const float4 gq = spix[pix];
     const float xf = small_int_to_float((uint32_t)pix & (GM_WIN - 1)), yf = small_int_to_float((uint32_t)pix / GM_WIN);
-    const float Dx = fmaf(dir.A.x, xf, fmaf(dir.B.x, yf, dir.C.x)), Dy = fmaf(dir.A.y, xf, fmaf(dir.B.y, yf, dir.C.y)),
-                Dz = fmaf(dir.A.z, xf, fmaf(dir.B.z, yf, dir.C.z));
+    const float xa = xf + wxf, ya = yf + wyf;   // pixel in the image (integers below 2^22: exact)
+    const float Dx = fmaf(dir.A.x, xa, fmaf(dir.B.x, ya, dir.C.x)), Dy = fmaf(dir.A.y, xa, fmaf(dir.B.y, ya, dir.C.y)),
+                Dz = fmaf(dir.A.z, xa, fmaf(dir.B.z, ya, dir.C.z));
     const float inv = fast_rsqrt(fmaf(Dx, Dx, fmaf(Dy, Dy, Dz * Dz)));
     float Y[K];
     sh_poly<K>(make_float3(Dx * inv, Dy * inv, Dz * inv), Y);
@@ -160,19 +234,22 @@ __device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, S
 
 // FMT: 0 = 16-byte LT entries, 2 = 8-byte entries (four halves, twice as many per pipeline stage).
 template <int TS, int DEG, int FMT>
-__global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __restrict__ rec, const float4* __restrict__ qs,
+__global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(const float4* __restrict__ rec, const float4* __restrict__ qs,
                                                              const uint32_t* __restrict__ gid_of_slot, const uint2* __restrict__ blk_desc,
                                                              const uint32_t* __restrict__ info, const uint32_t* __restrict__ st_off,
                                                              const uint4* __restrict__ rk_desc, const uint32_t* __restrict__ rk_gstart,
                                                              const uint32_t* __restrict__ gm_mask, const float4* __restrict__ lt,
-                                                             const float* __restrict__ dL_dC, CamF cam, int sup_x, Gacc gacc,
+                                                             const float* __restrict__ dL_dC, int width, int height, const DirAffine dir,
+                                                             int sup_x, Gacc gacc,
                                                              float4* __restrict__ grad4, uint32_t* __restrict__ counts) {
     constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
     constexpr int EB = FMT == 2 ? 8 : 16;                  // bytes per LT entry
-    constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage
-    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][GMB_STAGE_F4] LT stages, then dL/dC of the window
+    constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage (even)
+    constexpr int PF4 = GMB_PF4, PSTR = GMB_PF4;           // staged per-Gaussian data; odd lane stride: the lanes' 16-byte reads fall into distinct banks
+    extern __shared__ __align__(128) float4 dyn[];   // [warp][2][GMB_STAGE_F4] LT stages, dL/dC of the window, [thread][PF4] per-Gaussian data
     __shared__ __align__(8) uint64_t bars[GMB_WARPS][GMB_STAGES];
+    __shared__ uint32_t sgid[GMB_THREADS];   // staged id of the lane's Gaussian
     if (counts[GART_CNT_ERROR]) return;
     if (blockIdx.x >= info[GM_INFO_BLOCKS]) return;
     const uint2 bd = blk_desc[blockIdx.x];
@@ -189,40 +266,36 @@ __global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __
     for (int t = threadIdx.x; t < GMB_PIX; t += GMB_THREADS) {
         const int x = wx0 + (t & (GM_WIN - 1)), y = wy0 + t / GM_WIN;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (x < cam.width && y < cam.height) {
-            const float* gp = dL_dC + ((size_t)y * cam.width + x) * 3;
+        if (x < width && y < height) {
+            const float* gp = dL_dC + ((size_t)y * width + x) * 3;
             v.x = gp[0]; v.y = gp[1]; v.z = gp[2];
         }
         spix[t] = v;
     }
     __syncthreads();
-    DirAffine dir;
-    {
-        const float ifx = 1.0f / cam.fx, ify = 1.0f / cam.fy;
-        const float u0 = ((float)wx0 + 0.5f - cam.cx) * ifx, v0 = ((float)wy0 + 0.5f - cam.cy) * ify;
-        dir.A = make_float3(cam.r[0] * ifx, cam.r[1] * ifx, cam.r[2] * ifx);
-        dir.B = make_float3(cam.r[3] * ify, cam.r[4] * ify, cam.r[5] * ify);
-        dir.C = make_float3(fmaf(cam.r[0], u0, fmaf(cam.r[3], v0, cam.r[6])), fmaf(cam.r[1], u0, fmaf(cam.r[4], v0, cam.r[7])),
-                            fmaf(cam.r[2], u0, fmaf(cam.r[5], v0, cam.r[8])));
-    }
+    const float wxf = (float)wx0, wyf = (float)wy0;
 
     float4* my_stage = dyn + (size_t)warp * GMB_STAGES * GMB_STAGE_F4;
+    float4* my_par = spix + GMB_PIX + (size_t)(warp * 32 + lane) * PSTR;
     const uint32_t stage_addr = smem_u32(my_stage);
+    const uint32_t par_addr = smem_u32(my_par);
     const uint32_t bar_addr = smem_u32(&bars[warp][0]);
     const char* lt_bytes = reinterpret_cast<const char*>(lt);
-    // LT pipeline: unit u (a chunk of CH entries per lane) uses stage u % GMB_STAGES, and the wait for it uses parity
-    // (u / GMB_STAGES) & 1.  `unit` counts the units consumed, `produced` those whose copy has been issued; the producer
-    // cursor (pw, pk) = (group relative to the current one, chunk) runs up to GMB_STAGES units and two groups ahead.
+    // LT pipeline: unit u (a chunk of CH entries per lane, i.e. CH / 2 rows of 32 two-entry sectors) uses stage
+    // u % GMB_STAGES, and the wait for it uses parity (u / GMB_STAGES) & 1.  `unit` counts the units consumed, `produced`
+    // those whose copy has been issued; the producer cursor (pw, pk) = (group relative to the current one, chunk) runs up to
+    // GMB_STAGES units and two groups ahead.  A group holds 32 x (its largest count rounded up to even) entries.
     uint32_t unit = 0, produced = 0;
     int pw = 0, pk = 0;
-    auto produce = [&](const GmItem& a, const GmItem& b, const GmItem& c, const int maxw) {
+    auto produce = [&](const GmItem& a, const GmItem& b, const int c_cmax, const uint32_t c_gstart, const int maxw) {
         while (produced - unit < (uint32_t)GMB_STAGES && pw <= maxw) {
             int cm;
             uint32_t gs;
             if (pw == 0) { cm = a.cmax; gs = a.gstart; }
             else if (pw == 1) { cm = b.cmax; gs = b.gstart; }
-            else { cm = c.cmax; gs = c.gstart; }
+            else { cm = c_cmax; gs = c_gstart; }
             if (cm == 0) break;                                   // ranks descend in hit count: no later group has hits
+            cm += cm & 1;
             if (pk * CH >= cm) { ++pw; pk = 0; continue; }
             if (lane == 0) {
                 const int ne = min(CH, cm - pk * CH);
@@ -234,11 +307,36 @@ __global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __
             ++pk;
         }
     };
+    // copy the per-Gaussian data of a group's items into the lane's buffer, one group ahead: the evaluation record (read
+    // before the hit loop) and what the final conversion needs (quaternion, scale + opacity, id: read after the loop, so
+    // that they occupy no register across it)
+    const uint32_t gid_addr = smem_u32(&sgid[threadIdx.x]);
+    // Every issue closes one copy group, and the two kinds alternate (record of group j + 1 at the start of group j, tail
+    // of group j + 1 at its end), so "all groups but the newest have landed" is exactly what each reader needs: the record
+    // at the start of a group (the tail just issued may still fly), the tail at its end (the next record may still fly).
+    auto issue_rec = [&](const GmItem& d) {
+        if (d.valid) {
+            const float4* src = rec + (size_t)d.d.x * RS4;
+#pragma unroll
+            for (int q = 0; q < 5; ++q) cp_async16(par_addr + 16u * q, src + q);
+        }
+        cp_async_commit();
+    };
+    auto issue_tail = [&](const GmItem& d) {
+        if (d.valid && (d.d.w & GM_DESC_WHOLE)) {
+            const float4* sq = qs + 2 * (size_t)d.d.x;
+            cp_async16(par_addr + 16u * 5, sq);
+            cp_async16(par_addr + 16u * 6, sq + 1);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(gid_addr), "l"(gid_of_slot + d.d.x) : "memory");
+        }
+        cp_async_commit();
+    };
     auto fail = [&]() {
         // a copy never completed: report, give copies that may still be in flight a second bounded chance to land
         // before this warp's shared memory may be released, and stop
         if (lane == 0) atomicOr(&counts[GART_CNT_ERROR], GART_ERRBIT_TIMEOUT);
         for (uint32_t u = unit; u != produced; ++u) mbar_wait_bounded(bar_addr + 8u * (u % GMB_STAGES), (u / GMB_STAGES) & 1u);
+        cp_async_wait_all();
     };
 
     // The block's groups are [g0, g0 + GM_GROUPS_PER_BLOCK) of the super-tile; the warp's j-th group is
@@ -246,67 +344,93 @@ __global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __
     // gives every warp nearly the same number of iterations.
     const uint32_t g0 = bd.y * GM_GROUPS_PER_BLOCK;
     constexpr uint32_t ROUNDS = GM_GROUPS_PER_BLOCK / GMB_WARPS;
-    auto load = [&](uint32_t j) {
-        const uint32_t gi = g0 + j * GMB_WARPS + ((j & 1u) ? (uint32_t)(GMB_WARPS - 1 - warp) : (uint32_t)warp);
-        return gm_load_item(rk_desc, rk_gstart, begin, n, 32u * gi, j < ROUNDS, lane);
-    };
+    auto first_rank = [&](uint32_t j) { return 32u * (g0 + j * GMB_WARPS + ((j & 1u) ? (uint32_t)(GMB_WARPS - 1 - warp) : (uint32_t)warp)); };
+    auto load = [&](uint32_t j) { return gm_load_item(rk_desc, rk_gstart, begin, n, first_rank(j), j < ROUNDS, lane); };
+
     uint32_t gj = 0;
     GmItem cur = load(0);
+    issue_rec(cur);
+    issue_tail(cur);
     GmItem nxt = load(1);
+    bool first = true;
     while (__any_sync(0xffffffffu, cur.valid)) {
-        const GmItem nxt2 = load(gj + 2);
-        produce(cur, nxt, nxt2, 1);
-        // the item's Gaussian: evaluation record, and what the final conversion needs
+        const GmItem nxt2 = load(gj + 2);   // (two groups ahead: its loads are in flight during this group)
+        const int c2_cmax = nxt2.cmax;
+        const uint32_t c2_gstart = nxt2.gstart;
+        produce(cur, nxt, c2_cmax, c2_gstart, 1);
         const uint32_t sid = cur.d.x;
         const bool whole = (cur.d.w & GM_DESC_WHOLE) != 0u;
-        PreRec P;
-        if (cur.valid) {
-            P = load_pre(rec + (size_t)sid * RS4);
-        } else {
-            P = unpack_pre(make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 1.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f),
-                           make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f));
-        }
+        if (first) cp_async_wait_all(); else cp_async_wait_but_one();   // this lane's record has landed (a lane reads only what it copied itself)
+        first = false;
+        const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale data for lanes without item: never used)
+        issue_rec(nxt);        // the lane has read its record: that part of its buffer may be overwritten
         const ItemGeo IG = item_geo<TS>(P, cur.d, wx0, wy0);
+        // a 16-byte entry names its pixel (lt_pix); 8-byte entries have no room for that: their pixels come from the masks
         ItemWalk<TS> walk;
-        walk.start(gm_mask, cur.d, cur.c != 0);
+        if constexpr (FMT == 2) walk.start(gm_mask, cur.d, cur.c != 0);
         ShRegs<K> R;
         R.clear();
         float geo[11];
 #pragma unroll
         for (int q = 0; q < 11; ++q) geo[q] = 0.0f;
-        const int nchunks = (cur.cmax + CH - 1) / CH;
+        const int cme = cur.cmax + (cur.cmax & 1);
+        const int nchunks = (cme + CH - 1) / CH;
+        // lanes 4..7 of every eight read the second entry of their sector first: the eight lanes that a 16-byte shared load
+        // serves together then touch eight different bank groups (their sectors lie 32 bytes apart)
+        const bool flip = EB == 16 && (lane & 4) != 0;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % GMB_STAGES;
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / GMB_STAGES) & 1u))) { fail(); return; }
-            const char* sl = reinterpret_cast<const char*>(my_stage + s * GMB_STAGE_F4) + lane * EB;   // entry j of the stage: sl + j * 32 * EB
-            auto entry = [&](const char* q) {
-                if constexpr (FMT == 2) return lt_unpack_half(*reinterpret_cast<const uint2*>(q));
-                else return *reinterpret_cast<const float4*>(q);
-            };
+            // entries 2m and 2m + 1 of the lane: the 2 EB bytes at row m (32 lanes x 2 EB bytes) + lane x 2 EB
+            const char* se = reinterpret_cast<const char*>(my_stage + s * GMB_STAGE_F4) + lane * (2 * EB);
             const int e_end = min(cur.c, (k + 1) * CH);
-            // two hits per iteration: two independent dependency chains for the scheduler to interleave
-            int e = k * CH;
-            const char* se = sl;
-            for (; e + 1 < e_end; e += 2, se += 64 * EB) {
-                const int p0 = walk.next();
-                const int p1 = walk.next();
-                const float4 L0 = entry(se), L1 = entry(se + 32 * EB);
-                gm_hit<K>(IG, dir, R, geo, spix, p0, L0);
-                gm_hit<K>(IG, dir, R, geo, spix, p1, L1);
+            for (int e = k * CH; e < e_end; e += 2, se += 64 * EB) {
+                float4 L0, L1;
+                if constexpr (FMT == 2) {
+                    const uint4 t = *reinterpret_cast<const uint4*>(se);
+                    L0 = lt_unpack_half(make_uint2(t.x, t.y));
+                    L1 = lt_unpack_half(make_uint2(t.z, t.w));
+                } else {
+                    const float4 a = *reinterpret_cast<const float4*>(se + (flip ? 16 : 0));
+                    const float4 b = *reinterpret_cast<const float4*>(se + (flip ? 0 : 16));
+                    L0 = flip ? b : a;
+                    L1 = flip ? a : b;
+                }
+                // two hits per iteration: two independent dependency chains for the scheduler to interleave
+                int p0, p1 = 0;
+                if constexpr (FMT == 2) { p0 = walk.next(); if (e + 1 < e_end) p1 = walk.next(); }
+                else { p0 = (int)lt_pix(L0); p1 = (int)lt_pix(L1); }
+                if (e + 1 < e_end) {
+#if GMB_ABL == 1
+                    geo[0] += L0.x + L1.x + spix[p0].x + spix[p1].y;
+#else
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p0, L0);
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p1, L1);
+#endif
+                } else {
+#if GMB_ABL == 1
+                    geo[0] += L0.x + spix[p0].x;
+#else
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p0, L0);
+#endif
+                }
             }
-            if (e < e_end) gm_hit<K>(IG, dir, R, geo, spix, walk.next(), entry(se));
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
-            produce(cur, nxt, nxt2, 2);
+            produce(cur, nxt, c2_cmax, c2_gstart, 2);
         }
         // ---- the item's sums leave the registers
+#if GMB_ABL == 3
+        if (cur.valid && geo[0] == 123.456f) {
+#else
         if (cur.valid) {
+#endif
             if (whole) {
                 // the thread holds every hit of its Gaussian: convert the moments and write the gradient record once
-                // (quaternion, scale, opacity and id are fetched only now: they would occupy registers across the hit loop)
-                const float4 q4 = __ldg(qs + 2 * (size_t)sid), s4 = __ldg(qs + 2 * (size_t)sid + 1);
-                const uint32_t gid = __ldg(gid_of_slot + sid);
+                cp_async_wait_but_one();   // (the tail data of this group; the next group's record may still be in flight)
+                const float4 q4 = my_par[5], s4 = my_par[6];
+                const uint32_t gid = sgid[threadIdx.x];
                 const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
                 const float sc[3] = {s4.x, s4.y, s4.z};
                 const GeoGrad o = moments_to_grads(geo, geo + 3, qv, sc);
@@ -337,12 +461,14 @@ __global__ void __launch_bounds__(GMB_THREADS, 4) bwd_gm_kernel(const float4* __
                 }
             }
         }
+        issue_tail(nxt);   // (its conversion data: the lane has read the current item's)
         cur = nxt;
         nxt = nxt2;
         ++gj;
         --pw;
         if (pw < 0) { pw = 0; pk = 0; }   // (a group without hits leaves the producer behind: it restarts at the new current group)
     }
+    cp_async_wait_all();
 }
 
 // ---- the large Gaussians (cut into pieces): zero their accumulation records before, convert them after.  One thread
@@ -416,7 +542,7 @@ static gart_status launch_gm(int deg, unsigned grid, cudaStream_t st, const floa
         auto kern = bwd_gm_kernel<TS, D, FMT>;                                                                                   \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GMB_DYN_SMEM) != cudaSuccess) return GART_ERR_CUDA; \
         kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, v.gm_mask, lt, \
-                                                      dL_dC, cam, sup_x, gacc, grad4, counts);                                  \
+                                                      dL_dC, cam.width, cam.height, make_dir_affine(cam), sup_x, gacc, grad4, counts); \
     }
     switch (deg) {
         case 0: GART_GM(0); break;

@@ -165,10 +165,25 @@ __device__ __forceinline__ float4 lt_entry(float w, float alpha, float c0, float
                        __uint_as_float((__float_as_uint(w) & ~7u) | flags));
 }
 
+// In the primitive-major layout the entry also names the pixel it belongs to: the 10-bit index y * 32 + x of the hit's
+// pixel inside the 32 x 32-pixel window of the work item's owner replaces the three low mantissa bits of each of the
+// words 0..2 (bits 0..2, 3..5, 6..8 of the index) and bit 3 of word 3 (bit 9): a relative change below 2^-20 of
+// numbers needed to 1e-3.  The backward pass then finds a hit's pixel without walking any hit mask.
+__device__ __forceinline__ float4 lt_embed_pix(const float4 e, const uint32_t pix) {
+    return make_float4(__uint_as_float((__float_as_uint(e.x) & ~7u) | (pix & 7u)),
+                       __uint_as_float((__float_as_uint(e.y) & ~7u) | ((pix >> 3) & 7u)),
+                       __uint_as_float((__float_as_uint(e.z) & ~7u) | ((pix >> 6) & 7u)),
+                       __uint_as_float((__float_as_uint(e.w) & ~8u) | ((pix >> 6) & 8u)));
+}
+__device__ __forceinline__ uint32_t lt_pix(const float4 e) {
+    return (__float_as_uint(e.x) & 7u) | ((__float_as_uint(e.y) & 7u) << 3) | ((__float_as_uint(e.z) & 7u) << 6) |
+           ((__float_as_uint(e.w) & 8u) << 6);
+}
+
 // The per-channel weights dL/dc = w g of an LT entry (zero on clamped channels).
 __device__ __forceinline__ void lt_weights(const float4 L, const float3 g, float* wch) {
     const uint32_t b = __float_as_uint(L.w);
-    const float w = __uint_as_float(b & ~7u);
+    const float w = __uint_as_float(b & ~15u);
     wch[0] = (b & 1u) ? w * g.x : 0.0f;
     wch[1] = (b & 2u) ? w * g.y : 0.0f;
     wch[2] = (b & 4u) ? w * g.z : 0.0f;
@@ -188,7 +203,7 @@ __device__ __forceinline__ uint32_t lt_half_word9(float x, uint32_t flag) {
 }
 __device__ __forceinline__ uint2 lt_pack_half(const float4 e) {
     const uint32_t b = __float_as_uint(e.w);
-    const float w = __uint_as_float(b & ~7u);
+    const float w = __uint_as_float(b & ~15u);
     const uint32_t h3 = __half_as_ushort(__float2half_rn(w * LT_HALF_SCALE));
     return make_uint2(lt_half_word9(e.x, b & 1u) | (lt_half_word9(e.y, (b >> 1) & 1u) << 16),
                       lt_half_word9(e.z, (b >> 2) & 1u) | (h3 << 16));
@@ -360,6 +375,10 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// groups of per-thread copies: commit closes the group of the copies issued so far; wait_but_one returns when all groups
+// but the most recently committed one have landed
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 
 // 32-byte (one sector) global store / read-only load; the address must be 32-byte aligned
 __device__ __forceinline__ void st_global_32B(void* dst, const float4 a, const float4 b) {

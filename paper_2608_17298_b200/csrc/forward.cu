@@ -353,15 +353,16 @@ template <int MW>
 struct EvalDesc {
     PairMask<MW> pm;
     uint32_t sid, gstart;
+    uint32_t pbase;   // primitive-major layout: window index of the pair's tile origin
     int c;      // hits of this lane's pair
     int cmax;   // hits of the group's first pair (the largest)
 };
 
-// GMAJ: the LT slot of the pair's first hit comes from the primitive-major layout (gm_ltb, looked up by the pair's
-// primitive-major position) instead of the tile's rank groups; later hits follow 32 entries apart in both layouts.
+// GMAJ: rank_gstart holds the LT slot of the pair's first hit in the primitive-major layout (resolved per rank position
+// by gm_rank_ltb_kernel) instead of the start of the tile's rank group.
 template <int MW, bool GMAJ>
 __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
-                                                       const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ gm_ltb,
+                                                       const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ rank_pbase,
                                                        uint32_t begin, uint32_t n, uint32_t r0, int lane) {
     EvalDesc<MW> d;
     const bool act = r0 < n && r0 + lane < n;
@@ -369,8 +370,8 @@ __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restric
     d.pm.load(rank_mask, act ? q : 0u, act);
     d.c = d.pm.count();
     d.sid = act ? __ldg(rank_sid + q) : 0u;
-    d.gstart = act ? __ldg(rank_gstart + q) : 0u;   // (GMAJ: rank_gstart is the array of primitive-major positions)
-    if (GMAJ) d.gstart = act ? __ldg(gm_ltb + d.gstart) : 0u;
+    d.gstart = act ? __ldg(rank_gstart + q) : 0u;
+    d.pbase = (GMAJ && act) ? __ldg(rank_pbase + q) : 0u;
     d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
     return d;
 }
@@ -395,7 +396,7 @@ template <int TS, int DEG, bool GMAJ>
 __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
-                                                                const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ gm_ltb,
+                                                                const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ rank_pbase,
                                                                 const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
                                                                 uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PF4 = (20 + SW + 3) / 4;
@@ -450,12 +451,12 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     };
 
     uint32_t r0 = warp * 32;
-    EvalDesc<MW> cur = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0, lane);
+    EvalDesc<MW> cur = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0, lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
     issue_params(cur);
-    EvalDesc<MW> nxt = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0 + EVAL_THREADS, lane);
+    EvalDesc<MW> nxt = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0 + EVAL_THREADS, lane);
     while (true) {
-        const EvalDesc<MW> nxt2 = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, gm_ltb, begin, n, r0 + 2 * EVAL_THREADS, lane);
+        const EvalDesc<MW> nxt2 = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0 + 2 * EVAL_THREADS, lane);
         const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
         cp_async_wait_all();   // the copies this lane issued have landed
         __syncwarp();          // ... and so have those of the other lanes, which hold pieces of this lane's record
@@ -470,6 +471,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         if (nxt.cmax != 0) issue_params(nxt);
         uint32_t slot = GMAJ ? cur.gstart : lt_base + cur.gstart + lane;
         const float fbx = (float)(x0 - P.ix), fby = (float)(y0 - P.iy);
+        const uint32_t wdx = (cur.pbase / GM_SUP) & 1u, wdy = cur.pbase / (GM_WIN * GM_SUP);   // the tile's super-tile inside the owner's window
         // one hit: evaluate, take the next free place of the ray's segment, write the 32-byte record
         auto hit = [&](const int p, const uint32_t slot_e) {
             const float4 pa = spix_lane[EvalPix<TS>::index(p, 0, 0)], pb = spix_lane[EvalPix<TS>::index(p, 1, 0)];
@@ -486,17 +488,26 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                 c2 = fmaf(B[k], shc[3 * k + 2], c2);
             }
             float4* out = recs + ((size_t)__float_as_uint(pb.y) + pos) * 2;
+            // The lowest mantissa bit of the first two colour words tells the sweep in which of the 2 x 2 super-tiles of the
+            // owner's window this pixel lies (the primitive-major LT entry names its pixel inside that window).  The sweep
+            // composites the words without that bit, so both layouts composite the very same numbers.
+            c0 = __uint_as_float((__float_as_uint(fmaxf(c0, 0.0f)) & ~1u) | wdx);
+            c1 = __uint_as_float((__float_as_uint(fmaxf(c1, 0.0f)) & ~1u) | wdy);
             st_global_32B(out, make_float4(t, __uint_as_float(gid), __uint_as_float(slot_e), r.alpha),
-                          make_float4(fmaxf(c0, 0.0f), fmaxf(c1, 0.0f), fmaxf(c2, 0.0f), 0.0f));
+                          make_float4(c0, c1, fmaxf(c2, 0.0f), 0.0f));
         };
-        // two hits per iteration: two independent dependency chains for the scheduler to interleave
+        // two hits per iteration: two independent dependency chains for the scheduler to interleave.  The next hit's slot:
+        // 32 entries on in the tile-major layout; in the primitive-major layout entries go two by two (gm_slot):
+        // the odd one follows its even one, the next even one lies 63 further.
+        auto after = [](uint32_t sl) { return GMAJ ? ((sl & 1u) ? sl + 63u : sl + 1u) : sl + 32u; };
         int e = 0;
         for (; e + 1 < cur.c; e += 2) {
             const int p0 = cur.pm.next();
             const int p1 = cur.pm.next();
+            const uint32_t slot1 = after(slot);
             hit(p0, slot);
-            hit(p1, slot + 32u);
-            slot += 64u;
+            hit(p1, slot1);
+            slot = after(slot1);
         }
         if (e < cur.c) hit(cur.pm.next(), slot);
         if (nxt.cmax == 0) break;
@@ -575,10 +586,21 @@ __device__ __forceinline__ void sort_regs(uint32_t (&k)[R], int lane) {
     }
 }
 
-// Store a hit's LT entry in the format the caller asked for: all 16 bytes, only the weight word (4 bytes), or
-// the four words as halves (8 bytes).
-__device__ __forceinline__ void lt_store(float4* __restrict__ lt, int lt_fmt, uint32_t slot, const float4 e) {
-    if (lt_fmt == 0) lt[slot] = e;
+// A hit's colour words as they are composited: without the lowest mantissa bit of the first two (see pix_of).
+__device__ __forceinline__ float strip_low_bit(float c) { return __uint_as_float(__float_as_uint(c) & ~1u); }
+
+// Index of the ray's pixel inside the 32 x 32-pixel window of a hit's owner: pixlow = (y mod 16) * 32 + x mod 16 from the
+// ray, plus the super-tile offsets that the evaluation left in the lowest bit of the hit's first two colour words;
+// -1 (nothing to embed) where pixlow < 0, i.e. in the tile-major layout.
+__device__ __forceinline__ int pix_of(int pixlow, float c0, float c1) {
+    return pixlow < 0 ? -1 : pixlow + (int)((__float_as_uint(c0) & 1u) * GM_SUP + (__float_as_uint(c1) & 1u) * (GM_SUP * GM_WIN));
+}
+
+// Store a hit's LT entry in the format the caller asked for: all 16 bytes (with the pixel's window index in the low
+// mantissa bits where the layout is primitive-major: pix >= 0), only the weight word (4 bytes), or the four words as
+// halves (8 bytes).
+__device__ __forceinline__ void lt_store(float4* __restrict__ lt, int lt_fmt, uint32_t slot, const float4 e, int pix) {
+    if (lt_fmt == 0) lt[slot] = pix >= 0 ? lt_embed_pix(e, (uint32_t)pix) : e;
     else if (lt_fmt == 1) reinterpret_cast<float*>(lt)[slot] = e.w;
     else reinterpret_cast<uint2*>(lt)[slot] = lt_pack_half(e);
 }
@@ -592,7 +614,7 @@ __device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32
 // The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
 // slot as one float4, alpha apart; after the sort the three passes gather from there by sorted index.
 template <int R>
-__device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx,
+__device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx, int pixlow,
                                                float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                                                float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
@@ -688,7 +710,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
         for (int r = 0; r < R; ++r) {
             const float w0 = T * al[r];   // zero on padding positions
             const float4 c = s_cs[lane * R + r < n ? (k[r] & KEY_IDX_MASK) : 0u];
-            s0 = fmaf(w0, c.x, s0); s1 = fmaf(w0, c.y, s1); s2 = fmaf(w0, c.z, s2);
+            s0 = fmaf(w0, strip_low_bit(c.x), s0); s1 = fmaf(w0, strip_low_bit(c.y), s1); s2 = fmaf(w0, c.z, s2);
             T *= 1.0f - al[r];
         }
     }
@@ -715,9 +737,10 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const float4 cs = s_cs[c];
                 const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
-                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cs.x, cs.y, cs.z, k0, k1, k2));
+                const float cx = strip_low_bit(cs.x), cy = strip_low_bit(cs.y);
+                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2), pix_of(pixlow, cs.x, cs.y));
                 if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
-                k0 = fmaf(wgt, cs.x, k0); k1 = fmaf(wgt, cs.y, k1); k2 = fmaf(wgt, cs.z, k2);
+                k0 = fmaf(wgt, cx, k0); k1 = fmaf(wgt, cy, k1); k2 = fmaf(wgt, cs.z, k2);
             }
         }
     }
@@ -757,7 +780,7 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
     }
 }
 
-__device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int n_comp, int lane, size_t b, int64_t r,
+__device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int n_comp, int lane, size_t b, int64_t r, int pixlow,
                                             float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                             float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
     for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
@@ -813,7 +836,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
             rb = __ldg(&rec[2 * c + 1]);
             if (i >= n_comp) ra.w = 0.0f;   // behind the cap: not composited
             wgt = __uint_as_float((uint32_t)(key >> 32)) * ra.w;
-            v0 = wgt * rb.x; v1 = wgt * rb.y; v2 = wgt * rb.z;
+            v0 = wgt * strip_low_bit(rb.x); v1 = wgt * strip_low_bit(rb.y); v2 = wgt * rb.z;
         }
         float s0 = v0, s1 = v1, s2 = v2;
 #pragma unroll
@@ -827,7 +850,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
-            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, rb.x, rb.y, rb.z, k0 + e0, k1 + e1, k2 + e2));
+            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2), pix_of(pixlow, rb.x, rb.y));
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -856,7 +879,7 @@ struct SweepClass {
 template <int CLS, int FMT>   // FMT: the LT format (a compile-time constant keeps the store of the usual format free of tests)
 __global__ void __launch_bounds__(SWEEP_WARPS * 32, SweepClass<CLS>::MIN_BLOCKS)
 fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs, uint64_t* __restrict__ long_keys, int64_t n_rays,
-                      int width, int tile_size, int tiles_x,
+                      int width, int tile_size, int tiles_x, int embed_pix,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                       float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                       int max_comp, const uint32_t* __restrict__ counts) {
@@ -888,12 +911,13 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     }
     if (n <= SweepClass<CLS>::LO || (CLS < 2 && n > CAP)) return;
     const int n_comp = min(n, max_comp);   // hits that are composited (all of them unless the caller set a cap)
+    const int pixlow = embed_pix ? (int)((r / width) % GM_SUP) * GM_WIN + (int)((r % width) % GM_SUP) : -1;
     const float4* rec = recs + b * 2;
     extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, pixlow, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
@@ -901,7 +925,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
-        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
+        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, pixlow, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
     }
 #undef GART_SWEEP
 }
@@ -947,14 +971,14 @@ static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_p
 template <int TS, bool GMAJ>
 static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
-                               const uint32_t* tile_lt_base, const uint32_t* gm_ltb, const uint32_t* ray_off,
+                               const uint32_t* tile_lt_base, const uint32_t* rank_pbase, const uint32_t* ray_off,
                                const CamF& cam, const ForwardWs& w, uint32_t* counts) {
 #define GART_EVAL(D)                                                                                                        \
     {                                                                                                                      \
         auto kern = fwd_eval_kernel<TS, D, GMAJ>;                                                                          \
         constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
-        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, gm_ltb, ray_off, cam, \
+        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, rank_pbase, ray_off, cam, \
                                             w.recs, counts);                                                               \
     }
     switch (deg) {
@@ -1108,8 +1132,10 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
         if (s != GART_OK) return s;
         gm_blocks_kernel<<<(unsigned)ceil_div(v.ns, 256), 256, 0, st>>>(v.blk_off, v.st_parts, v.ns, v.blocks_cap, v.blk_desc, v.info, counts);
         GART_LAUNCH_CHECK();
-        if (ts == 8) gm_ltb_kernel<8><<<(unsigned)ceil_div(v.ns, 4), 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, counts);
-        else gm_ltb_kernel<16><<<(unsigned)ceil_div(v.ns, 4), 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, counts);
+        if (ts == 8) gm_ltb_kernel<8><<<(unsigned)v.ns, 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, v.gm_pbase, counts);
+        else gm_ltb_kernel<16><<<(unsigned)v.ns, 128, 0, st>>>(v.st_off, v.st_lt_base, v.ns, v.rk_desc, v.rk_gstart, v.gm_mask, v.gm_ltb, v.gm_pbase, counts);
+        GART_LAUNCH_CHECK();
+        gm_rank_ltb_kernel<<<(unsigned)ceil_div(cap_pairs, 256), 256, 0, st>>>(v.rank_gpos, v.gm_ltb, v.gm_pbase, v.rank_pbase, counts);
         GART_LAUNCH_CHECK();
     }
 
@@ -1120,11 +1146,11 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     GART_LAUNCH_CHECK();
 
     if (gmaj) {
-        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
-        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
+        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
     } else {
-        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
-        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.gm_ltb, ray_off, cf, w, counts);
+        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
+        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
     }
     if (s != GART_OK) return s;
 
@@ -1137,7 +1163,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     {                                                                                                                                           \
         if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
             return GART_ERR_CUDA;                                                                                                               \
-        fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0], \
+        fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, (gmaj && lt_fmt == 0) ? 1 : 0, bg[0], \
                                                                                                     bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, counts); \
         GART_LAUNCH_CHECK();                                                                                                                    \
     }

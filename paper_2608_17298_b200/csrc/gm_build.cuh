@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(256) gm_item_desc_kernel(const uint32_t* __res
 }
 
 // Warp per super-tile: stable counting sort of its items by descending hit count -> rk_desc; 32 consecutive ranks
-// form a group occupying 32 x (its largest count) LT entries -> rk_gstart (relative to the super-tile), st_len;
-// blocks of the backward for this super-tile -> st_parts.
+// form a group occupying 32 x (its largest count, rounded up to even) LT entries -> rk_gstart (relative to the
+// super-tile), st_len; blocks of the backward for this super-tile -> st_parts.
 constexpr int GM_RANK_WARPS = 4;
 constexpr int GM_RANK_BINS = GM_WIN * GM_WIN + 1;
 static __global__ void __launch_bounds__(GM_RANK_WARPS * 32) gm_rank_kernel(const uint32_t* __restrict__ st_off, const uint4* __restrict__ it_desc, int ns,
@@ -206,7 +206,8 @@ static __global__ void __launch_bounds__(GM_RANK_WARPS * 32) gm_rank_kernel(cons
         const bool act = r0 + lane < n;
         const uint32_t c = act ? (__ldcg(&rk_desc[begin + r0 + lane].w) & 0xffffu) : 0u;
         if (act) rk_gstart[begin + r0 + lane] = run;
-        run += 32u * __shfl_sync(0xffffffffu, c, 0);
+        const uint32_t cm = __shfl_sync(0xffffffffu, c, 0);
+        run += 32u * (cm + (cm & 1u));
     }
     if (lane == 0) {
         st_len[S] = run;
@@ -220,36 +221,56 @@ struct ArrayF {
     __device__ __forceinline__ uint32_t operator()(int64_t i) const { return a[i]; }
 };
 
-// Warp per super-tile: LT index of the first hit of every pair of every item (entry e of the item's hits sits at
-// group start + 32 e + lane; a pair's hits follow those of the item's earlier pairs), and the group starts made
-// absolute.
+// LT index of a work item's e-th hit (e counts through the item's pairs in turn) for the item of lane `lane` of a group
+// that starts at entry gs: entries are interleaved two by two, entries 2m and 2m + 1 of a lane share one 32-byte sector
+// (they are neighbouring pixels of one Gaussian, written by the forward close in time: whole-sector writes), the 32
+// lanes' sectors of the same m are consecutive (the backward reads them as one 1 KB row).
+__host__ __device__ __forceinline__ uint32_t gm_slot(uint32_t gs, uint32_t lane, uint32_t e) {
+    return gs + (e >> 1) * 64u + 2u * lane + (e & 1u);
+}
+
+// Block per super-tile, thread per item: LT index of the first hit of every pair of every item (a pair's hits follow
+// those of the item's earlier pairs), and the group starts made absolute.
 template <int TS>
 __global__ void __launch_bounds__(128) gm_ltb_kernel(const uint32_t* __restrict__ st_off, const uint32_t* __restrict__ st_lt_base, int ns,
                                                      const uint4* __restrict__ rk_desc, uint32_t* __restrict__ rk_gstart,
                                                      const uint32_t* __restrict__ gm_mask, uint32_t* __restrict__ gm_ltb,
-                                                     const uint32_t* __restrict__ counts) {
+                                                     uint32_t* __restrict__ gm_pbase, const uint32_t* __restrict__ counts) {
     constexpr int MW = TS * TS / 32;
     if (counts[GART_CNT_ERROR]) return;
-    const int lane = threadIdx.x & 31;
-    const int S = blockIdx.x * 4 + (threadIdx.x >> 5);
-    if (S >= ns) return;
+    const int S = blockIdx.x;
     const uint32_t begin = st_off[S], n = st_off[S + 1] - begin;
     const uint32_t base = st_lt_base[S];
-    for (uint32_t r = lane; r < n; r += 32) {
+    for (uint32_t r = threadIdx.x; r < n; r += blockDim.x) {
         const uint4 d = rk_desc[begin + r];
         const uint32_t gs = rk_gstart[begin + r] + base;
         rk_gstart[begin + r] = gs;
         const uint32_t stride = d.z & 0xffffu, ntx = (d.z >> 16) & 15u, nty = (d.z >> 20) & 15u;
+        const uint32_t otx = (d.z >> 24) & 15u, oty = (d.z >> 28) & 15u;
         uint32_t before = 0;
         for (uint32_t y = 0; y < nty; ++y)
             for (uint32_t x = 0; x < ntx; ++x) {
                 const uint32_t gp = d.y + y * stride + x;
-                gm_ltb[gp] = gs + (r & 31u) + 32u * before;
+                gm_ltb[gp] = gm_slot(gs, r & 31u, before);
+                gm_pbase[gp] = (oty + y) * TS * GM_WIN + (otx + x) * TS;
                 const uint32_t* m = gm_mask + (size_t)gp * MW;
 #pragma unroll
                 for (int q = 0; q < MW; ++q) before += __popc(__ldg(m + q));
             }
     }
+}
+
+// The LT index of every pair's first hit and the window index of its tile origin in the tile's rank order (what the
+// evaluation kernel walks); the former replaces, in place, the rank-ordered primitive-major positions.
+static __global__ void __launch_bounds__(256) gm_rank_ltb_kernel(uint32_t* __restrict__ rank_gpos, const uint32_t* __restrict__ gm_ltb,
+                                                                 const uint32_t* __restrict__ gm_pbase, uint32_t* __restrict__ rank_pbase,
+                                                                 const uint32_t* __restrict__ counts) {
+    if (counts[GART_CNT_ERROR]) return;
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= (int64_t)counts[GART_CNT_PAIRS]) return;
+    const uint32_t gp = rank_gpos[q];
+    rank_gpos[q] = __ldg(gm_ltb + gp);
+    rank_pbase[q] = __ldg(gm_pbase + gp);
 }
 
 // (super-tile, part) of every block of the backward; the block count.

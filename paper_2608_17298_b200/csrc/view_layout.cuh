@@ -30,6 +30,7 @@ struct ViewLayout {
     // tile-major
     uint32_t *pair_mask, *pair_order, *rank_sid, *rank_mask, *rank_gstart, *tile_lt_base;
     uint32_t *pair_gpos, *rank_gpos;   // primitive-major position of every pair, in pair order and in rank order
+    uint32_t *gm_pbase, *rank_pbase;   // index (y * GM_WIN + x) of the pair's tile origin in its owner's window, by primitive-major position and in rank order
     // primitive-major
     uint32_t* gpair_off;    // [n+1]  first primitive-major pair position of every slot
     uint32_t* gm_mask;      // [cap_pairs, MW] hit masks in primitive-major order (a Gaussian's tiles row by row)
@@ -78,6 +79,8 @@ static inline ViewLayout view_layout(void* base, int64_t n, int width, int heigh
     v.tile_lt_base = (uint32_t*)take((size_t)(T + 1) * 4);
     v.pair_gpos = (uint32_t*)take((size_t)cp * 4);
     v.rank_gpos = (uint32_t*)take((size_t)cp * 4);
+    v.gm_pbase = (uint32_t*)take((size_t)cp * 4);
+    v.rank_pbase = (uint32_t*)take((size_t)cp * 4);
     v.gpair_off = (uint32_t*)take((size_t)(nn + 1) * 4);
     v.gm_mask = (uint32_t*)take((size_t)cp * 4 * mw);
     v.gm_ltb = (uint32_t*)take((size_t)cp * 4);

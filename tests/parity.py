@@ -280,34 +280,52 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     dims = ntx[it_slot] | (it_ntx << 16) | (it_nty << 20) | ((fx - it_sx * tps) << 24) | ((fy - it_sy * tps) << 28)
     assert np.array_equal(desc[:, 2], dims[order])
     assert np.array_equal(desc[:, 3], (it_cnt | (it_whole.astype(np.int64) << 16))[order])
-    # groups of 32 ranks inside a super-tile occupy 32 x (largest count) entries
+    # groups of 32 ranks inside a super-tile occupy 32 x (largest count, rounded up to even) entries
     So, co = S_own[order], it_cnt[order]
     rank = np.arange(I) - st_off[So]
     first = rank % 32 == 0
-    gsize = 32 * co[first]
+    gsize = 32 * (co[first] + (co[first] & 1))
     gS = So[first]
     gstart = np.cumsum(gsize) - gsize                               # super-tiles are laid out one after the other
     assert np.array_equal(gpu["item_gstart"][:I].astype(np.int64), np.repeat(gstart, np.diff(np.r_[np.nonzero(first)[0], I])))
     st_len = np.bincount(gS, weights=gsize, minlength=NS).astype(np.int64)
     assert np.array_equal(gpu["st_lt_base"].astype(np.int64), np.concatenate([[0], np.cumsum(st_len)])) and st_len.sum() == L
-    # first LT entry of every pair
+    # LT entry of an item's e-th hit (e counts through the item's pairs in turn): entries go two by two, the two of a
+    # lane share a 32-byte sector, the 32 lanes' sectors of the same pair of entries are consecutive
+    def slot_of(gs, lane, e):
+        return gs + (e >> 1) * 64 + 2 * lane + (e & 1)
     pos_of_item = np.empty(I, np.int64)
     pos_of_item[order] = np.arange(I)
     g_of_item = gpu["item_gstart"][:I].astype(np.int64)[pos_of_item]
+    lane_of_item = rank[pos_of_item] % 32
     ltb = np.empty(P, np.int64)
-    ltb[pg] = g_of_item[pi] + rank[pos_of_item][pi] % 32 + 32 * before
+    ltb[pg] = slot_of(g_of_item[pi], lane_of_item[pi], before)
     assert np.array_equal(gpu["gm_ltb"].astype(np.int64), ltb)
+    item_of_gpos = np.empty(P, np.int64)
+    item_of_gpos[pg] = pi
+    before_g = np.empty(P, np.int64)
+    before_g[pg] = before
     # ---- per hit: on all rays, or on a random subset of them
     rays, idx = _sample_hits(cam, gpu, max_rays, seed)
     slots = gpu["ray_slot"][idx].astype(np.int64)
     gids = gpu["ray_gid"][idx].astype(np.int64)
     pair, below, _ = _locate_pairs(cam, cfg, gpu, rays, gids)
-    assert np.array_equal(slots, ltb[gpos[pair]] + 32 * below)      # the e-th hit of a pair: its e-th set mask bit in pixel order
+    it = item_of_gpos[gpos[pair]]                                   # the e-th hit of a pair: its e-th set mask bit in pixel order
+    assert np.array_equal(slots, slot_of(g_of_item[it], lane_of_item[it], before_g[gpos[pair]] + below))
     # LT: word 3 is the blending weight T alpha in (0, 1) with the three clamp flags in its low mantissa
     # bits; the vector part is finite.  (The values themselves are checked against the oracle's entries.)
     used = gpu["lt"][slots]
-    wgt = (np.ascontiguousarray(used[:, 3]).view(np.uint32) & np.uint32(0xFFFFFFF8)).view(np.float32)
+    bits = np.ascontiguousarray(used).view(np.uint32)
+    wgt = (bits[:, 3] & np.uint32(0xFFFFFFF0)).view(np.float32)
     assert np.all(np.isfinite(used)) and np.all(wgt >= 0) and np.all(wgt < 1.0)
+    # ... and the entry names its pixel inside the 32 x 32 window of the item's owner: ten bits spread over the low
+    # mantissa bits of the four words
+    pix = (bits[:, 0] & 7) | ((bits[:, 1] & 7) << 3) | ((bits[:, 2] & 7) << 6) | ((bits[:, 3] & 8) << 6)
+    own = S_own[it]
+    wx = rays % cam.width - (own % sup_x) * SUP
+    wy = rays // cam.width - (own // sup_x) * SUP
+    assert np.all((wx >= 0) & (wx < 2 * SUP) & (wy >= 0) & (wy < 2 * SUP))
+    assert np.array_equal(pix.astype(np.int64), wy * 2 * SUP + wx)
     assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
     return {"items": I, "whole_share": float(whole.mean()) if V else 1.0, "lt_padding": float(L) / max(H, 1)}
 
@@ -359,8 +377,12 @@ def check_structure_tile(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     rel = slots - base[tile]
     assert np.all(rel >= 0) and np.all(slots < base[tile + 1])
     assert np.array_equal(rel, slot0[pair] + 32 * below)
-    # the entries are the same numbers in both layouts
-    assert np.array_equal(t["lt"][slots], gpu["lt"][gpu["ray_slot"][idx].astype(np.int64)])
+    # the entries are the same numbers in both layouts, up to the low mantissa bits in which the primitive-major
+    # entries carry their pixel index
+    a = np.ascontiguousarray(t["lt"][slots]).view(np.uint32)
+    b = np.ascontiguousarray(gpu["lt"][gpu["ray_slot"][idx].astype(np.int64)]).view(np.uint32)
+    keep = np.array([0xFFFFFFF8, 0xFFFFFFF8, 0xFFFFFFF8, 0xFFFFFFF7], np.uint32)
+    assert np.array_equal(a & keep, b & keep)
 
 
 def _lists_for(ray_off, gid, rays):
