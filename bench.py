@@ -349,14 +349,14 @@ def run_ours(args):
     # ---- 8-byte LT entries (four halves per hit): forward and primitive-centric backward of the same view
     lt16_ms = None
     if args.lt16_reps > 0:
-        cfg_8 = dataclasses.replace(cfg, lt_format=2)
+        cfg_8 = dataclasses.replace(cfg, lt_format=2, lt_layout=G.LT_TILE_MAJOR)
         ft, bt = [], []
         for i in range(args.lt16_reps + 1):                      # one untimed run first
             e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
             e0.record(stream)
             G.run_forward(cfg_8, g, cams[last_v], buf, stream, ray_lists=False)
             e1.record(stream)
-            G.run_backward(cfg_8, g, cams[last_v], buf, dls[last_v], ga, stream)
+            G.run_backward_tile(cfg_8, g, cams[last_v], buf, dls[last_v], ga, stream)
             e2.record(stream)
             torch.cuda.synchronize()
             if i > 0:

@@ -80,7 +80,7 @@ typedef struct {
                              "Hybrid approach"); lt then holds cap_hits floats;
                              2 = the entry as four halves, 8 bytes per hit (the half-precision buffer that the
                              paper's limitations section, "VRAM Consumption", names as a way to save
-                             memory); gart_backward reads this format too */
+                             memory), for gart_backward_tile; formats 1 and 2 need lt_layout = GART_LT_TILE_MAJOR */
     int32_t max_hits;     /* 0: every hit of a ray is composited (the paper's benchmark sets no hit cap, Sec. 5).
                              m > 0: gart_forward composites only the first m hits of a ray in (t*, id)
                              order, the cap that the paper lists among the compromises of 3DGRT.  The hits behind
@@ -259,6 +259,10 @@ gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t ti
  *              formed among the items owned by one super-tile.  Entries go two by two: entry e of rank r sits at
  *              group start + 64 (e / 2) + 2 (r mod 32) + e mod 2 (the group's largest count is rounded up to even), so
  *              that a 32-byte sector holds two neighbouring hits of one Gaussian, which the forward writes close in time.
+ *              In this layout the entry also names its pixel: the 10-bit index y * 32 + x of the hit's pixel inside
+ *              the 32 x 32-pixel window whose corner is the owner super-tile's replaces the three low mantissa bits of
+ *              each of the words 0..2 (index bits 0..2, 3..5, 6..8) and bit 3 of word 3 (index bit 9) -- a relative
+ *              change below 2^-20 of numbers that are needed to 1e-3 -- so that the backward pass walks no hit mask.
  *   ray_off    [H*W+1] uint32 out; ray_gid, ray_slot [cap_hits] uint32 out: per ray, in
  *              compositing order, the Gaussian id and LT slot of each hit.  Only the pixel-centric
  *              baseline and parity checks read the two lists: pass NULL for both to skip them.
@@ -268,8 +272,8 @@ gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t ti
  *   by less than 32 x its largest count, and H <= S (the slot bound of gart_tile_map), so
  *   cap_hits = S + 32 tile_size^2 T (tile-major) or S + 32 * 1024 * NS (primitive-major) always suffices; the
  *   exact need is L.
- * Errors: INVALID_ARG also for an image wider or higher than 524280 pixels, and for lt_format 1 with the
- * primitive-major layout (the 4-byte format serves the hybrid pass, which is tile-major).
+ * Errors: INVALID_ARG also for an image wider or higher than 524280 pixels, and for lt_format 1 or 2 with the
+ * primitive-major layout (the 4- and 8-byte formats serve the tile-major passes).
  */
 size_t gart_forward_workspace_bytes(int32_t width, int32_t height, int32_t tile_size, int64_t cap_pairs, int64_t cap_hits);
 gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
@@ -294,11 +298,10 @@ gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const 
  *   view, cap_pairs: the view block that gart_forward filled and the capacity it was laid out for.
  *   counts: read (a set error bit skips the work); GART_ERRBIT_TIMEOUT is set if a wait on an
  *        asynchronous copy ran out, in which case grad is incomplete.
- * cfg->lt_format must be the one the forward wrote lt with, 0 or 2 (INVALID_ARG otherwise).  With 8-byte
- * entries every gradient word, being linear in the four words of its hits' entries, moves by at most 2^-10
- * of the sum of the absolute per-hit, per-channel terms of that word.
- * The main kernel uses 44 KB of dynamic shared memory per block: LT blocks are streamed in with bulk
- * asynchronous copies, one rank group ahead, beside dL/dC of the block's 32 x 32-pixel window.
+ * cfg->lt_format must be 0 (INVALID_ARG otherwise): the pass finds a hit's pixel in its 16-byte entry.
+ * The main kernel uses 54 KB of dynamic shared memory per block: LT blocks are streamed in with bulk
+ * asynchronous copies, one rank group ahead, beside dL/dC of the block's 32 x 32-pixel window and the
+ * Gaussians' records.
  */
 size_t gart_backward_workspace_bytes(int64_t n);
 gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
@@ -312,7 +315,9 @@ gart_status gart_backward(const gart_config *cfg, const gart_gaussians *g, const
  * (tile, Gaussian) pair; the thread walks the pair's hit pixels, accumulates in registers and performs one vector
  * atomic update per pair of the accumulation record of the Gaussian's slot; a per-Gaussian pass then converts the
  * accumulated moments and writes the gradient records.  Needs lt_layout = GART_LT_TILE_MAJOR.  Arguments, result
- * (up to summation order) and errors as gart_backward.  38 KB of dynamic shared memory per block.
+ * (up to summation order) and errors as gart_backward, but cfg->lt_format may be 0 or 2: with 8-byte
+ * entries every gradient word, being linear in the four words of its hits' entries, moves by at most 2^-10
+ * of the sum of the absolute per-hit, per-channel terms of that word.  38 KB of dynamic shared memory per block.
  */
 gart_status gart_backward_tile(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                                const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,

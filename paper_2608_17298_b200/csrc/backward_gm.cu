@@ -22,10 +22,6 @@
 #include "backward_common.cuh"
 #include "view_layout.cuh"
 
-#ifndef GMB_ABL
-#define GMB_ABL 0
-#endif
-
 namespace gart {
 
 constexpr int GMB_WARPS = 4;
@@ -33,10 +29,7 @@ constexpr int GMB_THREADS = GMB_WARPS * 32;
 constexpr int GMB_CHUNK = 6;                           // LT entries per lane and per pipeline stage (16-byte entries); even
 constexpr int GMB_STAGE_F4 = GMB_CHUNK * 32;           // float4 per stage
 constexpr int GMB_STAGES = 2;
-#ifndef GMB_MINB
-#define GMB_MINB 4
-#endif
-constexpr int GMB_MIN_BLOCKS = GMB_MINB;                      // resident blocks per SM that the register budget is set for
+constexpr int GMB_MIN_BLOCKS = 4;                      // resident blocks per SM that the register budget is set for
 constexpr int GMB_LT_SMEM = GMB_WARPS * GMB_STAGES * GMB_STAGE_F4 * 16;
 constexpr int GMB_PIX = GM_WIN * GM_WIN;
 constexpr int GMB_PF4 = 7;                             // float4 per lane of the staged per-Gaussian data: evaluation record 5, quaternion, scale + opacity
@@ -100,89 +93,6 @@ __device__ __forceinline__ ItemGeo item_geo(const PreRec& P, const uint4 d, int 
     return g;
 }
 
-// Walks the hit pixels of an item: its pairs row by row, each pair's mask bit by bit.  next() returns the pixel's index
-// in the window (y * GM_WIN + x); call it at most (hits of the item) times.
-template <int TS>
-struct ItemWalk {
-    static constexpr int MW = TS * TS / 32;
-    const uint32_t* mrow;   // masks of the current tile row of the item
-    uint32_t bits, stride;
-    int ntx, tx, wi, pbase, prow, togo;   // togo: pairs of the item after the current one
-    __device__ __forceinline__ void start(const uint32_t* __restrict__ gm_mask, const uint4 d, bool any) {
-        stride = d.z & 0xffffu;
-        ntx = (d.z >> 16) & 15;
-        const int otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
-        togo = ntx * (int)((d.z >> 20) & 15) - 1;
-        mrow = gm_mask + (size_t)d.y * MW;
-        tx = 0; wi = 0;
-        prow = oty * TS * GM_WIN + otx * TS;
-        pbase = prow;
-        bits = any ? __ldg(mrow) : 0u;
-    }
-    __device__ __forceinline__ int next() {
-        while (bits == 0u) {
-            if (++wi == MW) {
-                if (--togo < 0) return 0;   // (never: next() is called once per hit of the item; keeps a broken mask from spinning)
-                wi = 0;
-                pbase += TS;
-                if (++tx == ntx) { tx = 0; mrow += (size_t)stride * MW; prow += TS * GM_WIN; pbase = prow; }
-            }
-            bits = __ldg(mrow + tx * MW + wi);
-        }
-        const int b = __ffs((int)bits) - 1 + wi * 32;
-        bits &= bits - 1u;
-        return pbase + (b / TS) * GM_WIN + (b % TS);
-    }
-};
-
-// 64-pixel tiles: a pair's mask is one 8-byte word pair, and the mask of the pair after the current one is fetched
-// while the current one is walked (a lane changes pair every dozen hits, each lane at its own time: fetched on
-// demand, every change would stall the warp for a trip to L2).
-template <>
-struct ItemWalk<8> {
-    const uint2* mcur;      // mask of the pair being prefetched (row base + column)
-    uint32_t lo, hi, stride;
-    uint2 nx;               // the prefetched mask
-    int ntx, tx, ptx, togo, pbase, prow, boff;   // togo: pairs of the item after the current one
-    // fetch the mask of the pair `ahead` pairs after the current one (the cursor advances row by row)
-    __device__ __forceinline__ void prefetch(int ahead) {
-        if (togo >= ahead) {
-            if (++ptx == ntx) { ptx = 0; mcur += stride; }
-            nx = __ldg(mcur + ptx);
-        } else {
-            nx = make_uint2(0u, 0u);
-        }
-    }
-    __device__ __forceinline__ void start(const uint32_t* __restrict__ gm_mask, const uint4 d, bool any) {
-        stride = d.z & 0xffffu;
-        ntx = (d.z >> 16) & 15;
-        const int nty = (d.z >> 20) & 15, otx = (d.z >> 24) & 15, oty = (d.z >> 28) & 15;
-        mcur = reinterpret_cast<const uint2*>(gm_mask) + d.y;
-        tx = 0; ptx = 0; boff = 0;
-        prow = oty * 8 * GM_WIN + otx * 8;
-        pbase = prow;
-        togo = any ? ntx * nty - 1 : 0;
-        const uint2 m = any ? __ldg(mcur) : make_uint2(0u, 0u);
-        lo = m.x; hi = m.y;
-        prefetch(1);
-    }
-    __device__ __forceinline__ int next() {
-        while (lo == 0u) {
-            if (hi != 0u) { lo = hi; hi = 0u; boff = 32; }
-            else {
-                if (--togo < 0) return 0;   // (never: next() is called once per hit of the item; keeps a broken mask from spinning)
-                lo = nx.x; hi = nx.y; boff = 0;
-                pbase += 8;
-                if (++tx == ntx) { tx = 0; prow += 8 * GM_WIN; pbase = prow; }
-                prefetch(1);
-            }
-        }
-        const int b = __ffs((int)lo) - 1 + boff;
-        lo &= lo - 1u;
-        return pbase + (b >> 3) * GM_WIN + (b & 7);
-    }
-};
-
 // Coefficients of the un-normalised ray direction D = A x + B y + C through pixel (x, y) of the image: the same for the
 // whole launch, passed by value (operands from the constant bank: no registers).
 struct DirAffine {
@@ -232,19 +142,18 @@ __device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, f
     geo[6] = fmaf(tx, yy, geo[6]); geo[7] = fmaf(tx, yz, geo[7]); geo[8] = fmaf(ty, yz, geo[8]);
 }
 
-// FMT: 0 = 16-byte LT entries, 2 = 8-byte entries (four halves, twice as many per pipeline stage).
-template <int TS, int DEG, int FMT>
+template <int TS, int DEG>
 __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(const float4* __restrict__ rec, const float4* __restrict__ qs,
                                                              const uint32_t* __restrict__ gid_of_slot, const uint2* __restrict__ blk_desc,
                                                              const uint32_t* __restrict__ info, const uint32_t* __restrict__ st_off,
                                                              const uint4* __restrict__ rk_desc, const uint32_t* __restrict__ rk_gstart,
-                                                             const uint32_t* __restrict__ gm_mask, const float4* __restrict__ lt,
+                                                             const float4* __restrict__ lt,
                                                              const float* __restrict__ dL_dC, int width, int height, const DirAffine dir,
                                                              int sup_x, Gacc gacc,
                                                              float4* __restrict__ grad4, uint32_t* __restrict__ counts) {
     constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
-    constexpr int EB = FMT == 2 ? 8 : 16;                  // bytes per LT entry
+    constexpr int EB = 16;                                 // bytes per LT entry
     constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage (even)
     constexpr int PF4 = GMB_PF4, PSTR = GMB_PF4;           // staged per-Gaussian data; odd lane stride: the lanes' 16-byte reads fall into distinct banks
     extern __shared__ __align__(128) float4 dyn[];   // [warp][2][GMB_STAGE_F4] LT stages, dL/dC of the window, [thread][PF4] per-Gaussian data
@@ -365,9 +274,6 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
         const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale data for lanes without item: never used)
         issue_rec(nxt);        // the lane has read its record: that part of its buffer may be overwritten
         const ItemGeo IG = item_geo<TS>(P, cur.d, wx0, wy0);
-        // a 16-byte entry names its pixel (lt_pix); 8-byte entries have no room for that: their pixels come from the masks
-        ItemWalk<TS> walk;
-        if constexpr (FMT == 2) walk.start(gm_mask, cur.d, cur.c != 0);
         ShRegs<K> R;
         R.clear();
         float geo[11];
@@ -377,7 +283,7 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
         const int nchunks = (cme + CH - 1) / CH;
         // lanes 4..7 of every eight read the second entry of their sector first: the eight lanes that a 16-byte shared load
         // serves together then touch eight different bank groups (their sectors lie 32 bytes apart)
-        const bool flip = EB == 16 && (lane & 4) != 0;
+        const bool flip = (lane & 4) != 0;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % GMB_STAGES;
             if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / GMB_STAGES) & 1u))) { fail(); return; }
@@ -385,34 +291,16 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
             const char* se = reinterpret_cast<const char*>(my_stage + s * GMB_STAGE_F4) + lane * (2 * EB);
             const int e_end = min(cur.c, (k + 1) * CH);
             for (int e = k * CH; e < e_end; e += 2, se += 64 * EB) {
-                float4 L0, L1;
-                if constexpr (FMT == 2) {
-                    const uint4 t = *reinterpret_cast<const uint4*>(se);
-                    L0 = lt_unpack_half(make_uint2(t.x, t.y));
-                    L1 = lt_unpack_half(make_uint2(t.z, t.w));
-                } else {
-                    const float4 a = *reinterpret_cast<const float4*>(se + (flip ? 16 : 0));
-                    const float4 b = *reinterpret_cast<const float4*>(se + (flip ? 0 : 16));
-                    L0 = flip ? b : a;
-                    L1 = flip ? a : b;
-                }
-                // two hits per iteration: two independent dependency chains for the scheduler to interleave
-                int p0, p1 = 0;
-                if constexpr (FMT == 2) { p0 = walk.next(); if (e + 1 < e_end) p1 = walk.next(); }
-                else { p0 = (int)lt_pix(L0); p1 = (int)lt_pix(L1); }
+                const float4 a = *reinterpret_cast<const float4*>(se + (flip ? 16 : 0));
+                const float4 b = *reinterpret_cast<const float4*>(se + (flip ? 0 : 16));
+                const float4 L0 = flip ? b : a, L1 = flip ? a : b;
+                // two hits per iteration: two independent dependency chains for the scheduler to interleave; the entry
+                // names its pixel
                 if (e + 1 < e_end) {
-#if GMB_ABL == 1
-                    geo[0] += L0.x + L1.x + spix[p0].x + spix[p1].y;
-#else
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p0, L0);
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p1, L1);
-#endif
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L1), L1);
                 } else {
-#if GMB_ABL == 1
-                    geo[0] += L0.x + spix[p0].x;
-#else
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, p0, L0);
-#endif
+                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
                 }
             }
             fence_proxy_async();
@@ -421,11 +309,7 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
             produce(cur, nxt, c2_cmax, c2_gstart, 2);
         }
         // ---- the item's sums leave the registers
-#if GMB_ABL == 3
-        if (cur.valid && geo[0] == 123.456f) {
-#else
         if (cur.valid) {
-#endif
             if (whole) {
                 // the thread holds every hit of its Gaussian: convert the moments and write the gradient record once
                 cp_async_wait_but_one();   // (the tail data of this group; the next group's record may still be in flight)
@@ -533,15 +417,15 @@ static __global__ void __launch_bounds__(256) gm_fill_kernel(int64_t n, const ui
     }
 }
 
-template <int TS, int FMT>
+template <int TS>
 static gart_status launch_gm(int deg, unsigned grid, cudaStream_t st, const float4* rec, const float4* qs, const uint32_t* gid_of_slot,
                              const ViewLayout& v, const float4* lt, const float* dL_dC, const CamF& cam, int sup_x, const Gacc& gacc,
                              float4* grad4, uint32_t* counts) {
 #define GART_GM(D)                                                                                                                \
     {                                                                                                                            \
-        auto kern = bwd_gm_kernel<TS, D, FMT>;                                                                                   \
+        auto kern = bwd_gm_kernel<TS, D>;                                                                                   \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GMB_DYN_SMEM) != cudaSuccess) return GART_ERR_CUDA; \
-        kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, v.gm_mask, lt, \
+        kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, lt, \
                                                       dL_dC, cam.width, cam.height, make_dir_affine(cam), sup_x, gacc, grad4, counts); \
     }
     switch (deg) {
@@ -566,7 +450,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     (void)tile_off;
     if (!cfg || !g || !cam || !counts || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 0 && cfg->lt_format != 2) return GART_ERR_INVALID_ARG;   // this pass reads 16-byte or 8-byte LT entries
+    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;                          // this pass reads 16-byte LT entries (they name their pixel)
     if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR) return GART_ERR_INVALID_ARG;    // ... in the primitive-major layout
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
@@ -593,10 +477,8 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     GART_LAUNCH_CHECK();
     const unsigned grid = (unsigned)v.blocks_cap;
     gart_status s;
-#define GART_GM_TS(TSV, F) launch_gm<TSV, F>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts)
-    if (cfg->lt_format == 0) s = cfg->tile_size == 8 ? GART_GM_TS(8, 0) : GART_GM_TS(16, 0);
-    else s = cfg->tile_size == 8 ? GART_GM_TS(8, 2) : GART_GM_TS(16, 2);
-#undef GART_GM_TS
+    if (cfg->tile_size == 8) s = launch_gm<8>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts);
+    else s = launch_gm<16>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts);
     if (s != GART_OK) return s;
     gm_convert_big_kernel<<<slot_blocks, 256, 0, st>>>(srect, qs, gid_of_slot, gacc, grad4, counts);
     GART_LAUNCH_CHECK();

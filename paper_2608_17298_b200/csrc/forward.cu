@@ -591,9 +591,11 @@ __device__ __forceinline__ float strip_low_bit(float c) { return __uint_as_float
 
 // Index of the ray's pixel inside the 32 x 32-pixel window of a hit's owner: pixlow = (y mod 16) * 32 + x mod 16 from the
 // ray, plus the super-tile offsets that the evaluation left in the lowest bit of the hit's first two colour words;
-// -1 (nothing to embed) where pixlow < 0, i.e. in the tile-major layout.
-__device__ __forceinline__ int pix_of(int pixlow, float c0, float c1) {
-    return pixlow < 0 ? -1 : pixlow + (int)((__float_as_uint(c0) & 1u) * GM_SUP + (__float_as_uint(c1) & 1u) * (GM_SUP * GM_WIN));
+// -1 (nothing to embed) where pixlow < 0, i.e. in the tile-major layout.  A hit that is not composited (behind a hit cap)
+// gets index 0: its entry is all zero bits and adds exactly nothing, whatever pixel it names.
+__device__ __forceinline__ int pix_of(int pixlow, float c0, float c1, bool composited) {
+    if (pixlow < 0) return -1;
+    return composited ? pixlow + (int)((__float_as_uint(c0) & 1u) * GM_SUP + (__float_as_uint(c1) & 1u) * (GM_SUP * GM_WIN)) : 0;
 }
 
 // Store a hit's LT entry in the format the caller asked for: all 16 bytes (with the pixel's window index in the low
@@ -738,7 +740,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
                 const float cx = strip_low_bit(cs.x), cy = strip_low_bit(cs.y);
-                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2), pix_of(pixlow, cs.x, cs.y));
+                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2), pix_of(pixlow, cs.x, cs.y, i < n_comp));
                 if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cx, k0); k1 = fmaf(wgt, cy, k1); k2 = fmaf(wgt, cs.z, k2);
             }
@@ -850,7 +852,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
-            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2), pix_of(pixlow, rb.x, rb.y));
+            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2), pix_of(pixlow, rb.x, rb.y, i < n_comp));
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -1051,7 +1053,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0) return GART_ERR_INVALID_ARG;
     if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format == 1 && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // the 4-byte format serves the hybrid pass, which is tile-major
+    if (cfg->lt_format != 0 && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // the 4- and 8-byte formats serve the tile-major passes
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0 || cam->width > 65535 * 8 || cam->height > 65535 * 8) return GART_ERR_INVALID_ARG;

@@ -115,22 +115,16 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
             assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
             out["grad_hybrid"] = to_np(gh)[:g.n]
             assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
-        # 8-byte LT entries (four halves per hit): gart_backward on them (primitive-major) and the block-per-tile pass
+        # 8-byte LT entries (four halves per hit): the block-per-tile pass on them (tile-major layout)
         cfg_8t = dataclasses.replace(cfg_t, lt_format=2)
         G.run_forward(cfg_8t, g, cam, buf)
         g8 = torch.full_like(buf.grad, float("nan"))
         G.run_backward_tile(cfg_8t, g, cam, buf, dl, g8)
         torch.cuda.synchronize()
-        out["grad_lt16_tile"] = to_np(g8)[:g.n]
-        cfg_8 = dataclasses.replace(cfg, lt_format=2)
-        G.run_forward(cfg_8, g, cam, buf)
-        g8 = torch.full_like(buf.grad, float("nan"))
-        G.run_backward(cfg_8, g, cam, buf, dl, g8)
-        torch.cuda.synchronize()
         assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 0
         out["grad_lt16"] = to_np(g8)[:g.n]
-        out["lt16"] = to_np(buf.lt).reshape(-1).view(np.uint16)[:4 * counts[G.CNT_LT_SLOTS]].reshape(-1, 4).copy()
-        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_slot))[:H], out["ray_slot"])
+        out["lt16"] = to_np(buf.lt).reshape(-1).view(np.uint16)[:4 * tile["lt_slots"]].reshape(-1, 4).copy()
+        assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_slot))[:H], tile["ray_slot"])
     return out
 
 
@@ -325,7 +319,9 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     wx = rays % cam.width - (own % sup_x) * SUP
     wy = rays // cam.width - (own // sup_x) * SUP
     assert np.all((wx >= 0) & (wx < 2 * SUP) & (wy >= 0) & (wy < 2 * SUP))
-    assert np.array_equal(pix.astype(np.int64), wy * 2 * SUP + wx)
+    live = (idx - ray_off[rays] < cfg.max_hits) if cfg.max_hits > 0 else np.ones(idx.size, bool)   # composited hits
+    assert np.array_equal(pix.astype(np.int64)[live], (wy * 2 * SUP + wx)[live])
+    assert np.all((bits[~live] & np.uint32(0x7FFFFFF0)) == 0)      # a hit behind the cap: zero words (a sign or flag bit at most), pixel index 0
     assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
     return {"items": I, "whole_share": float(whole.mean()) if V else 1.0, "lt_padding": float(L) / max(H, 1)}
 
@@ -455,7 +451,7 @@ def check_lt16(gpu, ref):
     Only for a replay of every ray (the oracle's hit order is then the GPU's list order)."""
     import lt16
     entry, flags = ref["view"].lt_entries()
-    slots = gpu["ray_slot"].astype(np.int64)
+    slots = gpu["tile"]["ray_slot"].astype(np.int64)      # (8-byte entries live in the tile-major layout)
     assert entry.shape[0] == slots.size
     dec, f = lt16.decode(gpu["lt16"][slots])
     assert np.array_equal(f, flags)
