@@ -39,8 +39,8 @@
  *     entirely at depth <= near; it is "front" if the ellipsoid lies entirely
  *     at depth >= near, otherwise it "straddles" and its rectangle is the whole
  *     image unless its bounding sphere is outside one of the four side planes;
- *   - a ray hits a Gaussian iff alpha >= alpha_min and t* > 0; no early
- *     termination, no alpha clamp, no hit cap;
+ *   - a ray hits a Gaussian iff alpha >= alpha_min and t* > 0; by default no early
+ *     termination, no alpha clamp, no hit cap (each is an option, off unless set);
  *   - hits are ordered by (t*, id); colour is max(0, 0.5 + sum_k Y_k(d) sh_k)
  *     with d the unit ray direction; background colour multiplies T_final;
  *   - gradients are with respect to the given (activated) parameters; the
@@ -80,6 +80,12 @@ typedef struct {
     int64_t max_hits; /* 0: every hit is composited (the paper's setting).  m > 0: only the first m hits of a ray in
                          (t*, id) order, the cap on ray-primitive intersections that the paper lists among the
                          compromises of 3DGRT (comparison with prior work); later hits weigh nothing */
+    double t_min;     /* 0: off.  > 0: early termination, the other usual shortcut of such tracers: a ray ends before the
+                         first hit whose transmittance in front, T_i, is below t_min; that hit and all later ones weigh
+                         nothing (T_final is the transmittance reached) */
+    double alpha_max; /* >= 1: off.  < 1: a hit's alpha is min(sigma rho, alpha_max); where the clamp is active alpha is a
+                         constant, so the hit passes no gradient to opacity, mean, scale or rotation (its colour still
+                         gets one) */
 } orc_config;
 
 /* ------------------------------------------------------------------ threads */
@@ -323,6 +329,11 @@ typedef struct {
     double *Rs;        /* [H,3] colour composited behind the hit (after composite) */
     double *col;       /* [H,3] clamped colour of the hit */
     uint8_t *pos;      /* [H] bit c set if raw colour channel c > 0 */
+    double *ae;        /* [H] alpha as composited: min(alpha, alpha_max) (after composite) */
+    uint8_t *clamped;  /* [H] 1 where the clamp is active */
+    double *kap;       /* [H] kappa_i = sum over the composited hits j in front of i of alpha_j / (1 - alpha_j) */
+    double *Bk;        /* [H,3] conditioning of the colour behind the hit (see orc_view_lt_entries) */
+    double margin_t, margin_a; /* smallest |ln(T_i / t_min)| and |ln(alpha / alpha_max)| met by composite (decision margins) */
     int composited;
 } orc_view;
 
@@ -335,7 +346,9 @@ orc_view *orc_view_create(const orc_scene *s, const orc_camera *cam, const orc_c
 }
 static void view_free_hits(orc_view *v) {
     free(v->ray_off); free(v->gid); free(v->t); free(v->alpha); free(v->T); free(v->Rs); free(v->col); free(v->pos);
+    free(v->ae); free(v->clamped); free(v->kap); free(v->Bk);
     v->ray_off = NULL; v->gid = NULL; v->t = v->alpha = v->T = v->Rs = v->col = NULL; v->pos = NULL;
+    v->ae = v->kap = v->Bk = NULL; v->clamped = NULL;
     v->composited = 0;
 }
 void orc_view_destroy(orc_view *v) {
@@ -535,6 +548,10 @@ void orc_view_get_hits(const orc_view *v, uint64_t *ray_off, uint32_t *gid, doub
  * the hit (summed back to front), which the backward pass needs.
  * With a hit cap (cfg.max_hits > 0) the ray ends after its first max_hits hits: the hits behind keep their
  * place in the lists but get T_i = 0, so they add nothing to the colour, to T_final or to any gradient.
+ * Early termination (cfg.t_min > 0) ends the ray the same way before the first hit with T_i < t_min; the clamp
+ * (cfg.alpha_max < 1) composites min(alpha, alpha_max).
+ * Also kept per hit, for the error analysis of single-precision evaluations: kappa_i, the sum of alpha_j / (1 - alpha_j)
+ * over the composited hits in front (a relative error eps of every alpha_j moves ln T_i by at most eps kappa_i).
  */
 void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *hit_count) {
     const int64_t NR = v->n_rays;
@@ -545,46 +562,70 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
         v->Rs = (double *)malloc((size_t)(Hn + 1) * 3 * sizeof(double));
         v->col = (double *)malloc((size_t)(Hn + 1) * 3 * sizeof(double));
         v->pos = (uint8_t *)malloc((size_t)(Hn + 1));
+        v->ae = (double *)malloc((size_t)(Hn + 1) * sizeof(double));
+        v->clamped = (uint8_t *)malloc((size_t)(Hn + 1));
+        v->kap = (double *)malloc((size_t)(Hn + 1) * sizeof(double));
+        v->Bk = (double *)malloc((size_t)(Hn + 1) * 3 * sizeof(double));
     }
-#pragma omp parallel for schedule(dynamic, 64)
+    const double t_min = v->cfg.t_min, a_max = v->cfg.alpha_max;
+    double margin_t = INFINITY, margin_a = INFINITY;
+#pragma omp parallel for schedule(dynamic, 64) reduction(min : margin_t, margin_a)
     for (int64_t r = 0; r < NR; ++r) {
         const uint64_t b = v->ray_off[r], e = v->ray_off[r + 1];
-        double C[3] = {0, 0, 0}, T = 1.0;
+        double C[3] = {0, 0, 0}, T = 1.0, kappa = 0.0;
+        int ended = 0;
         if (e > b) {
             double d[3], Y[ORC_MAX_K];
             cam_ray_dir(&v->cam, (int)(r % v->cam.width), (int)(r / v->cam.width), d);
             orc_sh_basis(d, Y);
             for (uint64_t h = b; h < e; ++h) {
                 const double *sh = v->sc.sh + (size_t)v->gid[h] * K * 3;
-                const int capped = v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits;
+                if (!ended && t_min > 0.0) {
+                    if (fabs(log(T / t_min)) < margin_t) margin_t = fabs(log(T / t_min));
+                    if (T < t_min) ended = 1;
+                }
+                const int capped = ended || (v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits);
+                const double al = v->alpha[h] > a_max ? a_max : v->alpha[h];
+                v->ae[h] = al;
+                v->clamped[h] = v->alpha[h] > a_max;
+                if (a_max < 1.0 && !capped && fabs(log(v->alpha[h] / a_max)) < margin_a) margin_a = fabs(log(v->alpha[h] / a_max));
                 uint8_t pm = 0;
                 for (int c = 0; c < 3; ++c) {
                     double raw = 0.5;
                     for (int k = 0; k < K; ++k) raw += Y[k] * sh[3 * k + c];
                     if (raw > 0.0) pm |= (uint8_t)(1u << c);
                     v->col[3 * h + c] = raw > 0.0 ? raw : 0.0;
-                    if (!capped) C[c] += T * v->alpha[h] * v->col[3 * h + c];
+                    if (!capped) C[c] += T * al * v->col[3 * h + c];
                 }
                 v->pos[h] = pm;
                 v->T[h] = capped ? 0.0 : T;
-                if (!capped) T *= (1.0 - v->alpha[h]);
+                v->kap[h] = kappa;
+                if (!capped) { T *= (1.0 - al); kappa += al / (1.0 - al); }
             }
         }
         double Rb[3] = {T * v->cfg.bg[0], T * v->cfg.bg[1], T * v->cfg.bg[2]};
+        double Bk[3] = {kappa * fabs(Rb[0]), kappa * fabs(Rb[1]), kappa * fabs(Rb[2])};
         for (int c = 0; c < 3; ++c) C[c] += Rb[c];
         for (uint64_t h = e; h-- > b;) {
-            const int capped = v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits;
+            const int capped = v->T[h] == 0.0;   /* (not composited: behind a cap or behind the end of the ray) */
             for (int c = 0; c < 3; ++c) {
                 v->Rs[3 * h + c] = capped ? 0.0 : Rb[c];   /* nothing lies behind a hit that is not composited */
-                Rb[c] += v->T[h] * v->alpha[h] * v->col[3 * h + c];
+                v->Bk[3 * h + c] = capped ? 0.0 : Bk[c];
+                Rb[c] += v->T[h] * v->ae[h] * v->col[3 * h + c];
+                Bk[c] += (1.0 + v->kap[h]) * v->T[h] * v->ae[h] * v->col[3 * h + c];
             }
         }
         if (color) { color[3 * r] = C[0]; color[3 * r + 1] = C[1]; color[3 * r + 2] = C[2]; }
         if (t_final) t_final[r] = T;
         if (hit_count) hit_count[r] = (uint32_t)(e - b);
     }
+    v->margin_t = margin_t; v->margin_a = margin_a;
     v->composited = 1;
 }
+
+/* Smallest margins of the two floating-point decisions that the options add: out[0] = min |ln(T_i / t_min)| over the
+ * termination tests made, out[1] = min |ln(alpha / alpha_max)| over the composited hits (infinity where an option is off). */
+void orc_view_margins(const orc_view *v, double *out) { out[0] = v->margin_t; out[1] = v->margin_a; }
 
 /*
  * What the compact intermediate buffer (Sec. 4.3-4.4) has to hold per hit for the primitive-centric
@@ -594,15 +635,28 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
  *     alpha_i dC/dalpha_i = w c - alpha_i / (1 - alpha_i) B.
  * entry [H,4] receives that vector and w; flags [H] bit ch is set where colour channel ch is not
  * clamped (its SH gradient is w g_ch Y_k, zero otherwise).  Hit order = the view's lists.
+ * Where the alpha clamp is active alpha_i is a constant: the vector part, which only ever multiplies the derivative
+ * of alpha_i with respect to a parameter, is zero by definition; w = T_i alpha_max.
+ * cond [H,4] (may be NULL): how far a relative error eps of every alpha on the ray (what single precision leaves of
+ * alpha = sigma exp(-D^2 / 2)) can move each word, to first order, divided by eps.  With a_j = alpha_j / (1 - alpha_j)
+ * and kappa_i = sum of a_j over the composited hits in front: T_i moves by kappa_i eps (relative), w_i by
+ * (1 + kappa_i) eps, alpha_i / (1 - alpha_i) by (1 + a_i) eps, and B, a sum of w_j c_j behind and T_final bg, by
+ * sum (1 + kappa_j) w_j c_j + kappa_end T_final |bg| =: Bk.  Hence
+ *     cond[3] = (1 + kappa_i) w,   cond[c] = (1 + kappa_i) |w c_c| + alpha / (1 - alpha) ((1 + a_i) |B_c| + Bk_c).
  * Returns 0, or -1 if the view was not composited.
  */
-int orc_view_lt_entries(const orc_view *v, double *entry, uint8_t *flags) {
+int orc_view_lt_entries(const orc_view *v, double *entry, uint8_t *flags, double *cond) {
     if (!v->composited) return -1;
     const uint64_t Hn = v->ray_off[v->n_rays];
     for (uint64_t h = 0; h < Hn; ++h) {
-        const double al = v->alpha[h], w = v->T[h] * al;
-        for (int c = 0; c < 3; ++c) entry[4 * h + c] = w * v->col[3 * h + c] - al / (1.0 - al) * v->Rs[3 * h + c];
+        const double al = v->ae[h], w = v->T[h] * al, r = al / (1.0 - al);
+        for (int c = 0; c < 3; ++c) {
+            entry[4 * h + c] = v->clamped[h] ? 0.0 : w * v->col[3 * h + c] - r * v->Rs[3 * h + c];
+            if (cond) cond[4 * h + c] = v->clamped[h] ? 0.0 : (1.0 + v->kap[h]) * fabs(w * v->col[3 * h + c])
+                                                               + r * ((1.0 + r) * fabs(v->Rs[3 * h + c]) + v->Bk[3 * h + c]);
+        }
         entry[4 * h + 3] = w;
+        if (cond) cond[4 * h + 3] = (1.0 + v->kap[h]) * w;
         if (flags) flags[h] = v->pos[h];
     }
     return 0;
@@ -621,10 +675,14 @@ int orc_view_lt_entries(const orc_view *v, double *entry, uint8_t *flags) {
  * grad_abs_terms (may be NULL) splits once more: each channel's term is itself the difference of T alpha col_c and
  * alpha Rs_c / (1 - alpha), which nearly cancel where a hit has the colour of what lies behind it, and the scale
  * takes the sum of the two magnitudes: the mass of the products that any evaluation of Eq. 6-8 has to form.
+ * grad_cond (may be NULL): per gradient word, how far a relative error eps of every alpha (single-precision
+ * evaluation) can move it through the transmittances, divided by eps: the sum over the word's hits of the hit's
+ * sensitivity to its entry times the entry's conditioning `cond` of orc_view_lt_entries.  A hit behind nearly opaque
+ * ones (kappa in the hundreds) carries that factor however the sums are ordered.
  * Returns 0, or -1 if the view was not composited.
  */
 int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *grad_abs, double *grad_abs_elem,
-                      double *grad_abs_terms) {
+                      double *grad_abs_terms, double *grad_cond) {
     if (!v->composited) return -1;
     const int K = v->K, G = 11 + 3 * K;
     const int64_t NR = v->n_rays;
@@ -632,6 +690,7 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
     if (grad_abs) memset(grad_abs, 0, (size_t)v->sc.n * G * sizeof(double));
     if (grad_abs_elem) memset(grad_abs_elem, 0, (size_t)v->sc.n * G * sizeof(double));
     if (grad_abs_terms) memset(grad_abs_terms, 0, (size_t)v->sc.n * G * sizeof(double));
+    if (grad_cond) memset(grad_cond, 0, (size_t)v->sc.n * G * sizeof(double));
     double o[3];
     cam_origin(&v->cam, o);
 #pragma omp parallel for schedule(dynamic, 64)
@@ -644,18 +703,21 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
         const double *g = dL_dC + 3 * r;
         for (uint64_t h = b; h < e; ++h) {
             const int64_t i = v->gid[h];
-            const double al = v->alpha[h], T = v->T[h];
+            const double al = v->ae[h], T = v->T[h];
             double contrib[11 + 3 * ORC_MAX_K];
             /* colour -> SH */
             for (int k = 0; k < K; ++k) for (int c = 0; c < 3; ++c)
                 contrib[11 + 3 * k + c] = ((v->pos[h] >> c) & 1) ? Y[k] * T * al * g[c] : 0.0;
             /* alpha */
-            double dalpha = 0.0, dalpha_abs = 0.0, dalpha_terms = 0.0;
-            for (int c = 0; c < 3; ++c) {
+            double dalpha = 0.0, dalpha_abs = 0.0, dalpha_terms = 0.0, dalpha_cond = 0.0;
+            for (int c = 0; c < 3 && !v->clamped[h]; ++c) {   /* (a clamped alpha is a constant: no gradient through it) */
                 const double term = g[c] * (T * v->col[3 * h + c] - v->Rs[3 * h + c] / (1.0 - al));
                 dalpha += term;
                 dalpha_abs += fabs(term);
                 dalpha_terms += fabs(g[c]) * (fabs(T * v->col[3 * h + c]) + fabs(v->Rs[3 * h + c] / (1.0 - al)));
+                /* conditioning of alpha dL/dalpha = sum_c g_c entry_c, per unit of alpha (see orc_view_lt_entries) */
+                dalpha_cond += fabs(g[c]) * ((1.0 + v->kap[h]) * fabs(T * v->col[3 * h + c])
+                                             + ((1.0 + al / (1.0 - al)) * fabs(v->Rs[3 * h + c]) + v->Bk[3 * h + c]) / (1.0 - al));
             }
             const double sigma = v->sc.opacity[i];
             const double rho = al / sigma;
@@ -702,6 +764,17 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
                         const double a = fabs(contrib[k]) * (k < 11 ? split : 1.0);
 #pragma omp atomic
                         gt[k] += a;
+                    }
+                }
+            }
+            if (grad_cond) {
+                double *gc = grad_cond + (size_t)i * G;
+                const double split = dalpha != 0.0 ? dalpha_cond / fabs(dalpha) : 0.0;
+                for (int k = 0; k < G; ++k) {
+                    if (contrib[k] != 0.0) {
+                        const double a = fabs(contrib[k]) * (k < 11 ? split : 1.0 + v->kap[h]);
+#pragma omp atomic
+                        gc[k] += a;
                     }
                 }
             }

@@ -43,7 +43,8 @@ class _Scene(C.Structure):
 
 
 class _Config(C.Structure):
-    _fields_ = [("alpha_min", C.c_double), ("near_z", C.c_double), ("bg", C.c_double * 3), ("max_hits", C.c_int64)]
+    _fields_ = [("alpha_min", C.c_double), ("near_z", C.c_double), ("bg", C.c_double * 3), ("max_hits", C.c_int64),
+                ("t_min", C.c_double), ("alpha_max", C.c_double)]
 
 
 _lib = None
@@ -71,10 +72,11 @@ def lib():
         L.orc_view_num_hits.restype = C.c_int64
         L.orc_view_get_hits.argtypes = [C.c_void_p] + [C.c_void_p] * 4
         L.orc_view_composite.argtypes = [C.c_void_p] + [C.c_void_p] * 3
-        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 5
+        L.orc_view_backward.argtypes = [C.c_void_p] + [C.c_void_p] * 6
         L.orc_view_backward.restype = C.c_int
-        L.orc_view_lt_entries.argtypes = [C.c_void_p] + [C.c_void_p] * 2
+        L.orc_view_lt_entries.argtypes = [C.c_void_p] + [C.c_void_p] * 3
         L.orc_view_lt_entries.restype = C.c_int
+        L.orc_view_margins.argtypes = [C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -105,10 +107,11 @@ def _camera(cam) -> _Camera:
     return c
 
 
-def _config(alpha_min, near, bg, max_hits=0) -> _Config:
+def _config(alpha_min, near, bg, max_hits=0, t_min=0.0, alpha_max=1.0) -> _Config:
     c = _Config()
     c.alpha_min, c.near_z = float(alpha_min), float(near)
     c.max_hits = int(max_hits)
+    c.t_min, c.alpha_max = float(t_min), float(alpha_max)
     for i in range(3):
         c.bg[i] = float(bg[i])
     return c
@@ -183,10 +186,12 @@ PREFILTER = 1  # candidates from the projected bounding sphere, padded by one pi
 class View:
     """One camera view of a scene: hit discovery, ordering, compositing, backward."""
 
-    def __init__(self, scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, bg=(0.0, 0.0, 0.0), max_hits=0):
-        """max_hits > 0 composites only the first max_hits hits of every ray (0: all of them)."""
+    def __init__(self, scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, bg=(0.0, 0.0, 0.0), max_hits=0, t_min=0.0,
+                 alpha_max=1.0):
+        """max_hits > 0 composites only the first max_hits hits of every ray (0: all of them); t_min > 0 ends a ray before
+        the first hit with less than t_min transmittance in front of it; alpha_max < 1 clamps every hit's alpha."""
         self.scene, self.cam = scene, cam
-        self._c, self._g = _camera(cam), _config(alpha_min, near, bg, max_hits)
+        self._c, self._g = _camera(cam), _config(alpha_min, near, bg, max_hits, t_min, alpha_max)
         self.n_rays = int(cam.width) * int(cam.height)
         self._h = lib().orc_view_create(C.byref(scene.c), C.byref(self._c), C.byref(self._g))
         self._keep = None
@@ -239,32 +244,44 @@ class View:
         lib().orc_view_composite(self._h, _ptr(color), _ptr(t_final), _ptr(cnt))
         return color, t_final, cnt
 
-    def backward(self, dL_dC, with_abs=False, with_elem=False, with_terms=False):
+    def margins(self):
+        """(min |ln(T_i / t_min)| over the termination tests, min |ln(alpha / alpha_max)| over the composited hits) of
+        the last composite(): how close a floating-point decision of the two options came to flipping."""
+        out = np.zeros(2)
+        lib().orc_view_margins(self._h, _ptr(out))
+        return float(out[0]), float(out[1])
+
+    def backward(self, dL_dC, with_abs=False, with_elem=False, with_terms=False, with_cond=False):
         """Gradients [n, 11+3K] (mean 3, scale 3, quat 4, opacity 1, sh K*3) of sum <dL_dC, C>.
         with_abs adds the sums of absolute per-hit contributions, with_elem those of the contributions
         split by colour channel (the scale of an error that is relative to the per-hit quantities), with_terms
-        those with each channel's term split again into its two products (hit colour against colour behind)."""
+        those with each channel's term split again into its two products (hit colour against colour behind), with_cond
+        the first-order effect, per unit of relative error of every alpha, on each word through the transmittances."""
         g = _f64(dL_dC).reshape(self.n_rays, 3)
         G = self.scene.grad_words
         grad = np.zeros((self.scene.n, G))
         gabs = np.zeros((self.scene.n, G)) if with_abs else None
         gelem = np.zeros((self.scene.n, G)) if with_elem else None
         gterms = np.zeros((self.scene.n, G)) if with_terms else None
-        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs), _ptr(gelem), _ptr(gterms))
+        gcond = np.zeros((self.scene.n, G)) if with_cond else None
+        rc = lib().orc_view_backward(self._h, _ptr(g), _ptr(grad), _ptr(gabs), _ptr(gelem), _ptr(gterms), _ptr(gcond))
         if rc != 0:
             raise RuntimeError("composite() must run before backward()")
-        out = (grad,) + ((gabs,) if with_abs else ()) + ((gelem,) if with_elem else ()) + ((gterms,) if with_terms else ())
+        out = ((grad,) + ((gabs,) if with_abs else ()) + ((gelem,) if with_elem else ()) + ((gterms,) if with_terms else ())
+               + ((gcond,) if with_cond else ()))
         return out if len(out) > 1 else grad
 
-    def lt_entries(self):
+    def lt_entries(self, with_cond=False):
         """Per hit, in list order: (entry [H,4] = alpha dC/dalpha (3) and w = T alpha; flags [H] uint8, bit ch set
-        where colour channel ch is not clamped)."""
+        where colour channel ch is not clamped); with_cond adds cond [H,4], the first-order effect on each word of a
+        unit relative error of every alpha on the ray."""
         H = int(lib().orc_view_num_hits(self._h))
         entry = np.zeros((max(H, 1), 4))
         flags = np.zeros(max(H, 1), dtype=np.uint8)
-        if lib().orc_view_lt_entries(self._h, _ptr(entry), _ptr(flags)) != 0:
+        cond = np.zeros((max(H, 1), 4)) if with_cond else None
+        if lib().orc_view_lt_entries(self._h, _ptr(entry), _ptr(flags), _ptr(cond)) != 0:
             raise RuntimeError("composite() must run before lt_entries()")
-        return entry[:H], flags[:H]
+        return (entry[:H], flags[:H], cond[:H]) if with_cond else (entry[:H], flags[:H])
 
 
 def render(scene: OracleScene, cam, dL_dC=None, mode=BRUTE, pixel_mask=None, hit_lists=None, **kw):
