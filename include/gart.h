@@ -89,6 +89,14 @@ typedef struct {
                              read lt need no change; gart_backward_hybrid rejects a cap) */
     int32_t lt_layout;    /* GART_LT_PRIMITIVE_MAJOR (0, for gart_backward) or GART_LT_TILE_MAJOR (the ablation passes):
                              where gart_forward puts a hit's entry in lt.  The entries' contents are the same. */
+    float t_min;          /* 0: off (the paper's setting).  > 0: early termination, as in the tracers the paper compares with
+                             (Sec. 5.5): a ray ends before the first hit whose transmittance in front is below t_min; that
+                             hit and the later ones keep their place in every list and get a zero LT entry, like the hits
+                             behind max_hits; T_final is the transmittance reached */
+    float alpha_max;      /* >= 1: off (the paper's setting).  < 1: a hit's alpha is min(sigma rho, alpha_max).  Where the
+                             clamp is active alpha is a constant: the hit's LT entry has zero words 0..2 (no gradient to
+                             opacity, mean, scale, rotation) and w = T alpha_max (its colour still gets its gradient).
+                             gart_backward_hybrid takes neither option (it re-derives every alpha) */
 } gart_config;
 
 /* Host struct. */

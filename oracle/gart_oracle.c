@@ -333,6 +333,7 @@ typedef struct {
     uint8_t *clamped;  /* [H] 1 where the clamp is active */
     double *kap;       /* [H] kappa_i = sum over the composited hits j in front of i of alpha_j / (1 - alpha_j) */
     double *Bk;        /* [H,3] conditioning of the colour behind the hit (see orc_view_lt_entries) */
+    double *ray_margin; /* [n_rays, 2] the same two margins per ray */
     double margin_t, margin_a; /* smallest |ln(T_i / t_min)| and |ln(alpha / alpha_max)| met by composite (decision margins) */
     int composited;
 } orc_view;
@@ -346,7 +347,8 @@ orc_view *orc_view_create(const orc_scene *s, const orc_camera *cam, const orc_c
 }
 static void view_free_hits(orc_view *v) {
     free(v->ray_off); free(v->gid); free(v->t); free(v->alpha); free(v->T); free(v->Rs); free(v->col); free(v->pos);
-    free(v->ae); free(v->clamped); free(v->kap); free(v->Bk);
+    free(v->ae); free(v->clamped); free(v->kap); free(v->Bk); free(v->ray_margin);
+    v->ray_margin = NULL;
     v->ray_off = NULL; v->gid = NULL; v->t = v->alpha = v->T = v->Rs = v->col = NULL; v->pos = NULL;
     v->ae = v->kap = v->Bk = NULL; v->clamped = NULL;
     v->composited = 0;
@@ -566,13 +568,14 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
         v->clamped = (uint8_t *)malloc((size_t)(Hn + 1));
         v->kap = (double *)malloc((size_t)(Hn + 1) * sizeof(double));
         v->Bk = (double *)malloc((size_t)(Hn + 1) * 3 * sizeof(double));
+        v->ray_margin = (double *)malloc((size_t)(NR + 1) * 2 * sizeof(double));
     }
     const double t_min = v->cfg.t_min, a_max = v->cfg.alpha_max;
     double margin_t = INFINITY, margin_a = INFINITY;
 #pragma omp parallel for schedule(dynamic, 64) reduction(min : margin_t, margin_a)
     for (int64_t r = 0; r < NR; ++r) {
         const uint64_t b = v->ray_off[r], e = v->ray_off[r + 1];
-        double C[3] = {0, 0, 0}, T = 1.0, kappa = 0.0;
+        double C[3] = {0, 0, 0}, T = 1.0, kappa = 0.0, rm_t = INFINITY, rm_a = INFINITY;
         int ended = 0;
         if (e > b) {
             double d[3], Y[ORC_MAX_K];
@@ -581,14 +584,14 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
             for (uint64_t h = b; h < e; ++h) {
                 const double *sh = v->sc.sh + (size_t)v->gid[h] * K * 3;
                 if (!ended && t_min > 0.0) {
-                    if (fabs(log(T / t_min)) < margin_t) margin_t = fabs(log(T / t_min));
+                    if (fabs(log(T / t_min)) < rm_t) rm_t = fabs(log(T / t_min));
                     if (T < t_min) ended = 1;
                 }
                 const int capped = ended || (v->cfg.max_hits > 0 && h - b >= (uint64_t)v->cfg.max_hits);
                 const double al = v->alpha[h] > a_max ? a_max : v->alpha[h];
                 v->ae[h] = al;
                 v->clamped[h] = v->alpha[h] > a_max;
-                if (a_max < 1.0 && !capped && fabs(log(v->alpha[h] / a_max)) < margin_a) margin_a = fabs(log(v->alpha[h] / a_max));
+                if (a_max < 1.0 && !capped && fabs(log(v->alpha[h] / a_max)) < rm_a) rm_a = fabs(log(v->alpha[h] / a_max));
                 uint8_t pm = 0;
                 for (int c = 0; c < 3; ++c) {
                     double raw = 0.5;
@@ -618,6 +621,9 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
         if (color) { color[3 * r] = C[0]; color[3 * r + 1] = C[1]; color[3 * r + 2] = C[2]; }
         if (t_final) t_final[r] = T;
         if (hit_count) hit_count[r] = (uint32_t)(e - b);
+        v->ray_margin[2 * r] = rm_t; v->ray_margin[2 * r + 1] = rm_a;
+        if (rm_t < margin_t) margin_t = rm_t;
+        if (rm_a < margin_a) margin_a = rm_a;
     }
     v->margin_t = margin_t; v->margin_a = margin_a;
     v->composited = 1;
@@ -626,6 +632,13 @@ void orc_view_composite(orc_view *v, double *color, double *t_final, uint32_t *h
 /* Smallest margins of the two floating-point decisions that the options add: out[0] = min |ln(T_i / t_min)| over the
  * termination tests made, out[1] = min |ln(alpha / alpha_max)| over the composited hits (infinity where an option is off). */
 void orc_view_margins(const orc_view *v, double *out) { out[0] = v->margin_t; out[1] = v->margin_a; }
+
+/* The same two margins for every ray: out [n_rays, 2] (infinity where the ray met no such decision). */
+int orc_view_ray_margins(const orc_view *v, double *out) {
+    if (!v->composited) return 1;
+    memcpy(out, v->ray_margin, (size_t)v->cam.width * v->cam.height * 2 * sizeof(double));
+    return 0;
+}
 
 /*
  * What the compact intermediate buffer (Sec. 4.3-4.4) has to hold per hit for the primitive-centric

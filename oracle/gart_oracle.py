@@ -77,6 +77,8 @@ def lib():
         L.orc_view_lt_entries.argtypes = [C.c_void_p] + [C.c_void_p] * 3
         L.orc_view_lt_entries.restype = C.c_int
         L.orc_view_margins.argtypes = [C.c_void_p, C.c_void_p]
+        L.orc_view_ray_margins.argtypes = [C.c_void_p, C.c_void_p]
+        L.orc_view_ray_margins.restype = C.c_int
         _lib = L
     return _lib
 
@@ -250,6 +252,13 @@ class View:
         out = np.zeros(2)
         lib().orc_view_margins(self._h, _ptr(out))
         return float(out[0]), float(out[1])
+
+    def ray_margins(self):
+        """The same two margins per ray, [n_rays, 2] (infinity where a ray met no such decision)."""
+        out = np.zeros((self.n_rays, 2))
+        if lib().orc_view_ray_margins(self._h, _ptr(out)) != 0:
+            raise RuntimeError("composite() must run before ray_margins()")
+        return out
 
     def backward(self, dL_dC, with_abs=False, with_elem=False, with_terms=False, with_cond=False):
         """Gradients [n, 11+3K] (mean 3, scale 3, quat 4, opacity 1, sh K*3) of sum <dL_dC, C>.

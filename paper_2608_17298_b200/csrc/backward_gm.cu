@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
     constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
     constexpr int EB = 16;                                 // bytes per LT entry
     constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage (even)
-    constexpr int PF4 = GMB_PF4, PSTR = GMB_PF4;           // staged per-Gaussian data; odd lane stride: the lanes' 16-byte reads fall into distinct banks
+    constexpr int PSTR = GMB_PF4;                          // staged per-Gaussian data; odd lane stride: the lanes' 16-byte reads fall into distinct banks
     extern __shared__ __align__(128) float4 dyn[];   // [warp][2][GMB_STAGE_F4] LT stages, dL/dC of the window, [thread][PF4] per-Gaussian data
     __shared__ __align__(8) uint64_t bars[GMB_WARPS][GMB_STAGES];
     __shared__ uint32_t sgid[GMB_THREADS];   // staged id of the lane's Gaussian

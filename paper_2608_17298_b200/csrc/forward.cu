@@ -397,8 +397,8 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ rank_pbase,
-                                                                const uint32_t* __restrict__ ray_off, CamF cam, float4* __restrict__ recs,
-                                                                uint32_t* __restrict__ counts) {
+                                                                const uint32_t* __restrict__ ray_off, CamF cam, float alpha_max,
+                                                                float4* __restrict__ recs, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PF4 = (20 + SW + 3) / 4;
     constexpr int PSTR = PF4 | 1;   // odd lane stride: the lanes' 16-byte reads fall into distinct banks
     __shared__ __align__(16) float4 spix[EvalPix<TS>::F4];
@@ -493,7 +493,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
             // composites the words without that bit, so both layouts composite the very same numbers.
             c0 = __uint_as_float((__float_as_uint(fmaxf(c0, 0.0f)) & ~1u) | wdx);
             c1 = __uint_as_float((__float_as_uint(fmaxf(c1, 0.0f)) & ~1u) | wdy);
-            st_global_32B(out, make_float4(t, __uint_as_float(gid), __uint_as_float(slot_e), r.alpha),
+            st_global_32B(out, make_float4(t, __uint_as_float(gid), __uint_as_float(slot_e), fminf(r.alpha, alpha_max)),
                           make_float4(c0, c1, fmaxf(c2, 0.0f), 0.0f));
         };
         // two hits per iteration: two independent dependency chains for the scheduler to interleave.  The next hit's slot:
@@ -617,7 +617,7 @@ __device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32
 // slot as one float4, alpha apart; after the sort the three passes gather from there by sorted index.
 template <int R>
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx, int pixlow,
-                                               float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
+                                               float t_min, float alpha_max, float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                                                float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
     uint32_t k[R];
@@ -703,7 +703,29 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
     }
     float T0 = __shfl_up_sync(0xffffffffu, inc, 1);
     if (lane == 0) T0 = 1.0f;
-    const float Tfin = __shfl_sync(0xffffffffu, inc, 31);
+    float Tfin = __shfl_sync(0xffffffffu, inc, 31);
+    if (t_min > 0.0f) {
+        // early termination: the ray ends before the first hit whose transmittance in front is below t_min.  That hit and
+        // the later ones get alpha = 0 (they keep their place and their LT slot), T_final is the transmittance reached.
+        int first = 0x7fffffff;
+        float Tat = 0.0f, T = T0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (T < t_min && lane * R + r < n_comp && first == 0x7fffffff) { first = lane * R + r; Tat = T; }
+            T *= 1.0f - al[r];
+        }
+        int pstar = first;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pstar = min(pstar, __shfl_xor_sync(0xffffffffu, pstar, o));
+        if (pstar < n_comp) {
+            const unsigned owner = __ballot_sync(0xffffffffu, first == pstar);
+            Tfin = __shfl_sync(0xffffffffu, Tat, __ffs((int)owner) - 1);
+            n_comp = pstar;
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (lane * R + r >= pstar) al[r] = 0.0f;
+        }
+    }
     // back to front: colour composited behind every hit; first the lane totals ...
     float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f;
     {
@@ -740,7 +762,9 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const uint32_t slot = __float_as_uint(cs.w);
                 const float wgt = Ts[r] * al[r];
                 const float cx = strip_low_bit(cs.x), cy = strip_low_bit(cs.y);
-                lt_store(lt, lt_fmt, slot, lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2), pix_of(pixlow, cs.x, cs.y, i < n_comp));
+                float4 en = lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2);
+                if (al[r] >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }   // a clamped alpha is a constant: no gradient through it
+                lt_store(lt, lt_fmt, slot, en, pix_of(pixlow, cs.x, cs.y, i < n_comp));
                 if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cx, k0); k1 = fmaf(wgt, cy, k1); k2 = fmaf(wgt, cs.z, k2);
             }
@@ -783,7 +807,7 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
 }
 
 __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int n_comp, int lane, size_t b, int64_t r, int pixlow,
-                                            float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
+                                            float t_min, float alpha_max, float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                             float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
     for (int i = lane; i < n; i += 32) kp[i] = ((uint64_t)__float_as_uint(__ldg(&rec[2 * i].x)) << 32) | (uint64_t)i;
     __syncwarp();
@@ -806,6 +830,8 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         __syncwarp();
     }
     float carryT = 1.0f;
+    int pstar = 0x7fffffff;   // early termination: first position with less than t_min transmittance in front
+    float Tstar = 0.0f;
     for (int base = 0; base < n; base += 32) {
         const int i = base + lane;
         const bool valid = i < n;
@@ -822,8 +848,17 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         const float T = carryT * excl;
         if (valid) kp[i] = ((uint64_t)__float_as_uint(T) << 32) | (uint64_t)c;
         carryT *= __shfl_sync(0xffffffffu, prod, 31);
+        if (t_min > 0.0f && pstar == 0x7fffffff) {
+            const unsigned below = __ballot_sync(0xffffffffu, i < n_comp && T < t_min);
+            if (below) {
+                const int l0 = __ffs((int)below) - 1;
+                pstar = base + l0;
+                Tstar = __shfl_sync(0xffffffffu, T, l0);
+            }
+        }
     }
     __syncwarp();
+    if (pstar < n_comp) { n_comp = pstar; carryT = Tstar; }   // the hits from there on are not composited (their stored T is never used: alpha = 0)
     const float Tfin = carryT;
     float k0 = Tfin * bg0, k1 = Tfin * bg1, k2 = Tfin * bg2;
     for (int base = 0; base < n; base += 32) {
@@ -852,7 +887,9 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (lane == 0) { e0 = 0.0f; e1 = 0.0f; e2 = 0.0f; }
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
-            lt_store(lt, lt_fmt, slot, lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2), pix_of(pixlow, rb.x, rb.y, i < n_comp));
+            float4 en = lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2);
+            if (ra.w >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }
+            lt_store(lt, lt_fmt, slot, en, pix_of(pixlow, rb.x, rb.y, i < n_comp));
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -884,7 +921,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
                       int width, int tile_size, int tiles_x, int embed_pix,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                       float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
-                      int max_comp, const uint32_t* __restrict__ counts) {
+                      int max_comp, float t_min, float alpha_max, const uint32_t* __restrict__ counts) {
     constexpr int CAP = SweepClass<CLS>::CAP;
     constexpr int lt_fmt = FMT;
     if (counts[GART_CNT_ERROR]) return;
@@ -919,7 +956,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, pixlow, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
+#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
@@ -927,7 +964,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
-        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, pixlow, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
+        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
     }
 #undef GART_SWEEP
 }
@@ -974,14 +1011,14 @@ template <int TS, bool GMAJ>
 static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                const uint32_t* tile_lt_base, const uint32_t* rank_pbase, const uint32_t* ray_off,
-                               const CamF& cam, const ForwardWs& w, uint32_t* counts) {
+                               const CamF& cam, float alpha_max, const ForwardWs& w, uint32_t* counts) {
 #define GART_EVAL(D)                                                                                                        \
     {                                                                                                                      \
         auto kern = fwd_eval_kernel<TS, D, GMAJ>;                                                                          \
         constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
         kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, rank_pbase, ray_off, cam, \
-                                            w.recs, counts);                                                               \
+                                            alpha_max, w.recs, counts);                                                               \
     }
     switch (deg) {
         case 0: GART_EVAL(0); break;
@@ -1052,6 +1089,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0) return GART_ERR_INVALID_ARG;
+    if (!(cfg->t_min >= 0.0f) || !(cfg->t_min < 1.0f) || !(cfg->alpha_max > 0.0f)) return GART_ERR_INVALID_ARG;
     if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 0 && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // the 4- and 8-byte formats serve the tile-major passes
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
@@ -1075,6 +1113,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const bool gmaj = cfg->lt_layout == GART_LT_PRIMITIVE_MAJOR;
     const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
     gart_status s;
+    const float amax = cfg->alpha_max < 1.0f ? cfg->alpha_max : 2.0f;   // (2: no alpha reaches it, the clamp is off)
 
     // first primitive-major pair position of every slot (the mask kernel files every pair's mask there)
     if (cudaMemsetAsync(v.info, 0, GM_INFO_WORDS * 4, st) != cudaSuccess) return GART_ERR_CUDA;
@@ -1148,11 +1187,11 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     GART_LAUNCH_CHECK();
 
     if (gmaj) {
-        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
-        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
+        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
+        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
     } else {
-        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
-        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, w, counts);
+        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
+        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
     }
     if (s != GART_OK) return s;
 
@@ -1166,7 +1205,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
         if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
             return GART_ERR_CUDA;                                                                                                               \
         fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, (gmaj && lt_fmt == 0) ? 1 : 0, bg[0], \
-                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, counts); \
+                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, cfg->t_min, amax, counts); \
         GART_LAUNCH_CHECK();                                                                                                                    \
     }
 #define GART_SWEEP_BOTH(F) GART_SWEEP_LAUNCH(2, F) GART_SWEEP_LAUNCH(1, F)   // the longest rays first

@@ -48,7 +48,8 @@ class GartError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
-                ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32)]
+                ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32), ("t_min", C.c_float),
+                ("alpha_max", C.c_float)]
 
 
 class _Camera(C.Structure):
@@ -123,6 +124,8 @@ class Config:
     lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid); 2: 8 bytes (gart_backward)
     max_hits: int = 0           # > 0: only the first max_hits hits of a ray are composited (0: all, the paper's setting)
     lt_layout: int = 0          # 0: primitive-major LT (gart_backward); 1: tile-major (gart_backward_tile, _warp, _hybrid)
+    t_min: float = 0.0          # > 0: a ray ends before the first hit with less than t_min transmittance in front (0: off)
+    alpha_max: float = 1.0      # < 1: every hit's alpha is clamped to alpha_max (>= 1: off)
 
     def c(self) -> _Config:
         s = _Config()
@@ -130,6 +133,7 @@ class Config:
         s.lt_format = int(self.lt_format)
         s.max_hits = int(self.max_hits)
         s.lt_layout = int(self.lt_layout)
+        s.t_min, s.alpha_max = float(self.t_min), float(self.alpha_max)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s
@@ -142,6 +146,14 @@ class Config:
     @property
     def near_f32(self) -> float:
         return float(C.c_float(self.near_z).value)
+
+    @property
+    def t_min_f32(self) -> float:
+        return float(C.c_float(self.t_min).value)
+
+    @property
+    def alpha_max_f32(self) -> float:
+        return float(C.c_float(self.alpha_max).value)
 
 
 def camera_struct(cam) -> _Camera:

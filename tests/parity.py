@@ -105,7 +105,7 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         # the other outputs of the forward do not depend on the LT layout
         assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
         assert np.array_equal(tile["pair_mask"], out["pair_mask"])
-        if cfg.max_hits == 0:   # (the hybrid backward re-derives every alpha in its pixel pass: it takes no hit cap)
+        if cfg.max_hits == 0 and cfg.t_min == 0 and cfg.alpha_max >= 1:   # (the hybrid backward re-derives every alpha in its pixel pass: no cap, early end or clamp)
             # hybrid backward: the forward again with 4-byte LT entries
             cfg_h = dataclasses.replace(cfg_t, lt_format=1)
             G.run_forward(cfg_h, g, cam, buf)
@@ -319,9 +319,13 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     wx = rays % cam.width - (own % sup_x) * SUP
     wy = rays // cam.width - (own // sup_x) * SUP
     assert np.all((wx >= 0) & (wx < 2 * SUP) & (wy >= 0) & (wy < 2 * SUP))
-    live = (idx - ray_off[rays] < cfg.max_hits) if cfg.max_hits > 0 else np.ones(idx.size, bool)   # composited hits
-    assert np.array_equal(pix.astype(np.int64)[live], (wy * 2 * SUP + wx)[live])
-    assert np.all((bits[~live] & np.uint32(0x7FFFFFF0)) == 0)      # a hit behind the cap: zero words (a sign or flag bit at most), pixel index 0
+    # (a hit that is not composited -- behind a cap or behind the end of its ray -- has zero words, a sign or flag bit at
+    # most, and pixel index 0: it adds exactly nothing whatever pixel it names)
+    dead = np.all((bits & np.uint32(0x7FFFFFF0)) == 0, axis=1)
+    assert np.all((pix.astype(np.int64) == wy * 2 * SUP + wx) | (dead & (pix == 0)))
+    if cfg.max_hits > 0:
+        capped = idx - ray_off[rays] >= cfg.max_hits
+        assert np.all(dead[capped]) and (cfg.t_min > 0 or not dead[~capped].any())
     assert np.all(np.isfinite(gpu["color"])) and np.all(np.isfinite(gpu["grad"]))
     return {"items": I, "whole_share": float(whole.mean()) if V else 1.0, "lt_padding": float(L) / max(H, 1)}
 
@@ -436,15 +440,49 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     stats["identical_lists"] = bool(identical)
     assert stats["band_hit"] + stats["band_order"] <= max(2, 1e-3 * stats["oracle_hits"])
     # replay the GPU's lists
-    v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits)
+    v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits,
+                  t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0)
     v2.set_hits(g_new_off, g_sel_gid)
     color, t_final, cnt = v2.composite()
-    grad, gabs, gelem, gterms = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True, with_terms=True)
-    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "gelem": gelem, "gterms": gterms, "stats": stats,
+    stats["margin_t_min"], stats["margin_alpha_max"] = v2.margins()
+    grad, gabs, gelem, gterms, gcond = v2.backward(np.asarray(dL_dC, dtype=np.float64), with_abs=True, with_elem=True, with_terms=True,
+                                                   with_cond=True)
+    return {"color": color, "t_final": t_final, "grad": grad, "gabs": gabs, "gelem": gelem, "gterms": gterms, "gcond": gcond, "stats": stats,
             "sel": sel, "view": v2}
 
 
-def check_lt16(gpu, ref):
+LT32_EPS = 1e-5
+
+
+def check_lt32(gpu, ref, keep_rays=None):
+    """The 16-byte entries the forward wrote, in both layouts, against the oracle's entries of the same hits: the clamp
+    flags identical on every composited hit, and every word within LT32_EPS times the oracle's conditioning figure of the
+    word (the mass of the two products it is a difference of, plus the effect of a unit relative error of every alpha in
+    front of and at the hit: (1 + kappa) |w c| + r ((1 + r) |B| + B_kappa) with r = alpha / (1 - alpha); (1 + kappa) w for
+    the weight).  LT32_EPS = 1e-5 covers an alpha evaluated in single precision (a few 1e-6: the exponent is a
+    quadratic form of rounded inputs, and where its terms cancel, as for a camera inside a large Gaussian, its absolute error
+    of a few 1e-6 is alpha's relative error) plus the roundings of the products and of the sums B and T, and 2e-6 of the word for the (at most four) low mantissa bits that carry the flags and, in the
+    primitive-major layout, the pixel index.  Only for a replay of every ray.  Returns the largest error in units of
+    the bound."""
+    entry, flags, cond = ref["view"].lt_entries(with_cond=True)
+    hk = np.ones(entry.shape[0], bool) if keep_rays is None else np.repeat(keep_rays, np.diff(gpu["ray_off"].astype(np.int64)))
+    worst = 0.0
+    for lt, slots, mask in ((gpu["lt"], gpu["ray_slot"], (~7, ~7, ~7, ~15)), (gpu["tile"]["lt"], gpu["tile"]["ray_slot"], (~0, ~0, ~0, ~7))):
+        assert slots.size == entry.shape[0]
+        bits = np.ascontiguousarray(lt[slots.astype(np.int64)]).view(np.uint32).reshape(-1, 4)
+        f = (bits[:, 3] & 7).astype(np.uint8)
+        val = (bits & np.array(mask, np.int64).astype(np.uint32)).view(np.float32).astype(np.float64)
+        live = hk & (entry[:, 3] > 0)
+        assert np.array_equal(f[live], flags[live])
+        tol = LT32_EPS * cond + 2e-6 * np.abs(entry) + 1e-30
+        err = np.abs(val - entry)[hk] / tol[hk]
+        assert np.all(err <= 1.0), ("LT entry outside its bound", float(err.max()))
+        assert np.all(val[hk & (entry[:, 3] == 0)] == 0)           # a hit that is not composited: zero entry
+        worst = max(worst, float(err.max(initial=0.0)))
+    return worst
+
+
+def check_lt16(gpu, ref, keep_rays=None):
     """The 8-byte entries the forward wrote (lt_format 2) against the oracle's entries of the same hits: flags
     identical, every colour word within the encoding's 2^-10 and the weight within 2^-11, plus the fp32 error of
     the encoder's input (the colour word is a difference of two products of size about w and alpha/(1-alpha) B).
@@ -454,6 +492,9 @@ def check_lt16(gpu, ref):
     slots = gpu["tile"]["ray_slot"].astype(np.int64)      # (8-byte entries live in the tile-major layout)
     assert entry.shape[0] == slots.size
     dec, f = lt16.decode(gpu["lt16"][slots])
+    if keep_rays is not None:       # (rays left out of the comparison: see the caller)
+        hk = np.repeat(keep_rays, np.diff(gpu["ray_off"].astype(np.int64)))
+        entry, flags, dec, f = entry[hk], flags[hk], dec[hk], f[hk]
     assert np.array_equal(f, flags)
     x, w = entry[:, :3], entry[:, 3]
     fp32 = 1e-5 * (np.abs(x) + 8.0 * w[:, None])

@@ -11,6 +11,11 @@ terms whatever the summation order):
     as sum_c |g_c| (|T alpha col_c| + |alpha Rs_c / (1 - alpha)|) -- a hit whose colour is close to the colour behind it
     cancels inside one term.  A sum whose terms cancel to less than COND = 2% of their mass cannot reach a
     relative 1e-3 in fp32 in any summation order, so the relative bar is measured against that floor;
+    plus EPS_ALPHA * K, where K is the oracle's first-order effect on the word of a unit relative error of every alpha on
+    the word's rays (through the transmittances: a hit with alpha close to 1 in front multiplies the error of its own
+    alpha by alpha / (1 - alpha) in everything behind it, which no fp32 path avoids) and EPS_ALPHA = 3e-6 bounds the
+    relative error of an alpha evaluated in single precision (an exponential of a quadratic form of rounded inputs: a few
+    ulp of 6e-8 each from the form, the exponential and the product);
   * gradients from 8-byte LT entries (lt_format 2): the same bar plus 1.05 * 2^-10 * E, where E is the sum of
     the absolute per-hit terms split by colour channel.  Every gradient word is linear in the four words of the
     hit's entry, each stored to a relative 2^-10 (2^-11 for the weight), so that is the bound of the encoding;
@@ -31,6 +36,7 @@ import parity as P
 pytestmark = pytest.mark.gpu
 
 COND = 0.02
+EPS_ALPHA = 3e-6
 
 
 def assert_color(gpu, ref, sel, cam):
@@ -43,9 +49,9 @@ def assert_grad(gpu_grad, ref, K, rows=None):
     gw = 11 + 3 * K
     rows = np.arange(ref["grad"].shape[0]) if rows is None else rows
     g = gpu_grad[rows][:, :gw].astype(np.float64)
-    r, a = ref["grad"][rows], ref["gterms"][rows]
+    r, a, kc = ref["grad"][rows], ref["gterms"][rows], ref["gcond"][rows]
     d = np.abs(g - r)
-    ok = (d <= 1e-3 * np.maximum(np.abs(r), COND * a)) | (d <= 1e-6)
+    ok = (d <= 1e-3 * np.maximum(np.abs(r), COND * a) + EPS_ALPHA * kc) | (d <= 1e-6)
     assert ok.all(), ("gradient outside tolerance", int((~ok).sum()), float(d[~ok].max()))
     assert np.all(gpu_grad[rows][:, gw:] == 0)
     strict = (d <= 1e-3 * np.abs(r)) | (d <= 1e-6)
@@ -69,19 +75,43 @@ def assert_grad_lt16(gpu_grad, ref, K, rows=None):
 VARIANTS = ("grad", "grad_tile", "grad_atomic", "grad_hybrid", "grad_warp")   # every backward pass on 16-byte (4-byte: hybrid) entries
 
 
+OPTION_BAND = 1e-3    # rays with a termination or clamp decision closer than this (in ln) to its threshold carry no upstream gradient
+
+
+def option_band(scene, cam, cfg):
+    """Rays on which a decision of the options t_min / alpha_max comes within OPTION_BAND of flipping under float64:
+    |ln(T_i / t_min)| or |ln(alpha / alpha_max)| below the band.  Each option puts one more floating-point comparison on
+    the compositing path; on these rays single precision may take it the other way, which changes the ray's colour and its
+    hits' entries by a whole term.  The tests give such rays a zero upstream gradient and leave their colour unchecked (at
+    most a few per thousand); on every other ray the decisions are then required to be the oracle's."""
+    v = orc.View(orc.OracleScene.from_scene(scene), cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, max_hits=cfg.max_hits,
+                 t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0)
+    v.find_hits()
+    v.composite()
+    return (v.ray_margins() < OPTION_BAND).any(axis=1)
+
+
 def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
     g = gs.upstream_gradient(cam, 0) if g is None else g
+    keep = np.ones(cam.width * cam.height, bool)
+    if cfg.t_min > 0 or cfg.alpha_max < 1:
+        keep = ~option_band(scene, cam, cfg)
+        assert keep.mean() > 0.99
+        g = (np.asarray(g).reshape(-1, 3) * keep[:, None]).reshape(np.asarray(g).shape).astype(np.float32)
     gpu = P.run_gpu(scene, cam, cfg, g)
     assert gpu["counts"][G.CNT_ERROR] == 0
     m = P.check_maps(scene, cam, cfg, gpu)
     P.check_structure(cam, cfg, gpu)
     P.check_structure_tile(cam, cfg, gpu)
     ref = P.check_hits_and_replay(m["osc"], cam, cfg, gpu, g, None, mode)
-    assert_color(gpu, ref, ref["sel"], cam)
+    assert ref["view"].ray_margins()[keep].min(initial=np.inf) > 0.1 * OPTION_BAND   # (the replayed lists are the GPU's: a guard-band hit may move a margin a little)
+    ref["keep"] = keep
+    assert_color(gpu, ref, ref["sel"][keep], cam)
     K = (scene.sh_degree + 1) ** 2
     strict = {v: assert_grad(gpu[v], ref, K) for v in VARIANTS if v in gpu}
     assert min(strict.values()) > 0.995, strict            # the conditioning floor is the exception, not the rule
-    P.check_lt16(gpu, ref)
+    ref["lt32_worst"] = P.check_lt32(gpu, ref, keep)
+    P.check_lt16(gpu, ref, keep)
     assert assert_grad_lt16(gpu["grad_lt16"], ref, K) > 0.85
     ref["strict"] = strict
     return gpu, ref
@@ -133,20 +163,18 @@ def test_hit_cap(m):
 @pytest.mark.parametrize("seed", [101, 102, 103, 104, 105, 106])
 def test_random_configurations(seed):
     """Random combinations of image size (ragged against both tile sizes), field of view, SH degree, tile size, background,
-    alpha_min and hit cap on a random cluster, every ray and every backward variant against the oracle."""
+    alpha_min, hit cap, early termination and alpha clamp on a random cluster, every ray and every backward variant against the oracle."""
     rng = np.random.default_rng(seed)
     deg = int(rng.integers(0, 4))
     width, height = int(rng.integers(40, 150)), int(rng.integers(30, 110))
     scene, cams = gs.config_cluster(n=int(rng.integers(500, 5000)), sh_degree=deg, width=width, height=height, seed=seed)
-    # opacities below 0.98: behind a hit with 1 - alpha of a few 1e-4 the transmittance, and with it every gradient word of
-    # the Gaussians behind, carries the fp32 error of that alpha (1e-6) divided by 1 - alpha, which no fp32 path can avoid
-    scene.opacity[:] = np.minimum(scene.opacity, 0.98)
     # a camera somewhere around the cluster (centre (0, 0, 3)), looking near its centre, any field of view
     dirv = rng.normal(size=3)
     pos = np.array([0.0, 0.0, 3.0]) + float(rng.uniform(2.0, 4.0)) * dirv / np.linalg.norm(dirv)
     cam = gs.pinhole(width, height, float(rng.uniform(25.0, 75.0)), gs.look_at(pos, np.array([0.0, 0.0, 3.0]) + rng.uniform(-0.2, 0.2, 3)))
     cfg = G.Config(tile_size=int(rng.choice([8, 16])), background=tuple(float(v) for v in rng.uniform(0, 1, 3)),
                    alpha_min=float(rng.choice([1.0 / 255.0, 0.01, 0.03])), max_hits=int(rng.choice([0, 0, 3, 17])))
+    cfg.t_min, cfg.alpha_max = float(rng.choice([0.0, 0.0, 0.03, 0.2])), float(rng.choice([1.0, 1.0, 0.95, 0.6]))
     gpu, ref = full_parity(scene, cam, cfg, g=gs.upstream_gradient(cam, seed))
     assert gpu["counts"][G.CNT_HITS] > 100
 
@@ -162,7 +190,7 @@ def test_random_cameras_inside_the_cloud(seed):
     mean = rng.uniform(-1.0, 1.0, (n, 3))
     scale = np.exp(rng.uniform(np.log(0.003), np.log(0.6), (n, 3)))
     scene = gs.Scene(mean.astype(np.float32), scale.astype(np.float32), gs._unit_quats(rng, n).astype(np.float32),
-                     np.minimum(gs._sigmoid(rng.normal(0, 2.0, n)), 0.98).astype(np.float32), gs._sh(rng, n, deg), deg)
+                     gs._sigmoid(rng.normal(0, 2.0, n)).astype(np.float32), gs._sh(rng, n, deg), deg)
     cam = gs.pinhole(width, height, float(rng.uniform(20.0, 100.0)), gs.look_at(rng.uniform(-1.5, 1.5, 3), rng.uniform(-0.5, 0.5, 3)))
     cam = gs.Camera(cam.width, cam.height, cam.fx, cam.fx * float(rng.uniform(0.8, 1.25)), cam.cx + float(rng.uniform(-5, 5)),
                     cam.cy + float(rng.uniform(-5, 5)), cam.w2c)
@@ -170,6 +198,37 @@ def test_random_cameras_inside_the_cloud(seed):
                    alpha_min=float(rng.choice([1.0 / 255.0, 0.02])), max_hits=int(rng.choice([0, 0, 0, 5])))
     gpu, ref = full_parity(scene, cam, cfg, g=gs.upstream_gradient(cam, seed))
     assert gpu["counts"][G.CNT_HITS] > 0
+
+
+def test_early_termination():
+    """t_min: a ray ends before the first hit with less than t_min transmittance in front of it; colour, T_final, LT
+    entries and every gradient follow the oracle's early-terminated compositing; lists and counts still hold every hit."""
+    scene, cams = gs.config_cluster(n=4000, width=120, height=96, seed=23)
+    cam = cams[0]
+    t_min = 0.05
+    gpu, ref = full_parity(scene, cam, G.Config(t_min=t_min, background=(0.2, 0.1, 0.3)))
+    free, _ = full_parity(scene, cam, G.Config(background=(0.2, 0.1, 0.3)))
+    keep = ref["keep"].reshape(cam.height, cam.width)
+    assert not keep.all()                                           # (the band is met on a view of this size: the protocol is exercised)
+    assert np.array_equal(gpu["ray_gid"], free["ray_gid"]) and np.array_equal(gpu["hit_count"], free["hit_count"])
+    ended = gpu["t_final"] < t_min
+    assert 0.05 < ended.mean() < 0.95
+    assert np.all(gpu["t_final"] >= free["t_final"] - 1e-6) and np.abs(gpu["color"] - free["color"]).max() > 1e-3
+    same = ~ended & (free["t_final"] >= 1.01 * t_min)              # rays that never meet the threshold are untouched, to the bit
+    assert same.any() and np.array_equal(gpu["color"][same], free["color"][same])
+
+
+def test_alpha_clamp():
+    """alpha_max: every hit composites min(alpha, alpha_max); a clamped hit passes no gradient through alpha."""
+    scene, cams = gs.config_cluster(n=4000, width=120, height=96, seed=24)
+    scene.opacity[::3] = np.float32(0.97)
+    cam = cams[0]
+    a_max = 0.9
+    gpu, ref = full_parity(scene, cam, G.Config(alpha_max=a_max))
+    free, _ = full_parity(scene, cam, G.Config())
+    assert np.abs(gpu["color"] - free["color"]).max() > 1e-3 and np.all(gpu["t_final"] >= free["t_final"] - 1e-7)
+    # both options with a cap, on the tile-major passes too (full_parity runs every variant)
+    full_parity(scene, cam, G.Config(alpha_max=a_max, max_hits=9, tile_size=16))
 
 
 def test_stricter_alpha_min():
@@ -423,13 +482,16 @@ def test_invalid_arguments_return_status():
         (G.run_backward_hybrid, G.Config(lt_format=2, lt_layout=TM)),
         (G.run_backward_hybrid, G.Config(lt_format=1)),
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, max_hits=4)),
+        (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, t_min=0.01)),
+        (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, alpha_max=0.99)),
         (G.run_backward_hybrid, G.Config(lt_format=0, lt_layout=TM)),
     ]
     for fn, cfg_bad in refused:
         with pytest.raises(G.GartError) as e:
             fn(cfg_bad, g, cam, buf, dl)
         assert e.value.status == 1, (fn.__name__, cfg_bad)
-    for cfg_bad in (G.Config(max_hits=-1), G.Config(lt_format=3), G.Config(lt_layout=2), G.Config(lt_format=1), G.Config(lt_format=2)):
+    for cfg_bad in (G.Config(max_hits=-1), G.Config(lt_format=3), G.Config(lt_layout=2), G.Config(lt_format=1), G.Config(lt_format=2),
+                    G.Config(t_min=1.0), G.Config(t_min=-0.1), G.Config(alpha_max=0.0)):
         with pytest.raises(G.GartError) as e:
             G.run_forward(cfg_bad, g, cam, buf)
         assert e.value.status == 1, cfg_bad
