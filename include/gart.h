@@ -97,6 +97,13 @@ typedef struct {
                              clamp is active alpha is a constant: the hit's LT entry has zero words 0..2 (no gradient to
                              opacity, mean, scale, rotation) and w = T alpha_max (its colour still gets its gradient).
                              gart_backward_hybrid takes neither option (it re-derives every alpha) */
+    int32_t wait_polls;   /* 0: the library's limit (2^22 polls) on every wait of a kernel for one of its own asynchronous
+                             copies; > 0: that many polls; < 0: no poll at all, so every such wait gives up at once (a test
+                             hook for the path below).  A wait that gives up sets GART_ERRBIT_TIMEOUT in
+                             counts[GART_CNT_ERROR]; the warp then waits, with the library's limit, for its copies in flight
+                             and returns.  The call's outputs are then undefined, the context stays usable, and
+                             gart_sync_status returns GART_ERR_TIMEOUT.  Read by gart_backward, gart_backward_tile and
+                             gart_backward_hybrid (the kernels that stream the intermediate buffer through shared memory). */
 } gart_config;
 
 /* Host struct. */

@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base,
                                                                 const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                Gacc gacc, uint32_t* __restrict__ counts) {
+                                                                Gacc gacc, uint32_t* __restrict__ counts, const uint32_t wait_limit) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;   // accumulator words, multiple of 4
     constexpr int EB = FMT == 2 ? 8 : 16;                  // bytes per LT entry
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
         const int nchunks = (cur.cmax + CH - 1) / CH;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % BWD_STAGES;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / BWD_STAGES) & 1u))) { fail(); return; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / BWD_STAGES) & 1u, wait_limit))) { fail(); return; }
             const char* sl = reinterpret_cast<const char*>(my_stage + s * BWD_STAGE_F4) + lane * EB;   // entry j of the stage: sl + j * 32 * EB
             auto entry = [&](const char* q) {
                 if constexpr (FMT == 2) return lt_unpack_half(*reinterpret_cast<const uint2*>(q));
@@ -291,11 +291,11 @@ template <int TS, int DEG, int FMT>
 static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                     const uint32_t* tile_lt_base, const float4* lt,
-                                    const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
+                                    const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts, uint32_t wait_limit) {
     auto kern = bwd_pairs_kernel<TS, DEG, FMT>;
     constexpr int smem = BWD_DYN_SMEM;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
-    kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts);
+    kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }
@@ -304,9 +304,9 @@ template <int TS, int FMT>
 static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                 const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                 const uint32_t* tile_lt_base, const float4* lt,
-                                const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts) {
+                                const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts, uint32_t wait_limit) {
 #define GART_PAIRS(D) \
-    return launch_pairs_deg<TS, D, FMT>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts)
+    return launch_pairs_deg<TS, D, FMT>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit)
     switch (deg) {
         case 0: GART_PAIRS(0);
         case 1: GART_PAIRS(1);
@@ -360,7 +360,7 @@ extern "C" gart_status gart_backward_tile(const gart_config* cfg, const gart_gau
     const int T = cf.tiles_x * cf.tiles_y;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
-#define GART_PAIRS_TS(TSV, F) launch_pairs<TSV, F>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts)
+#define GART_PAIRS_TS(TSV, F) launch_pairs<TSV, F>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts, wait_limit_of(cfg->wait_polls))
     if (cfg->lt_format == 0) s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 0) : GART_PAIRS_TS(16, 0);
     else s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 2) : GART_PAIRS_TS(16, 2);
 #undef GART_PAIRS_TS

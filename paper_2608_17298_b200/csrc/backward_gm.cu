@@ -150,7 +150,8 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
                                                              const float4* __restrict__ lt,
                                                              const float* __restrict__ dL_dC, int width, int height, const DirAffine dir,
                                                              int sup_x, Gacc gacc,
-                                                             float4* __restrict__ grad4, uint32_t* __restrict__ counts) {
+                                                             float4* __restrict__ grad4, uint32_t* __restrict__ counts,
+                                                             const uint32_t wait_limit) {
     constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
     constexpr int EB = 16;                                 // bytes per LT entry
@@ -286,7 +287,7 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
         const bool flip = (lane & 4) != 0;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % GMB_STAGES;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / GMB_STAGES) & 1u))) { fail(); return; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / GMB_STAGES) & 1u, wait_limit))) { fail(); return; }
             // entries 2m and 2m + 1 of the lane: the 2 EB bytes at row m (32 lanes x 2 EB bytes) + lane x 2 EB
             const char* se = reinterpret_cast<const char*>(my_stage + s * GMB_STAGE_F4) + lane * (2 * EB);
             const int e_end = min(cur.c, (k + 1) * CH);
@@ -420,13 +421,13 @@ static __global__ void __launch_bounds__(256) gm_fill_kernel(int64_t n, const ui
 template <int TS>
 static gart_status launch_gm(int deg, unsigned grid, cudaStream_t st, const float4* rec, const float4* qs, const uint32_t* gid_of_slot,
                              const ViewLayout& v, const float4* lt, const float* dL_dC, const CamF& cam, int sup_x, const Gacc& gacc,
-                             float4* grad4, uint32_t* counts) {
+                             float4* grad4, uint32_t* counts, uint32_t wait_limit) {
 #define GART_GM(D)                                                                                                                \
     {                                                                                                                            \
         auto kern = bwd_gm_kernel<TS, D>;                                                                                   \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GMB_DYN_SMEM) != cudaSuccess) return GART_ERR_CUDA; \
         kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, lt, \
-                                                      dL_dC, cam.width, cam.height, make_dir_affine(cam), sup_x, gacc, grad4, counts); \
+                                                      dL_dC, cam.width, cam.height, make_dir_affine(cam), sup_x, gacc, grad4, counts, wait_limit); \
     }
     switch (deg) {
         case 0: GART_GM(0); break;
@@ -477,8 +478,8 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     GART_LAUNCH_CHECK();
     const unsigned grid = (unsigned)v.blocks_cap;
     gart_status s;
-    if (cfg->tile_size == 8) s = launch_gm<8>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts);
-    else s = launch_gm<16>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts);
+    if (cfg->tile_size == 8) s = launch_gm<8>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
+    else s = launch_gm<16>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
     if (s != GART_OK) return s;
     gm_convert_big_kernel<<<slot_blocks, 256, 0, st>>>(srect, qs, gid_of_slot, gacc, grad4, counts);
     GART_LAUNCH_CHECK();

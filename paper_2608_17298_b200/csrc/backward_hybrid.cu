@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
                                                              const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                              const uint32_t* __restrict__ tile_lt_base, const float* __restrict__ lt_w,
                                                              const float* __restrict__ dL_dC, CamF cam, Gacc gacc,
-                                                             uint32_t* __restrict__ counts) {
+                                                             uint32_t* __restrict__ counts, const uint32_t wait_limit) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PIXF4 = PixLayout<TS>::F4;
     constexpr int AW = (11 + SW + 3) & ~3;
     __shared__ __align__(128) float stage[HYB_WARPS][HYB_STAGES][HYB_STAGE_WORDS];
@@ -108,7 +108,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
         const int nchunks = (cur.cmax + HYB_CHUNK - 1) / HYB_CHUNK;
         for (int k = 0; k < nchunks; ++k) {
             const uint32_t s = unit % HYB_STAGES;
-            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / HYB_STAGES) & 1u))) { fail(); return; }
+            if (!__all_sync(0xffffffffu, mbar_wait_bounded(bar_addr + 8u * s, (unit / HYB_STAGES) & 1u, wait_limit))) { fail(); return; }
             const float* sl = &stage[warp][s][lane];
             const int e_end = min(cur.c, (k + 1) * HYB_CHUNK);
             auto hit = [&](const int p, const float wv) {
@@ -222,8 +222,8 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
 template <int TS>
 static gart_status launch_sh(int deg, int T, cudaStream_t st, const uint32_t* tile_off, const uint32_t* rank_sid, const uint32_t* rank_mask,
                              const uint32_t* rank_gstart, const uint32_t* tile_lt_base, const float* lt_w, const float* dL_dC,
-                             const CamF& cam, const Gacc& gacc, uint32_t* counts) {
-#define GART_SH(D) bwd_sh_kernel<TS, D><<<T, HYB_THREADS, 0, st>>>(tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dC, cam, gacc, counts)
+                             const CamF& cam, const Gacc& gacc, uint32_t* counts, uint32_t wait_limit) {
+#define GART_SH(D) bwd_sh_kernel<TS, D><<<T, HYB_THREADS, 0, st>>>(tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dC, cam, gacc, counts, wait_limit)
     switch (deg) {
         case 0: GART_SH(0); break;
         case 1: GART_SH(1); break;
@@ -264,8 +264,8 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int T = cf.tiles_x * cf.tiles_y;
     const float4* rec = reinterpret_cast<const float4*>(pre);
-    if (cfg->tile_size == 8) s = launch_sh<8>(g->sh_degree, T, st, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dcolor, cf, gacc, counts);
-    else s = launch_sh<16>(g->sh_degree, T, st, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dcolor, cf, gacc, counts);
+    if (cfg->tile_size == 8) s = launch_sh<8>(g->sh_degree, T, st, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dcolor, cf, gacc, counts, wait_limit_of(cfg->wait_polls));
+    else s = launch_sh<16>(g->sh_degree, T, st, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt_w, dL_dcolor, cf, gacc, counts, wait_limit_of(cfg->wait_polls));
     if (s != GART_OK) return s;
     const int64_t n_rays = (int64_t)cam->width * cam->height;
     const unsigned blocks = (unsigned)ceil_div(n_rays, 128);

@@ -361,8 +361,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0u;
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < ASYNC_WAIT_LIMIT; ++i)
+// the limit a configuration asks for (gart_config::wait_polls)
+static inline uint32_t wait_limit_of(int32_t wait_polls) {
+    return wait_polls == 0 ? ASYNC_WAIT_LIMIT : (wait_polls < 0 ? 0u : (uint32_t)wait_polls);
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = ASYNC_WAIT_LIMIT) {
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -49,7 +49,7 @@ class GartError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
                 ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32), ("t_min", C.c_float),
-                ("alpha_max", C.c_float)]
+                ("alpha_max", C.c_float), ("wait_polls", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -126,6 +126,7 @@ class Config:
     lt_layout: int = 0          # 0: primitive-major LT (gart_backward); 1: tile-major (gart_backward_tile, _warp, _hybrid)
     t_min: float = 0.0          # > 0: a ray ends before the first hit with less than t_min transmittance in front (0: off)
     alpha_max: float = 1.0      # < 1: every hit's alpha is clamped to alpha_max (>= 1: off)
+    wait_polls: int = 0         # 0: library limit on a kernel's waits for its own copies; > 0: polls; < 0: every wait gives up (test hook)
 
     def c(self) -> _Config:
         s = _Config()
@@ -134,6 +135,7 @@ class Config:
         s.max_hits = int(self.max_hits)
         s.lt_layout = int(self.lt_layout)
         s.t_min, s.alpha_max = float(self.t_min), float(self.alpha_max)
+        s.wait_polls = int(self.wait_polls)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s

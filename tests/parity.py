@@ -46,7 +46,31 @@ def _view_arrays(buf, names, P, mw):
     return out
 
 
-def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, atomic=True):
+GUARD_BYTES = 1024
+GUARDED = ("rect", "cls", "pre", "slot_of_gid", "gid_of_slot", "tile_off", "pair_gid", "view", "color", "t_final", "hit_count", "lt",
+           "ray_off", "ray_gid", "ray_slot", "grad", "workspace")
+
+
+def guard_buffers(buf):
+    """Re-seat every device buffer of the view between two guard zones of GUARD_BYTES filled with a pattern (the buffer
+    keeps its size, type and 256-byte alignment).  Returns the backing tensors for check_guards."""
+    backing = {}
+    for nme in GUARDED:
+        t = getattr(buf, nme)
+        nb = t.numel() * t.element_size()
+        flat = torch.full((nb + 2 * GUARD_BYTES,), 0xA5, dtype=torch.uint8, device=t.device)
+        setattr(buf, nme, flat[GUARD_BYTES:GUARD_BYTES + nb].view(t.dtype).view(t.shape))
+        backing[nme] = (flat, nb)
+    return backing
+
+
+def check_guards(backing):
+    """No kernel wrote in front of or behind any buffer."""
+    for nme, (flat, nb) in backing.items():
+        assert bool((flat[:GUARD_BYTES] == 0xA5).all()) and bool((flat[GUARD_BYTES + nb:] == 0xA5).all()), ("guard zone of %s overwritten" % nme)
+
+
+def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, atomic=True, guard=False):
     """Full device path for one view; returns numpy copies of every output.  The view runs in the primitive-major LT
     layout (gart_backward); with atomic=True the other backward variants follow: the pixel-centric baseline on the
     same buffers, then the forward again in the tile-major layout for the block-per-tile pass, the warp-per-pair pass
@@ -58,6 +82,7 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         cap_pairs = P if cap_pairs is None else cap_pairs
         cap_hits = S if cap_hits is None else cap_hits
     buf = G.ViewBuffers(g.n, g.sh_degree, cam, cfg, cap_pairs, cap_hits)
+    backing = guard_buffers(buf) if guard else None
     buf.grad.fill_(float("nan"))          # every record must be written by the backward pass
     dl = torch.from_numpy(np.ascontiguousarray(dL_dC, dtype=np.float32)).cuda()
     G.run_bounds_tile_map(cfg, g, cam, buf)
@@ -70,6 +95,8 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
     out["rect"], out["cls"] = to_np(buf.rect)[:g.n], to_np(buf.cls)[:g.n]
     out["tile_off"] = u32(to_np(buf.tile_off))
     if counts[G.CNT_ERROR]:
+        if guard:
+            check_guards(backing)
         return out
     out["pair_gid"] = u32(to_np(buf.pair_gid))[:P]
     out["slot_of_gid"], out["gid_of_slot"] = u32(to_np(buf.slot_of_gid))[:g.n], u32(to_np(buf.gid_of_slot))[:g.n]
@@ -125,6 +152,9 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         out["grad_lt16"] = to_np(g8)[:g.n]
         out["lt16"] = to_np(buf.lt).reshape(-1).view(np.uint16)[:4 * tile["lt_slots"]].reshape(-1, 4).copy()
         assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_slot))[:H], tile["ray_slot"])
+    if guard:
+        torch.cuda.synchronize()
+        check_guards(backing)
     return out
 
 

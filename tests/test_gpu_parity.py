@@ -91,14 +91,14 @@ def option_band(scene, cam, cfg):
     return (v.ray_margins() < OPTION_BAND).any(axis=1)
 
 
-def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE):
+def full_parity(scene, cam, cfg, g=None, mode=orc.BRUTE, guard=False, caps=(None, None)):
     g = gs.upstream_gradient(cam, 0) if g is None else g
     keep = np.ones(cam.width * cam.height, bool)
     if cfg.t_min > 0 or cfg.alpha_max < 1:
         keep = ~option_band(scene, cam, cfg)
         assert keep.mean() > 0.99
         g = (np.asarray(g).reshape(-1, 3) * keep[:, None]).reshape(np.asarray(g).shape).astype(np.float32)
-    gpu = P.run_gpu(scene, cam, cfg, g)
+    gpu = P.run_gpu(scene, cam, cfg, g, cap_pairs=caps[0], cap_hits=caps[1], guard=guard)
     assert gpu["counts"][G.CNT_ERROR] == 0
     m = P.check_maps(scene, cam, cfg, gpu)
     P.check_structure(cam, cfg, gpu)
@@ -229,6 +229,22 @@ def test_alpha_clamp():
     assert np.abs(gpu["color"] - free["color"]).max() > 1e-3 and np.all(gpu["t_final"] >= free["t_final"] - 1e-7)
     # both options with a cap, on the tile-major passes too (full_parity runs every variant)
     full_parity(scene, cam, G.Config(alpha_max=a_max, max_hits=9, tile_size=16))
+
+
+@pytest.mark.parametrize("ts", [8, 16])
+def test_no_write_outside_any_buffer(ts):
+    """Every device buffer of the view sits between two guard zones; after the whole path in every variant (both LT
+    layouts, three entry formats, five backward passes) with the capacities at their exact need, the zones are untouched."""
+    scene, cams = gs.config_cluster(n=3000, width=150, height=90, seed=31)
+    cfg = G.Config(tile_size=ts)
+    g = G.Gaussians.from_numpy(scene)
+    pairs, _ = G.size_view(cfg, g, cams[0], slack=1.0)
+    probe = P.run_gpu(scene, cams[0], cfg, gs.upstream_gradient(cams[0], 0))
+    need = max(int(probe["counts"][G.CNT_LT_SLOTS]), int(probe["tile"]["lt_slots"]))     # (the larger of the two layouts' needs)
+    full_parity(scene, cams[0], cfg, guard=True, caps=(pairs - 1, need))
+    # one entry short: the forward reports it and writes nothing outside
+    short = P.run_gpu(scene, cams[0], cfg, gs.upstream_gradient(cams[0], 0), cap_pairs=pairs - 1, cap_hits=need - 1, atomic=False, guard=True)
+    assert short["counts"][G.CNT_ERROR] != 0
 
 
 def test_stricter_alpha_min():
@@ -442,6 +458,39 @@ def test_capacity_errors_are_reported_not_fatal():
     # and the context is still usable afterwards
     gpu = P.run_gpu(scene, cam, cfg, g, atomic=False)
     assert gpu["counts"][G.CNT_ERROR] == 0 and gpu["counts"][G.CNT_HITS] == 7373
+
+
+@pytest.mark.parametrize("variant", ["primitive", "tile", "hybrid"])
+def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(variant):
+    """wait_polls < 0: every wait of the streaming kernel for its own copies gives up without a poll.  The call returns,
+    the time-out bit is set and gart_sync_status says so; the view run again on the same buffers with the normal limit gives
+    the oracle's gradients.  Nothing faults and nothing hangs: the waits that give up are the kernel's own bounded ones."""
+    scene, cams = gs.config_tiny()
+    cam = cams[0]
+    cfg = {"primitive": G.Config(), "tile": G.Config(lt_layout=G.LT_TILE_MAJOR),
+           "hybrid": G.Config(lt_layout=G.LT_TILE_MAJOR, lt_format=1)}[variant]
+    fn = {"primitive": G.run_backward, "tile": G.run_backward_tile, "hybrid": G.run_backward_hybrid}[variant]
+    g = G.Gaussians.from_numpy(scene)
+    pairs, slots = G.size_view(cfg, g, cam)
+    buf = G.ViewBuffers(g.n, g.sh_degree, cam, cfg, pairs, slots)
+    dl_np = gs.upstream_gradient(cam, 0)
+    dl = torch.from_numpy(np.ascontiguousarray(dl_np, dtype=np.float32)).cuda()
+
+    def view(c):
+        G.run_bounds_tile_map(c, g, cam, buf)
+        G.run_forward(c, g, cam, buf)
+        buf.grad.fill_(float("nan"))
+        fn(c, g, cam, buf, dl)
+        return G.gart_sync_status(buf.counts)
+
+    assert view(dataclasses.replace(cfg, wait_polls=-1)) == 5                       # GART_ERR_TIMEOUT
+    assert G.gart_read_counts(buf.counts)[G.CNT_ERROR] == 4                         # GART_ERRBIT_TIMEOUT alone
+    assert view(dataclasses.replace(cfg, wait_polls=1 << 20)) == G.GART_OK          # (an explicit limit)
+    assert view(cfg) == G.GART_OK
+    got = buf.grad.cpu().numpy()[:g.n]
+    ref = orc.render(orc.OracleScene.from_scene(scene), cam, dL_dC=dl_np, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    K = (scene.sh_degree + 1) ** 2
+    assert np.allclose(got[:, :11 + 3 * K], ref["grad"], rtol=2e-3, atol=2e-5)
 
 
 def test_invalid_arguments_return_status():
