@@ -49,12 +49,25 @@ def _radix_passes(n_keys: int) -> int:
     return (bits + 7) // 8
 
 
-def launches_per_step(tiles_x: int, tiles_y: int) -> int:
-    """Kernel launches of one step (memsets are not kernels).  A radix pass is histogram + three scan kernels + scatter."""
-    bounds = 1 + _radix_passes(tiles_y) * 5 + 1                  # bounds kernel, slot sort on the tile row, record gather
-    tile_map = 1 + 3 + 1 + 1 + _radix_passes(tiles_x * tiles_y - 1) * 5 + 1   # areas, scan, total, emission, pair sort, offsets
-    forward = 1 + 1 + 3 + 3 + 1 + 1 + 2          # mask, tile sort, two scans, totals, evaluation, sweep per ray-length class
-    backward = 4                                # zero, pair kernel, per-slot conversion, scatter of the SH gradient
+def launches_per_step(width: int, height: int, tile_size: int, layout: str = "tile") -> int:
+    """Kernel launches of one step (memsets are not kernels).  A scan is three kernels, a radix pass histogram + scan +
+    scatter."""
+    tiles = -(-width // tile_size) * -(-height // tile_size)
+    sups_x, sups_y = -(-width // 16), -(-height // 16)           # super-tiles of 16 x 16 pixels
+    scan, radix = 3, 5
+    tile_map = 1 + scan + 1 + 1 + _radix_passes(tiles - 1) * radix + 1   # areas, scan, total, emission, pair sort, offsets
+    if layout == "tile":
+        bounds = 1 + _radix_passes(sups_y) * radix + 1           # bounds kernel, slot sort on the corner's super-tile row, record gather
+        forward = 1 + 1 + scan + scan + 1 + 1 + 2                # mask, tile sort, entries per tile, ray offsets, totals, evaluation, sweep per ray-length class
+        backward = 4                                             # zero, pair kernel, per-slot conversion, scatter of the SH gradient
+        return bounds + tile_map + forward + backward
+    sups = sups_x * sups_y
+    bounds = 1 + _radix_passes(sups) * radix + 1                 # ... slot sort on the corner's super-tile
+    forward = (scan + 1 + 1 + scan                               # pairs per slot, mask, tile sort, entries per tile
+               + scan + 1 + 1 + _radix_passes(sups - 1) * radix  # items per slot, total, emission, item sort on the super-tile
+               + 1 + 1 + 1 + scan + scan + 1 + 1 + 1             # segment offsets, descriptors, ranking, two scans, blocks, LT bases, per-rank copy
+               + scan + 1 + 1 + 2)                               # ray offsets, totals, evaluation, sweep per ray-length class
+    backward = 4                                                 # records of cut Gaussians zeroed, zero rows, item kernel, conversion of cut Gaussians
     return bounds + tile_map + forward + backward
 
 
@@ -65,18 +78,28 @@ def algorithmic_bytes_backward(H, P, n_vis, n_pixels, K):
     return 16 * H + 4 * P + 4 * (13 + 3 * K) * n_vis + 4 * (11 + 3 * K) * n_vis + 28 * n_pixels
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the four kernels of gart_backward, from the ncu capture
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels of gart_backward, from the ncu captures
 # summarised in profiles/dram_traffic_unbounded6m_crop.md (8x8 tiles, SH degree 3, central crop of a view), each
-# divided by the unit it grows with: the pair kernel by hits, zeroing and conversion by visible Gaussians, the
-# scatter's reads by visible Gaussians and its writes by all Gaussians.
-TRAFFIC_MODEL = {"pairs_per_hit": 45.0, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
-                 "scatter_read_per_visible": 186.0, "scatter_write_per_gaussian": 220.7}
+# divided by the unit it grows with.  Tile-major layout: the pair kernel by hits, zeroing and conversion by visible
+# Gaussians, the scatter's reads by visible Gaussians and its writes by all Gaussians.  Primitive-major layout: the item
+# kernel's reads by LT entries (it streams the padded buffer) and its writes by visible Gaussians, the zero rows by the
+# Gaussians without a slot, the two kernels for cut Gaussians by visible Gaussians.  `--crop 0.5` prints the units of the captured case in roofline.traffic_units, so
+# that a fresh capture divides into these figures.
+TRAFFIC_MODEL = {
+    "tile": {"pairs_per_hit": 45.0, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
+             "scatter_read_per_visible": 186.0, "scatter_write_per_gaussian": 220.7},
+    "primitive": {"items_read_per_lt_entry": 21.91, "items_write_per_visible": 235.7, "fill_write_per_invisible": 238.6,
+                  "fill_read_per_gaussian": 4.0, "big_per_visible": 38.8},
+}
 
 
-def measured_traffic_backward(H, n_vis, n):
-    t = TRAFFIC_MODEL
-    return (t["pairs_per_hit"] * H + (t["zero_per_visible"] + t["convert_per_visible"] + t["scatter_read_per_visible"]) * n_vis
-            + t["scatter_write_per_gaussian"] * n)
+def measured_traffic_backward(layout, H, L, n_vis, n):
+    t = TRAFFIC_MODEL[layout]
+    if layout == "tile":
+        return (t["pairs_per_hit"] * H + (t["zero_per_visible"] + t["convert_per_visible"] + t["scatter_read_per_visible"]) * n_vis
+                + t["scatter_write_per_gaussian"] * n)
+    return (t["items_read_per_lt_entry"] * L + (t["items_write_per_visible"] + t["big_per_visible"]) * n_vis
+            + t["fill_write_per_invisible"] * (n - n_vis) + t["fill_read_per_gaussian"] * n)
 
 
 def fp32_instr_backward(H, K):
@@ -165,22 +188,43 @@ def oracle_sample(scene, cam, seed=0, frac=0.02, tile=8):
     return np.ascontiguousarray(mask.astype(np.uint8))
 
 
-def time_oracle(scene, cam, dL_dC, frac, threads=None):
-    """Oracle (as it stands) on a bounded sample of the view: hit discovery + ordering + compositing +
-    backward for the sampled rays.  Returns (hits, seconds, threads)."""
+def time_oracle(scene, cam, dL_dC, frac, threads=None, split=False):
+    """Oracle (as it stands) on a bounded sample of the view (frac >= 1: every ray): hit discovery + ordering +
+    compositing + backward for the sampled rays.  Returns (hits, seconds, threads, rays); with split=True the seconds are
+    (forward, backward)."""
     from oracle import gart_oracle as orc
+    all_threads = orc.max_threads()
     if threads:
         orc.set_threads(threads)
     osc = orc.OracleScene.from_scene(scene)
-    mask = oracle_sample(scene, cam, frac=frac)
+    mask = oracle_sample(scene, cam, frac=frac) if frac < 1.0 else None
     t0 = time.perf_counter()
     v = orc.View(osc, cam, alpha_min=float(np.float32(1.0 / 255.0)), near=float(np.float32(0.01)))
     H = v.find_hits(orc.PREFILTER, mask)
     v.composite()
+    t1 = time.perf_counter()
     v.backward(np.asarray(dL_dC, dtype=np.float64))
-    dt = time.perf_counter() - t0
+    t2 = time.perf_counter()
     v.close()
-    return H, dt, orc.max_threads(), int(mask.sum())
+    used = orc.max_threads()
+    if threads:
+        orc.set_threads(all_threads)
+    rays = int(mask.sum()) if mask is not None else cam.width * cam.height
+    return H, ((t1 - t0, t2 - t1) if split else t2 - t0), used, rays
+
+
+def oracle_detail(config="cluster10k"):
+    """The oracle on every ray of one view of a small configuration, forward (hit discovery, ordering, compositing) and
+    backward timed separately, with all host threads and with one."""
+    scene, cams = gs.make(config)
+    cam = cams[0]
+    g = gs.upstream_gradient(cam, 0)
+    out = {"workload": config, "unit": UNIT}
+    for key, thr in (("all_threads", None), ("one_thread", 1)):
+        H, (tf, tb), used, rays = time_oracle(scene, cam, g, 1.0, threads=thr, split=True)
+        out[key] = {"cores": used, "hits": H, "forward_s": tf, "backward_s": tb, "value": H / (tf + tb),
+                    "forward_hits_per_s": H / tf, "backward_hits_per_s": H / tb}
+    return out
 
 
 def run_reference(args):
@@ -227,7 +271,9 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    cfg = G.Config(tile_size=args.tile_size)
+    tile_major = args.lt_layout == "tile"
+    cfg = G.Config(tile_size=args.tile_size, lt_layout=G.LT_TILE_MAJOR if tile_major else G.LT_PRIMITIVE_MAJOR)
+    run_backward = G.run_backward_tile if tile_major else G.run_backward
     scene, cams = make_workload(args.config, crop=args.crop)
     mine = shard_views(len(cams), rank, world)
     g = G.Gaussians.from_numpy(scene, dev)
@@ -246,7 +292,7 @@ def run_ours(args):
         if ev: ev[1].record(stream)
         G.run_forward(cfg, g, cam, buf, stream, ray_lists=False)   # the ordered per-ray lists serve only the atomic baseline
         if ev: ev[2].record(stream)
-        G.run_backward(cfg, g, cam, buf, dls[v], None, stream)
+        run_backward(cfg, g, cam, buf, dls[v], None, stream)
         if ev: ev[3].record(stream)
 
     for s in range(args.warmup):
@@ -292,26 +338,10 @@ def run_ours(args):
     else:
         total_ms_all, hits_all = total_ms, float(hits_total)
 
-    # ---- atomic backward (pixel-centric baseline) on the last view's buffers
+    # ---- the other backward passes, each on the last view's buffers
+    import dataclasses
     last_v = mine[(args.steps - 1) % len(mine)]
     ga = torch.empty_like(buf.grad)
-    at = []
-    if args.atomic_reps > 0:
-        G.run_forward(cfg, g, cams[last_v], buf, stream, ray_lists=True)   # same view again, this time with the lists
-    for i in range(args.atomic_reps + 1 if args.atomic_reps > 0 else 0):   # one untimed run first
-        a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
-        a0.record(stream)
-        G.run_backward_atomic(cfg, g, cams[last_v], buf, dls[last_v], ga, stream)
-        a1.record(stream)
-        torch.cuda.synchronize()
-        if i > 0:
-            at.append(a0.elapsed_time(a1))
-    atomic_ms = float(np.mean(at)) if at else None
-    # ---- the paper's decomposition (block per tile, one vector atomic update per pair) and the ownership ablation (a warp
-    # per pair instead of a thread): the forward again in the tile-major LT layout, same view
-    import dataclasses
-    cfg_t = dataclasses.replace(cfg, lt_layout=G.LT_TILE_MAJOR)
-    warp_ms, tile_ms, tile_fwd_ms = None, None, None
 
     def timed(fn, reps):
         ts_ = []
@@ -325,43 +355,66 @@ def run_ours(args):
                 ts_.append(a0.elapsed_time(a1))
         return float(np.mean(ts_))
 
-    if args.tile_reps > 0 or args.warp_reps > 0:
-        tile_fwd_ms = timed(lambda: G.run_forward(cfg_t, g, cams[last_v], buf, stream, ray_lists=False), max(1, args.tile_reps))
-        if args.tile_reps > 0:
-            tile_ms = timed(lambda: G.run_backward_tile(cfg_t, g, cams[last_v], buf, dls[last_v], ga, stream), args.tile_reps)
-        if args.warp_reps > 0:
-            warp_ms = timed(lambda: G.run_backward_warp(cfg_t, g, cams[last_v], buf, dls[last_v], ga, stream), args.warp_reps)
-    # ---- hybrid backward (colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric), same view
+    # pixel-centric baselines (Sec. 3.5): one atomicAdd per gradient word per hit, and the same sums as 16-byte vector reductions
+    atomic_ms, atomic_vec_ms = None, None
+    if args.atomic_reps > 0:
+        G.run_forward(cfg, g, cams[last_v], buf, stream, ray_lists=True)   # same view again, this time with the lists
+        atomic_ms = timed(lambda: G.run_backward_atomic(cfg, g, cams[last_v], buf, dls[last_v], ga, stream), args.atomic_reps)
+        cfg_v = dataclasses.replace(cfg, atomic_mode=1)
+        atomic_vec_ms = timed(lambda: G.run_backward_atomic(cfg_v, g, cams[last_v], buf, dls[last_v], ga, stream), args.atomic_reps)
+    # the other layout of the intermediate buffer and the backward pass that reads it (primitive-major: a thread walks all
+    # hits of a Gaussian and writes its gradient record once; tile-major: the paper's block per tile with one vector atomic
+    # update per pair), bounds to backward of the same view in buffers of its own (the slot order follows the layout)
+    other_layout = None
+    if args.layout_reps > 0:
+        cfg_a = dataclasses.replace(cfg, lt_layout=G.LT_PRIMITIVE_MAJOR if tile_major else G.LT_TILE_MAJOR)
+        pa, ha = G.size_view(cfg_a, g, cams[last_v], slack=1.0, device=dev)
+        ba = G.ViewBuffers(g.n, g.sh_degree, cams[last_v], cfg_a, pa, ha, dev)
+        other_layout = {"layout": "primitive" if tile_major else "tile",
+                        "bounds_tile_map": timed(lambda: G.run_bounds_tile_map(cfg_a, g, cams[last_v], ba, stream), args.layout_reps),
+                        "forward": timed(lambda: G.run_forward(cfg_a, g, cams[last_v], ba, stream, ray_lists=False), args.layout_reps),
+                        "backward": timed(lambda: G.run_backward(cfg_a, g, cams[last_v], ba, dls[last_v], None, stream), args.layout_reps)}
+        ca = G.gart_read_counts(ba.counts)
+        if ca[G.CNT_ERROR]:
+            raise RuntimeError("capacity exceeded in the other layout: %s" % ca)
+        other_layout["lt_entries"] = int(ca[G.CNT_LT_SLOTS])
+        del ba
+        torch.cuda.empty_cache()
+    # the ownership ablation (a warp per pair instead of a thread), tile-major layout
+    cfg_t = dataclasses.replace(cfg, lt_layout=G.LT_TILE_MAJOR)
+    warp_ms = None
+    if args.warp_reps > 0:
+        G.run_forward(cfg_t, g, cams[last_v], buf, stream, ray_lists=False)
+        warp_ms = timed(lambda: G.run_backward_warp(cfg_t, g, cams[last_v], buf, dls[last_v], ga, stream), args.warp_reps)
+    # hybrid backward (colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric), same view
     hybrid_ms = None
     if args.hybrid_reps > 0:
         cfg_h = dataclasses.replace(cfg, lt_format=1, lt_layout=G.LT_TILE_MAJOR)
         G.run_forward(cfg_h, g, cams[last_v], buf, stream, ray_lists=True)
-        ht = []
-        for i in range(args.hybrid_reps + 1):                    # one untimed run first
-            a0 = torch.cuda.Event(enable_timing=True); a1 = torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            G.run_backward_hybrid(cfg_h, g, cams[last_v], buf, dls[last_v], ga, stream)
-            a1.record(stream)
-            torch.cuda.synchronize()
-            if i > 0:
-                ht.append(a0.elapsed_time(a1))
-        hybrid_ms = float(np.mean(ht))
-    # ---- 8-byte LT entries (four halves per hit): forward and primitive-centric backward of the same view
+        hybrid_ms = timed(lambda: G.run_backward_hybrid(cfg_h, g, cams[last_v], buf, dls[last_v], ga, stream), args.hybrid_reps)
+    # 8-byte LT entries (four halves per hit): forward and block-per-tile backward of the same view
     lt16_ms = None
     if args.lt16_reps > 0:
         cfg_8 = dataclasses.replace(cfg, lt_format=2, lt_layout=G.LT_TILE_MAJOR)
-        ft, bt = [], []
-        for i in range(args.lt16_reps + 1):                      # one untimed run first
-            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-            e0.record(stream)
-            G.run_forward(cfg_8, g, cams[last_v], buf, stream, ray_lists=False)
-            e1.record(stream)
-            G.run_backward_tile(cfg_8, g, cams[last_v], buf, dls[last_v], ga, stream)
-            e2.record(stream)
-            torch.cuda.synchronize()
-            if i > 0:
-                ft.append(e0.elapsed_time(e1)); bt.append(e1.elapsed_time(e2))
-        lt16_ms = {"forward": float(np.mean(ft)), "backward": float(np.mean(bt))}
+        f8 = timed(lambda: G.run_forward(cfg_8, g, cams[last_v], buf, stream, ray_lists=False), args.lt16_reps)
+        b8 = timed(lambda: G.run_backward_tile(cfg_8, g, cams[last_v], buf, dls[last_v], ga, stream), args.lt16_reps)
+        lt16_ms = {"forward": f8, "backward": b8}
+    # the other tile size: the whole step of the same view in buffers of its own
+    other_ts = None
+    if args.other_ts_reps > 0:
+        cfg_o = dataclasses.replace(cfg, tile_size=16 if cfg.tile_size == 8 else 8)
+        po, ho = G.size_view(cfg_o, g, cams[last_v], slack=1.0, device=dev)
+        bo = G.ViewBuffers(g.n, g.sh_degree, cams[last_v], cfg_o, po, ho, dev)
+        other_ts = {"tile_size": cfg_o.tile_size,
+                    "bounds_tile_map": timed(lambda: G.run_bounds_tile_map(cfg_o, g, cams[last_v], bo, stream), args.other_ts_reps),
+                    "forward": timed(lambda: G.run_forward(cfg_o, g, cams[last_v], bo, stream, ray_lists=False), args.other_ts_reps),
+                    "backward": timed(lambda: G.run_backward(cfg_o, g, cams[last_v], bo, dls[last_v], None, stream), args.other_ts_reps)}
+        co = G.gart_read_counts(bo.counts)
+        if co[G.CNT_ERROR]:
+            raise RuntimeError("capacity exceeded at the other tile size: %s" % co)
+        other_ts["pairs"] = int(co[G.CNT_PAIRS])
+        del bo
+        torch.cuda.empty_cache()
     last = cl[-1]
     prim_last_ms = float(stage[-1, 2])
     del ga
@@ -413,18 +466,22 @@ def run_ours(args):
     hbm, hbm_src, sm_max = measured_peaks()
     n_pix = cams[0].width * cams[0].height
     Hm, Pm, Nv = float(np.mean(cl[:, G.CNT_HITS])), float(np.mean(cl[:, G.CNT_PAIRS])), float(np.mean(cl[:, G.CNT_VISIBLE]))
+    Lm = float(np.mean(cl[:, G.CNT_LT_SLOTS]))
     B = algorithmic_bytes_backward(Hm, Pm, Nv, n_pix, K)
     achieved = B / (bwd_ms * 1e-3) / 1e9
     F = fp32_instr_backward(Hm, K)
     alu_peak = 148 * 128 * sm_max * 1e6            # FP32 lane-instructions per second at the maximum SM clock
     roof = {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm, "traffic": None,
-            "peak_source": hbm_src, "kernel": "gart_backward (bwd_zero + bwd_pairs + bwd_convert + bwd_scatter kernels)",
+            "peak_source": hbm_src,
+            "kernel": ("gart_backward, tile-major (bwd_zero + bwd_pairs + bwd_convert + bwd_scatter kernels)" if tile_major else
+                       "gart_backward, primitive-major (bwd_gm item kernel + gm_fill zero rows + gm_zero_big / gm_convert_big for cut Gaussians)"),
             "algorithmic_bytes": B, "ms": bwd_ms,
             "alu": {"fp32_lane_instr": F, "peak_lane_instr_per_s": alu_peak, "frac": F / (bwd_ms * 1e-3) / alu_peak}}
     if cfg.tile_size == 8 and scene.sh_degree == 3:
         # captured on a cropped view of unbounded6m and scaled by the units each kernel's traffic grows with
-        roof["traffic"] = measured_traffic_backward(Hm, Nv, scene.n)
+        roof["traffic"] = measured_traffic_backward(args.lt_layout, Hm, Lm, Nv, scene.n)
         roof["traffic_source"] = "ncu capture of a cropped view, scaled (profiles/dram_traffic_unbounded6m_crop.md)"
+    roof["traffic_units"] = {"hits": Hm, "lt_entries": Lm, "visible": Nv, "gaussians": scene.n, "model": TRAFFIC_MODEL[args.lt_layout]}
 
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
@@ -433,14 +490,15 @@ def run_ours(args):
         H, dt, thr, npx = time_oracle(scene, cam, gs.upstream_gradient(cam, mine[0]), args.oracle_frac)
         cpu = {"value": H / dt, "unit": UNIT, "cores": thr, "kind": "oracle",
                "sample": "random %.1f%% of the 8x8 tiles of view %d (%d rays, %d hits), all Gaussians, %.1f s" % (
-                   100 * args.oracle_frac, mine[0], npx, H, dt)}
+                   100 * args.oracle_frac, mine[0], npx, H, dt),
+               "small_config": oracle_detail()}
 
     line = {
         "metric": METRIC, "value": hits_all / (total_ms_all * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms_all / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.config, "n_gaussians": scene.n, "width": cams[0].width, "height": cams[0].height,
-                   "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "views": len(cams), "crop": args.crop,
+                   "sh_degree": scene.sh_degree, "tile_size": cfg.tile_size, "lt_layout": args.lt_layout, "views": len(cams), "crop": args.crop,
                    "l2": "inputs larger than L2 (parameters %.2f GB, LT %.2f GB per view)" % (
                        4e-9 * scene.n * (11 + 3 * K), 16e-9 * Hm),
                    "hits_per_view": Hm, "pairs_per_view": Pm, "visible_per_view": Nv,
@@ -448,13 +506,15 @@ def run_ours(args):
         "stages_ms": {"bounds_tile_map": float(np.mean(stage[:, 0])), "forward": float(np.mean(stage[:, 1])),
                       "backward": bwd_ms, "backward_median": float(np.median(stage[:, 2]))},
         "backward_hits_per_s": Hm / (bwd_ms * 1e-3),
-        "backward_atomic_ms": atomic_ms,
-        "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,
+        "backward_atomic_ms": atomic_ms, "backward_atomic_vector_ms": atomic_vec_ms,
+        "speedup_vs_atomic": (atomic_ms / prim_last_ms) if atomic_ms else None,                 # scalar atomicAdd per word (Sec. 3.5)
+        "speedup_vs_atomic_vector": (atomic_vec_ms / prim_last_ms) if atomic_vec_ms else None,  # the same sums as 16-byte reductions
         "backward_hybrid_ms": hybrid_ms,
         "lt_8byte_ms": lt16_ms,
         "backward_warp_per_pair_ms": warp_ms,
-        "backward_tile_ms": tile_ms, "forward_tile_major_ms": tile_fwd_ms,
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(-(-cams[0].width // cfg.tile_size), -(-cams[0].height // cfg.tile_size)) * args.steps,
+        "other_layout_ms": other_layout,
+        "other_tile_size_ms": other_ts,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step(cams[0].width, cams[0].height, cfg.tile_size, args.lt_layout) * args.steps,
         "roofline": roof, "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
@@ -470,13 +530,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="unbounded6m", choices=list(gs.CONFIGS))
     ap.add_argument("--tile-size", type=int, default=8, choices=[8, 16])
+    ap.add_argument("--lt-layout", default="tile", choices=["primitive", "tile"],
+                    help="layout of the intermediate buffer and the backward pass that reads it: primitive-major (gart_backward) or tile-major (gart_backward_tile)")
     ap.add_argument("--slack", type=float, default=1.25)
     ap.add_argument("--atomic-reps", type=int, default=2)
     ap.add_argument("--warp-reps", type=int, default=1, help="timed runs of the warp-per-pair backward on the last view (0: skip)")
-    ap.add_argument("--tile-reps", type=int, default=2, help="timed runs of the block-per-tile backward (tile-major LT layout) on the last view (0: skip)")
+    ap.add_argument("--layout-reps", type=int, default=2, help="timed runs of the whole step in the other layout on the last view (0: skip)")
     ap.add_argument("--hybrid-reps", type=int, default=1, help="timed runs of the hybrid backward on the last view (0: skip)")
     ap.add_argument("--lt16-reps", type=int, default=2, help="timed runs of forward + backward with 8-byte LT entries on the last view (0: skip)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--other-ts-reps", type=int, default=2, help="timed runs of the whole step at the other tile size on the last view (0: skip)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--oracle-frac", type=float, default=0.08)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--crop", type=float, default=1.0, help="central crop of every view (profiling on a smaller case)")

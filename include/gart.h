@@ -97,6 +97,10 @@ typedef struct {
                              clamp is active alpha is a constant: the hit's LT entry has zero words 0..2 (no gradient to
                              opacity, mean, scale, rotation) and w = T alpha_max (its colour still gets its gradient).
                              gart_backward_hybrid takes neither option (it re-derives every alpha) */
+    int32_t atomic_mode;  /* gart_backward_atomic only.  GART_ATOMIC_SCALAR (0): one atomicAdd per gradient word per hit, the
+                             form Sec. 3.5 describes; GART_ATOMIC_VECTOR (1): the same sums as 16-byte vector reductions,
+                             ceil((11 + 3K) / 4) per hit (15 at degree 3), the strongest plain form of the scatter on
+                             this hardware */
     int32_t wait_polls;   /* 0: the library's limit (2^22 polls) on every wait of a kernel for one of its own asynchronous
                              copies; > 0: that many polls; < 0: no poll at all, so every such wait gives up at once (a test
                              hook for the path below).  A wait that gives up sets GART_ERRBIT_TIMEOUT in
@@ -137,6 +141,9 @@ enum {
     GART_CNT_LT_SLOTS = 8,  /* L >= H: entries of LT in use, including the padding of its interleaved layout */
     GART_COUNTS_WORDS = 12
 };
+#define GART_ATOMIC_SCALAR 0
+#define GART_ATOMIC_VECTOR 1
+
 #define GART_ERRBIT_PAIRS 1u
 #define GART_ERRBIT_HITS 2u
 #define GART_ERRBIT_TIMEOUT 4u   /* a bounded wait on an asynchronous copy gave up (never expected) */
@@ -342,8 +349,8 @@ gart_status gart_backward_tile(const gart_config *cfg, const gart_gaussians *g, 
 
 /*
  * Pixel-centric baseline (Sec. 3.5): one thread per ray walks the ray's hits and issues one
- * atomicAdd per gradient word per hit (11 + 3K; 59 at degree 3).  Same result as gart_backward
- * up to summation order.  Reads 16-byte LT entries through ray_slot, so either layout serves; needs the
+ * atomicAdd per gradient word per hit (11 + 3K; 59 at degree 3), or, with cfg->atomic_mode = GART_ATOMIC_VECTOR,
+ * one 16-byte vector reduction per four words.  Same result as gart_backward up to summation order.  Reads 16-byte LT entries through ray_slot, so either layout serves; needs the
  * per-ray lists of gart_forward (INVALID_ARG if they are NULL).
  */
 gart_status gart_backward_atomic(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam,

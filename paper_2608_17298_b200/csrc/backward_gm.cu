@@ -451,8 +451,11 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     (void)tile_off;
     if (!cfg || !g || !cam || !counts || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;                          // this pass reads 16-byte LT entries (they name their pixel)
-    if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR) return GART_ERR_INVALID_ARG;    // ... in the primitive-major layout
+    if (cfg->lt_layout == GART_LT_TILE_MAJOR)    // the other layout: the block-per-tile pass reads it
+        return gart_backward_tile(cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, view_bytes, cap_pairs, lt, dL_dcolor, grad, counts,
+                                  workspace, workspace_bytes, stream);
+    if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;                          // the item pass reads 16-byte LT entries (they name their pixel)
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;

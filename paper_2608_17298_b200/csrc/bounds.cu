@@ -140,7 +140,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
             q5 = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
             q6 = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
         }
-        keys[i] = vis ? (uint32_t)((y0 / GM_SUP) * sup_x + x0 / GM_SUP) : key_none;   // super-tile of the rectangle's corner
+        // super-tile of the rectangle's corner (its row alone where the caller sorts by rows: sup_x = 1)
+        keys[i] = vis ? (uint32_t)((y0 / GM_SUP) * sup_x + (sup_x > 1 ? x0 / GM_SUP : 0)) : key_none;
         vals[i] = (uint32_t)i;
     }
     {
@@ -306,8 +307,12 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     c.width = cam->width; c.height = cam->height;
     c.fx = cam->fx; c.fy = cam->fy; c.cx = cam->cx; c.cy = cam->cy;
     for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
-    const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
-    const uint32_t key_none = (uint32_t)gm_super_tiles(cam->width, cam->height);   // sorts after every super-tile
+    // Slots are numbered in the order of the super-tile (16 x 16 pixels) of the rectangle's corner: neighbours in the image
+    // are neighbours in every per-slot array.  The primitive-major layout wants the full order (its work items of a
+    // super-tile are then consecutive slots); for the tile-major layout the row alone gives the locality and needs one
+    // radix pass less.
+    const int sup_x = cfg->lt_layout == GART_LT_PRIMITIVE_MAJOR ? (cam->width + GM_SUP - 1) / GM_SUP : 1;
+    const uint32_t key_none = (uint32_t)(sup_x * ((cam->height + GM_SUP - 1) / GM_SUP));   // sorts after every visible Gaussian
     int bits = 1;
     while ((1u << bits) <= key_none) ++bits;
     uint32_t* const kbuf[2] = {w.keys0, w.keys1};

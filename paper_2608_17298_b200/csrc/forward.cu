@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
     float4 ra[5];
     // the pair's place in the primitive-major order: first pair of its Gaussian + its tile's index in the rectangle's tiles
     auto gpos_of = [&](uint32_t sid, bool act) {
-        if (!act) return 0u;
+        if (!act || !gm_mask) return 0u;   // (gm_mask is NULL in the tile-major layout)
         const int4 r = __ldg(srect + sid);
         const int gx0 = r.x / TS, gy0 = r.y / TS;
         return __ldg(gpair_off + sid) + (uint32_t)((ty - gy0) * (r.z / TS - gx0 + 1) + (tx - gx0));
@@ -193,9 +193,11 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
             }
 #pragma unroll
             for (int q = 0; q < MW; ++q) pair_mask[(size_t)j * MW + q] = w[q];
+            if (gm_mask) {
 #pragma unroll
-            for (int q = 0; q < MW; ++q) gm_mask[(size_t)gpa * MW + q] = w[q];
-            pair_gpos[j] = gpa;
+                for (int q = 0; q < MW; ++q) gm_mask[(size_t)gpa * MW + q] = w[q];
+                pair_gpos[j] = gpa;
+            }
         }
         // hits per pixel: one shared-memory increment per hit
 #pragma unroll
@@ -302,7 +304,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
 #pragma unroll
             for (int m = 0; m < MW; ++m) wv[u][m] = act ? __ldg(pair_mask + (size_t)j[u] * MW + m) : 0u;
             sid[u] = act ? __ldg(pair_sid + j[u]) : 0u;
-            gp[u] = act ? __ldg(pair_gpos + j[u]) : 0u;
+            gp[u] = (act && rank_gpos) ? __ldg(pair_gpos + j[u]) : 0u;   // (rank_gpos is NULL in the tile-major layout)
         }
 #pragma unroll
         for (int u = 0; u < TSU; ++u) {
@@ -314,7 +316,7 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) tile_sort_kernel(const uint32
 #pragma unroll
                 for (int m = 0; m < MW; ++m) rank_mask[q * MW + m] = wv[u][m];
                 rank_sid[q] = sid[u];
-                rank_gpos[q] = gp[u];
+                if (rank_gpos) rank_gpos[q] = gp[u];
                 rank_gstart[q] = run;
             }
             const uint32_t cmax = __shfl_sync(0xffffffffu, c, 0);
@@ -615,7 +617,7 @@ __device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32
 
 // The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
 // slot as one float4, alpha apart; after the sort the three passes gather from there by sorted index.
-template <int R>
+template <int R, bool GM, bool OPT>   // GM: entries carry their pixel's window index; OPT: early termination or alpha clamp may be on
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx, int pixlow,
                                                float t_min, float alpha_max, float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
@@ -704,7 +706,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
     float T0 = __shfl_up_sync(0xffffffffu, inc, 1);
     if (lane == 0) T0 = 1.0f;
     float Tfin = __shfl_sync(0xffffffffu, inc, 31);
-    if (t_min > 0.0f) {
+    if (OPT && t_min > 0.0f) {
         // early termination: the ray ends before the first hit whose transmittance in front is below t_min.  That hit and
         // the later ones get alpha = 0 (they keep their place and their LT slot), T_final is the transmittance reached.
         int first = 0x7fffffff;
@@ -763,8 +765,8 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 const float wgt = Ts[r] * al[r];
                 const float cx = strip_low_bit(cs.x), cy = strip_low_bit(cs.y);
                 float4 en = lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2);
-                if (al[r] >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }   // a clamped alpha is a constant: no gradient through it
-                lt_store(lt, lt_fmt, slot, en, pix_of(pixlow, cs.x, cs.y, i < n_comp));
+                if (OPT && al[r] >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }   // a clamped alpha is a constant: no gradient through it
+                lt_store(lt, lt_fmt, slot, en, GM ? pix_of(pixlow, cs.x, cs.y, i < n_comp) : -1);
                 if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cx, k0); k1 = fmaf(wgt, cy, k1); k2 = fmaf(wgt, cs.z, k2);
             }
@@ -806,6 +808,7 @@ __device__ __forceinline__ void warp_sort(uint64_t* a, int n, int lane) {
     }
 }
 
+template <bool GM, bool OPT>
 __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint64_t* __restrict__ kp, int n, int n_comp, int lane, size_t b, int64_t r, int pixlow,
                                             float t_min, float alpha_max, float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                             float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot) {
@@ -848,7 +851,7 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         const float T = carryT * excl;
         if (valid) kp[i] = ((uint64_t)__float_as_uint(T) << 32) | (uint64_t)c;
         carryT *= __shfl_sync(0xffffffffu, prod, 31);
-        if (t_min > 0.0f && pstar == 0x7fffffff) {
+        if (OPT && t_min > 0.0f && pstar == 0x7fffffff) {
             const unsigned below = __ballot_sync(0xffffffffu, i < n_comp && T < t_min);
             if (below) {
                 const int l0 = __ffs((int)below) - 1;
@@ -888,8 +891,8 @@ __device__ __noinline__ void sweep_ray_long(const float4* __restrict__ rec, uint
         if (valid) {
             const uint32_t slot = __float_as_uint(ra.z);
             float4 en = lt_entry(wgt, ra.w, strip_low_bit(rb.x), strip_low_bit(rb.y), rb.z, k0 + e0, k1 + e1, k2 + e2);
-            if (ra.w >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }
-            lt_store(lt, lt_fmt, slot, en, pix_of(pixlow, rb.x, rb.y, i < n_comp));
+            if (OPT && ra.w >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }
+            lt_store(lt, lt_fmt, slot, en, GM ? pix_of(pixlow, rb.x, rb.y, i < n_comp) : -1);
             if (ray_gid) { ray_gid[b + i] = __float_as_uint(ra.y); ray_slot[b + i] = slot; }
         }
         k0 += __shfl_sync(0xffffffffu, s0, 31);
@@ -915,10 +918,12 @@ struct SweepClass {
     static constexpr int SMEM = SWEEP_WARPS * CAP * 28;
 };
 
-template <int CLS, int FMT>   // FMT: the LT format (a compile-time constant keeps the store of the usual format free of tests)
+// FMT: the LT format; GM: primitive-major layout with 16-byte entries (they carry their pixel's window index); OPT: early
+// termination or the alpha clamp may be on.  Compile-time constants keep the usual case free of their tests and registers.
+template <int CLS, int FMT, bool GM, bool OPT>
 __global__ void __launch_bounds__(SWEEP_WARPS * 32, SweepClass<CLS>::MIN_BLOCKS)
 fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __restrict__ recs, uint64_t* __restrict__ long_keys, int64_t n_rays,
-                      int width, int tile_size, int tiles_x, int embed_pix,
+                      int width, int tile_size, int tiles_x,
                       float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                       float4* __restrict__ lt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                       int max_comp, float t_min, float alpha_max, const uint32_t* __restrict__ counts) {
@@ -950,13 +955,13 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     }
     if (n <= SweepClass<CLS>::LO || (CLS < 2 && n > CAP)) return;
     const int n_comp = min(n, max_comp);   // hits that are composited (all of them unless the caller set a cap)
-    const int pixlow = embed_pix ? (int)((r / width) % GM_SUP) * GM_WIN + (int)((r % width) % GM_SUP) : -1;
+    const int pixlow = GM ? (int)((r / width) % GM_SUP) * GM_WIN + (int)((r % width) % GM_SUP) : -1;
     const float4* rec = recs + b * 2;
     extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
     uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
     float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R>(rec, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
+#define GART_SWEEP(R) sweep_ray_regs<R, GM, OPT>(rec, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
@@ -964,7 +969,7 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
         else GART_SWEEP(8);
     } else {
         if (n <= SORT_CAP) GART_SWEEP(16);
-        else sweep_ray_long(rec, long_keys + b, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
+        else sweep_ray_long<GM, OPT>(rec, long_keys + b, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot);
     }
 #undef GART_SWEEP
 }
@@ -1120,21 +1125,22 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (cudaMemsetAsync(v.st_off, 0, (size_t)(v.ns + 1) * 4, st) != cudaSuccess) return GART_ERR_CUDA;
     // (a visible Gaussian has at least one pair: without a capacity error the slots in use number at most cap_pairs)
     const int64_t nscan = g->n < cap_pairs ? g->n : cap_pairs;
-    if (nscan > 0) {
+    if (gmaj && nscan > 0) {
         SlotTilesF tf{srect, counts, ts};
         s = exclusive_scan(tf, nscan, v.gpair_off, w.total_gm, w.scan_ws, st);
         if (s != GART_OK) return s;
     }
 
-    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, v.gm_mask, v.pair_gpos, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, v.gm_mask, v.pair_gpos, hit_count, counts);
+    uint32_t* const gm_mask = gmaj ? v.gm_mask : nullptr;
+    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
     // (in the primitive-major layout the evaluation looks the LT slot up by the pair's primitive-major position: the
     // rank-ordered copy of those positions takes the place of the tile layout's group starts)
-    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, v.rank_gpos, w.tile_slots, counts);
-    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, v.rank_gpos, w.tile_slots, counts);
+    if (ts == 8) tile_sort_kernel<8><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, gmaj ? v.rank_gpos : nullptr, w.tile_slots, counts);
+    else tile_sort_kernel<16><<<sblocks, SORT_WARPS * 32, 0, st>>>(tile_off, w.pair_sid, v.pair_mask, v.pair_gpos, T, v.pair_order, v.rank_sid, v.rank_mask, v.rank_gstart, gmaj ? v.rank_gpos : nullptr, w.tile_slots, counts);
     GART_LAUNCH_CHECK();
 
     TileSlotsF tsf{w.tile_slots};
@@ -1200,18 +1206,24 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const int lt_fmt = cfg->lt_format;
     const int max_comp = cfg->max_hits > 0 ? cfg->max_hits : 0x7fffffff;
     const float* bg = cfg->background;
-#define GART_SWEEP_LAUNCH(C, F)                                                                                                                 \
-    {                                                                                                                                           \
-        if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
-            return GART_ERR_CUDA;                                                                                                               \
-        fwd_sort_sweep_kernel<C, F><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, (gmaj && lt_fmt == 0) ? 1 : 0, bg[0], \
-                                                                                                    bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, cfg->t_min, amax, counts); \
-        GART_LAUNCH_CHECK();                                                                                                                    \
+#define GART_SWEEP_LAUNCH(C, F, GM, OPT)                                                                                                                 \
+    {                                                                                                                                                    \
+        if (cudaFuncSetAttribute(fwd_sort_sweep_kernel<C, F, GM, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SweepClass<C>::SMEM) != cudaSuccess) \
+            return GART_ERR_CUDA;                                                                                                                        \
+        fwd_sort_sweep_kernel<C, F, GM, OPT><<<(unsigned)blocks, SWEEP_WARPS * 32, SweepClass<C>::SMEM, st>>>(ray_off, w.recs, w.long_keys, n_rays, cam->width, ts, cf.tiles_x, bg[0],   \
+                                                                                                             bg[1], bg[2], color, t_final, lt4, ray_gid, ray_slot, max_comp, cfg->t_min, amax, counts); \
+        GART_LAUNCH_CHECK();                                                                                                                             \
     }
-#define GART_SWEEP_BOTH(F) GART_SWEEP_LAUNCH(2, F) GART_SWEEP_LAUNCH(1, F)   // the longest rays first
-    if (lt_fmt == 0) { GART_SWEEP_BOTH(0) }
-    else if (lt_fmt == 1) { GART_SWEEP_BOTH(1) }
-    else { GART_SWEEP_BOTH(2) }
+#define GART_SWEEP_BOTH(F, GM, OPT) GART_SWEEP_LAUNCH(2, F, GM, OPT) GART_SWEEP_LAUNCH(1, F, GM, OPT)   // the longest rays first
+    const bool opt = cfg->t_min > 0.0f || cfg->alpha_max < 1.0f;
+    if (lt_fmt == 0) {
+        if (gmaj) { if (opt) { GART_SWEEP_BOTH(0, true, true) } else { GART_SWEEP_BOTH(0, true, false) } }
+        else { if (opt) { GART_SWEEP_BOTH(0, false, true) } else { GART_SWEEP_BOTH(0, false, false) } }
+    } else if (lt_fmt == 1) {
+        GART_SWEEP_BOTH(1, false, false)     // (the hybrid pass takes neither option)
+    } else {
+        if (opt) { GART_SWEEP_BOTH(2, false, true) } else { GART_SWEEP_BOTH(2, false, false) }
+    }
 #undef GART_SWEEP_BOTH
 #undef GART_SWEEP_LAUNCH
     GART_LAUNCH_CHECK();

@@ -49,7 +49,7 @@ class GartError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
                 ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32), ("t_min", C.c_float),
-                ("alpha_max", C.c_float), ("wait_polls", C.c_int32)]
+                ("alpha_max", C.c_float), ("atomic_mode", C.c_int32), ("wait_polls", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -123,9 +123,10 @@ class Config:
     tile_size: int = 8
     lt_format: int = 0          # 0: 16-byte LT entries (gart_backward); 1: 4 bytes per hit (gart_backward_hybrid); 2: 8 bytes (gart_backward)
     max_hits: int = 0           # > 0: only the first max_hits hits of a ray are composited (0: all, the paper's setting)
-    lt_layout: int = 0          # 0: primitive-major LT (gart_backward); 1: tile-major (gart_backward_tile, _warp, _hybrid)
+    lt_layout: int = LT_TILE_MAJOR   # LT_TILE_MAJOR (1, the faster whole step: block-per-tile backward) or LT_PRIMITIVE_MAJOR (0: item backward, half the DRAM traffic)
     t_min: float = 0.0          # > 0: a ray ends before the first hit with less than t_min transmittance in front (0: off)
     alpha_max: float = 1.0      # < 1: every hit's alpha is clamped to alpha_max (>= 1: off)
+    atomic_mode: int = 0        # gart_backward_atomic: 0 scalar atomicAdd per word, 1 one 16-byte vector reduction per four words
     wait_polls: int = 0         # 0: library limit on a kernel's waits for its own copies; > 0: polls; < 0: every wait gives up (test hook)
 
     def c(self) -> _Config:
@@ -135,7 +136,7 @@ class Config:
         s.max_hits = int(self.max_hits)
         s.lt_layout = int(self.lt_layout)
         s.t_min, s.alpha_max = float(self.t_min), float(self.alpha_max)
-        s.wait_polls = int(self.wait_polls)
+        s.wait_polls, s.atomic_mode = int(self.wait_polls), int(self.atomic_mode)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s

@@ -76,6 +76,7 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
     same buffers, then the forward again in the tile-major layout for the block-per-tile pass, the warp-per-pair pass
     and the hybrid pass, and the forward with 8-byte entries for gart_backward on them."""
     import dataclasses
+    cfg = dataclasses.replace(cfg, lt_layout=G.LT_PRIMITIVE_MAJOR)
     g = G.Gaussians.from_numpy(scene)
     if cap_pairs is None or cap_hits is None:
         P, S = G.size_view(cfg, g, cam, slack=1.0)
@@ -114,6 +115,10 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         G.run_backward_atomic(cfg, g, cam, buf, dl, ga)
         torch.cuda.synchronize()
         out["grad_atomic"] = to_np(ga)[:g.n]
+        gv = torch.full_like(buf.grad, float("nan"))
+        G.run_backward_atomic(dataclasses.replace(cfg, atomic_mode=1), g, cam, buf, dl, gv)     # the same sums as vector reductions
+        torch.cuda.synchronize()
+        out["grad_atomic_vec"] = to_np(gv)[:g.n]
         # ---- tile-major layout: block-per-tile pass and warp-per-pair pass (same buffers, the forward again)
         cfg_t = dataclasses.replace(cfg, lt_layout=G.LT_TILE_MAJOR)
         G.run_forward(cfg_t, g, cam, buf)

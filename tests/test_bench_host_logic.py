@@ -22,14 +22,23 @@ def test_shard_views_partition():
 
 
 def test_launch_count_and_bytes():
-    assert bench.launches_per_step(155, 103) == 7 + (7 + 2 * 5) + 12 + 4     # 7 row bits -> 1 pass, 14 tile bits -> 2 passes
-    assert bench.launches_per_step(8, 8) == 7 + (7 + 5) + 12 + 4
+    # 155 x 103 tiles of 8 pixels (14 key bits: two radix passes of five kernels), 78 x 52 super-tiles (12 bits: two passes)
+    assert bench.launches_per_step(1240, 824, 8, "primitive") == (1 + 10 + 1) + (7 + 10) + (8 + (5 + 10) + 12 + 7) + 4
+    # 8 x 8 tiles, 4 x 4 super-tiles: one pass each
+    assert bench.launches_per_step(64, 64, 8, "primitive") == (1 + 5 + 1) + (7 + 5) + (8 + (5 + 5) + 12 + 7) + 4
+    # tile-major layout: the slot sort has 52 super-tile rows (one pass), the forward no item lists
+    assert bench.launches_per_step(1240, 824, 8, "tile") == (1 + 5 + 1) + (7 + 10) + 12 + 4
+    assert bench.launches_per_step(1240, 824, 8) == bench.launches_per_step(1240, 824, 8, "tile")
     B = bench.algorithmic_bytes_backward(H=100, P=10, n_vis=5, n_pixels=64, K=16)
     assert B == 1600 + 40 + 4 * 61 * 5 + 4 * 59 * 5 + 28 * 64
     # the traffic model adds its per-unit figures
     t = bench.TRAFFIC_MODEL
-    assert bench.measured_traffic_backward(0, 0, 10) == 10 * t["scatter_write_per_gaussian"]
-    assert bench.measured_traffic_backward(7, 0, 0) == 7 * t["pairs_per_hit"]
+    tp = t["primitive"]
+    assert bench.measured_traffic_backward("primitive", 0, 0, 0, 10) == 10 * (tp["fill_write_per_invisible"] + tp["fill_read_per_gaussian"])
+    assert bench.measured_traffic_backward("primitive", 5, 7, 0, 0) == 7 * tp["items_read_per_lt_entry"]
+    assert bench.measured_traffic_backward("primitive", 0, 0, 10, 10) == 10 * (tp["items_write_per_visible"] + tp["big_per_visible"] + tp["fill_read_per_gaussian"])
+    assert bench.measured_traffic_backward("tile", 0, 0, 0, 10) == 10 * t["tile"]["scatter_write_per_gaussian"]
+    assert bench.measured_traffic_backward("tile", 7, 9, 0, 0) == 7 * t["tile"]["pairs_per_hit"]
 
 
 def _worker(rank, world, port, out):

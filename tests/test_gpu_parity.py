@@ -72,7 +72,7 @@ def assert_grad_lt16(gpu_grad, ref, K, rows=None):
     return float(((d <= 3e-3 * np.maximum(np.abs(r), COND * a)) | (d <= 1e-6)).mean())
 
 
-VARIANTS = ("grad", "grad_tile", "grad_atomic", "grad_hybrid", "grad_warp")   # every backward pass on 16-byte (4-byte: hybrid) entries
+VARIANTS = ("grad", "grad_tile", "grad_atomic", "grad_atomic_vec", "grad_hybrid", "grad_warp")   # every backward pass on 16-byte (4-byte: hybrid) entries
 
 
 OPTION_BAND = 1e-3    # rays with a termination or clamp decision closer than this (in ln) to its threshold carry no upstream gradient
@@ -410,14 +410,14 @@ def test_shell200k_sampled(view):
 
 def test_unbounded1m_sampled():
     scene, cams = gs.config_unbounded_1m()
-    sampled_parity(scene, cams[0], G.Config(tile_size=8), 0)
-    sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=100, n_tiles=20)
+    sampled_parity(scene, cams[0], G.Config(tile_size=8), 0, n_gauss=200, n_tiles=40, n_large=14)
+    sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=60, n_tiles=12, n_large=6)
 
 
 def test_unbounded6m_sampled():
     """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles)."""
     scene, cams = gs.config_unbounded_6m()
-    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=150, n_tiles=30, n_large=6, large_max_area=15000)
+    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=110, n_tiles=22, n_large=5, large_max_area=15000)
     assert gpu["counts"][G.CNT_HITS] > 1e8
 
 
@@ -467,7 +467,7 @@ def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(variant)
     the oracle's gradients.  Nothing faults and nothing hangs: the waits that give up are the kernel's own bounded ones."""
     scene, cams = gs.config_tiny()
     cam = cams[0]
-    cfg = {"primitive": G.Config(), "tile": G.Config(lt_layout=G.LT_TILE_MAJOR),
+    cfg = {"primitive": G.Config(lt_layout=G.LT_PRIMITIVE_MAJOR), "tile": G.Config(lt_layout=G.LT_TILE_MAJOR),
            "hybrid": G.Config(lt_layout=G.LT_TILE_MAJOR, lt_format=1)}[variant]
     fn = {"primitive": G.run_backward, "tile": G.run_backward_tile, "hybrid": G.run_backward_hybrid}[variant]
     g = G.Gaussians.from_numpy(scene)
@@ -518,18 +518,18 @@ def test_invalid_arguments_return_status():
     assert e.value.status == 1                     # workspace not 256-byte aligned
     # each backward variant wants its own LT format, and the forward knows three
     dl = torch.zeros((cam.height, cam.width, 3), dtype=torch.float32, device="cuda")
-    TM = G.LT_TILE_MAJOR
+    TM, PM = G.LT_TILE_MAJOR, G.LT_PRIMITIVE_MAJOR
     refused = [
-        (G.run_backward, G.Config(lt_format=1)),                      # gart_backward reads 16-byte entries ...
-        (G.run_backward, G.Config(lt_format=2)),
-        (G.run_backward, G.Config(lt_layout=TM)),                     # ... in the primitive-major layout
-        (G.run_backward_tile, G.Config()),                            # the tile-major passes want the tile-major layout
+        (G.run_backward, G.Config(lt_format=1, lt_layout=PM)),        # the item pass reads 16-byte entries ...
+        (G.run_backward, G.Config(lt_format=2, lt_layout=PM)),
+        (G.run_backward, G.Config(lt_format=1, lt_layout=TM)),        # ... the block-per-tile pass 16- or 8-byte entries
+        (G.run_backward_tile, G.Config(lt_layout=PM)),                # the tile-major passes want the tile-major layout
         (G.run_backward_tile, G.Config(lt_format=1, lt_layout=TM)),
-        (G.run_backward_warp, G.Config()),
+        (G.run_backward_warp, G.Config(lt_layout=PM)),
         (G.run_backward_warp, G.Config(lt_format=1, lt_layout=TM)),
         (G.run_backward_warp, G.Config(lt_format=2, lt_layout=TM)),
         (G.run_backward_hybrid, G.Config(lt_format=2, lt_layout=TM)),
-        (G.run_backward_hybrid, G.Config(lt_format=1)),
+        (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=PM)),
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, max_hits=4)),
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, t_min=0.01)),
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, alpha_max=0.99)),
@@ -539,8 +539,9 @@ def test_invalid_arguments_return_status():
         with pytest.raises(G.GartError) as e:
             fn(cfg_bad, g, cam, buf, dl)
         assert e.value.status == 1, (fn.__name__, cfg_bad)
-    for cfg_bad in (G.Config(max_hits=-1), G.Config(lt_format=3), G.Config(lt_layout=2), G.Config(lt_format=1), G.Config(lt_format=2),
-                    G.Config(t_min=1.0), G.Config(t_min=-0.1), G.Config(alpha_max=0.0)):
+    for cfg_bad in (G.Config(max_hits=-1), G.Config(lt_format=3), G.Config(lt_layout=2), G.Config(lt_format=1, lt_layout=G.LT_PRIMITIVE_MAJOR),
+                    G.Config(lt_format=2, lt_layout=G.LT_PRIMITIVE_MAJOR),
+                    G.Config(t_min=1.0), G.Config(t_min=-0.1), G.Config(alpha_max=0.0)):   # (refused by gart_forward)
         with pytest.raises(G.GartError) as e:
             G.run_forward(cfg_bad, g, cam, buf)
         assert e.value.status == 1, cfg_bad
