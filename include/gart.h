@@ -212,7 +212,10 @@ gart_status gart_tile_map(const gart_config *cfg, const int32_t *rect, int64_t n
  *     GART_TILE_MAP_STATIC_BYTES (about n + 3 cap_pairs words: e.g. n = 200k with cap_pairs = 500k);
  *     larger problems are refused with GART_ERR_WORKSPACE_TOO_SMALL before any work is queued.
  *   - The first call on a device looks up the array's device address (a host-side query, done with
- *     that device current); make that first call before any stream capture begins.
+ *     that device current) and keeps it for the life of the process; make that first call before any
+ *     stream capture begins.  Host threads may make it together.  `stream` must belong to the device
+ *     that is current in the calling thread (the array used is the current device's).  cudaDeviceReset
+ *     invalidates the kept address: do not call this entry point after a reset of its device.
  *   - All calls on a device share the array: calls that may overlap on the GPU (different streams
  *     without ordering) race on it.  The array keeps the previous call's contents; the tile map
  *     writes every scratch word before reading it, so nothing has to be cleared.

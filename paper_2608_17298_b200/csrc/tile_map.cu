@@ -5,6 +5,8 @@
 // caller's capacity and read the actual count.
 #include "radix.cuh"
 
+#include <atomic>
+
 namespace gart {
 
 struct TileCountF {
@@ -195,22 +197,24 @@ static __device__ __align__(256) unsigned char g_tile_map_scratch[GART_TILE_MAP_
 // In host code the array's name is only a stand-in for the symbol, not a device address: the
 // address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device
 // current.
-static void* g_tile_map_scratch_ptr[64] = {nullptr};
+// Threads that make a device's first call together may all run the query; they store the same value, atomically.
+static std::atomic<void*> g_tile_map_scratch_ptr[64];
 
 extern "C" gart_status gart_tile_map_static(const gart_config* cfg, const int32_t* rect, int64_t n, int32_t width, int32_t height,
                                             uint32_t* tile_off, uint32_t* pair_gid, int64_t cap_pairs, uint32_t* counts,
                                             void* stream) {
+    // the argument checks of gart_tile_map that the size test below relies on, then the size test: a problem beyond the
+    // fixed array is refused before anything is launched
+    if (!cfg || (cfg->tile_size != 8 && cfg->tile_size != 16)) return GART_ERR_INVALID_ARG;
     if (n < 0 || cap_pairs < 0 || width <= 0 || height <= 0) return GART_ERR_INVALID_ARG;
-    // sizes beyond the fixed array are refused before anything is launched
-    if (gart_tile_map_workspace_bytes(n, width, height, cfg ? cfg->tile_size : 8, cap_pairs) > (size_t)GART_TILE_MAP_STATIC_BYTES)
+    if (gart_tile_map_workspace_bytes(n, width, height, cfg->tile_size, cap_pairs) > (size_t)GART_TILE_MAP_STATIC_BYTES)
         return GART_ERR_WORKSPACE_TOO_SMALL;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GART_ERR_CUDA;
-    if (!g_tile_map_scratch_ptr[dev]) {
-        void* p = nullptr;
+    void* p = g_tile_map_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress(&p, g_tile_map_scratch) != cudaSuccess || !p) return GART_ERR_CUDA;
-        g_tile_map_scratch_ptr[dev] = p;
+        g_tile_map_scratch_ptr[dev].store(p, std::memory_order_release);
     }
-    return gart_tile_map(cfg, rect, n, width, height, tile_off, pair_gid, cap_pairs, counts, g_tile_map_scratch_ptr[dev],
-                         (size_t)GART_TILE_MAP_STATIC_BYTES, stream);
+    return gart_tile_map(cfg, rect, n, width, height, tile_off, pair_gid, cap_pairs, counts, p, (size_t)GART_TILE_MAP_STATIC_BYTES, stream);
 }

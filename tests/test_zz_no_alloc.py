@@ -4,8 +4,10 @@ It serves callers that cannot allocate device memory when they call (a host that
 device budget to its own arena, a plug-in under a quota, a loop that must not touch the allocator).
 The test calls it through the C ABI twice in a row -- the second call finds the first call's
 leftovers in the shared array -- and requires exactly the outputs of gart_tile_map, which are
-integers: tile offsets, pair lists and the counts block must be identical.  It also checks that a
-problem too large for the fixed array is refused with a clear status.
+integers: tile offsets, pair lists and the counts block must be identical; the same outputs are
+compared with the oracle's tile map, and the device's free memory must be the same before and
+after the second call (nothing was allocated).  It also checks that a problem too large for the
+fixed array is refused with a clear status.
 """
 import numpy as np
 import pytest
@@ -13,6 +15,7 @@ import torch
 
 import gart_scenes as gs
 import paper_2608_17298_b200.gart as G
+from oracle import gart_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -32,6 +35,19 @@ def _tile_maps(scene, cam, cfg):
     G.gart_tile_map_static(cfg, buf.rect, g.n, cam, tile_off, pair_gid, P, buf.counts)
     torch.cuda.synchronize()
     got = (tile_off.cpu().numpy(), pair_gid.cpu().numpy()[:P - 1], G.gart_read_counts(buf.counts))
+    # once more into the same arrays: the address of the fixed array is known by now, so the call must not touch the allocator
+    free0 = torch.cuda.mem_get_info()[0]
+    G.gart_tile_map_static(cfg, buf.rect, g.n, cam, tile_off, pair_gid, P, buf.counts)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert np.array_equal(tile_off.cpu().numpy(), got[0]) and np.array_equal(pair_gid.cpu().numpy()[:P - 1], got[1])
+    # and the oracle's tile map of the oracle's own rectangles (identical unless a rectangle edge lies within 1e-9 of a pixel centre)
+    osc = orc.OracleScene.from_scene(scene)
+    rect, cls, margin = orc.bounds(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    if (margin > 1e-9).all():
+        o_off, o_gid, _ = orc.tile_map(rect, cam.width, cam.height, cfg.tile_size)
+        assert np.array_equal(got[0].astype(np.int64), np.asarray(o_off, dtype=np.int64))
+        assert np.array_equal(got[1].astype(np.int64), np.asarray(o_gid, dtype=np.int64)[:P - 1])
     return ref, got
 
 
