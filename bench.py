@@ -436,8 +436,19 @@ def run_ours(args):
         # free the resident buffers first: the arena holds its own copy of everything
         del buf
         torch.cuda.empty_cache()
-        arena = torch.empty(G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam0.width, cam0.height, cfg.tile_size,
-                                                         cap_pairs, cap_hits), dtype=torch.uint8, device=dev)
+        arena_bytes = G.gart_view_host_arena_bytes(scene.n, scene.sh_degree, cam0.width, cam0.height, cfg.tile_size, cap_pairs, cap_hits)
+        h2d = 4 * scene.n * (3 + 3 + 4 + 1 + 3 * K) + 12 * cam0.width * cam0.height
+        d2h = 4 * scene.n * G.GRAD_WORDS + 12 * cam0.width * cam0.height + 4 * G.COUNTS_WORDS
+
+        def reduce_e2e(hits, secs):
+            if world > 1:
+                tt = torch.tensor([secs], dtype=torch.float64, device=dev); dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+                hh = torch.tensor([hits], dtype=torch.float64, device=dev); dist.all_reduce(hh, op=dist.ReduceOp.SUM)
+                return float(hh.item()) / float(tt.item())
+            return hits / secs
+
+        # (a) one view at a time: gart_view_host returns when the view's results are on the host
+        arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
         e_hits, e_t = 0, 0.0
         for s in range(args.e2e_steps + 1):
             v = mine[s % len(mine)]
@@ -447,15 +458,50 @@ def run_ours(args):
             dt = time.perf_counter() - t0
             if s > 0:
                 e_hits += c[G.CNT_HITS]; e_t += dt
-        e_val = e_hits / e_t
-        if world > 1:
-            tt = torch.tensor([e_t], dtype=torch.float64, device=dev); dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            hh = torch.tensor([e_hits], dtype=torch.float64, device=dev); dist.all_reduce(hh, op=dist.ReduceOp.SUM)
-            e_val = float(hh.item()) / float(tt.item())
-        h2d = 4 * scene.n * (3 + 3 + 4 + 1 + 3 * K) + 12 * cam0.width * cam0.height
-        d2h = 4 * scene.n * G.GRAD_WORDS + 12 * cam0.width * cam0.height + 4 * G.COUNTS_WORDS
-        e2e = {"value": e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": 1e3 * e_t / args.e2e_steps, "steps": args.e2e_steps}
+        serial = {"value": reduce_e2e(e_hits, e_t), "ms_per_step": 1e3 * e_t / args.e2e_steps}
+        # (b) several views in flight (gart_view_host_async on one stream each, with an arena and host arrays of its own): one
+        # view's uploads overlap another's downloads and kernels.  Same bytes per step, every copy inside the timed region.
+        NS = args.e2e_inflight
+        slots = [{"arena": arena, "color": color_h, "grad": grad_h, "stream": torch.cuda.Stream(dev)}]
+        for _ in range(NS - 1):
+            slots.append({"arena": torch.empty(arena_bytes, dtype=torch.uint8, device=dev),
+                          "color": torch.empty_like(color_h).pin_memory(), "grad": torch.empty_like(grad_h).pin_memory(),
+                          "stream": torch.cuda.Stream(dev)})
+        for sl in slots:
+            sl["counts"] = torch.zeros(G.COUNTS_WORDS, dtype=torch.int32).pin_memory()
+            sl["busy"] = False
+        p_hits = 0
+
+        def drain(sl):
+            if sl["busy"]:
+                sl["stream"].synchronize()
+                st = G.gart_counts_status(sl["counts"])
+                if st != G.GART_OK:
+                    raise RuntimeError("gart_view_host_async: status %d" % st)
+                sl["busy"] = False
+                return int(sl["counts"].numpy().view(np.uint32)[G.CNT_HITS])
+            return 0
+
+        n_pipe = NS * args.e2e_steps
+        for s in range(NS + n_pipe):                    # one untimed view per slot first
+            if s == NS:
+                for sl in slots:
+                    drain(sl)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+            sl = slots[s % NS]
+            got = drain(sl)                             # the slot's previous view has landed on the host: its arrays are free again
+            if s >= 2 * NS:
+                p_hits += got
+            v = mine[s % len(mine)]
+            G.gart_view_host_async(cfg, hs, cams[v], hdl[v], sl["color"], sl["grad"], cap_pairs, cap_hits, sl["counts"], sl["arena"], sl["stream"])
+            sl["busy"] = True
+        for sl in slots:
+            p_hits += drain(sl)
+        p_t = time.perf_counter() - t0
+        e2e = {"value": reduce_e2e(p_hits, p_t), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * p_t / n_pipe, "steps": n_pipe, "mode": "%d views in flight (gart_view_host_async, one stream each)" % NS,
+               "one_view_at_a_time": serial}
 
     if rank != 0:
         if world > 1:
@@ -540,6 +586,7 @@ def main():
     ap.add_argument("--lt16-reps", type=int, default=2, help="timed runs of forward + backward with 8-byte LT entries on the last view (0: skip)")
     ap.add_argument("--other-ts-reps", type=int, default=2, help="timed runs of the whole step at the other tile size on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-inflight", type=int, default=3, help="views in flight in the end-to-end measurement (each holds an arena on the device)")
     ap.add_argument("--oracle-frac", type=float, default=0.08)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--crop", type=float, default=1.0, help="central crop of every view (profiling on a smaller case)")

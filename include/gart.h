@@ -413,6 +413,21 @@ gart_status gart_view_host(const gart_config *cfg, const gart_gaussians *g_host,
                            int64_t cap_pairs, int64_t cap_hits, uint32_t *counts_host,
                            void *arena, size_t arena_bytes, void *stream);
 
+/*
+ * The same, without waiting: every copy and kernel of the view is queued on `stream` and the call returns.  The host
+ * arrays (pinned, for the copies to be asynchronous) and counts_host are valid once the stream has been synchronised;
+ * gart_counts_status(counts_host) then gives the status gart_view_host would have returned.  Two views in flight on two
+ * streams, each with an arena and output arrays of its own, overlap one view's uploads with the other's downloads
+ * (the two directions of the host link) and with its kernels.
+ */
+gart_status gart_view_host_async(const gart_config *cfg, const gart_gaussians *g_host, const gart_camera *cam,
+                           const float *dL_dcolor_host, float *color_host, float *grad_host,
+                           int64_t cap_pairs, int64_t cap_hits, uint32_t *counts_host,
+                           void *arena, size_t arena_bytes, void *stream);
+
+/* The status that a counts block copied to the host encodes: GART_ERR_TIMEOUT, GART_ERR_CAPACITY_EXCEEDED or GART_OK. */
+gart_status gart_counts_status(const uint32_t *counts_host);
+
 #ifdef __cplusplus
 }
 #endif

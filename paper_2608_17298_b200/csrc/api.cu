@@ -79,10 +79,10 @@ extern "C" size_t gart_view_host_arena_bytes(int64_t n, int32_t sh_degree, int32
     return gart::arena_layout(nullptr, n, K, width, height, tile_size, cap_pairs, cap_hits).bytes;
 }
 
-extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussians* gh, const gart_camera* cam,
-                                      const float* dL_dcolor_host, float* color_host, float* grad_host,
-                                      int64_t cap_pairs, int64_t cap_hits, uint32_t* counts_host,
-                                      void* arena, size_t arena_bytes, void* stream) {
+extern "C" gart_status gart_view_host_async(const gart_config* cfg, const gart_gaussians* gh, const gart_camera* cam,
+                                            const float* dL_dcolor_host, float* color_host, float* grad_host,
+                                            int64_t cap_pairs, int64_t cap_hits, uint32_t* counts_host,
+                                            void* arena, size_t arena_bytes, void* stream) {
     using namespace gart;
     if (!cfg || !gh || !cam || !dL_dcolor_host || !color_host || !counts_host || !arena) return GART_ERR_INVALID_ARG;
     if (gh->n < 0 || gh->sh_degree < 0 || gh->sh_degree > 3) return GART_ERR_INVALID_ARG;
@@ -123,9 +123,24 @@ extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussia
     if (cudaMemcpyAsync(color_host, a.color, (size_t)hw * 12, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GART_ERR_CUDA;
     if (n > 0 && cudaMemcpyAsync(grad_host, a.grad, (size_t)n * GART_GRAD_WORDS * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return GART_ERR_CUDA;
-    s = gart_read_counts(a.counts, counts_host, stream);
-    if (s != GART_OK) return s;
+    if (cudaMemcpyAsync(counts_host, a.counts, GART_COUNTS_WORDS * sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return GART_ERR_CUDA;
+    return GART_OK;
+}
+
+extern "C" gart_status gart_counts_status(const uint32_t* counts_host) {
+    if (!counts_host) return GART_ERR_INVALID_ARG;
     if (counts_host[GART_CNT_ERROR] & GART_ERRBIT_TIMEOUT) return GART_ERR_TIMEOUT;
     if (counts_host[GART_CNT_ERROR]) return GART_ERR_CAPACITY_EXCEEDED;
     return GART_OK;
+}
+
+extern "C" gart_status gart_view_host(const gart_config* cfg, const gart_gaussians* gh, const gart_camera* cam,
+                                      const float* dL_dcolor_host, float* color_host, float* grad_host,
+                                      int64_t cap_pairs, int64_t cap_hits, uint32_t* counts_host,
+                                      void* arena, size_t arena_bytes, void* stream) {
+    const gart_status s = gart_view_host_async(cfg, gh, cam, dL_dcolor_host, color_host, grad_host, cap_pairs, cap_hits, counts_host, arena,
+                                               arena_bytes, stream);
+    if (s != GART_OK) return s;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return GART_ERR_CUDA;
+    return gart_counts_status(counts_host);
 }

@@ -36,7 +36,7 @@ EXPORTS = [
     "gart_forward_workspace_bytes", "gart_forward",
     "gart_backward_workspace_bytes", "gart_backward", "gart_backward_tile", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp",
     "gart_workspace_bytes", "gart_read_counts", "gart_sync_status",
-    "gart_view_host_arena_bytes", "gart_view_host",
+    "gart_view_host_arena_bytes", "gart_view_host", "gart_view_host_async", "gart_counts_status",
 ]
 
 
@@ -107,8 +107,10 @@ def lib():
         L.gart_view_host_arena_bytes.restype = sz
         L.gart_view_host_arena_bytes.argtypes = [i64, i32, i32, i32, i32, i64, i64]
         L.gart_view_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
+        L.gart_view_host_async.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp, vp, sz, vp]
+        L.gart_counts_status.argtypes = [vp]
         for fn in ("gart_bounds", "gart_tile_map", "gart_forward", "gart_backward", "gart_backward_tile", "gart_backward_atomic",
-                   "gart_backward_hybrid", "gart_backward_warp", "gart_read_counts", "gart_sync_status", "gart_view_host", "gart_view_array"):
+                   "gart_backward_hybrid", "gart_backward_warp", "gart_read_counts", "gart_sync_status", "gart_view_host", "gart_view_host_async", "gart_counts_status", "gart_view_array"):
             getattr(L, fn).restype = C.c_int
         _lib = L
     return _lib
@@ -391,6 +393,36 @@ def gart_sync_status(counts, stream=None) -> int:
 def gart_view_host_arena_bytes(n, sh_degree, width, height, tile_size, cap_pairs, cap_hits) -> int:
     return int(lib().gart_view_host_arena_bytes(int(n), int(sh_degree), int(width), int(height), int(tile_size),
                                                 int(cap_pairs), int(cap_hits)))
+
+
+def _host_ptr(t, what, dtype=torch.float32):
+    if not (isinstance(t, torch.Tensor) and not t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError("%s must be a contiguous CPU %s tensor" % (what, dtype))
+    return t.data_ptr()
+
+
+def _host_scene(scene) -> _Gaussians:
+    gs = _Gaussians()
+    gs.n, gs.sh_degree = int(scene.mean.shape[0]), int(scene.sh_degree)
+    gs.mean, gs.scale, gs.quat = _host_ptr(scene.mean, "mean"), _host_ptr(scene.scale, "scale"), _host_ptr(scene.quat, "quat")
+    gs.opacity, gs.sh = _host_ptr(scene.opacity, "opacity"), _host_ptr(scene.sh, "sh")
+    return gs
+
+
+def gart_view_host_async(cfg: Config, scene, cam, dL_dcolor, color_out, grad_out, cap_pairs, cap_hits, counts_out, arena, stream=None):
+    """gart_view_host without waiting: everything is queued on ``stream``.  ``counts_out`` is a pinned CPU int32 tensor of
+    COUNTS_WORDS words; after synchronising the stream, gart_counts_status(counts_out) gives the status."""
+    gs = _host_scene(scene)
+    c, cs = cfg.c(), camera_struct(cam)
+    if counts_out.numel() < COUNTS_WORDS:
+        raise ValueError("counts_out must hold COUNTS_WORDS words")
+    _check(lib().gart_view_host_async(C.byref(c), C.byref(gs), C.byref(cs), _host_ptr(dL_dcolor, "dL_dcolor"), _host_ptr(color_out, "color_out"),
+                                      _host_ptr(grad_out, "grad_out"), int(cap_pairs), int(cap_hits), _host_ptr(counts_out, "counts_out", torch.int32),
+                                      _dev(arena, torch.uint8, "arena"), arena.numel(), _stream_ptr(stream)), "gart_view_host_async")
+
+
+def gart_counts_status(counts_out) -> int:
+    return int(lib().gart_counts_status(_host_ptr(counts_out, "counts_out", torch.int32)))
 
 
 def gart_view_host(cfg: Config, scene, cam, dL_dcolor, color_out, grad_out, cap_pairs, cap_hits, arena, stream=None):

@@ -574,7 +574,7 @@ def test_invalid_arguments_return_status():
 
 def test_host_entry_point_matches_device_path():
     scene, cams = gs.config_cluster(n=2000, width=96, height=64)
-    cam, cfg = cams[0], G.Config(tile_size=8)
+    cam, cfg = cams[0], G.Config(tile_size=8, lt_layout=G.LT_PRIMITIVE_MAJOR)
     g = gs.upstream_gradient(cam, 0)
     gpu = P.run_gpu(scene, cam, cfg, g, atomic=False)
     Pn, Hn = gpu["counts"][G.CNT_PAIRS], gpu["counts"][G.CNT_HITS]
@@ -610,3 +610,32 @@ def test_host_entry_point_matches_device_path():
     assert np.array_equal(color.numpy(), gpu2["color"]) and np.abs(gpu2["color"] - gpu["color"]).max() > 1e-3
     a, b = grad.numpy().astype(np.float64), gpu2["grad_lt16"].astype(np.float64)
     assert np.all(np.abs(a - b) <= 1e-4 * np.abs(b) + 1e-5 * np.abs(b).max(axis=1, keepdims=True) + 1e-7)
+    # two views in flight on two streams (gart_view_host_async), each with its own arena and host arrays: the results of
+    # the one-at-a-time calls, to the bit for colour and, for the item pass on Gaussians that are one item, for the gradient
+    cfg = G.Config(tile_size=8, lt_layout=G.LT_PRIMITIVE_MAJOR)
+    want = []
+    for v in (0, 1):
+        gv = torch.from_numpy(gs.upstream_gradient(cam, v)).pin_memory()
+        G.gart_view_host(cfg, hs, cam, gv, color, grad, Pn + 5, Ln + 5, arena)
+        want.append((gv, color.clone(), grad.clone()))
+    slots = []
+    for v in (0, 1):
+        slots.append({"color": torch.empty_like(color).pin_memory(), "grad": torch.empty_like(grad).pin_memory(),
+                      "counts": torch.zeros(G.COUNTS_WORDS, dtype=torch.int32).pin_memory(), "stream": torch.cuda.Stream(),
+                      "arena": torch.empty_like(arena)})
+    torch.cuda.synchronize()
+    for v, sl in enumerate(slots):
+        G.gart_view_host_async(cfg, hs, cam, want[v][0], sl["color"], sl["grad"], Pn + 5, Ln + 5, sl["counts"], sl["arena"], sl["stream"])
+    for v, sl in enumerate(slots):
+        sl["stream"].synchronize()
+        assert G.gart_counts_status(sl["counts"]) == G.GART_OK
+        assert sl["counts"].numpy().view(np.uint32)[G.CNT_HITS] == Hn
+        assert np.array_equal(sl["color"].numpy(), want[v][1].numpy())
+        a, b = sl["grad"].numpy().astype(np.float64), want[v][2].numpy().astype(np.float64)
+        assert np.all(np.abs(a - b) <= 1e-4 * np.abs(b) + 1e-5 * np.abs(b).max(axis=1, keepdims=True) + 1e-7)
+    assert np.abs(slots[0]["grad"].numpy() - slots[1]["grad"].numpy()).max() > 0      # (two different upstream gradients)
+    # a capacity error shows in the counts block once the stream is done
+    sl = slots[0]
+    G.gart_view_host_async(cfg, hs, cam, want[0][0], sl["color"], sl["grad"], Pn + 5, Hn // 2, sl["counts"], sl["arena"], sl["stream"])
+    sl["stream"].synchronize()
+    assert G.gart_counts_status(sl["counts"]) == 3
