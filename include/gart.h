@@ -9,10 +9,12 @@
  *   gart_forward   ray evaluation: hits ordered by maximum-response distance, compositing,
  *                  and the compact per-hit buffer LT (16 bytes per hit: alpha dC/dalpha and the
  *                  blending weight T alpha, see gart_forward)
- *   gart_backward  primitive-centric backward: a thread gathers the gradients of one Gaussian over
- *                  the hit pixels of its (tile, Gaussian) pairs, with the sums in registers
- *   gart_backward_tile     the same pass in the paper's decomposition: block per tile, thread per pair,
- *                          one vector atomic update per pair
+ *   gart_backward  primitive-centric backward, in the decomposition that matches the layout of LT
+ *                  (cfg->lt_layout): tile-major -- the paper's: block per tile, thread per (tile, Gaussian)
+ *                  pair, one vector atomic update per pair (the faster whole step on B200); primitive-major
+ *                  -- a thread gathers the gradients of one Gaussian over the hit pixels of all its pairs
+ *                  and writes its record once (half the DRAM traffic of the pass, a dearer forward)
+ *   gart_backward_tile     the tile-major pass by name (what gart_backward runs for that layout)
  *   gart_backward_atomic   the pixel-centric baseline: one thread per ray, atomicAdd per hit
  *   gart_backward_warp     gart_backward_tile with a warp per pair (ownership ablation)
  *   gart_backward_hybrid   colour gradients primitive-centric from 4 bytes per hit, the rest pixel-centric
@@ -65,8 +67,10 @@ typedef enum {
 
 /* Layouts of the intermediate buffer LT (gart_config.lt_layout). */
 enum {
-    GART_LT_PRIMITIVE_MAJOR = 0,  /* hits grouped by Gaussian: what gart_backward reads */
-    GART_LT_TILE_MAJOR = 1        /* hits grouped by (tile, Gaussian) pair inside each tile: gart_backward_tile, _warp, _hybrid */
+    GART_LT_PRIMITIVE_MAJOR = 0,  /* hits grouped by Gaussian (work items of a 16 x 16-pixel super-tile): gart_backward's item pass */
+    GART_LT_TILE_MAJOR = 1        /* hits grouped by (tile, Gaussian) pair inside each tile: gart_backward's block-per-tile pass
+                                     (= gart_backward_tile), gart_backward_warp, gart_backward_hybrid.  The faster whole step:
+                                     callers that do not care should set this one (the Python binding's default). */
 };
 
 /* Host struct. */
@@ -87,8 +91,10 @@ typedef struct {
                              the cap keep their place in every list and their LT slot, with a zero entry: they
                              add nothing to the colour, to T_final or to a gradient (the backward passes that
                              read lt need no change; gart_backward_hybrid rejects a cap) */
-    int32_t lt_layout;    /* GART_LT_PRIMITIVE_MAJOR (0, for gart_backward) or GART_LT_TILE_MAJOR (the ablation passes):
-                             where gart_forward puts a hit's entry in lt.  The entries' contents are the same. */
+    int32_t lt_layout;    /* GART_LT_PRIMITIVE_MAJOR (0) or GART_LT_TILE_MAJOR (1): where gart_forward puts a hit's entry in lt,
+                             and with it which pass gart_backward runs.  The entries' contents are the same (the
+                             primitive-major entries also carry their pixel's index in low mantissa bits).  gart_bounds
+                             reads it too (the order of the slots follows the layout): use one value for a whole view. */
     float t_min;          /* 0: off (the paper's setting).  > 0: early termination, as in the tracers the paper compares with
                              (Sec. 5.5): a ray ends before the first hit whose transmittance in front is below t_min; that
                              hit and the later ones keep their place in every list and get a zero LT entry, like the hits
@@ -310,20 +316,22 @@ gart_status gart_forward(const gart_config *cfg, const gart_gaussians *g, const 
                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * Step 4 -- primitive-centric backward (Sec. 4.4).  A thread gathers the gradient sums of ONE work item of the
+ * Step 4 -- primitive-centric backward (Sec. 4.4).  With cfg->lt_layout = GART_LT_TILE_MAJOR this call IS
+ * gart_backward_tile (below).  With GART_LT_PRIMITIVE_MAJOR a thread gathers the gradient sums of ONE work item of the
  * primitive-major order: it walks the item's (tile, Gaussian) pairs one after the other and, per pair, the pair's hit
  * pixels, reads their LT entries (coalesced across the warp thanks to the interleaved layout) and accumulates in
  * registers.  No per-pixel atomics.  An item that is a whole Gaussian (its rectangle fits a 32 x 32-pixel window: nearly
  * all of them) ends with the conversion of the moments and ONE write of the 256-byte gradient record -- no atomic, no
  * accumulation record; the pieces of larger Gaussians add to an accumulation record with one vector atomic per 16 bytes
- * and piece, converted by a small per-slot pass.  Needs gart_forward run with lt_layout = GART_LT_PRIMITIVE_MAJOR.
+ * and piece, converted by a small per-slot pass.  gart_bounds and gart_forward must have run with the same lt_layout.
  *   dL_dcolor [H,W,3] in.
  *   grad [n,GART_GRAD_WORDS] out, fully overwritten: d mean, d scale, d quat, d opacity, d sh
  *        of L = sum <dL_dcolor, color>; zero for Gaussians without hits.
  *   view, cap_pairs: the view block that gart_forward filled and the capacity it was laid out for.
  *   counts: read (a set error bit skips the work); GART_ERRBIT_TIMEOUT is set if a wait on an
  *        asynchronous copy ran out, in which case grad is incomplete.
- * cfg->lt_format must be 0 (INVALID_ARG otherwise): the pass finds a hit's pixel in its 16-byte entry.
+ * In the primitive-major layout cfg->lt_format must be 0 (INVALID_ARG otherwise): the pass finds a hit's pixel in its
+ * 16-byte entry.
  * The main kernel uses 54 KB of dynamic shared memory per block: LT blocks are streamed in with bulk
  * asynchronous copies, one rank group ahead, beside dL/dC of the block's 32 x 32-pixel window and the
  * Gaussians' records.
