@@ -236,11 +236,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
             if (k + 1 < nchunks) produce(cur, nxt, nxt2, 2);   // refill the stage just released (after the last chunk it first serves the flush)
         }
         {
-            // Flush through the stage just released, so that consecutive lanes add consecutive 16-byte pieces of one
+            // Flush through the stage just released, so that neighbouring lanes add neighbouring 16-byte pieces of one
             // record: the atomics of a record then reach L2 as whole 32-byte sectors (about 9 sector updates per pair
             // instead of 15).  Two rounds of FLUSH_Q pieces per lane, then the last piece directly.
             constexpr int NQ = AW / 4, FLUSH_Q = BWD_CHUNK;
-            static_assert(NQ <= 2 * FLUSH_Q + 1 && NQ >= 1, "flush rounds");
+            static_assert(NQ <= 2 * FLUSH_Q + 1 && NQ >= 1 && FLUSH_Q <= 8, "flush rounds");
             float4* tb = my_stage + ((unit - 1u) % BWD_STAGES) * BWD_STAGE_F4;
             const uint32_t tag = cur.c != 0 ? cur.sid : 0xffffffffu;
             const uint64_t pol_keep = l2_policy_evict_last();   // (made where they are used: the policies hold no register across the hit loop)
@@ -253,6 +253,11 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                 }
                 return make_float4(v[0], v[1], v[2], v[3]);
             };
+            // Reading the staged pieces back, eight lanes serve one record: lanes 8 g .. 8 g + nq - 1 take the round's nq
+            // pieces of record 4 j + g.  A lane's piece, and with it the array, the row stride and the offset in the row, is
+            // then the same for all eight reads of a round, and the address of a reduction is one multiply-add (with the
+            // pieces dealt lane by lane across records it took an integer division per read).
+            const int hl = lane >> 3, pc = lane & 7;
 #pragma unroll
             for (int q0 = 0; q0 + 1 < NQ; q0 += FLUSH_Q) {
                 const int nq = NQ - 1 - q0 < FLUSH_Q ? NQ - 1 - q0 : FLUSH_Q;   // compile-time after unrolling
@@ -260,13 +265,17 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                 for (int j = 0; j < FLUSH_Q; ++j)
                     if (j < nq) tb[lane * nq + j] = piece(q0 + j);
                 __syncwarp();
+                const int q = q0 + pc;
+                const bool in_a = q < GACC_A_WORDS / 4;
+                char* const row0 = in_a ? reinterpret_cast<char*>(gacc.a) + 16 * q : reinterpret_cast<char*>(gacc.b) + 16 * (q - GACC_A_WORDS / 4);
+                const uint32_t row_bytes = in_a ? GACC_A_WORDS * 4u : GACC_B_WORDS * 4u;
+                const float4* tl = tb + hl * nq + pc;
 #pragma unroll
-                for (int j = 0; j < FLUSH_Q; ++j) {
-                    if (j < nq) {
-                        const int i = j * 32 + lane, pr = i / nq, q = q0 + i - pr * nq;
-                        const float4 v = tb[i];
-                        const uint32_t sd = __shfl_sync(0xffffffffu, tag, pr);
-                        if (sd != 0xffffffffu) red_add_f4_hint(gacc_piece(gacc, sd, q), v.x, v.y, v.z, v.w, pol_keep);
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t sd = __shfl_sync(0xffffffffu, tag, 4 * j + hl);
+                    if (pc < nq && sd != 0xffffffffu) {
+                        const float4 v = tl[4 * j * nq];
+                        red_add_f4_hint(reinterpret_cast<float4*>(row0 + (size_t)sd * row_bytes), v.x, v.y, v.z, v.w, pol_keep);
                     }
                 }
                 __syncwarp();
