@@ -86,7 +86,14 @@ typedef struct {
     double alpha_max; /* >= 1: off.  < 1: a hit's alpha is min(sigma rho, alpha_max); where the clamp is active alpha is a
                          constant, so the hit passes no gradient to opacity, mean, scale or rotation (its colour still
                          gets one) */
+    int64_t kernel_degree; /* k of the response rho = exp(-D^k / 2), D the Mahalanobis distance of the ray's closest point
+                         (Eq. 4 is k = 2, the paper's benchmark setting, Sec. 5.2; 0 means 2).  An even k > 2 is a "narrow"
+                         kernel, the last of the compromises the paper lists for 3DGRT (Sec. 5.5): flatter top, faster
+                         fall-off, and a clamping radius alpha_c = (2 ln(sigma / alpha_min))^(1/k) in place of Eq. 9-10's
+                         square root.  The maximum-response point along a ray does not depend on k */
 } orc_config;
+
+static int kernel_degree_of(const orc_config *cfg) { return cfg->kernel_degree > 0 ? (int)cfg->kernel_degree : 2; }
 
 /* ------------------------------------------------------------------ threads */
 int orc_max_threads(void) {
@@ -177,7 +184,7 @@ static void gauss_geometry(const orc_scene *s, int64_t i, const orc_camera *cam,
     const double sigma = s->opacity[i];
     g->cls = 0; g->cls_margin = fabs(sigma - cfg->alpha_min);
     if (!(sigma > cfg->alpha_min)) return;
-    g->alpha_c = sqrt(2.0 * log(sigma / cfg->alpha_min));
+    g->alpha_c = pow(2.0 * log(sigma / cfg->alpha_min), 1.0 / kernel_degree_of(cfg));   /* Eq. 9-10 for exp(-D^k / 2) */
     double R[9];
     quat_to_R(s->quat + 4 * i, R);
     const double *sc = s->scale + 3 * i;
@@ -370,7 +377,7 @@ static void gauss_local(const orc_scene *s, int64_t i, const double *o, double *
 }
 
 /* Response of Gaussian (Wm, og, sigma) along unit direction d: t*, alpha, x_g (Eq. 4, 5, 8). */
-static void ray_response(const double *Wm, const double *og, double sigma, const double *d,
+static void ray_response(const double *Wm, const double *og, double sigma, const double *d, int kdeg,
                          double *tstar, double *alpha, double *xg) {
     double dg[3];
     for (int k = 0; k < 3; ++k) dg[k] = Wm[3 * k] * d[0] + Wm[3 * k + 1] * d[1] + Wm[3 * k + 2] * d[2];
@@ -381,7 +388,7 @@ static void ray_response(const double *Wm, const double *og, double sigma, const
     for (int k = 0; k < 3; ++k) x[k] = og[k] + ts * dg[k];
     const double D2 = x[0] * x[0] + x[1] * x[1] + x[2] * x[2];
     *tstar = ts;
-    *alpha = sigma * exp(-0.5 * D2);
+    *alpha = sigma * exp(-0.5 * pow(D2, 0.5 * kdeg));   /* Eq. 4 at k = 2 */
     if (xg) { xg[0] = x[0]; xg[1] = x[1]; xg[2] = x[2]; }
 }
 
@@ -391,7 +398,7 @@ void orc_view_eval_pair(const orc_view *v, int64_t ray, int64_t gid, double *out
     cam_origin(&v->cam, o);
     cam_ray_dir(&v->cam, (int)(ray % v->cam.width), (int)(ray / v->cam.width), d);
     gauss_local(&v->sc, gid, o, Wm, og);
-    ray_response(Wm, og, v->sc.opacity[gid], d, &out[1], &out[0], NULL);
+    ray_response(Wm, og, v->sc.opacity[gid], d, kernel_degree_of(&v->cfg), &out[1], &out[0], NULL);
 }
 
 /*
@@ -460,7 +467,7 @@ int64_t orc_view_find_hits(orc_view *v, int mode, const uint8_t *pixel_mask) {
                 if (pixel_mask && !pixel_mask[ray]) continue;
                 double d[3], ts, al;
                 cam_ray_dir(&v->cam, x, y, d);
-                ray_response(Wm, og, sigma, d, &ts, &al, NULL);
+                ray_response(Wm, og, sigma, d, kernel_degree_of(&v->cfg), &ts, &al, NULL);
                 if (!(al >= v->cfg.alpha_min && ts > 0.0)) continue;
                 if (pass == 0) {
 #pragma omp atomic
@@ -527,7 +534,7 @@ void orc_view_set_hits(orc_view *v, const uint64_t *ray_off, const uint32_t *gid
         for (uint64_t h = ray_off[r]; h < ray_off[r + 1]; ++h) {
             double Wm[9], og[3];
             gauss_local(&v->sc, gid[h], o, Wm, og);
-            ray_response(Wm, og, v->sc.opacity[gid[h]], d, &v->t[h], &v->alpha[h], NULL);
+            ray_response(Wm, og, v->sc.opacity[gid[h]], d, kernel_degree_of(&v->cfg), &v->t[h], &v->alpha[h], NULL);
         }
     }
 }
@@ -735,11 +742,15 @@ int orc_view_backward(orc_view *v, const double *dL_dC, double *grad, double *gr
             const double sigma = v->sc.opacity[i];
             const double rho = al / sigma;
             contrib[10] = dalpha * rho;
-            const double Gd = -0.5 * al * dalpha; /* dL / d(D^2); d(D^2)/dt* = 0 at the maximum */
             /* geometry */
             double Wm[9], og[3], ts, a2, xg[3];
             gauss_local(&v->sc, i, o, Wm, og);
-            ray_response(Wm, og, sigma, d, &ts, &a2, xg);
+            const int kdeg = kernel_degree_of(&v->cfg);
+            ray_response(Wm, og, sigma, d, kdeg, &ts, &a2, xg);
+            /* dL / d(D^2) with alpha = sigma exp(-(D^2)^(k/2) / 2): d alpha / d(D^2) = -alpha (k/4) (D^2)^(k/2 - 1), i.e.
+             * -alpha / 2 at k = 2; d(D^2)/dt* = 0 at the maximum */
+            const double D2 = xg[0] * xg[0] + xg[1] * xg[1] + xg[2] * xg[2];
+            const double Gd = -0.25 * kdeg * pow(D2, 0.5 * kdeg - 1.0) * al * dalpha;
             const double *mu = v->sc.mean + 3 * i, *sc = v->sc.scale + 3 * i, *q = v->sc.quat + 4 * i;
             const double xw[3] = {o[0] + ts * d[0] - mu[0], o[1] + ts * d[1] - mu[1], o[2] + ts * d[2] - mu[2]};
             for (int j = 0; j < 3; ++j)

@@ -44,7 +44,7 @@ class _Scene(C.Structure):
 
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_double), ("near_z", C.c_double), ("bg", C.c_double * 3), ("max_hits", C.c_int64),
-                ("t_min", C.c_double), ("alpha_max", C.c_double)]
+                ("t_min", C.c_double), ("alpha_max", C.c_double), ("kernel_degree", C.c_int64)]
 
 
 _lib = None
@@ -109,8 +109,9 @@ def _camera(cam) -> _Camera:
     return c
 
 
-def _config(alpha_min, near, bg, max_hits=0, t_min=0.0, alpha_max=1.0) -> _Config:
+def _config(alpha_min, near, bg, max_hits=0, t_min=0.0, alpha_max=1.0, kernel_degree=2) -> _Config:
     c = _Config()
+    c.kernel_degree = int(kernel_degree)
     c.alpha_min, c.near_z = float(alpha_min), float(near)
     c.max_hits = int(max_hits)
     c.t_min, c.alpha_max = float(t_min), float(alpha_max)
@@ -158,12 +159,13 @@ def ray(cam, x, y):
     return o, d
 
 
-def bounds(scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR):
-    """Eq. 9-14: returns rect [n,4] int32 (x0,y0,x1,y1 inclusive), cls [n] uint8, margin [n] float64."""
+def bounds(scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, kernel_degree=2):
+    """Eq. 9-14: returns rect [n,4] int32 (x0,y0,x1,y1 inclusive), cls [n] uint8, margin [n] float64.
+    kernel_degree k: the response is exp(-D^k / 2) (k = 2: Eq. 4), so the clamping radius is (2 ln(sigma/alpha_min))^(1/k)."""
     rect = np.zeros((scene.n, 4), dtype=np.int32)
     cls = np.zeros(scene.n, dtype=np.uint8)
     margin = np.zeros(scene.n, dtype=np.float64)
-    c, g = _camera(cam), _config(alpha_min, near, (0, 0, 0))
+    c, g = _camera(cam), _config(alpha_min, near, (0, 0, 0), kernel_degree=kernel_degree)
     lib().orc_bounds(C.byref(scene.c), C.byref(c), C.byref(g), _ptr(rect), _ptr(cls), _ptr(margin))
     return rect, cls, margin
 
@@ -189,11 +191,12 @@ class View:
     """One camera view of a scene: hit discovery, ordering, compositing, backward."""
 
     def __init__(self, scene: OracleScene, cam, alpha_min=ALPHA_MIN, near=NEAR, bg=(0.0, 0.0, 0.0), max_hits=0, t_min=0.0,
-                 alpha_max=1.0):
+                 alpha_max=1.0, kernel_degree=2):
         """max_hits > 0 composites only the first max_hits hits of every ray (0: all of them); t_min > 0 ends a ray before
-        the first hit with less than t_min transmittance in front of it; alpha_max < 1 clamps every hit's alpha."""
+        the first hit with less than t_min transmittance in front of it; alpha_max < 1 clamps every hit's alpha;
+        kernel_degree k > 2 (even) makes the response exp(-D^k / 2), a narrow kernel (k = 2: the Gaussian of Eq. 4)."""
         self.scene, self.cam = scene, cam
-        self._c, self._g = _camera(cam), _config(alpha_min, near, bg, max_hits, t_min, alpha_max)
+        self._c, self._g = _camera(cam), _config(alpha_min, near, bg, max_hits, t_min, alpha_max, kernel_degree)
         self.n_rays = int(cam.width) * int(cam.height)
         self._h = lib().orc_view_create(C.byref(scene.c), C.byref(self._c), C.byref(self._g))
         self._keep = None
