@@ -114,6 +114,14 @@ typedef struct {
                              and returns.  The call's outputs are then undefined, the context stays usable, and
                              gart_sync_status returns GART_ERR_TIMEOUT.  Read by gart_backward, gart_backward_tile and
                              gart_backward_hybrid (the kernels that stream the intermediate buffer through shared memory). */
+    int32_t kernel_degree; /* k of the response rho = exp(-D^k / 2), D the Mahalanobis distance of the ray's closest point (Eq. 5).
+                             0 or 2: the Gaussian of Eq. 4, the paper's setting (Sec. 5.2).  4: a narrow kernel, the last of the
+                             compromises that Sec. 5.5 lists for 3DGRT (flatter top, faster fall-off); the paper prints no
+                             formula for it, this is the reading taken.  The clamping radius of Eq. 9-10 becomes
+                             (2 ln(sigma / alpha_min))^(1/k), the maximum-response point and t* do not change, and
+                             d alpha / d(D^2) = -alpha (k/4) (D^2)^(k/2 - 1).  Read by gart_bounds, gart_forward and every
+                             backward pass (use one value for a whole view); other values are GART_ERR_INVALID_ARG, and so is
+                             4 in gart_backward_hybrid */
 } gart_config;
 
 /* Host struct. */

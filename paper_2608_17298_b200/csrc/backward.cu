@@ -66,8 +66,10 @@ __device__ __forceinline__ void pair_geo_at(const PairGeo& P, float u, float v, 
 // Gradient terms of one hit (pixel p of the tile, LT entry L) added to the pair's accumulators:
 // geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz), geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh.
 // With y = d_g x (o_g x d_g) and a = |d_g|^2 the maximum-response point is x_g = y / a, so
-// G x_g = (G / a) y and G x_g x_g^T = (G / a^2) y y^T.
-template <int TS, int K>
+// G x_g = (G / a) y and G x_g x_g^T = (G / a^2) y y^T.  G = dL/d(D^2) = -(alpha dL/dalpha) (KD / 4) (D^2)^(KD/2 - 1) for the
+// response exp(-D^KD / 2): -1/2 of alpha dL/dalpha for the Gaussian (KD = 2), -D^2 times it for the degree-4 kernel, with
+// D^2 = |o_g x d_g|^2 / a.
+template <int TS, int K, int KD = 2>
 __device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* geo, const float4* spix, int p, const float4 L) {
     const float4 pa = spix[PixLayout<TS>::index(p, 0, 0)], pb = spix[PixLayout<TS>::index(p, 1, 0)];   // spix points at the lane's copy
     float3 dg, cr;
@@ -82,7 +84,9 @@ __device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* g
     const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
     geo[9] += ad;
     const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
-    const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+    float s1 = -0.5f * ad * inv_a;
+    if constexpr (KD == 4) s1 *= 2.0f * inv_a * fmaf(cr.x, cr.x, fmaf(cr.y, cr.y, cr.z * cr.z));
+    const float s2 = s1 * inv_a;
     geo[0] = fmaf(s1, yx, geo[0]); geo[1] = fmaf(s1, yy, geo[1]); geo[2] = fmaf(s1, yz, geo[2]);
     const float tx = s2 * yx, ty = s2 * yy, tz = s2 * yz;
     geo[3] = fmaf(tx, yx, geo[3]); geo[4] = fmaf(ty, yy, geo[4]); geo[5] = fmaf(tz, yz, geo[5]);
@@ -90,7 +94,7 @@ __device__ __forceinline__ void bwd_hit(const PairGeo& P, ShRegs<K>& R, float* g
 }
 
 // FMT: 0 = 16-byte LT entries, 2 = 8-byte entries (four halves, twice as many per pipeline stage).
-template <int TS, int DEG, int FMT>
+template <int TS, int DEG, int FMT, int KD>
 __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4* __restrict__ rec,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
@@ -226,10 +230,10 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
                 const int p0 = cur.pm.next();
                 const int p1 = cur.pm.next();
                 const float4 L0 = entry(se), L1 = entry(se + 32 * EB);
-                bwd_hit<TS, K>(P, R, geo, spix_lane, p0, L0);
-                bwd_hit<TS, K>(P, R, geo, spix_lane, p1, L1);
+                bwd_hit<TS, K, KD>(P, R, geo, spix_lane, p0, L0);
+                bwd_hit<TS, K, KD>(P, R, geo, spix_lane, p1, L1);
             }
-            if (e < e_end) bwd_hit<TS, K>(P, R, geo, spix_lane, cur.pm.next(), entry(se));
+            if (e < e_end) bwd_hit<TS, K, KD>(P, R, geo, spix_lane, cur.pm.next(), entry(se));
             fence_proxy_async();
             __syncwarp();   // every lane is done with this stage before a later copy may overwrite it
             ++unit;
@@ -296,12 +300,12 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     }
 }
 
-template <int TS, int DEG, int FMT>
+template <int TS, int DEG, int FMT, int KD>
 static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                     const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                     const uint32_t* tile_lt_base, const float4* lt,
                                     const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts, uint32_t wait_limit) {
-    auto kern = bwd_pairs_kernel<TS, DEG, FMT>;
+    auto kern = bwd_pairs_kernel<TS, DEG, FMT, KD>;
     constexpr int smem = BWD_DYN_SMEM;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA;
     kern<<<T, BWD_THREADS, smem, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit);
@@ -310,12 +314,13 @@ static gart_status launch_pairs_deg(int T, cudaStream_t st, const float4* rec, c
 }
 
 template <int TS, int FMT>
-static gart_status launch_pairs(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
+static gart_status launch_pairs(int deg, bool narrow, int T, cudaStream_t st, const float4* rec, const uint32_t* tile_off,
                                 const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                 const uint32_t* tile_lt_base, const float4* lt,
                                 const float* dL_dC, const CamF& cam, const Gacc& gacc, uint32_t* counts, uint32_t wait_limit) {
-#define GART_PAIRS(D) \
-    return launch_pairs_deg<TS, D, FMT>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit)
+#define GART_PAIRS(D)                                                                                                                                       \
+    return narrow ? launch_pairs_deg<TS, D, FMT, 4>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit) \
+                  : launch_pairs_deg<TS, D, FMT, 2>(T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt, dL_dC, cam, gacc, counts, wait_limit)
     switch (deg) {
         case 0: GART_PAIRS(0);
         case 1: GART_PAIRS(1);
@@ -338,6 +343,7 @@ static gart_status tile_pass_args(const gart_config* cfg, const gart_gaussians* 
     if (!cfg || !g || !cam || !counts || !tile_off || !dL_dcolor) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // these passes read LT in the tile-major layout
+    if (!gart::kernel_degree_ok(cfg->kernel_degree)) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
@@ -369,7 +375,7 @@ extern "C" gart_status gart_backward_tile(const gart_config* cfg, const gart_gau
     const int T = cf.tiles_x * cf.tiles_y;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
-#define GART_PAIRS_TS(TSV, F) launch_pairs<TSV, F>(g->sh_degree, T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts, wait_limit_of(cfg->wait_polls))
+#define GART_PAIRS_TS(TSV, F) launch_pairs<TSV, F>(g->sh_degree, kernel_degree_is4(cfg->kernel_degree), T, st, rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts, wait_limit_of(cfg->wait_polls))
     if (cfg->lt_format == 0) s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 0) : GART_PAIRS_TS(16, 0);
     else s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 2) : GART_PAIRS_TS(16, 2);
 #undef GART_PAIRS_TS
@@ -403,7 +409,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
                                                                      const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
                                                                      const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ tile_lt_base,
                                                                      const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                                     Gacc gacc, const uint32_t* __restrict__ counts) {
+                                                                     Gacc gacc, const uint32_t* __restrict__ counts, const bool narrow) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
     constexpr int AW = (11 + SW + 3) & ~3;
     __shared__ __align__(16) float4 spix[NT * 2];   // (d, u), (g, v) per pixel, one copy: the lanes of a warp read different pixels
@@ -457,7 +463,9 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
             lt_weights(L, g, w);
             const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));
             const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
-            const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+            float s1 = -0.5f * ad * inv_a;
+            if (narrow) s1 *= 2.0f * inv_a * fmaf(cr.x, cr.x, fmaf(cr.y, cr.y, cr.z * cr.z));   // degree-4 kernel: dL/d(D^2) = -D^2 alpha dL/dalpha
+            const float s2 = s1 * inv_a;
             acc[0] = fmaf(s1, yx, acc[0]); acc[1] = fmaf(s1, yy, acc[1]); acc[2] = fmaf(s1, yz, acc[2]);
             acc[3] = fmaf(s2 * yx, yx, acc[3]); acc[4] = fmaf(s2 * yy, yy, acc[4]); acc[5] = fmaf(s2 * yz, yz, acc[5]);
             acc[6] = fmaf(s2 * yx, yy, acc[6]); acc[7] = fmaf(s2 * yx, yz, acc[7]); acc[8] = fmaf(s2 * yy, yz, acc[8]);
@@ -509,7 +517,7 @@ extern "C" gart_status gart_backward_warp(const gart_config* cfg, const gart_gau
     const int T = cf.tiles_x * cf.tiles_y;
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
-#define GART_WARP(TS, D) bwd_pairs_warp_kernel<TS, D><<<T, BWD_THREADS, 0, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts)
+#define GART_WARP(TS, D) bwd_pairs_warp_kernel<TS, D><<<T, BWD_THREADS, 0, st>>>(rec, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, lt4, dL_dcolor, cf, gacc, counts, kernel_degree_is4(cfg->kernel_degree))
     if (cfg->tile_size == 8) {
         switch (g->sh_degree) { case 0: GART_WARP(8, 0); break; case 1: GART_WARP(8, 1); break; case 2: GART_WARP(8, 2); break; default: GART_WARP(8, 3); break; }
     } else {

@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
                                                          const float* __restrict__ opacity, const uint32_t* __restrict__ ray_off,
                                                          const uint32_t* __restrict__ ray_gid, const uint32_t* __restrict__ ray_slot,
                                                          const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
-                                                         float* __restrict__ grad, const uint32_t* __restrict__ counts) {
+                                                         float* __restrict__ grad, const uint32_t* __restrict__ counts, const bool narrow) {
     constexpr int K = (DEG + 1) * (DEG + 1), RS4 = (20 + 3 * K + 3) / 4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -34,8 +34,9 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
         float wch[3];
         lt_weights(L, g, wch);
         const float ad = fmaf(g.x, L.x, fmaf(g.y, L.y, g.z * L.z));   // alpha dL/dalpha
-        const float G = -0.5f * ad;
         const float3 xg = ray_xg(r);
+        // dL/d(D^2): -1/2 alpha dL/dalpha for the Gaussian, -D^2 alpha dL/dalpha for the degree-4 kernel (D^2 = |x_g|^2)
+        const float G = narrow ? -ad * fmaf(xg.x, xg.x, fmaf(xg.y, xg.y, xg.z * xg.z)) : -0.5f * ad;
         const float v[3] = {G * xg.x, G * xg.y, G * xg.z};
         const float Q[6] = {v[0] * xg.x, v[1] * xg.y, v[2] * xg.z, v[0] * xg.y, v[0] * xg.z, v[1] * xg.z};
         const float q[4] = {quat[4 * gid], quat[4 * gid + 1], quat[4 * gid + 2], quat[4 * gid + 3]};
@@ -91,6 +92,7 @@ extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_g
     if (!grad || !pre || !slot_of_gid || !g->scale || !g->quat || !g->opacity || !ray_gid || !ray_slot || !lt) return GART_ERR_INVALID_ARG;
     if (cfg->atomic_mode != GART_ATOMIC_SCALAR && cfg->atomic_mode != GART_ATOMIC_VECTOR) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;   // reads 16-byte LT entries (either layout: the slot of every hit comes from ray_slot)
+    if (!kernel_degree_ok(cfg->kernel_degree)) return GART_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(grad, 0, (size_t)g->n * GART_GRAD_WORDS * sizeof(float), st) != cudaSuccess) return GART_ERR_CUDA;
     const CamF cf = make_camf(cam, cfg->tile_size);
@@ -98,7 +100,7 @@ extern "C" gart_status gart_backward_atomic(const gart_config* cfg, const gart_g
     const float4* rec = reinterpret_cast<const float4*>(pre);
     const float4* lt4 = reinterpret_cast<const float4*>(lt);
     const unsigned blocks = (unsigned)ceil_div(n_rays, 128);
-#define GART_ATOMIC_ARGS <<<blocks, 128, 0, st>>>(rec, slot_of_gid, g->scale, g->quat, g->opacity, ray_off, ray_gid, ray_slot, lt4, dL_dcolor, cf, grad, counts)
+#define GART_ATOMIC_ARGS <<<blocks, 128, 0, st>>>(rec, slot_of_gid, g->scale, g->quat, g->opacity, ray_off, ray_gid, ray_slot, lt4, dL_dcolor, cf, grad, counts, kernel_degree_is4(cfg->kernel_degree))
 #define GART_ATOMIC(D)                                                             \
     if (cfg->atomic_mode == GART_ATOMIC_VECTOR) bwd_atomic_kernel<D, true> GART_ATOMIC_ARGS; \
     else bwd_atomic_kernel<D, false> GART_ATOMIC_ARGS

@@ -111,7 +111,7 @@ static inline DirAffine make_dir_affine(const CamF& cam) {
 
 // Gradient terms of one hit added to the item's accumulators: geo[0..2] = v, geo[3..8] = Q (xx, yy, zz, xy, xz, yz),
 // geo[9] = sum alpha dL/dalpha, R.acc = dL/dsh against the bare SH polynomials.
-template <int K>
+template <int K, int KD>
 __device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, float wxf, float wyf, ShRegs<K>& R, float* geo, const float4* __restrict__ spix, int pix, const float4 L) {
     const float4 gq = spix[pix];
     const float xf = small_int_to_float((uint32_t)pix & (GM_WIN - 1)), yf = small_int_to_float((uint32_t)pix / GM_WIN);
@@ -135,14 +135,16 @@ __device__ __forceinline__ void gm_hit(const ItemGeo& P, const DirAffine& dir, f
     const float inv_a = fast_rcp(fmaf(dg.x, dg.x, fmaf(dg.y, dg.y, dg.z * dg.z)));
     // y = d_g x (o_g x d_g); x_g = y / |d_g|^2
     const float yx = dg.y * cr.z - dg.z * cr.y, yy = dg.z * cr.x - dg.x * cr.z, yz = dg.x * cr.y - dg.y * cr.x;
-    const float s1 = -0.5f * ad * inv_a, s2 = s1 * inv_a;
+    float s1 = -0.5f * ad * inv_a;
+    if constexpr (KD == 4) s1 *= 2.0f * inv_a * fmaf(cr.x, cr.x, fmaf(cr.y, cr.y, cr.z * cr.z));   // degree-4 kernel: dL/d(D^2) = -D^2 alpha dL/dalpha
+    const float s2 = s1 * inv_a;
     geo[0] = fmaf(s1, yx, geo[0]); geo[1] = fmaf(s1, yy, geo[1]); geo[2] = fmaf(s1, yz, geo[2]);
     const float tx = s2 * yx, ty = s2 * yy, tz = s2 * yz;
     geo[3] = fmaf(tx, yx, geo[3]); geo[4] = fmaf(ty, yy, geo[4]); geo[5] = fmaf(tz, yz, geo[5]);
     geo[6] = fmaf(tx, yy, geo[6]); geo[7] = fmaf(tx, yz, geo[7]); geo[8] = fmaf(ty, yz, geo[8]);
 }
 
-template <int TS, int DEG>
+template <int TS, int DEG, int KD>
 __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(const float4* __restrict__ rec, const float4* __restrict__ qs,
                                                              const uint32_t* __restrict__ gid_of_slot, const uint2* __restrict__ blk_desc,
                                                              const uint32_t* __restrict__ info, const uint32_t* __restrict__ st_off,
@@ -298,10 +300,10 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
                 // two hits per iteration: two independent dependency chains for the scheduler to interleave; the entry
                 // names its pixel
                 if (e + 1 < e_end) {
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L1), L1);
+                    gm_hit<K, KD>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
+                    gm_hit<K, KD>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L1), L1);
                 } else {
-                    gm_hit<K>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
+                    gm_hit<K, KD>(IG, dir, wxf, wyf, R, geo, spix, (int)lt_pix(L0), L0);
                 }
             }
             fence_proxy_async();
@@ -419,12 +421,12 @@ static __global__ void __launch_bounds__(256) gm_fill_kernel(int64_t n, const ui
 }
 
 template <int TS>
-static gart_status launch_gm(int deg, unsigned grid, cudaStream_t st, const float4* rec, const float4* qs, const uint32_t* gid_of_slot,
+static gart_status launch_gm(int deg, bool narrow, unsigned grid, cudaStream_t st, const float4* rec, const float4* qs, const uint32_t* gid_of_slot,
                              const ViewLayout& v, const float4* lt, const float* dL_dC, const CamF& cam, int sup_x, const Gacc& gacc,
                              float4* grad4, uint32_t* counts, uint32_t wait_limit) {
 #define GART_GM(D)                                                                                                                \
     {                                                                                                                            \
-        auto kern = bwd_gm_kernel<TS, D>;                                                                                   \
+        auto kern = narrow ? bwd_gm_kernel<TS, D, 4> : bwd_gm_kernel<TS, D, 2>;                                                   \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GMB_DYN_SMEM) != cudaSuccess) return GART_ERR_CUDA; \
         kern<<<grid, GMB_THREADS, GMB_DYN_SMEM, st>>>(rec, qs, gid_of_slot, v.blk_desc, v.info, v.st_off, v.rk_desc, v.rk_gstart, lt, \
                                                       dL_dC, cam.width, cam.height, make_dir_affine(cam), sup_x, gacc, grad4, counts, wait_limit); \
@@ -456,6 +458,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
                                   workspace, workspace_bytes, stream);
     if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 0) return GART_ERR_INVALID_ARG;                          // the item pass reads 16-byte LT entries (they name their pixel)
+    if (!kernel_degree_ok(cfg->kernel_degree)) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
@@ -481,8 +484,8 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     GART_LAUNCH_CHECK();
     const unsigned grid = (unsigned)v.blocks_cap;
     gart_status s;
-    if (cfg->tile_size == 8) s = launch_gm<8>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
-    else s = launch_gm<16>(g->sh_degree, grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
+    if (cfg->tile_size == 8) s = launch_gm<8>(g->sh_degree, kernel_degree_is4(cfg->kernel_degree), grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
+    else s = launch_gm<16>(g->sh_degree, kernel_degree_is4(cfg->kernel_degree), grid, st, rec, qs, gid_of_slot, v, lt4, dL_dcolor, cf, sup_x, gacc, grad4, counts, wait_limit_of(cfg->wait_polls));
     if (s != GART_OK) return s;
     gm_convert_big_kernel<<<slot_blocks, 256, 0, st>>>(srect, qs, gid_of_slot, gacc, grad4, counts);
     GART_LAUNCH_CHECK();

@@ -248,6 +248,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 1 || cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // this pass reads the 4-byte LT format, tile-major
     if (cfg->max_hits != 0 || cfg->t_min > 0.0f || cfg->alpha_max < 1.0f) return GART_ERR_INVALID_ARG;   // its pixel-centric part re-derives every hit's alpha: no cap, no early end, no clamp
+    if (cfg->kernel_degree != 0 && cfg->kernel_degree != 2) return GART_ERR_INVALID_ARG;                   // ... with the Gaussian response
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;

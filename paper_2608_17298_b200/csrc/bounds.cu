@@ -30,7 +30,7 @@ __device__ __forceinline__ void quat_to_rot(const double w, const double x, cons
 
 __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* __restrict__ mean, const float* __restrict__ scale,
                                                      const float* __restrict__ quat, const float* __restrict__ opacity,
-                                                     CamD cam, double alpha_min, double near_z,
+                                                     CamD cam, double alpha_min, int narrow, double near_z,
                                                      int sup_x, uint32_t key_none,
                                                      int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
                                                      float4* __restrict__ pre4, uint32_t* __restrict__ keys,
@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
         int x0 = 0, y0 = 0, x1 = -1, y1 = -1, c = 0;
         const double sigma = (double)opacity[i];
         if (sigma > alpha_min) {
-            const double alpha_c = sqrt(2.0 * log(sigma / alpha_min));  // Eq. 10
+            const double tau_c = 2.0 * log(sigma / alpha_min);
+            const double alpha_c = narrow ? sqrt(sqrt(tau_c)) : sqrt(tau_c);  // Eq. 10 (fourth root for the degree-4 kernel)
             double R[9];
             quat_to_rot((double)quat[4 * i], (double)quat[4 * i + 1], (double)quat[4 * i + 2], (double)quat[4 * i + 3], R);
             const double s[3] = {(double)scale[3 * i], (double)scale[3 * i + 1], (double)scale[3 * i + 2]};
@@ -294,6 +295,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     if (!cfg || !g || !cam || !counts) return GART_ERR_INVALID_ARG;
     if (g->n < 0 || g->n > 0xfffffff0ll || g->sh_degree < 0 || g->sh_degree > 3) return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
+    if (!kernel_degree_ok(cfg->kernel_degree)) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0 || !(cam->fx > 0.0) || !(cam->fy > 0.0)) return GART_ERR_INVALID_ARG;
     if (g->n > 0 && (!g->mean || !g->scale || !g->quat || !g->opacity || !g->sh || !rect || !cls || !pre || !slot_of_gid || !gid_of_slot))
         return GART_ERR_INVALID_ARG;
@@ -321,7 +323,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     const int threads = 128;
     const int64_t blocks = ceil_div(g->n, threads);
     bounds_kernel<<<(unsigned)blocks, threads, 0, st>>>(g->n, g->mean, g->scale, g->quat, g->opacity, c,
-                                                       (double)cfg->alpha_min, (double)cfg->near_z, sup_x, key_none, rect, cls,
+                                                       (double)cfg->alpha_min, kernel_degree_is4(cfg->kernel_degree) ? 1 : 0, (double)cfg->near_z, sup_x, key_none, rect, cls,
                                                        w.pre_tmp, kbuf[cur], vbuf[cur], counts);
     GART_LAUNCH_CHECK();
     gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);

@@ -121,9 +121,13 @@ struct RayEval {
     float3 cr;     // o_g x d_g
 };
 
+// The configuration's kernel degree: 2 (also for 0) or 4; anything else is refused.
+static inline bool kernel_degree_ok(int32_t k) { return k == 0 || k == 2 || k == 4; }
+static inline bool kernel_degree_is4(int32_t k) { return k == 4; }
+
 // Response of the Gaussian along the ray through the pixel at offset (dx, dy) pixels from the
-// record's reference position.
-__device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy) {
+// record's reference position.  narrow: the degree-4 kernel exp(-D^4 / 2) instead of exp(-D^2 / 2).
+__device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy, bool narrow = false) {
     RayEval r;
     const float ex = fmaf(p.c0.x, dx, p.c1.x * dy);
     const float ey = fmaf(p.c0.y, dx, p.c1.y * dy);
@@ -136,7 +140,7 @@ __device__ __forceinline__ RayEval ray_eval(const PreRec& p, float dx, float dy)
     const float cc = fmaf(r.cr.x, r.cr.x, fmaf(r.cr.y, r.cr.y, r.cr.z * r.cr.z));
     r.inv_a = fast_rcp(a);
     const float D2 = cc * r.inv_a;
-    r.alpha = p.sigma * fast_exp2(-0.72134752044448170f * D2);
+    r.alpha = p.sigma * fast_exp2(-0.72134752044448170f * (narrow ? D2 * D2 : D2));
     r.tnum = fmaf(p.m.x, r.dg.x, fmaf(p.m.y, r.dg.y, p.m.z * r.dg.z));
     return r;
 }

@@ -102,7 +102,7 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
 template <int TS>
 __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4* __restrict__ rec, int rs4, const uint32_t* __restrict__ slot_of_gid,
                                                                    const uint32_t* __restrict__ tile_off,
-                                                                   const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min,
+                                                                   const uint32_t* __restrict__ pair_gid, CamF cam, float alpha_min, bool narrow,
                                                                    uint32_t* __restrict__ pair_mask, uint32_t* __restrict__ pair_sid,
                                                                    const int4* __restrict__ srect, const uint32_t* __restrict__ gpair_off,
                                                                    uint32_t* __restrict__ gm_mask, uint32_t* __restrict__ pair_gpos,
@@ -158,7 +158,9 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
         for (int q = 0; q < MW; ++q) w[q] = 0u;
         if (j < end) {
             const PreRec P = unpack_pre(ra[0], ra[1], ra[2], ra[3], ra[4]);
-            const float tau = 1.3862943611198906f * __log2f(P.sigma * inv_amin);   // 2 ln(sigma / alpha_min)
+            // 2 ln(sigma / alpha_min); the degree-4 kernel reaches alpha_min where D^4 = that, i.e. D^2 = its square root
+            const float tau2 = 1.3862943611198906f * __log2f(P.sigma * inv_amin);
+            const float tau = narrow ? fast_sqrt(fmaxf(tau2, 0.0f)) : tau2;
             const float3 a1 = make_float3(P.c0.y * P.m.z - P.c0.z * P.m.y, P.c0.z * P.m.x - P.c0.x * P.m.z, P.c0.x * P.m.y - P.c0.y * P.m.x);
             const float3 b1 = make_float3(P.c1.y * P.m.z - P.c1.z * P.m.y, P.c1.z * P.m.x - P.c1.x * P.m.z, P.c1.x * P.m.y - P.c1.y * P.m.x);
             // o_g x d_g and d_g at the pixel of the tile nearest to the reference position
@@ -399,7 +401,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ rank_pbase,
-                                                                const uint32_t* __restrict__ ray_off, CamF cam, float alpha_max,
+                                                                const uint32_t* __restrict__ ray_off, CamF cam, float alpha_max, bool narrow,
                                                                 float4* __restrict__ recs, uint32_t* __restrict__ counts) {
     constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, PF4 = (20 + SW + 3) / 4;
     constexpr int PSTR = PF4 | 1;   // odd lane stride: the lanes' 16-byte reads fall into distinct banks
@@ -478,7 +480,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         auto hit = [&](const int p, const uint32_t slot_e) {
             const float4 pa = spix_lane[EvalPix<TS>::index(p, 0, 0)], pb = spix_lane[EvalPix<TS>::index(p, 1, 0)];
             const uint32_t pos = atomicAdd(&scur[p], 1u);
-            const RayEval r = ray_eval(P, (fbx + pa.w) - P.rx, (fby + pb.x) - P.ry);   // small integers: the sums are exact
+            const RayEval r = ray_eval(P, (fbx + pa.w) - P.rx, (fby + pb.x) - P.ry, narrow);   // small integers: the sums are exact
             const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
             float B[K];
             sh_poly<K>(make_float3(pa.x, pa.y, pa.z), B);
@@ -1016,14 +1018,14 @@ template <int TS, bool GMAJ>
 static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                const uint32_t* tile_lt_base, const uint32_t* rank_pbase, const uint32_t* ray_off,
-                               const CamF& cam, float alpha_max, const ForwardWs& w, uint32_t* counts) {
+                               const CamF& cam, float alpha_max, bool narrow, const ForwardWs& w, uint32_t* counts) {
 #define GART_EVAL(D)                                                                                                        \
     {                                                                                                                      \
         auto kern = fwd_eval_kernel<TS, D, GMAJ>;                                                                          \
         constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
         kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, rank_pbase, ray_off, cam, \
-                                            alpha_max, w.recs, counts);                                                               \
+                                            alpha_max, narrow, w.recs, counts);                                                               \
     }
     switch (deg) {
         case 0: GART_EVAL(0); break;
@@ -1093,7 +1095,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (!cfg || !g || !cam || !tile_off || !color || !t_final || !hit_count || !ray_off || !counts)
         return GART_ERR_INVALID_ARG;
     if (cfg->tile_size != 8 && cfg->tile_size != 16) return GART_ERR_INVALID_ARG;
-    if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0) return GART_ERR_INVALID_ARG;
+    if (cfg->lt_format < 0 || cfg->lt_format > 2 || cfg->max_hits < 0 || !kernel_degree_ok(cfg->kernel_degree)) return GART_ERR_INVALID_ARG;
     if (!(cfg->t_min >= 0.0f) || !(cfg->t_min < 1.0f) || !(cfg->alpha_max > 0.0f)) return GART_ERR_INVALID_ARG;
     if (cfg->lt_layout != GART_LT_PRIMITIVE_MAJOR && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;
     if (cfg->lt_format != 0 && cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // the 4- and 8-byte formats serve the tile-major passes
@@ -1119,6 +1121,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
     gart_status s;
     const float amax = cfg->alpha_max < 1.0f ? cfg->alpha_max : 2.0f;   // (2: no alpha reaches it, the clamp is off)
+    const bool narrow = kernel_degree_is4(cfg->kernel_degree);
 
     // first primitive-major pair position of every slot (the mask kernel files every pair's mask there)
     if (cudaMemsetAsync(v.info, 0, GM_INFO_WORDS * 4, st) != cudaSuccess) return GART_ERR_CUDA;
@@ -1132,8 +1135,8 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     }
 
     uint32_t* const gm_mask = gmaj ? v.gm_mask : nullptr;
-    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
-    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
+    if (ts == 8) fwd_mask_kernel<8><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, narrow, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
+    else fwd_mask_kernel<16><<<T, MASK_WARPS * 32, 0, st>>>(rec, rs4, slot_of_gid, tile_off, pair_gid, cf, cfg->alpha_min, narrow, v.pair_mask, w.pair_sid, srect, v.gpair_off, gm_mask, v.pair_gpos, hit_count, counts);
     GART_LAUNCH_CHECK();
 
     const int sblocks = (int)ceil_div(T, SORT_WARPS);
@@ -1193,11 +1196,11 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     GART_LAUNCH_CHECK();
 
     if (gmaj) {
-        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
-        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
+        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
     } else {
-        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
-        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, w, counts);
+        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
     }
     if (s != GART_OK) return s;
 

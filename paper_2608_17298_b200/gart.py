@@ -49,7 +49,7 @@ class GartError(RuntimeError):
 class _Config(C.Structure):
     _fields_ = [("alpha_min", C.c_float), ("near_z", C.c_float), ("background", C.c_float * 3), ("tile_size", C.c_int32),
                 ("lt_format", C.c_int32), ("max_hits", C.c_int32), ("lt_layout", C.c_int32), ("t_min", C.c_float),
-                ("alpha_max", C.c_float), ("atomic_mode", C.c_int32), ("wait_polls", C.c_int32)]
+                ("alpha_max", C.c_float), ("atomic_mode", C.c_int32), ("wait_polls", C.c_int32), ("kernel_degree", C.c_int32)]
 
 
 class _Camera(C.Structure):
@@ -130,6 +130,7 @@ class Config:
     alpha_max: float = 1.0      # < 1: every hit's alpha is clamped to alpha_max (>= 1: off)
     atomic_mode: int = 0        # gart_backward_atomic: 0 scalar atomicAdd per word, 1 one 16-byte vector reduction per four words
     wait_polls: int = 0         # 0: library limit on a kernel's waits for its own copies; > 0: polls; < 0: every wait gives up (test hook)
+    kernel_degree: int = 2      # k of the response exp(-D^k / 2): 2 the Gaussian (the paper's setting), 4 a narrow kernel
 
     def c(self) -> _Config:
         s = _Config()
@@ -139,6 +140,7 @@ class Config:
         s.lt_layout = int(self.lt_layout)
         s.t_min, s.alpha_max = float(self.t_min), float(self.alpha_max)
         s.wait_polls, s.atomic_mode = int(self.wait_polls), int(self.atomic_mode)
+        s.kernel_degree = int(self.kernel_degree)
         for i in range(3):
             s.background[i] = float(self.background[i])
         return s

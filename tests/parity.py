@@ -137,7 +137,7 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
         # the other outputs of the forward do not depend on the LT layout
         assert np.array_equal(to_np(buf.color), out["color"]) and np.array_equal(u32(to_np(buf.ray_gid))[:H], out["ray_gid"])
         assert np.array_equal(tile["pair_mask"], out["pair_mask"])
-        if cfg.max_hits == 0 and cfg.t_min == 0 and cfg.alpha_max >= 1:   # (the hybrid backward re-derives every alpha in its pixel pass: no cap, early end or clamp)
+        if cfg.max_hits == 0 and cfg.t_min == 0 and cfg.alpha_max >= 1 and cfg.kernel_degree == 2:   # (the hybrid backward re-derives every alpha in its pixel pass: no cap, early end or clamp, Gaussian response)
             # hybrid backward: the forward again with 4-byte LT entries
             cfg_h = dataclasses.replace(cfg_t, lt_format=1)
             G.run_forward(cfg_h, g, cam, buf)
@@ -166,7 +166,7 @@ def run_gpu(scene, cam, cfg: G.Config, dL_dC, cap_pairs=None, cap_hits=None, ato
 def check_maps(scene, cam, cfg: G.Config, gpu):
     """Rectangles, classes and tile lists against the oracle (bit-exact outside the 1e-9 margin)."""
     osc = orc.OracleScene.from_scene(scene)
-    rect, cls, margin = orc.bounds(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32)
+    rect, cls, margin = orc.bounds(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, kernel_degree=cfg.kernel_degree)
     safe = margin > 1e-9
     assert safe.mean() > 0.999
     assert np.array_equal(gpu["cls"][safe], cls[safe])
@@ -437,7 +437,7 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     colour, t_final, gradient, gradient conditioning and statistics."""
     n_rays = cam.width * cam.height
     sel = np.arange(n_rays) if pixel_mask is None else np.nonzero(pixel_mask.reshape(-1))[0]
-    v = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background)
+    v = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, kernel_degree=cfg.kernel_degree)
     v.find_hits(mode, pixel_mask)
     o_off, o_gid, o_t, o_alpha = v.hits()
     g_off, g_gid = gpu["ray_off"].astype(np.int64), gpu["ray_gid"]
@@ -476,7 +476,7 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     assert stats["band_hit"] + stats["band_order"] <= max(2, 1e-3 * stats["oracle_hits"])
     # replay the GPU's lists
     v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits,
-                  t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0)
+                  t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0, kernel_degree=cfg.kernel_degree)
     v2.set_hits(g_new_off, g_sel_gid)
     color, t_final, cnt = v2.composite()
     stats["margin_t_min"], stats["margin_alpha_max"] = v2.margins()

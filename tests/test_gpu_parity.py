@@ -85,7 +85,7 @@ def option_band(scene, cam, cfg):
     hits' entries by a whole term.  The tests give such rays a zero upstream gradient and leave their colour unchecked (at
     most a few per thousand); on every other ray the decisions are then required to be the oracle's."""
     v = orc.View(orc.OracleScene.from_scene(scene), cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, max_hits=cfg.max_hits,
-                 t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0)
+                 t_min=cfg.t_min_f32, alpha_max=cfg.alpha_max_f32 if cfg.alpha_max < 1.0 else 1.0, kernel_degree=cfg.kernel_degree)
     v.find_hits()
     v.composite()
     return (v.ray_margins() < OPTION_BAND).any(axis=1)
@@ -163,7 +163,7 @@ def test_hit_cap(m):
 @pytest.mark.parametrize("seed", [101, 102, 103, 104, 105, 106])
 def test_random_configurations(seed):
     """Random combinations of image size (ragged against both tile sizes), field of view, SH degree, tile size, background,
-    alpha_min, hit cap, early termination and alpha clamp on a random cluster, every ray and every backward variant against the oracle."""
+    alpha_min, hit cap, early termination, alpha clamp and kernel degree on a random cluster, every ray and every backward variant against the oracle."""
     rng = np.random.default_rng(seed)
     deg = int(rng.integers(0, 4))
     width, height = int(rng.integers(40, 150)), int(rng.integers(30, 110))
@@ -175,6 +175,7 @@ def test_random_configurations(seed):
     cfg = G.Config(tile_size=int(rng.choice([8, 16])), background=tuple(float(v) for v in rng.uniform(0, 1, 3)),
                    alpha_min=float(rng.choice([1.0 / 255.0, 0.01, 0.03])), max_hits=int(rng.choice([0, 0, 3, 17])))
     cfg.t_min, cfg.alpha_max = float(rng.choice([0.0, 0.0, 0.03, 0.2])), float(rng.choice([1.0, 1.0, 0.95, 0.6]))
+    cfg.kernel_degree = int(np.random.default_rng([seed, 7]).choice([2, 2, 4]))   # (a stream of its own: the other draws stay what they were)
     gpu, ref = full_parity(scene, cam, cfg, g=gs.upstream_gradient(cam, seed))
     assert gpu["counts"][G.CNT_HITS] > 100
 
@@ -229,6 +230,22 @@ def test_alpha_clamp():
     assert np.abs(gpu["color"] - free["color"]).max() > 1e-3 and np.all(gpu["t_final"] >= free["t_final"] - 1e-7)
     # both options with a cap, on the tile-major passes too (full_parity runs every variant)
     full_parity(scene, cam, G.Config(alpha_max=a_max, max_hits=9, tile_size=16))
+
+
+@pytest.mark.parametrize("ts", [8, 16])
+def test_narrow_kernel(ts):
+    """kernel_degree = 4: response exp(-D^4 / 2).  Rectangles (clamping radius tau^(1/4)), hit lists, colour, LT entries and the
+    gradients of every backward pass that takes the option follow the oracle's; the footprints shrink, the hybrid pass refuses."""
+    scene, cams = gs.config_cluster(n=4000, width=120, height=96, seed=27)
+    cam = cams[0]
+    cfg = G.Config(kernel_degree=4, tile_size=ts, background=(0.1, 0.2, 0.3))
+    gpu, ref = full_parity(scene, cam, cfg)
+    free, _ = full_parity(scene, cam, G.Config(tile_size=ts, background=(0.1, 0.2, 0.3)))
+    assert 0 < gpu["counts"][G.CNT_PAIRS] < free["counts"][G.CNT_PAIRS] and 0 < gpu["counts"][G.CNT_HITS] < free["counts"][G.CNT_HITS]
+    assert np.abs(gpu["color"] - free["color"]).max() > 1e-3
+    assert "grad_hybrid" not in gpu and "grad_hybrid" in free
+    # with the options of the other compromises too
+    full_parity(scene, cam, G.Config(kernel_degree=4, tile_size=ts, alpha_max=0.9, max_hits=12))
 
 
 @pytest.mark.parametrize("ts", [8, 16])
@@ -534,6 +551,9 @@ def test_invalid_arguments_return_status():
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, t_min=0.01)),
         (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, alpha_max=0.99)),
         (G.run_backward_hybrid, G.Config(lt_format=0, lt_layout=TM)),
+        (G.run_backward_hybrid, G.Config(lt_format=1, lt_layout=TM, kernel_degree=4)),   # its pixel pass knows the Gaussian response only
+        (G.run_backward_tile, G.Config(kernel_degree=3)),             # the library builds the degrees 2 and 4
+        (G.run_backward, G.Config(lt_layout=PM, kernel_degree=6)),
     ]
     for fn, cfg_bad in refused:
         with pytest.raises(G.GartError) as e:
@@ -541,7 +561,7 @@ def test_invalid_arguments_return_status():
         assert e.value.status == 1, (fn.__name__, cfg_bad)
     for cfg_bad in (G.Config(max_hits=-1), G.Config(lt_format=3), G.Config(lt_layout=2), G.Config(lt_format=1, lt_layout=G.LT_PRIMITIVE_MAJOR),
                     G.Config(lt_format=2, lt_layout=G.LT_PRIMITIVE_MAJOR),
-                    G.Config(t_min=1.0), G.Config(t_min=-0.1), G.Config(alpha_max=0.0)):   # (refused by gart_forward)
+                    G.Config(t_min=1.0), G.Config(t_min=-0.1), G.Config(alpha_max=0.0), G.Config(kernel_degree=3)):   # (refused by gart_forward)
         with pytest.raises(G.GartError) as e:
             G.run_forward(cfg_bad, g, cam, buf)
         assert e.value.status == 1, cfg_bad
