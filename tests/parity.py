@@ -447,8 +447,10 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
     # fast path: concatenate selected lists and compare wholesale
     g_new_off, g_sel_gid = _lists_for(gpu["ray_off"].astype(np.int64), g_gid, sel)
     identical = np.array_equal(g_cnt, o_cnt) and np.array_equal(g_sel_gid, o_gid)
+    band_bound = {}      # ray -> bound on what its guard-band decisions can move its colour by (see below)
     if not identical:
         amin = cfg.alpha_min_f32
+        cb = 0.5 + np.abs(osc.sh).max(axis=2).sum(axis=1)      # |colour| of a Gaussian is at most this (|Y_k| <= 1)
         for k, r in enumerate(sel):
             gl = g_gid[g_off[r]:g_off[r + 1]]
             ol = o_gid[o_off[r]:o_off[r + 1]]
@@ -460,6 +462,8 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
                 assert abs(np.log(alpha / amin)) < BAND_HIT or (alpha >= amin and abs(t) < 1e-6), \
                     ("hit decision differs outside the guard band", int(r), int(gid), alpha, t)
                 stats["band_hit"] += 1
+                # a hit more or less moves the colour by T alpha (c - colour behind): at most alpha (|c| + largest colour)
+                band_bound[int(r)] = band_bound.get(int(r), 0.0) + alpha * (cb[gid] + max(cb[gl].max(initial=0.0), float(np.max(np.abs(cfg.background)))))
             # order of the GPU list must be non-decreasing in float64 t* up to the band
             ts_ = np.array([v.eval_pair(int(r), int(gid))[1] for gid in gl])
             if ts_.size > 1:
@@ -472,7 +476,26 @@ def check_hits_and_replay(osc, cam, cfg: G.Config, gpu, dL_dC, pixel_mask=None, 
                 common = [x for x in gl.tolist() if x in os_]
                 common_o = [x for x in ol.tolist() if x in gs]
                 stats["band_order"] += int(common != common_o)
+                if common != common_o:
+                    # two hits composited the other way round move the colour by T alpha_i alpha_j (c_i - c_j)
+                    pos_o = {x: i for i, x in enumerate(common_o)}
+                    al = {int(x): v.eval_pair(int(r), int(x))[0] for x in common}
+                    b = 0.0
+                    for i in range(len(common)):
+                        for j in range(i + 1, len(common)):
+                            if pos_o[common[i]] > pos_o[common[j]]:
+                                b += al[common[i]] * al[common[j]] * (cb[common[i]] + cb[common[j]])
+                    band_bound[int(r)] = band_bound.get(int(r), 0.0) + b
     stats["identical_lists"] = bool(identical)
+    stats["band_rays"] = len(band_bound)
+    if band_bound and cfg.max_hits == 0 and cfg.t_min == 0 and cfg.alpha_max >= 1:
+        # On the rays with a guard-band decision the GPU's colour is also held against the colour of the oracle's OWN lists,
+        # within what those decisions can move it by (the replay below checks the arithmetic on the GPU's lists).
+        own, _, _ = v.composite()
+        own = own.reshape(-1, 3)
+        gcol = gpu["color"].reshape(-1, 3).astype(np.float64)
+        for r, b in band_bound.items():
+            assert np.all(np.abs(gcol[r] - own[r]) <= b + 1e-4 * np.abs(own[r]) + 1e-6), ("banded ray moved further than its decisions allow", r, gcol[r], own[r], b)
     assert stats["band_hit"] + stats["band_order"] <= max(2, 1e-3 * stats["oracle_hits"])
     # replay the GPU's lists
     v2 = orc.View(osc, cam, alpha_min=cfg.alpha_min_f32, near=cfg.near_f32, bg=cfg.background, max_hits=cfg.max_hits,
