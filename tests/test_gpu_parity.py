@@ -434,7 +434,7 @@ def test_unbounded1m_sampled():
 def test_unbounded6m_sampled():
     """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles)."""
     scene, cams = gs.config_unbounded_6m()
-    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=110, n_tiles=22, n_large=5, large_max_area=15000)
+    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=90, n_tiles=18, n_large=5, large_max_area=15000)
     assert gpu["counts"][G.CNT_HITS] > 1e8
 
 
