@@ -97,6 +97,18 @@ __device__ __forceinline__ uint32_t row_hits(const RowQuad& q, bool regular, flo
     return bits;
 }
 
+// Transpose of the 32 x 32 bit matrix whose row l is lane l's word x: the result's bit i is bit `lane` of lane i's x.
+// Five exchanges of half-blocks with the lane 16, 8, 4, 2, 1 away.
+__device__ __forceinline__ uint32_t warp_transpose_bits(uint32_t x, int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const uint32_t m = s == 16 ? 0x0000FFFFu : s == 8 ? 0x00FF00FFu : s == 4 ? 0x0F0F0F0Fu : s == 2 ? 0x33333333u : 0x55555555u;
+        const uint32_t y = __shfl_xor_sync(0xffffffffu, x, s);
+        x = (lane & s) ? (((y >> s) & m) | (x & ~m)) : ((x & m) | ((y & m) << s));
+    }
+    return x;
+}
+
 // Block per tile, thread per (tile, Gaussian) pair: row by row the interval of hit columns -> the pair's mask.
 // Hits per pixel: a shared-memory counter per pixel.
 template <int TS>
@@ -118,6 +130,9 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
     const uint32_t begin = tile_off[tile], end = tile_off[tile + 1];
     for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) scnt[p] = 0u;
     __syncthreads();
+    uint32_t pcnt[MW];   // hits of pixel 32 q + lane among the pairs this warp has seen
+#pragma unroll
+    for (int q = 0; q < MW; ++q) pcnt[q] = 0u;
     const float inv_amin = 1.0f / alpha_min;
     // the chain pair -> Gaussian -> slot -> record is three dependent loads: slot ids run two iterations ahead,
     // records one
@@ -201,20 +216,18 @@ __global__ void __launch_bounds__(MASK_WARPS * 32) fwd_mask_kernel(const float4*
                 pair_gpos[j] = gpa;
             }
         }
-        // hits per pixel: one shared-memory increment per hit
+        // hits per pixel: the warp's 32 masks are a 32 x 32 bit matrix per mask word (row = pair); transposed, lane b holds
+        // the column of pixel 32 q + b, whose population count is the number of this iteration's pairs that hit the pixel
+        // (a loop of one shared-memory increment per hit ran as long as the warp's largest pair and took half the kernel)
 #pragma unroll
-        for (int q = 0; q < MW; ++q) {
-            uint32_t m = w[q];
-            while (m) {
-                const int b = __ffs((int)m) - 1;
-                m &= m - 1u;
-                atomicAdd(&scnt[q * 32 + b], 1u);
-            }
-        }
+        for (int q = 0; q < MW; ++q) pcnt[q] += __popc(warp_transpose_bits(w[q], lane));
 #pragma unroll
         for (int q = 0; q < 5; ++q) ra[q] = rb[q];
         gpa = gpb;
     }
+#pragma unroll
+    for (int q = 0; q < MW; ++q)
+        if (pcnt[q]) atomicAdd(&scnt[q * 32 + lane], pcnt[q]);
     __syncthreads();
     uint32_t m = 0;
     for (int p = threadIdx.x; p < NT; p += MASK_WARPS * 32) {
