@@ -185,9 +185,10 @@ int32_t gart_mask_words(int32_t tile_size);
  *   cls    [n]   uint8 out: 0 culled (sigma <= alpha_min, or support entirely at depth <= near_z),
  *                1 in front of the near plane, 2 straddling it (rectangle = whole image unless
  *                the bounding sphere is outside a side plane of the frustum).
- *   pre    [n * gart_pre_words(sh_degree)] fp32 out: per slot, the evaluation record followed by a copy
- *                of its SH coefficients (times the basis constants), and behind all records quaternion, scale,
- *                opacity and the rectangle in slot order; contents are private to the library.
+ *   pre    [n * gart_pre_words(sh_degree)] fp32 out: per slot, the 80-byte evaluation record, and behind all
+ *                records quaternion, scale, opacity and the rectangle in slot order; contents are private to the
+ *                library.  (The SH coefficients are not copied: gart_forward and gart_backward_hybrid read them
+ *                from g->sh by Gaussian id, so g->sh must stay valid, unchanged and 16-byte aligned for the view.)
  *   slot_of_gid [n] uint32 out: slot of every Gaussian, 0xffffffff if it has none.
  *   gid_of_slot [n] uint32 out: the inverse (first V entries; 0xffffffff beyond).
  *   counts [GART_COUNTS_WORDS] uint32 out: zeroed, then VISIBLE and STRADDLE are set.
@@ -273,7 +274,8 @@ gart_status gart_view_array(int64_t n, int32_t width, int32_t height, int32_t ti
  * For every pixel ray and every Gaussian of its tile list: t* = -(o_g.d_g)/(d_g.d_g),
  * alpha = sigma exp(-|o_g + t* d_g|^2 / 2); a hit iff alpha >= alpha_min and t* > 0.  Hits of a
  * ray are ordered by (t*, id) and composited front to back, C = sum T_i alpha_i c_i + T_final bg,
- * c_i = max(0, 0.5 + sum_k Y_k(d) sh_ik).
+ * c_i = max(0, 0.5 + sum_k Y_k(d) sh_ik).  The coefficients sh_ik are read from g->sh (device memory, by Gaussian id,
+ * 16-byte aligned: INVALID_ARG otherwise); everything else of a Gaussian comes from `pre`.
  *   color      [H,W,3] out;  t_final [H,W] out;  hit_count [H,W] uint32 out.
  *   lt         [cap_hits,4] out: per hit, with w = T alpha its blending weight (T the transmittance
  *              in front of it), c its clamped colour and B the colour composited BEHIND it

@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(BWD_THREADS, 4) bwd_pairs_kernel(const float4*
     constexpr int CH = BWD_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage
     // evaluation record of a lane's Gaussian (the first 5 float4 of the slot's record), staged through shared
     // memory one group ahead
-    constexpr int PF4 = BWD_PF4, RS4 = (20 + SW + 3) / 4;
+    constexpr int PF4 = BWD_PF4, RS4 = REC_F4;
     constexpr int PSTR = PF4;       // lane stride in the buffer, odd: the lanes' 16-byte reads fall into distinct banks
     extern __shared__ __align__(128) float4 dyn[];   // [warp][2][BWD_STAGE_F4] LT stages, then [warp][32][5] evaluation records
     __shared__ __align__(16) float4 spix[PIXF4];
@@ -380,7 +380,7 @@ extern "C" gart_status gart_backward_tile(const gart_config* cfg, const gart_gau
     else s = cfg->tile_size == 8 ? GART_PAIRS_TS(8, 2) : GART_PAIRS_TS(16, 2);
 #undef GART_PAIRS_TS
     if (s != GART_OK) return s;
-    const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);   // per slot: quaternion, scale, opacity (behind the records)
+    const float4* qs = rec + (size_t)g->n * REC_F4;   // per slot: quaternion, scale, opacity (behind the records)
     return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);
 }
 
@@ -410,7 +410,7 @@ __global__ void __launch_bounds__(BWD_THREADS) bwd_pairs_warp_kernel(const float
                                                                      const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ tile_lt_base,
                                                                      const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
                                                                      Gacc gacc, const uint32_t* __restrict__ counts, const bool narrow) {
-    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int NT = TS * TS, MW = NT / 32, K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = REC_F4;
     constexpr int AW = (11 + SW + 3) & ~3;
     __shared__ __align__(16) float4 spix[NT * 2];   // (d, u), (g, v) per pixel, one copy: the lanes of a warp read different pixels
     if (counts[GART_CNT_ERROR]) return;
@@ -525,6 +525,6 @@ extern "C" gart_status gart_backward_warp(const gart_config* cfg, const gart_gau
     }
 #undef GART_WARP
     GART_LAUNCH_CHECK();
-    const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);
+    const float4* qs = rec + (size_t)g->n * REC_F4;
     return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);
 }

@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(128) bwd_atomic_kernel(const float4* __restric
                                                          const uint32_t* __restrict__ ray_gid, const uint32_t* __restrict__ ray_slot,
                                                          const float4* __restrict__ lt, const float* __restrict__ dL_dC, CamF cam,
                                                          float* __restrict__ grad, const uint32_t* __restrict__ counts, const bool narrow) {
-    constexpr int K = (DEG + 1) * (DEG + 1), RS4 = (20 + 3 * K + 3) / 4;
+    constexpr int K = (DEG + 1) * (DEG + 1), RS4 = REC_F4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (ray >= (int64_t)cam.width * cam.height) return;

@@ -154,7 +154,7 @@ __global__ void __launch_bounds__(GMB_THREADS, GMB_MIN_BLOCKS) bwd_gm_kernel(con
                                                              int sup_x, Gacc gacc,
                                                              float4* __restrict__ grad4, uint32_t* __restrict__ counts,
                                                              const uint32_t wait_limit) {
-    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = REC_F4;
     constexpr int AW = (11 + SW + 3) & ~3;                 // accumulator words, multiple of 4
     constexpr int EB = 16;                                 // bytes per LT entry
     constexpr int CH = GMB_STAGE_F4 * 16 / (32 * EB);      // entries per lane and per stage (even)
@@ -472,7 +472,7 @@ extern "C" gart_status gart_backward(const gart_config* cfg, const gart_gaussian
     const CamF cf = make_camf(cam, cfg->tile_size);
     const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
     const float4* rec = reinterpret_cast<const float4*>(pre);
-    const int rs4 = rec_f4(g->sh_degree);
+    const int rs4 = REC_F4;
     const float4* qs = rec + (size_t)g->n * rs4;                                         // per slot: quaternion, scale, opacity
     const int4* srect = reinterpret_cast<const int4*>(rec + (size_t)g->n * (rs4 + 2));   // per slot: rectangle
     const float4* lt4 = reinterpret_cast<const float4*>(lt);

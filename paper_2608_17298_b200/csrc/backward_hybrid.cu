@@ -157,11 +157,11 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
 // One thread per ray; per hit three 16-byte vector reductions on the moments of the Gaussian's accumulation record
 // (v, Q, sum alpha dL/dalpha: the same record that the primitive-centric pass fills, converted afterwards).
 template <int DEG>
-__global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ slot_of_gid,
+__global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const float* __restrict__ sh, const uint32_t* __restrict__ slot_of_gid,
                                                             const uint32_t* __restrict__ ray_off, const uint32_t* __restrict__ ray_gid,
                                                             const float* __restrict__ dL_dC, CamF cam, float bg0, float bg1, float bg2,
                                                             Gacc gacc, const uint32_t* __restrict__ counts) {
-    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = (20 + SW + 3) / 4;
+    constexpr int K = (DEG + 1) * (DEG + 1), SW = 3 * K, RS4 = REC_F4;
     if (counts[GART_CNT_ERROR]) return;
     const int64_t ray = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (ray >= (int64_t)cam.width * cam.height) return;
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
     if (b == e) return;
     const int x = (int)(ray % cam.width), y = (int)(ray / cam.width);
     float B[K];
-    sh_poly<K>(pixel_dir(cam, x, y), B);   // the records' SH coefficients carry the basis constants
+    sh_basis<K>(pixel_dir(cam, x, y), B);   // (with the basis constants: the coefficients come straight from the caller's array)
     const float3 g = make_float3(dL_dC[3 * ray], dL_dC[3 * ray + 1], dL_dC[3 * ray + 2]);
     const uint64_t pol_keep = l2_policy_evict_last();
     // front to back: log of the final transmittance
@@ -182,25 +182,18 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
     // back to front
     float cb0 = bg0, cb1 = bg1, cb2 = bg2;
     for (uint32_t h = e; h-- > b;) {
-        const uint32_t sid = __ldg(slot_of_gid + ray_gid[h]);
+        const uint32_t gid = ray_gid[h];
+        const uint32_t sid = __ldg(slot_of_gid + gid);
         const float4* rp = rec + (size_t)sid * RS4;
         const PreRec P = load_pre(rp);
         const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
         float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
+        const float* sp = sh + (size_t)gid * SW;
 #pragma unroll
-        for (int q = 0; q < (SW + 3) / 4; ++q) {
-            const float4 t = __ldg(rp + 5 + q);
-            const float sv[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int wd = 4 * q + i;
-                if (wd < SW) {
-                    const float term = B[wd / 3] * sv[i];
-                    if (wd % 3 == 0) c0 += term;
-                    else if (wd % 3 == 1) c1 += term;
-                    else c2 += term;
-                }
-            }
+        for (int k = 0; k < K; ++k) {
+            c0 = fmaf(B[k], __ldg(sp + 3 * k), c0);
+            c1 = fmaf(B[k], __ldg(sp + 3 * k + 1), c1);
+            c2 = fmaf(B[k], __ldg(sp + 3 * k + 2), c2);
         }
         c0 = fmaxf(c0, 0.0f); c1 = fmaxf(c1, 0.0f); c2 = fmaxf(c2, 0.0f);
         logT -= log1pf(-r.alpha);                       // log of the transmittance in front of this hit
@@ -249,7 +242,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     if (cfg->lt_format != 1 || cfg->lt_layout != GART_LT_TILE_MAJOR) return GART_ERR_INVALID_ARG;   // this pass reads the 4-byte LT format, tile-major
     if (cfg->max_hits != 0 || cfg->t_min > 0.0f || cfg->alpha_max < 1.0f) return GART_ERR_INVALID_ARG;   // its pixel-centric part re-derives every hit's alpha: no cap, no early end, no clamp
     if (cfg->kernel_degree != 0 && cfg->kernel_degree != 2) return GART_ERR_INVALID_ARG;                   // ... with the Gaussian response
-    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0) return GART_ERR_INVALID_ARG;
+    if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || (g->n > 0 && !g->sh)) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0) return GART_ERR_INVALID_ARG;
     if (g->n == 0) return GART_OK;
     if (!grad || !pre || !slot_of_gid || !gid_of_slot || !lt_w || !ray_gid || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
@@ -271,7 +264,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     const int64_t n_rays = (int64_t)cam->width * cam->height;
     const unsigned blocks = (unsigned)ceil_div(n_rays, 128);
     const float* bg = cfg->background;
-#define GART_GEO(D) bwd_pixel_geo_kernel<D><<<blocks, 128, 0, st>>>(rec, slot_of_gid, ray_off, ray_gid, dL_dcolor, cf, bg[0], bg[1], bg[2], gacc, counts)
+#define GART_GEO(D) bwd_pixel_geo_kernel<D><<<blocks, 128, 0, st>>>(rec, g->sh, slot_of_gid, ray_off, ray_gid, dL_dcolor, cf, bg[0], bg[1], bg[2], gacc, counts)
     switch (g->sh_degree) {
         case 0: GART_GEO(0); break;
         case 1: GART_GEO(1); break;
@@ -280,6 +273,6 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     }
 #undef GART_GEO
     GART_LAUNCH_CHECK();
-    const float4* qs = rec + (size_t)g->n * rec_f4(g->sh_degree);
+    const float4* qs = rec + (size_t)g->n * REC_F4;
     return launch_finalize(g->n, qs, slot_of_gid, gid_of_slot, gacc, grad, counts, st);
 }

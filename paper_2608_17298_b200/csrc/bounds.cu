@@ -168,24 +168,15 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
     }
 }
 
-// One thread per 16 bytes of a slot's record: 5 float4 of the evaluation record, then the SH
-// coefficients (zero padded to the record stride).  Also fills the two maps between ids and slots.
-__constant__ float c_sh_norm[16] = {sh_norm(0), sh_norm(1), sh_norm(2), sh_norm(3), sh_norm(4), sh_norm(5), sh_norm(6), sh_norm(7),
-                                    sh_norm(8), sh_norm(9), sh_norm(10), sh_norm(11), sh_norm(12), sh_norm(13), sh_norm(14), sh_norm(15)};
-
+// One thread per 16 bytes of a slot's evaluation record (5 float4).  Also fills the two maps between ids and slots.
 constexpr int GATHER_UNROLL = 2;
 
-template <int DEG>
 __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
-                                                             const float4* __restrict__ pre_tmp, const float* __restrict__ sh,
-                                                             const int4* __restrict__ rect,
+                                                             const float4* __restrict__ pre_tmp, const int4* __restrict__ rect,
                                                              float4* __restrict__ rec, float4* __restrict__ qs, int4* __restrict__ srect,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
-    constexpr uint32_t SW = 3 * (DEG + 1) * (DEG + 1), RS4 = (20 + SW + 3) / 4;   // (compile-time: the divisions below are multiplications)
-    __shared__ float s_norm[16];   // lanes index it divergently: shared memory, not the constant bank
-    if (threadIdx.x < 16) s_norm[threadIdx.x] = c_sh_norm[threadIdx.x];
-    __syncthreads();
+    constexpr uint32_t RS4 = REC_F4;   // (compile-time: the divisions below are multiplications)
     // GATHER_UNROLL pieces per thread, their loads issued together (the chain id -> record otherwise leaves too few bytes in flight)
     uint32_t slot[GATHER_UNROLL], q[GATHER_UNROLL], gid[GATHER_UNROLL];
     bool vis[GATHER_UNROLL];
@@ -206,21 +197,7 @@ __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_
 #pragma unroll
     for (int u = 0; u < GATHER_UNROLL; ++u) {
         v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (!vis[u]) continue;
-        if (q[u] < 5) {
-            v[u] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + q[u]];
-        } else {
-            const uint32_t e = (q[u] - 5) * 4;
-            const float* sp = sh + (size_t)gid[u] * SW;
-            if (SW % 4 == 0) {
-                v[u] = __ldg(reinterpret_cast<const float4*>(sp + e));
-            } else {
-                v[u].x = e < SW ? sp[e] : 0.0f;
-                v[u].y = e + 1 < SW ? sp[e + 1] : 0.0f;
-                v[u].z = e + 2 < SW ? sp[e + 2] : 0.0f;
-                v[u].w = e + 3 < SW ? sp[e + 3] : 0.0f;
-            }
-        }
+        if (vis[u]) v[u] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + q[u]];
     }
 #pragma unroll
     for (int u = 0; u < GATHER_UNROLL; ++u) {
@@ -230,14 +207,6 @@ __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_
             qs[2 * (size_t)slot[u] + 1] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 6];
         }
         if (q[u] == 2) srect[slot[u]] = rect[gid[u]];   // the rectangle in slot order
-        if (q[u] >= 5) {
-            // scaled by the basis function's normalisation constant: the forward evaluates the bare polynomials
-            const uint32_t e = (q[u] - 5) * 4;
-            v[u].x *= e < SW ? s_norm[e / 3] : 0.0f;
-            v[u].y *= e + 1 < SW ? s_norm[(e + 1) / 3] : 0.0f;
-            v[u].z *= e + 2 < SW ? s_norm[(e + 2) / 3] : 0.0f;
-            v[u].w *= e + 3 < SW ? s_norm[(e + 3) / 3] : 0.0f;
-        }
         rec[(size_t)slot[u] * RS4 + q[u]] = v[u];
     }
 }
@@ -282,9 +251,9 @@ extern "C" const char* gart_status_string(gart_status s) {
 
 extern "C" int32_t gart_mask_words(int32_t tile_size) { return tile_size * tile_size / 32; }
 
-// Per Gaussian: the slot record (evaluation record + SH coefficients, padded to 16 bytes); in a second
-// block behind all records, 8 words (quaternion, scale, opacity) in slot order; in a third, the rectangle.
-extern "C" int32_t gart_pre_words(int32_t sh_degree) { return 4 * gart::rec_f4(sh_degree) + 8 + 4; }
+// Per Gaussian: the slot's evaluation record (20 words); in a second block behind all records, 8 words (quaternion, scale,
+// opacity) in slot order; in a third, the rectangle.  (The same for every SH degree: the coefficients are read in place.)
+extern "C" int32_t gart_pre_words(int32_t sh_degree) { (void)sh_degree; return 4 * gart::REC_F4 + 8 + 4; }
 
 extern "C" size_t gart_bounds_workspace_bytes(int64_t n) { return gart::bounds_layout(nullptr, n).bytes; }
 
@@ -328,21 +297,13 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     GART_LAUNCH_CHECK();
     gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);
     if (s != GART_OK) return s;
-    const int rs4 = rec_f4(g->sh_degree);
+    const int rs4 = REC_F4;
     const int64_t gthreads = g->n * rs4;
-    if (gthreads >= (int64_t)1 << 32) return GART_ERR_INVALID_ARG;   // (n beyond 1e8 at SH degree 3: 32-bit thread indices)
+    if (gthreads >= (int64_t)1 << 32) return GART_ERR_INVALID_ARG;   // (32-bit thread indices)
     float4* rec_out = reinterpret_cast<float4*>(pre);
-#define GART_GATHER(D)                                                                                                                        \
-    gather_records_kernel<D><<<(unsigned)ceil_div(gthreads, 256 * GATHER_UNROLL), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp, g->sh, \
-                                                                                reinterpret_cast<const int4*>(rect), rec_out, rec_out + (size_t)g->n * rs4,        \
-                                                                                reinterpret_cast<int4*>(rec_out + (size_t)g->n * (rs4 + 2)), slot_of_gid, gid_of_slot)
-    switch (g->sh_degree) {
-        case 0: GART_GATHER(0); break;
-        case 1: GART_GATHER(1); break;
-        case 2: GART_GATHER(2); break;
-        default: GART_GATHER(3); break;
-    }
-#undef GART_GATHER
+    gather_records_kernel<<<(unsigned)ceil_div(gthreads, 256 * GATHER_UNROLL), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp,
+                                                                                reinterpret_cast<const int4*>(rect), rec_out, rec_out + (size_t)g->n * rs4,
+                                                                                reinterpret_cast<int4*>(rec_out + (size_t)g->n * (rs4 + 2)), slot_of_gid, gid_of_slot);
     GART_LAUNCH_CHECK();
     return GART_OK;
 }

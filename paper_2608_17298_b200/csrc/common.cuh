@@ -93,9 +93,9 @@ __device__ __forceinline__ PreRec unpack_pre(const float4& a, const float4& b, c
     return p;
 }
 
-// A slot's record: 5 float4 of PreRec, then the 3K SH coefficients (coefficient-major, channel-minor),
-// zero padded to a multiple of 4 floats.  rs4 = float4 per record.
-static inline int rec_f4(int sh_degree) { return ((20 + 3 * (sh_degree + 1) * (sh_degree + 1) + 3) & ~3) / 4; }
+// A slot's record: the 5 float4 of PreRec.  (The SH coefficients are not copied per view: the evaluation reads them from
+// the caller's array by Gaussian id.)
+constexpr int REC_F4 = 5;
 
 __device__ __forceinline__ PreRec load_pre(const float4* __restrict__ rec) {
     return unpack_pre(__ldg(rec), __ldg(rec + 1), __ldg(rec + 2), __ldg(rec + 3), __ldg(rec + 4));
@@ -334,6 +334,9 @@ __device__ __forceinline__ void sh_poly(const float3 d, float* B) {
         }
     }
 }
+__device__ __forceinline__ constexpr float sh_norm(int k);
+// normalisation constant of SH word e = 3 k + channel (1 beyond the 16 basis functions: padding words)
+__device__ __forceinline__ constexpr float sh_norm_word(int e) { return e < 48 ? sh_norm(e / 3) : 0.0f; }
 __device__ __forceinline__ constexpr float sh_norm(int k) {
     return k == 0 ? 0.28209479177387814f
          : k == 1 ? -0.4886025119029199f : k == 2 ? 0.4886025119029199f : k == 3 ? -0.4886025119029199f
@@ -381,6 +384,9 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 // copy, which every lane would have to issue by itself); completion by cp.async.wait_all of the issuing thread.
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // groups of per-thread copies: commit closes the group of the copies issued so far; wait_but_one returns when all groups

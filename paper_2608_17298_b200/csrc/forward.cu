@@ -370,6 +370,7 @@ template <int MW>
 struct EvalDesc {
     PairMask<MW> pm;
     uint32_t sid, gstart;
+    uint32_t gid;     // id of the pair's Gaussian (its SH coefficients are read from the caller's array)
     uint32_t pbase;   // primitive-major layout: window index of the pair's tile origin
     int c;      // hits of this lane's pair
     int cmax;   // hits of the group's first pair (the largest)
@@ -380,6 +381,7 @@ struct EvalDesc {
 template <int MW, bool GMAJ>
 __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restrict__ rank_sid, const uint32_t* __restrict__ rank_mask,
                                                        const uint32_t* __restrict__ rank_gstart, const uint32_t* __restrict__ rank_pbase,
+                                                       const uint32_t* __restrict__ gid_of_slot,
                                                        uint32_t begin, uint32_t n, uint32_t r0, int lane) {
     EvalDesc<MW> d;
     const bool act = r0 < n && r0 + lane < n;
@@ -390,6 +392,7 @@ __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restric
     d.gstart = act ? __ldg(rank_gstart + q) : 0u;
     d.pbase = (GMAJ && act) ? __ldg(rank_pbase + q) : 0u;
     d.cmax = __shfl_sync(0xffffffffu, d.c, 0);
+    d.gid = (act && d.c != 0) ? __ldg(gid_of_slot + d.sid) : 0u;   // (two groups ahead of its use: the chain slot -> id -> coefficients is hidden)
     return d;
 }
 
@@ -410,7 +413,7 @@ struct EvalPix {
 // current group is evaluated.  The colour is 0.5 + sum_k B_k(d) sh'_k with the bare SH polynomials B_k and
 // the record's coefficients sh'_k, which carry the normalisation constants.
 template <int TS, int DEG, bool GMAJ>
-__global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const uint32_t* __restrict__ gid_of_slot,
+__global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __restrict__ rec, const float* __restrict__ sh, const uint32_t* __restrict__ gid_of_slot,
                                                                 const uint32_t* __restrict__ tile_off, const uint32_t* __restrict__ rank_sid,
                                                                 const uint32_t* __restrict__ rank_mask, const uint32_t* __restrict__ rank_gstart,
                                                                 const uint32_t* __restrict__ tile_lt_base, const uint32_t* __restrict__ rank_pbase,
@@ -446,9 +449,13 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
     const float4* spix_lane = spix + (lane & (EvalPix<TS>::COPIES - 1));
     float4* my_par = spar + (size_t)(warp * 32 + lane) * PSTR;
     const uint32_t par_addr = smem_u32(my_par);
-    // Copy the records of a group's 32 Gaussians: LP lanes take the first LP 16-byte pieces of one record (contiguous:
-    // whole sectors per request instead of one request per piece), 32 / LP records per instruction; a lane copies the
-    // pieces beyond LP of its own record.  A lane therefore writes other lanes' buffers: warp barriers around the use.
+    // Copy what the lanes need of a group's 32 Gaussians into the warp's buffers: per lane the 5 float4 of the evaluation
+    // record (by slot) followed by the 3K SH coefficients (from the caller's array, by Gaussian id).  Where a row of
+    // coefficients is a whole number of 16-byte pieces (degrees 1 and 3), LP lanes take the first LP pieces of one lane's
+    // buffer (contiguous sources: whole sectors per request instead of one request per piece), 32 / LP buffers per
+    // instruction, and a lane copies the pieces beyond LP of its own buffer; otherwise (degrees 0 and 2: rows of 12 and 108
+    // bytes) a lane copies its own row word by word.  A lane therefore writes other lanes' buffers: warp barriers around the use.
+    constexpr bool SH16 = SW % 4 == 0;
     constexpr int LP = PF4 <= 8 ? 8 : 16, PPI = 32 / LP;
     const uint32_t warp_par_addr = smem_u32(spar + (size_t)warp * 32 * PSTR);
     auto issue_params = [&](const EvalDesc<MW>& d) {
@@ -458,31 +465,42 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         for (int i = 0; i < 32 / PPI; ++i) {
             const int pair = i * PPI + lane / LP;
             const uint32_t sd = __shfl_sync(0xffffffffu, tag, pair);
-            if (sd != 0xffffffffu && piece < PF4) cp_async16(warp_par_addr + 16u * (uint32_t)(pair * PSTR + piece), rec + (size_t)sd * PF4 + piece);
+            const uint32_t gd = __shfl_sync(0xffffffffu, d.gid, pair);
+            if (sd != 0xffffffffu && piece < (SH16 ? PF4 : REC_F4)) {
+                const void* src = piece < REC_F4 ? reinterpret_cast<const void*>(rec + (size_t)sd * REC_F4 + piece)
+                                                 : reinterpret_cast<const void*>(sh + (size_t)gd * SW + 4 * (piece - REC_F4));
+                cp_async16(warp_par_addr + 16u * (uint32_t)(pair * PSTR + piece), src);
+            }
         }
         if (d.c != 0) {
-            const float4* src = rec + (size_t)d.sid * PF4;
+            if constexpr (SH16) {
 #pragma unroll
-            for (int q = LP; q < PF4; ++q) cp_async16(par_addr + 16u * q, src + q);
+                for (int q = LP; q < PF4; ++q) cp_async16(par_addr + 16u * q, sh + (size_t)d.gid * SW + 4 * (q - REC_F4));
+            } else {
+                const float* src = sh + (size_t)d.gid * SW;
+#pragma unroll
+                for (int e = 0; e < SW; ++e) cp_async4(par_addr + 4u * (uint32_t)(4 * REC_F4 + e), src + e);
+            }
         }
     };
 
     uint32_t r0 = warp * 32;
-    EvalDesc<MW> cur = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0, lane);
+    EvalDesc<MW> cur = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, gid_of_slot, begin, n, r0, lane);
     if (cur.cmax == 0) return;   // ranks descend in hit count: nothing for this warp
     issue_params(cur);
-    EvalDesc<MW> nxt = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0 + EVAL_THREADS, lane);
+    EvalDesc<MW> nxt = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, gid_of_slot, begin, n, r0 + EVAL_THREADS, lane);
     while (true) {
-        const EvalDesc<MW> nxt2 = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, begin, n, r0 + 2 * EVAL_THREADS, lane);
-        const uint32_t gid = cur.c != 0 ? __ldg(gid_of_slot + cur.sid) : 0u;
+        const EvalDesc<MW> nxt2 = load_eval_desc<MW, GMAJ>(rank_sid, rank_mask, rank_gstart, rank_pbase, gid_of_slot, begin, n, r0 + 2 * EVAL_THREADS, lane);
+        const uint32_t gid = cur.gid;
         cp_async_wait_all();   // the copies this lane issued have landed
         __syncwarp();          // ... and so have those of the other lanes, which hold pieces of this lane's record
         const PreRec P = unpack_pre(my_par[0], my_par[1], my_par[2], my_par[3], my_par[4]);   // (stale for lanes without hits: unused)
         float shc[SW + 3];
 #pragma unroll
         for (int q = 0; q < (SW + 3) / 4; ++q) {
-            const float4 t = my_par[5 + q];
-            shc[4 * q] = t.x; shc[4 * q + 1] = t.y; shc[4 * q + 2] = t.z; shc[4 * q + 3] = t.w;
+            const float4 t = my_par[5 + q];   // (times the basis constants: the hits evaluate the bare polynomials)
+            shc[4 * q] = t.x * sh_norm_word(4 * q); shc[4 * q + 1] = t.y * sh_norm_word(4 * q + 1);
+            shc[4 * q + 2] = t.z * sh_norm_word(4 * q + 2); shc[4 * q + 3] = t.w * sh_norm_word(4 * q + 3);
         }
         __syncwarp();                           // every lane has read its record: the buffers may be overwritten
         if (nxt.cmax != 0) issue_params(nxt);
@@ -1028,7 +1046,7 @@ static ForwardWs forward_layout(void* base, int64_t n_rays, int T, int64_t cap_p
 }
 
 template <int TS, bool GMAJ>
-static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const uint32_t* gid_of_slot, const uint32_t* tile_off,
+static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* rec, const float* sh, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                const uint32_t* rank_sid, const uint32_t* rank_mask, const uint32_t* rank_gstart,
                                const uint32_t* tile_lt_base, const uint32_t* rank_pbase, const uint32_t* ray_off,
                                const CamF& cam, float alpha_max, bool narrow, const ForwardWs& w, uint32_t* counts) {
@@ -1037,7 +1055,7 @@ static gart_status launch_eval(int deg, int T, cudaStream_t st, const float4* re
         auto kern = fwd_eval_kernel<TS, D, GMAJ>;                                                                          \
         constexpr int smem = EVAL_THREADS * (((20 + 3 * (D + 1) * (D + 1) + 3) / 4) | 1) * 16;                             \
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GART_ERR_CUDA; \
-        kern<<<T, EVAL_THREADS, smem, st>>>(rec, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, rank_pbase, ray_off, cam, \
+        kern<<<T, EVAL_THREADS, smem, st>>>(rec, sh, gid_of_slot, tile_off, rank_sid, rank_mask, rank_gstart, tile_lt_base, rank_pbase, ray_off, cam, \
                                             alpha_max, narrow, w.recs, counts);                                                               \
     }
     switch (deg) {
@@ -1115,7 +1133,8 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (g->n < 0 || g->sh_degree < 0 || g->sh_degree > 3 || cap_pairs < 0 || cap_hits < 0) return GART_ERR_INVALID_ARG;
     if (cap_hits > 0xfffffff0ll || cap_pairs > 0xfffffff0ll) return GART_ERR_INVALID_ARG;
     if (cam->width <= 0 || cam->height <= 0 || cam->width > 65535 * 8 || cam->height > 65535 * 8) return GART_ERR_INVALID_ARG;
-    if (cap_pairs > 0 && (!pair_gid || !pre || !slot_of_gid || !gid_of_slot)) return GART_ERR_INVALID_ARG;
+    if (cap_pairs > 0 && (!pair_gid || !pre || !slot_of_gid || !gid_of_slot || (g->n > 0 && !g->sh))) return GART_ERR_INVALID_ARG;
+    if (((uintptr_t)g->sh & 15) != 0) return GART_ERR_INVALID_ARG;   // the evaluation copies rows of coefficients in 16-byte pieces
     if (cap_hits > 0 && (!lt || (ray_gid == nullptr) != (ray_slot == nullptr))) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255) || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
     const int ts = cfg->tile_size;
@@ -1128,7 +1147,7 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     if (v.bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = (cudaStream_t)stream;
     const float4* rec = reinterpret_cast<const float4*>(pre);
-    const int rs4 = rec_f4(g->sh_degree);
+    const int rs4 = REC_F4;
     const int4* srect = reinterpret_cast<const int4*>(rec + (size_t)g->n * (rs4 + 2));   // the rectangles in slot order, behind the records
     const bool gmaj = cfg->lt_layout == GART_LT_PRIMITIVE_MAJOR;
     const int sup_x = (cam->width + GM_SUP - 1) / GM_SUP;
@@ -1209,11 +1228,11 @@ extern "C" gart_status gart_forward(const gart_config* cfg, const gart_gaussians
     GART_LAUNCH_CHECK();
 
     if (gmaj) {
-        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
-        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        if (ts == 8) s = launch_eval<8, true>(g->sh_degree, T, st, rec, g->sh, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        else s = launch_eval<16, true>(g->sh_degree, T, st, rec, g->sh, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gpos, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
     } else {
-        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
-        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        if (ts == 8) s = launch_eval<8, false>(g->sh_degree, T, st, rec, g->sh, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
+        else s = launch_eval<16, false>(g->sh_degree, T, st, rec, g->sh, gid_of_slot, tile_off, v.rank_sid, v.rank_mask, v.rank_gstart, v.tile_lt_base, v.rank_pbase, ray_off, cf, amax, narrow, w, counts);
     }
     if (s != GART_OK) return s;
 

@@ -26,7 +26,7 @@ def test_every_declared_symbol_is_exported():
 
 def test_host_only_queries():
     assert G.gart_mask_words(8) == 2 and G.gart_mask_words(16) == 8
-    assert [G.gart_pre_words(d) for d in range(4)] == [36, 44, 60, 80]
+    assert [G.gart_pre_words(d) for d in range(4)] == [32, 32, 32, 32]   # evaluation record 20 + quaternion, scale, opacity 8 + rectangle 4
     # accumulation records: 60 words per Gaussian in two arrays, each rounded up to 256 bytes
     assert G.gart_backward_workspace_bytes(1000) == 64_000 + 176_128 and G.gart_bounds_workspace_bytes(1000) > 80_000
     assert G.lib().gart_status_string(0) == b"ok" and G.lib().gart_status_string(2) == b"workspace too small"
