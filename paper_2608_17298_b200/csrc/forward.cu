@@ -554,7 +554,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
 
 // ------------------------------------------------------------------------------------------ phase 4
 constexpr int SORT_CAP = 512;    // hits per ray sorted in registers; longer rays sort in global memory
-constexpr int SWEEP_WARPS = 1;    // a block is one ray: a warp whose ray belongs to the other length class (or has ended) holds no shared memory of a block that is still sweeping
+constexpr int SWEEP_WARPS = 1;   // rays per block: with several, a block's shared memory and registers stay allocated until its longest ray is done
 
 // ---- rays of up to SORT_CAP hits: one warp, keys in registers (R per lane, lane l holds positions l R .. l R + R - 1)
 // A key is one 32-bit word: the bits of t* (a non-negative float: its bit pattern orders like its value)
