@@ -189,11 +189,27 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
         const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
         float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
         const float* sp = sh + (size_t)gid * SW;
+        if constexpr (SW % 4 == 0) {   // rows of whole 16-byte pieces (degrees 1 and 3; the array is 16-byte aligned)
 #pragma unroll
-        for (int k = 0; k < K; ++k) {
-            c0 = fmaf(B[k], __ldg(sp + 3 * k), c0);
-            c1 = fmaf(B[k], __ldg(sp + 3 * k + 1), c1);
-            c2 = fmaf(B[k], __ldg(sp + 3 * k + 2), c2);
+            for (int q = 0; q < SW / 4; ++q) {
+                const float4 t = __ldg(reinterpret_cast<const float4*>(sp) + q);
+                const float sv[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int wd = 4 * q + i;
+                    const float term = B[wd / 3] * sv[i];
+                    if (wd % 3 == 0) c0 += term;
+                    else if (wd % 3 == 1) c1 += term;
+                    else c2 += term;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                c0 = fmaf(B[k], __ldg(sp + 3 * k), c0);
+                c1 = fmaf(B[k], __ldg(sp + 3 * k + 1), c1);
+                c2 = fmaf(B[k], __ldg(sp + 3 * k + 2), c2);
+            }
         }
         c0 = fmaxf(c0, 0.0f); c1 = fmaxf(c1, 0.0f); c2 = fmaxf(c2, 0.0f);
         logT -= log1pf(-r.alpha);                       // log of the transmittance in front of this hit

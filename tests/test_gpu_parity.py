@@ -565,6 +565,13 @@ def test_invalid_arguments_return_status():
         with pytest.raises(G.GartError) as e:
             G.run_forward(cfg_bad, g, cam, buf)
         assert e.value.status == 1, cfg_bad
+    # the evaluation copies rows of SH coefficients from the caller's array in 16-byte pieces: an array that is not 16-byte
+    # aligned is refused on the host
+    import dataclasses
+    skew = torch.zeros(g.sh.numel() + 1, dtype=torch.float32, device="cuda")[1:].view(g.sh.shape)
+    with pytest.raises(G.GartError) as e:
+        G.run_forward(G.Config(), dataclasses.replace(g, sh=skew), cam, buf)
+    assert e.value.status == 1
     # pointers that a pass dereferences: refused on the host instead of faulting on the device
     with pytest.raises(G.GartError) as e:     # the pixel-centric baseline without the per-ray lists
         G.gart_backward_atomic(G.Config(), g, cam, buf.pre, buf.slot_of_gid, buf.ray_off, None, None, buf.lt, dl, buf.grad, buf.counts)
