@@ -450,6 +450,18 @@ int64_t orc_view_find_hits(orc_view *v, int mode, const uint8_t *pixel_mask) {
     double o[3];
     cam_origin(&v->cam, o);
     uint64_t *cnt = (uint64_t *)calloc((size_t)NR + 1, sizeof(uint64_t));
+    /* per image row the span of requested pixels (hi < lo: none), so that a sparse request does not walk the whole image
+     * for every Gaussian; the rays visited and what is computed for them are the same */
+    const int Hh = v->cam.height;
+    int *row_lo = (int *)malloc((size_t)Hh * sizeof(int)), *row_hi = (int *)malloc((size_t)Hh * sizeof(int));
+    for (int y = 0; y < Hh; ++y) {
+        row_lo[y] = 0; row_hi[y] = W - 1;
+        if (pixel_mask) {
+            int lo = W, hi = -1;
+            for (int x = 0; x < W; ++x) if (pixel_mask[(int64_t)y * W + x]) { if (x < lo) lo = x; hi = x; }
+            row_lo[y] = lo; row_hi[y] = hi;
+        }
+    }
     for (int pass = 0; pass < 2; ++pass) {
 #pragma omp parallel for schedule(dynamic, 256)
         for (int64_t i = 0; i < v->sc.n; ++i) {
@@ -462,7 +474,7 @@ int64_t orc_view_find_hits(orc_view *v, int mode, const uint8_t *pixel_mask) {
             double Wm[9], og[3];
             gauss_local(&v->sc, i, o, Wm, og);
             const double sigma = v->sc.opacity[i];
-            for (int y = y0; y <= y1; ++y) for (int x = x0; x <= x1; ++x) {
+            for (int y = y0; y <= y1; ++y) for (int x = (x0 > row_lo[y] ? x0 : row_lo[y]); x <= (x1 < row_hi[y] ? x1 : row_hi[y]); ++x) {
                 const int64_t ray = (int64_t)y * W + x;
                 if (pixel_mask && !pixel_mask[ray]) continue;
                 double d[3], ts, al;
@@ -490,7 +502,7 @@ int64_t orc_view_find_hits(orc_view *v, int mode, const uint8_t *pixel_mask) {
             v->alpha = (double *)malloc((size_t)(run + 1) * sizeof(double));
         }
     }
-    free(cnt);
+    free(cnt); free(row_lo); free(row_hi);
     /* order every ray's hits by (t*, id) */
 #pragma omp parallel
     {
