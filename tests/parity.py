@@ -228,6 +228,18 @@ def _locate_pairs(cam, cfg, gpu, rays, gids):
     return pair, below, tile
 
 
+def all_distinct_below(a, bound):
+    """True if the non-negative integers of `a` are pairwise distinct and all below `bound` (a flag per value: linear time)."""
+    a = np.asarray(a).astype(np.int64, copy=False)
+    if a.size == 0:
+        return True
+    if int(a.max()) >= bound or int(a.min()) < 0:
+        return False
+    seen = np.zeros(int(bound), dtype=bool)
+    seen[a] = True
+    return int(np.count_nonzero(seen)) == a.size
+
+
 def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     """Properties that hold at any size, checked on the whole view without the oracle (the per-hit part on a random
     subset of rays when the view has more than a few million hits): ray offsets, hit masks, slot numbering, and the
@@ -242,7 +254,7 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     assert pc.sum() == H and L >= H
     # every hit owns exactly one slot
     slots_all = gpu["ray_slot"]
-    assert np.unique(slots_all).size == H and (int(slots_all.max()) if H else -1) < L
+    assert slots_all.size == H and all_distinct_below(slots_all, L)
     P = pc.size
     # ---- slots: visible Gaussians in the order of the super-tile of their rectangle's corner, ids ascending inside one
     rect_ = gpu["rect"].astype(np.int64)
@@ -267,7 +279,7 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     sl = gpu["slot_of_gid"][gpu["pair_gid"]].astype(np.int64)
     ptx, pty = tile_of_pair % tiles_x, tile_of_pair // tiles_x
     gpos = gpo[sl] + (pty - ty0[sl]) * ntx[sl] + (ptx - tx0[sl])
-    assert np.array_equal(gpu["pair_gpos"].astype(np.int64), gpos) and np.unique(gpos).size == P
+    assert np.array_equal(gpu["pair_gpos"].astype(np.int64), gpos) and all_distinct_below(gpos, P)
     assert np.array_equal(gpu["gm_mask"][gpos], gpu["pair_mask"])
     pc_g = np.empty(P, np.int64)
     pc_g[gpos] = pc                                                # hits per pair, by primitive-major position
@@ -295,7 +307,7 @@ def check_structure(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     pi = np.repeat(np.arange(I), npair)
     kk = np.arange(npair.sum()) - np.repeat(np.cumsum(npair) - npair, npair)
     pg = gpos0[pi] + (kk // it_ntx[pi]) * ntx[it_slot][pi] + kk % it_ntx[pi]      # primitive-major position of the item's k-th pair
-    assert np.unique(pg).size == P                                  # the items partition the pairs
+    assert pg.size == P and all_distinct_below(pg, P)               # the items partition the pairs
     it_cnt = np.bincount(pi, weights=pc_g[pg], minlength=I).astype(np.int64)
     csum = np.cumsum(pc_g[pg]) - pc_g[pg]
     before = csum - np.repeat((np.cumsum(it_cnt) - it_cnt), npair)
@@ -371,7 +383,7 @@ def check_structure_tile(cam, cfg: G.Config, gpu, max_rays=20000, seed=0):
     H, L = gpu["counts"][G.CNT_HITS], t["lt_slots"]
     pc = np.bitwise_count(t["pair_mask"]).sum(axis=1).astype(np.int64)
     slots_all = t["ray_slot"]
-    assert np.unique(slots_all).size == H and (int(slots_all.max()) if H else -1) < L and L >= H
+    assert slots_all.size == H and all_distinct_below(slots_all, L) and L >= H
     tile_off, base = gpu["tile_off"].astype(np.int64), t["tile_lt_base"].astype(np.int64)
     assert base[0] == 0 and base[-1] == L and np.all(np.diff(base) >= 0)
     n_tile = np.diff(tile_off)

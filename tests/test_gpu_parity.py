@@ -427,14 +427,17 @@ def test_shell200k_sampled(view):
 
 def test_unbounded1m_sampled():
     scene, cams = gs.config_unbounded_1m()
-    sampled_parity(scene, cams[0], G.Config(tile_size=8), 0, n_gauss=150, n_tiles=30, n_large=14)
-    sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=40, n_tiles=8, n_large=6)
+    sampled_parity(scene, cams[0], G.Config(tile_size=8), 0, n_gauss=200, n_tiles=40, n_large=14)
+    sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=60, n_tiles=12, n_large=6)
 
 
 def test_unbounded6m_sampled():
     """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles)."""
     scene, cams = gs.config_unbounded_6m()
-    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=60, n_tiles=12, n_large=5, large_max_area=15000)
+    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=150, n_tiles=30, n_large=8, large_max_area=15000)
+    assert gpu["counts"][G.CNT_HITS] > 1e8
+    del gpu, ref
+    gpu, ref = sampled_parity(scene, cams[12], G.Config(tile_size=8), 12, n_gauss=60, n_tiles=12, n_large=3, large_max_area=15000)   # a second view of the orbit
     assert gpu["counts"][G.CNT_HITS] > 1e8
 
 
