@@ -431,13 +431,15 @@ def test_unbounded1m_sampled():
     sampled_parity(scene, cams[0], G.Config(tile_size=16), 1, n_gauss=60, n_tiles=12, n_large=6)
 
 
-def test_unbounded6m_sampled():
-    """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles)."""
+@pytest.mark.parametrize("view", [5, 0, 9, 12])
+def test_unbounded6m_sampled(view):
+    """The benchmark's configuration, in the launch configuration bench.py times (8x8 tiles): four views of the orbit,
+    the first with the larger sample."""
     scene, cams = gs.config_unbounded_6m()
-    gpu, ref = sampled_parity(scene, cams[5], G.Config(tile_size=8), 5, n_gauss=150, n_tiles=30, n_large=8, large_max_area=15000)
-    assert gpu["counts"][G.CNT_HITS] > 1e8
-    del gpu, ref
-    gpu, ref = sampled_parity(scene, cams[12], G.Config(tile_size=8), 12, n_gauss=60, n_tiles=12, n_large=3, large_max_area=15000)   # a second view of the orbit
+    if view == 5:
+        gpu, ref = sampled_parity(scene, cams[view], G.Config(tile_size=8), view, n_gauss=200, n_tiles=40, n_large=12, large_max_area=20000)
+    else:
+        gpu, ref = sampled_parity(scene, cams[view], G.Config(tile_size=8), view, n_gauss=80, n_tiles=16, n_large=4, large_max_area=15000)
     assert gpu["counts"][G.CNT_HITS] > 1e8
 
 
