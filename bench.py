@@ -86,7 +86,7 @@ def algorithmic_bytes_backward(H, P, n_vis, n_pixels, K):
 # Gaussians without a slot, the two kernels for cut Gaussians by visible Gaussians.  `--crop 0.5` prints the units of the captured case in roofline.traffic_units, so
 # that a fresh capture divides into these figures.
 TRAFFIC_MODEL = {
-    "tile": {"pairs_per_hit": 45.0, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
+    "tile": {"pairs_per_hit": 39.9, "zero_per_visible": 214.6, "convert_per_visible": 153.3,
              "scatter_read_per_visible": 186.0, "scatter_write_per_gaussian": 220.7},
     "primitive": {"items_read_per_lt_entry": 21.91, "items_write_per_visible": 235.7, "fill_write_per_invisible": 238.6,
                   "fill_read_per_gaussian": 4.0, "big_per_visible": 38.8},
