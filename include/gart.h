@@ -398,6 +398,7 @@ gart_status gart_backward_warp(const gart_config *cfg, const gart_gaussians *g, 
  * the ray in its pixel-centric part, keeps 4).  Same result as gart_backward up to rounding and summation order;
  * same workspace as gart_backward.  Errors as gart_backward; INVALID_ARG if cfg->lt_format != 1.
  */
+size_t gart_backward_hybrid_workspace_bytes(int64_t n, int32_t sh_degree);   /* gart_backward_workspace_bytes(n) + a copy of the coefficient rows in slot order */
 gart_status gart_backward_hybrid(const gart_config *cfg, const gart_gaussians *g, const gart_camera *cam, const float *pre,
                                  const uint32_t *slot_of_gid, const uint32_t *gid_of_slot, const uint32_t *tile_off,
                                  const void *view, size_t view_bytes, int64_t cap_pairs,

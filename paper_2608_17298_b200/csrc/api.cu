@@ -65,7 +65,7 @@ extern "C" size_t gart_workspace_bytes(int64_t n, int32_t width, int32_t height,
     size_t b = gart_bounds_workspace_bytes(nn);
     const size_t w1 = gart_tile_map_workspace_bytes(nn, width, height, tile_size, cap_pairs);
     const size_t w2 = gart_forward_workspace_bytes(width, height, tile_size, cap_pairs, cap_hits);
-    const size_t w3 = gart_backward_workspace_bytes(nn);
+    const size_t w3 = gart_backward_hybrid_workspace_bytes(nn, 3);   // (the largest backward need: the hybrid pass at SH degree 3)
     if (w1 > b) b = w1;
     if (w2 > b) b = w2;
     if (w3 > b) b = w3;

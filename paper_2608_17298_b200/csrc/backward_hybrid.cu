@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(HYB_THREADS) bwd_sh_kernel(const uint32_t* __r
 // One thread per ray; per hit three 16-byte vector reductions on the moments of the Gaussian's accumulation record
 // (v, Q, sum alpha dL/dalpha: the same record that the primitive-centric pass fills, converted afterwards).
 template <int DEG>
-__global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const float* __restrict__ sh, const uint32_t* __restrict__ slot_of_gid,
+__global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __restrict__ rec, const float4* __restrict__ sh_slot, const uint32_t* __restrict__ slot_of_gid,
                                                             const uint32_t* __restrict__ ray_off, const uint32_t* __restrict__ ray_gid,
                                                             const float* __restrict__ dL_dC, CamF cam, float bg0, float bg1, float bg2,
                                                             Gacc gacc, const uint32_t* __restrict__ counts) {
@@ -188,27 +188,20 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
         const PreRec P = load_pre(rp);
         const RayEval r = ray_eval(P, (float)(x - P.ix) - P.rx, (float)(y - P.iy) - P.ry);
         float c0 = 0.5f, c1 = 0.5f, c2 = 0.5f;
-        const float* sp = sh + (size_t)gid * SW;
-        if constexpr (SW % 4 == 0) {   // rows of whole 16-byte pieces (degrees 1 and 3; the array is 16-byte aligned)
+        const float4* sp = sh_slot + (size_t)sid * ((SW + 3) / 4);   // the slot's coefficient row (a copy in slot order: rays of a warp meet the same few rows)
 #pragma unroll
-            for (int q = 0; q < SW / 4; ++q) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(sp) + q);
-                const float sv[4] = {t.x, t.y, t.z, t.w};
+        for (int q = 0; q < (SW + 3) / 4; ++q) {
+            const float4 t = __ldg(sp + q);
+            const float sv[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int wd = 4 * q + i;
+            for (int i = 0; i < 4; ++i) {
+                const int wd = 4 * q + i;
+                if (wd < SW) {
                     const float term = B[wd / 3] * sv[i];
                     if (wd % 3 == 0) c0 += term;
                     else if (wd % 3 == 1) c1 += term;
                     else c2 += term;
                 }
-            }
-        } else {
-#pragma unroll
-            for (int k = 0; k < K; ++k) {
-                c0 = fmaf(B[k], __ldg(sp + 3 * k), c0);
-                c1 = fmaf(B[k], __ldg(sp + 3 * k + 1), c1);
-                c2 = fmaf(B[k], __ldg(sp + 3 * k + 2), c2);
             }
         }
         c0 = fmaxf(c0, 0.0f); c1 = fmaxf(c1, 0.0f); c2 = fmaxf(c2, 0.0f);
@@ -226,6 +219,23 @@ __global__ void __launch_bounds__(128) bwd_pixel_geo_kernel(const float4* __rest
         const float om = 1.0f - r.alpha;
         cb0 = fmaf(r.alpha, c0, om * cb0); cb1 = fmaf(r.alpha, c1, om * cb1); cb2 = fmaf(r.alpha, c2, om * cb2);
     }
+}
+
+// The coefficient rows of the view's slots, copied once per call in slot order (rows padded to whole 16-byte pieces): the
+// pixel pass reads a hit's row once per hit, and read by Gaussian id those reads scatter over the whole scene.
+static __global__ void __launch_bounds__(256) hyb_gather_sh_kernel(const float* __restrict__ sh, const uint32_t* __restrict__ gid_of_slot, int sw,
+                                                                   float* __restrict__ sh_slot, const uint32_t* __restrict__ counts) {
+    const int swp = (sw + 3) & ~3;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t slot = t / swp;
+    const int e = (int)(t - slot * swp);
+    if (slot >= (int64_t)counts[GART_CNT_VISIBLE]) return;
+    sh_slot[t] = e < sw ? __ldg(sh + (size_t)gid_of_slot[slot] * sw + e) : 0.0f;
+}
+
+static inline size_t hybrid_sh_bytes(int64_t n, int sh_degree) {
+    const int sw = 3 * (sh_degree + 1) * (sh_degree + 1);
+    return align256((size_t)n * ((sw + 3) & ~3) * 4);
 }
 
 template <int TS>
@@ -246,6 +256,11 @@ static gart_status launch_sh(int deg, int T, cudaStream_t st, const uint32_t* ti
 
 }  // namespace gart
 
+extern "C" size_t gart_backward_hybrid_workspace_bytes(int64_t n, int32_t sh_degree) {
+    const int64_t nn = n > 0 ? n : 1;
+    return gart_backward_workspace_bytes(nn) + gart::hybrid_sh_bytes(nn, sh_degree < 0 ? 0 : (sh_degree > 3 ? 3 : sh_degree));
+}
+
 extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_gaussians* g, const gart_camera* cam, const float* pre,
                                             const uint32_t* slot_of_gid, const uint32_t* gid_of_slot, const uint32_t* tile_off,
                                             const void* view, size_t view_bytes, int64_t cap_pairs,
@@ -263,7 +278,7 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     if (g->n == 0) return GART_OK;
     if (!grad || !pre || !slot_of_gid || !gid_of_slot || !lt_w || !ray_gid || !view || ((uintptr_t)view & 255)) return GART_ERR_INVALID_ARG;
     if (!workspace || ((uintptr_t)workspace & 255)) return GART_ERR_INVALID_ARG;
-    if (gart_backward_workspace_bytes(g->n) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
+    if (gart_backward_hybrid_workspace_bytes(g->n, g->sh_degree) > workspace_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     const ViewLayout v = view_layout(const_cast<void*>(view), g->n, cam->width, cam->height, cfg->tile_size, cap_pairs);
     if (v.bytes > view_bytes) return GART_ERR_WORKSPACE_TOO_SMALL;
     const uint32_t *rank_sid = v.rank_sid, *rank_mask = v.rank_mask, *rank_gstart = v.rank_gstart, *tile_lt_base = v.tile_lt_base;
@@ -280,7 +295,13 @@ extern "C" gart_status gart_backward_hybrid(const gart_config* cfg, const gart_g
     const int64_t n_rays = (int64_t)cam->width * cam->height;
     const unsigned blocks = (unsigned)ceil_div(n_rays, 128);
     const float* bg = cfg->background;
-#define GART_GEO(D) bwd_pixel_geo_kernel<D><<<blocks, 128, 0, st>>>(rec, g->sh, slot_of_gid, ray_off, ray_gid, dL_dcolor, cf, bg[0], bg[1], bg[2], gacc, counts)
+    float* sh_slot = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + gart_backward_workspace_bytes(g->n));
+    {
+        const int sw = 3 * (g->sh_degree + 1) * (g->sh_degree + 1), swp = (sw + 3) & ~3;
+        hyb_gather_sh_kernel<<<(unsigned)ceil_div(g->n * (int64_t)swp, 256), 256, 0, st>>>(g->sh, gid_of_slot, sw, sh_slot, counts);
+        GART_LAUNCH_CHECK();
+    }
+#define GART_GEO(D) bwd_pixel_geo_kernel<D><<<blocks, 128, 0, st>>>(rec, reinterpret_cast<const float4*>(sh_slot), slot_of_gid, ray_off, ray_gid, dL_dcolor, cf, bg[0], bg[1], bg[2], gacc, counts)
     switch (g->sh_degree) {
         case 0: GART_GEO(0); break;
         case 1: GART_GEO(1); break;

@@ -34,7 +34,8 @@ EXPORTS = [
     "gart_status_string", "gart_mask_words", "gart_pre_words", "gart_bounds_workspace_bytes", "gart_bounds",
     "gart_tile_map_workspace_bytes", "gart_tile_map", "gart_tile_map_static", "gart_view_bytes", "gart_view_array",
     "gart_forward_workspace_bytes", "gart_forward",
-    "gart_backward_workspace_bytes", "gart_backward", "gart_backward_tile", "gart_backward_atomic", "gart_backward_hybrid", "gart_backward_warp",
+    "gart_backward_workspace_bytes", "gart_backward_hybrid_workspace_bytes", "gart_backward", "gart_backward_tile", "gart_backward_atomic", "gart_backward_hybrid",
+    "gart_backward_warp",
     "gart_workspace_bytes", "gart_read_counts", "gart_sync_status",
     "gart_view_host_arena_bytes", "gart_view_host", "gart_view_host_async", "gart_counts_status",
 ]
@@ -96,6 +97,8 @@ def lib():
         L.gart_forward.argtypes = [vp] * 8 + [i64] + [vp] * 4 + [i64] + [vp] * 4 + [sz, vp, vp, sz, vp]
         L.gart_backward_workspace_bytes.restype = sz
         L.gart_backward_workspace_bytes.argtypes = [i64]
+        L.gart_backward_hybrid_workspace_bytes.restype = sz
+        L.gart_backward_hybrid_workspace_bytes.argtypes = [i64, i32]
         for fn in ("gart_backward", "gart_backward_tile", "gart_backward_warp"):
             getattr(L, fn).argtypes = [vp] * 8 + [sz, i64] + [vp] * 5 + [sz, vp]
         L.gart_backward_atomic.argtypes = [vp] * 13
@@ -322,6 +325,10 @@ def gart_forward(cfg: Config, g: Gaussians, cam, pre, slot_of_gid, gid_of_slot, 
 
 def gart_backward_workspace_bytes(n) -> int:
     return int(lib().gart_backward_workspace_bytes(int(n)))
+
+
+def gart_backward_hybrid_workspace_bytes(n, sh_degree) -> int:
+    return int(lib().gart_backward_hybrid_workspace_bytes(int(n), int(sh_degree)))
 
 
 def _backward_call(name, cfg, g, cam, pre, slot_of_gid, gid_of_slot, tile_off, view, cap_pairs, lt, dL_dcolor, grad, counts,

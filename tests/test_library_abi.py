@@ -39,7 +39,9 @@ def test_host_only_queries():
     assert G.gart_view_host_arena_bytes(1000, 3, 640, 480, 8, 10_000, 100_000) > f1
     # one query for the whole view: the largest of the four
     assert G.gart_workspace_bytes(1000, 640, 480, 8, 10_000, 100_000) == max(
-        f1, a, G.gart_bounds_workspace_bytes(1000), G.gart_backward_workspace_bytes(1000))
+        f1, a, G.gart_bounds_workspace_bytes(1000), G.gart_backward_hybrid_workspace_bytes(1000, 3))
+    assert G.gart_backward_hybrid_workspace_bytes(1000, 3) == G.gart_backward_workspace_bytes(1000) + 1000 * 48 * 4
+    assert G.gart_backward_hybrid_workspace_bytes(1000, 0) == G.gart_backward_workspace_bytes(1000) + 16128   # 1000 rows of 4 words, to 256 bytes
     # the view block: grows with the pair capacity; its named arrays lie inside it, 256-byte aligned, in order
     v1, v2 = G.gart_view_bytes(1000, 640, 480, 8, 10_000), G.gart_view_bytes(1000, 640, 480, 8, 20_000)
     assert 0 < v1 < v2 and v1 % 256 == 0 and G.gart_view_bytes(1000, 640, 480, 12, 10_000) == 0
