@@ -586,7 +586,7 @@ def main():
     ap.add_argument("--lt16-reps", type=int, default=2, help="timed runs of forward + backward with 8-byte LT entries on the last view (0: skip)")
     ap.add_argument("--other-ts-reps", type=int, default=2, help="timed runs of the whole step at the other tile size on the last view (0: skip)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--e2e-inflight", type=int, default=3, help="views in flight in the end-to-end measurement (each holds an arena on the device)")
+    ap.add_argument("--e2e-inflight", type=int, default=4, help="views in flight in the end-to-end measurement (each holds an arena on the device)")
     ap.add_argument("--oracle-frac", type=float, default=0.08)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--crop", type=float, default=1.0, help="central crop of every view (profiling on a smaller case)")
