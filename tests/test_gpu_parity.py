@@ -443,6 +443,49 @@ def test_unbounded6m_sampled(view):
     assert gpu["counts"][G.CNT_HITS] > 1e8
 
 
+def test_unbounded6m_whole_orbit_layouts_agree():
+    """Every one of the benchmark's 16 views, without the oracle: the view's invariants (hit totals, transmittances in [0, 1],
+    finite colours and gradients, no error word, every gradient record written) and agreement of the two decompositions of
+    the backward pass, whose forward passes lay the intermediate buffer out differently: identical hit counts, colours and
+    transmittances, gradients equal up to the rounding of differently ordered sums.  Compared on the device."""
+    import dataclasses
+    scene, cams = gs.config_unbounded_6m()
+    g = G.Gaussians.from_numpy(scene)
+    cfg_t = G.Config(tile_size=8, lt_layout=G.LT_TILE_MAJOR)
+    cfg_p = dataclasses.replace(cfg_t, lt_layout=G.LT_PRIMITIVE_MAJOR)
+    cap_pairs, cap_hits = 0, 0
+    for cam in (cams[0], cams[8]):
+        for cfg in (cfg_t, cfg_p):
+            P, S = G.size_view(cfg, g, cam, slack=1.3)
+            cap_pairs, cap_hits = max(cap_pairs, P), max(cap_hits, S)
+    buf = G.ViewBuffers(g.n, g.sh_degree, cams[0], cfg_t, cap_pairs, cap_hits)
+    gt, gp = torch.empty_like(buf.grad), torch.empty_like(buf.grad)
+    worst = 0.0
+    for v, cam in enumerate(cams):
+        dl = torch.from_numpy(gs.upstream_gradient(cam, v)).cuda()
+        outs = []
+        for cfg, grad, back in ((cfg_t, gt, G.run_backward_tile), (cfg_p, gp, G.run_backward)):
+            grad.fill_(float("nan"))
+            G.run_bounds_tile_map(cfg, g, cam, buf)
+            G.run_forward(cfg, g, cam, buf, ray_lists=False)
+            back(cfg, g, cam, buf, dl, grad)
+            cnt = G.gart_read_counts(buf.counts)
+            assert cnt[G.CNT_ERROR] == 0, (v, cnt)
+            assert int(buf.hit_count.view(torch.int32).sum(dtype=torch.int64)) == cnt[G.CNT_HITS] > 1e8
+            assert bool(torch.isfinite(buf.color).all()) and bool(torch.isfinite(grad).all())
+            assert float(buf.t_final.min()) >= 0.0 and float(buf.t_final.max()) <= 1.0
+            outs.append((buf.color.clone(), buf.t_final.clone(), buf.hit_count.clone(), cnt[G.CNT_HITS], cnt[G.CNT_PAIRS]))
+        a, b = outs
+        assert a[3] == b[3] and a[4] == b[4] and torch.equal(a[2], b[2])
+        assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])          # both layouts composite the very same numbers
+        x, y = gt[:, :59].double(), gp[:, :59].double()
+        tol = 1e-3 * torch.maximum(x.abs(), y.abs()) + 1e-5 * x.abs().amax(dim=1, keepdim=True) + 1e-6
+        bad = (x - y).abs() > tol
+        assert not bool(bad.any()), (v, int(bad.sum()))
+        worst = max(worst, float(((x - y).abs() / tol).max()))
+    print("whole orbit: 16 views, largest difference between the two backward decompositions %.2f of the tolerance" % worst)
+
+
 # ------------------------------------------------------------------------------------------ edge cases and errors
 def _empty_scene(deg=1):
     K = (deg + 1) ** 2
