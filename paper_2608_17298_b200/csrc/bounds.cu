@@ -19,6 +19,7 @@ constexpr int PRE_TMP_F4 = 7;   // float4 per Gaussian in the id-ordered tempora
 struct CamD {
     int width, height;
     double fx, fy, cx, cy;
+    double ifx, ify;   // 1 / fx, 1 / fy: the record's quotients are products (fp64 divisions are what this kernel's time goes to)
     double w2c[12];
 };
 
@@ -105,7 +106,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
                                          -(M[2] * M[3] + M[6] * M[7] + M[10] * M[11])};
 #pragma unroll
                     for (int k = 0; k < 3; ++k) {
-                        const double w0 = R[k] / s[k], w1 = R[3 + k] / s[k], w2 = R[6 + k] / s[k];  // row k of W
+                        const double is = 1.0 / s[k];
+                        const double w0 = R[k] * is, w1 = R[3 + k] * is, w2 = R[6 + k] * is;  // row k of W
 #pragma unroll
                         for (int j = 0; j < 3; ++j) Wc[3 * k + j] = w0 * M[4 * j] + w1 * M[4 * j + 1] + w2 * M[4 * j + 2];
                         m[k] = w0 * (mu[0] - o[0]) + w1 * (mu[1] - o[1]) + w2 * (mu[2] - o[2]);
@@ -113,13 +115,14 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
                     // reference position: projected centre when that is a sane pixel coordinate
                     double rpx = cam.cx, rpy = cam.cy;
                     if (c == 1) {
-                        const double ppx = cam.fx * muc[0] / muc[2] + cam.cx, ppy = cam.fy * muc[1] / muc[2] + cam.cy;
+                        const double iz = 1.0 / muc[2];
+                        const double ppx = cam.fx * muc[0] * iz + cam.cx, ppy = cam.fy * muc[1] * iz + cam.cy;
                         if (fabs(ppx) < 1.0e6 && fabs(ppy) < 1.0e6) { rpx = ppx; rpy = ppy; }
                     }
                     const double fix = floor(rpx), fiy = floor(rpy);
                     const float rx = (float)(rpx - 0.5 - fix), ry = (float)(rpy - 0.5 - fiy);
                     const double ex_px = fix + 0.5 + (double)rx, ex_py = fiy + 0.5 + (double)ry;  // exactly what the kernels use
-                    const double du = (ex_px - cam.cx) / cam.fx, dv = (ex_py - cam.cy) / cam.fy;
+                    const double du = (ex_px - cam.cx) * cam.ifx, dv = (ex_py - cam.cy) * cam.ify;
                     double dgr[3], kk[3];
 #pragma unroll
                     for (int k = 0; k < 3; ++k) dgr[k] = Wc[3 * k] * du + Wc[3 * k + 1] * dv + Wc[3 * k + 2];
@@ -127,8 +130,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
                     kk[0] = dgr[1] * m[2] - dgr[2] * m[1];
                     kk[1] = dgr[2] * m[0] - dgr[0] * m[2];
                     kk[2] = dgr[0] * m[1] - dgr[1] * m[0];
-                    q0 = make_float4((float)(Wc[0] / cam.fx), (float)(Wc[3] / cam.fx), (float)(Wc[6] / cam.fx), (float)(Wc[1] / cam.fy));
-                    q1 = make_float4((float)(Wc[4] / cam.fy), (float)(Wc[7] / cam.fy), (float)dgr[0], (float)dgr[1]);
+                    q0 = make_float4((float)(Wc[0] * cam.ifx), (float)(Wc[3] * cam.ifx), (float)(Wc[6] * cam.ifx), (float)(Wc[1] * cam.ify));
+                    q1 = make_float4((float)(Wc[4] * cam.ify), (float)(Wc[7] * cam.ify), (float)dgr[0], (float)dgr[1]);
                     q2 = make_float4((float)dgr[2], (float)m[0], (float)m[1], (float)m[2]);
                     q3 = make_float4((float)kk[0], (float)kk[1], (float)kk[2], (float)sigma);
                     q4 = make_float4(rx, ry, __int_as_float((int)fix), __int_as_float((int)fiy));
@@ -277,6 +280,7 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     gart::CamD c;
     c.width = cam->width; c.height = cam->height;
     c.fx = cam->fx; c.fy = cam->fy; c.cx = cam->cx; c.cy = cam->cy;
+    c.ifx = 1.0 / c.fx; c.ify = 1.0 / c.fy;
     for (int i = 0; i < 12; ++i) c.w2c[i] = cam->w2c[i];
     // Slots are numbered in the order of the super-tile (16 x 16 pixels) of the rectangle's corner: neighbours in the image
     // are neighbours in every per-slot array.  The primitive-major layout wants the full order (its work items of a

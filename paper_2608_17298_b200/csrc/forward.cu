@@ -425,17 +425,18 @@ __device__ __forceinline__ EvalDesc<MW> load_eval_desc(const uint32_t* __restric
     return d;
 }
 
-// Per-pixel data of the tile in shared memory, two float4 per pixel: (d.x, d.y, d.z, x) and (y, ray_off, -, -), d the
-// unit ray direction, (x, y) the position in the tile, ray_off the start of the ray's segment of hit records.
+// Per-pixel data of the tile in shared memory, one float4 per pixel: the unit ray direction.
 // Lanes read DIFFERENT pixels at the same time; with 8 copies, copy j confined to the 16-byte bank group j and
 // lane l reading copy l mod 8, the 8 lanes served together by a 16-byte shared load never collide.
 template <int TS>
 struct EvalPix {
     static constexpr int COPIES = TS == 8 ? 8 : 1;
-    static constexpr int STRIDE = COPIES == 1 ? 3 : 2;
-    static constexpr int F4 = TS * TS * STRIDE * COPIES;
-    __device__ static __forceinline__ int index(int p, int h, int copy) { return (p * STRIDE + h) * COPIES + copy; }
+    static constexpr int F4 = TS * TS * COPIES;
+    __device__ static __forceinline__ int index(int p, int copy) { return p * COPIES + copy; }
 };
+
+// A small non-negative integer as a float without a conversion instruction (exact below 2^23).
+__device__ __forceinline__ float small_int_float(int v) { return __uint_as_float(0x4b000000u | (uint32_t)v) - 8388608.0f; }
 
 // Block per tile, one thread per (tile, Gaussian) pair; warps walk the rank groups.  The records of the
 // next group's Gaussians are copied into shared memory (16-byte asynchronous copies of each lane) while the
@@ -464,14 +465,10 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         const int x = x0 + p % TS, y = y0 + p / TS;
         const float3 d = pixel_dir(cam, min(x, cam.width - 1), min(y, cam.height - 1));
         const uint32_t ro = (x < cam.width && y < cam.height) ? ray_off[(size_t)y * cam.width + x] : 0u;
-        const float4 a = make_float4(d.x, d.y, d.z, (float)(p % TS));
-        const float4 b = make_float4((float)(p / TS), __uint_as_float(ro), 0.0f, 0.0f);
+        const float4 a = make_float4(d.x, d.y, d.z, 0.0f);
 #pragma unroll
-        for (int c = 0; c < EvalPix<TS>::COPIES; ++c) {
-            spix[EvalPix<TS>::index(p, 0, c)] = a;
-            spix[EvalPix<TS>::index(p, 1, c)] = b;
-        }
-        scur[p] = 0u;
+        for (int c = 0; c < EvalPix<TS>::COPIES; ++c) spix[EvalPix<TS>::index(p, c)] = a;
+        scur[p] = ro;   // the next free place of the ray's segment of hit records
     }
     __syncthreads();
     const uint32_t lt_base = tile_lt_base[tile];
@@ -538,9 +535,9 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
         const uint32_t wdx = (cur.pbase / GM_SUP) & 1u, wdy = cur.pbase / (GM_WIN * GM_SUP);   // the tile's super-tile inside the owner's window
         // one hit: evaluate, take the next free place of the ray's segment, write the 32-byte record
         auto hit = [&](const int p, const uint32_t slot_e) {
-            const float4 pa = spix_lane[EvalPix<TS>::index(p, 0, 0)], pb = spix_lane[EvalPix<TS>::index(p, 1, 0)];
+            const float4 pa = spix_lane[EvalPix<TS>::index(p, 0)];
             const uint32_t pos = atomicAdd(&scur[p], 1u);
-            const RayEval r = ray_eval(P, (fbx + pa.w) - P.rx, (fby + pb.x) - P.ry, narrow);   // small integers: the sums are exact
+            const RayEval r = ray_eval(P, (fbx + small_int_float(p % TS)) - P.rx, (fby + small_int_float(p / TS)) - P.ry, narrow);   // small integers: the sums are exact
             const float t = fmaxf(r.tnum * r.inv_a, 0.0f);
             float B[K];
             sh_poly<K>(make_float3(pa.x, pa.y, pa.z), B);
@@ -551,7 +548,7 @@ __global__ void __launch_bounds__(EVAL_THREADS) fwd_eval_kernel(const float4* __
                 c1 = fmaf(B[k], shc[3 * k + 1], c1);
                 c2 = fmaf(B[k], shc[3 * k + 2], c2);
             }
-            float4* out = recs + ((size_t)__float_as_uint(pb.y) + pos) * 2;
+            float4* out = recs + (size_t)pos * 2;
             // The lowest mantissa bit of the first two colour words tells the sweep in which of the 2 x 2 super-tiles of the
             // owner's window this pixel lies (the primitive-major LT entry names its pixel inside that window).  The sweep
             // composites the words without that bit, so both layouts composite the very same numbers.
