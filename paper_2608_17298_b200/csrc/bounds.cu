@@ -14,7 +14,9 @@
 
 namespace gart {
 
-constexpr int PRE_TMP_F4 = 7;   // float4 per Gaussian in the id-ordered temporary: 5 of the record, quaternion, scale + opacity
+constexpr int PRE_TMP_F4 = 8;   // float4 per Gaussian in the id-ordered temporary: 5 of the record, quaternion, scale + opacity, rectangle
+                                // (128 bytes: the gather reads one whole line per Gaussian and nothing else)
+constexpr int PRE_TMP_PAD = PRE_TMP_F4 + 1;   // lane stride of the staging rows in shared memory (odd: no bank conflicts)
 
 struct CamD {
     int width, height;
@@ -36,10 +38,10 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
                                                      int32_t* __restrict__ rect, uint8_t* __restrict__ cls,
                                                      float4* __restrict__ pre4, uint32_t* __restrict__ keys,
                                                      uint32_t* __restrict__ vals, uint32_t* __restrict__ counts) {
-    __shared__ float4 s_out[128 * PRE_TMP_F4];   // the block's 128 temporaries, staged so that the stores are whole rows
+    __shared__ float4 s_out[128 * PRE_TMP_PAD];   // the block's 128 temporaries, staged so that the stores are whole rows
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int vis = 0, straddle = 0;
-    float4 q0 = make_float4(0, 0, 0, 0), q1 = q0, q2 = q0, q3 = q0, q4 = q0, q5 = q0, q6 = q0;
+    float4 q0 = make_float4(0, 0, 0, 0), q1 = q0, q2 = q0, q3 = q0, q4 = q0, q5 = q0, q6 = q0, q7 = q0;
     if (i < n) {
         int x0 = 0, y0 = 0, x1 = -1, y1 = -1, c = 0;
         const double sigma = (double)opacity[i];
@@ -143,6 +145,7 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
         if (vis) {   // quaternion, scale, opacity ride along so that the gather reads one contiguous piece
             q5 = make_float4(quat[4 * i], quat[4 * i + 1], quat[4 * i + 2], quat[4 * i + 3]);
             q6 = make_float4(scale[3 * i], scale[3 * i + 1], scale[3 * i + 2], opacity[i]);
+            q7 = make_float4(__int_as_float(x0), __int_as_float(y0), __int_as_float(x1), __int_as_float(y1));
         }
         // super-tile of the rectangle's corner (its row alone where the caller sorts by rows: sup_x = 1)
         keys[i] = vis ? (uint32_t)((y0 / GM_SUP) * sup_x + (sup_x > 1 ? x0 / GM_SUP : 0)) : key_none;
@@ -151,9 +154,9 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
     {
         // a warp's 32 temporaries are contiguous in memory: through shared memory (lane stride 7 float4, odd: no bank
         // conflicts) and out as 7 coalesced 512-byte rows
-        const int lane = threadIdx.x & 31, wbase = (threadIdx.x & ~31) * PRE_TMP_F4;
-        float4* mine = s_out + wbase + lane * PRE_TMP_F4;
-        mine[0] = q0; mine[1] = q1; mine[2] = q2; mine[3] = q3; mine[4] = q4; mine[5] = q5; mine[6] = q6;
+        const int lane = threadIdx.x & 31, wbase = (threadIdx.x & ~31) * PRE_TMP_PAD;
+        float4* mine = s_out + wbase + lane * PRE_TMP_PAD;
+        mine[0] = q0; mine[1] = q1; mine[2] = q2; mine[3] = q3; mine[4] = q4; mine[5] = q5; mine[6] = q6; mine[7] = q7;
         __syncwarp();
         const int64_t i_w = i - lane;                      // first Gaussian of the warp
         const int64_t left = (n - i_w) * PRE_TMP_F4;       // float4 of this warp that exist
@@ -161,7 +164,7 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
 #pragma unroll
         for (int j = 0; j < PRE_TMP_F4; ++j) {
             const int idx = j * 32 + lane;
-            if (idx < left) dst[idx] = s_out[wbase + idx];
+            if (idx < left) dst[idx] = s_out[wbase + (idx / PRE_TMP_F4) * PRE_TMP_PAD + idx % PRE_TMP_F4];
         }
     }
     const unsigned bv = __ballot_sync(0xffffffffu, vis), bs = __ballot_sync(0xffffffffu, straddle);
@@ -171,23 +174,25 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
     }
 }
 
-// One thread per 16 bytes of a slot's evaluation record (5 float4).  Also fills the two maps between ids and slots.
+// One thread per 16 bytes of a slot's 128-byte temporary: eight threads read the whole line of their Gaussian and write
+// the evaluation record (5 float4), the quaternion and scale + opacity (2) and the rectangle (1) into their
+// slot-ordered arrays.  Also fills the two maps between ids and slots.
 constexpr int GATHER_UNROLL = 2;
 
 __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_t key_none,
                                                              const uint32_t* __restrict__ keys_sorted, const uint32_t* __restrict__ vals_sorted,
-                                                             const float4* __restrict__ pre_tmp, const int4* __restrict__ rect,
+                                                             const float4* __restrict__ pre_tmp,
                                                              float4* __restrict__ rec, float4* __restrict__ qs, int4* __restrict__ srect,
                                                              uint32_t* __restrict__ slot_of_gid, uint32_t* __restrict__ gid_of_slot) {
-    constexpr uint32_t RS4 = REC_F4;   // (compile-time: the divisions below are multiplications)
+    constexpr uint32_t RS4 = REC_F4;
     // GATHER_UNROLL pieces per thread, their loads issued together (the chain id -> record otherwise leaves too few bytes in flight)
     uint32_t slot[GATHER_UNROLL], q[GATHER_UNROLL], gid[GATHER_UNROLL];
     bool vis[GATHER_UNROLL];
 #pragma unroll
     for (int u = 0; u < GATHER_UNROLL; ++u) {
         const uint32_t t = (blockIdx.x * GATHER_UNROLL + u) * blockDim.x + threadIdx.x;
-        slot[u] = t / RS4;
-        q[u] = t - slot[u] * RS4;
+        slot[u] = t / PRE_TMP_F4;
+        q[u] = t % PRE_TMP_F4;
         const bool in = slot[u] < n;
         gid[u] = in ? vals_sorted[slot[u]] : 0u;
         vis[u] = in && keys_sorted[slot[u]] != key_none;
@@ -205,12 +210,9 @@ __global__ void __launch_bounds__(256) gather_records_kernel(uint32_t n, uint32_
 #pragma unroll
     for (int u = 0; u < GATHER_UNROLL; ++u) {
         if (!vis[u]) continue;
-        if (q[u] == 1) {   // quaternion, scale and opacity in slot order for the backward's per-Gaussian pass
-            qs[2 * (size_t)slot[u]] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 5];
-            qs[2 * (size_t)slot[u] + 1] = pre_tmp[(size_t)gid[u] * PRE_TMP_F4 + 6];
-        }
-        if (q[u] == 2) srect[slot[u]] = rect[gid[u]];   // the rectangle in slot order
-        rec[(size_t)slot[u] * RS4 + q[u]] = v[u];
+        if (q[u] < RS4) rec[(size_t)slot[u] * RS4 + q[u]] = v[u];
+        else if (q[u] < RS4 + 2) qs[2 * (size_t)slot[u] + (q[u] - RS4)] = v[u];   // quaternion; scale and opacity (the backward's per-Gaussian pass)
+        else srect[slot[u]] = make_int4(__float_as_int(v[u].x), __float_as_int(v[u].y), __float_as_int(v[u].z), __float_as_int(v[u].w));
     }
 }
 
@@ -302,11 +304,11 @@ extern "C" gart_status gart_bounds(const gart_config* cfg, const gart_gaussians*
     gart_status s = radix_sort_pairs(kbuf, vbuf, cur, bits, g->n, nullptr, (uint32_t)g->n, nullptr, w.table, w.scan_ws, w.total64, st);
     if (s != GART_OK) return s;
     const int rs4 = REC_F4;
-    const int64_t gthreads = g->n * rs4;
+    const int64_t gthreads = g->n * PRE_TMP_F4;
     if (gthreads >= (int64_t)1 << 32) return GART_ERR_INVALID_ARG;   // (32-bit thread indices)
     float4* rec_out = reinterpret_cast<float4*>(pre);
     gather_records_kernel<<<(unsigned)ceil_div(gthreads, 256 * GATHER_UNROLL), 256, 0, st>>>((uint32_t)g->n, key_none, kbuf[0], vbuf[0], w.pre_tmp,
-                                                                                reinterpret_cast<const int4*>(rect), rec_out, rec_out + (size_t)g->n * rs4,
+                                                                                rec_out, rec_out + (size_t)g->n * rs4,
                                                                                 reinterpret_cast<int4*>(rec_out + (size_t)g->n * (rs4 + 2)), slot_of_gid, gid_of_slot);
     GART_LAUNCH_CHECK();
     return GART_OK;
