@@ -152,8 +152,8 @@ __global__ void __launch_bounds__(128, 6) bounds_kernel(int64_t n, const float* 
         vals[i] = (uint32_t)i;
     }
     {
-        // a warp's 32 temporaries are contiguous in memory: through shared memory (lane stride 7 float4, odd: no bank
-        // conflicts) and out as 7 coalesced 512-byte rows
+        // a warp's 32 temporaries are contiguous in memory: through shared memory (lane stride 9 float4, odd: no bank
+        // conflicts) and out as 8 coalesced 512-byte rows
         const int lane = threadIdx.x & 31, wbase = (threadIdx.x & ~31) * PRE_TMP_PAD;
         float4* mine = s_out + wbase + lane * PRE_TMP_PAD;
         mine[0] = q0; mine[1] = q1; mine[2] = q2; mine[3] = q3; mine[4] = q4; mine[5] = q5; mine[6] = q6; mine[7] = q7;
