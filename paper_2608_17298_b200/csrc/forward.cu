@@ -583,10 +583,10 @@ constexpr int SORT_CAP = 512;    // hits per ray sorted in registers; longer ray
 constexpr int SWEEP_WARPS = 1;   // rays per block: with several, a block's shared memory and registers stay allocated until its longest ray is done
 
 // ---- rays of up to SORT_CAP hits: one warp, keys in registers (R per lane, lane l holds positions l R .. l R + R - 1)
-// A key is one 32-bit word: the bits of t* (a non-negative float: its bit pattern orders like its value)
-// with the low KEY_IDX_BITS mantissa bits replaced by the record index.  Sorting these orders the hits
-// by t* up to a relative 2^-14; neighbours whose truncated t* coincide are then put in exact (t*, id)
-// order by a few odd-even exchanges on the full values (rare).  Padding keys are all ones and sort last.
+// A key is one 32-bit word: t* in 23 bits of fixed point over the ray's own depth range, above KEY_IDX_BITS bits of
+// record index.  Sorting these orders the hits by t* up to 2^-23 of that range; neighbours whose quantised t* coincide
+// are then put in exact (t*, id) order by a few odd-even exchanges on the full values (rare).  Padding keys are all
+// ones and sort last (the largest quantised t* is 2^23 - 2).
 constexpr int KEY_IDX_BITS = 9;
 static_assert((1 << KEY_IDX_BITS) >= SORT_CAP, "record index must fit the key");
 constexpr uint32_t KEY_IDX_MASK = (1u << KEY_IDX_BITS) - 1u;
@@ -682,6 +682,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
                                                float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
     uint32_t k[R];
+    float tlo = 3.0e38f, thi = 0.0f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         // load striped (coalesced), the network does not care about the initial arrangement
@@ -690,11 +691,26 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
         if (i < n) {
             float4 ra, rb;
             ld_global_nc_32B(&rec[2 * i], ra, rb);
-            k[r] = (__float_as_uint(ra.x) & ~KEY_IDX_MASK) | (uint32_t)i;
+            k[r] = __float_as_uint(ra.x);
+            tlo = fminf(tlo, ra.x); thi = fmaxf(thi, ra.x);
             s_cs[i] = make_float4(rb.x, rb.y, rb.z, ra.z);
             s_al[i] = ra.w;
             s_tg[i] = make_uint2(__float_as_uint(ra.x), __float_as_uint(ra.y));
         }
+    }
+    // The key's upper bits: t* on a scale of 2^23 - 2 steps between the ray's nearest and farthest hit (monotone in t*:
+    // a difference and a product with a positive number round monotonically), finer than the leading bits of the
+    // float itself by the ratio of t* to the ray's depth range, so that far fewer neighbours tie.
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        tlo = fminf(tlo, __shfl_xor_sync(0xffffffffu, tlo, o));
+        thi = fmaxf(thi, __shfl_xor_sync(0xffffffffu, thi, o));
+    }
+    const float kscale = thi > tlo ? 8388606.0f / (thi - tlo) : 0.0f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int i = r * 32 + lane;
+        if (i < n) k[r] = (min(__float2uint_rd((__uint_as_float(k[r]) - tlo) * kscale), 8388606u) << KEY_IDX_BITS) | (uint32_t)i;
     }
     __syncwarp();
     sort_regs<R>(k, lane);
