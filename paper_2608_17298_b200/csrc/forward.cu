@@ -668,10 +668,12 @@ __device__ __forceinline__ void lt_store(float4* __restrict__ lt, int lt_fmt, ui
     else reinterpret_cast<uint2*>(lt)[slot] = lt_pack_half(e);
 }
 
-// true if record a must come after record b: larger t*, or equal t* and larger Gaussian id  (s_tg: t* bits and id per record)
-__device__ __forceinline__ bool rec_after(const uint2* __restrict__ s_tg, uint32_t ka, uint32_t kb) {
-    const uint2 a = s_tg[ka & KEY_IDX_MASK], b = s_tg[kb & KEY_IDX_MASK];
-    return a.x > b.x || (a.x == b.x && a.y > b.y);   // t* >= 0: its bit pattern orders like its value
+// true if record a must come after record b: larger t*, or equal t* and larger Gaussian id  (read from the ray's records
+// in global memory: with keys as fine as they are this is asked for a few rays in a hundred)
+__device__ __forceinline__ bool rec_after(const float4* __restrict__ rec, uint32_t ka, uint32_t kb) {
+    const float4 a = __ldg(&rec[2 * (ka & KEY_IDX_MASK)]), b = __ldg(&rec[2 * (kb & KEY_IDX_MASK)]);
+    const uint32_t ta = __float_as_uint(a.x), tb = __float_as_uint(b.x);   // t* >= 0: its bit pattern orders like its value
+    return ta > tb || (ta == tb && __float_as_uint(a.y) > __float_as_uint(b.y));
 }
 
 // The warp first stages the ray's records in shared memory (one coalesced 32-byte read per hit): colour and LT
@@ -680,7 +682,7 @@ template <int R, bool GM, bool OPT>   // GM: entries carry their pixel's window 
 __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, int n, int n_comp, int lane, size_t b, int64_t r_idx, int pixlow,
                                                float t_min, float alpha_max, float bg0, float bg1, float bg2, float* __restrict__ color, float* __restrict__ t_final,
                                                float4* __restrict__ lt, int lt_fmt, uint32_t* __restrict__ ray_gid, uint32_t* __restrict__ ray_slot,
-                                               float4* __restrict__ s_cs, float* __restrict__ s_al, uint2* __restrict__ s_tg) {
+                                               float4* __restrict__ s_cs, float* __restrict__ s_al) {
     uint32_t k[R];
     float tlo = 3.0e38f, thi = 0.0f;
 #pragma unroll
@@ -695,7 +697,6 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
             tlo = fminf(tlo, ra.x); thi = fmaxf(thi, ra.x);
             s_cs[i] = make_float4(rb.x, rb.y, rb.z, ra.z);
             s_al[i] = ra.w;
-            s_tg[i] = make_uint2(__float_as_uint(ra.x), __float_as_uint(ra.y));
         }
     }
     // The key's upper bits: t* on a scale of 2^23 - 2 steps between the ray's nearest and farthest hit (monotone in t*:
@@ -730,11 +731,11 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 // isolated pairs (the usual case): one exact comparison each
 #pragma unroll
                 for (int r = 0; r + 1 < R; ++r) {
-                    if (((tm >> r) & 1u) && rec_after(s_tg, k[r], k[r + 1])) { const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; }
+                    if (((tm >> r) & 1u) && rec_after(rec, k[r], k[r + 1])) { const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; }
                 }
                 const bool mine = (tm >> (R - 1)) & 1u;
                 if (__any_sync(0xffffffffu, mine)) {   // pairs across a lane boundary
-                    const bool swap = mine && rec_after(s_tg, k[R - 1], nb);
+                    const bool swap = mine && rec_after(rec, k[R - 1], nb);
                     const uint32_t from_prev = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
                     const bool prev_swapped = __shfl_up_sync(0xffffffffu, (int)swap, 1) != 0 && lane > 0;
                     if (swap) k[R - 1] = nb;
@@ -746,7 +747,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                     bool moved = false;
 #pragma unroll
                     for (int r = 0; r + 1 < R; ++r) {
-                        if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(s_tg, k[r], k[r + 1])) {
+                        if (lane * R + r + 1 < n && (k[r] >> KEY_IDX_BITS) == (k[r + 1] >> KEY_IDX_BITS) && rec_after(rec, k[r], k[r + 1])) {
                             const uint32_t t = k[r]; k[r] = k[r + 1]; k[r + 1] = t; moved = true;
                         }
                     }
@@ -754,9 +755,9 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                     const uint32_t up = __shfl_down_sync(0xffffffffu, k[0], 1), dn = __shfl_up_sync(0xffffffffu, k[R - 1], 1);
                     const bool lead = ((lane ^ round) & 1) == 0;
                     if (lead) {
-                        if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(s_tg, k[R - 1], up)) { k[R - 1] = up; moved = true; }
+                        if (lane < 31 && (lane + 1) * R < n && (k[R - 1] >> KEY_IDX_BITS) == (up >> KEY_IDX_BITS) && rec_after(rec, k[R - 1], up)) { k[R - 1] = up; moved = true; }
                     } else {
-                        if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(s_tg, dn, k[0])) { k[0] = dn; moved = true; }
+                        if (lane > 0 && lane * R < n && (dn >> KEY_IDX_BITS) == (k[0] >> KEY_IDX_BITS) && rec_after(rec, dn, k[0])) { k[0] = dn; moved = true; }
                     }
                     if (!__any_sync(0xffffffffu, moved) && (round & 1)) break;
                 }
@@ -842,7 +843,7 @@ __device__ __forceinline__ void sweep_ray_regs(const float4* __restrict__ rec, i
                 float4 en = lt_entry(wgt, al[r], cx, cy, cs.z, k0, k1, k2);
                 if (OPT && al[r] >= alpha_max) { en.x = 0.0f; en.y = 0.0f; en.z = 0.0f; }   // a clamped alpha is a constant: no gradient through it
                 lt_store(lt, lt_fmt, slot, en, GM ? pix_of(pixlow, cs.x, cs.y, i < n_comp) : -1);
-                if (ray_gid) { ray_gid[b + i] = s_tg[c].y; ray_slot[b + i] = slot; }
+                if (ray_gid) { ray_gid[b + i] = __float_as_uint(__ldg(&rec[2 * c].y)); ray_slot[b + i] = slot; }
                 k0 = fmaf(wgt, cx, k0); k1 = fmaf(wgt, cy, k1); k2 = fmaf(wgt, cs.z, k2);
             }
         }
@@ -990,7 +991,7 @@ struct SweepClass {
     static constexpr int LO = CLS == 1 ? 0 : 256;                    // exclusive lower bound of n
     static constexpr int CAP = CLS == 1 ? 256 : SORT_CAP;            // entries staged per warp
     static constexpr int MIN_BLOCKS = CLS == 1 ? 24 : 16;
-    static constexpr int SMEM = SWEEP_WARPS * CAP * 28;
+    static constexpr int SMEM = SWEEP_WARPS * CAP * 20;
 };
 
 // FMT: the LT format; GM: primitive-major layout with 16-byte entries (they carry their pixel's window index); OPT: early
@@ -1032,11 +1033,10 @@ fwd_sort_sweep_kernel(const uint32_t* __restrict__ ray_off, const float4* __rest
     const int n_comp = min(n, max_comp);   // hits that are composited (all of them unless the caller set a cap)
     const int pixlow = GM ? (int)((r / width) % GM_SUP) * GM_WIN + (int)((r % width) % GM_SUP) : -1;
     const float4* rec = recs + b * 2;
-    extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then uint2 (t*, id), then float (alpha)
+    extern __shared__ __align__(16) float4 sweep_smem[];   // CAP entries per warp: float4 (colour, slot), then float (alpha)
     float4* s_cs = sweep_smem + (size_t)warp * CAP;
-    uint2* s_tg = reinterpret_cast<uint2*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
-    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP * 3 / 2) + (size_t)warp * CAP;
-#define GART_SWEEP(R) sweep_ray_regs<R, GM, OPT>(rec, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al, s_tg)
+    float* s_al = reinterpret_cast<float*>(sweep_smem + (size_t)SWEEP_WARPS * CAP) + (size_t)warp * CAP;
+#define GART_SWEEP(R) sweep_ray_regs<R, GM, OPT>(rec, n, n_comp, lane, b, r, pixlow, t_min, alpha_max, bg0, bg1, bg2, color, t_final, lt, lt_fmt, ray_gid, ray_slot, s_cs, s_al)
     if (CLS == 1) {
         if (n <= 32) GART_SWEEP(1);
         else if (n <= 64) GART_SWEEP(2);
