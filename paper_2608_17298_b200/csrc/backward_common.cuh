@@ -68,9 +68,8 @@ __device__ __forceinline__ GeoGrad moments_to_grads(const float* v, const float*
 // with d the unit ray direction, g = dL/dC and (x, y) the pixel's position in the tile.  Lanes of a warp read
 // DIFFERENT pixels at the same time, so a single copy suffers bank conflicts at random; with C copies, copy j
 // laid out in the 16-byte bank groups j, j + C, ... only and lane l reading copy l mod C, the 8 lanes that a
-// 16-byte shared load serves together collide 8 / C at a time at most.  Four copies (8 KB), not eight: the block's
-// shared memory then fits the next smaller carve-out of the multiprocessor, which leaves the L1 (through which the
-// reductions of the flush leave) twice the size; measured 0.02 ms faster than eight, two copies 0.01 ms slower.
+// 16-byte shared load serves together collide 8 / C at a time at most.  Four copies (8 KB): measured 0.02 ms faster
+// per view than eight, which never collide but take twice as long to fill for every tile; two copies are 0.03 ms slower.
 // (Tiles of 256 pixels keep one copy, 3 float4 apart.)
 template <int TS>
 struct PixLayout {
